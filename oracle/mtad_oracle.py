@@ -1,0 +1,430 @@
+"""CPU oracle for one MTAD / MMTAD iteration (arxiv 2407.09722).
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain fp64 statement of what
+the verification hot path computes.  It is imported by the tests, by the smoke
+check and by the benchmark's CPU-baseline leg, never by the product path, and
+it shares no code with the CUDA kernels.
+
+What follows the paper, and where:
+  * target forward over the draft rows, giving P[i, :] = p(. | x_{1:i-1}, input)
+    (Algorithm 1, the line "P <- M_p(input, X)"; Sec. 3.3 for the tree form
+    with tree attention);
+  * joint likelihood of every draft prefix as a running product along the
+    path (Sec. 3.2 "Draft Tokens Verification"; Algorithm 1 loop), kept in
+    the log domain here;
+  * chain rule: prefix j passes iff min(1, p/q) > tau, the longest passing
+    prefix is accepted, every prefix is tested (Sec. 3.2);
+  * tree rule: candidate passes iff p(candidate) / q(x**_{1:i}) clears tau,
+    longest accepted candidate wins, ties by target likelihood (Sec. 3.3,
+    the displayed acceptance equation and the paragraph after it);
+  * one extra token sampled from the target row after the accepted prefix
+    (Algorithm 1, "t ~ p'"), drawn with the Gumbel-max identity from caller
+    supplied uniforms so that the draw is a pure function of its inputs;
+  * beam sampling draft with the auxiliary model (Sec. 2.1, the p_beam
+    equation), sampled without replacement with Gumbel-top-b.
+
+The decoder itself is only named by the paper (Llama / OPT families); the
+definition used is the Llama one: pre-RMSNorm, rotary embedding with
+half-split pairing, grouped-query softmax attention, SwiGLU FFN, untied LM
+head.  The KV cache stores bf16 (round-to-nearest-even), a storage decision
+both sides of the parity tests take; every other quantity is fp64.
+
+Parity pins (tests/test_oracle_*.py): chain-shaped tree == token-by-token
+causal decoding; every tree node == the chain of its own path; cross-check
+against stock torch fp64 ops; log-softmax normalisation; prefix sums vs
+products of probabilities; hand-built accept cases incl. the non-monotone
+one; exhaustive enumeration at vocab 8, gamma 3; sampler frequencies.
+The *distribution* of the beam-sampling draft is pinned only through the
+Gumbel-top-b inclusion probabilities at vocab 8: beyond that it is
+"parity unpinned".
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+NEG_INF = float("-inf")
+
+
+# ----------------------------------------------------------------------------
+# bf16 <-> fp64
+# ----------------------------------------------------------------------------
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Widen bf16 bit patterns (uint16) to fp64 exactly."""
+    b = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def f64_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round to bf16, nearest-even, through fp32 (the value first becomes an fp32, as it is on the device)."""
+    u = np.ascontiguousarray(x, dtype=np.float64).astype(np.float32).view(np.uint32)
+    rounded = u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))
+    return (rounded >> np.uint32(16)).astype(np.uint16)
+
+
+# ----------------------------------------------------------------------------
+# model container
+# ----------------------------------------------------------------------------
+
+@dataclass
+class OracleModel:
+    """A decoder given as bf16 bit patterns (uint16 arrays), matrices row-major [out, in].
+
+    `layers` is any indexable of per-layer dicts with keys attn_norm, wq, wk, wv, wo, ffn_norm,
+    w_gate, w_up, w_down (it may build a layer on demand so that large shapes stream through memory).
+    """
+    n_layers: int
+    d_model: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    d_ffn: int
+    vocab: int
+    rope_base: float
+    rms_eps: float
+    embed: np.ndarray
+    lm_head: np.ndarray
+    final_norm: np.ndarray
+    layers: Sequence[dict]
+
+
+def rmsnorm(x: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
+    """x / sqrt(mean(x^2) + eps) * gain, row-wise."""
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * gain
+
+
+def rope(x: np.ndarray, pos: np.ndarray, base: float) -> np.ndarray:
+    """Rotary embedding, half-split pairing: element i pairs with i + hd/2, angle pos * base^(-2i/hd).
+
+    x: [R, H, hd]; pos: [R]."""
+    hd = x.shape[-1]
+    half = hd // 2
+    inv_freq = base ** (-2.0 * np.arange(half, dtype=np.float64) / hd)
+    ang = pos.astype(np.float64)[:, None] * inv_freq[None, :]          # [R, half]
+    c, s = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+    a, b = x[..., :half], x[..., half:]
+    return np.concatenate([a * c - b * s, b * c + a * s], axis=-1)
+
+
+def silu(x: np.ndarray) -> np.ndarray:
+    return x / (1.0 + np.exp(-x))
+
+
+def log_softmax(z: np.ndarray) -> np.ndarray:
+    """log P[r, j] = z[r, j] - log sum_k exp z[r, k], with the row maximum subtracted first."""
+    m = np.max(z, axis=-1, keepdims=True)
+    return z - (m + np.log(np.sum(np.exp(z - m), axis=-1, keepdims=True)))
+
+
+def decoder_rows(model: OracleModel, cache: np.ndarray, L: int, row_tok: Sequence[int], row_pos: Sequence[int],
+                 row_slot: Sequence[int], row_visible: Sequence[Sequence[int]]) -> np.ndarray:
+    """Run R new rows through the decoder against one sequence's KV cache.
+
+    cache: uint16 [layers, 2, Hkv, capacity, hd] (bf16 bits), positions [0, L) committed.  Row r has token
+    row_tok[r], rotary position row_pos[r]; its K and V are rounded to bf16 and written at cache slot
+    row_slot[r] (>= L); it attends to every committed position and to the slots listed in row_visible[r]
+    (which must include its own slot).  Returns the fp64 logits [R, vocab].
+    """
+    R = len(row_tok)
+    Hq, Hkv, hd = model.n_q_heads, model.n_kv_heads, model.head_dim
+    group = Hq // Hkv
+    pos = np.asarray(row_pos, dtype=np.int64)
+    h = bf16_bits_to_f64(model.embed[np.asarray(row_tok, dtype=np.int64)])        # [R, d]
+    hi_slot = max(row_slot) + 1
+    # visibility mask over cache slots [0, hi_slot): committed prefix + listed speculative slots
+    vis = np.zeros((R, hi_slot), dtype=bool)
+    vis[:, :L] = True
+    for r in range(R):
+        assert row_slot[r] in row_visible[r]
+        for s in row_visible[r]:
+            assert s >= L
+            vis[r, s] = True
+    for l in range(model.n_layers):
+        w = model.layers[l]
+        a = rmsnorm(h, bf16_bits_to_f64(w["attn_norm"]), model.rms_eps)
+        q = (a @ bf16_bits_to_f64(w["wq"]).T).reshape(R, Hq, hd)
+        k = (a @ bf16_bits_to_f64(w["wk"]).T).reshape(R, Hkv, hd)
+        v = (a @ bf16_bits_to_f64(w["wv"]).T).reshape(R, Hkv, hd)
+        q = rope(q, pos, model.rope_base)
+        k = rope(k, pos, model.rope_base)
+        for r in range(R):
+            cache[l, 0, :, row_slot[r], :] = f64_to_bf16_bits(k[r])
+            cache[l, 1, :, row_slot[r], :] = f64_to_bf16_bits(v[r])
+        o = np.zeros((R, Hq, hd), dtype=np.float64)
+        for g in range(Hkv):
+            Kc = bf16_bits_to_f64(cache[l, 0, g, :hi_slot, :])                    # [S, hd]
+            Vc = bf16_bits_to_f64(cache[l, 1, g, :hi_slot, :])
+            for hq in range(g * group, (g + 1) * group):
+                s = (q[:, hq, :] @ Kc.T) / math.sqrt(hd)                          # [R, S]
+                s = np.where(vis, s, NEG_INF)
+                s = s - np.max(s, axis=-1, keepdims=True)
+                p = np.exp(s)
+                p = p / np.sum(p, axis=-1, keepdims=True)
+                o[:, hq, :] = p @ Vc
+        h = h + o.reshape(R, Hq * hd) @ bf16_bits_to_f64(w["wo"]).T
+        f = rmsnorm(h, bf16_bits_to_f64(w["ffn_norm"]), model.rms_eps)
+        gate = f @ bf16_bits_to_f64(w["w_gate"]).T
+        up = f @ bf16_bits_to_f64(w["w_up"]).T
+        h = h + (silu(gate) * up) @ bf16_bits_to_f64(w["w_down"]).T
+    hn = rmsnorm(h, bf16_bits_to_f64(model.final_norm), model.rms_eps)
+    return hn @ bf16_bits_to_f64(model.lm_head).T
+
+
+# ----------------------------------------------------------------------------
+# tree bookkeeping
+# ----------------------------------------------------------------------------
+
+def node_depths(parent: Sequence[int]) -> List[int]:
+    """1-based depth of every node; parent[n] = -1 means the node follows the root row directly."""
+    d: List[int] = []
+    for n, p in enumerate(parent):
+        assert -1 <= p < n, "nodes must be topologically sorted (parent[n] < n)"
+        d.append(1 if p < 0 else d[p] + 1)
+    return d
+
+
+def tree_rows(L: int, root_tok: int, tok: Sequence[int], parent: Sequence[int]):
+    """Rows of the verify forward: row 0 = root (last emitted token, position L), row n+1 = node n at
+    position L + depth(n); a row sees the committed context, its ancestors and itself."""
+    depth = node_depths(parent)
+    row_tok = [root_tok] + list(tok)
+    row_pos = [L] + [L + d for d in depth]
+    row_slot = [L + r for r in range(len(row_tok))]
+    visible = [[L]]
+    for n, p in enumerate(parent):
+        visible.append(visible[p + 1] + [L + n + 1])
+    return row_tok, row_pos, row_slot, visible
+
+
+def node_logprobs(logits: np.ndarray, tok: Sequence[int], parent: Sequence[int]):
+    """lp[n] = log P[row(parent(n)), tok[n]]: the target's conditional log-probability of node n's token given
+    its path (row i of P predicts the token after x_{1:i-1}; Algorithm 1's comment on P).  Also the log-sum-exp
+    of each row."""
+    logp = log_softmax(logits)
+    lp = np.array([logp[parent[n] + 1, tok[n]] for n in range(len(tok))], dtype=np.float64)
+    m = np.max(logits, axis=-1)
+    lse = m + np.log(np.sum(np.exp(logits - m[:, None]), axis=-1))
+    return lp, lse
+
+
+def path_prefix_sums(lp: Sequence[float], parent: Sequence[int]) -> np.ndarray:
+    """LP[n] = LP[parent(n)] + lp[n], LP[root] = 0: log of the running product p <- p * P[i, x_i]."""
+    LP = np.zeros(len(lp), dtype=np.float64)
+    for n, p in enumerate(parent):
+        LP[n] = (0.0 if p < 0 else LP[p]) + lp[n]
+    return LP
+
+
+# ----------------------------------------------------------------------------
+# accept rules
+# ----------------------------------------------------------------------------
+
+def accept_chain(LP: Sequence[float], logq: Sequence[float], log_tau: float):
+    """Longest prefix j with log p(x_{1:j}) - log q(x_{1:j}) > log tau; every j is tested, a failure does not
+    stop the scan.  min(1, p/q) > tau is the same test because tau < 1.  Returns (eta, margin) with margin the
+    smallest distance of any tested prefix from the threshold."""
+    eta, margin = 0, float("inf")
+    for j in range(len(LP)):
+        gap = (LP[j] - logq[j]) - log_tau
+        if gap > 0:
+            eta = j + 1
+        if math.isfinite(gap):
+            margin = min(margin, abs(gap))
+    return eta, margin
+
+
+def accept_tree(LP: Sequence[float], parent: Sequence[int], logq_ref: Sequence[float], log_tau: float):
+    """Candidate n (depth i) passes iff LP[n] - log q(x**_{1:i}) > log tau.  Winner: deepest passing node, then
+    highest LP, then lowest index; no passing node -> the root (-1).  Returns (winner, eta, path, margin_accept,
+    margin_tie) where margin_tie is the LP gap between the winner and the best other passing node of its depth."""
+    depth = node_depths(parent)
+    winner, best = -1, (0, NEG_INF)
+    margin = float("inf")
+    for n in range(len(LP)):
+        gap = (LP[n] - logq_ref[depth[n] - 1]) - log_tau
+        if math.isfinite(gap):
+            margin = min(margin, abs(gap))
+        if gap > 0 and (depth[n], LP[n]) > best:          # strict: ties keep the lower index
+            winner, best = n, (depth[n], LP[n])
+    path: List[int] = []
+    n = winner
+    while n >= 0:
+        path.append(n)
+        n = parent[n]
+    path.reverse()
+    tie = float("inf")
+    if winner >= 0:
+        for n in range(len(LP)):
+            if n != winner and depth[n] == depth[winner] and \
+                    (LP[n] - logq_ref[depth[n] - 1]) - log_tau > 0:
+                tie = min(tie, LP[winner] - LP[n])
+    return winner, len(path), path, margin, tie
+
+
+def gumbel_argmax(z: np.ndarray, u: np.ndarray):
+    """A draw from softmax(z): argmax_j (z_j + g_j), g_j = -log(-log u_j), lowest index on ties.
+    Returns (token, gap between the best and second-best perturbed value)."""
+    y = np.asarray(z, dtype=np.float64) - np.log(-np.log(np.asarray(u, dtype=np.float64)))
+    t = int(np.argmax(y))
+    second = np.max(np.delete(y, t)) if y.size > 1 else NEG_INF
+    return t, float(y[t] - second)
+
+
+def inverse_cdf_sample(p: np.ndarray, u: float) -> int:
+    """The other exact sampler (used only in the small enumeration tests): t = min{k : C_k > u}."""
+    c = np.cumsum(np.asarray(p, dtype=np.float64))
+    return int(min(np.searchsorted(c, u, side="right"), len(c) - 1))
+
+
+# ----------------------------------------------------------------------------
+# one verification step and the cache commit
+# ----------------------------------------------------------------------------
+
+@dataclass
+class VerifyResult:
+    eta: int
+    winner: int                 # node index of the accepted candidate, -1 = none (root)
+    path: List[int]             # node ids root-to-winner
+    out_tok: List[int]          # [tok[path_1..eta], bonus]
+    out_lp: List[float]         # their target log-probs
+    node_lp: np.ndarray
+    node_LP: np.ndarray
+    row_lse: np.ndarray
+    row_cand: np.ndarray        # Gumbel-argmax token of every row
+    row_cand_lp: np.ndarray
+    margin_accept: float
+    margin_tie: float
+    margin_bonus: float
+    logits: Optional[np.ndarray] = None
+
+
+def verify_from_logits(logits: np.ndarray, tok, parent, logq_or_ref, log_tau: float, u: np.ndarray,
+                       chain: bool) -> VerifyResult:
+    lp, lse = node_logprobs(logits, tok, parent)
+    LP = path_prefix_sums(lp, parent)
+    if chain:
+        eta, m_acc = accept_chain(LP, logq_or_ref, log_tau)
+        winner, path, m_tie = eta - 1, list(range(eta)), float("inf")
+    else:
+        winner, eta, path, m_acc, m_tie = accept_tree(LP, parent, logq_or_ref, log_tau)
+    R = logits.shape[0]
+    cand = np.zeros(R, dtype=np.int64)
+    cand_lp = np.zeros(R, dtype=np.float64)
+    gaps = np.zeros(R, dtype=np.float64)
+    for r in range(R):
+        cand[r], gaps[r] = gumbel_argmax(logits[r], u)
+        cand_lp[r] = logits[r, cand[r]] - lse[r]
+    wrow = winner + 1
+    out_tok = [int(tok[n]) for n in path] + [int(cand[wrow])]
+    out_lp = [float(lp[n]) for n in path] + [float(cand_lp[wrow])]
+    return VerifyResult(eta, winner, path, out_tok, out_lp, lp, LP, lse, cand, cand_lp, m_acc, m_tie,
+                        float(gaps[wrow]), logits)
+
+
+def verify_chain(model: OracleModel, cache: np.ndarray, L: int, root_tok: int, draft_tok, draft_logq,
+                 log_tau: float, u: np.ndarray) -> VerifyResult:
+    """Algorithm 1 from "P <- M_p(input, X)" to the return: draft_logq[i] = log q(x_{1:i+1} | input)."""
+    parent = list(range(-1, len(draft_tok) - 1))
+    rows = tree_rows(L, root_tok, draft_tok, parent)
+    logits = decoder_rows(model, cache, L, *rows)
+    return verify_from_logits(logits, draft_tok, parent, draft_logq, log_tau, u, chain=True)
+
+
+def verify_tree(model: OracleModel, cache: np.ndarray, L: int, root_tok: int, tok, parent, logq_ref,
+                log_tau: float, u: np.ndarray) -> VerifyResult:
+    """Sec. 3.3: all candidates in one forward under the tree mask, normalised by the output beam's likelihood."""
+    assert max(node_depths(parent), default=0) <= len(logq_ref)
+    rows = tree_rows(L, root_tok, tok, parent)
+    logits = decoder_rows(model, cache, L, *rows)
+    return verify_from_logits(logits, tok, parent, logq_ref, log_tau, u, chain=False)
+
+
+def kv_commit(cache: np.ndarray, L: int, path: Sequence[int]) -> int:
+    """Keep the root row and the accepted path: node path[i] (slot L + 1 + path[i]) moves to position L + 1 + i.
+    Everything after is dropped (the "rollback").  Returns the new committed length L + eta + 1."""
+    for i, n in enumerate(path):
+        src, dst = L + 1 + n, L + 1 + i
+        assert src >= dst
+        if src != dst:
+            cache[:, :, :, dst, :] = cache[:, :, :, src, :]
+    return L + len(path) + 1
+
+
+# ----------------------------------------------------------------------------
+# beam-sampling draft with the auxiliary model
+# ----------------------------------------------------------------------------
+
+@dataclass
+class DraftResult:
+    tok: List[int]
+    parent: List[int]
+    depth: List[int]
+    logq: List[float]           # joint log q of the path ending at each node
+    best_path: List[int]        # node ids of x** (the final beam with the highest draft likelihood)
+    logq_ref: List[float]       # log q(x**_{1:i})
+
+
+def gumbel_top_b(scores: np.ndarray, u: np.ndarray, b: int) -> List[int]:
+    """Sample b distinct flat indices without replacement, successive draws proportional to exp(scores):
+    the b largest of scores + Gumbel noise, in decreasing order (lowest index first on ties)."""
+    y = np.asarray(scores, dtype=np.float64).ravel() - np.log(-np.log(np.asarray(u, dtype=np.float64).ravel()))
+    order = sorted(range(y.size), key=lambda i: (-y[i], i))
+    return order[:b]
+
+
+def draft_beam(model: OracleModel, cache: np.ndarray, L: int, pending_tok: Sequence[int], gamma: int, b: int,
+               u: np.ndarray) -> DraftResult:
+    """Beam sampling of width b for gamma steps (Sec. 2.1): at each step the b kept sequences are drawn without
+    replacement from p_beam over (beam, token) pairs, i.e. proportionally to the joint likelihood
+    q(beam) * q(token | beam).  Every intermediate beam becomes a tree node (Sec. 3.3).
+
+    pending_tok: tokens not yet in the auxiliary cache, oldest first, ending with the root (last emitted token);
+    they occupy positions L .. L+len-1 and are run causally in the first step.  u: [gamma, b, vocab] uniforms.
+    Speculative node n uses cache slot L + len(pending) + n.
+    """
+    P = len(pending_tok)
+    base = L + P
+    tok: List[int] = []
+    parent: List[int] = []
+    depth: List[int] = []
+    logq: List[float] = []
+    # step 1: the context is the only beam
+    vis = [[L + i for i in range(r + 1)] for r in range(P)]
+    logits = decoder_rows(model, cache, L, list(pending_tok), [L + i for i in range(P)],
+                          [L + i for i in range(P)], vis)
+    beams = [-1]                                   # node ids of the current beams (-1 = context)
+    beam_logq = np.array([0.0])
+    beam_logp = log_softmax(logits[P - 1:P])       # [n_beams, V]
+    root_vis = vis[P - 1]
+    node_vis = {-1: root_vis}
+    for step in range(gamma):
+        scores = beam_logq[:, None] + beam_logp    # joint log-likelihood of every (beam, token) pair
+        picks = gumbel_top_b(scores, u[step, :len(beams), :], b)
+        V = scores.shape[1]
+        new_nodes = []
+        for flat in picks:
+            j, v = divmod(flat, V)
+            n = len(tok)
+            tok.append(int(v)); parent.append(beams[j]); depth.append(step + 1)
+            logq.append(float(scores[j, v]))
+            node_vis[n] = node_vis[beams[j]] + [base + n]
+            new_nodes.append(n)
+        beams = new_nodes
+        beam_logq = np.array([logq[n] for n in beams])
+        if step + 1 < gamma:
+            logits = decoder_rows(model, cache, L, [tok[n] for n in beams], [base - 1 + depth[n] for n in beams],
+                                  [base + n for n in beams], [node_vis[n] for n in beams])
+            beam_logp = log_softmax(logits)
+    best = max(beams, key=lambda n: (logq[n], -n))
+    path = []
+    n = best
+    while n >= 0:
+        path.append(n)
+        n = parent[n]
+    path.reverse()
+    return DraftResult(tok, parent, depth, logq, path, [logq[n] for n in path])

@@ -1,0 +1,306 @@
+"""Pins for the oracle's accept rules, prefix sums, samplers and draft: hand-built cases stated in
+probabilities, invariants from the paper's text and proofs, and exhaustive enumeration at vocab 8."""
+import itertools
+import math
+
+import numpy as np
+import pytest
+
+import mtad_synth as S
+from oracle import mtad_oracle as O
+
+V, GAMMA = 8, 3
+
+
+def _tables(seed, closeness):
+    """Two explicit 'models': conditional tables p(.|context), q(.|context) for every context of length 0..3."""
+    rng = np.random.default_rng(seed)
+    p, q = {}, {}
+    for k in range(GAMMA + 1):
+        for ctx in itertools.product(range(V), repeat=k):
+            z = rng.standard_normal(V) * 1.5
+            p[ctx] = np.exp(O.log_softmax(z[None])[0])
+            q[ctx] = np.exp(O.log_softmax((z + closeness * rng.standard_normal(V))[None])[0])
+    return p, q
+
+
+def _chain_inputs(p, q, x):
+    logits = np.stack([np.log(p[tuple(x[:i])]) for i in range(len(x) + 1)])
+    logq = np.cumsum([math.log(q[tuple(x[:i])][x[i]]) for i in range(len(x))])
+    return logits, logq
+
+
+def test_prefix_sums_are_products_of_probabilities():
+    rng = np.random.default_rng(0)
+    tr = S.beam_tree(4, 8, 2, 1000, stream=1)
+    prob = rng.uniform(0.05, 0.9, size=len(tr.tok))
+    LP = O.path_prefix_sums(np.log(prob), tr.parent)
+    for n in range(len(tr.tok)):
+        prod, m = 1.0, n
+        while m >= 0:
+            prod *= prob[m]; m = tr.parent[m]
+        assert abs(math.exp(LP[n]) - prod) < 1e-15
+
+
+def test_node_logprobs_pick_the_parent_row():
+    rng = np.random.default_rng(1)
+    logits = rng.standard_normal((4, 6))
+    P = np.exp(logits) / np.exp(logits).sum(-1, keepdims=True)
+    tok, parent = [2, 5, 0], [-1, -1, 1]
+    lp, lse = O.node_logprobs(logits, tok, parent)
+    assert np.allclose(np.exp(lp), [P[0, 2], P[0, 5], P[2, 0]])
+    assert np.allclose(lse, np.log(np.exp(logits).sum(-1)))
+
+
+def _chain_from_probs(p_tok, q_tok, tau):
+    LP = np.cumsum(np.log(p_tok)); LQ = np.cumsum(np.log(q_tok))
+    return O.accept_chain(LP, LQ, math.log(tau) if tau > 0 else O.NEG_INF)[0]
+
+
+def test_chain_rule_hand_cases():
+    # all prefixes pass: p >= q everywhere
+    assert _chain_from_probs([.5, .5, .5], [.4, .4, .4], 0.5) == 3
+    # none pass: joint ratios .1, .01, .001
+    assert _chain_from_probs([.05, .05, .05], [.5, .5, .5], 0.3) == 0
+    # non-monotone: ratio after 1 token 0.2 (fails tau=.5), after 2 tokens 0.2*4=0.8 (passes), after 3: 0.08
+    assert _chain_from_probs([.1, .8, .05], [.5, .2, .5], 0.5) == 2
+    # a later pass overrides an earlier pass too: ratios .9, .09, .9
+    assert _chain_from_probs([.45, .05, .5], [.5, .5, .05], 0.5) == 3
+    # strict comparison at equality (ratio exactly tau): p/q = 0.5 -> not accepted
+    assert _chain_from_probs([.25], [.5], 0.5) == 0
+    # tau = 0 accepts everything with p > 0
+    assert _chain_from_probs([1e-30, 1e-30], [.9, .9], 0.0) == 2
+    # min(1, p/q) never blocks: ratio 50 passes for tau just below 1
+    assert _chain_from_probs([.5], [.01], 0.999) == 1
+
+
+def test_chain_invariants_on_random_inputs():
+    rng = np.random.default_rng(2)
+    for _ in range(500):
+        g = int(rng.integers(1, 9))
+        pt, qt = rng.uniform(.01, 1, g), rng.uniform(.01, 1, g)
+        tau = float(rng.uniform(.05, .95))
+        eta = _chain_from_probs(pt, qt, tau)
+        P, Q = np.cumprod(pt), np.cumprod(qt)
+        if eta > 0:
+            assert P[eta - 1] / Q[eta - 1] > tau                          # accepted prefix clears the threshold
+            if Q[eta - 1] > P[eta - 1]:
+                assert (Q[eta - 1] - P[eta - 1]) / P[eta - 1] < 1 / tau - 1  # bounded relative error (Sec. 3.2)
+        for j in range(eta, g):
+            assert not (min(1.0, P[j] / Q[j]) > tau)                      # every longer prefix fails
+
+
+def test_gamma_zero_is_plain_autoregressive_sampling():
+    rng = np.random.default_rng(3)
+    logits = rng.standard_normal((1, 50))
+    u = rng.uniform(size=50)
+    res = O.verify_from_logits(logits, [], [], [], math.log(0.3), u, chain=True)
+    t, _ = O.gumbel_argmax(logits[0], u)
+    assert res.eta == 0 and res.out_tok == [t]
+    assert abs(res.out_lp[0] - O.log_softmax(logits)[0, t]) < 1e-12
+
+
+def test_theorem_short_prefixes_always_accepted():
+    # proof of the bound gamma_bar >= |log tau| / U: a prefix of length j <= |log tau| / U always passes
+    p, q = _tables(7, 0.15)
+    U = max(np.max(np.abs(np.log(p[c]) - np.log(q[c]))) for c in p if len(c) < GAMMA)
+    for tau in (0.05, 0.2, 0.5):
+        jmax = int(math.floor(abs(math.log(tau)) / U))
+        assert jmax >= 1 or tau == 0.5
+        for x in itertools.product(range(V), repeat=GAMMA):
+            logits, logq = _chain_inputs(p, q, x)
+            lp, _ = O.node_logprobs(logits, x, list(range(-1, GAMMA - 1)))
+            LP = O.path_prefix_sums(lp, list(range(-1, GAMMA - 1)))
+            assert np.allclose(np.exp(LP), np.cumprod([p[tuple(x[:i])][x[i]] for i in range(GAMMA)]))
+            eta, _ = O.accept_chain(LP, logq, math.log(tau))
+            # strictness: the theorem's bound is non-strict, equality has measure zero with these tables
+            assert eta >= min(jmax, GAMMA)
+
+
+def _chi_square_ok(counts, expected, n, min_expected=5.0, z=5.0):
+    """Pearson statistic over cells with enough mass (rest pooled); passes if within z sigma of its mean."""
+    stat, dof, pool_c, pool_e = 0.0, 0, 0.0, 0.0
+    for key, e in expected.items():
+        c = counts.get(key, 0)
+        if e * n >= min_expected:
+            stat += (c - e * n) ** 2 / (e * n); dof += 1
+        else:
+            pool_c += c; pool_e += e * n
+    if pool_e >= min_expected:
+        stat += (pool_c - pool_e) ** 2 / pool_e; dof += 1
+    dof -= 1
+    assert set(counts) <= set(expected)
+    return stat < dof + z * math.sqrt(2 * dof), (stat, dof)
+
+
+@pytest.mark.parametrize("sampler", ["gumbel", "inverse_cdf"])
+def test_exact_output_distribution_by_enumeration(sampler):
+    """Draft x ~ q (beam sampling of width 1 is ancestral sampling), verify with the chain rule, bonus ~ p.
+    The law of the returned block [x_1..x_eta, t] is sum_x q(x) 1[eta(x)] p(t | x_{1:eta}); enumerate it."""
+    p, q = _tables(11, 1.5)
+    tau = 0.6
+    exact = {}
+    for x in itertools.product(range(V), repeat=GAMMA):
+        qx = math.prod(q[tuple(x[:i])][x[i]] for i in range(GAMMA))
+        logits, logq = _chain_inputs(p, q, x)
+        LP = np.cumsum([math.log(p[tuple(x[:i])][x[i]]) for i in range(GAMMA)])
+        eta = max([j + 1 for j in range(GAMMA) if math.exp(LP[j] - logq[j]) > tau], default=0)
+        for t in range(V):
+            key = tuple(x[:eta]) + (t,)
+            exact[key] = exact.get(key, 0.0) + qx * p[tuple(x[:eta])][t]
+    assert abs(sum(exact.values()) - 1.0) < 1e-12
+    etas = {len(k) - 1 for k, v in exact.items() if v > 0}
+    assert etas == {0, 1, 2, 3}                                   # every accepted length occurs
+    rng = np.random.default_rng(5)
+    n, counts = 40000, {}
+    for _ in range(n):
+        x = []
+        for i in range(GAMMA):                                    # the oracle's own draft sampler, width 1
+            x.append(O.gumbel_top_b(np.log(q[tuple(x)])[None], rng.uniform(size=(1, V)), 1)[0])
+        logits, logq = _chain_inputs(p, q, x)
+        if sampler == "gumbel":
+            res = O.verify_from_logits(logits, x, list(range(-1, GAMMA - 1)), logq, math.log(tau),
+                                       rng.uniform(size=V), chain=True)
+            key = tuple(res.out_tok)
+            assert key[:-1] == tuple(x[:res.eta])
+        else:
+            lp, _ = O.node_logprobs(logits, x, list(range(-1, GAMMA - 1)))
+            eta, _ = O.accept_chain(O.path_prefix_sums(lp, list(range(-1, GAMMA - 1))), logq, math.log(tau))
+            key = tuple(x[:eta]) + (O.inverse_cdf_sample(p[tuple(x[:eta])], rng.uniform()),)
+        counts[key] = counts.get(key, 0) + 1
+    ok, info = _chi_square_ok(counts, exact, n)
+    assert ok, info
+
+
+def test_samplers_at_vocab_8():
+    rng = np.random.default_rng(6)
+    z = rng.standard_normal(V) * 1.3
+    pz = np.exp(O.log_softmax(z[None])[0])
+    n = 60000
+    counts = np.zeros(V)
+    for _ in range(n):
+        counts[O.gumbel_argmax(z, rng.uniform(size=V))[0]] += 1
+    assert np.all(np.abs(counts / n - pz) < 5 * np.sqrt(pz * (1 - pz) / n))
+    # inverse CDF: token k owns an interval of length p_k
+    edges = np.concatenate([[0.0], np.cumsum(pz)])
+    for k in range(V):
+        mid = 0.5 * (edges[k] + edges[k + 1])
+        assert O.inverse_cdf_sample(pz, mid) == k
+        assert abs((edges[k + 1] - edges[k]) - pz[k]) < 1e-15
+    # ties -> lowest index; margin is the gap to the runner-up
+    t, gap = O.gumbel_argmax(np.array([1.0, 3.0, 3.0]), np.array([.5, .5, .5]))
+    assert t == 1 and gap == 0.0
+
+
+def test_gumbel_top_b_inclusion_probabilities():
+    # ordered pair (i, j) without replacement has probability p_i * p_j / (1 - p_i)
+    rng = np.random.default_rng(8)
+    s = rng.standard_normal((2, 4))                              # two beams x four tokens, flat index = beam*4+tok
+    w = np.exp(s).ravel(); w /= w.sum()
+    n, counts = 60000, {}
+    for _ in range(n):
+        pick = tuple(O.gumbel_top_b(s, rng.uniform(size=(2, 4)), 2))
+        assert pick[0] != pick[1]
+        counts[pick] = counts.get(pick, 0) + 1
+    exact = {(i, j): w[i] * w[j] / (1 - w[i]) for i in range(8) for j in range(8) if i != j}
+    ok, info = _chi_square_ok(counts, exact, n)
+    assert ok, info
+
+
+def test_tree_rule_hand_cases():
+    #      root -> 0 (d1) -> 2 (d2)
+    #           -> 1 (d1) -> 3 (d2)
+    parent = [-1, -1, 0, 1]
+    ref = [math.log(.5), math.log(.25)]
+    lt = math.log(.5)
+    # deepest passing wins even if a shallower node has a larger ratio
+    LP = np.log([.9, .1, .13, .01])
+    assert O.accept_tree(LP, parent, ref, lt)[:3] == (2, 2, [0, 2])
+    # same depth: higher target likelihood wins
+    LP = np.log([.3, .4, .01, .01])
+    assert O.accept_tree(LP, parent, ref, lt)[:3] == (1, 1, [1])
+    # exact LP tie at the same depth: lowest index
+    LP = np.log([.4, .4, .01, .01])
+    w, eta, path, _, tie = O.accept_tree(LP, parent, ref, lt)
+    assert (w, eta, path, tie) == (0, 1, [0], 0.0)
+    # nobody passes -> root, eta 0, empty path
+    LP = np.log([.2, .2, .1, .1])
+    assert O.accept_tree(LP, parent, ref, lt)[:3] == (-1, 0, [])
+    # a child may pass although its parent failed (joint likelihood recovers)
+    LP = np.log([.2, .01, .19, .001])
+    assert O.accept_tree(LP, parent, ref, lt)[:3] == (2, 2, [0, 2])
+    # strict threshold: ratio exactly tau fails
+    LP = np.log([.25, .01, .01, .001])
+    assert O.accept_tree(LP, parent, ref, lt)[1] == 0
+
+
+def test_chain_shaped_tree_equals_chain_rule_and_tree_never_shorter():
+    rng = np.random.default_rng(9)
+    for trial in range(300):
+        tr = S.beam_tree(4, 4, 2, 1000, stream=trial)
+        lp = -rng.exponential(7.0, size=len(tr.tok))
+        LP = O.path_prefix_sums(lp, tr.parent)
+        log_tau = math.log(float(rng.uniform(.05, .9)))
+        w, eta_tree, path, _, _ = O.accept_tree(LP, tr.parent, tr.logq_ref, log_tau)
+        assert [tr.depth[n] for n in path] == list(range(1, eta_tree + 1))
+        # the output beam alone, as a chain and as a chain-shaped tree
+        LPb = [LP[n] for n in tr.best_path]
+        eta_chain, m1 = O.accept_chain(LPb, tr.logq_ref, log_tau)
+        wc, eta_ct, pc, m2, _ = O.accept_tree(LPb, list(range(-1, 3)), tr.logq_ref, log_tau)
+        assert (eta_ct, pc, m1) == (eta_chain, list(range(eta_chain)), m2)
+        assert eta_tree >= eta_chain                                # Sec. 3.3 theorem, per instance
+        # sibling order does not matter (no exact ties with continuous values)
+        perm = list(range(len(tr.tok)))
+        for d in range(1, 5):
+            idx = [i for i in perm if tr.depth[i] == d]
+            sh = list(rng.permutation(idx))
+            for a, b in zip(idx, sh):
+                perm[a] = b
+        inv = {old: new for new, old in enumerate(perm)}
+        parent2 = [(-1 if tr.parent[o] < 0 else inv[tr.parent[o]]) for o in perm]
+        if all(p < i for i, p in enumerate(parent2)):
+            LP2 = [LP[o] for o in perm]
+            w2, eta2, path2, _, _ = O.accept_tree(LP2, parent2, tr.logq_ref, log_tau)
+            assert eta2 == eta_tree and [perm[n] for n in path2] == path
+
+
+def test_draft_beam_bookkeeping():
+    """Structure of the beam-sampling draft: b distinct first tokens, node_logq = sum of aux log-probs along the
+    path, x** has the largest final joint q, width 1 reduces to ancestral sampling with the same noise."""
+    from oracle.adapters import oracle_model
+    shape = S.WORKLOADS["tiny"].aux
+    model = oracle_model(S.make_model(shape, 1))
+    gamma, b, L = 3, 4, 0
+    cap = 40
+    cache = np.zeros((shape.layers, 2, shape.n_kv_heads, cap, shape.head_dim), dtype=np.uint16)
+    pend = S.token_ids(0, 31, 5, shape.vocab).tolist()
+    u = S.uniforms(0, 32, gamma * b * shape.vocab).view(gamma, b, shape.vocab).numpy()
+    dr = O.draft_beam(model, cache, L, pend, gamma, b, u)
+    assert len(dr.tok) == gamma * b and dr.depth == [1] * b + [2] * b + [3] * b
+    assert len(set(dr.tok[:b])) == b and all(p == -1 for p in dr.parent[:b])
+    pairs = {(dr.parent[n], dr.tok[n]) for n in range(len(dr.tok))}
+    assert len(pairs) == len(dr.tok)
+    finals = [n for n in range(len(dr.tok)) if dr.depth[n] == gamma]
+    assert dr.best_path[-1] in finals and dr.logq[dr.best_path[-1]] == max(dr.logq[n] for n in finals)
+    assert dr.logq_ref == [dr.logq[n] for n in dr.best_path]
+    # joint log q along x** equals per-token aux log-softmax values from causal token-by-token decoding
+    seq = pend + [dr.tok[n] for n in dr.best_path]
+    c2 = np.zeros_like(cache)
+    acc, want = 0.0, []
+    for i, t in enumerate(seq[:-1]):
+        lg = O.decoder_rows(model, c2, i, [t], [i], [i], [[i]])
+        if i >= len(pend) - 1:
+            acc += O.log_softmax(lg)[0, seq[i + 1]]
+            want.append(acc)
+    assert np.allclose(want, dr.logq_ref, atol=1e-10)
+    # width 1: each step is one Gumbel-max draw from q(. | prefix)
+    cache1 = np.zeros_like(cache)
+    d1 = O.draft_beam(model, cache1, L, pend, gamma, 1, u[:, :1])
+    c3 = np.zeros_like(cache)
+    for i, t in enumerate(pend[:-1]):
+        O.decoder_rows(model, c3, i, [t], [i], [i], [[i]])
+    cur, pos = pend[-1], len(pend) - 1
+    for step in range(gamma):
+        lg = O.decoder_rows(model, c3, pos, [cur], [pos], [pos], [[pos]])[0]
+        cur, _ = O.gumbel_argmax(lg, u[step, 0]); pos += 1
+        assert cur == d1.tok[step]
