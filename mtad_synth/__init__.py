@@ -105,9 +105,10 @@ def token_ids(seed: int, stream: int, n: int, vocab: int, device="cpu") -> torch
 
 
 def uniforms(seed: int, stream: int, n: int, device="cpu") -> torch.Tensor:
-    """fp32 uniforms strictly inside (0, 1): (24 hashed bits + 0.5) / 2^24 (exact in fp32)."""
+    """fp32 uniforms strictly inside (0, 1): (23 hashed bits + 0.5) / 2^23, every value exact in fp32
+    (smallest 2^-24, largest 1 - 2^-24)."""
     h = hash_u64(seed, stream, 0, n, device)
-    return ((_lsr(h, 40).to(torch.float64) + 0.5) / float(1 << 24)).to(torch.float32)
+    return ((_lsr(h, 41).to(torch.float64) + 0.5) / float(1 << 23)).to(torch.float32)
 
 
 # ----------------------------------------------------------------------------
