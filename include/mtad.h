@@ -1,0 +1,172 @@
+/*
+ * mtad.h - C ABI of the MTAD / MMTAD verification hot path (arxiv 2407.09722) for NVIDIA B200 (sm_100a).
+ *
+ * One iteration of the method (Algorithm 1; Sec. 3.3 for the multi-candidate form) is
+ *     draft with the auxiliary model  ->  one target forward over all draft rows  ->  joint likelihood of
+ *     every draft prefix  ->  threshold test  ->  longest accepted prefix + one extra token from the target.
+ * This library runs everything from the target forward on (mtad_verify_chain / mtad_verify_tree), the KV-cache
+ * roll-forward that the paper calls the rollback operation (kv_commit), and the beam-sampling draft
+ * (mtad_draft).  Every step executes in CUDA kernels of this library; there is no CPU fallback.
+ *
+ * Conventions
+ *   - Every function returns an int status: MTAD_OK (0) or a negative MTAD_E_* code.  Nothing throws, exits
+ *     or aborts.  mtad_status_str() names a code.
+ *   - "device" pointers are CUDA device memory owned by the caller for the whole lifetime of the context;
+ *     "host" pointers are ordinary memory read during the call only.  The library allocates no device memory:
+ *     all scratch lives in the workspace the caller hands to mtad_create.
+ *   - All device work is enqueued on the stream passed in (a cudaStream_t cast to void*; NULL = the legacy
+ *     default stream) and the call returns without synchronising, unless stated otherwise.
+ *   - Rows.  A verify call runs R = 1 + N rows per sequence: row 0 is the *root*, the last emitted token whose
+ *     K/V are not yet cached (position L, the committed length); row n+1 is draft node n at position
+ *     L + depth(n).  Row r writes its K/V to cache slot L + r.  A row attends to positions [0, L) and to the
+ *     rows of its ancestors and itself (tree attention, Sec. 3.3).
+ *   - Matrices are bf16, row-major [out_features, in_features].  Accumulation, norms, softmax and the residual
+ *     stream are fp32.  The KV cache stores bf16.
+ *   - A context is not thread-safe; use one context per stream.
+ */
+#ifndef MTAD_H_
+#define MTAD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    MTAD_OK = 0,
+    MTAD_E_INVALID = -1,       /* bad argument: null pointer, size out of range, tau outside [0,1), NaN */
+    MTAD_E_CAPACITY = -2,      /* batch, node count, depth or KV capacity exceeded */
+    MTAD_E_CUDA = -3,          /* a CUDA call failed; mtad_last_cuda_error() gives the code */
+    MTAD_E_TIMEOUT = -4,       /* a bounded device-side wait gave up (reported through the status words) */
+    MTAD_E_UNIMPLEMENTED = -5,
+    MTAD_E_WORKSPACE = -6      /* workspace missing, misaligned or too small */
+};
+
+#define MTAD_MAX_BATCH 64        /* sequences per call */
+#define MTAD_MAX_NODES 255       /* draft nodes per sequence per call */
+#define MTAD_MAX_DEPTH 32        /* deepest draft node */
+#define MTAD_LAYER_TENSORS 9     /* attn_norm, wq, wk, wv, wo, ffn_norm, w_gate, w_up, w_down */
+
+/* Bits of the per-sequence device status word (mtad_result.status), written by the kernels.  A sequence with
+ * a non-zero status produced no valid result and its cache is not touched by kv_commit. */
+#define MTAD_ST_BAD_PARENT   1u  /* parent[n] >= n or < -1 */
+#define MTAD_ST_BAD_TOKEN    2u  /* token id outside [0, vocab) */
+#define MTAD_ST_KV_OVERFLOW  4u  /* L + rows > kv_capacity */
+#define MTAD_ST_TOO_DEEP     8u  /* depth > max_depth passed to the call */
+#define MTAD_ST_BAD_COUNT   16u  /* n_nodes[b] outside [0, max_nodes] */
+#define MTAD_ST_TIMEOUT     32u  /* a bounded wait inside a kernel gave up */
+
+/* A Llama-style decoder (pre-RMSNorm, rotary embedding with half-split pairing (i, i + head_dim/2), grouped-
+ * query attention scaled by 1/sqrt(head_dim), SwiGLU FFN, no biases, untied LM head).  The paper names model
+ * families only (Sec. 5); this is the decoder its Llama pairs use. */
+typedef struct mtad_model_desc {
+    int32_t layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    float rope_base, rms_eps;
+    const void* embed;                 /* device bf16 [vocab, d_model] */
+    const void* lm_head;               /* device bf16 [vocab, d_model] */
+    const void* final_norm;            /* device bf16 [d_model] */
+    const void* const* layer_weights;  /* HOST array of layers * MTAD_LAYER_TENSORS device bf16 pointers, in the
+                                          order attn_norm[d], wq[Hq*hd, d], wk[Hkv*hd, d], wv[Hkv*hd, d],
+                                          wo[d, Hq*hd], ffn_norm[d], w_gate[F, d], w_up[F, d], w_down[d, F] */
+    void* kv_cache;                    /* device bf16 [layers][max_batch][2 (K,V)][n_kv_heads][kv_capacity][head_dim];
+                                          K is stored after the rotary embedding */
+    int64_t kv_capacity;               /* positions per sequence */
+} mtad_model_desc;
+
+/* Outputs of a verify call; device arrays owned by the caller.  B = sequences in the call, N = max_nodes of the
+ * call, D = max_depth of the call (chain: N = D = gamma).  Optional members may be NULL. */
+typedef struct mtad_result {
+    int32_t* eta;          /* [B]   accepted draft tokens (length of the winning path) */
+    int32_t* winner;       /* [B]   node index of the accepted candidate, -1 = none (only the root is kept) */
+    int32_t* path;         /* [B,D] node ids root-to-winner, first eta entries valid */
+    int32_t* n_out;        /* [B]   eta + 1 */
+    int32_t* out_tok;      /* [B,D+1] accepted tokens followed by the extra token drawn from the target */
+    float*   out_lp;       /* [B,D+1] their target log-probabilities (conditional, per token) */
+    float*   node_lp;      /* [B,N] log p(tok[n] | path to n), optional */
+    float*   node_LP;      /* [B,N] joint log-likelihood of the path ending at n, optional */
+    float*   row_lse;      /* [B,N+1] log-sum-exp of each row's logits, optional */
+    int32_t* row_cand;     /* [B,N+1] Gumbel-argmax token of each row, optional */
+    float*   row_cand_lp;  /* [B,N+1] its log-probability, optional */
+    float*   margin;       /* [B,2] smallest |log p - log q - log tau| over the tested nodes; LP gap between the
+                                    winner and the best other passing node of its depth (+inf if none), optional */
+    uint32_t* status;      /* [B]   MTAD_ST_* bits, 0 = fine */
+} mtad_result;
+
+typedef struct mtad_ctx mtad_ctx;
+
+/* Bytes of device workspace a context for these models needs.  aux may be NULL (no draft model). */
+int mtad_workspace_bytes(const mtad_model_desc* target, const mtad_model_desc* aux, int max_batch, int max_nodes,
+                         size_t* out_bytes);
+
+/* Create a context.  workspace: device memory, 256-byte aligned, at least mtad_workspace_bytes(); it is zeroed
+ * and the call synchronises the device.  The descriptors (and the host pointer arrays in them) are copied; the
+ * device memory they point to stays the caller's.  All sequences start empty (L = 0, root token 0). */
+int mtad_create(const mtad_model_desc* target, const mtad_model_desc* aux, int max_batch, int max_nodes,
+                void* workspace, size_t workspace_bytes, mtad_ctx** out);
+int mtad_destroy(mtad_ctx* ctx);
+
+/* Set sequence `seq` to committed length kv_len (positions [0, kv_len) of the target cache are taken as valid,
+ * e.g. injected by the caller) with `root_token` as the last emitted token.  kv_len = 0 starts a fresh sequence;
+ * a prompt is then pushed as draft chains with log_tau = -INFINITY (tau = 0 accepts every prefix) and kv_commit.
+ * aux_len is the committed length of the auxiliary cache (<= kv_len); the kv_len - aux_len tokens in between
+ * (at most MTAD_MAX_DEPTH) are given in pending_tok (host; may be NULL when aux_len == kv_len) and are replayed
+ * by the next mtad_draft. */
+int mtad_seq_set(mtad_ctx* ctx, int seq, int32_t kv_len, int32_t root_token, int32_t aux_len,
+                 const int32_t* pending_tok, void* stream);
+
+/* Read back the committed length and root token of a sequence.  Synchronises the stream. */
+int mtad_seq_get(mtad_ctx* ctx, int seq, int32_t* kv_len, int32_t* root_token, void* stream);
+
+/* Draft with the auxiliary model: beam sampling of width beam_width for gamma steps (Sec. 2.1, the p_beam
+ * equation; every intermediate beam becomes a tree node, Sec. 3.3).  At each step the beam_width kept sequences
+ * are drawn without replacement, proportionally to their joint likelihood, as the beam_width largest values of
+ * log q(beam) + log q(token | beam) + Gumbel noise, noise = -log(-log(u)).
+ *   seqs        host  [B]                 sequence ids
+ *   uniforms    device [B, gamma, beam_width, vocab] fp32 in (0,1)
+ *   tok,parent,depth  device [B, gamma*beam_width] int32  node arrays, layer by layer (parent = -1: child of root)
+ *   node_logq   device [B, gamma*beam_width] fp32  joint draft log-likelihood of the path ending at each node
+ *   logq_ref    device [B, gamma] fp32   log q(x**_{1:i}), x** = final beam with the highest likelihood
+ *   best_path   device [B, gamma] int32  node ids of x**
+ * The chain of Algorithm 1 is best_path with logq_ref. */
+int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_width, const float* uniforms,
+               int32_t* tok, int32_t* parent, int32_t* depth, float* node_logq, float* logq_ref,
+               int32_t* best_path, void* stream);
+
+/* Verify a draft chain x_1..x_gamma (Algorithm 1 from "P <- M_p(input, X)" to the return).
+ *   seqs         host   [B]
+ *   draft_tok    device [B, gamma] int32
+ *   draft_logq   device [B, gamma] fp32, draft_logq[b,i] = log q(x_{1:i+1} | input) (joint)
+ *   log_tau      log of the threshold tau in [0,1): <= 0, -INFINITY for tau = 0.  Prefix j passes iff
+ *                log p(x_{1:j}) - log q(x_{1:j}) > log_tau (min(1, p/q) > tau, Sec. 3.2); the longest passing
+ *                prefix is accepted, all gamma prefixes are tested.
+ *   bonus_uniform device [B, vocab] fp32 in (0,1): the extra token is argmax_j(logit_j - log(-log u_j)), a draw
+ *                from the target row after the accepted prefix. */
+int mtad_verify_chain(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, const int32_t* draft_tok,
+                      const float* draft_logq, float log_tau, const float* bonus_uniform,
+                      const mtad_result* out, void* stream);
+
+/* Verify a candidate tree (Sec. 3.3).  Node n of sequence b has token tok[b,n] and parent parent[b,n] (< n, or
+ * -1 for a child of the root); n_nodes[b] <= max_nodes nodes are valid (n_nodes NULL: all max_nodes).
+ * Candidate n at depth i passes iff log p(path to n) - logq_ref[b, i-1] > log_tau with
+ * logq_ref[b, i-1] = log q(x**_{1:i}); the deepest passing node wins, ties by the larger target likelihood,
+ * then by the lower index.
+ *   n_nodes   device [B] int32;  tok, parent device [B, max_nodes] int32;  logq_ref device [B, max_depth] fp32 */
+int mtad_verify_tree(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_nodes, int max_nodes,
+                     int max_depth, const int32_t* tok, const int32_t* parent, const float* logq_ref,
+                     float log_tau, const float* bonus_uniform, const mtad_result* out, void* stream);
+
+/* Keep the root row and the accepted path of the last verify call on this context (res = the same arrays, B and
+ * seqs the same), drop every other draft row, advance L by eta + 1 and make the extra token the new root; the
+ * auxiliary cache rolls forward the same way when the context has one and mtad_draft produced the tree.
+ * Sequences whose status is non-zero are left untouched. */
+int kv_commit(mtad_ctx* ctx, int B, const int32_t* seqs, const mtad_result* res, void* stream);
+
+const char* mtad_status_str(int status);
+int mtad_last_cuda_error(const mtad_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MTAD_H_ */

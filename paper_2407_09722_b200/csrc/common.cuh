@@ -1,0 +1,107 @@
+// Internal declarations shared by the host dispatcher and the kernel translation units.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "mtad.h"
+
+#define MTAD_MASK_WORDS 8          // ancestor bitmask words per row (rows per sequence <= 256)
+#define MTAD_ATTN_TILE 64          // keys staged per attention tile
+#define MTAD_ROW_CHUNK 8           // rows per GEMM / attention pass in the CUDA-core kernels
+
+namespace mtad {
+
+// Per-call view of the rows (device arrays inside the workspace). Global row t = bi * R + r.
+struct RowMeta {
+    int32_t* tok;        // [T]
+    int32_t* pos;        // [T] rotary position
+    int32_t* slot;       // [T] cache slot, -1 = row inactive (padding, rejected sequence)
+    int32_t* seq;        // [T] sequence id
+    int32_t* depth;      // [T]
+    uint32_t* mask;      // [T][MTAD_MASK_WORDS] visible rows of the same sequence (ancestors and self)
+    int32_t* n_rows;     // [B] active rows of sequence bi (n_nodes + 1, 0 if the sequence is rejected)
+    int32_t* kv_base;    // [B] committed length L seen by this call
+    int32_t* call_seq;   // [B] sequence ids of the call
+};
+
+struct ModelView {
+    mtad_model_desc d;
+    std::vector<const void*> lw;   // layers * 9 device pointers
+    int max_batch;
+    const __nv_bfloat16* w(int layer, int which) const {
+        return static_cast<const __nv_bfloat16*>(lw[(size_t)layer * MTAD_LAYER_TENSORS + which]);
+    }
+};
+
+struct SeqState {        // device arrays, [max_batch]
+    int32_t* kv_len;
+    int32_t* root_tok;
+    int32_t* aux_len;
+    int32_t* aux_npend;
+    int32_t* aux_pend;   // [max_batch][MTAD_MAX_DEPTH + 1]
+};
+
+struct Scratch {
+    float* hidden;       // [T, d]
+    float* xn;           // [T, d]
+    float* qkv;          // [T, (Hq + 2 Hkv) hd]
+    float* attn;         // [T, Hq hd]
+    float* act;          // [T, F]
+    float* rope;         // [T, hd/2, 2]
+    float* attn_part;    // [T, Hq, nsplit, hd + 2]
+    float* logits;       // [T, V]
+    float* node_lp;      // [T]
+    float* row_lse;      // [T]
+    int32_t* row_cand;   // [T]
+    float* row_cand_lp;  // [T]
+};
+
+inline int attn_split_cap(int n_q_heads) {
+    int s = (4 * 148 + n_q_heads - 1) / n_q_heads;
+    return s < 1 ? 1 : (s > 32 ? 32 : s);
+}
+
+// ---- launchers (each enqueues on `st`, returns the launch error) -------------------------------------------------
+
+struct PrepareArgs {
+    int B, R, max_depth;
+    const int32_t* n_nodes;    // device [B] or nullptr (all sequences have R-1 nodes)
+    const int32_t* tok;        // device [B, R-1]
+    const int32_t* parent;     // device [B, R-1] or nullptr (chain)
+};
+
+cudaError_t launch_prepare(const ModelView& m, const SeqState& s, const RowMeta& rm, const Scratch& sc,
+                           const PrepareArgs& a, uint32_t* status, cudaStream_t st);
+cudaError_t launch_rmsnorm(const float* x, const __nv_bfloat16* gain, float* y, int T, int d, float eps,
+                           cudaStream_t st);
+// y[t, col0 + n] (=|+=) sum_k x[t,k] W[n,k];  mode 0 store, 1 add into y, 2 SwiGLU with W2 (y = silu(xW^T) * (xW2^T))
+cudaError_t launch_gemm_rows(const float* x, int ldx, const __nv_bfloat16* W, const __nv_bfloat16* W2, float* y,
+                             int ldy, int col0, int T, int N, int K, int mode, cudaStream_t st);
+cudaError_t launch_rope_append(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int T,
+                               cudaStream_t st);
+cudaError_t launch_attention(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int B, int R,
+                             int nsplit, int chunk, cudaStream_t st);
+cudaError_t launch_lm_reduce(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R,
+                             const float* bonus_uniform, const int32_t* tok, const int32_t* parent,
+                             cudaStream_t st);
+struct AcceptArgs {
+    int B, R, max_depth;
+    const int32_t* tok;        // [B, R-1]
+    const int32_t* parent;     // [B, R-1] or nullptr (chain)
+    const float* logq_ref;     // [B, max_depth]
+    float log_tau;
+};
+cudaError_t launch_accept(const RowMeta& rm, const Scratch& sc, const AcceptArgs& a, const mtad_result& out,
+                          cudaStream_t st);
+cudaError_t launch_kv_commit(const ModelView& m, const SeqState& s, int B, const int32_t* call_seq_dev,
+                             const mtad_result& res, int max_depth, cudaStream_t st);
+cudaError_t launch_seq_advance(const SeqState& s, int B, const int32_t* call_seq_dev, const mtad_result& res,
+                               int max_depth, cudaStream_t st);
+cudaError_t launch_seq_set(const SeqState& s, int seq, int kv_len, int root, int aux_len, int npend,
+                           const int32_t* pend_host, cudaStream_t st);
+
+}  // namespace mtad

@@ -1,0 +1,182 @@
+// Tree-masked attention of the draft rows against the KV cache: split-KV partial pass + deterministic combine.
+// A row attends to the committed positions [0, L) of its sequence and to the cache slots L + s of the rows s that
+// are its ancestors or itself (tree attention, Sec. 3.3 of the paper; the chain case is causal attention).
+#include <math_constants.h>
+
+#include "common.cuh"
+
+namespace mtad {
+
+template <int HD>
+__global__ void __launch_bounds__(128) attn_partial_kernel(const float* __restrict__ qkv, int ldq,
+                                                           const __nv_bfloat16* __restrict__ cache, RowMeta rm,
+                                                           float* __restrict__ part, int layer, int max_batch, int Hq,
+                                                           int Hkv, long long cap, int R, int nsplit, int chunk) {
+    constexpr int TILE = MTAD_ATTN_TILE;           // 64 keys
+    constexpr int PAD = HD + 8;                    // bf16 elements per staged row (16-byte pad against bank conflicts)
+    constexpr int DPL = HD / 32;                   // output dims per lane
+    __shared__ __align__(16) __nv_bfloat16 Ks[TILE * PAD];
+    __shared__ __align__(16) __nv_bfloat16 Vs[TILE * PAD];
+    __shared__ __align__(16) float qs[MTAD_ROW_CHUNK][HD];
+    __shared__ float ps[4][TILE];
+
+    const int h = blockIdx.x, sp = blockIdx.y, bi = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nrows = rm.n_rows[bi];
+    if (nrows == 0) return;
+    const int seq = rm.call_seq[bi];
+    const int L = rm.kv_base[bi];
+    const int nkeys = L + nrows;
+    const int c0 = sp * chunk;
+    const int c1 = min(c0 + chunk, nkeys);
+    const int g = h / (Hq / Hkv);
+    const __nv_bfloat16* Kg = cache + (((((size_t)layer * max_batch + seq) * 2 + 0) * Hkv + g) * cap) * HD;
+    const __nv_bfloat16* Vg = cache + (((((size_t)layer * max_batch + seq) * 2 + 1) * Hkv + g) * cap) * HD;
+
+    for (int rc = 0; rc < nrows; rc += MTAD_ROW_CHUNK) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < MTAD_ROW_CHUNK * HD; i += blockDim.x) {
+            const int r = rc + i / HD;
+            qs[i / HD][i % HD] = (r < nrows) ? qkv[(size_t)(bi * R + r) * ldq + h * HD + (i % HD)] : 0.f;
+        }
+        float m[2] = {-CUDART_INF_F, -CUDART_INF_F}, l[2] = {0.f, 0.f};
+        float o[2][DPL];
+#pragma unroll
+        for (int a = 0; a < 2; ++a)
+#pragma unroll
+            for (int d = 0; d < DPL; ++d) o[a][d] = 0.f;
+
+        for (int j0 = c0; j0 < c1; j0 += TILE) {
+            __syncthreads();
+            for (int i = threadIdx.x; i < TILE * (HD / 8); i += blockDim.x) {
+                const int key = i / (HD / 8), piece = i % (HD / 8);
+                uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
+                if (j0 + key < c1) {
+                    kv4 = *reinterpret_cast<const uint4*>(Kg + (size_t)(j0 + key) * HD + piece * 8);
+                    vv4 = *reinterpret_cast<const uint4*>(Vg + (size_t)(j0 + key) * HD + piece * 8);
+                }
+                *reinterpret_cast<uint4*>(&Ks[key * PAD + piece * 8]) = kv4;
+                *reinterpret_cast<uint4*>(&Vs[key * PAD + piece * 8]) = vv4;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int a = 0; a < 2; ++a) {
+                const int rl = warp * 2 + a;                 // row within the chunk
+                const int r = rc + rl;
+                if (r >= nrows) continue;                    // warp-uniform
+                const uint32_t* mk = rm.mask + (size_t)(bi * R + r) * MTAD_MASK_WORDS;
+                float s[2];
+#pragma unroll
+                for (int kk = 0; kk < 2; ++kk) {
+                    const int key = lane + 32 * kk;
+                    const int j = j0 + key;
+                    float acc = 0.f;
+#pragma unroll
+                    for (int p = 0; p < HD / 8; ++p) {
+                        const uint4 w = *reinterpret_cast<const uint4*>(&Ks[key * PAD + p * 8]);
+                        const float4 qa = *reinterpret_cast<const float4*>(&qs[rl][p * 8]);
+                        const float4 qb = *reinterpret_cast<const float4*>(&qs[rl][p * 8 + 4]);
+                        acc = fmaf(qa.x, __uint_as_float(w.x << 16), acc);
+                        acc = fmaf(qa.y, __uint_as_float(w.x & 0xffff0000u), acc);
+                        acc = fmaf(qa.z, __uint_as_float(w.y << 16), acc);
+                        acc = fmaf(qa.w, __uint_as_float(w.y & 0xffff0000u), acc);
+                        acc = fmaf(qb.x, __uint_as_float(w.z << 16), acc);
+                        acc = fmaf(qb.y, __uint_as_float(w.z & 0xffff0000u), acc);
+                        acc = fmaf(qb.z, __uint_as_float(w.w << 16), acc);
+                        acc = fmaf(qb.w, __uint_as_float(w.w & 0xffff0000u), acc);
+                    }
+                    bool vis = j < c1;
+                    if (vis && j >= L) {
+                        const int sr = j - L;
+                        vis = (mk[sr >> 5] >> (sr & 31)) & 1u;
+                    }
+                    s[kk] = vis ? acc : -CUDART_INF_F;
+                }
+                float mx = fmaxf(s[0], s[1]);
+#pragma unroll
+                for (int ofs = 16; ofs > 0; ofs >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, ofs));
+                const float mn = fmaxf(m[a], mx);
+                float p0 = 0.f, p1 = 0.f, corr = 1.f;
+                if (mn != -CUDART_INF_F) {
+                    p0 = expf(s[0] - mn);
+                    p1 = expf(s[1] - mn);
+                    corr = expf(m[a] - mn);
+                }
+                float psum = p0 + p1;
+#pragma unroll
+                for (int ofs = 16; ofs > 0; ofs >>= 1) psum += __shfl_xor_sync(0xffffffffu, psum, ofs);
+                l[a] = l[a] * corr + psum;
+                m[a] = mn;
+                __syncwarp();
+                ps[warp][lane] = p0;
+                ps[warp][lane + 32] = p1;
+                __syncwarp();
+#pragma unroll
+                for (int d = 0; d < DPL; ++d) o[a][d] *= corr;
+                for (int key = 0; key < TILE; ++key) {
+                    const float p = ps[warp][key];
+#pragma unroll
+                    for (int d = 0; d < DPL; ++d)
+                        o[a][d] = fmaf(p, __bfloat162float(Vs[key * PAD + lane * DPL + d]), o[a][d]);
+                }
+            }
+        }
+#pragma unroll
+        for (int a = 0; a < 2; ++a) {
+            const int r = rc + warp * 2 + a;
+            if (r >= nrows) continue;
+            float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
+            if (lane == 0) { dst[0] = m[a]; dst[1] = l[a]; }
+#pragma unroll
+            for (int d = 0; d < DPL; ++d) dst[2 + lane * DPL + d] = o[a][d];
+        }
+    }
+}
+
+// merge the split partials of one (row, head) in split order
+template <int HD>
+__global__ void attn_combine_kernel(const float* __restrict__ part, float* __restrict__ out, const int32_t* slot,
+                                    int Hq, int nsplit) {
+    const int t = blockIdx.x, h = blockIdx.y, d = threadIdx.x;
+    float* dst = out + ((size_t)t * Hq + h) * HD + d;
+    if (slot[t] < 0) { *dst = 0.f; return; }
+    const float* p = part + (((size_t)t * Hq + h) * nsplit) * (HD + 2);
+    float M = -CUDART_INF_F;
+    for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p[s * (HD + 2)]);
+    float lsum = 0.f, acc = 0.f;
+    for (int s = 0; s < nsplit; ++s) {
+        const float ms = p[s * (HD + 2)];
+        if (ms == -CUDART_INF_F) continue;
+        const float w = expf(ms - M);
+        lsum += p[s * (HD + 2) + 1] * w;
+        acc += p[s * (HD + 2) + 2 + d] * w;
+    }
+    *dst = acc / lsum;
+}
+
+cudaError_t launch_attention(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int B, int R,
+                             int nsplit, int chunk, cudaStream_t st) {
+    const int Hq = m.d.n_q_heads, Hkv = m.d.n_kv_heads, hd = m.d.head_dim;
+    const int ldq = (Hq + 2 * Hkv) * hd;
+    dim3 grid(Hq, nsplit, B);
+    const __nv_bfloat16* cache = static_cast<const __nv_bfloat16*>(m.d.kv_cache);
+    dim3 cgrid(B * R, Hq);
+    if (hd == 128) {
+        attn_partial_kernel<128><<<grid, 128, 0, st>>>(sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
+                                                       Hkv, (long long)m.d.kv_capacity, R, nsplit, chunk);
+        attn_combine_kernel<128><<<cgrid, 128, 0, st>>>(sc.attn_part, sc.attn, rm.slot, Hq, nsplit);
+    } else if (hd == 64) {
+        attn_partial_kernel<64><<<grid, 128, 0, st>>>(sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
+                                                      Hkv, (long long)m.d.kv_capacity, R, nsplit, chunk);
+        attn_combine_kernel<64><<<cgrid, 64, 0, st>>>(sc.attn_part, sc.attn, rm.slot, Hq, nsplit);
+    } else if (hd == 32) {
+        attn_partial_kernel<32><<<grid, 128, 0, st>>>(sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
+                                                      Hkv, (long long)m.d.kv_capacity, R, nsplit, chunk);
+        attn_combine_kernel<32><<<cgrid, 32, 0, st>>>(sc.attn_part, sc.attn, rm.slot, Hq, nsplit);
+    } else {
+        return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace mtad
