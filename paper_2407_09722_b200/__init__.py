@@ -1,0 +1,9 @@
+"""B200-native verification hot path of multi-token assisted decoding (MTAD / MMTAD, arxiv 2407.09722).
+
+The product is the C-ABI library built from csrc/ (see include/mtad.h); this package is its thin Python binding.
+"""
+from .binding import (Context, ModelDesc, MtadError, Result, ResultBuffers, load_library, log_tau, make_desc,
+                      mtad_workspace_bytes, EXPORTS, LIB_PATH)
+
+__all__ = ["Context", "ModelDesc", "MtadError", "Result", "ResultBuffers", "load_library", "log_tau", "make_desc",
+           "mtad_workspace_bytes", "EXPORTS", "LIB_PATH"]

@@ -1,0 +1,317 @@
+// Host dispatcher behind the C ABI: argument validation, workspace carving, and the launch sequence of one
+// verification step.  No device memory is allocated here; everything lives in the caller's workspace.
+#include <math.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+#include "common.cuh"
+
+using namespace mtad;
+
+struct mtad_ctx {
+    ModelView target, aux;
+    bool has_aux = false;
+    int max_batch = 0, max_nodes = 0, T_max = 0;
+    SeqState st{};
+    RowMeta rm{};
+    Scratch sc{};
+    std::vector<long long> len_ub;      // host upper bound of each sequence's committed length
+    int last_B = 0, last_R = 0, last_D = 0;
+    int32_t last_seqs[MTAD_MAX_BATCH];
+    int last_cuda = 0;
+};
+
+namespace {
+
+struct Carver {
+    char* base;
+    size_t off = 0;
+    explicit Carver(void* b) : base(static_cast<char*>(b)) {}
+    template <typename T>
+    T* take(size_t count) {
+        off = (off + 255) & ~size_t(255);
+        T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+        off += count * sizeof(T);
+        return p;
+    }
+};
+
+bool model_ok(const mtad_model_desc* m) {
+    if (!m) return false;
+    if (m->layers < 1 || m->d_model < 8 || m->n_q_heads < 1 || m->n_kv_heads < 1 || m->d_ffn < 8 || m->vocab < 1)
+        return false;
+    if (m->head_dim != 32 && m->head_dim != 64 && m->head_dim != 128) return false;
+    if (m->n_q_heads % m->n_kv_heads) return false;
+    if (m->d_model % 8 || m->d_ffn % 8 || (m->n_q_heads * m->head_dim) % 8) return false;
+    if (!(m->rope_base > 1.f) || !(m->rms_eps >= 0.f)) return false;
+    return true;
+}
+
+bool model_ptrs_ok(const mtad_model_desc* m) {
+    if (!m->embed || !m->lm_head || !m->final_norm || !m->layer_weights || !m->kv_cache) return false;
+    if (m->kv_capacity < 1) return false;
+    for (int i = 0; i < m->layers * MTAD_LAYER_TENSORS; ++i)
+        if (!m->layer_weights[i]) return false;
+    return true;
+}
+
+// Lays out the workspace; with base == nullptr only measures it.
+size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, int max_batch, int max_nodes,
+             void* base) {
+    Carver k(base);
+    const size_t T = (size_t)max_batch * (max_nodes + 1);
+    auto mx = [&](auto f) { size_t v = f(t); if (a) v = std::max(v, (size_t)f(a)); return v; };
+    const size_t d = mx([](const mtad_model_desc* m) { return (size_t)m->d_model; });
+    const size_t qkv = mx([](const mtad_model_desc* m) { return (size_t)(m->n_q_heads + 2 * m->n_kv_heads) * m->head_dim; });
+    const size_t qd = mx([](const mtad_model_desc* m) { return (size_t)m->n_q_heads * m->head_dim; });
+    const size_t F = mx([](const mtad_model_desc* m) { return (size_t)m->d_ffn; });
+    const size_t V = mx([](const mtad_model_desc* m) { return (size_t)m->vocab; });
+    const size_t hh = mx([](const mtad_model_desc* m) { return (size_t)m->head_dim / 2; });
+    const size_t part = mx([](const mtad_model_desc* m) {
+        return (size_t)m->n_q_heads * attn_split_cap(m->n_q_heads) * (m->head_dim + 2);
+    });
+    SeqState st;
+    st.kv_len = k.take<int32_t>(max_batch);
+    st.root_tok = k.take<int32_t>(max_batch);
+    st.aux_len = k.take<int32_t>(max_batch);
+    st.aux_npend = k.take<int32_t>(max_batch);
+    st.aux_pend = k.take<int32_t>((size_t)max_batch * (MTAD_MAX_DEPTH + 1));
+    RowMeta rm;
+    rm.tok = k.take<int32_t>(T);
+    rm.pos = k.take<int32_t>(T);
+    rm.slot = k.take<int32_t>(T);
+    rm.seq = k.take<int32_t>(T);
+    rm.depth = k.take<int32_t>(T);
+    rm.mask = k.take<uint32_t>(T * MTAD_MASK_WORDS);
+    rm.n_rows = k.take<int32_t>(max_batch);
+    rm.kv_base = k.take<int32_t>(max_batch);
+    rm.call_seq = k.take<int32_t>(max_batch);
+    Scratch sc;
+    sc.hidden = k.take<float>(T * d);
+    sc.xn = k.take<float>(T * d);
+    sc.qkv = k.take<float>(T * qkv);
+    sc.attn = k.take<float>(T * qd);
+    sc.act = k.take<float>(T * F);
+    sc.rope = k.take<float>(T * hh * 2);
+    sc.attn_part = k.take<float>(T * part);
+    sc.logits = k.take<float>(T * V);
+    sc.node_lp = k.take<float>(T);
+    sc.row_lse = k.take<float>(T);
+    sc.row_cand = k.take<int32_t>(T);
+    sc.row_cand_lp = k.take<float>(T);
+    if (c) { c->st = st; c->rm = rm; c->sc = sc; }
+    return (k.off + 255) & ~size_t(255);
+}
+
+#define CU(call)                                                  \
+    do {                                                          \
+        cudaError_t e__ = (call);                                 \
+        if (e__ != cudaSuccess) { ctx->last_cuda = (int)e__; return MTAD_E_CUDA; } \
+    } while (0)
+
+// One decoder forward over T = B * R prepared rows, leaving fp32 logits in the workspace.
+int forward_rows(mtad_ctx* ctx, const ModelView& m, int B, int R, long long len_ub, cudaStream_t s) {
+    const int T = B * R;
+    const mtad_model_desc& d = m.d;
+    const int qd = d.n_q_heads * d.head_dim, kvd = d.n_kv_heads * d.head_dim, ldq = qd + 2 * kvd;
+    const Scratch& sc = ctx->sc;
+    // split the keys [0, L + R) over CTAs: about four waves of (head, split, sequence) blocks
+    const long long total = std::min<long long>(len_ub, d.kv_capacity) + R;
+    int nsplit = (int)std::min<long long>(attn_split_cap(d.n_q_heads), (total + MTAD_ATTN_TILE - 1) / MTAD_ATTN_TILE);
+    nsplit = std::max(1, std::min(nsplit, (4 * 148 + d.n_q_heads * B - 1) / (d.n_q_heads * B)));
+    long long chunk = (total + nsplit - 1) / nsplit;
+    chunk = (chunk + MTAD_ATTN_TILE - 1) / MTAD_ATTN_TILE * MTAD_ATTN_TILE;
+    for (int l = 0; l < d.layers; ++l) {
+        CU(launch_rmsnorm(sc.hidden, m.w(l, 0), sc.xn, T, d.d_model, d.rms_eps, s));
+        CU(launch_gemm_rows(sc.xn, d.d_model, m.w(l, 1), nullptr, sc.qkv, ldq, 0, T, qd, d.d_model, 0, s));
+        CU(launch_gemm_rows(sc.xn, d.d_model, m.w(l, 2), nullptr, sc.qkv, ldq, qd, T, kvd, d.d_model, 0, s));
+        CU(launch_gemm_rows(sc.xn, d.d_model, m.w(l, 3), nullptr, sc.qkv, ldq, qd + kvd, T, kvd, d.d_model, 0, s));
+        CU(launch_rope_append(m, l, ctx->rm, sc, T, s));
+        CU(launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, s));
+        CU(launch_gemm_rows(sc.attn, qd, m.w(l, 4), nullptr, sc.hidden, d.d_model, 0, T, d.d_model, qd, 1, s));
+        CU(launch_rmsnorm(sc.hidden, m.w(l, 5), sc.xn, T, d.d_model, d.rms_eps, s));
+        CU(launch_gemm_rows(sc.xn, d.d_model, m.w(l, 6), m.w(l, 7), sc.act, d.d_ffn, 0, T, d.d_ffn, d.d_model, 2, s));
+        CU(launch_gemm_rows(sc.act, d.d_ffn, m.w(l, 8), nullptr, sc.hidden, d.d_model, 0, T, d.d_model, d.d_ffn, 1, s));
+    }
+    CU(launch_rmsnorm(sc.hidden, static_cast<const __nv_bfloat16*>(d.final_norm), sc.xn, T, d.d_model, d.rms_eps, s));
+    CU(launch_gemm_rows(sc.xn, d.d_model, static_cast<const __nv_bfloat16*>(d.lm_head), nullptr, sc.logits, d.vocab, 0,
+                        T, d.vocab, d.d_model, 0, s));
+    return MTAD_OK;
+}
+
+bool seqs_ok(const mtad_ctx* ctx, int B, const int32_t* seqs) {
+    if (!seqs || B < 1 || B > ctx->max_batch || B > MTAD_MAX_BATCH) return false;
+    for (int i = 0; i < B; ++i) {
+        if (seqs[i] < 0 || seqs[i] >= ctx->max_batch) return false;
+        for (int j = 0; j < i; ++j)
+            if (seqs[j] == seqs[i]) return false;
+    }
+    return true;
+}
+
+bool result_ok(const mtad_result* r) {
+    return r && r->eta && r->winner && r->path && r->n_out && r->out_tok && r->out_lp && r->status;
+}
+
+int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_nodes, int N, int D,
+                  const int32_t* tok, const int32_t* parent, const float* logq_ref, float log_tau,
+                  const float* bonus_uniform, const mtad_result* out, void* stream) {
+    if (!ctx) return MTAD_E_INVALID;
+    if (!seqs_ok(ctx, B, seqs)) return B > (ctx ? ctx->max_batch : 0) ? MTAD_E_CAPACITY : MTAD_E_INVALID;
+    if (N < 0 || D < 0) return MTAD_E_INVALID;
+    if (N > ctx->max_nodes || N > MTAD_MAX_NODES || D > MTAD_MAX_DEPTH) return MTAD_E_CAPACITY;
+    if (N > 0 && (!tok || !logq_ref || D < 1)) return MTAD_E_INVALID;
+    if (!bonus_uniform || !result_ok(out)) return MTAD_E_INVALID;
+    if (isnan(log_tau) || !(log_tau < 0.f)) return MTAD_E_INVALID;       // tau in [0, 1)
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int R = N + 1;
+    long long ub = 0;
+    for (int i = 0; i < B; ++i) ub = std::max(ub, ctx->len_ub[seqs[i]]);
+
+    CU(cudaMemsetAsync(out->status, 0, sizeof(uint32_t) * B, s));
+    PrepareArgs pa{};
+    for (int i = 0; i < B; ++i) pa.seqs.v[i] = seqs[i];
+    pa.B = B; pa.R = R; pa.max_depth = D; pa.n_nodes = n_nodes; pa.tok = tok; pa.parent = parent;
+    CU(launch_prepare(ctx->target, ctx->st, ctx->rm, ctx->sc, pa, out->status, s));
+    int rc = forward_rows(ctx, ctx->target, B, R, ub, s);
+    if (rc != MTAD_OK) return rc;
+    CU(launch_lm_reduce(ctx->target, ctx->rm, ctx->sc, B, R, bonus_uniform, tok, parent, s));
+    AcceptArgs aa{B, R, D, tok, parent, logq_ref, log_tau};
+    CU(launch_accept(ctx->rm, ctx->sc, aa, *out, s));
+    ctx->last_B = B; ctx->last_R = R; ctx->last_D = D;
+    memcpy(ctx->last_seqs, seqs, sizeof(int32_t) * B);
+    return MTAD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int mtad_workspace_bytes(const mtad_model_desc* target, const mtad_model_desc* aux, int max_batch, int max_nodes,
+                         size_t* out_bytes) {
+    if (!out_bytes || !model_ok(target) || (aux && !model_ok(aux))) return MTAD_E_INVALID;
+    if (max_batch < 1 || max_nodes < 0) return MTAD_E_INVALID;
+    if (max_batch > MTAD_MAX_BATCH || max_nodes > MTAD_MAX_NODES) return MTAD_E_CAPACITY;
+    *out_bytes = carve(nullptr, target, aux, max_batch, max_nodes, nullptr);
+    return MTAD_OK;
+}
+
+int mtad_create(const mtad_model_desc* target, const mtad_model_desc* aux, int max_batch, int max_nodes,
+                void* workspace, size_t workspace_bytes, mtad_ctx** out) {
+    if (!out) return MTAD_E_INVALID;
+    *out = nullptr;
+    size_t need = 0;
+    int rc = mtad_workspace_bytes(target, aux, max_batch, max_nodes, &need);
+    if (rc != MTAD_OK) return rc;
+    if (!model_ptrs_ok(target) || (aux && !model_ptrs_ok(aux))) return MTAD_E_INVALID;
+    if (aux && aux->vocab != target->vocab) return MTAD_E_INVALID;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < need) return MTAD_E_WORKSPACE;
+    mtad_ctx* ctx = new (std::nothrow) mtad_ctx();
+    if (!ctx) return MTAD_E_INVALID;
+    auto fill = [&](ModelView& v, const mtad_model_desc* m) {
+        v.d = *m;
+        v.lw.assign(m->layer_weights, m->layer_weights + (size_t)m->layers * MTAD_LAYER_TENSORS);
+        v.d.layer_weights = v.lw.data();
+        v.max_batch = max_batch;
+    };
+    fill(ctx->target, target);
+    if (aux) { fill(ctx->aux, aux); ctx->has_aux = true; }
+    ctx->max_batch = max_batch;
+    ctx->max_nodes = max_nodes;
+    ctx->T_max = max_batch * (max_nodes + 1);
+    ctx->len_ub.assign(max_batch, 0);
+    carve(ctx, target, aux, max_batch, max_nodes, workspace);
+    cudaError_t e = cudaMemset(workspace, 0, need);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { delete ctx; return MTAD_E_CUDA; }
+    *out = ctx;
+    return MTAD_OK;
+}
+
+int mtad_destroy(mtad_ctx* ctx) {
+    delete ctx;
+    return MTAD_OK;
+}
+
+int mtad_seq_set(mtad_ctx* ctx, int seq, int32_t kv_len, int32_t root_token, int32_t aux_len,
+                 const int32_t* pending_tok, void* stream) {
+    if (!ctx || seq < 0 || seq >= ctx->max_batch) return MTAD_E_INVALID;
+    if (kv_len < 0 || root_token < 0 || root_token >= ctx->target.d.vocab) return MTAD_E_INVALID;
+    if (kv_len > ctx->target.d.kv_capacity) return MTAD_E_CAPACITY;
+    if (aux_len < 0 || aux_len > kv_len) return MTAD_E_INVALID;
+    const int npend = kv_len - aux_len;
+    if (npend > MTAD_MAX_DEPTH) return MTAD_E_CAPACITY;
+    if (npend > 0 && !pending_tok) return MTAD_E_INVALID;
+    CU(launch_seq_set(ctx->st, seq, kv_len, root_token, aux_len, npend, pending_tok, static_cast<cudaStream_t>(stream)));
+    ctx->len_ub[seq] = kv_len;
+    return MTAD_OK;
+}
+
+int mtad_seq_get(mtad_ctx* ctx, int seq, int32_t* kv_len, int32_t* root_token, void* stream) {
+    if (!ctx || seq < 0 || seq >= ctx->max_batch) return MTAD_E_INVALID;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t v[2];
+    CU(cudaMemcpyAsync(&v[0], ctx->st.kv_len + seq, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    CU(cudaMemcpyAsync(&v[1], ctx->st.root_tok + seq, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    CU(cudaStreamSynchronize(s));
+    ctx->len_ub[seq] = v[0];
+    if (kv_len) *kv_len = v[0];
+    if (root_token) *root_token = v[1];
+    return MTAD_OK;
+}
+
+int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_width, const float* uniforms,
+               int32_t* tok, int32_t* parent, int32_t* depth, float* node_logq, float* logq_ref,
+               int32_t* best_path, void* stream) {
+    (void)ctx; (void)B; (void)seqs; (void)gamma; (void)beam_width; (void)uniforms; (void)tok; (void)parent;
+    (void)depth; (void)node_logq; (void)logq_ref; (void)best_path; (void)stream;
+    return MTAD_E_UNIMPLEMENTED;
+}
+
+int mtad_verify_chain(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, const int32_t* draft_tok,
+                      const float* draft_logq, float log_tau, const float* bonus_uniform,
+                      const mtad_result* out, void* stream) {
+    // a chain is the tree parent[n] = n - 1; node j has depth j + 1, so log q(x**_{1:j+1}) = draft_logq[j]
+    return verify_common(ctx, B, seqs, nullptr, gamma, gamma, draft_tok, nullptr, draft_logq, log_tau,
+                         bonus_uniform, out, stream);
+}
+
+int mtad_verify_tree(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_nodes, int max_nodes,
+                     int max_depth, const int32_t* tok, const int32_t* parent, const float* logq_ref,
+                     float log_tau, const float* bonus_uniform, const mtad_result* out, void* stream) {
+    if (max_nodes > 0 && !parent) return MTAD_E_INVALID;
+    return verify_common(ctx, B, seqs, n_nodes, max_nodes, max_depth, tok, parent, logq_ref, log_tau,
+                         bonus_uniform, out, stream);
+}
+
+int kv_commit(mtad_ctx* ctx, int B, const int32_t* seqs, const mtad_result* res, void* stream) {
+    if (!ctx || !result_ok(res)) return MTAD_E_INVALID;
+    if (!seqs_ok(ctx, B, seqs)) return MTAD_E_INVALID;
+    if (B != ctx->last_B || memcmp(seqs, ctx->last_seqs, sizeof(int32_t) * B) != 0) return MTAD_E_INVALID;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CU(launch_kv_commit(ctx->target, ctx->st, B, ctx->rm.call_seq, *res, ctx->last_D, s));
+    CU(launch_seq_advance(ctx->st, B, ctx->rm.call_seq, *res, ctx->last_D, s));
+    for (int i = 0; i < B; ++i)
+        ctx->len_ub[seqs[i]] = std::min<long long>(ctx->len_ub[seqs[i]] + ctx->last_D + 1, ctx->target.d.kv_capacity);
+    ctx->last_B = 0;
+    return MTAD_OK;
+}
+
+const char* mtad_status_str(int status) {
+    switch (status) {
+        case MTAD_OK: return "ok";
+        case MTAD_E_INVALID: return "invalid argument";
+        case MTAD_E_CAPACITY: return "capacity exceeded";
+        case MTAD_E_CUDA: return "CUDA error";
+        case MTAD_E_TIMEOUT: return "device wait timed out";
+        case MTAD_E_UNIMPLEMENTED: return "not implemented";
+        case MTAD_E_WORKSPACE: return "workspace missing, misaligned or too small";
+        default: return "unknown status";
+    }
+}
+
+int mtad_last_cuda_error(const mtad_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+
+}  // extern "C"

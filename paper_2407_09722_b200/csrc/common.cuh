@@ -67,7 +67,12 @@ inline int attn_split_cap(int n_q_heads) {
 
 // ---- launchers (each enqueues on `st`, returns the launch error) -------------------------------------------------
 
+struct SeqList {
+    int32_t v[MTAD_MAX_BATCH];
+};
+
 struct PrepareArgs {
+    SeqList seqs;              // sequence ids of the call, by value
     int B, R, max_depth;
     const int32_t* n_nodes;    // device [B] or nullptr (all sequences have R-1 nodes)
     const int32_t* tok;        // device [B, R-1]

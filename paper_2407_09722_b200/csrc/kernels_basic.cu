@@ -70,7 +70,7 @@ __global__ void prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, i
                                long long kv_capacity, SeqState s, RowMeta rm, float* __restrict__ hidden,
                                float* __restrict__ rope, PrepareArgs a, uint32_t* status) {
     const int t = blockIdx.x, bi = t / a.R, r = t % a.R;
-    const int seq = rm.call_seq[bi];
+    const int seq = a.seqs.v[bi];
     const int L = s.kv_len[seq];
     const int N = a.R - 1;
     int nn = a.n_nodes ? a.n_nodes[bi] : N;
@@ -117,6 +117,7 @@ __global__ void prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, i
         if (r == 0) {
             rm.n_rows[bi] = seq_ok ? nn + 1 : 0;
             rm.kv_base[bi] = L;
+            rm.call_seq[bi] = seq;
         }
         sh_tok = tok;
         sh_pos = L + depth;

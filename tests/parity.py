@@ -1,0 +1,191 @@
+"""Parity harness: runs one verification step through the C-ABI on the GPU and through the CPU oracle on the same
+seeded inputs and compares them.  Test infrastructure (imports the oracle)."""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+import mtad_synth as S
+import paper_2407_09722_b200 as M
+from oracle import mtad_oracle as O
+from oracle.adapters import oracle_model, bits
+
+LP_TOL = 2e-3          # absolute tolerance on log-probabilities (per token and joint)
+MARGIN = 1e-3          # decisions closer than this to a boundary are counted, not compared
+
+
+class GpuModel:
+    """Seeded weights + KV cache on the device, the library context, and a lazily built oracle twin."""
+
+    def __init__(self, target: S.ModelShape, max_batch: int, max_nodes: int, capacity: int, seed: int = 0,
+                 aux: Optional[S.ModelShape] = None, aux_capacity: Optional[int] = None):
+        dev = "cuda"
+        self.shape, self.aux_shape, self.seed = target, aux, seed
+        self.max_batch, self.max_nodes, self.capacity = max_batch, max_nodes, capacity
+        self.weights = S.make_model(target, 0, seed, dev)
+        self.cache = torch.zeros(S.kv_cache_shape(target, max_batch, capacity), dtype=torch.bfloat16, device=dev)
+        self._keep: list = []
+        self.desc = M.make_desc(target, self.weights, self.cache, self._keep)
+        self.aux_desc = None
+        if aux is not None:
+            self.aux_weights = S.make_model(aux, 1, seed, dev)
+            self.aux_cache = torch.zeros(S.kv_cache_shape(aux, max_batch, aux_capacity or capacity),
+                                         dtype=torch.bfloat16, device=dev)
+            self.aux_desc = M.make_desc(aux, self.aux_weights, self.aux_cache, self._keep)
+        self.ctx = M.Context(self.desc, self.aux_desc, max_batch, max_nodes, keep=self._keep)
+        self._oracle = None
+
+    def oracle(self) -> O.OracleModel:
+        if self._oracle is None:
+            s = self.shape
+            w = self.weights
+            self._oracle = oracle_model(
+                {"shape": s, "embed": w["embed"], "lm_head": w["lm_head"], "final_norm": w["final_norm"]},
+                layer_maker=lambda l: w["layers"][l])
+        return self._oracle
+
+    def inject(self, seq: int, length: int):
+        S.fill_kv_cache(self.cache, 0, seq, length, self.seed)
+
+    def cache_bits(self, seq: int, upto: int) -> np.ndarray:
+        """Host copy of one sequence's cache [layers, 2, Hkv, capacity, hd] as bf16 bits (only [0, upto) filled)."""
+        out = np.zeros((self.shape.layers, 2, self.shape.n_kv_heads, self.capacity, self.shape.head_dim), np.uint16)
+        out[:, :, :, :upto] = bits(self.cache[:, seq, :, :, :upto].contiguous())
+        return out
+
+
+@dataclass
+class SeqCase:
+    seq: int
+    L: int
+    root: int
+    tree: S.DraftTree
+    n_nodes: Optional[int] = None      # use only the first n nodes (ragged batches)
+
+
+@dataclass
+class ParityStats:
+    max_lp_err: float = 0.0
+    max_LP_err: float = 0.0
+    max_lse_err: float = 0.0
+    n_seq: int = 0
+    eta_match: int = 0
+    path_match: int = 0
+    tok_match: int = 0
+    near_ties: int = 0
+    cache_rows: int = 0
+    cache_exact: int = 0
+    cache_max_rel: float = 0.0
+    etas: List[int] = field(default_factory=list)
+
+    def ok(self) -> bool:
+        clean = self.n_seq - self.near_ties
+        return (self.max_lp_err <= LP_TOL and self.max_LP_err <= LP_TOL and self.eta_match >= clean
+                and self.path_match >= clean and self.tok_match >= clean)
+
+
+def _trim(tree: S.DraftTree, n: Optional[int]) -> S.DraftTree:
+    if n is None or n >= len(tree.tok):
+        return tree
+    return S.DraftTree(tree.tok[:n], tree.parent[:n], tree.depth[:n], tree.logq[:n], tree.best_path, tree.logq_ref)
+
+
+def run_gpu(gm: GpuModel, cases: Sequence[SeqCase], log_tau: float, u: torch.Tensor, chain: bool,
+            commit: bool = True) -> M.ResultBuffers:
+    """One verify call (+ kv_commit) through the C-ABI. u: [B, vocab] device uniforms."""
+    B = len(cases)
+    seqs = [c.seq for c in cases]
+    for c in cases:
+        gm.ctx.mtad_seq_set(c.seq, c.L, c.root)
+    if chain:
+        g = len(cases[0].tree.tok)
+        assert all(len(c.tree.tok) == g and c.n_nodes is None for c in cases)
+        tok = torch.tensor([c.tree.tok for c in cases], dtype=torch.int32, device="cuda").view(B, g)
+        lq = torch.tensor([c.tree.logq_ref for c in cases], dtype=torch.float32, device="cuda").view(B, g)
+        res = M.ResultBuffers(B, g, g)
+        gm.ctx.mtad_verify_chain(seqs, g, tok if g else None, lq if g else None, log_tau, u, res)
+    else:
+        N = max(len(c.tree.tok) for c in cases)
+        D = max(max(c.tree.depth, default=1) for c in cases)
+        tok = torch.zeros(B, N, dtype=torch.int32)
+        par = torch.full((B, N), -1, dtype=torch.int32)
+        ref = torch.zeros(B, D, dtype=torch.float32)
+        nn = torch.zeros(B, dtype=torch.int32)
+        for i, c in enumerate(cases):
+            t = _trim(c.tree, c.n_nodes)
+            n = len(t.tok)
+            tok[i, :n] = torch.tensor(t.tok, dtype=torch.int32)
+            par[i, :n] = torch.tensor(t.parent, dtype=torch.int32)
+            ref[i, :len(t.logq_ref)] = torch.tensor(t.logq_ref, dtype=torch.float32)
+            nn[i] = n
+        res = M.ResultBuffers(B, N, D)
+        gm.ctx.mtad_verify_tree(seqs, nn.cuda(), N, D, tok.cuda(), par.cuda(), ref.cuda(), log_tau, u, res)
+    if commit:
+        gm.ctx.kv_commit(seqs, res)
+    torch.cuda.synchronize()
+    return res
+
+
+def run_oracle(gm: GpuModel, case: SeqCase, cache_before: np.ndarray, log_tau: float, u_row: np.ndarray,
+               chain: bool):
+    t = _trim(case.tree, case.n_nodes)
+    model = gm.oracle()
+    cache = cache_before
+    if chain:
+        # the device receives fp32 draft log-likelihoods; the oracle gets the same values
+        lq = np.asarray(t.logq_ref, dtype=np.float32).astype(np.float64)
+        r = O.verify_chain(model, cache, case.L, case.root, t.tok, lq, log_tau, u_row)
+    else:
+        ref = np.asarray(t.logq_ref, dtype=np.float32).astype(np.float64)
+        r = O.verify_tree(model, cache, case.L, case.root, t.tok, t.parent, ref, log_tau, u_row)
+    newL = O.kv_commit(cache, case.L, r.path)
+    return r, cache, newL
+
+
+def compare(gm: GpuModel, cases: Sequence[SeqCase], log_tau: float, u: torch.Tensor, chain: bool,
+            stats: Optional[ParityStats] = None, check_cache: bool = True) -> ParityStats:
+    """Run both sides on the same inputs and accumulate the comparison."""
+    stats = stats or ParityStats()
+    before = [gm.cache_bits(c.seq, c.L) for c in cases]
+    res = run_gpu(gm, cases, log_tau, u, chain)
+    h = res.host()
+    u_host = u.cpu().numpy()
+    for i, c in enumerate(cases):
+        assert int(h["status"][i]) == 0, f"device status {int(h['status'][i])}"
+        r, ocache, newL = run_oracle(gm, c, before[i], log_tau, u_host[i], chain)
+        n = len(r.node_lp)
+        if n:
+            stats.max_lp_err = max(stats.max_lp_err, float(np.max(np.abs(h["node_lp"][i, :n].numpy() - r.node_lp))))
+            stats.max_LP_err = max(stats.max_LP_err, float(np.max(np.abs(h["node_LP"][i, :n].numpy() - r.node_LP))))
+        stats.max_lse_err = max(stats.max_lse_err,
+                                float(np.max(np.abs(h["row_lse"][i, :n + 1].numpy() - r.row_lse))))
+        stats.n_seq += 1
+        stats.etas.append(r.eta)
+        near = min(r.margin_accept, r.margin_tie, r.margin_bonus) < MARGIN
+        stats.near_ties += int(near)
+        g_eta = int(h["eta"][i])
+        g_path = h["path"][i, :g_eta].tolist()
+        g_tok = h["out_tok"][i, :g_eta + 1].tolist()
+        e_ok = g_eta == r.eta
+        p_ok = e_ok and g_path == r.path and int(h["winner"][i]) == r.winner
+        t_ok = p_ok and g_tok == r.out_tok and int(h["n_out"][i]) == r.eta + 1
+        stats.eta_match += int(e_ok)
+        stats.path_match += int(p_ok)
+        stats.tok_match += int(t_ok)
+        if t_ok:
+            lp_err = np.max(np.abs(h["out_lp"][i, :g_eta + 1].numpy() - np.asarray(r.out_lp)))
+            stats.max_lp_err = max(stats.max_lp_err, float(lp_err))
+        if check_cache and p_ok:
+            gL, groot = gm.ctx.mtad_seq_get(c.seq)
+            assert gL == newL and groot == r.out_tok[-1] or not t_ok, (gL, newL)
+            got = O.bf16_bits_to_f64(bits(gm.cache[:, c.seq, :, :, c.L:newL].contiguous()))
+            want = O.bf16_bits_to_f64(ocache[:, :, :, c.L:newL])
+            stats.cache_rows += got.size
+            stats.cache_exact += int(np.sum(got == want))
+            denom = np.maximum(np.abs(want), 1e-3)
+            stats.cache_max_rel = max(stats.cache_max_rel, float(np.max(np.abs(got - want) / denom)))
+    return stats
