@@ -1,0 +1,386 @@
+#!/usr/bin/env python
+"""Benchmark of the MTAD verification hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 7b_chain] [--impl ours|reference]
+
+A step is one pass of the whole hot path over one batch of synthetic drafts: mtad_verify_chain / mtad_verify_tree
+followed by kv_commit.  Consecutive steps are consecutive decode iterations (the committed length grows).  Prints
+one JSON line (rank 0).  With N > 1 every rank runs an independent replica (the path does not shard).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import mtad_synth as S  # noqa: E402
+
+TAU = 0.1
+SEED = 0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def step_trees(w: S.Workload, it: int):
+    return [S.workload_tree(w, seq=b, seed=SEED, iteration=it) for b in range(w.batch)]
+
+
+def algorithmic_bytes(w: S.Workload, lens) -> float:
+    """bf16 weight bytes streamed once per step + committed K/V bytes of every sequence read once."""
+    return w.target.streamed_weight_bytes() + w.target.kv_bytes_per_token() * float(sum(lens))
+
+
+class ClockSampler:
+    def __init__(self, index: int):
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            pass
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# reference arm and CPU baseline: the oracle, as it stands, on the host cores
+# ---------------------------------------------------------------------------------------------------------------
+
+def _blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+class OracleSampler:
+    """Times the oracle's verify step on a model truncated to `n_layers` layers (same shapes and inputs) and on the
+    same model with no layers (embedding, final norm, LM head, accept rule); the full-depth time is extrapolated
+    as t0 + layers * (tn - t0) / n.  Accepted tokens are those of the truncated model's own decision."""
+
+    def __init__(self, w: S.Workload, n_layers: int):
+        from oracle import mtad_oracle as O
+        from oracle.adapters import oracle_model, bits
+        import numpy as np
+        self.O, self.np, self.w, self.n = O, np, w, n_layers
+        s = w.target
+        dev = "cuda" if torch.cuda.is_available() else "cpu"
+        head = {"shape": s, "embed": S.make_tensor(s, 0, "embed", seed=SEED, device=dev),
+                "lm_head": S.make_tensor(s, 0, "lm_head", seed=SEED, device=dev),
+                "final_norm": S.make_tensor(s, 0, "final_norm", seed=SEED, device=dev)}
+        layers = [{k: bits(v) for k, v in S.make_layer(s, 0, l, SEED, dev).items()} for l in range(n_layers)]
+        self.models = {}
+        for n in (0, n_layers):
+            m = oracle_model(head, layer_maker=lambda l: None)
+            m.layers = layers
+            m.n_layers = n
+            self.models[n] = m
+        self.lens = S.kv_lengths(w, SEED)
+        cap = max(self.lens) + w.n_nodes + 8
+        cache = torch.zeros(S.kv_cache_shape(S.ModelShape(n_layers, s.d_model, s.n_q_heads, s.n_kv_heads, s.head_dim,
+                                                          s.d_ffn, s.vocab), 1, cap), dtype=torch.bfloat16)
+        S.fill_kv_cache(cache, 0, 0, self.lens[0], SEED)
+        self.cache = bits(cache[:, 0]).copy()
+        self.step(0)                      # untimed first touch (page faults, BLAS start-up)
+
+    def step(self, it: int):
+        """One sampled step for sequence 0 of the workload. Returns (estimated full-depth seconds for the whole
+        batch, accepted tokens for the whole batch)."""
+        O, np, w = self.O, self.np, self.w
+        tree = S.workload_tree(w, seq=0, seed=SEED, iteration=it)
+        u = S.bonus_uniforms(SEED, it, w.batch, w.target.vocab)[0].numpy()
+        ref = np.asarray(tree.logq_ref, np.float32).astype(np.float64)
+        ts = {}
+        acc = 0
+        for n in (0, self.n):
+            cache = self.cache.copy()
+            t0 = time.perf_counter()
+            if w.kind == "chain":
+                r = O.verify_chain(self.models[n], cache, self.lens[0], 1, tree.tok, ref, math.log(TAU), u)
+            else:
+                r = O.verify_tree(self.models[n], cache, self.lens[0], 1, tree.tok, tree.parent, ref, math.log(TAU), u)
+            ts[n] = time.perf_counter() - t0
+            acc = r.eta + 1
+        per_layer = max(ts[self.n] - ts[0], 0.0) / self.n
+        est = (ts[0] + w.target.layers * per_layer) * w.batch
+        return est, acc * w.batch, ts
+
+
+def run_reference(args, w: S.Workload):
+    n_layers = 1
+    smp = OracleSampler(w, n_layers)
+    for i in range(args.warmup):
+        smp.step(i)
+    tot_t, tot_a = 0.0, 0
+    for i in range(args.steps):
+        est, acc, _ = smp.step(args.warmup + i)
+        tot_t += est
+        tot_a += acc
+    value = tot_a / tot_t
+    sample = (f"each step: oracle verify step of sequence 0 on the {w.name} shapes truncated to {n_layers} layer(s) "
+              f"and to 0 layers; full depth extrapolated as t0 + {w.target.layers} * (t{n_layers} - t0) / {n_layers}, "
+              f"times batch {w.batch}")
+    cores = _blas_threads()
+    line = {"impl": "reference", "metric": "accepted_tokens_per_s", "value": value, "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * tot_t / max(args.steps, 1), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "tau": TAU},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def cpu_baseline(w: S.Workload):
+    n_layers = 2
+    smp = OracleSampler(w, n_layers)
+    est, acc, ts = smp.step(0)
+    return {"value": acc / est, "unit": "tokens/s", "cores": _blas_threads(), "kind": "oracle",
+            "sample": (f"one oracle verify step of sequence 0 truncated to {n_layers} of {w.target.layers} layers "
+                       f"({ts[n_layers]:.1f} s) and to 0 layers ({ts[0]:.1f} s); full depth extrapolated linearly, "
+                       f"times batch {w.batch}: {est:.1f} s per step"),
+            "est_step_s": est}
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------------------------------------------
+
+def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
+    import paper_2407_09722_b200 as M
+    from paper_2407_09722_b200.runtime import DeviceModel, StepInputs
+
+    torch.cuda.set_device(local_rank)
+    lens = S.kv_lengths(w, SEED)
+    chain = w.kind == "chain"
+    rows = w.n_nodes + 1
+    total_steps = args.warmup + args.steps
+    cap = max(lens) + (total_steps + 2) * (w.gamma + 1) + rows + 8
+    cap = (cap + 63) // 64 * 64
+    dm = DeviceModel(w.target, w.batch, w.n_nodes, cap, SEED)
+    for b, L in enumerate(lens):
+        dm.inject(b, L)
+    ctx = dm.ctx
+    seqs = list(range(w.batch))
+    V = w.target.vocab
+    log_tau = math.log(TAU)
+
+    inputs = [StepInputs(step_trees(w, i), chain, pin=True) for i in range(total_steps)]
+    unis_host = [S.bonus_uniforms(SEED, i, w.batch, V).pin_memory() for i in range(total_steps)]
+    unis = [u.cuda() for u in unis_host]
+    res = M.ResultBuffers(w.batch, inputs[0].N, inputs[0].D)
+
+    def reset():
+        for b, L in enumerate(lens):
+            ctx.mtad_seq_set(b, L, 1)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def reduce_max(x: float) -> float:
+        if world > 1:
+            t = torch.tensor([x], dtype=torch.float64, device="cuda")
+            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+            return float(t.item())
+        return x
+
+    def reduce_sum(x: float) -> float:
+        if world > 1:
+            t = torch.tensor([x], dtype=torch.float64, device="cuda")
+            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.SUM)
+            return float(t.item())
+        return x
+
+    # ---- device-resident timing ---------------------------------------------------------------------------------
+    reset()
+    for i in range(args.warmup):
+        inputs[i].verify(ctx, seqs, log_tau, unis[i], res)
+        ctx.kv_commit(seqs, res)
+    acc_dev = torch.zeros((), dtype=torch.int64, device="cuda")
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    sampler = ClockSampler(local_rank)
+    launches0 = M.mtad_kernel_launches()
+    ev[0].record()
+    for k in range(args.steps):
+        i = args.warmup + k
+        inputs[i].verify(ctx, seqs, log_tau, unis[i], res)
+        ctx.kv_commit(seqs, res)
+        acc_dev += res.n_out.sum()
+        ev[k + 1].record()
+    barrier()
+    launches = M.mtad_kernel_launches() - launches0
+    clocks = sampler.stop()
+    total_ms = reduce_max(ev[0].elapsed_time(ev[-1]))
+    step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
+    accepted = reduce_sum(float(acc_dev.item()))
+    value = accepted / (total_ms * 1e-3)
+    final_lens = [ctx.mtad_seq_get(b)[0] for b in seqs]
+
+    # ---- per-kernel pass: same steps again with an event pair around every launch ---------------------------------
+    reset()
+    prof_steps = min(args.steps, 4)
+    for i in range(min(args.warmup, 1)):
+        inputs[i].verify(ctx, seqs, log_tau, unis[i], res)
+        ctx.kv_commit(seqs, res)
+    ctx.mtad_profile_begin(prof_steps * (w.target.layers * 16 + 32))
+    for k in range(prof_steps):
+        i = args.warmup + k
+        inputs[i].verify(ctx, seqs, log_tau, unis[i], res)
+        ctx.kv_commit(seqs, res)
+    prof = ctx.mtad_profile_end()
+    gemm = prof["gemm"]
+    peak, peak_kind = measured_peaks()
+    achieved = gemm["bytes"] / (gemm["ms"] * 1e-3) / 1e9 if gemm["ms"] > 0 else 0.0
+    prof_total = sum(v["ms"] for v in prof.values())
+    roofline = {"bound": "hbm", "kernel": "skinny GEMM (all weight matrices + LM head)", "achieved": achieved,
+                "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                "launches_per_step": gemm["launches"] / prof_steps,
+                "avg_launch_us": 1e3 * gemm["ms"] / max(gemm["launches"], 1),
+                "share_of_step": gemm["ms"] / prof_total if prof_total else None,
+                "per_class_ms_per_step": {k: v["ms"] / prof_steps for k, v in prof.items()}}
+
+    # ---- end to end: host buffers in, host results out, every step --------------------------------------------------
+    reset()
+    stage = {k: torch.empty_like(v, device="cuda") for k, v in inputs[0].host.items()}
+    u_stage = torch.empty_like(unis[0])
+    out_host = {n: torch.empty_like(getattr(res, n), device="cpu").pin_memory()
+                for n in ("eta", "n_out", "out_tok", "out_lp", "status")}
+    h2d = sum(v.numel() * v.element_size() for v in inputs[0].host.values()) + u_stage.numel() * 4
+    d2h = sum(v.numel() * v.element_size() for v in out_host.values())
+
+    def e2e_step(i):
+        for k, v in inputs[i].host.items():
+            stage[k].copy_(v, non_blocking=True)
+        u_stage.copy_(unis_host[i], non_blocking=True)
+        inputs[i].verify(ctx, seqs, log_tau, u_stage, res, dev=stage)
+        ctx.kv_commit(seqs, res)
+        for n, t in out_host.items():
+            t.copy_(getattr(res, n), non_blocking=True)
+        torch.cuda.synchronize()
+        return int(out_host["n_out"].sum())
+
+    for i in range(args.warmup):
+        e2e_step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record()
+    acc_e2e = 0
+    for k in range(args.steps):
+        acc_e2e += e2e_step(args.warmup + k)
+    e1.record()
+    barrier()
+    wall = time.perf_counter() - t0
+    e2e_ms = reduce_max(max(e0.elapsed_time(e1), wall * 1e3))
+    e2e_value = reduce_sum(float(acc_e2e)) / (e2e_ms * 1e-3)
+
+    if rank != 0:
+        return
+    mid_lens = [(a + b) / 2 for a, b in zip(lens, final_lens)]
+    step_bytes = algorithmic_bytes(w, mid_lens)
+    ms_per_step = total_ms / args.steps
+    line = {
+        "metric": "accepted_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 weights, f32 accumulate", "data": "synthetic",
+        "config": {"workload": w.name, "tau": TAU, "batch": w.batch, "rows_per_seq": rows, "kv_len_start": lens,
+                   "replicas": world, "l2": "inputs larger than L2 (weights streamed once per step)",
+                   "block_efficiency": accepted / (args.steps * w.batch * world)},
+        "verify_step_us": {"median": 1e3 * statistics.median(step_ms), "min": 1e3 * min(step_ms),
+                           "max": 1e3 * max(step_ms)},
+        "step_hbm": {"algorithmic_gb": step_bytes / 1e9, "achieved_gbs": step_bytes / (ms_per_step * 1e-3) / 1e9,
+                     "frac_of_measured_copy": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
+                     "frac_of_8000": step_bytes / (ms_per_step * 1e-3) / 1e9 / 8000.0},
+        "roofline": roofline,
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms / args.steps},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        del dm, ctx
+        torch.cuda.empty_cache()
+        line["cpu_baseline"] = cpu_baseline(w)
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=32)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--workload", default="7b_chain", choices=sorted(S.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = S.WORKLOADS[args.workload]
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, w)
+        return
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    try:
+        run_ours(args, w, rank, world, local_rank)
+    finally:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -163,6 +163,19 @@ int mtad_verify_tree(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n
  * Sequences whose status is non-zero are left untouched. */
 int kv_commit(mtad_ctx* ctx, int B, const int32_t* seqs, const mtad_result* res, void* stream);
 
+/* Instrumentation (not part of the method).  Kernel classes for mtad_profile_end. */
+enum { MTAD_K_PREPARE = 0, MTAD_K_NORM, MTAD_K_GEMM, MTAD_K_ROPE, MTAD_K_ATTN, MTAD_K_LMRED, MTAD_K_ACCEPT,
+       MTAD_K_COMMIT, MTAD_K_CLASSES };
+
+/* Start bracketing every kernel launch of this context with a pair of CUDA events on the launching stream (room
+ * for max_launches launches; later launches go unrecorded).  Creates events, no device memory. */
+int mtad_profile_begin(mtad_ctx* ctx, int max_launches);
+/* Stop, synchronise the device and sum per kernel class: elapsed milliseconds, algorithmic bytes (bf16 weight
+ * bytes of the GEMM launches; 0 for the other classes) and launch count.  Arrays of MTAD_K_CLASSES, host. */
+int mtad_profile_end(mtad_ctx* ctx, double* ms, double* bytes, int64_t* launches);
+/* Kernels of this library enqueued by this process so far. */
+uint64_t mtad_kernel_launches(void);
+
 const char* mtad_status_str(int status);
 int mtad_last_cuda_error(const mtad_ctx* ctx);
 

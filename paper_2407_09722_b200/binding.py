@@ -38,7 +38,9 @@ class Result(C.Structure):
 
 
 EXPORTS = ("mtad_workspace_bytes", "mtad_create", "mtad_destroy", "mtad_seq_set", "mtad_seq_get", "mtad_draft",
-           "mtad_verify_chain", "mtad_verify_tree", "kv_commit", "mtad_status_str", "mtad_last_cuda_error")
+           "mtad_verify_chain", "mtad_verify_tree", "kv_commit", "mtad_status_str", "mtad_last_cuda_error",
+           "mtad_profile_begin", "mtad_profile_end", "mtad_kernel_launches")
+KERNEL_CLASSES = ("prepare", "norm", "gemm", "rope_append", "attention", "lm_reduce", "accept", "commit")
 
 _lib = None
 
@@ -67,9 +69,13 @@ def load_library() -> C.CDLL:
     lib.mtad_status_str.argtypes = [I]
     lib.mtad_status_str.restype = C.c_char_p
     lib.mtad_last_cuda_error.argtypes = [P]
+    lib.mtad_profile_begin.argtypes = [P, I]
+    lib.mtad_profile_end.argtypes = [P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    lib.mtad_kernel_launches.argtypes = []
     for n in EXPORTS:
-        if n != "mtad_status_str":
+        if n not in ("mtad_status_str", "mtad_kernel_launches"):
             getattr(lib, n).restype = I
+    lib.mtad_kernel_launches.restype = C.c_uint64
     _lib = lib
     return lib
 
@@ -223,6 +229,15 @@ class Context:
             self._check(rc, "kv_commit")
         return rc
 
+    def mtad_profile_begin(self, max_launches: int = 8192):
+        self._check(self._lib.mtad_profile_begin(self.handle, max_launches), "mtad_profile_begin")
+
+    def mtad_profile_end(self) -> Dict[str, dict]:
+        n = len(KERNEL_CLASSES)
+        ms, by, cnt = (C.c_double * n)(), (C.c_double * n)(), (C.c_int64 * n)()
+        self._check(self._lib.mtad_profile_end(self.handle, ms, by, cnt), "mtad_profile_end")
+        return {k: {"ms": ms[i], "bytes": by[i], "launches": cnt[i]} for i, k in enumerate(KERNEL_CLASSES)}
+
     def mtad_draft(self, seqs, gamma: int, beam_width: int, uniforms, tok, parent, depth, node_logq, logq_ref,
                    best_path, stream=None, check=True) -> int:
         rc = self._lib.mtad_draft(self.handle, len(seqs), _seqs(seqs), gamma, beam_width,
@@ -232,6 +247,10 @@ class Context:
         if check:
             self._check(rc, "mtad_draft")
         return rc
+
+
+def mtad_kernel_launches() -> int:
+    return int(load_library().mtad_kernel_launches())
 
 
 def log_tau(tau: float) -> float:

@@ -21,7 +21,15 @@ struct mtad_ctx {
     int last_B = 0, last_R = 0, last_D = 0;
     int32_t last_seqs[MTAD_MAX_BATCH];
     int last_cuda = 0;
+    // optional per-kernel-class timing (cudaEvent pairs around each launch)
+    bool prof_on = false;
+    std::vector<cudaEvent_t> prof_ev;        // pool, used pairwise
+    std::vector<int> prof_cls;               // class of each recorded pair
+    std::vector<double> prof_bytes;          // algorithmic bytes of each recorded pair
+    size_t prof_used = 0;
 };
+
+unsigned long long g_kernel_launches = 0;    // kernels of this library enqueued since load
 
 namespace {
 
@@ -111,6 +119,27 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
         if (e__ != cudaSuccess) { ctx->last_cuda = (int)e__; return MTAD_E_CUDA; } \
     } while (0)
 
+// Enqueue one launcher; when profiling is on, bracket it with an event pair on the same stream.
+template <class F>
+int timed(mtad_ctx* ctx, int cls, double bytes, int kernels, cudaStream_t s, F&& f) {
+    const bool rec = ctx->prof_on && ctx->prof_used + 2 <= ctx->prof_ev.size();
+    if (rec) CU(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s));
+    CU(f());
+    g_kernel_launches += kernels;
+    if (rec) {
+        CU(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s));
+        ctx->prof_cls.push_back(cls);
+        ctx->prof_bytes.push_back(bytes);
+        ctx->prof_used += 2;
+    }
+    return MTAD_OK;
+}
+#define RUN(cls, bytes, kernels, call)                                                    \
+    do {                                                                                  \
+        int rc__ = timed(ctx, cls, bytes, kernels, s, [&]() -> cudaError_t { return (call); }); \
+        if (rc__ != MTAD_OK) return rc__;                                                 \
+    } while (0)
+
 // One decoder forward over T = B * R prepared rows, leaving fp32 logits in the workspace.
 int forward_rows(mtad_ctx* ctx, const ModelView& m, int B, int R, long long len_ub, cudaStream_t s) {
     const int T = B * R;
@@ -123,21 +152,30 @@ int forward_rows(mtad_ctx* ctx, const ModelView& m, int B, int R, long long len_
     nsplit = std::max(1, std::min(nsplit, (4 * 148 + d.n_q_heads * B - 1) / (d.n_q_heads * B)));
     long long chunk = (total + nsplit - 1) / nsplit;
     chunk = (chunk + MTAD_ATTN_TILE - 1) / MTAD_ATTN_TILE * MTAD_ATTN_TILE;
+    const double wb = 2.0;   // bytes per bf16 weight
     for (int l = 0; l < d.layers; ++l) {
-        CU(launch_rmsnorm(sc.hidden, m.w(l, 0), sc.xn, T, d.d_model, d.rms_eps, s));
-        CU(launch_gemm_rows(sc.xn, d.d_model, m.w(l, 1), nullptr, sc.qkv, ldq, 0, T, qd, d.d_model, 0, s));
-        CU(launch_gemm_rows(sc.xn, d.d_model, m.w(l, 2), nullptr, sc.qkv, ldq, qd, T, kvd, d.d_model, 0, s));
-        CU(launch_gemm_rows(sc.xn, d.d_model, m.w(l, 3), nullptr, sc.qkv, ldq, qd + kvd, T, kvd, d.d_model, 0, s));
-        CU(launch_rope_append(m, l, ctx->rm, sc, T, s));
-        CU(launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, s));
-        CU(launch_gemm_rows(sc.attn, qd, m.w(l, 4), nullptr, sc.hidden, d.d_model, 0, T, d.d_model, qd, 1, s));
-        CU(launch_rmsnorm(sc.hidden, m.w(l, 5), sc.xn, T, d.d_model, d.rms_eps, s));
-        CU(launch_gemm_rows(sc.xn, d.d_model, m.w(l, 6), m.w(l, 7), sc.act, d.d_ffn, 0, T, d.d_ffn, d.d_model, 2, s));
-        CU(launch_gemm_rows(sc.act, d.d_ffn, m.w(l, 8), nullptr, sc.hidden, d.d_model, 0, T, d.d_model, d.d_ffn, 1, s));
+        RUN(MTAD_K_NORM, 0, 1, launch_rmsnorm(sc.hidden, m.w(l, 0), sc.xn, T, d.d_model, d.rms_eps, s));
+        RUN(MTAD_K_GEMM, wb * qd * d.d_model, 1,
+            launch_gemm_rows(sc.xn, d.d_model, m.w(l, 1), nullptr, sc.qkv, ldq, 0, T, qd, d.d_model, 0, s));
+        RUN(MTAD_K_GEMM, wb * kvd * d.d_model, 1,
+            launch_gemm_rows(sc.xn, d.d_model, m.w(l, 2), nullptr, sc.qkv, ldq, qd, T, kvd, d.d_model, 0, s));
+        RUN(MTAD_K_GEMM, wb * kvd * d.d_model, 1,
+            launch_gemm_rows(sc.xn, d.d_model, m.w(l, 3), nullptr, sc.qkv, ldq, qd + kvd, T, kvd, d.d_model, 0, s));
+        RUN(MTAD_K_ROPE, 0, 1, launch_rope_append(m, l, ctx->rm, sc, T, s));
+        RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, s));
+        RUN(MTAD_K_GEMM, wb * d.d_model * qd, 1,
+            launch_gemm_rows(sc.attn, qd, m.w(l, 4), nullptr, sc.hidden, d.d_model, 0, T, d.d_model, qd, 1, s));
+        RUN(MTAD_K_NORM, 0, 1, launch_rmsnorm(sc.hidden, m.w(l, 5), sc.xn, T, d.d_model, d.rms_eps, s));
+        RUN(MTAD_K_GEMM, wb * 2.0 * d.d_ffn * d.d_model, 1,
+            launch_gemm_rows(sc.xn, d.d_model, m.w(l, 6), m.w(l, 7), sc.act, d.d_ffn, 0, T, d.d_ffn, d.d_model, 2, s));
+        RUN(MTAD_K_GEMM, wb * d.d_model * d.d_ffn, 1,
+            launch_gemm_rows(sc.act, d.d_ffn, m.w(l, 8), nullptr, sc.hidden, d.d_model, 0, T, d.d_model, d.d_ffn, 1, s));
     }
-    CU(launch_rmsnorm(sc.hidden, static_cast<const __nv_bfloat16*>(d.final_norm), sc.xn, T, d.d_model, d.rms_eps, s));
-    CU(launch_gemm_rows(sc.xn, d.d_model, static_cast<const __nv_bfloat16*>(d.lm_head), nullptr, sc.logits, d.vocab, 0,
-                        T, d.vocab, d.d_model, 0, s));
+    RUN(MTAD_K_NORM, 0, 1,
+        launch_rmsnorm(sc.hidden, static_cast<const __nv_bfloat16*>(d.final_norm), sc.xn, T, d.d_model, d.rms_eps, s));
+    RUN(MTAD_K_GEMM, wb * d.vocab * d.d_model, 1,
+        launch_gemm_rows(sc.xn, d.d_model, static_cast<const __nv_bfloat16*>(d.lm_head), nullptr, sc.logits, d.vocab, 0,
+                         T, d.vocab, d.d_model, 0, s));
     return MTAD_OK;
 }
 
@@ -174,12 +212,13 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
     PrepareArgs pa{};
     for (int i = 0; i < B; ++i) pa.seqs.v[i] = seqs[i];
     pa.B = B; pa.R = R; pa.max_depth = D; pa.n_nodes = n_nodes; pa.tok = tok; pa.parent = parent;
-    CU(launch_prepare(ctx->target, ctx->st, ctx->rm, ctx->sc, pa, out->status, s));
+    RUN(MTAD_K_PREPARE, 0, 1, launch_prepare(ctx->target, ctx->st, ctx->rm, ctx->sc, pa, out->status, s));
     int rc = forward_rows(ctx, ctx->target, B, R, ub, s);
     if (rc != MTAD_OK) return rc;
-    CU(launch_lm_reduce(ctx->target, ctx->rm, ctx->sc, B, R, bonus_uniform, tok, parent, s));
+    RUN(MTAD_K_LMRED, 0, R > 1 ? 2 : 1,
+        launch_lm_reduce(ctx->target, ctx->rm, ctx->sc, B, R, bonus_uniform, tok, parent, s));
     AcceptArgs aa{B, R, D, tok, parent, logq_ref, log_tau};
-    CU(launch_accept(ctx->rm, ctx->sc, aa, *out, s));
+    RUN(MTAD_K_ACCEPT, 0, 1, launch_accept(ctx->rm, ctx->sc, aa, *out, s));
     ctx->last_B = B; ctx->last_R = R; ctx->last_D = D;
     memcpy(ctx->last_seqs, seqs, sizeof(int32_t) * B);
     return MTAD_OK;
@@ -231,9 +270,44 @@ int mtad_create(const mtad_model_desc* target, const mtad_model_desc* aux, int m
 }
 
 int mtad_destroy(mtad_ctx* ctx) {
+    if (ctx)
+        for (cudaEvent_t e : ctx->prof_ev) cudaEventDestroy(e);
     delete ctx;
     return MTAD_OK;
 }
+
+int mtad_profile_begin(mtad_ctx* ctx, int max_launches) {
+    if (!ctx || max_launches < 1 || max_launches > (1 << 20)) return MTAD_E_INVALID;
+    while (ctx->prof_ev.size() < (size_t)max_launches * 2) {
+        cudaEvent_t e;
+        CU(cudaEventCreate(&e));
+        ctx->prof_ev.push_back(e);
+    }
+    ctx->prof_cls.clear();
+    ctx->prof_bytes.clear();
+    ctx->prof_used = 0;
+    ctx->prof_on = true;
+    return MTAD_OK;
+}
+
+int mtad_profile_end(mtad_ctx* ctx, double* ms, double* bytes, int64_t* launches) {
+    if (!ctx || !ms || !bytes || !launches) return MTAD_E_INVALID;
+    ctx->prof_on = false;
+    for (int c = 0; c < MTAD_K_CLASSES; ++c) { ms[c] = 0; bytes[c] = 0; launches[c] = 0; }
+    CU(cudaDeviceSynchronize());
+    for (size_t i = 0; i < ctx->prof_cls.size(); ++i) {
+        float t = 0.f;
+        CU(cudaEventElapsedTime(&t, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]));
+        const int c = ctx->prof_cls[i];
+        ms[c] += t;
+        bytes[c] += ctx->prof_bytes[i];
+        launches[c] += 1;
+    }
+    ctx->prof_used = 0;
+    return MTAD_OK;
+}
+
+uint64_t mtad_kernel_launches(void) { return g_kernel_launches; }
 
 int mtad_seq_set(mtad_ctx* ctx, int seq, int32_t kv_len, int32_t root_token, int32_t aux_len,
                  const int32_t* pending_tok, void* stream) {
@@ -244,7 +318,8 @@ int mtad_seq_set(mtad_ctx* ctx, int seq, int32_t kv_len, int32_t root_token, int
     const int npend = kv_len - aux_len;
     if (npend > MTAD_MAX_DEPTH) return MTAD_E_CAPACITY;
     if (npend > 0 && !pending_tok) return MTAD_E_INVALID;
-    CU(launch_seq_set(ctx->st, seq, kv_len, root_token, aux_len, npend, pending_tok, static_cast<cudaStream_t>(stream)));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    RUN(MTAD_K_PREPARE, 0, 1, launch_seq_set(ctx->st, seq, kv_len, root_token, aux_len, npend, pending_tok, s));
     ctx->len_ub[seq] = kv_len;
     return MTAD_OK;
 }
@@ -291,8 +366,8 @@ int kv_commit(mtad_ctx* ctx, int B, const int32_t* seqs, const mtad_result* res,
     if (!seqs_ok(ctx, B, seqs)) return MTAD_E_INVALID;
     if (B != ctx->last_B || memcmp(seqs, ctx->last_seqs, sizeof(int32_t) * B) != 0) return MTAD_E_INVALID;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    CU(launch_kv_commit(ctx->target, ctx->st, B, ctx->rm.call_seq, *res, ctx->last_D, s));
-    CU(launch_seq_advance(ctx->st, B, ctx->rm.call_seq, *res, ctx->last_D, s));
+    RUN(MTAD_K_COMMIT, 0, 1, launch_kv_commit(ctx->target, ctx->st, B, ctx->rm.call_seq, *res, ctx->last_D, s));
+    RUN(MTAD_K_COMMIT, 0, 1, launch_seq_advance(ctx->st, B, ctx->rm.call_seq, *res, ctx->last_D, s));
     for (int i = 0; i < B; ++i)
         ctx->len_ub[seqs[i]] = std::min<long long>(ctx->len_ub[seqs[i]] + ctx->last_D + 1, ctx->target.d.kv_capacity);
     ctx->last_B = 0;

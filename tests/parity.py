@@ -11,6 +11,7 @@ import torch
 
 import mtad_synth as S
 import paper_2407_09722_b200 as M
+from paper_2407_09722_b200.runtime import DeviceModel
 from oracle import mtad_oracle as O
 from oracle.adapters import oracle_model, bits
 
@@ -18,25 +19,11 @@ LP_TOL = 2e-3          # absolute tolerance on log-probabilities (per token and 
 MARGIN = 1e-3          # decisions closer than this to a boundary are counted, not compared
 
 
-class GpuModel:
+class GpuModel(DeviceModel):
     """Seeded weights + KV cache on the device, the library context, and a lazily built oracle twin."""
 
-    def __init__(self, target: S.ModelShape, max_batch: int, max_nodes: int, capacity: int, seed: int = 0,
-                 aux: Optional[S.ModelShape] = None, aux_capacity: Optional[int] = None):
-        dev = "cuda"
-        self.shape, self.aux_shape, self.seed = target, aux, seed
-        self.max_batch, self.max_nodes, self.capacity = max_batch, max_nodes, capacity
-        self.weights = S.make_model(target, 0, seed, dev)
-        self.cache = torch.zeros(S.kv_cache_shape(target, max_batch, capacity), dtype=torch.bfloat16, device=dev)
-        self._keep: list = []
-        self.desc = M.make_desc(target, self.weights, self.cache, self._keep)
-        self.aux_desc = None
-        if aux is not None:
-            self.aux_weights = S.make_model(aux, 1, seed, dev)
-            self.aux_cache = torch.zeros(S.kv_cache_shape(aux, max_batch, aux_capacity or capacity),
-                                         dtype=torch.bfloat16, device=dev)
-            self.aux_desc = M.make_desc(aux, self.aux_weights, self.aux_cache, self._keep)
-        self.ctx = M.Context(self.desc, self.aux_desc, max_batch, max_nodes, keep=self._keep)
+    def __init__(self, *a, **k):
+        super().__init__(*a, **k)
         self._oracle = None
 
     def oracle(self) -> O.OracleModel:
@@ -47,9 +34,6 @@ class GpuModel:
                 {"shape": s, "embed": w["embed"], "lm_head": w["lm_head"], "final_norm": w["final_norm"]},
                 layer_maker=lambda l: w["layers"][l])
         return self._oracle
-
-    def inject(self, seq: int, length: int):
-        S.fill_kv_cache(self.cache, 0, seq, length, self.seed)
 
     def cache_bits(self, seq: int, upto: int) -> np.ndarray:
         """Host copy of one sequence's cache [layers, 2, Hkv, capacity, hd] as bf16 bits (only [0, upto) filled)."""

@@ -28,7 +28,7 @@ def _desc(shape, ptrs=False):
 
 def test_every_declared_symbol_is_exported(lib):
     header = open(os.path.join(ROOT, "include", "mtad.h")).read()
-    declared = set(re.findall(r"^(?:int|const char\*)\s+(\w+)\(", header, flags=re.M))
+    declared = set(re.findall(r"^(?:int|uint64_t|const char\*)\s+(\w+)\(", header, flags=re.M))
     assert declared == set(M.EXPORTS)
     for name in declared:
         assert hasattr(lib, name), name
