@@ -243,13 +243,13 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
 
     # ---- device-resident timing ---------------------------------------------------------------------------------
     reset()
+    sampler = ClockSampler(local_rank)       # started before the warm-up: nvidia-smi needs a moment to come up
     for i in range(args.warmup):
         inputs[i].verify(ctx, seqs, log_tau, unis[i], res)
         ctx.kv_commit(seqs, res)
     acc_dev = torch.zeros((), dtype=torch.int64, device="cuda")
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
-    sampler = ClockSampler(local_rank)
     launches0 = M.mtad_kernel_launches()
     ev[0].record()
     for k in range(args.steps):
