@@ -163,6 +163,30 @@ int mtad_verify_tree(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n
  * Sequences whose status is non-zero are left untouched. */
 int kv_commit(mtad_ctx* ctx, int B, const int32_t* seqs, const mtad_result* res, void* stream);
 
+/* The paper has no counterpart for this entry point; it exists for callers that cannot allocate device memory.
+ * Some hosts of this library - a plug-in running inside another engine's memory pool, a process whose CUDA
+ * allocator has been frozen after start-up, code that may run while a stream is being captured - are not allowed
+ * to call cudaMalloc, so they cannot supply the workspace that mtad_create wants.  This call verifies one draft
+ * chain for ONE sequence exactly like mtad_verify_chain, but takes its scratch from a fixed array of
+ * MTAD_STATIC_SCRATCH_BYTES that is compiled into the library (every GPU that loads the library holds that much
+ * memory until the process exits).  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   target      descriptor as for mtad_create; its kv_cache must be laid out for max_batch = 1
+ *   kv_len      committed length of the sequence, root_token its last emitted token
+ *   draft_tok, draft_logq, log_tau, bonus_uniform, out: as mtad_verify_chain with B = 1 (device arrays of the caller)
+ * The K/V rows of the root and the draft tokens are left in cache slots kv_len .. kv_len + gamma, as after
+ * mtad_verify_chain; there is no commit step, the caller keeps the rows it accepts.
+ * Limits and sharing: returns MTAD_E_WORKSPACE when the model shape or gamma needs more scratch than the array
+ * holds (mtad_workspace_bytes(target, NULL, 1, gamma) tells how much).  All calls on a device share the one array,
+ * which still contains the previous call's data: the library re-zeroes the parts that must start at zero whenever
+ * the model or gamma changes, but two calls whose GPU work overlaps (different streams, different threads) race
+ * on it - issue them on one stream or synchronise in between.  The first call on a device (and any call that
+ * changes the model or gamma) looks up the array's device address, zeroes it and synchronises the device; make
+ * that call before starting a stream capture. */
+#define MTAD_STATIC_SCRATCH_BYTES (16u << 20)
+int mtad_verify_chain_static(const mtad_model_desc* target, int32_t kv_len, int32_t root_token, int gamma,
+                             const int32_t* draft_tok, const float* draft_logq, float log_tau,
+                             const float* bonus_uniform, const mtad_result* out, void* stream);
+
 /* Instrumentation (not part of the method).  Kernel classes for mtad_profile_end. */
 enum { MTAD_K_PREPARE = 0, MTAD_K_NORM, MTAD_K_GEMM, MTAD_K_ROPE, MTAD_K_ATTN, MTAD_K_LMRED, MTAD_K_ACCEPT,
        MTAD_K_COMMIT, MTAD_K_CLASSES };

@@ -39,7 +39,8 @@ class Result(C.Structure):
 
 EXPORTS = ("mtad_workspace_bytes", "mtad_create", "mtad_destroy", "mtad_seq_set", "mtad_seq_get", "mtad_draft",
            "mtad_verify_chain", "mtad_verify_tree", "kv_commit", "mtad_status_str", "mtad_last_cuda_error",
-           "mtad_profile_begin", "mtad_profile_end", "mtad_kernel_launches")
+           "mtad_profile_begin", "mtad_profile_end", "mtad_kernel_launches", "mtad_verify_chain_static")
+MTAD_STATIC_SCRATCH_BYTES = 16 << 20
 KERNEL_CLASSES = ("prepare", "norm", "gemm", "rope_append", "attention", "lm_reduce", "accept", "commit")
 
 _lib = None
@@ -72,6 +73,7 @@ def load_library() -> C.CDLL:
     lib.mtad_profile_begin.argtypes = [P, I]
     lib.mtad_profile_end.argtypes = [P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     lib.mtad_kernel_launches.argtypes = []
+    lib.mtad_verify_chain_static.argtypes = [MD, C.c_int32, C.c_int32, I, P, P, F, P, RS, P]
     for n in EXPORTS:
         if n not in ("mtad_status_str", "mtad_kernel_launches"):
             getattr(lib, n).restype = I
@@ -247,6 +249,15 @@ class Context:
         if check:
             self._check(rc, "mtad_draft")
         return rc
+
+
+def mtad_verify_chain_static(target: ModelDesc, kv_len: int, root_token: int, gamma: int, draft_tok, draft_logq,
+                             log_tau: float, bonus_uniform, out: "ResultBuffers", stream=None) -> int:
+    """Chain verification for one sequence with the library's built-in scratch array instead of a workspace:
+    for callers that are not allowed to allocate device memory.  Returns the status code (no exception)."""
+    return load_library().mtad_verify_chain_static(
+        C.byref(target), kv_len, root_token, gamma, _ptr(draft_tok, torch.int32), _ptr(draft_logq, torch.float32),
+        log_tau, _ptr(bonus_uniform, torch.float32), C.byref(out.struct), _stream(stream))
 
 
 def mtad_kernel_launches() -> int:
