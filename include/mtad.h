@@ -199,6 +199,10 @@ int mtad_profile_begin(mtad_ctx* ctx, int max_launches);
 int mtad_profile_end(mtad_ctx* ctx, double* ms, double* bytes, int64_t* launches);
 /* Kernels of this library enqueued by this process so far. */
 uint64_t mtad_kernel_launches(void);
+/* Runs the weight-streaming tensor-core GEMM alone: y[T, N] (fp32, device) = x[T, K] (fp32, device) * W[N, K]^T
+ * (bf16, device, 16-byte aligned), T <= 256, K a multiple of 8 and at most the context's largest FFN width.
+ * For unit tests and kernel timing; uses the context's workspace. */
+int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, int T, float* y, void* stream);
 
 const char* mtad_status_str(int status);
 int mtad_last_cuda_error(const mtad_ctx* ctx);

@@ -39,7 +39,8 @@ class Result(C.Structure):
 
 EXPORTS = ("mtad_workspace_bytes", "mtad_create", "mtad_destroy", "mtad_seq_set", "mtad_seq_get", "mtad_draft",
            "mtad_verify_chain", "mtad_verify_tree", "kv_commit", "mtad_status_str", "mtad_last_cuda_error",
-           "mtad_profile_begin", "mtad_profile_end", "mtad_kernel_launches", "mtad_verify_chain_static")
+           "mtad_profile_begin", "mtad_profile_end", "mtad_kernel_launches", "mtad_verify_chain_static",
+           "mtad_debug_gemm")
 MTAD_STATIC_SCRATCH_BYTES = 16 << 20
 KERNEL_CLASSES = ("prepare", "norm", "gemm", "rope_append", "attention", "lm_reduce", "accept", "commit")
 
@@ -73,6 +74,7 @@ def load_library() -> C.CDLL:
     lib.mtad_profile_begin.argtypes = [P, I]
     lib.mtad_profile_end.argtypes = [P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     lib.mtad_kernel_launches.argtypes = []
+    lib.mtad_debug_gemm.argtypes = [P, P, I, I, P, I, P, P]
     lib.mtad_verify_chain_static.argtypes = [MD, C.c_int32, C.c_int32, I, P, P, F, P, RS, P]
     for n in EXPORTS:
         if n not in ("mtad_status_str", "mtad_kernel_launches"):
@@ -229,6 +231,15 @@ class Context:
         rc = self._lib.kv_commit(self.handle, len(seqs), _seqs(seqs), C.byref(res.struct), _stream(stream))
         if check:
             self._check(rc, "kv_commit")
+        return rc
+
+    def mtad_debug_gemm(self, W: torch.Tensor, x: torch.Tensor, y: torch.Tensor, stream=None, check=True) -> int:
+        N, K = W.shape
+        T = x.shape[0]
+        rc = self._lib.mtad_debug_gemm(self.handle, _ptr(W, torch.bfloat16), N, K, _ptr(x, torch.float32), T,
+                                       _ptr(y, torch.float32), _stream(stream))
+        if check:
+            self._check(rc, "mtad_debug_gemm")
         return rc
 
     def mtad_profile_begin(self, max_launches: int = 8192):

@@ -1,16 +1,30 @@
 // Host dispatcher behind the C ABI: argument validation, workspace carving, and the launch sequence of one
 // verification step.  No device memory is allocated here; everything lives in the caller's workspace.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
 #include <new>
 
 #include "common.cuh"
+#include "tc_gemm.cuh"
 
 using namespace mtad;
 
+constexpr int kCtas = 148;     // one persistent CTA per SM in the tensor-core GEMM
+
+// Host-side tensor maps of one model's weight matrices.
+struct WeightMaps {
+    std::vector<CUtensorMap> wq, wk, wv, wo, gate, up, down;
+    CUtensorMap lm_head;
+    bool ok = false;
+};
+
 struct mtad_ctx {
+    WeightMaps tmaps, amaps;
+    bool use_tc = false, use_pdl = false;
+    size_t tc_ws_floats = 0, tc_counter_n = 0, xf_elems = 0;
     ModelView target, aux;
     bool has_aux = false;
     int max_batch = 0, max_nodes = 0, T_max = 0;
@@ -109,7 +123,47 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     sc.row_lse = k.take<float>(T);
     sc.row_cand = k.take<int32_t>(T);
     sc.row_cand_lp = k.take<float>(T);
-    if (c) { c->st = st; c->rm = rm; c->sc = sc; }
+    rm.prow = k.take<int32_t>(T);
+    // tensor-core path buffers (operand rows are always TC_X_ROWS high so that the TMA box never leaves them)
+    const size_t Tc = std::min<size_t>(T, TC_MAX_ROWS);
+    const size_t rpad = (Tc + 15) / 16 * 16;
+    sc.xd_hi = k.take<__nv_bfloat16>((size_t)TC_X_ROWS * d);
+    sc.xd_lo = k.take<__nv_bfloat16>((size_t)TC_X_ROWS * d);
+    sc.xa_hi = k.take<__nv_bfloat16>((size_t)TC_X_ROWS * qd);
+    sc.xa_lo = k.take<__nv_bfloat16>((size_t)TC_X_ROWS * qd);
+    sc.xf_hi = k.take<__nv_bfloat16>((size_t)TC_X_ROWS * F);
+    sc.xf_lo = k.take<__nv_bfloat16>((size_t)TC_X_ROWS * F);
+    const size_t dt = (d + TC_TILE_N - 1) / TC_TILE_N;
+    sc.sumsq_a = k.take<float>(dt * TC_X_ROWS);
+    sc.sumsq_b = k.take<float>(dt * TC_X_ROWS);
+    size_t ws_tiles = 0, max_tiles = 0, lm_tiles = 0;
+    auto shape_ws = [&](const mtad_model_desc* m) {
+        const int qdm = m->n_q_heads * m->head_dim, kvm = m->n_kv_heads * m->head_dim;
+        const int shapes[5][2] = {{(qdm + 127) / 128 + 2 * ((kvm + 127) / 128), m->d_model},
+                                  {(m->d_model + 127) / 128, qdm},
+                                  {(m->d_ffn + 63) / 64, m->d_model},
+                                  {(m->d_model + 127) / 128, m->d_ffn},
+                                  {(m->vocab + 127) / 128, m->d_model}};
+        for (auto& sh : shapes) {
+            TcGemmParams tp{};
+            tc_decompose(tp, sh[0], sh[1], 1, kCtas);
+            ws_tiles = std::max(ws_tiles, (size_t)sh[0] * tp.max_contrib);
+            max_tiles = std::max(max_tiles, (size_t)sh[0]);
+        }
+        lm_tiles = std::max(lm_tiles, (size_t)(m->vocab + 127) / 128);
+    };
+    shape_ws(t);
+    if (a) shape_ws(a);
+    sc.tc_ws = k.take<float>(ws_tiles * rpad * TC_TILE_N);
+    sc.tc_counters = k.take<int32_t>(max_tiles);
+    sc.lm_part = k.take<float4>(Tc * lm_tiles);
+    sc.node_z = k.take<float>(T);
+    if (c) {
+        c->st = st; c->rm = rm; c->sc = sc;
+        c->tc_ws_floats = ws_tiles * rpad * TC_TILE_N;
+        c->tc_counter_n = max_tiles;
+        c->xf_elems = (size_t)TC_X_ROWS * F;
+    }
     return (k.off + 255) & ~size_t(255);
 }
 
@@ -162,7 +216,7 @@ int forward_rows(mtad_ctx* ctx, const ModelView& m, int B, int R, long long len_
         RUN(MTAD_K_GEMM, wb * kvd * d.d_model, 1,
             launch_gemm_rows(sc.xn, d.d_model, m.w(l, 3), nullptr, sc.qkv, ldq, qd + kvd, T, kvd, d.d_model, 0, s));
         RUN(MTAD_K_ROPE, 0, 1, launch_rope_append(m, l, ctx->rm, sc, T, s));
-        RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, s));
+        RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, false, s));
         RUN(MTAD_K_GEMM, wb * d.d_model * qd, 1,
             launch_gemm_rows(sc.attn, qd, m.w(l, 4), nullptr, sc.hidden, d.d_model, 0, T, d.d_model, qd, 1, s));
         RUN(MTAD_K_NORM, 0, 1, launch_rmsnorm(sc.hidden, m.w(l, 5), sc.xn, T, d.d_model, d.rms_eps, s));
@@ -176,6 +230,110 @@ int forward_rows(mtad_ctx* ctx, const ModelView& m, int B, int R, long long len_
     RUN(MTAD_K_GEMM, wb * d.vocab * d.d_model, 1,
         launch_gemm_rows(sc.xn, d.d_model, static_cast<const __nv_bfloat16*>(d.lm_head), nullptr, sc.logits, d.vocab, 0,
                          T, d.vocab, d.d_model, 0, s));
+    return MTAD_OK;
+}
+
+bool build_weight_maps(const ModelView& m, WeightMaps& w) {
+    const mtad_model_desc& d = m.d;
+    const int qd = d.n_q_heads * d.head_dim, kvd = d.n_kv_heads * d.head_dim;
+    auto aligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; };
+    auto mk = [&](CUtensorMap* o, const void* base, long long rows, long long cols, int box) {
+        return aligned(base) && tc_make_map(o, base, rows, cols, box) == 0;
+    };
+    w.wq.resize(d.layers); w.wk.resize(d.layers); w.wv.resize(d.layers); w.wo.resize(d.layers);
+    w.gate.resize(d.layers); w.up.resize(d.layers); w.down.resize(d.layers);
+    bool ok = true;
+    for (int l = 0; l < d.layers && ok; ++l) {
+        ok = ok && mk(&w.wq[l], m.w(l, 1), qd, d.d_model, 128);
+        ok = ok && mk(&w.wk[l], m.w(l, 2), kvd, d.d_model, 128);
+        ok = ok && mk(&w.wv[l], m.w(l, 3), kvd, d.d_model, 128);
+        ok = ok && mk(&w.wo[l], m.w(l, 4), d.d_model, qd, 128);
+        ok = ok && mk(&w.gate[l], m.w(l, 6), d.d_ffn, d.d_model, 64);
+        ok = ok && mk(&w.up[l], m.w(l, 7), d.d_ffn, d.d_model, 64);
+        ok = ok && mk(&w.down[l], m.w(l, 8), d.d_model, d.d_ffn, 128);
+    }
+    ok = ok && mk(&w.lm_head, d.lm_head, d.vocab, d.d_model, 128);
+    w.ok = ok;
+    return ok;
+}
+
+// The same forward on the tensor-core path: every projection is one launch of the TMA + tcgen05 GEMM with a fused
+// epilogue; activations travel between launches as bf16 hi/lo operand rows plus per-row sums of squares, so the
+// RMSNorm is applied as a per-row scale in the consumer's epilogue.  Leaves lm_part / node_z for launch_lm_merge.
+int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int B, int R, long long len_ub,
+                    const float* uniforms, uint32_t* status, cudaStream_t s) {
+    const int T = B * R;
+    const mtad_model_desc& d = m.d;
+    const int qd = d.n_q_heads * d.head_dim, kvd = d.n_kv_heads * d.head_dim;
+    const Scratch& sc = ctx->sc;
+    const long long total = std::min<long long>(len_ub, d.kv_capacity) + R;
+    int nsplit = (int)std::min<long long>(attn_split_cap(d.n_q_heads), (total + MTAD_ATTN_TILE - 1) / MTAD_ATTN_TILE);
+    nsplit = std::max(1, std::min(nsplit, (4 * 148 + d.n_q_heads * B - 1) / (d.n_q_heads * B)));
+    long long chunk = (total + nsplit - 1) / nsplit;
+    chunk = (chunk + MTAD_ATTN_TILE - 1) / MTAD_ATTN_TILE * MTAD_ATTN_TILE;
+    const int rpad = (T + 15) / 16 * 16;
+    const int dt = (d.d_model + TC_TILE_N - 1) / TC_TILE_N;
+    const bool pdl = ctx->use_pdl;
+    // activation operand maps for this call's row count
+    CUtensorMap xd_hi, xd_lo, xa_hi, xa_lo, xf_hi, xf_lo;
+    if (tc_make_map(&xd_hi, sc.xd_hi, TC_X_ROWS, d.d_model, rpad) || tc_make_map(&xd_lo, sc.xd_lo, TC_X_ROWS, d.d_model, rpad) ||
+        tc_make_map(&xa_hi, sc.xa_hi, TC_X_ROWS, qd, rpad) || tc_make_map(&xa_lo, sc.xa_lo, TC_X_ROWS, qd, rpad) ||
+        tc_make_map(&xf_hi, sc.xf_hi, TC_X_ROWS, d.d_ffn, rpad) || tc_make_map(&xf_lo, sc.xf_lo, TC_X_ROWS, d.d_ffn, rpad))
+        return MTAD_E_CUDA;
+    TcGemmParams base{};
+    base.ws = sc.tc_ws; base.counters = sc.tc_counters; base.status = status;
+    base.inv_dim = 1.f / (float)d.d_model; base.eps = d.rms_eps;
+    base.Hq = d.n_q_heads; base.Hkv = d.n_kv_heads; base.hd = d.head_dim;
+    base.q_out = sc.qkv; base.rope = sc.rope; base.cache = static_cast<__nv_bfloat16*>(d.kv_cache);
+    base.slot = ctx->rm.slot; base.seq = ctx->rm.seq; base.max_batch = m.max_batch; base.cap = d.kv_capacity;
+    base.hidden = sc.hidden; base.R = R; base.prow = ctx->rm.prow; base.tok = ctx->rm.tok; base.node_z = sc.node_z;
+    base.lm_part = sc.lm_part; base.uniforms = uniforms;
+    const double wb = 2.0;
+    for (int l = 0; l < d.layers; ++l) {
+        {   // QKV + rotary + append
+            TcGemmParams p = base; TcMaps mp{};
+            const int qt = (qd + 127) / 128, kt = (kvd + 127) / 128;
+            tc_decompose(p, qt + 2 * kt, d.d_model, T, kCtas);
+            p.mode = TC_QKV; p.N = qd; p.seg_k_tile = qt; p.seg_v_tile = qt + kt; p.layer = l;
+            p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = (l == 0) ? 1 : dt;
+            mp.a0 = wm.wq[l]; mp.a1 = wm.wk[l]; mp.a2 = wm.wv[l]; mp.xhi = xd_hi; mp.xlo = xd_lo;
+            RUN(MTAD_K_GEMM, wb * (qd + 2.0 * kvd) * d.d_model, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
+        }
+        RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, true, s));
+        {   // O projection + residual, emits the FFN norm's operand rows
+            TcGemmParams p = base; TcMaps mp{};
+            tc_decompose(p, dt, qd, T, kCtas);
+            p.mode = TC_RESID; p.N = d.d_model; p.sumsq_in_parts = 0;
+            p.gain = m.w(l, 5); p.x_hi = sc.xd_hi; p.x_lo = sc.xd_lo; p.ldx = d.d_model; p.sumsq_out = sc.sumsq_b;
+            mp.a0 = wm.wo[l]; mp.xhi = xa_hi; mp.xlo = xa_lo;
+            RUN(MTAD_K_GEMM, wb * d.d_model * qd, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
+        }
+        {   // gate / up + SwiGLU
+            TcGemmParams p = base; TcMaps mp{};
+            tc_decompose(p, (d.d_ffn + 63) / 64, d.d_model, T, kCtas);
+            p.mode = TC_SWIGLU; p.N = d.d_ffn; p.sumsq_in = sc.sumsq_b; p.sumsq_in_parts = dt;
+            p.x_hi = sc.xf_hi; p.x_lo = sc.xf_lo; p.ldx = d.d_ffn;
+            mp.a0 = wm.gate[l]; mp.a1 = wm.up[l]; mp.xhi = xd_hi; mp.xlo = xd_lo;
+            RUN(MTAD_K_GEMM, wb * 2.0 * d.d_ffn * d.d_model, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
+        }
+        {   // down projection + residual, emits the next norm's operand rows
+            TcGemmParams p = base; TcMaps mp{};
+            tc_decompose(p, dt, d.d_ffn, T, kCtas);
+            p.mode = TC_RESID; p.N = d.d_model; p.sumsq_in_parts = 0;
+            p.gain = (l + 1 < d.layers) ? m.w(l + 1, 0) : static_cast<const __nv_bfloat16*>(d.final_norm);
+            p.x_hi = sc.xd_hi; p.x_lo = sc.xd_lo; p.ldx = d.d_model; p.sumsq_out = sc.sumsq_a;
+            mp.a0 = wm.down[l]; mp.xhi = xf_hi; mp.xlo = xf_lo;
+            RUN(MTAD_K_GEMM, wb * d.d_model * d.d_ffn, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
+        }
+    }
+    {   // LM head + per-tile log-softmax / Gumbel-argmax partials + gather of the drafted tokens' logits
+        TcGemmParams p = base; TcMaps mp{};
+        tc_decompose(p, (d.vocab + 127) / 128, d.d_model, T, kCtas);
+        p.mode = TC_LMHEAD; p.N = d.vocab; p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = dt;
+        mp.a0 = wm.lm_head; mp.xhi = xd_hi; mp.xlo = xd_lo;
+        RUN(MTAD_K_GEMM, wb * d.vocab * d.d_model, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
+        RUN(MTAD_K_LMRED, 0, 2, launch_lm_merge(m, ctx->rm, sc, B, R, p.n_tiles, uniforms, s));
+    }
     return MTAD_OK;
 }
 
@@ -212,11 +370,21 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
     PrepareArgs pa{};
     for (int i = 0; i < B; ++i) pa.seqs.v[i] = seqs[i];
     pa.B = B; pa.R = R; pa.max_depth = D; pa.n_nodes = n_nodes; pa.tok = tok; pa.parent = parent;
+    const bool tc = ctx->use_tc && ctx->tmaps.ok && B * R <= TC_MAX_ROWS;
+    if (tc) {
+        pa.gain0 = ctx->target.w(0, 0); pa.x_hi = ctx->sc.xd_hi; pa.x_lo = ctx->sc.xd_lo;
+        pa.sumsq_out = ctx->sc.sumsq_a;
+    }
     RUN(MTAD_K_PREPARE, 0, 1, launch_prepare(ctx->target, ctx->st, ctx->rm, ctx->sc, pa, out->status, s));
-    int rc = forward_rows(ctx, ctx->target, B, R, ub, s);
-    if (rc != MTAD_OK) return rc;
-    RUN(MTAD_K_LMRED, 0, R > 1 ? 2 : 1,
-        launch_lm_reduce(ctx->target, ctx->rm, ctx->sc, B, R, bonus_uniform, tok, parent, s));
+    if (tc) {
+        int rc = forward_rows_tc(ctx, ctx->target, ctx->tmaps, B, R, ub, bonus_uniform, out->status, s);
+        if (rc != MTAD_OK) return rc;
+    } else {
+        int rc = forward_rows(ctx, ctx->target, B, R, ub, s);
+        if (rc != MTAD_OK) return rc;
+        RUN(MTAD_K_LMRED, 0, R > 1 ? 2 : 1,
+            launch_lm_reduce(ctx->target, ctx->rm, ctx->sc, B, R, bonus_uniform, tok, parent, s));
+    }
     AcceptArgs aa{B, R, D, tok, parent, logq_ref, log_tau};
     RUN(MTAD_K_ACCEPT, 0, 1, launch_accept(ctx->rm, ctx->sc, aa, *out, s));
     ctx->last_B = B; ctx->last_R = R; ctx->last_D = D;
@@ -262,6 +430,12 @@ int mtad_create(const mtad_model_desc* target, const mtad_model_desc* aux, int m
     ctx->T_max = max_batch * (max_nodes + 1);
     ctx->len_ub.assign(max_batch, 0);
     carve(ctx, target, aux, max_batch, max_nodes, workspace);
+    // tensor-core path unless MTAD_PATH=simt asks for the CUDA-core kernels (or a weight pointer is not 16-byte aligned)
+    const char* path = getenv("MTAD_PATH");
+    ctx->use_tc = !(path && strcmp(path, "simt") == 0) && build_weight_maps(ctx->target, ctx->tmaps);
+    if (ctx->use_tc && aux) build_weight_maps(ctx->aux, ctx->amaps);
+    const char* pdl = getenv("MTAD_PDL");
+    ctx->use_pdl = pdl && strcmp(pdl, "1") == 0;
     cudaError_t e = cudaMemset(workspace, 0, need);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete ctx; return MTAD_E_CUDA; }
@@ -308,6 +482,26 @@ int mtad_profile_end(mtad_ctx* ctx, double* ms, double* bytes, int64_t* launches
 }
 
 uint64_t mtad_kernel_launches(void) { return g_kernel_launches; }
+
+int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, int T, float* y, void* stream) {
+    if (!ctx || !W || !x || !y || N < 1 || K < 8 || (K % 8) || T < 1) return MTAD_E_INVALID;
+    if (T > TC_MAX_ROWS || (size_t)TC_X_ROWS * K > ctx->xf_elems) return MTAD_E_CAPACITY;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    TcGemmParams p{};
+    tc_decompose(p, (N + TC_TILE_N - 1) / TC_TILE_N, K, T, kCtas);
+    if ((size_t)p.n_tiles * p.max_contrib * p.rpad * TC_TILE_N > ctx->tc_ws_floats ||
+        (size_t)p.n_tiles > ctx->tc_counter_n)
+        return MTAD_E_WORKSPACE;
+    TcMaps mp{};
+    if (tc_make_map(&mp.a0, W, N, K, 128) || tc_make_map(&mp.xhi, ctx->sc.xf_hi, TC_X_ROWS, K, p.rpad) ||
+        tc_make_map(&mp.xlo, ctx->sc.xf_lo, TC_X_ROWS, K, p.rpad))
+        return MTAD_E_CUDA;
+    p.mode = TC_PLAIN; p.N = N; p.out = y; p.ldo = N;
+    p.ws = ctx->sc.tc_ws; p.counters = ctx->sc.tc_counters; p.status = nullptr;
+    RUN(MTAD_K_PREPARE, 0, 1, launch_split_rows(x, K, ctx->sc.xf_hi, ctx->sc.xf_lo, K, T, K, s));
+    RUN(MTAD_K_GEMM, 2.0 * N * K, 1, launch_tc_gemm(mp, p, kCtas, false, s));
+    return MTAD_OK;
+}
 
 int mtad_seq_set(mtad_ctx* ctx, int seq, int32_t kv_len, int32_t root_token, int32_t aux_len,
                  const int32_t* pending_tok, void* stream) {

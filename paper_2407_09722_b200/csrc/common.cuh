@@ -26,6 +26,7 @@ struct RowMeta {
     int32_t* n_rows;     // [B] active rows of sequence bi (n_nodes + 1, 0 if the sequence is rejected)
     int32_t* kv_base;    // [B] committed length L seen by this call
     int32_t* call_seq;   // [B] sequence ids of the call
+    int32_t* prow;       // [T] global row of a node row's parent, -1 for roots and inactive rows
 };
 
 struct ModelView {
@@ -58,6 +59,16 @@ struct Scratch {
     float* row_lse;      // [T]
     int32_t* row_cand;   // [T]
     float* row_cand_lp;  // [T]
+    // tensor-core path: bf16 hi/lo operand rows, deferred-norm statistics, split-K workspace, LM-head partials
+    __nv_bfloat16 *xd_hi, *xd_lo;      // [256, d]   input of QKV / gate-up / LM head (un-normalised hidden * gain)
+    __nv_bfloat16 *xa_hi, *xa_lo;      // [256, Hq hd] attention output
+    __nv_bfloat16 *xf_hi, *xf_lo;      // [256, F]   SwiGLU output
+    float* sumsq_a;      // [tiles(d)][256] sums of squares of the hidden rows (after down proj / embedding)
+    float* sumsq_b;      // [tiles(d)][256] the same after the O projection
+    float* tc_ws;        // split-K partial tiles
+    int32_t* tc_counters;
+    float4* lm_part;     // [T][tiles(V)]
+    float* node_z;       // [T]
 };
 
 inline int attn_split_cap(int n_q_heads) {
@@ -77,6 +88,10 @@ struct PrepareArgs {
     const int32_t* n_nodes;    // device [B] or nullptr (all sequences have R-1 nodes)
     const int32_t* tok;        // device [B, R-1]
     const int32_t* parent;     // device [B, R-1] or nullptr (chain)
+    // tensor-core path (null otherwise): first layer's norm gains, operand rows and row statistics to emit
+    const __nv_bfloat16* gain0;
+    __nv_bfloat16 *x_hi, *x_lo;
+    float* sumsq_out;
 };
 
 cudaError_t launch_prepare(const ModelView& m, const SeqState& s, const RowMeta& rm, const Scratch& sc,
@@ -89,7 +104,9 @@ cudaError_t launch_gemm_rows(const float* x, int ldx, const __nv_bfloat16* W, co
 cudaError_t launch_rope_append(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int T,
                                cudaStream_t st);
 cudaError_t launch_attention(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int B, int R,
-                             int nsplit, int chunk, cudaStream_t st);
+                             int nsplit, int chunk, bool emit_split, cudaStream_t st);
+cudaError_t launch_lm_merge(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int n_tiles,
+                            const float* bonus_uniform, cudaStream_t st);
 cudaError_t launch_lm_reduce(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R,
                              const float* bonus_uniform, const int32_t* tok, const int32_t* parent,
                              cudaStream_t st);

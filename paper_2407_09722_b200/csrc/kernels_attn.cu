@@ -136,10 +136,16 @@ __global__ void __launch_bounds__(128) attn_partial_kernel(const float* __restri
 // merge the split partials of one (row, head) in split order
 template <int HD>
 __global__ void attn_combine_kernel(const float* __restrict__ part, float* __restrict__ out, const int32_t* slot,
-                                    int Hq, int nsplit) {
+                                    int Hq, int nsplit, __nv_bfloat16* __restrict__ x_hi,
+                                    __nv_bfloat16* __restrict__ x_lo) {
     const int t = blockIdx.x, h = blockIdx.y, d = threadIdx.x;
-    float* dst = out + ((size_t)t * Hq + h) * HD + d;
-    if (slot[t] < 0) { *dst = 0.f; return; }
+    const size_t idx = ((size_t)t * Hq + h) * HD + d;
+    float* dst = out + idx;
+    if (slot[t] < 0) {
+        *dst = 0.f;
+        if (x_hi) { x_hi[idx] = __float2bfloat16_rn(0.f); x_lo[idx] = __float2bfloat16_rn(0.f); }
+        return;
+    }
     const float* p = part + (((size_t)t * Hq + h) * nsplit) * (HD + 2);
     float M = -CUDART_INF_F;
     for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p[s * (HD + 2)]);
@@ -151,28 +157,36 @@ __global__ void attn_combine_kernel(const float* __restrict__ part, float* __res
         lsum += p[s * (HD + 2) + 1] * w;
         acc += p[s * (HD + 2) + 2 + d] * w;
     }
-    *dst = acc / lsum;
+    const float y = acc / lsum;
+    *dst = y;
+    if (x_hi) {      // operand rows of the O projection: bf16 hi + lo
+        const __nv_bfloat16 hb = __float2bfloat16_rn(y);
+        x_hi[idx] = hb;
+        x_lo[idx] = __float2bfloat16_rn(y - __bfloat162float(hb));
+    }
 }
 
 cudaError_t launch_attention(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int B, int R,
-                             int nsplit, int chunk, cudaStream_t st) {
+                             int nsplit, int chunk, bool emit_split, cudaStream_t st) {
     const int Hq = m.d.n_q_heads, Hkv = m.d.n_kv_heads, hd = m.d.head_dim;
     const int ldq = (Hq + 2 * Hkv) * hd;
     dim3 grid(Hq, nsplit, B);
     const __nv_bfloat16* cache = static_cast<const __nv_bfloat16*>(m.d.kv_cache);
     dim3 cgrid(B * R, Hq);
+    __nv_bfloat16* xh = emit_split ? sc.xa_hi : nullptr;
+    __nv_bfloat16* xl = emit_split ? sc.xa_lo : nullptr;
     if (hd == 128) {
         attn_partial_kernel<128><<<grid, 128, 0, st>>>(sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
                                                        Hkv, (long long)m.d.kv_capacity, R, nsplit, chunk);
-        attn_combine_kernel<128><<<cgrid, 128, 0, st>>>(sc.attn_part, sc.attn, rm.slot, Hq, nsplit);
+        attn_combine_kernel<128><<<cgrid, 128, 0, st>>>(sc.attn_part, sc.attn, rm.slot, Hq, nsplit, xh, xl);
     } else if (hd == 64) {
         attn_partial_kernel<64><<<grid, 128, 0, st>>>(sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
                                                       Hkv, (long long)m.d.kv_capacity, R, nsplit, chunk);
-        attn_combine_kernel<64><<<cgrid, 64, 0, st>>>(sc.attn_part, sc.attn, rm.slot, Hq, nsplit);
+        attn_combine_kernel<64><<<cgrid, 64, 0, st>>>(sc.attn_part, sc.attn, rm.slot, Hq, nsplit, xh, xl);
     } else if (hd == 32) {
         attn_partial_kernel<32><<<grid, 128, 0, st>>>(sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
                                                       Hkv, (long long)m.d.kv_capacity, R, nsplit, chunk);
-        attn_combine_kernel<32><<<cgrid, 32, 0, st>>>(sc.attn_part, sc.attn, rm.slot, Hq, nsplit);
+        attn_combine_kernel<32><<<cgrid, 32, 0, st>>>(sc.attn_part, sc.attn, rm.slot, Hq, nsplit, xh, xl);
     } else {
         return cudaErrorInvalidValue;
     }

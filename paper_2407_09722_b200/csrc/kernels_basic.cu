@@ -114,6 +114,12 @@ __global__ void prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, i
         rm.seq[t] = seq;
 #pragma unroll
         for (int i = 0; i < MTAD_MASK_WORDS; ++i) rm.mask[(size_t)t * MTAD_MASK_WORDS + i] = mask[i];
+        int pr = -1;
+        if (active && r > 0 && !(st & MTAD_ST_BAD_PARENT)) {
+            const int p0 = a.parent ? a.parent[bi * N + (r - 1)] : r - 2;
+            pr = bi * a.R + p0 + 1;
+        }
+        rm.prow[t] = pr;
         if (r == 0) {
             rm.n_rows[bi] = seq_ok ? nn + 1 : 0;
             rm.kv_base[bi] = L;
@@ -126,8 +132,23 @@ __global__ void prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, i
     __syncthreads();
     const int tok = sh_tok;
     const bool ok = sh_ok;
-    for (int i = threadIdx.x; i < d; i += blockDim.x)
-        hidden[(size_t)t * d + i] = ok ? __bfloat162float(embed[(size_t)tok * d + i]) : 0.f;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        const float v = ok ? __bfloat162float(embed[(size_t)tok * d + i]) : 0.f;
+        hidden[(size_t)t * d + i] = v;
+        if (a.x_hi) {
+            const float y = v * __bfloat162float(a.gain0[i]);
+            const __nv_bfloat16 h = __float2bfloat16_rn(y);
+            a.x_hi[(size_t)t * d + i] = h;
+            a.x_lo[(size_t)t * d + i] = __float2bfloat16_rn(y - __bfloat162float(h));
+            ss += v * v;
+        }
+    }
+    if (a.x_hi) {
+        __shared__ float red[32];
+        ss = block_sum(ss, red);
+        if (threadIdx.x == 0) a.sumsq_out[t] = ss;
+    }
     // rotary table in double: angle = pos * base^(-2i/hd)
     for (int i = threadIdx.x; i < hd / 2; i += blockDim.x) {
         const double inv = exp2(-(2.0 * i / hd) * log2(rope_base));
@@ -415,6 +436,72 @@ cudaError_t launch_lm_reduce(const ModelView& m, const RowMeta& rm, const Scratc
         e = cudaGetLastError();
     }
     return e;
+}
+
+// Merge of the LM-head kernel's per-(row, vocab tile) partials, in tile order: log-sum-exp, Gumbel-argmax candidate
+// and its log-probability per row, then the log-probability of every node's token under its parent row.
+__global__ void lm_merge_kernel(const float4* __restrict__ part, int n_tiles, int V, int R,
+                                const float* __restrict__ uni, const int32_t* __restrict__ slot,
+                                float* __restrict__ row_lse, int32_t* __restrict__ row_cand,
+                                float* __restrict__ row_cand_lp) {
+    const int t = blockIdx.x, bi = t / R;
+    if (slot[t] < 0) {
+        if (threadIdx.x == 0) { row_lse[t] = 0.f; row_cand[t] = 0; row_cand_lp[t] = 0.f; }
+        return;
+    }
+    float m = -CUDART_INF_F, s = 0.f;
+    Best best{-CUDART_INF_F, 0x7fffffff};
+    for (int j = threadIdx.x; j < n_tiles; j += blockDim.x) {
+        const float4 q = part[(size_t)t * n_tiles + j];
+        const float mm = fmaxf(m, q.x);
+        s = (m == -CUDART_INF_F ? 0.f : s * expf(m - mm)) + (q.x == -CUDART_INF_F ? 0.f : q.y * expf(q.x - mm));
+        m = mm;
+        best = better(best, Best{q.z, __float_as_int(q.w)});
+    }
+    __shared__ float sm[256], ss[256], sv[256];
+    __shared__ int si[256];
+    sm[threadIdx.x] = m; ss[threadIdx.x] = s; sv[threadIdx.x] = best.v; si[threadIdx.x] = best.i;
+    __syncthreads();
+    for (int o = blockDim.x >> 1; o > 0; o >>= 1) {
+        if (threadIdx.x < o) {
+            const float m1 = sm[threadIdx.x], m2 = sm[threadIdx.x + o];
+            const float mm = fmaxf(m1, m2);
+            const float s1 = (m1 == -CUDART_INF_F) ? 0.f : ss[threadIdx.x] * expf(m1 - mm);
+            const float s2 = (m2 == -CUDART_INF_F) ? 0.f : ss[threadIdx.x + o] * expf(m2 - mm);
+            sm[threadIdx.x] = mm; ss[threadIdx.x] = s1 + s2;
+            const Best b = better(Best{sv[threadIdx.x], si[threadIdx.x]},
+                                  Best{sv[threadIdx.x + o], si[threadIdx.x + o]});
+            sv[threadIdx.x] = b.v; si[threadIdx.x] = b.i;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const float lse = sm[0] + logf(ss[0]);
+        const int c = si[0];
+        row_lse[t] = lse;
+        row_cand[t] = c;
+        // the partial keeps logit + noise; take the noise off again to get the candidate's logit
+        const float g = -logf(-logf(uni[(size_t)bi * V + c]));
+        row_cand_lp[t] = (sv[0] - g) - lse;
+    }
+}
+
+__global__ void node_lp_from_z_kernel(const float* __restrict__ node_z, const int32_t* __restrict__ prow,
+                                      const float* __restrict__ row_lse, float* __restrict__ node_lp, int T) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    const int pr = prow[t];
+    node_lp[t] = pr >= 0 ? node_z[t] - row_lse[pr] : 0.f;
+}
+
+cudaError_t launch_lm_merge(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int n_tiles,
+                            const float* bonus_uniform, cudaStream_t st) {
+    lm_merge_kernel<<<B * R, 256, 0, st>>>(sc.lm_part, n_tiles, m.d.vocab, R, bonus_uniform, rm.slot, sc.row_lse,
+                                           sc.row_cand, sc.row_cand_lp);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    node_lp_from_z_kernel<<<(B * R + 127) / 128, 128, 0, st>>>(sc.node_z, rm.prow, sc.row_lse, sc.node_lp, B * R);
+    return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------------------------------------------

@@ -1,0 +1,613 @@
+// Tensor-core weight-streaming GEMM for the skinny projections of the verification step.
+//
+//   acc[n, r] = sum_k W[n, k] * (x_hi[r, k] + x_lo[r, k])          n: output feature, r: draft row
+//
+// The weight matrix is the 128-row MMA operand (A), the draft rows are the MMA N dimension (B), both K-major bf16
+// tiles of 64 elements (one 128-byte swizzled row) brought in by TMA; fp32 accumulators live in tensor memory.
+// The fp32 activations arrive split into bf16 hi + lo rows, so the tensor cores see them to ~2^-17 relative;
+// the two products accumulate into the same TMEM columns.  Work is cut into (tile, k-block) units dealt out
+// evenly to the CTAs (one per SM); a tile whose k-range spans several CTAs is completed by whichever of them
+// arrives last, which sums the partial tiles in CTA order (deterministic) and runs the fused epilogue.
+//
+// Warp roles: 0 = TMA producer, 1 = TMEM owner + MMA issuer, 2..5 = epilogue (one TMEM lane quadrant each).
+// Every wait on an mbarrier is bounded; on a time-out the kernel raises MTAD_ST_TIMEOUT, waits (bounded) for its
+// own copies in flight, frees its tensor memory and returns.
+#include <math_constants.h>
+
+#include "tc_gemm.cuh"
+
+namespace mtad {
+namespace {
+
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr int MAX_STAGES = 12;
+constexpr int EPI_THREADS = 128;
+constexpr int EPI_ROWS = 16;                      // draft rows finished per epilogue pass
+constexpr uint64_t HINT_STREAM = 0x12F0000000000000ull;   // evict-first: weights are read once
+constexpr uint64_t HINT_KEEP = 0x14F0000000000000ull;     // evict-last: activation operands are re-read by every CTA
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out here or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        if (mbar_test(bar, parity)) return true;
+        if (it > 64) __nanosleep(32);
+        if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y,
+                                            uint64_t hint) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y), "l"(hint)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// D[tmem] (+)= A[smem desc] * B[smem desc]^T, bf16 operands, fp32 accumulate, M = 128.
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// K-major, 128-byte swizzle: 8-row groups 1024 bytes apart; start address advances 32 bytes per 16-element k step.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15},"
+        " [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+__device__ __forceinline__ void split_store(float y, __nv_bfloat16* hi, __nv_bfloat16* lo) {
+    const __nv_bfloat16 h = __float2bfloat16_rn(y);
+    *hi = h;
+    *lo = __float2bfloat16_rn(y - __bfloat162float(h));
+}
+
+struct Smem {
+    uint8_t* ring;
+    float (*epi)[TC_TILE_N + 1];
+    float* rstd;
+    float* red;            // [4][EPI_ROWS] floats, also reused as [4][EPI_ROWS] float4 via red4
+    float4* red4;
+    uint64_t* full;
+    uint64_t* empty;
+    uint64_t* tfull;
+    uint64_t* tempty;
+    uint32_t* tmem_ptr;
+    int* abort_flag;
+    int* flags;            // [0] last-arriver flag, [1..4] epilogue warp wait results
+};
+
+__device__ __forceinline__ Smem carve(uint8_t* base, int stages, int stage_bytes) {
+    Smem s;
+    s.ring = base;
+    uint8_t* p = base + (size_t)stages * stage_bytes;
+    s.epi = reinterpret_cast<float(*)[TC_TILE_N + 1]>(p);
+    p += sizeof(float) * EPI_ROWS * (TC_TILE_N + 1);
+    s.rstd = reinterpret_cast<float*>(p);
+    p += sizeof(float) * TC_MAX_ROWS;
+    p = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(p) + 15) & ~uintptr_t(15));
+    s.red4 = reinterpret_cast<float4*>(p);
+    s.red = reinterpret_cast<float*>(p);
+    p += sizeof(float4) * 4 * EPI_ROWS * 2;
+    s.full = reinterpret_cast<uint64_t*>(p);
+    p += 8 * MAX_STAGES;
+    s.empty = reinterpret_cast<uint64_t*>(p);
+    p += 8 * MAX_STAGES;
+    s.tfull = reinterpret_cast<uint64_t*>(p);
+    p += 16;
+    s.tempty = reinterpret_cast<uint64_t*>(p);
+    p += 16;
+    s.tmem_ptr = reinterpret_cast<uint32_t*>(p);
+    p += 8;
+    s.abort_flag = reinterpret_cast<int*>(p);
+    p += 8;
+    s.flags = reinterpret_cast<int*>(p);
+    return s;
+}
+
+constexpr size_t SMEM_TAIL = sizeof(float) * EPI_ROWS * (TC_TILE_N + 1) + sizeof(float) * TC_MAX_ROWS + 16 +
+                             sizeof(float4) * 4 * EPI_ROWS * 2 + 8 * MAX_STAGES * 2 + 16 + 16 + 8 + 8 + 32;
+
+// ---------------------------------------------------------------------------------------------------------------
+// epilogues: called by the 128 epilogue threads for a block of EPI_ROWS finished rows held in s.epi[j][i]
+// (j: row r0 + j, i: feature n0 + i of the tile).  e = epilogue thread index 0..127.
+// ---------------------------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ void epi_plain(const TcGemmParams& p, const Smem& s, int tile, int r0, int e) {
+    const int n = tile * TC_TILE_N + e;
+    if (n >= p.N) return;
+    for (int j = 0; j < EPI_ROWS && r0 + j < p.T; ++j) p.out[(size_t)(r0 + j) * p.ldo + n] = s.epi[j][e];
+}
+
+__device__ __forceinline__ void epi_qkv(const TcGemmParams& p, const Smem& s, int tile, int r0, int e) {
+    const int hd = p.hd, half = hd >> 1;
+    int seg, tin;
+    if (tile < p.seg_k_tile) { seg = 0; tin = tile; }
+    else if (tile < p.seg_v_tile) { seg = 1; tin = tile - p.seg_k_tile; }
+    else { seg = 2; tin = tile - p.seg_v_tile; }
+    const int f = tin * TC_TILE_N + e;
+    const int head = f / hd, jin = f % hd;
+    const int heads = seg == 0 ? p.Hq : p.Hkv;
+    if (head >= heads) return;
+    const int ldq = (p.Hq + 2 * p.Hkv) * hd;
+    const float scale = rsqrtf((float)hd);
+    for (int j = 0; j < EPI_ROWS && r0 + j < p.T; ++j) {
+        const int t = r0 + j;
+        if (seg == 2) {
+            const int sl = p.slot[t];
+            if (sl < 0) continue;
+            const size_t base = (((((size_t)p.layer * p.max_batch + p.seq[t]) * 2 + 1) * p.Hkv + head) * p.cap + sl) * hd;
+            p.cache[base + jin] = __float2bfloat16_rn(s.epi[j][e]);
+        } else if (jin < half) {
+            const float c = p.rope[((size_t)t * half + jin) * 2], sn = p.rope[((size_t)t * half + jin) * 2 + 1];
+            const float a = s.epi[j][e], b = s.epi[j][e + half];
+            const float ra = a * c - b * sn, rb = b * c + a * sn;
+            if (seg == 0) {
+                float* q = p.q_out + (size_t)t * ldq + head * hd;
+                q[jin] = ra * scale;
+                q[jin + half] = rb * scale;
+            } else {
+                const int sl = p.slot[t];
+                if (sl < 0) continue;
+                const size_t base =
+                    (((((size_t)p.layer * p.max_batch + p.seq[t]) * 2 + 0) * p.Hkv + head) * p.cap + sl) * hd;
+                p.cache[base + jin] = __float2bfloat16_rn(ra);
+                p.cache[base + jin + half] = __float2bfloat16_rn(rb);
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void epi_resid(const TcGemmParams& p, const Smem& s, int tile, int r0, int e) {
+    const int n = tile * TC_TILE_N + e;
+    const bool ok = n < p.N;
+    const float g = ok ? __bfloat162float(p.gain[n]) : 0.f;
+    const int warp = e >> 5, lane = e & 31;
+    for (int j = 0; j < EPI_ROWS; ++j) {
+        const int t = r0 + j;
+        float y = 0.f;
+        if (ok && t < p.T) {
+            y = p.hidden[(size_t)t * p.N + n] + s.epi[j][e];
+            p.hidden[(size_t)t * p.N + n] = y;
+            split_store(y * g, p.x_hi + (size_t)t * p.ldx + n, p.x_lo + (size_t)t * p.ldx + n);
+        }
+        float sq = y * y;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+        if (lane == 0) s.red[warp * EPI_ROWS + j] = sq;
+    }
+    epi_bar();
+    if (e < EPI_ROWS && r0 + e < p.T)
+        p.sumsq_out[(size_t)tile * TC_X_ROWS + r0 + e] =
+            (s.red[e] + s.red[EPI_ROWS + e]) + (s.red[2 * EPI_ROWS + e] + s.red[3 * EPI_ROWS + e]);
+}
+
+__device__ __forceinline__ void epi_swiglu(const TcGemmParams& p, const Smem& s, int tile, int r0, int e) {
+    if (e >= 64) return;
+    const int f = tile * 64 + e;
+    if (f >= p.N) return;
+    for (int j = 0; j < EPI_ROWS && r0 + j < p.T; ++j) {
+        const float g = s.epi[j][e], u = s.epi[j][e + 64];
+        const float a = g / (1.f + expf(-g)) * u;
+        split_store(a, p.x_hi + (size_t)(r0 + j) * p.ldx + f, p.x_lo + (size_t)(r0 + j) * p.ldx + f);
+    }
+}
+
+__device__ __forceinline__ void epi_lmhead(const TcGemmParams& p, const Smem& s, int tile, int r0, int e) {
+    const int v = tile * TC_TILE_N + e;
+    const bool ok = v < p.N;
+    const int warp = e >> 5, lane = e & 31;
+    for (int j = 0; j < EPI_ROWS; ++j) {
+        const int t = r0 + j;
+        float m = -CUDART_INF_F, sum = 0.f, bv = -CUDART_INF_F;
+        int bi = 0x7fffffff;
+        if (ok && t < p.T) {
+            const float z = s.epi[j][e];
+            m = z;
+            sum = 1.f;
+            const float u = p.uniforms[(size_t)(t / p.R) * p.N + v];
+            bv = z - logf(-logf(u));
+            bi = v;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, sum, o);
+            const float v2 = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int i2 = __shfl_xor_sync(0xffffffffu, bi, o);
+            const float mm = fmaxf(m, m2);
+            sum = (m == -CUDART_INF_F ? 0.f : sum * expf(m - mm)) + (m2 == -CUDART_INF_F ? 0.f : s2 * expf(m2 - mm));
+            m = mm;
+            if (v2 > bv || (v2 == bv && i2 < bi)) { bv = v2; bi = i2; }
+        }
+        if (lane == 0) s.red4[warp * EPI_ROWS + j] = make_float4(m, sum, bv, __int_as_float(bi));
+    }
+    epi_bar();
+    if (e < EPI_ROWS && r0 + e < p.T) {
+        float4 a = s.red4[e];
+        for (int w = 1; w < 4; ++w) {
+            const float4 b = s.red4[w * EPI_ROWS + e];
+            const float mm = fmaxf(a.x, b.x);
+            const float sa = a.x == -CUDART_INF_F ? 0.f : a.y * expf(a.x - mm);
+            const float sb = b.x == -CUDART_INF_F ? 0.f : b.y * expf(b.x - mm);
+            a.x = mm;
+            a.y = sa + sb;
+            if (b.z > a.z || (b.z == a.z && __float_as_int(b.w) < __float_as_int(a.w))) { a.z = b.z; a.w = b.w; }
+        }
+        p.lm_part[(size_t)(r0 + e) * p.n_tiles + tile] = a;
+    }
+    // gather: logit of each node's token under its parent row, when both fall into this block of rows and this tile
+    const int n0 = tile * TC_TILE_N;
+    for (int t = e; t < p.T; t += EPI_THREADS) {
+        const int pr = p.prow[t];
+        if (pr < r0 || pr >= r0 + EPI_ROWS) continue;
+        const int tk = p.tok[t] - n0;
+        if (tk >= 0 && tk < TC_TILE_N) p.node_z[t] = s.epi[pr - r0][tk];
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// kernel
+// ---------------------------------------------------------------------------------------------------------------
+
+__global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__ TcMaps maps, const TcGemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int b_bytes = p.rpad * 128;
+    const int stage_bytes = TC_TILE_N * 128 + 2 * b_bytes;
+    const Smem s = carve(smem_base, p.stages, stage_bytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int u_begin = blockIdx.x * p.units_per_cta;
+    const int u_end = min(u_begin + p.units_per_cta, p.total_units);
+    const int n_units = max(u_end - u_begin, 0);
+    const int KB = p.k_blocks;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < 2 * p.rpad) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < p.stages; ++i) {
+            mbar_init(smem_u32(&s.full[i]), 1);
+            mbar_init(smem_u32(&s.empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&s.tfull[i]), 1);
+            mbar_init(smem_u32(&s.tempty[i]), 4);
+        }
+        *s.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s.tmem_ptr)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *s.tmem_ptr;
+    // let the next kernel in the stream start its own prologue (it waits for this grid before it reads our output)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    volatile int* abort_flag = s.abort_flag;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0 && n_units > 0) {
+            const int box_half = p.mode == TC_SWIGLU;
+            auto issue_a = [&](int i) {
+                const int u = u_begin + i, tile = u / KB, kb = u % KB, st = i % p.stages;
+                const uint32_t bar = smem_u32(&s.full[st]);
+                const uint32_t dst = smem_u32(s.ring + (size_t)st * stage_bytes);
+                mbar_expect_tx(bar, (uint32_t)stage_bytes);
+                if (box_half) {
+                    tma_load_2d(dst, &maps.a0, bar, kb * TC_TILE_K, tile * 64, HINT_STREAM);
+                    tma_load_2d(dst + 64 * 128, &maps.a1, bar, kb * TC_TILE_K, tile * 64, HINT_STREAM);
+                } else if (p.mode == TC_QKV) {
+                    const CUtensorMap* m = tile < p.seg_k_tile ? &maps.a0 : (tile < p.seg_v_tile ? &maps.a1 : &maps.a2);
+                    const int tin = tile < p.seg_k_tile ? tile : (tile < p.seg_v_tile ? tile - p.seg_k_tile
+                                                                                       : tile - p.seg_v_tile);
+                    tma_load_2d(dst, m, bar, kb * TC_TILE_K, tin * TC_TILE_N, HINT_STREAM);
+                } else {
+                    tma_load_2d(dst, &maps.a0, bar, kb * TC_TILE_K, tile * TC_TILE_N, HINT_STREAM);
+                }
+            };
+            auto issue_b = [&](int i) {
+                const int u = u_begin + i, kb = u % KB, st = i % p.stages;
+                const uint32_t bar = smem_u32(&s.full[st]);
+                const uint32_t dst = smem_u32(s.ring + (size_t)st * stage_bytes) + TC_TILE_N * 128;
+                tma_load_2d(dst, &maps.xhi, bar, kb * TC_TILE_K, 0, HINT_KEEP);
+                tma_load_2d(dst + b_bytes, &maps.xlo, bar, kb * TC_TILE_K, 0, HINT_KEEP);
+            };
+            // weights do not depend on the previous kernel: start streaming them before waiting for it
+            const int pre = min(p.stages, n_units);
+            for (int i = 0; i < pre; ++i) issue_a(i);
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            for (int i = 0; i < pre; ++i) issue_b(i);
+            bool ok = true;
+            for (int i = pre; i < n_units && ok; ++i) {
+                const int st = i % p.stages;
+                const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+                ok = mbar_wait(smem_u32(&s.empty[st]), ph ^ 1u, abort_flag);
+                if (!ok) break;
+                issue_a(i);
+                issue_b(i);
+            }
+            if (*abort_flag) {
+                // give our own copies in flight a bounded chance to land before the CTA exits
+                const int first = max(0, n_units - p.stages);
+                for (int i = first; i < n_units; ++i) {
+                    const uint32_t bar = smem_u32(&s.full[i % p.stages]);
+                    const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+                    for (uint32_t it = 0; it < (1u << 16) && !mbar_test(bar, ph); ++it) __nanosleep(64);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0 && n_units > 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.rpad >> 3) << 17) |
+                                   ((uint32_t)(TC_TILE_N >> 4) << 24);
+            int i = 0, seg = 0;
+            bool ok = true;
+            while (i < n_units && ok) {
+                const int u = u_begin + i;
+                const int kb0 = u % KB;
+                const int len = min(KB - kb0, n_units - i);
+                const int buf = seg & 1;
+                const uint32_t aph = (uint32_t)(seg >> 1) & 1u;
+                ok = mbar_wait(smem_u32(&s.tempty[buf]), aph ^ 1u, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.rpad);
+                for (int k = 0; k < len && ok; ++k, ++i) {
+                    const int st = i % p.stages;
+                    const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+                    ok = mbar_wait(smem_u32(&s.full[st]), ph, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(s.ring + (size_t)st * stage_bytes);
+                    const uint32_t bh_addr = a_addr + TC_TILE_N * 128;
+                    const uint32_t bl_addr = bh_addr + b_bytes;
+#pragma unroll
+                    for (int k4 = 0; k4 < TC_TILE_K / 16; ++k4) {
+                        const uint64_t ad = smem_desc(a_addr + k4 * 32);
+                        tc_mma(d_tmem, ad, smem_desc(bh_addr + k4 * 32), idesc, (k > 0 || k4 > 0) ? 1u : 0u);
+                        tc_mma(d_tmem, ad, smem_desc(bl_addr + k4 * 32), idesc, 1u);
+                    }
+                    tc_commit(smem_u32(&s.empty[st]));      // frees the smem stage once these MMAs have read it
+                }
+                if (ok) tc_commit(smem_u32(&s.tfull[buf]));  // accumulator of this segment complete
+                ++seg;
+            }
+        }
+    } else {
+        // ---------------- epilogue ----------------
+        const int e = threadIdx.x - 64;                 // 0..127
+        const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
+        const int feat = quad * 32 + lane;              // feature (TMEM lane) within the tile
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        // deferred RMSNorm scale of every row
+        for (int r = e; r < TC_MAX_ROWS; r += EPI_THREADS) {
+            float v = 1.f;
+            if (r < p.T && p.sumsq_in_parts > 0) {
+                float acc = 0.f;
+                for (int q = 0; q < p.sumsq_in_parts; ++q) acc += p.sumsq_in[(size_t)q * TC_X_ROWS + r];
+                v = rsqrtf(acc * p.inv_dim + p.eps);
+            }
+            s.rstd[r] = v;
+        }
+        epi_bar();
+        int i = 0, seg = 0;
+        while (i < n_units) {
+            const int u = u_begin + i;
+            const int tile = u / KB, kb0 = u % KB;
+            const int len = min(KB - kb0, n_units - i);
+            const int buf = seg & 1;
+            const uint32_t aph = (uint32_t)(seg >> 1) & 1u;
+            bool ok = true;
+            if (lane == 0) ok = mbar_wait(smem_u32(&s.tfull[buf]), aph, abort_flag);
+            if (lane == 0) s.flags[1 + (warp - 2)] = ok ? 1 : 0;
+            epi_bar();
+            if (!(s.flags[1] && s.flags[2] && s.flags[3] && s.flags[4])) break;   // uniform over the 128 threads
+            tc_fence_after();
+            // contributors of this tile, in CTA order
+            const int c_first = (tile * KB) / p.units_per_cta;
+            const int c_last = ((tile + 1) * KB - 1) / p.units_per_cta;
+            const int n_contrib = c_last - c_first + 1;
+            const int slot_idx = (int)blockIdx.x - c_first;
+            float* part = p.ws + ((size_t)tile * p.max_contrib + slot_idx) * ((size_t)p.rpad * TC_TILE_N);
+            for (int c0 = 0; c0 < p.T; c0 += 16) {
+                float v[16];
+                tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * p.rpad + c0), v);
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (c0 + j < p.T) part[(size_t)(c0 + j) * TC_TILE_N + feat] = v[j];
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s.tempty[buf]));   // MMA may reuse this accumulator
+            __threadfence();
+            epi_bar();
+            if (e == 0) {
+                const int old = atomicAdd(&p.counters[tile], 1);
+                s.flags[0] = (old + 1 == n_contrib);
+            }
+            epi_bar();
+            if (s.flags[0]) {
+                __threadfence();
+                const float* tile_ws = p.ws + (size_t)tile * p.max_contrib * ((size_t)p.rpad * TC_TILE_N);
+                for (int r0 = 0; r0 < p.T; r0 += EPI_ROWS) {
+                    for (int j = 0; j < EPI_ROWS; ++j) {
+                        const int r = r0 + j;
+                        float acc = 0.f;
+                        if (r < p.T) {
+                            for (int c = 0; c < n_contrib; ++c)
+                                acc += __ldcg(tile_ws + (size_t)c * p.rpad * TC_TILE_N + (size_t)r * TC_TILE_N + e);
+                            acc *= s.rstd[r];
+                        }
+                        s.epi[j][e] = acc;
+                    }
+                    epi_bar();
+                    switch (p.mode) {
+                        case TC_PLAIN: epi_plain(p, s, tile, r0, e); break;
+                        case TC_QKV: epi_qkv(p, s, tile, r0, e); break;
+                        case TC_RESID: epi_resid(p, s, tile, r0, e); break;
+                        case TC_SWIGLU: epi_swiglu(p, s, tile, r0, e); break;
+                        default: epi_lmhead(p, s, tile, r0, e); break;
+                    }
+                    epi_bar();
+                }
+                if (e == 0) p.counters[tile] = 0;          // ready for the next launch
+            }
+            i += len;
+            ++seg;
+        }
+    }
+    // ---------------- teardown ----------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+    if (threadIdx.x == 0 && *abort_flag && p.status) atomicOr(p.status, MTAD_ST_TIMEOUT);
+}
+
+__global__ void split_rows_kernel(const float* __restrict__ x, int ldx_in, __nv_bfloat16* __restrict__ hi,
+                                  __nv_bfloat16* __restrict__ lo, int ld, int K) {
+    const int t = blockIdx.x;
+    for (int k = threadIdx.x; k < K; k += blockDim.x)
+        split_store(x[(size_t)t * ldx_in + k], hi + (size_t)t * ld + k, lo + (size_t)t * ld + k);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(f);
+    }
+    return fn;
+}
+
+}  // namespace
+
+int tc_make_map(CUtensorMap* out, const void* base, long long rows, long long cols, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return -1;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)TC_TILE_K, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : -1;
+}
+
+void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int ctas) {
+    p.n_tiles = n_tiles;
+    p.k_blocks = (K + TC_TILE_K - 1) / TC_TILE_K;
+    p.total_units = n_tiles * p.k_blocks;
+    p.units_per_cta = (p.total_units + ctas - 1) / ctas;
+    p.max_contrib = (p.k_blocks + p.units_per_cta - 1) / p.units_per_cta + 1;
+    p.T = T;
+    p.rpad = (T + 15) / 16 * 16;
+}
+
+size_t tc_workspace_floats(int n_tiles_max, int max_contrib_max, int rpad_max) {
+    return (size_t)n_tiles_max * max_contrib_max * rpad_max * TC_TILE_N;
+}
+
+cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p_in, int ctas, bool pdl, cudaStream_t st) {
+    TcGemmParams p = p_in;
+    const int stage_bytes = TC_TILE_N * 128 + 2 * p.rpad * 128;
+    // two CTAs of consecutive kernels share an SM while one drains and the next prefetches: stay under half of it
+    const size_t budget = (p.rpad <= 32 ? 100 : 200) * 1024;
+    int stages = (int)((budget - SMEM_TAIL - 1024) / stage_bytes);
+    stages = stages > MAX_STAGES ? MAX_STAGES : stages;
+    if (stages < 2) return cudaErrorInvalidValue;
+    p.stages = stages;
+    const size_t smem = (size_t)stages * stage_bytes + SMEM_TAIL + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int grid = (p.total_units + p.units_per_cta - 1) / p.units_per_cta;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    (void)ctas;
+    return cudaLaunchKernelEx(&cfg, tc_gemm_kernel, maps, p);
+}
+
+cudaError_t launch_split_rows(const float* x, int ldx_in, __nv_bfloat16* hi, __nv_bfloat16* lo, int ld, int T, int K,
+                              cudaStream_t st) {
+    split_rows_kernel<<<T, 256, 0, st>>>(x, ldx_in, hi, lo, ld, K);
+    return cudaGetLastError();
+}
+
+}  // namespace mtad

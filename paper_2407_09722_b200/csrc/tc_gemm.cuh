@@ -1,0 +1,86 @@
+// Interface of the tensor-core weight-streaming GEMM (tcgen05 + TMEM + TMA) and its fused epilogues.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace mtad {
+
+constexpr int TC_TILE_N = 128;      // output features per tile (the MMA M dimension: weights are operand A)
+constexpr int TC_TILE_K = 64;       // bf16 elements per k-block: one 128-byte swizzle row
+constexpr int TC_MAX_ROWS = 256;    // activation rows per launch (the MMA N dimension)
+constexpr int TC_X_ROWS = 256;      // rows allocated in every activation operand buffer
+
+enum TcMode {
+    TC_PLAIN = 0,     // out[r, n] = acc
+    TC_QKV = 1,       // rotary embedding; q -> fp32 (scaled), k, v -> bf16 KV cache
+    TC_RESID = 2,     // hidden[r, n] += acc; emits hidden * gain as bf16 hi/lo and per-tile sums of squares
+    TC_SWIGLU = 3,    // rows 0..63 of a tile are gate, 64..127 up: silu(gate) * up as bf16 hi/lo
+    TC_LMHEAD = 4     // per (row, tile): max, sum-exp, best perturbed logit; gathers the drafted tokens' logits
+};
+
+struct TcGemmParams {
+    // decomposition
+    int n_tiles, k_blocks, total_units, units_per_cta, max_contrib;
+    int T;                 // valid activation rows
+    int rpad;              // MMA N: T rounded up to 16
+    int stages;            // smem ring depth
+    int mode;
+    int N;                 // output features (bound for stores)
+    // split-K fix-up
+    float* ws;             // [n_tiles][max_contrib][rpad][128] partial tiles
+    int* counters;         // [n_tiles], zero between launches
+    uint32_t* status;      // device status word for time-outs (may be null)
+    // deferred RMSNorm of the input: rstd[r] = rsqrt(sum_parts / dim + eps); parts == 0 -> 1
+    const float* sumsq_in;
+    int sumsq_in_parts;
+    float inv_dim, eps;
+    // TC_PLAIN
+    float* out;
+    int ldo;
+    // TC_QKV
+    int seg_k_tile, seg_v_tile;     // first tile of the K rows and of the V rows
+    int Hq, Hkv, hd;
+    float* q_out;                   // [T, (Hq + 2 Hkv) hd], q part written
+    const float* rope;              // [T, hd/2, 2]
+    __nv_bfloat16* cache;
+    const int32_t* slot;
+    const int32_t* seq;
+    int layer, max_batch;
+    long long cap;
+    // TC_RESID / TC_SWIGLU outputs
+    float* hidden;                  // [T, N]
+    const __nv_bfloat16* gain;      // [N] gains of the norm that follows (TC_RESID)
+    __nv_bfloat16* x_hi;            // [TC_X_ROWS, ldx] operand buffers for the next GEMM
+    __nv_bfloat16* x_lo;
+    int ldx;
+    float* sumsq_out;               // [n_tiles][TC_X_ROWS]
+    // TC_LMHEAD
+    float4* lm_part;                // [T][n_tiles] (max, sumexp, best value, best index bits)
+    const float* uniforms;          // [B, V]
+    int R;                          // rows per sequence
+    const int32_t* prow;            // [T] parent row of a node row, -1 otherwise
+    const int32_t* tok;             // [T]
+    float* node_z;                  // [T] logit of the row's token under its parent row
+};
+
+struct TcMaps {
+    CUtensorMap a0, a1, a2;         // weight maps (QKV: wq, wk, wv; SwiGLU: gate, up; else a0)
+    CUtensorMap xhi, xlo;           // activation operand maps
+};
+
+// Encodes a 2-D bf16 tensor map (row-major [rows, cols], 128-byte swizzle, box [box_rows, 64]).
+int tc_make_map(CUtensorMap* out, const void* base, long long rows, long long cols, int box_rows);
+
+// Fills the decomposition fields of p for a problem of n_tiles x k_blocks on `ctas` CTAs.
+void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int ctas);
+size_t tc_workspace_floats(int n_tiles_max, int max_contrib_max, int rpad_max);
+
+cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p, int ctas, bool pdl, cudaStream_t st);
+
+// Splits fp32 rows into bf16 hi + lo operand rows (hi = bf16(x), lo = bf16(x - hi)).
+cudaError_t launch_split_rows(const float* x, int ldx_in, __nv_bfloat16* hi, __nv_bfloat16* lo, int ld, int T, int K,
+                              cudaStream_t st);
+
+}  // namespace mtad

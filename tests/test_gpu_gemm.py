@@ -1,0 +1,50 @@
+"""The tensor-core weight-streaming GEMM alone (mtad_debug_gemm) against an fp64 matmul of the same bf16 weights."""
+import pytest
+import torch
+
+import mtad_synth as S
+from paper_2407_09722_b200.runtime import DeviceModel
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def small_ctx():
+    # F = 1408 bounds K, vocab 4096 bounds the tile count of the workspace
+    return DeviceModel(S.ModelShape(1, 256, 4, 4, 64, 1408, 4096), max_batch=1, max_nodes=255, capacity=320)
+
+
+def _check(dm, N, K, T, seed):
+    W = S.normal_bf16(seed, 1000 + N + K, N * K, 0.02, "cuda").view(N, K)
+    x = S.normal_bf16(seed, 2000 + T + K, T * K, 1.0, "cuda").float().view(T, K)
+    x = x * (1.0 + 1e-3 * torch.arange(T * K, device="cuda").view(T, K).remainder(7))     # not bf16-representable
+    y = torch.full((T, N), float("nan"), device="cuda")
+    dm.ctx.mtad_debug_gemm(W, x, y)
+    torch.cuda.synchronize()
+    ref = x.double() @ W.double().t()
+    err = (y.double() - ref).abs().max().item()
+    scale = ref.abs().max().item()
+    assert err <= 2e-5 * max(scale, 1.0), (N, K, T, err, scale)
+
+
+@pytest.mark.parametrize("N,K,T", [(128, 64, 1), (128, 256, 5), (256, 256, 16), (384, 688, 17), (200, 136, 3),
+                                   (1024, 1408, 65), (4096, 256, 129), (640, 1024, 256), (4096, 1408, 5)])
+def test_debug_gemm_shapes(small_ctx, N, K, T):
+    _check(small_ctx, N, K, T, 0)
+
+
+def test_debug_gemm_twice_is_bit_identical(small_ctx):
+    N, K, T = 1024, 1408, 33
+    W = S.normal_bf16(1, 7, N * K, 0.02, "cuda").view(N, K)
+    x = torch.randn(T, K, device="cuda")
+    a = torch.empty(T, N, device="cuda"); b = torch.empty(T, N, device="cuda")
+    small_ctx.ctx.mtad_debug_gemm(W, x, a)
+    small_ctx.ctx.mtad_debug_gemm(W, x, b)
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+
+
+def test_debug_gemm_7b_shapes():
+    dm = DeviceModel(S.ModelShape(1, 4096, 32, 32, 128, 11008, 32000), max_batch=1, max_nodes=8, capacity=64)
+    for (N, K, T) in [(4096, 4096, 5), (4096, 11008, 5), (32000, 4096, 9)]:
+        _check(dm, N, K, T, 2)
