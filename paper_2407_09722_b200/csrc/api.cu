@@ -12,7 +12,7 @@
 
 using namespace mtad;
 
-constexpr int kCtas = 148;     // one persistent CTA per SM in the tensor-core GEMM
+static const int kCtas = getenv("MTAD_TC_CTAS") ? atoi(getenv("MTAD_TC_CTAS")) : 148;   // CTAs of the tensor-core GEMM (one per SM)
 
 // Host-side tensor maps of one model's weight matrices.
 struct WeightMaps {

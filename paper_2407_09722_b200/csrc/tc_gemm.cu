@@ -13,6 +13,7 @@
 // Every wait on an mbarrier is bounded; on a time-out the kernel raises MTAD_ST_TIMEOUT, waits (bounded) for its
 // own copies in flight, frees its tensor memory and returns.
 #include <math_constants.h>
+#include <stdlib.h>
 
 #include "tc_gemm.cuh"
 
@@ -308,8 +309,13 @@ __global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__
     const int u_end = min(u_begin + p.units_per_cta, p.total_units);
     const int n_units = max(u_end - u_begin, 0);
     const int KB = p.k_blocks;
+    // hi and lo operand rows sit back to back in a stage, so one MMA of N = 2 * rpad multiplies both (their products
+    // land in neighbouring column blocks and are added when the accumulator is drained); beyond N = 256 two MMAs
+    // accumulate into the same columns instead
+    const bool stacked = 2 * p.rpad <= 256;
+    const int acc_cols = stacked ? 2 * p.rpad : p.rpad;
     uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < 2 * p.rpad) tmem_cols <<= 1;
+    while ((int)tmem_cols < 2 * acc_cols) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.stages; ++i) {
@@ -393,7 +399,8 @@ __global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0 && n_units > 0) {
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.rpad >> 3) << 17) |
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) |
+                                   ((uint32_t)((stacked ? 2 * p.rpad : p.rpad) >> 3) << 17) |
                                    ((uint32_t)(TC_TILE_N >> 4) << 24);
             int i = 0, seg = 0;
             bool ok = true;
@@ -406,7 +413,7 @@ __global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__
                 ok = mbar_wait(smem_u32(&s.tempty[buf]), aph ^ 1u, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.rpad);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * acc_cols);
                 for (int k = 0; k < len && ok; ++k, ++i) {
                     const int st = i % p.stages;
                     const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
@@ -420,7 +427,7 @@ __global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__
                     for (int k4 = 0; k4 < TC_TILE_K / 16; ++k4) {
                         const uint64_t ad = smem_desc(a_addr + k4 * 32);
                         tc_mma(d_tmem, ad, smem_desc(bh_addr + k4 * 32), idesc, (k > 0 || k4 > 0) ? 1u : 0u);
-                        tc_mma(d_tmem, ad, smem_desc(bl_addr + k4 * 32), idesc, 1u);
+                        if (!stacked) tc_mma(d_tmem, ad, smem_desc(bl_addr + k4 * 32), idesc, 1u);
                     }
                     tc_commit(smem_u32(&s.empty[st]));      // frees the smem stage once these MMAs have read it
                 }
@@ -466,7 +473,14 @@ __global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__
             float* part = p.ws + ((size_t)tile * p.max_contrib + slot_idx) * ((size_t)p.rpad * TC_TILE_N);
             for (int c0 = 0; c0 < p.T; c0 += 16) {
                 float v[16];
-                tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * p.rpad + c0), v);
+                const uint32_t col = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * acc_cols + c0);
+                tc_ld16(col, v);
+                if (stacked) {
+                    float w[16];
+                    tc_ld16(col + (uint32_t)p.rpad, w);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] += w[j];
+                }
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
                     if (c0 + j < p.T) part[(size_t)(c0 + j) * TC_TILE_N + feat] = v[j];
@@ -554,7 +568,9 @@ int tc_make_map(CUtensorMap* out, const void* base, long long rows, long long co
     const cuuint32_t box[2] = {(cuuint32_t)TC_TILE_K, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          getenv("MTAD_TC_L2P") ? (CUtensorMapL2promotion)atoi(getenv("MTAD_TC_L2P"))
+                                                : CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? 0 : -1;
 }
@@ -577,7 +593,8 @@ cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p_in, int cta
     TcGemmParams p = p_in;
     const int stage_bytes = TC_TILE_N * 128 + 2 * p.rpad * 128;
     // two CTAs of consecutive kernels share an SM while one drains and the next prefetches: stay under half of it
-    const size_t budget = (p.rpad <= 32 ? 100 : 200) * 1024;
+    static const int budget_kb_env = getenv("MTAD_TC_SMEM_KB") ? atoi(getenv("MTAD_TC_SMEM_KB")) : 0;
+    const size_t budget = budget_kb_env > 0 ? (size_t)budget_kb_env * 1024 : (p.rpad <= 32 ? 113 : 200) * 1024;
     int stages = (int)((budget - SMEM_TAIL - 1024) / stage_bytes);
     stages = stages > MAX_STAGES ? MAX_STAGES : stages;
     if (stages < 2) return cudaErrorInvalidValue;
