@@ -32,7 +32,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", LIB] + sources()
+           "-o", LIB] + os.environ.get("MTAD_NVCC_FLAGS", "").split() + sources()
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
         print(" ".join(cmd))

@@ -15,9 +15,9 @@ using namespace mtad;
 static const int kCtas = getenv("MTAD_TC_CTAS") ? atoi(getenv("MTAD_TC_CTAS")) : 148;   // CTAs of the tensor-core GEMM (one per SM)
 
 // Host-side tensor maps of one model's weight matrices.
-struct WeightMaps {
-    std::vector<CUtensorMap> wq, wk, wv, wo, gate, up, down;
-    CUtensorMap lm_head;
+struct WeightMaps {                      // index 0, 1, 2: tiles of 128, 256, 512 rows (1, 2, 4 halves)
+    std::vector<CUtensorMap> wq[3], wk[3], wv[3], wo[3], gate[3], up[3], down[3];
+    CUtensorMap lm_head[3];
     bool ok = false;
 };
 
@@ -127,12 +127,11 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     // tensor-core path buffers (operand rows are always TC_X_ROWS high so that the TMA box never leaves them)
     const size_t Tc = std::min<size_t>(T, TC_MAX_ROWS);
     const size_t rpad = (Tc + 15) / 16 * 16;
-    sc.xd_hi = k.take<__nv_bfloat16>((size_t)TC_X_ROWS * d);
-    sc.xd_lo = k.take<__nv_bfloat16>((size_t)TC_X_ROWS * d);
-    sc.xa_hi = k.take<__nv_bfloat16>((size_t)TC_X_ROWS * qd);
-    sc.xa_lo = k.take<__nv_bfloat16>((size_t)TC_X_ROWS * qd);
-    sc.xf_hi = k.take<__nv_bfloat16>((size_t)TC_X_ROWS * F);
-    sc.xf_lo = k.take<__nv_bfloat16>((size_t)TC_X_ROWS * F);
+    // operand rows, hi and lo interleaved: row 2t = hi(t), row 2t + 1 = lo(t)
+    sc.xd_hi = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * d);
+    sc.xa_hi = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * qd);
+    sc.xf_hi = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * F);
+    sc.xd_lo = sc.xa_lo = sc.xf_lo = nullptr;
     const size_t dt = (d + TC_TILE_N - 1) / TC_TILE_N;
     sc.sumsq_a = k.take<float>(dt * TC_X_ROWS);
     sc.sumsq_b = k.take<float>(dt * TC_X_ROWS);
@@ -145,10 +144,13 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
                                   {(m->d_model + 127) / 128, m->d_ffn},
                                   {(m->vocab + 127) / 128, m->d_model}};
         for (auto& sh : shapes) {
-            TcGemmParams tp{};
-            tc_decompose(tp, sh[0], sh[1], 1, kCtas);
-            ws_tiles = std::max(ws_tiles, (size_t)sh[0] * tp.max_contrib);
-            max_tiles = std::max(max_tiles, (size_t)sh[0]);
+            for (int mh = 1; mh <= 4; mh *= 2) {
+                TcGemmParams tp{};
+                const int tiles = (sh[0] + mh - 1) / mh;
+                tc_decompose(tp, tiles, sh[1], 1, kCtas);
+                ws_tiles = std::max(ws_tiles, (size_t)tiles * tp.max_contrib * mh);
+                max_tiles = std::max(max_tiles, (size_t)tiles);
+            }
         }
         lm_tiles = std::max(lm_tiles, (size_t)(m->vocab + 127) / 128);
     };
@@ -162,7 +164,7 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
         c->st = st; c->rm = rm; c->sc = sc;
         c->tc_ws_floats = ws_tiles * rpad * TC_TILE_N;
         c->tc_counter_n = max_tiles;
-        c->xf_elems = (size_t)TC_X_ROWS * F;
+        c->xf_elems = (size_t)2 * TC_X_ROWS * F;
     }
     return (k.off + 255) & ~size_t(255);
 }
@@ -216,7 +218,7 @@ int forward_rows(mtad_ctx* ctx, const ModelView& m, int B, int R, long long len_
         RUN(MTAD_K_GEMM, wb * kvd * d.d_model, 1,
             launch_gemm_rows(sc.xn, d.d_model, m.w(l, 3), nullptr, sc.qkv, ldq, qd + kvd, T, kvd, d.d_model, 0, s));
         RUN(MTAD_K_ROPE, 0, 1, launch_rope_append(m, l, ctx->rm, sc, T, s));
-        RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, false, s));
+        RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, false, false, s));
         RUN(MTAD_K_GEMM, wb * d.d_model * qd, 1,
             launch_gemm_rows(sc.attn, qd, m.w(l, 4), nullptr, sc.hidden, d.d_model, 0, T, d.d_model, qd, 1, s));
         RUN(MTAD_K_NORM, 0, 1, launch_rmsnorm(sc.hidden, m.w(l, 5), sc.xn, T, d.d_model, d.rms_eps, s));
@@ -240,19 +242,24 @@ bool build_weight_maps(const ModelView& m, WeightMaps& w) {
     auto mk = [&](CUtensorMap* o, const void* base, long long rows, long long cols, int box) {
         return aligned(base) && tc_make_map(o, base, rows, cols, box) == 0;
     };
-    w.wq.resize(d.layers); w.wk.resize(d.layers); w.wv.resize(d.layers); w.wo.resize(d.layers);
-    w.gate.resize(d.layers); w.up.resize(d.layers); w.down.resize(d.layers);
     bool ok = true;
-    for (int l = 0; l < d.layers && ok; ++l) {
-        ok = ok && mk(&w.wq[l], m.w(l, 1), qd, d.d_model, 128);
-        ok = ok && mk(&w.wk[l], m.w(l, 2), kvd, d.d_model, 128);
-        ok = ok && mk(&w.wv[l], m.w(l, 3), kvd, d.d_model, 128);
-        ok = ok && mk(&w.wo[l], m.w(l, 4), d.d_model, qd, 128);
-        ok = ok && mk(&w.gate[l], m.w(l, 6), d.d_ffn, d.d_model, 64);
-        ok = ok && mk(&w.up[l], m.w(l, 7), d.d_ffn, d.d_model, 64);
-        ok = ok && mk(&w.down[l], m.w(l, 8), d.d_model, d.d_ffn, 128);
+    for (int i = 0; i < 3 && ok; ++i) {
+        const int halves = 1 << i;
+        const int box = halves == 1 ? 128 : 256;          // a 512-row tile is fetched as two 256-row boxes
+        w.wq[i].resize(d.layers); w.wk[i].resize(d.layers); w.wv[i].resize(d.layers); w.wo[i].resize(d.layers);
+        w.gate[i].resize(d.layers); w.up[i].resize(d.layers); w.down[i].resize(d.layers);
+        for (int l = 0; l < d.layers && ok; ++l) {
+            ok = ok && mk(&w.wq[i][l], m.w(l, 1), qd, d.d_model, box);
+            ok = ok && mk(&w.wk[i][l], m.w(l, 2), kvd, d.d_model, box);
+            ok = ok && mk(&w.wv[i][l], m.w(l, 3), kvd, d.d_model, box);
+            ok = ok && mk(&w.wo[i][l], m.w(l, 4), d.d_model, qd, box);
+            // gate and up share a tile: its first half are gate rows, its second half the matching up rows
+            ok = ok && mk(&w.gate[i][l], m.w(l, 6), d.d_ffn, d.d_model, 64 * halves);
+            ok = ok && mk(&w.up[i][l], m.w(l, 7), d.d_ffn, d.d_model, 64 * halves);
+            ok = ok && mk(&w.down[i][l], m.w(l, 8), d.d_model, d.d_ffn, box);
+        }
+        ok = ok && mk(&w.lm_head[i], d.lm_head, d.vocab, d.d_model, box);
     }
-    ok = ok && mk(&w.lm_head, d.lm_head, d.vocab, d.d_model, 128);
     w.ok = ok;
     return ok;
 }
@@ -274,11 +281,16 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
     const int rpad = (T + 15) / 16 * 16;
     const int dt = (d.d_model + TC_TILE_N - 1) / TC_TILE_N;
     const bool pdl = ctx->use_pdl;
-    // activation operand maps for this call's row count
-    CUtensorMap xd_hi, xd_lo, xa_hi, xa_lo, xf_hi, xf_lo;
-    if (tc_make_map(&xd_hi, sc.xd_hi, TC_X_ROWS, d.d_model, rpad) || tc_make_map(&xd_lo, sc.xd_lo, TC_X_ROWS, d.d_model, rpad) ||
-        tc_make_map(&xa_hi, sc.xa_hi, TC_X_ROWS, qd, rpad) || tc_make_map(&xa_lo, sc.xa_lo, TC_X_ROWS, qd, rpad) ||
-        tc_make_map(&xf_hi, sc.xf_hi, TC_X_ROWS, d.d_ffn, rpad) || tc_make_map(&xf_lo, sc.xf_lo, TC_X_ROWS, d.d_ffn, rpad))
+    const int mh = tc_halves(T);                          // weight halves per tile, as many as tensor memory allows
+    int mq = mh;                                          // QKV tiles must not straddle q | k | v
+    while (mq > 1 && (qd % (128 * mq) || kvd % (128 * mq))) mq /= 2;
+    auto ix = [](int halves) { return halves == 1 ? 0 : (halves == 2 ? 1 : 2); };
+    auto up = [](int a, int b) { return (a + b - 1) / b; };
+    // operand-row maps for this call's row count: box = all 2 * rpad interleaved rows (two boxes beyond 256)
+    const int xbox = 2 * rpad > 256 ? rpad : 2 * rpad;
+    CUtensorMap xd, xa, xf;
+    if (tc_make_map(&xd, sc.xd_hi, 2 * TC_X_ROWS, d.d_model, xbox) || tc_make_map(&xa, sc.xa_hi, 2 * TC_X_ROWS, qd, xbox) ||
+        tc_make_map(&xf, sc.xf_hi, 2 * TC_X_ROWS, d.d_ffn, xbox))
         return MTAD_E_CUDA;
     TcGemmParams base{};
     base.ws = sc.tc_ws; base.counters = sc.tc_counters; base.status = status;
@@ -292,47 +304,53 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
     for (int l = 0; l < d.layers; ++l) {
         {   // QKV + rotary + append
             TcGemmParams p = base; TcMaps mp{};
-            const int qt = (qd + 127) / 128, kt = (kvd + 127) / 128;
-            tc_decompose(p, qt + 2 * kt, d.d_model, T, kCtas);
+            const int qt = up(qd, 128), kt = up(kvd, 128);
+            tc_decompose(p, (qt + 2 * kt) / mq, d.d_model, T, kCtas);
+            p.mh = mq; p.n_rows_total = (qt + 2 * kt) * 128;
             p.mode = TC_QKV; p.N = qd; p.seg_k_tile = qt; p.seg_v_tile = qt + kt; p.layer = l;
             p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = (l == 0) ? 1 : dt;
-            mp.a0 = wm.wq[l]; mp.a1 = wm.wk[l]; mp.a2 = wm.wv[l]; mp.xhi = xd_hi; mp.xlo = xd_lo;
+            mp.a0 = wm.wq[ix(mq)][l]; mp.a1 = wm.wk[ix(mq)][l]; mp.a2 = wm.wv[ix(mq)][l]; mp.x = xd;
             RUN(MTAD_K_GEMM, wb * (qd + 2.0 * kvd) * d.d_model, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
         }
-        RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, true, s));
+        RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, true, pdl, s));
         {   // O projection + residual, emits the FFN norm's operand rows
             TcGemmParams p = base; TcMaps mp{};
-            tc_decompose(p, dt, qd, T, kCtas);
+            tc_decompose(p, up(d.d_model, 128 * mh), qd, T, kCtas);
+            p.mh = mh; p.n_rows_total = d.d_model;
             p.mode = TC_RESID; p.N = d.d_model; p.sumsq_in_parts = 0;
-            p.gain = m.w(l, 5); p.x_hi = sc.xd_hi; p.x_lo = sc.xd_lo; p.ldx = d.d_model; p.sumsq_out = sc.sumsq_b;
-            mp.a0 = wm.wo[l]; mp.xhi = xa_hi; mp.xlo = xa_lo;
+            p.gain = m.w(l, 5); p.x_hi = sc.xd_hi; p.x_lo = sc.xd_hi + d.d_model; p.ldx = 2 * d.d_model;
+            p.sumsq_out = sc.sumsq_b;
+            mp.a0 = wm.wo[ix(mh)][l]; mp.x = xa;
             RUN(MTAD_K_GEMM, wb * d.d_model * qd, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
         }
         {   // gate / up + SwiGLU
             TcGemmParams p = base; TcMaps mp{};
-            tc_decompose(p, (d.d_ffn + 63) / 64, d.d_model, T, kCtas);
+            tc_decompose(p, up(d.d_ffn, 64 * mh), d.d_model, T, kCtas);
+            p.mh = mh; p.n_rows_total = d.d_ffn;
             p.mode = TC_SWIGLU; p.N = d.d_ffn; p.sumsq_in = sc.sumsq_b; p.sumsq_in_parts = dt;
-            p.x_hi = sc.xf_hi; p.x_lo = sc.xf_lo; p.ldx = d.d_ffn;
-            mp.a0 = wm.gate[l]; mp.a1 = wm.up[l]; mp.xhi = xd_hi; mp.xlo = xd_lo;
+            p.x_hi = sc.xf_hi; p.x_lo = sc.xf_hi + d.d_ffn; p.ldx = 2 * d.d_ffn;
+            mp.a0 = wm.gate[ix(mh)][l]; mp.a1 = wm.up[ix(mh)][l]; mp.x = xd;
             RUN(MTAD_K_GEMM, wb * 2.0 * d.d_ffn * d.d_model, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
         }
         {   // down projection + residual, emits the next norm's operand rows
             TcGemmParams p = base; TcMaps mp{};
-            tc_decompose(p, dt, d.d_ffn, T, kCtas);
+            tc_decompose(p, up(d.d_model, 128 * mh), d.d_ffn, T, kCtas);
+            p.mh = mh; p.n_rows_total = d.d_model;
             p.mode = TC_RESID; p.N = d.d_model; p.sumsq_in_parts = 0;
             p.gain = (l + 1 < d.layers) ? m.w(l + 1, 0) : static_cast<const __nv_bfloat16*>(d.final_norm);
-            p.x_hi = sc.xd_hi; p.x_lo = sc.xd_lo; p.ldx = d.d_model; p.sumsq_out = sc.sumsq_a;
-            mp.a0 = wm.down[l]; mp.xhi = xf_hi; mp.xlo = xf_lo;
+            p.x_hi = sc.xd_hi; p.x_lo = sc.xd_hi + d.d_model; p.ldx = 2 * d.d_model; p.sumsq_out = sc.sumsq_a;
+            mp.a0 = wm.down[ix(mh)][l]; mp.x = xf;
             RUN(MTAD_K_GEMM, wb * d.d_model * d.d_ffn, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
         }
     }
     {   // LM head + per-tile log-softmax / Gumbel-argmax partials + gather of the drafted tokens' logits
         TcGemmParams p = base; TcMaps mp{};
-        tc_decompose(p, (d.vocab + 127) / 128, d.d_model, T, kCtas);
+        tc_decompose(p, up(d.vocab, 128 * mh), d.d_model, T, kCtas);
+        p.mh = mh; p.n_rows_total = d.vocab; p.n_tiles128 = up(d.vocab, 128);
         p.mode = TC_LMHEAD; p.N = d.vocab; p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = dt;
-        mp.a0 = wm.lm_head; mp.xhi = xd_hi; mp.xlo = xd_lo;
+        mp.a0 = wm.lm_head[ix(mh)]; mp.x = xd;
         RUN(MTAD_K_GEMM, wb * d.vocab * d.d_model, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
-        RUN(MTAD_K_LMRED, 0, 2, launch_lm_merge(m, ctx->rm, sc, B, R, p.n_tiles, uniforms, s));
+        RUN(MTAD_K_LMRED, 0, 2, launch_lm_merge(m, ctx->rm, sc, B, R, p.n_tiles128, uniforms, s));
     }
     return MTAD_OK;
 }
@@ -372,7 +390,7 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
     pa.B = B; pa.R = R; pa.max_depth = D; pa.n_nodes = n_nodes; pa.tok = tok; pa.parent = parent;
     const bool tc = ctx->use_tc && ctx->tmaps.ok && B * R <= TC_MAX_ROWS;
     if (tc) {
-        pa.gain0 = ctx->target.w(0, 0); pa.x_hi = ctx->sc.xd_hi; pa.x_lo = ctx->sc.xd_lo;
+        pa.gain0 = ctx->target.w(0, 0); pa.x_hi = ctx->sc.xd_hi; pa.x_lo = ctx->sc.xd_hi + ctx->target.d.d_model;
         pa.sumsq_out = ctx->sc.sumsq_a;
     }
     RUN(MTAD_K_PREPARE, 0, 1, launch_prepare(ctx->target, ctx->st, ctx->rm, ctx->sc, pa, out->status, s));
@@ -435,7 +453,7 @@ int mtad_create(const mtad_model_desc* target, const mtad_model_desc* aux, int m
     ctx->use_tc = !(path && strcmp(path, "simt") == 0) && build_weight_maps(ctx->target, ctx->tmaps);
     if (ctx->use_tc && aux) build_weight_maps(ctx->aux, ctx->amaps);
     const char* pdl = getenv("MTAD_PDL");
-    ctx->use_pdl = pdl && strcmp(pdl, "1") == 0;
+    ctx->use_pdl = !(pdl && strcmp(pdl, "0") == 0);        // programmatic dependent launch unless MTAD_PDL=0
     cudaError_t e = cudaMemset(workspace, 0, need);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete ctx; return MTAD_E_CUDA; }
@@ -485,20 +503,22 @@ uint64_t mtad_kernel_launches(void) { return g_kernel_launches; }
 
 int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, int T, float* y, void* stream) {
     if (!ctx || !W || !x || !y || N < 1 || K < 8 || (K % 8) || T < 1) return MTAD_E_INVALID;
-    if (T > TC_MAX_ROWS || (size_t)TC_X_ROWS * K > ctx->xf_elems) return MTAD_E_CAPACITY;
+    if (T > TC_MAX_ROWS || (size_t)2 * TC_X_ROWS * K > ctx->xf_elems) return MTAD_E_CAPACITY;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     TcGemmParams p{};
-    tc_decompose(p, (N + TC_TILE_N - 1) / TC_TILE_N, K, T, kCtas);
-    if ((size_t)p.n_tiles * p.max_contrib * p.rpad * TC_TILE_N > ctx->tc_ws_floats ||
+    const int mh = tc_halves(T);
+    tc_decompose(p, (N + TC_TILE_N * mh - 1) / (TC_TILE_N * mh), K, T, kCtas);
+    p.mh = mh; p.n_rows_total = N;
+    if ((size_t)p.n_tiles * p.max_contrib * mh * p.rpad * TC_TILE_N > ctx->tc_ws_floats ||
         (size_t)p.n_tiles > ctx->tc_counter_n)
         return MTAD_E_WORKSPACE;
     TcMaps mp{};
-    if (tc_make_map(&mp.a0, W, N, K, 128) || tc_make_map(&mp.xhi, ctx->sc.xf_hi, TC_X_ROWS, K, p.rpad) ||
-        tc_make_map(&mp.xlo, ctx->sc.xf_lo, TC_X_ROWS, K, p.rpad))
+    const int xbox = 2 * p.rpad > 256 ? p.rpad : 2 * p.rpad;
+    if (tc_make_map(&mp.a0, W, N, K, mh == 1 ? 128 : 256) || tc_make_map(&mp.x, ctx->sc.xf_hi, 2 * TC_X_ROWS, K, xbox))
         return MTAD_E_CUDA;
     p.mode = TC_PLAIN; p.N = N; p.out = y; p.ldo = N;
     p.ws = ctx->sc.tc_ws; p.counters = ctx->sc.tc_counters; p.status = nullptr;
-    RUN(MTAD_K_PREPARE, 0, 1, launch_split_rows(x, K, ctx->sc.xf_hi, ctx->sc.xf_lo, K, T, K, s));
+    RUN(MTAD_K_PREPARE, 0, 1, launch_split_rows(x, K, ctx->sc.xf_hi, ctx->sc.xf_hi + K, 2 * K, T, K, s));
     RUN(MTAD_K_GEMM, 2.0 * N * K, 1, launch_tc_gemm(mp, p, kCtas, false, s));
     return MTAD_OK;
 }

@@ -76,6 +76,27 @@ inline int attn_split_cap(int n_q_heads) {
     return s < 1 ? 1 : (s > 32 ? 32 : s);
 }
 
+// Launch with the programmatic-dependent-launch attribute: the kernel may start while its predecessor in the stream
+// is still draining; it must execute griddepcontrol.wait before it touches anything the predecessor writes.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- launchers (each enqueues on `st`, returns the launch error) -------------------------------------------------
 
 struct SeqList {
@@ -104,7 +125,7 @@ cudaError_t launch_gemm_rows(const float* x, int ldx, const __nv_bfloat16* W, co
 cudaError_t launch_rope_append(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int T,
                                cudaStream_t st);
 cudaError_t launch_attention(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int B, int R,
-                             int nsplit, int chunk, bool emit_split, cudaStream_t st);
+                             int nsplit, int chunk, bool emit_split, bool pdl, cudaStream_t st);
 cudaError_t launch_lm_merge(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int n_tiles,
                             const float* bonus_uniform, cudaStream_t st);
 cudaError_t launch_lm_reduce(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R,

@@ -22,6 +22,8 @@ __global__ void __launch_bounds__(128) attn_partial_kernel(const float* __restri
 
     const int h = blockIdx.x, sp = blockIdx.y, bi = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_wait();          // q, the appended K/V rows and the row metadata come from the kernels before
+    pdl_trigger();
     const int nrows = rm.n_rows[bi];
     if (nrows == 0) return;
     const int seq = rm.call_seq[bi];
@@ -139,11 +141,14 @@ __global__ void attn_combine_kernel(const float* __restrict__ part, float* __res
                                     int Hq, int nsplit, __nv_bfloat16* __restrict__ x_hi,
                                     __nv_bfloat16* __restrict__ x_lo) {
     const int t = blockIdx.x, h = blockIdx.y, d = threadIdx.x;
+    pdl_wait();
+    pdl_trigger();
     const size_t idx = ((size_t)t * Hq + h) * HD + d;
+    const size_t xidx = ((size_t)2 * t * Hq + h) * HD + d;     // interleaved operand rows: hi at row 2t, lo at 2t + 1
     float* dst = out + idx;
     if (slot[t] < 0) {
         *dst = 0.f;
-        if (x_hi) { x_hi[idx] = __float2bfloat16_rn(0.f); x_lo[idx] = __float2bfloat16_rn(0.f); }
+        if (x_hi) { x_hi[xidx] = __float2bfloat16_rn(0.f); x_lo[xidx] = __float2bfloat16_rn(0.f); }
         return;
     }
     const float* p = part + (((size_t)t * Hq + h) * nsplit) * (HD + 2);
@@ -161,36 +166,43 @@ __global__ void attn_combine_kernel(const float* __restrict__ part, float* __res
     *dst = y;
     if (x_hi) {      // operand rows of the O projection: bf16 hi + lo
         const __nv_bfloat16 hb = __float2bfloat16_rn(y);
-        x_hi[idx] = hb;
-        x_lo[idx] = __float2bfloat16_rn(y - __bfloat162float(hb));
+        x_hi[xidx] = hb;
+        x_lo[xidx] = __float2bfloat16_rn(y - __bfloat162float(hb));
     }
 }
 
 cudaError_t launch_attention(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int B, int R,
-                             int nsplit, int chunk, bool emit_split, cudaStream_t st) {
+                             int nsplit, int chunk, bool emit_split, bool pdl, cudaStream_t st) {
     const int Hq = m.d.n_q_heads, Hkv = m.d.n_kv_heads, hd = m.d.head_dim;
     const int ldq = (Hq + 2 * Hkv) * hd;
     dim3 grid(Hq, nsplit, B);
     const __nv_bfloat16* cache = static_cast<const __nv_bfloat16*>(m.d.kv_cache);
     dim3 cgrid(B * R, Hq);
+    cudaError_t e = cudaSuccess;
     __nv_bfloat16* xh = emit_split ? sc.xa_hi : nullptr;
-    __nv_bfloat16* xl = emit_split ? sc.xa_lo : nullptr;
+    __nv_bfloat16* xl = emit_split ? sc.xa_hi + (size_t)Hq * hd : nullptr;
     if (hd == 128) {
-        attn_partial_kernel<128><<<grid, 128, 0, st>>>(sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
+        e = launch_pdl(attn_partial_kernel<128>, grid, dim3(128), 0, st, pdl, sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
                                                        Hkv, (long long)m.d.kv_capacity, R, nsplit, chunk);
-        attn_combine_kernel<128><<<cgrid, 128, 0, st>>>(sc.attn_part, sc.attn, rm.slot, Hq, nsplit, xh, xl);
+        if (e == cudaSuccess)
+            e = launch_pdl(attn_combine_kernel<128>, cgrid, dim3(128), 0, st, pdl, (const float*)sc.attn_part, sc.attn,
+                           (const int32_t*)rm.slot, Hq, nsplit, xh, xl);
     } else if (hd == 64) {
-        attn_partial_kernel<64><<<grid, 128, 0, st>>>(sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
+        e = launch_pdl(attn_partial_kernel<64>, grid, dim3(128), 0, st, pdl, sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
                                                       Hkv, (long long)m.d.kv_capacity, R, nsplit, chunk);
-        attn_combine_kernel<64><<<cgrid, 64, 0, st>>>(sc.attn_part, sc.attn, rm.slot, Hq, nsplit, xh, xl);
+        if (e == cudaSuccess)
+            e = launch_pdl(attn_combine_kernel<64>, cgrid, dim3(64), 0, st, pdl, (const float*)sc.attn_part, sc.attn,
+                           (const int32_t*)rm.slot, Hq, nsplit, xh, xl);
     } else if (hd == 32) {
-        attn_partial_kernel<32><<<grid, 128, 0, st>>>(sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
+        e = launch_pdl(attn_partial_kernel<32>, grid, dim3(128), 0, st, pdl, sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
                                                       Hkv, (long long)m.d.kv_capacity, R, nsplit, chunk);
-        attn_combine_kernel<32><<<cgrid, 32, 0, st>>>(sc.attn_part, sc.attn, rm.slot, Hq, nsplit, xh, xl);
+        if (e == cudaSuccess)
+            e = launch_pdl(attn_combine_kernel<32>, cgrid, dim3(32), 0, st, pdl, (const float*)sc.attn_part, sc.attn,
+                           (const int32_t*)rm.slot, Hq, nsplit, xh, xl);
     } else {
         return cudaErrorInvalidValue;
     }
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace mtad

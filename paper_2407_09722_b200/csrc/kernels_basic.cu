@@ -139,8 +139,8 @@ __global__ void prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, i
         if (a.x_hi) {
             const float y = v * __bfloat162float(a.gain0[i]);
             const __nv_bfloat16 h = __float2bfloat16_rn(y);
-            a.x_hi[(size_t)t * d + i] = h;
-            a.x_lo[(size_t)t * d + i] = __float2bfloat16_rn(y - __bfloat162float(h));
+            a.x_hi[(size_t)t * 2 * d + i] = h;                      // interleaved operand rows: stride 2 d
+            a.x_lo[(size_t)t * 2 * d + i] = __float2bfloat16_rn(y - __bfloat162float(h));
             ss += v * v;
         }
     }

@@ -9,7 +9,8 @@
 // evenly to the CTAs (one per SM); a tile whose k-range spans several CTAs is completed by whichever of them
 // arrives last, which sums the partial tiles in CTA order (deterministic) and runs the fused epilogue.
 //
-// Warp roles: 0 = TMA producer, 1 = TMEM owner + MMA issuer, 2..5 = epilogue (one TMEM lane quadrant each).
+// Warp roles: 0 = TMA producer, 1..4 = MMA issuers (one per 128-row half of a stage; a single thread cannot issue
+// the many small MMAs of a skinny problem fast enough), 5..8 = epilogue (one TMEM lane quadrant each).
 // Every wait on an mbarrier is bounded; on a time-out the kernel raises MTAD_ST_TIMEOUT, waits (bounded) for its
 // own copies in flight, frees its tensor memory and returns.
 #include <math_constants.h>
@@ -23,7 +24,9 @@ namespace {
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr int MAX_STAGES = 12;
 constexpr int EPI_THREADS = 128;
-constexpr int EPI_ROWS = 16;                      // draft rows finished per epilogue pass
+constexpr int EPI_ROWS = 8;                       // draft rows finished per epilogue pass
+constexpr int MAX_HALVES = 4;                     // 128-row weight halves per stage, one MMA-issuing warp each
+constexpr int TC_THREADS = 32 * (1 + MAX_HALVES + 4);
 constexpr uint64_t HINT_STREAM = 0x12F0000000000000ull;   // evict-first: weights are read once
 constexpr uint64_t HINT_KEEP = 0x14F0000000000000ull;     // evict-last: activation operands are re-read by every CTA
 
@@ -111,9 +114,20 @@ __device__ __forceinline__ void split_store(float y, __nv_bfloat16* hi, __nv_bfl
     *lo = __float2bfloat16_rn(y - __bfloat162float(h));
 }
 
+#ifdef MTAD_TC_TRACE
+__device__ unsigned long long g_trace[1024 * 8];
+__device__ __forceinline__ void trace(int k) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    g_trace[blockIdx.x * 8 + k] = t;
+}
+#else
+__device__ __forceinline__ void trace(int) {}
+#endif
+
 struct Smem {
     uint8_t* ring;
-    float (*epi)[TC_TILE_N + 1];
+    float (*epi)[EPI_ROWS][TC_TILE_N + 1];   // [half][row][feature]
     float* rstd;
     float* red;            // [4][EPI_ROWS] floats, also reused as [4][EPI_ROWS] float4 via red4
     float4* red4;
@@ -130,8 +144,8 @@ __device__ __forceinline__ Smem carve(uint8_t* base, int stages, int stage_bytes
     Smem s;
     s.ring = base;
     uint8_t* p = base + (size_t)stages * stage_bytes;
-    s.epi = reinterpret_cast<float(*)[TC_TILE_N + 1]>(p);
-    p += sizeof(float) * EPI_ROWS * (TC_TILE_N + 1);
+    s.epi = reinterpret_cast<float(*)[EPI_ROWS][TC_TILE_N + 1]>(p);
+    p += sizeof(float) * MAX_HALVES * EPI_ROWS * (TC_TILE_N + 1);
     s.rstd = reinterpret_cast<float*>(p);
     p += sizeof(float) * TC_MAX_ROWS;
     p = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(p) + 15) & ~uintptr_t(15));
@@ -154,21 +168,22 @@ __device__ __forceinline__ Smem carve(uint8_t* base, int stages, int stage_bytes
     return s;
 }
 
-constexpr size_t SMEM_TAIL = sizeof(float) * EPI_ROWS * (TC_TILE_N + 1) + sizeof(float) * TC_MAX_ROWS + 16 +
+constexpr size_t SMEM_TAIL = sizeof(float) * MAX_HALVES * EPI_ROWS * (TC_TILE_N + 1) + sizeof(float) * TC_MAX_ROWS + 16 +
                              sizeof(float4) * 4 * EPI_ROWS * 2 + 8 * MAX_STAGES * 2 + 16 + 16 + 8 + 8 + 32;
 
 // ---------------------------------------------------------------------------------------------------------------
-// epilogues: called by the 128 epilogue threads for a block of EPI_ROWS finished rows held in s.epi[j][i]
-// (j: row r0 + j, i: feature n0 + i of the tile).  e = epilogue thread index 0..127.
+// epilogues: called by the 128 epilogue threads for a block of EPI_ROWS finished rows of one 128-feature tile held
+// in epi[j][i] (j: row r0 + j, i: feature tile * 128 + i).  e = epilogue thread index 0..127.
+typedef float (*EpiTile)[TC_TILE_N + 1];
 // ---------------------------------------------------------------------------------------------------------------
 
-__device__ __forceinline__ void epi_plain(const TcGemmParams& p, const Smem& s, int tile, int r0, int e) {
+__device__ __forceinline__ void epi_plain(const TcGemmParams& p, EpiTile epi, int tile, int r0, int e) {
     const int n = tile * TC_TILE_N + e;
     if (n >= p.N) return;
-    for (int j = 0; j < EPI_ROWS && r0 + j < p.T; ++j) p.out[(size_t)(r0 + j) * p.ldo + n] = s.epi[j][e];
+    for (int j = 0; j < EPI_ROWS && r0 + j < p.T; ++j) p.out[(size_t)(r0 + j) * p.ldo + n] = epi[j][e];
 }
 
-__device__ __forceinline__ void epi_qkv(const TcGemmParams& p, const Smem& s, int tile, int r0, int e) {
+__device__ __forceinline__ void epi_qkv(const TcGemmParams& p, EpiTile epi, int tile, int r0, int e) {
     const int hd = p.hd, half = hd >> 1;
     int seg, tin;
     if (tile < p.seg_k_tile) { seg = 0; tin = tile; }
@@ -186,10 +201,10 @@ __device__ __forceinline__ void epi_qkv(const TcGemmParams& p, const Smem& s, in
             const int sl = p.slot[t];
             if (sl < 0) continue;
             const size_t base = (((((size_t)p.layer * p.max_batch + p.seq[t]) * 2 + 1) * p.Hkv + head) * p.cap + sl) * hd;
-            p.cache[base + jin] = __float2bfloat16_rn(s.epi[j][e]);
+            p.cache[base + jin] = __float2bfloat16_rn(epi[j][e]);
         } else if (jin < half) {
             const float c = p.rope[((size_t)t * half + jin) * 2], sn = p.rope[((size_t)t * half + jin) * 2 + 1];
-            const float a = s.epi[j][e], b = s.epi[j][e + half];
+            const float a = epi[j][e], b = epi[j][e + half];
             const float ra = a * c - b * sn, rb = b * c + a * sn;
             if (seg == 0) {
                 float* q = p.q_out + (size_t)t * ldq + head * hd;
@@ -207,7 +222,8 @@ __device__ __forceinline__ void epi_qkv(const TcGemmParams& p, const Smem& s, in
     }
 }
 
-__device__ __forceinline__ void epi_resid(const TcGemmParams& p, const Smem& s, int tile, int r0, int e) {
+__device__ __forceinline__ void epi_resid(const TcGemmParams& p, const Smem& s, EpiTile epi, int tile, int r0,
+                                          int e) {
     const int n = tile * TC_TILE_N + e;
     const bool ok = n < p.N;
     const float g = ok ? __bfloat162float(p.gain[n]) : 0.f;
@@ -216,7 +232,7 @@ __device__ __forceinline__ void epi_resid(const TcGemmParams& p, const Smem& s, 
         const int t = r0 + j;
         float y = 0.f;
         if (ok && t < p.T) {
-            y = p.hidden[(size_t)t * p.N + n] + s.epi[j][e];
+            y = p.hidden[(size_t)t * p.N + n] + epi[j][e];
             p.hidden[(size_t)t * p.N + n] = y;
             split_store(y * g, p.x_hi + (size_t)t * p.ldx + n, p.x_lo + (size_t)t * p.ldx + n);
         }
@@ -229,20 +245,36 @@ __device__ __forceinline__ void epi_resid(const TcGemmParams& p, const Smem& s, 
     if (e < EPI_ROWS && r0 + e < p.T)
         p.sumsq_out[(size_t)tile * TC_X_ROWS + r0 + e] =
             (s.red[e] + s.red[EPI_ROWS + e]) + (s.red[2 * EPI_ROWS + e] + s.red[3 * EPI_ROWS + e]);
+    epi_bar();       // the scratch is reused by the next tile half
 }
 
 __device__ __forceinline__ void epi_swiglu(const TcGemmParams& p, const Smem& s, int tile, int r0, int e) {
-    if (e >= 64) return;
-    const int f = tile * 64 + e;
-    if (f >= p.N) return;
-    for (int j = 0; j < EPI_ROWS && r0 + j < p.T; ++j) {
-        const float g = s.epi[j][e], u = s.epi[j][e + 64];
-        const float a = g / (1.f + expf(-g)) * u;
-        split_store(a, p.x_hi + (size_t)(r0 + j) * p.ldx + f, p.x_lo + (size_t)(r0 + j) * p.ldx + f);
+    // the first half of a tile's weight rows are gate rows, the second half the matching up rows
+    if (p.mh == 1) {
+        if (e >= 64) return;
+        const int f = tile * 64 + e;
+        if (f >= p.N) return;
+        for (int j = 0; j < EPI_ROWS && r0 + j < p.T; ++j) {
+            const float g = s.epi[0][j][e], u = s.epi[0][j][e + 64];
+            split_store(g / (1.f + expf(-g)) * u, p.x_hi + (size_t)(r0 + j) * p.ldx + f,
+                        p.x_lo + (size_t)(r0 + j) * p.ldx + f);
+        }
+        return;
+    }
+    const int hh = p.mh / 2;
+    for (int h = 0; h < hh; ++h) {
+        const int f = tile * 64 * p.mh + h * TC_TILE_N + e;
+        if (f >= p.N) break;
+        for (int j = 0; j < EPI_ROWS && r0 + j < p.T; ++j) {
+            const float g = s.epi[h][j][e], u = s.epi[h + hh][j][e];
+            split_store(g / (1.f + expf(-g)) * u, p.x_hi + (size_t)(r0 + j) * p.ldx + f,
+                        p.x_lo + (size_t)(r0 + j) * p.ldx + f);
+        }
     }
 }
 
-__device__ __forceinline__ void epi_lmhead(const TcGemmParams& p, const Smem& s, int tile, int r0, int e) {
+__device__ __forceinline__ void epi_lmhead(const TcGemmParams& p, const Smem& s, EpiTile epi, int tile, int r0,
+                                           int e) {
     const int v = tile * TC_TILE_N + e;
     const bool ok = v < p.N;
     const int warp = e >> 5, lane = e & 31;
@@ -251,7 +283,7 @@ __device__ __forceinline__ void epi_lmhead(const TcGemmParams& p, const Smem& s,
         float m = -CUDART_INF_F, sum = 0.f, bv = -CUDART_INF_F;
         int bi = 0x7fffffff;
         if (ok && t < p.T) {
-            const float z = s.epi[j][e];
+            const float z = epi[j][e];
             m = z;
             sum = 1.f;
             const float u = p.uniforms[(size_t)(t / p.R) * p.N + v];
@@ -282,7 +314,7 @@ __device__ __forceinline__ void epi_lmhead(const TcGemmParams& p, const Smem& s,
             a.y = sa + sb;
             if (b.z > a.z || (b.z == a.z && __float_as_int(b.w) < __float_as_int(a.w))) { a.z = b.z; a.w = b.w; }
         }
-        p.lm_part[(size_t)(r0 + e) * p.n_tiles + tile] = a;
+        p.lm_part[(size_t)(r0 + e) * p.n_tiles128 + tile] = a;
     }
     // gather: logit of each node's token under its parent row, when both fall into this block of rows and this tile
     const int n0 = tile * TC_TILE_N;
@@ -290,40 +322,50 @@ __device__ __forceinline__ void epi_lmhead(const TcGemmParams& p, const Smem& s,
         const int pr = p.prow[t];
         if (pr < r0 || pr >= r0 + EPI_ROWS) continue;
         const int tk = p.tok[t] - n0;
-        if (tk >= 0 && tk < TC_TILE_N) p.node_z[t] = s.epi[pr - r0][tk];
+        if (tk >= 0 && tk < TC_TILE_N) p.node_z[t] = epi[pr - r0][tk];
     }
+    epi_bar();       // the scratch is reused by the next tile half
 }
 
 // ---------------------------------------------------------------------------------------------------------------
 // kernel
 // ---------------------------------------------------------------------------------------------------------------
 
-__global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__ TcMaps maps, const TcGemmParams p) {
+__global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_constant__ TcMaps maps, const TcGemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int b_bytes = p.rpad * 128;
-    const int stage_bytes = TC_TILE_N * 128 + 2 * b_bytes;
+    const int mh = p.mh;                               // 128-row weight halves per stage (1, 2 or 4)
+    const int a_bytes = mh * TC_TILE_N * 128;
+    const int acc_cols = 2 * p.rpad;                   // one column per operand row: hi and lo of a draft row are neighbours
+    const int n_bbox = acc_cols > 256 ? 2 : 1;         // TMA boxes (and MMAs per k step and half) that cover the operand rows
+    const int bbox_rows = acc_cols / n_bbox;
+    const int stage_bytes = a_bytes + acc_cols * 128;
     const Smem s = carve(smem_base, p.stages, stage_bytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        trace(0);
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps.a0)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps.x)) : "memory");
+        if (p.mode == TC_QKV || p.mode == TC_SWIGLU)
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps.a1)) : "memory");
+        if (p.mode == TC_QKV)
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps.a2)) : "memory");
+    }
     const int u_begin = blockIdx.x * p.units_per_cta;
     const int u_end = min(u_begin + p.units_per_cta, p.total_units);
     const int n_units = max(u_end - u_begin, 0);
     const int KB = p.k_blocks;
-    // hi and lo operand rows sit back to back in a stage, so one MMA of N = 2 * rpad multiplies both (their products
-    // land in neighbouring column blocks and are added when the accumulator is drained); beyond N = 256 two MMAs
-    // accumulate into the same columns instead
-    const bool stacked = 2 * p.rpad <= 256;
-    const int acc_cols = stacked ? 2 * p.rpad : p.rpad;
+    const int nbuf = p.nbuf;
     uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < 2 * acc_cols) tmem_cols <<= 1;
+    while ((int)tmem_cols < nbuf * mh * acc_cols) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.stages; ++i) {
             mbar_init(smem_u32(&s.full[i]), 1);
-            mbar_init(smem_u32(&s.empty[i]), 1);
+            mbar_init(smem_u32(&s.empty[i]), mh);        // one commit per MMA-issuing warp
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(smem_u32(&s.tfull[i]), 1);
+            mbar_init(smem_u32(&s.tfull[i]), mh);
             mbar_init(smem_u32(&s.tempty[i]), 4);
         }
         *s.abort_flag = 0;
@@ -340,53 +382,86 @@ __global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *s.tmem_ptr;
+    if (threadIdx.x == 0) trace(1);
     // let the next kernel in the stream start its own prologue (it waits for this grid before it reads our output)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     volatile int* abort_flag = s.abort_flag;
 
     if (warp == 0) {
-        // ---------------- TMA producer ----------------
-        if (lane == 0 && n_units > 0) {
-            const int box_half = p.mode == TC_SWIGLU;
-            auto issue_a = [&](int i) {
+        // ---------------- TMA producer: the whole warp walks the units, lane l issues the l-th copy of a stage ------
+        if (n_units > 0) {
+            // copies of one stage: weight boxes first (gate|up, or two 256-row boxes of a 512-row tile), then the
+            // operand-row boxes
+            const int n_a = (p.mode == TC_SWIGLU || mh == 4) ? 2 : 1;
+            auto issue = [&](int i, bool do_a, bool do_b) {
                 const int u = u_begin + i, tile = u / KB, kb = u % KB, st = i % p.stages;
                 const uint32_t bar = smem_u32(&s.full[st]);
-                const uint32_t dst = smem_u32(s.ring + (size_t)st * stage_bytes);
-                mbar_expect_tx(bar, (uint32_t)stage_bytes);
-                if (box_half) {
-                    tma_load_2d(dst, &maps.a0, bar, kb * TC_TILE_K, tile * 64, HINT_STREAM);
-                    tma_load_2d(dst + 64 * 128, &maps.a1, bar, kb * TC_TILE_K, tile * 64, HINT_STREAM);
-                } else if (p.mode == TC_QKV) {
-                    const CUtensorMap* m = tile < p.seg_k_tile ? &maps.a0 : (tile < p.seg_v_tile ? &maps.a1 : &maps.a2);
-                    const int tin = tile < p.seg_k_tile ? tile : (tile < p.seg_v_tile ? tile - p.seg_k_tile
-                                                                                       : tile - p.seg_v_tile);
-                    tma_load_2d(dst, m, bar, kb * TC_TILE_K, tin * TC_TILE_N, HINT_STREAM);
+                const uint32_t base = smem_u32(s.ring + (size_t)st * stage_bytes);
+                if (do_a && lane == 0) mbar_expect_tx(bar, (uint32_t)stage_bytes);
+                __syncwarp();
+                const CUtensorMap* m = nullptr;
+                uint32_t dst = 0;
+                int y = 0;
+                uint64_t hint = HINT_STREAM;
+                if (lane < n_a) {
+                    if (!do_a) return;
+                    if (p.mode == TC_SWIGLU) {
+                        // gate rows fill the first half of the stage's weight rows, up rows the second half
+                        const int rows = 64 * mh;
+                        m = lane == 0 ? &maps.a0 : &maps.a1;
+                        dst = base + lane * rows * 128;
+                        y = tile * rows;
+                    } else if (p.mode == TC_QKV) {
+                        const int t128 = tile * mh;
+                        m = t128 < p.seg_k_tile ? &maps.a0 : (t128 < p.seg_v_tile ? &maps.a1 : &maps.a2);
+                        y = (t128 < p.seg_k_tile ? t128 : (t128 < p.seg_v_tile ? t128 - p.seg_k_tile
+                                                                               : t128 - p.seg_v_tile)) * TC_TILE_N +
+                            lane * 256;
+                        dst = base + lane * 256 * 128;
+                    } else {
+                        m = &maps.a0;
+                        y = tile * mh * TC_TILE_N + lane * 256;
+                        dst = base + lane * 256 * 128;
+                    }
+                } else if (lane < n_a + n_bbox) {
+                    if (!do_b) return;
+                    const int b = lane - n_a;
+                    m = &maps.x;
+                    dst = base + a_bytes + b * bbox_rows * 128;
+                    y = b * bbox_rows;
+                    hint = HINT_KEEP;
                 } else {
-                    tma_load_2d(dst, &maps.a0, bar, kb * TC_TILE_K, tile * TC_TILE_N, HINT_STREAM);
+                    return;
                 }
-            };
-            auto issue_b = [&](int i) {
-                const int u = u_begin + i, kb = u % KB, st = i % p.stages;
-                const uint32_t bar = smem_u32(&s.full[st]);
-                const uint32_t dst = smem_u32(s.ring + (size_t)st * stage_bytes) + TC_TILE_N * 128;
-                tma_load_2d(dst, &maps.xhi, bar, kb * TC_TILE_K, 0, HINT_KEEP);
-                tma_load_2d(dst + b_bytes, &maps.xlo, bar, kb * TC_TILE_K, 0, HINT_KEEP);
+                tma_load_2d(dst, m, bar, kb * TC_TILE_K, y, hint);
             };
             // weights do not depend on the previous kernel: start streaming them before waiting for it
             const int pre = min(p.stages, n_units);
-            for (int i = 0; i < pre; ++i) issue_a(i);
+            for (int i = 0; i < pre; ++i) issue(i, true, false);
             asm volatile("griddepcontrol.wait;" ::: "memory");
-            for (int i = 0; i < pre; ++i) issue_b(i);
+            for (int i = 0; i < pre; ++i) issue(i, false, true);
+            if (lane == 0) trace(2);
             bool ok = true;
-            for (int i = pre; i < n_units && ok; ++i) {
+#ifdef MTAD_TC_TRACE
+            unsigned long long t_wait = 0, t_all0 = clock64();
+#endif
+            for (int i = pre; i < n_units; ++i) {
                 const int st = i % p.stages;
                 const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-                ok = mbar_wait(smem_u32(&s.empty[st]), ph ^ 1u, abort_flag);
+#ifdef MTAD_TC_TRACE
+                unsigned long long c0 = clock64();
+                if (lane == 0) ok = mbar_wait(smem_u32(&s.empty[st]), ph ^ 1u, abort_flag);
+                t_wait += clock64() - c0;
+                if (lane == 0 && i == n_units - 1)
+                    g_trace[blockIdx.x * 8 + 7] = (t_wait << 32) | ((clock64() - t_all0) & 0xffffffffull);
+#else
+                if (lane == 0) ok = mbar_wait(smem_u32(&s.empty[st]), ph ^ 1u, abort_flag);
+#endif
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
-                issue_a(i);
-                issue_b(i);
+                issue(i, true, true);
             }
-            if (*abort_flag) {
+            if (lane == 0 && *abort_flag) {
                 // give our own copies in flight a bounded chance to land before the CTA exits
                 const int first = max(0, n_units - p.stages);
                 for (int i = first; i < n_units; ++i) {
@@ -396,50 +471,75 @@ __global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__
                 }
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0 && n_units > 0) {
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) |
-                                   ((uint32_t)((stacked ? 2 * p.rpad : p.rpad) >> 3) << 17) |
+    } else if (warp <= MAX_HALVES) {
+        // ---------------- MMA issuers: warp 1 + h owns the 128-row half h of every stage and its accumulator --------
+        const int h = warp - 1;
+        if (lane == 0 && n_units > 0 && h < mh) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bbox_rows >> 3) << 17) |
                                    ((uint32_t)(TC_TILE_N >> 4) << 24);
             int i = 0, seg = 0;
             bool ok = true;
+#ifdef MTAD_TC_TRACE
+            unsigned long long mma_wait = 0, mma_t0 = clock64(), mma_issue = 0, mma_commit = 0;
+#endif
             while (i < n_units && ok) {
                 const int u = u_begin + i;
                 const int kb0 = u % KB;
                 const int len = min(KB - kb0, n_units - i);
-                const int buf = seg & 1;
-                const uint32_t aph = (uint32_t)(seg >> 1) & 1u;
+                const int buf = seg % nbuf;
+                const uint32_t aph = (uint32_t)(seg / nbuf) & 1u;
                 ok = mbar_wait(smem_u32(&s.tempty[buf]), aph ^ 1u, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * acc_cols);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * mh * acc_cols);
                 for (int k = 0; k < len && ok; ++k, ++i) {
                     const int st = i % p.stages;
                     const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+#ifdef MTAD_TC_TRACE
+                    unsigned long long c0 = clock64();
                     ok = mbar_wait(smem_u32(&s.full[st]), ph, abort_flag);
+                    if (i > 0) mma_wait += clock64() - c0;
+#else
+                    ok = mbar_wait(smem_u32(&s.full[st]), ph, abort_flag);
+#endif
                     if (!ok) break;
+                    if (i == 0 && h == 0) trace(3);
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(s.ring + (size_t)st * stage_bytes);
-                    const uint32_t bh_addr = a_addr + TC_TILE_N * 128;
-                    const uint32_t bl_addr = bh_addr + b_bytes;
+                    const uint32_t b_addr = a_addr + a_bytes;
+#ifdef MTAD_TC_TRACE
+                    unsigned long long ci0 = clock64();
+#endif
 #pragma unroll
                     for (int k4 = 0; k4 < TC_TILE_K / 16; ++k4) {
-                        const uint64_t ad = smem_desc(a_addr + k4 * 32);
-                        tc_mma(d_tmem, ad, smem_desc(bh_addr + k4 * 32), idesc, (k > 0 || k4 > 0) ? 1u : 0u);
-                        if (!stacked) tc_mma(d_tmem, ad, smem_desc(bl_addr + k4 * 32), idesc, 1u);
+                        const uint32_t acc = (k > 0 || k4 > 0) ? 1u : 0u;
+                        const uint64_t ad = smem_desc(a_addr + h * TC_TILE_N * 128 + k4 * 32);
+                        for (int b = 0; b < n_bbox; ++b)
+                            tc_mma(d_tmem + (uint32_t)(h * acc_cols + b * bbox_rows), ad,
+                                   smem_desc(b_addr + b * bbox_rows * 128 + k4 * 32), idesc, acc);
                     }
+#ifdef MTAD_TC_TRACE
+                    unsigned long long ci1 = clock64();
+#endif
                     tc_commit(smem_u32(&s.empty[st]));      // frees the smem stage once these MMAs have read it
+#ifdef MTAD_TC_TRACE
+                    mma_issue += ci1 - ci0; mma_commit += clock64() - ci1;
+#endif
                 }
                 if (ok) tc_commit(smem_u32(&s.tfull[buf]));  // accumulator of this segment complete
                 ++seg;
             }
+            if (h == 0) trace(4);
+#ifdef MTAD_TC_TRACE
+            if (h == 0) g_trace[blockIdx.x * 8 + 5] = (mma_wait << 32) | ((clock64() - mma_t0) & 0xffffffffull);
+            if (h == 0) g_trace[blockIdx.x * 8 + 6] = (mma_issue << 32) | (mma_commit & 0xffffffffull);
+#endif
         }
     } else {
         // ---------------- epilogue ----------------
-        const int e = threadIdx.x - 64;                 // 0..127
+        const int e = threadIdx.x - 32 * (1 + MAX_HALVES);   // 0..127
         const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
-        const int feat = quad * 32 + lane;              // feature (TMEM lane) within the tile
+        const int feat = quad * 32 + lane;              // feature (TMEM lane) within a 128-row half
         asm volatile("griddepcontrol.wait;" ::: "memory");
         // deferred RMSNorm scale of every row
         for (int r = e; r < TC_MAX_ROWS; r += EPI_THREADS) {
@@ -452,16 +552,18 @@ __global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__
             s.rstd[r] = v;
         }
         epi_bar();
+        const size_t half_floats = (size_t)p.rpad * TC_TILE_N;
+        const size_t part_floats = (size_t)mh * half_floats;
         int i = 0, seg = 0;
         while (i < n_units) {
             const int u = u_begin + i;
             const int tile = u / KB, kb0 = u % KB;
             const int len = min(KB - kb0, n_units - i);
-            const int buf = seg & 1;
-            const uint32_t aph = (uint32_t)(seg >> 1) & 1u;
+            const int buf = seg % nbuf;
+            const uint32_t aph = (uint32_t)(seg / nbuf) & 1u;
             bool ok = true;
             if (lane == 0) ok = mbar_wait(smem_u32(&s.tfull[buf]), aph, abort_flag);
-            if (lane == 0) s.flags[1 + (warp - 2)] = ok ? 1 : 0;
+            if (lane == 0) s.flags[1 + (warp - 1 - MAX_HALVES)] = ok ? 1 : 0;
             epi_bar();
             if (!(s.flags[1] && s.flags[2] && s.flags[3] && s.flags[4])) break;   // uniform over the 128 threads
             tc_fence_after();
@@ -470,20 +572,18 @@ __global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__
             const int c_last = ((tile + 1) * KB - 1) / p.units_per_cta;
             const int n_contrib = c_last - c_first + 1;
             const int slot_idx = (int)blockIdx.x - c_first;
-            float* part = p.ws + ((size_t)tile * p.max_contrib + slot_idx) * ((size_t)p.rpad * TC_TILE_N);
-            for (int c0 = 0; c0 < p.T; c0 += 16) {
-                float v[16];
-                const uint32_t col = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * acc_cols + c0);
-                tc_ld16(col, v);
-                if (stacked) {
-                    float w[16];
-                    tc_ld16(col + (uint32_t)p.rpad, w);
+            float* part = p.ws + ((size_t)tile * p.max_contrib + slot_idx) * part_floats;
+            for (int h = 0; h < mh; ++h) {
+                for (int c0 = 0; c0 < 2 * p.T; c0 += 16) {
+                    float v[16];
+                    tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) +
+                                (uint32_t)(buf * mh * acc_cols + h * acc_cols + c0), v);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] += w[j];
+                    for (int j = 0; j < 8; ++j) {
+                        const int r = (c0 >> 1) + j;
+                        if (r < p.T) part[h * half_floats + (size_t)r * TC_TILE_N + feat] = v[2 * j] + v[2 * j + 1];
+                    }
                 }
-#pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    if (c0 + j < p.T) part[(size_t)(c0 + j) * TC_TILE_N + feat] = v[j];
             }
             tc_fence_before();
             __syncwarp();
@@ -497,25 +597,46 @@ __global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__
             epi_bar();
             if (s.flags[0]) {
                 __threadfence();
-                const float* tile_ws = p.ws + (size_t)tile * p.max_contrib * ((size_t)p.rpad * TC_TILE_N);
+                const float* tile_ws = p.ws + (size_t)tile * p.max_contrib * part_floats;
                 for (int r0 = 0; r0 < p.T; r0 += EPI_ROWS) {
-                    for (int j = 0; j < EPI_ROWS; ++j) {
-                        const int r = r0 + j;
-                        float acc = 0.f;
-                        if (r < p.T) {
-                            for (int c = 0; c < n_contrib; ++c)
-                                acc += __ldcg(tile_ws + (size_t)c * p.rpad * TC_TILE_N + (size_t)r * TC_TILE_N + e);
-                            acc *= s.rstd[r];
+                    for (int h = 0; h < mh; ++h) {
+                        float acc[EPI_ROWS];
+#pragma unroll
+                        for (int j = 0; j < EPI_ROWS; ++j) acc[j] = 0.f;
+                        // partials are added in CTA order (deterministic); four contributors' loads are issued
+                        // together so that the L2 latency is paid once per group, not once per contributor
+                        for (int c = 0; c < n_contrib; c += 4) {
+                            float v[4][EPI_ROWS];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const float* src = tile_ws + (size_t)(c + q) * part_floats + h * half_floats + e;
+#pragma unroll
+                                for (int j = 0; j < EPI_ROWS; ++j)
+                                    v[q][j] = (c + q < n_contrib && r0 + j < p.T)
+                                                  ? __ldcg(src + (size_t)(r0 + j) * TC_TILE_N) : 0.f;
+                            }
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                                for (int j = 0; j < EPI_ROWS; ++j) acc[j] += v[q][j];
                         }
-                        s.epi[j][e] = acc;
+#pragma unroll
+                        for (int j = 0; j < EPI_ROWS; ++j) s.epi[h][j][e] = (r0 + j < p.T) ? acc[j] * s.rstd[r0 + j] : 0.f;
                     }
                     epi_bar();
-                    switch (p.mode) {
-                        case TC_PLAIN: epi_plain(p, s, tile, r0, e); break;
-                        case TC_QKV: epi_qkv(p, s, tile, r0, e); break;
-                        case TC_RESID: epi_resid(p, s, tile, r0, e); break;
-                        case TC_SWIGLU: epi_swiglu(p, s, tile, r0, e); break;
-                        default: epi_lmhead(p, s, tile, r0, e); break;
+                    if (p.mode == TC_SWIGLU) {
+                        epi_swiglu(p, s, tile, r0, e);
+                    } else {
+                        for (int h = 0; h < mh; ++h) {
+                            const int t128 = tile * mh + h;
+                            if (t128 * TC_TILE_N >= p.n_rows_total) break;      // half beyond the last weight row
+                            switch (p.mode) {
+                                case TC_PLAIN: epi_plain(p, s.epi[h], t128, r0, e); break;
+                                case TC_QKV: epi_qkv(p, s.epi[h], t128, r0, e); break;
+                                case TC_RESID: epi_resid(p, s, s.epi[h], t128, r0, e); break;
+                                default: epi_lmhead(p, s, s.epi[h], t128, r0, e); break;
+                            }
+                        }
                     }
                     epi_bar();
                 }
@@ -529,6 +650,7 @@ __global__ void __launch_bounds__(192, 1) tc_gemm_kernel(const __grid_constant__
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
+        __syncwarp();
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
@@ -560,6 +682,12 @@ EncodeTiledFn encode_fn() {
 
 }  // namespace
 
+#ifdef MTAD_TC_TRACE
+extern "C" int mtad_debug_trace(unsigned long long* out, int n) {
+    return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(unsigned long long) * n);
+}
+#endif
+
 int tc_make_map(CUtensorMap* out, const void* base, long long rows, long long cols, int box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return -1;
@@ -585,16 +713,27 @@ void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int ctas) {
     p.rpad = (T + 15) / 16 * 16;
 }
 
+int tc_halves(int T) {
+    // TMEM holds 2 buffers x halves x 2 * rpad columns <= 512; two halves (two MMA-issuing warps) already keep the
+    // tensor pipe ahead of HBM, and smaller stages fill and drain faster than 512-row ones
+    static const int cap = getenv("MTAD_TC_MH") ? atoi(getenv("MTAD_TC_MH")) : 2;
+    const int rpad = (T + 15) / 16 * 16;
+    const int fit = rpad <= 32 ? 4 : (rpad <= 64 ? 2 : 1);
+    return fit < cap ? fit : cap;
+}
+
 size_t tc_workspace_floats(int n_tiles_max, int max_contrib_max, int rpad_max) {
     return (size_t)n_tiles_max * max_contrib_max * rpad_max * TC_TILE_N;
 }
 
 cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p_in, int ctas, bool pdl, cudaStream_t st) {
     TcGemmParams p = p_in;
-    const int stage_bytes = TC_TILE_N * 128 + 2 * p.rpad * 128;
-    // two CTAs of consecutive kernels share an SM while one drains and the next prefetches: stay under half of it
+    if (p.mh != 1 && p.mh != 2 && p.mh != 4) return cudaErrorInvalidValue;
+    p.nbuf = (2 * p.mh * 2 * p.rpad <= 512) ? 2 : 1;
+    if (p.mh * 2 * p.rpad > 512) return cudaErrorInvalidValue;
+    const int stage_bytes = p.mh * TC_TILE_N * 128 + 2 * p.rpad * 128;
     static const int budget_kb_env = getenv("MTAD_TC_SMEM_KB") ? atoi(getenv("MTAD_TC_SMEM_KB")) : 0;
-    const size_t budget = budget_kb_env > 0 ? (size_t)budget_kb_env * 1024 : (p.rpad <= 32 ? 113 : 200) * 1024;
+    const size_t budget = (size_t)(budget_kb_env > 0 ? budget_kb_env : 226) * 1024;
     int stages = (int)((budget - SMEM_TAIL - 1024) / stage_bytes);
     stages = stages > MAX_STAGES ? MAX_STAGES : stages;
     if (stages < 2) return cudaErrorInvalidValue;
@@ -609,7 +748,7 @@ cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p_in, int cta
     const int grid = (p.total_units + p.units_per_cta - 1) / p.units_per_cta;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(192);
+    cfg.blockDim = dim3(TC_THREADS);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute at[1];

@@ -24,12 +24,16 @@ struct TcGemmParams {
     // decomposition
     int n_tiles, k_blocks, total_units, units_per_cta, max_contrib;
     int T;                 // valid activation rows
-    int rpad;              // MMA N: T rounded up to 16
+    int rpad;              // T rounded up to 16; the operand tile has 2 * rpad rows (hi and lo of a row are neighbours)
+    int mh;                // 128-row weight halves per tile and stage (1 or 2); a tile is mh * 128 output features
+    int nbuf;              // TMEM accumulator buffers (set by the launcher)
+    int n_rows_total;      // weight rows, for skipping a half that lies beyond them
+    int n_tiles128;        // ceil(N / 128): row stride of lm_part
     int stages;            // smem ring depth
     int mode;
     int N;                 // output features (bound for stores)
     // split-K fix-up
-    float* ws;             // [n_tiles][max_contrib][rpad][128] partial tiles
+    float* ws;             // [n_tiles][max_contrib][mh][rpad][128] partial tiles
     int* counters;         // [n_tiles], zero between launches
     uint32_t* status;      // device status word for time-outs (may be null)
     // deferred RMSNorm of the input: rstd[r] = rsqrt(sum_parts / dim + eps); parts == 0 -> 1
@@ -52,8 +56,8 @@ struct TcGemmParams {
     // TC_RESID / TC_SWIGLU outputs
     float* hidden;                  // [T, N]
     const __nv_bfloat16* gain;      // [N] gains of the norm that follows (TC_RESID)
-    __nv_bfloat16* x_hi;            // [TC_X_ROWS, ldx] operand buffers for the next GEMM
-    __nv_bfloat16* x_lo;
+    __nv_bfloat16* x_hi;            // operand rows for the next GEMM: row t of the hi part at x_hi + t * ldx,
+    __nv_bfloat16* x_lo;            // of the lo part at x_lo + t * ldx (interleaved buffer: x_lo = x_hi + K, ldx = 2 K)
     int ldx;
     float* sumsq_out;               // [n_tiles][TC_X_ROWS]
     // TC_LMHEAD
@@ -67,7 +71,7 @@ struct TcGemmParams {
 
 struct TcMaps {
     CUtensorMap a0, a1, a2;         // weight maps (QKV: wq, wk, wv; SwiGLU: gate, up; else a0)
-    CUtensorMap xhi, xlo;           // activation operand maps
+    CUtensorMap x;                  // operand rows [2 * TC_X_ROWS, K]: row 2t = hi(t), row 2t + 1 = lo(t)
 };
 
 // Encodes a 2-D bf16 tensor map (row-major [rows, cols], 128-byte swizzle, box [box_rows, 64]).
@@ -75,6 +79,8 @@ int tc_make_map(CUtensorMap* out, const void* base, long long rows, long long co
 
 // Fills the decomposition fields of p for a problem of n_tiles x k_blocks on `ctas` CTAs.
 void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int ctas);
+// Weight halves per tile that fit tensor memory for T rows (2 up to 64 rows, else 1).
+int tc_halves(int T);
 size_t tc_workspace_floats(int n_tiles_max, int max_contrib_max, int rpad_max);
 
 cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p, int ctas, bool pdl, cudaStream_t st);
