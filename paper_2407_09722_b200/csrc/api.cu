@@ -91,8 +91,11 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     const size_t F = mx([](const mtad_model_desc* m) { return (size_t)m->d_ffn; });
     const size_t V = mx([](const mtad_model_desc* m) { return (size_t)m->vocab; });
     const size_t hh = mx([](const mtad_model_desc* m) { return (size_t)m->head_dim / 2; });
-    const size_t part = mx([](const mtad_model_desc* m) {
-        return (size_t)m->n_q_heads * attn_split_cap(m->n_q_heads) * (m->head_dim + 2);
+    // split-KV partials: one split per 64 keys on the tensor-core attention path
+    const size_t part = mx([&](const mtad_model_desc* m) {
+        const size_t splits = std::max<size_t>(attn_split_cap(m->n_q_heads),
+                                               (size_t)((m->kv_capacity + max_nodes + 1 + 63) / 64));
+        return (size_t)m->n_q_heads * splits * (m->head_dim + 2);
     });
     SeqState st;
     st.kv_len = k.take<int32_t>(max_batch);
@@ -312,7 +315,13 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             mp.a0 = wm.wq[ix(mq)][l]; mp.a1 = wm.wk[ix(mq)][l]; mp.a2 = wm.wv[ix(mq)][l]; mp.x = xd;
             RUN(MTAD_K_GEMM, wb * (qd + 2.0 * kvd) * d.d_model, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
         }
-        RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, true, pdl, s));
+        if (d.head_dim == 64 || d.head_dim == 128) {
+            const int ns = (int)((total + 63) / 64);
+            RUN(MTAD_K_ATTN, 0, 2, launch_attention_mma(m, l, ctx->rm, sc, B, R, ns, pdl, s));
+            RUN(MTAD_K_ATTN, 0, 0, launch_attention_combine(m, ctx->rm, sc, B, R, ns, true, pdl, s));
+        } else {
+            RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, true, pdl, s));
+        }
         {   // O projection + residual, emits the FFN norm's operand rows
             TcGemmParams p = base; TcMaps mp{};
             tc_decompose(p, up(d.d_model, 128 * mh), qd, T, kCtas);

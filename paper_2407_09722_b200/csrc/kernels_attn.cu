@@ -205,4 +205,19 @@ cudaError_t launch_attention(const ModelView& m, int layer, const RowMeta& rm, c
     return e;
 }
 
+cudaError_t launch_attention_combine(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int nsplit,
+                                     bool emit_split, bool pdl, cudaStream_t st) {
+    const int Hq = m.d.n_q_heads, hd = m.d.head_dim;
+    dim3 cgrid(B * R, Hq);
+    __nv_bfloat16* xh = emit_split ? sc.xa_hi : nullptr;
+    __nv_bfloat16* xl = emit_split ? sc.xa_hi + (size_t)Hq * hd : nullptr;
+    if (hd == 128)
+        return launch_pdl(attn_combine_kernel<128>, cgrid, dim3(128), 0, st, pdl, (const float*)sc.attn_part, sc.attn,
+                          (const int32_t*)rm.slot, Hq, nsplit, xh, xl);
+    if (hd == 64)
+        return launch_pdl(attn_combine_kernel<64>, cgrid, dim3(64), 0, st, pdl, (const float*)sc.attn_part, sc.attn,
+                          (const int32_t*)rm.slot, Hq, nsplit, xh, xl);
+    return cudaErrorInvalidValue;
+}
+
 }  // namespace mtad
