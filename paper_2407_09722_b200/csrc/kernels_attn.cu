@@ -135,7 +135,8 @@ __global__ void __launch_bounds__(128) attn_partial_kernel(const float* __restri
     }
 }
 
-// merge the split partials of one (row, head) in split order
+// merge the split partials of one (row, head), in split order: the split weights exp(m_s - M) are computed once by
+// the block, then every thread sums its output dimension over the splits with independent loads
 template <int HD>
 __global__ void attn_combine_kernel(const float* __restrict__ part, float* __restrict__ out, const int32_t* slot,
                                     int Hq, int nsplit, __nv_bfloat16* __restrict__ x_hi,
@@ -151,18 +152,33 @@ __global__ void attn_combine_kernel(const float* __restrict__ part, float* __res
         if (x_hi) { x_hi[xidx] = __float2bfloat16_rn(0.f); x_lo[xidx] = __float2bfloat16_rn(0.f); }
         return;
     }
+    extern __shared__ float wsm[];                  // [nsplit] weights, then [1] the normaliser
     const float* p = part + (((size_t)t * Hq + h) * nsplit) * (HD + 2);
-    float M = -CUDART_INF_F;
-    for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p[s * (HD + 2)]);
-    float lsum = 0.f, acc = 0.f;
-    for (int s = 0; s < nsplit; ++s) {
-        const float ms = p[s * (HD + 2)];
-        if (ms == -CUDART_INF_F) continue;
-        const float w = expf(ms - M);
-        lsum += p[s * (HD + 2) + 1] * w;
-        acc += p[s * (HD + 2) + 2 + d] * w;
+    __shared__ float s_max;
+    if (threadIdx.x < 32) {
+        float M = -CUDART_INF_F;
+        for (int s = threadIdx.x; s < nsplit; s += 32) M = fmaxf(M, p[(size_t)s * (HD + 2)]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        if (threadIdx.x == 0) s_max = M;
     }
-    const float y = acc / lsum;
+    __syncthreads();
+    const float M = s_max;
+    for (int s = threadIdx.x; s < nsplit; s += blockDim.x) {
+        const float ms = p[(size_t)s * (HD + 2)];
+        wsm[s] = (ms == -CUDART_INF_F) ? 0.f : expf(ms - M);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {                          // fixed order: deterministic
+        float lsum = 0.f;
+        for (int s = 0; s < nsplit; ++s) lsum += p[(size_t)s * (HD + 2) + 1] * wsm[s];
+        wsm[nsplit] = lsum;
+    }
+    float acc = 0.f;
+#pragma unroll 8
+    for (int s = 0; s < nsplit; ++s) acc += p[(size_t)s * (HD + 2) + 2 + d] * wsm[s];
+    __syncthreads();
+    const float y = acc / wsm[nsplit];
     *dst = y;
     if (x_hi) {      // operand rows of the O projection: bf16 hi + lo
         const __nv_bfloat16 hb = __float2bfloat16_rn(y);
@@ -185,19 +201,19 @@ cudaError_t launch_attention(const ModelView& m, int layer, const RowMeta& rm, c
         e = launch_pdl(attn_partial_kernel<128>, grid, dim3(128), 0, st, pdl, sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
                                                        Hkv, (long long)m.d.kv_capacity, R, nsplit, chunk);
         if (e == cudaSuccess)
-            e = launch_pdl(attn_combine_kernel<128>, cgrid, dim3(128), 0, st, pdl, (const float*)sc.attn_part, sc.attn,
+            e = launch_pdl(attn_combine_kernel<128>, cgrid, dim3(128), (nsplit + 1) * sizeof(float), st, pdl, (const float*)sc.attn_part, sc.attn,
                            (const int32_t*)rm.slot, Hq, nsplit, xh, xl);
     } else if (hd == 64) {
         e = launch_pdl(attn_partial_kernel<64>, grid, dim3(128), 0, st, pdl, sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
                                                       Hkv, (long long)m.d.kv_capacity, R, nsplit, chunk);
         if (e == cudaSuccess)
-            e = launch_pdl(attn_combine_kernel<64>, cgrid, dim3(64), 0, st, pdl, (const float*)sc.attn_part, sc.attn,
+            e = launch_pdl(attn_combine_kernel<64>, cgrid, dim3(64), (nsplit + 1) * sizeof(float), st, pdl, (const float*)sc.attn_part, sc.attn,
                            (const int32_t*)rm.slot, Hq, nsplit, xh, xl);
     } else if (hd == 32) {
         e = launch_pdl(attn_partial_kernel<32>, grid, dim3(128), 0, st, pdl, sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
                                                       Hkv, (long long)m.d.kv_capacity, R, nsplit, chunk);
         if (e == cudaSuccess)
-            e = launch_pdl(attn_combine_kernel<32>, cgrid, dim3(32), 0, st, pdl, (const float*)sc.attn_part, sc.attn,
+            e = launch_pdl(attn_combine_kernel<32>, cgrid, dim3(32), (nsplit + 1) * sizeof(float), st, pdl, (const float*)sc.attn_part, sc.attn,
                            (const int32_t*)rm.slot, Hq, nsplit, xh, xl);
     } else {
         return cudaErrorInvalidValue;
@@ -212,10 +228,10 @@ cudaError_t launch_attention_combine(const ModelView& m, const RowMeta& rm, cons
     __nv_bfloat16* xh = emit_split ? sc.xa_hi : nullptr;
     __nv_bfloat16* xl = emit_split ? sc.xa_hi + (size_t)Hq * hd : nullptr;
     if (hd == 128)
-        return launch_pdl(attn_combine_kernel<128>, cgrid, dim3(128), 0, st, pdl, (const float*)sc.attn_part, sc.attn,
+        return launch_pdl(attn_combine_kernel<128>, cgrid, dim3(128), (nsplit + 1) * sizeof(float), st, pdl, (const float*)sc.attn_part, sc.attn,
                           (const int32_t*)rm.slot, Hq, nsplit, xh, xl);
     if (hd == 64)
-        return launch_pdl(attn_combine_kernel<64>, cgrid, dim3(64), 0, st, pdl, (const float*)sc.attn_part, sc.attn,
+        return launch_pdl(attn_combine_kernel<64>, cgrid, dim3(64), (nsplit + 1) * sizeof(float), st, pdl, (const float*)sc.attn_part, sc.attn,
                           (const int32_t*)rm.slot, Hq, nsplit, xh, xl);
     return cudaErrorInvalidValue;
 }
