@@ -121,6 +121,8 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     sc.act = k.take<float>(T * F);
     sc.rope = k.take<float>(T * hh * 2);
     sc.attn_part = k.take<float>(T * part);
+    sc.q_hi = k.take<__nv_bfloat16>(T * qd);
+    sc.q_lo = k.take<__nv_bfloat16>(T * qd);
     sc.logits = k.take<float>(T * V);
     sc.node_lp = k.take<float>(T);
     sc.row_lse = k.take<float>(T);
@@ -299,7 +301,7 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
     base.ws = sc.tc_ws; base.counters = sc.tc_counters; base.status = status;
     base.inv_dim = 1.f / (float)d.d_model; base.eps = d.rms_eps;
     base.Hq = d.n_q_heads; base.Hkv = d.n_kv_heads; base.hd = d.head_dim;
-    base.q_out = sc.qkv; base.rope = sc.rope; base.cache = static_cast<__nv_bfloat16*>(d.kv_cache);
+    base.q_out = sc.qkv; base.q_hi = sc.q_hi; base.q_lo = sc.q_lo; base.rope = sc.rope; base.cache = static_cast<__nv_bfloat16*>(d.kv_cache);
     base.slot = ctx->rm.slot; base.seq = ctx->rm.seq; base.max_batch = m.max_batch; base.cap = d.kv_capacity;
     base.hidden = sc.hidden; base.R = R; base.prow = ctx->rm.prow; base.tok = ctx->rm.tok; base.node_z = sc.node_z;
     base.lm_part = sc.lm_part; base.uniforms = uniforms;

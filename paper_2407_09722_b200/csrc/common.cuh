@@ -54,6 +54,7 @@ struct Scratch {
     float* act;          // [T, F]
     float* rope;         // [T, hd/2, 2]
     float* attn_part;    // [T, Hq, nsplit, hd + 2]
+    __nv_bfloat16 *q_hi, *q_lo;   // [T, Hq hd] query rows as bf16 hi / lo (tensor-core attention operands)
     float* logits;       // [T, V]
     float* node_lp;      // [T]
     float* row_lse;      // [T]

@@ -51,19 +51,25 @@ __device__ __forceinline__ void split2(float x, float y, uint32_t& hi, uint32_t&
 }  // namespace
 
 // part[(t * Hq + h) * nsplit + split] = (running max m, sum l, unnormalised output o[HD]) of row t, head h over the
-// keys of the split; attn_combine_kernel merges the splits in order.
+// keys of the split; attn_combine_kernel merges the splits in order.  q_hi / q_lo hold the query rows times
+// log2(e) / sqrt(HD), so the softmax numerators are exp2(s - m); m is stored back in natural-log units.
 template <int HD>
-__global__ void __launch_bounds__(128) attn_mma_kernel(const float* __restrict__ qkv, int ldq,
-                                                       const __nv_bfloat16* __restrict__ cache, RowMeta rm,
-                                                       float* __restrict__ part, int layer, int max_batch, int Hq,
-                                                       int Hkv, long long cap, int R, int nsplit) {
+__global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* __restrict__ q_hi,
+                                                          const __nv_bfloat16* __restrict__ q_lo,
+                                                          const __nv_bfloat16* __restrict__ cache, RowMeta rm,
+                                                          float* __restrict__ part, int layer, int max_batch, int Hq,
+                                                          int Hkv, long long cap, int R, int nsplit, int nslab) {
     constexpr int ROWB = HD * 2;          // bytes of one key row
     constexpr int CPR = HD / 8;           // 16-byte pieces per row
     constexpr int NDT = HD / 8;           // 8-wide output tiles over the head dim
+    constexpr int SLAB = 2 * 16 * ROWB;   // one query tile: 16 rows hi, then 16 rows lo
+    constexpr int PARK = HD + 8;          // row stride (floats) of a parked output tile
+    constexpr float LN2 = 0.6931471805599453f;
     extern __shared__ __align__(128) uint8_t smem[];
     uint8_t* Ks = smem;                               // [KT][HD] bf16, piece c of row k stored at piece c ^ (k & 7)
     uint8_t* Vs = smem + KT * ROWB;
-    uint8_t* Qs = smem + 2 * KT * ROWB;               // per warp: [16][HD] hi then [16][HD] lo, same swizzle
+    uint8_t* Qs = smem + 2 * KT * ROWB;               // nslab query tiles, same swizzle
+    float* ml = reinterpret_cast<float*>(Qs + nslab * SLAB);           // [4 warps][16 rows][m, l]
 
     const int sp = blockIdx.x, g = blockIdx.y, bi = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -75,9 +81,10 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const float* __restrict__
     const int nkeys = L + nrows;
     const int k_begin = sp * KT;
     const int G = Hq / Hkv;
+    const int n_q = G * nrows;                        // query rows of this KV head: (head in group, draft row)
     if (k_begin >= nkeys) {
         // empty split: leave neutral partials so that the combine pass can read every split
-        for (int i = threadIdx.x; i < G * nrows; i += blockDim.x) {
+        for (int i = threadIdx.x; i < n_q; i += blockDim.x) {
             const int h = g * G + i / nrows, r = i % nrows;
             float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
             dst[0] = -CUDART_INF_F;
@@ -88,7 +95,30 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const float* __restrict__
     const int seq = rm.call_seq[bi];
     const __nv_bfloat16* Kg = cache + (((((size_t)layer * max_batch + seq) * 2 + 0) * Hkv + g) * cap) * HD;
     const __nv_bfloat16* Vg = cache + (((((size_t)layer * max_batch + seq) * 2 + 1) * Hkv + g) * cap) * HD;
+    const int n_mt = (n_q + 15) / 16;
+    // With fewer than three query tiles the warps share a tile and split its 64 keys instead (kparts warps per
+    // tile, merged through shared memory below); otherwise every warp runs whole tiles against all 64 keys.
+    const int kparts = n_mt >= 3 ? 1 : (n_mt == 2 ? 2 : 4);
+    const int cnt = 4 / kparts;                       // 16-key groups per task
+    const int kt0 = (warp % kparts) * cnt;            // first 16-key group of this warp's tasks
 
+    // query tile mt -> slab (16-byte async copies by `nthr` threads; rows past the last query are zero-filled)
+    auto stage_q = [&](int mt, int slab, int tid, int nthr) {
+        uint8_t* dst = Qs + slab * SLAB;
+        for (int i = tid; i < 2 * 16 * CPR; i += nthr) {
+            const int which = i / (16 * CPR), row = (i / CPR) % 16, c = i % CPR;
+            const int qi = mt * 16 + row;
+            const bool valid = qi < n_q;
+            const int hg = valid ? qi / nrows : 0, r = valid ? qi % nrows : 0;
+            const __nv_bfloat16* src = (which ? q_lo : q_hi) + ((size_t)(bi * R + r) * Hq + g * G + hg) * HD + c * 8;
+            cp_async16(s_u32(dst + which * 16 * ROWB + row * ROWB + ((c ^ (row & 7)) << 4)), src, valid);
+        }
+    };
+    if (kparts > 1) {
+        for (int mt = 0; mt < n_mt; ++mt) stage_q(mt, mt, threadIdx.x, blockDim.x);
+    } else if (warp < n_mt) {
+        stage_q(warp, warp, lane, 32);
+    }
     // ---- K and V rows of this split -> shared memory (zero-filled past the last key) ----
     for (int i = threadIdx.x; i < KT * CPR; i += blockDim.x) {
         const int key = i / CPR, c = i % CPR;
@@ -99,47 +129,27 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const float* __restrict__
         cp_async16(s_u32(Vs + soff), Vg + goff, valid);
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
-
-    const int n_q = G * nrows;                        // query rows of this KV head: (head in group, draft row)
-    const int n_mt = (n_q + 15) / 16;
-    uint8_t* Qw = Qs + warp * (2 * 16 * ROWB);
-    const int gq = lane >> 2, tq = lane & 3;          // fragment coordinates
-    const bool spec = k_begin + KT > L;               // the split reaches into the draft rows: masks apply
-
-    // 16 query rows of tile mt as bf16 hi / lo in this warp's slab
-    auto stage_q = [&](int mt) {
-        for (int i = lane; i < 16 * (HD / 2); i += 32) {
-            const int row = i / (HD / 2), d2 = (i % (HD / 2)) * 2;
-            const int qi = mt * 16 + row;
-            float x = 0.f, y = 0.f;
-            if (qi < n_q) {
-                const int hg = qi / nrows, r = qi % nrows;
-                const float2 v =
-                    *reinterpret_cast<const float2*>(qkv + (size_t)(bi * R + r) * ldq + (g * G + hg) * HD + d2);
-                x = v.x;
-                y = v.y;
-            }
-            uint32_t hi, lo;
-            split2(x, y, hi, lo);
-            const uint32_t off = row * ROWB + (((d2 >> 3) ^ (row & 7)) << 4) + (d2 & 7) * 2;
-            *reinterpret_cast<uint32_t*>(Qw + off) = hi;
-            *reinterpret_cast<uint32_t*>(Qw + 16 * ROWB + off) = lo;
-        }
-    };
-    if (warp < n_mt) stage_q(warp);                   // overlaps the K/V copies in flight
     asm volatile("cp.async.wait_all;" ::: "memory");
     __syncthreads();
 
-    const uint32_t ks_base = s_u32(Ks), vs_base = s_u32(Vs), qh_base = s_u32(Qw), ql_base = s_u32(Qw + 16 * ROWB);
+    const int gq = lane >> 2, tq = lane & 3;          // fragment coordinates
+    const bool spec = k_begin + KT > L;               // the split reaches into the draft rows: masks apply
+    const uint32_t ks_base = s_u32(Ks), vs_base = s_u32(Vs);
     const int lrow = lane & 7, lid = lane >> 3;       // ldmatrix: row within an 8x8 matrix, matrix id
+    float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, l0 = 0.f, l1 = 0.f;
+    float oacc[NDT][4];
 
-    for (int mt = warp; mt < n_mt; mt += 4) {
-        if (mt != warp) {
+    for (int mt = warp / kparts; mt < n_mt; mt += 4 / kparts) {
+        const int slab = kparts > 1 ? mt : warp;
+        if (kparts == 1 && mt != warp) {
+            __syncwarp();                             // the previous tile's fragments have been read
+            stage_q(mt, slab, lane, 32);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_all;" ::: "memory");
             __syncwarp();
-            stage_q(mt);
         }
-        __syncwarp();
-        // ---- S = Q K^T over the 64 keys: 8 key tiles of 8, accumulated over HD in steps of 16 ----
+        const uint32_t qh_base = s_u32(Qs + slab * SLAB), ql_base = qh_base + 16 * ROWB;
+        // ---- S = Q K^T over this task's keys: key tiles of 8, accumulated over HD in steps of 16 ----
         float sacc[8][4];
 #pragma unroll
         for (int n = 0; n < 8; ++n)
@@ -156,97 +166,102 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const float* __restrict__
             }
 #pragma unroll
             for (int n2 = 0; n2 < 4; ++n2) {
-                const int key = n2 * 16 + (lid >> 1) * 8 + lrow, c = ks * 2 + (lid & 1);
-                uint32_t b0, b1, b2, b3;
-                ldsm4(ks_base + key * ROWB + ((c ^ (key & 7)) << 4), b0, b1, b2, b3);
-                mma16816(sacc[2 * n2], ah, b0, b1);
-                mma16816(sacc[2 * n2], al, b0, b1);
-                mma16816(sacc[2 * n2 + 1], ah, b2, b3);
-                mma16816(sacc[2 * n2 + 1], al, b2, b3);
+                if (n2 < cnt) {                       // sacc[2 * n2 ..] covers keys (kt0 + n2) * 16 ..
+                    const int key = (kt0 + n2) * 16 + (lid >> 1) * 8 + lrow, c = ks * 2 + (lid & 1);
+                    uint32_t b0, b1, b2, b3;
+                    ldsm4(ks_base + key * ROWB + ((c ^ (key & 7)) << 4), b0, b1, b2, b3);
+                    mma16816(sacc[2 * n2], ah, b0, b1);
+                    mma16816(sacc[2 * n2], al, b0, b1);
+                    mma16816(sacc[2 * n2 + 1], ah, b2, b3);
+                    mma16816(sacc[2 * n2 + 1], al, b2, b3);
+                }
             }
         }
         // ---- visibility: keys past the last one, and draft rows that are not ancestors-or-self ----
         // this thread holds rows gq and gq + 8 of the tile and, per key tile n, keys n * 8 + 2 * tq + {0, 1}
         const int qi0 = mt * 16 + gq, qi1 = qi0 + 8;
-        const uint32_t* mk0 = nullptr;
-        const uint32_t* mk1 = nullptr;
-        if (spec) {
-            if (qi0 < n_q) mk0 = rm.mask + (size_t)(bi * R + qi0 % nrows) * MTAD_MASK_WORDS;
-            if (qi1 < n_q) mk1 = rm.mask + (size_t)(bi * R + qi1 % nrows) * MTAD_MASK_WORDS;
-        }
-        if (spec || k_begin + KT > nkeys) {
+        const int kfirst = k_begin + kt0 * 16;
+        if (kfirst + cnt * 16 > min(L, nkeys)) {
+            const uint32_t* mk0 = (spec && qi0 < n_q) ? rm.mask + (size_t)(bi * R + qi0 % nrows) * MTAD_MASK_WORDS : nullptr;
+            const uint32_t* mk1 = (spec && qi1 < n_q) ? rm.mask + (size_t)(bi * R + qi1 % nrows) * MTAD_MASK_WORDS : nullptr;
 #pragma unroll
             for (int n = 0; n < 8; ++n)
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
-                    const int j = k_begin + n * 8 + 2 * tq + c;
-                    bool v0 = j < nkeys, v1 = j < nkeys;
-                    if (j >= L && j < nkeys) {
-                        const int sr = j - L;
-                        v0 = mk0 && ((mk0[sr >> 5] >> (sr & 31)) & 1u);
-                        v1 = mk1 && ((mk1[sr >> 5] >> (sr & 31)) & 1u);
+                    if (n < 2 * cnt) {
+                        const int j = kfirst + n * 8 + 2 * tq + c;
+                        bool v0 = j < nkeys, v1 = v0;
+                        if (v0 && j >= L) {
+                            const int sr = j - L;
+                            v0 = mk0 && ((mk0[sr >> 5] >> (sr & 31)) & 1u);
+                            v1 = mk1 && ((mk1[sr >> 5] >> (sr & 31)) & 1u);
+                        }
+                        if (!v0) sacc[n][c] = -CUDART_INF_F;
+                        if (!v1) sacc[n][2 + c] = -CUDART_INF_F;
                     }
-                    if (!v0) sacc[n][c] = -CUDART_INF_F;
-                    if (!v1) sacc[n][2 + c] = -CUDART_INF_F;
                 }
         }
-        // ---- softmax numerators over this split ----
-        float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;
+        // ---- softmax numerators over this task's keys ----
+        m0 = -CUDART_INF_F; m1 = -CUDART_INF_F;
 #pragma unroll
-        for (int n = 0; n < 8; ++n) {
-            m0 = fmaxf(m0, fmaxf(sacc[n][0], sacc[n][1]));
-            m1 = fmaxf(m1, fmaxf(sacc[n][2], sacc[n][3]));
-        }
+        for (int n = 0; n < 8; ++n)
+            if (n < 2 * cnt) {
+                m0 = fmaxf(m0, fmaxf(sacc[n][0], sacc[n][1]));
+                m1 = fmaxf(m1, fmaxf(sacc[n][2], sacc[n][3]));
+            }
         m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1));
         m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
         m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1));
         m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
-        float l0 = 0.f, l1 = 0.f;
+        l0 = 0.f; l1 = 0.f;
+        const float s0 = (m0 == -CUDART_INF_F) ? 0.f : m0, s1 = (m1 == -CUDART_INF_F) ? 0.f : m1;
 #pragma unroll
-        for (int n = 0; n < 8; ++n) {
+        for (int n = 0; n < 8; ++n)
+            if (n < 2 * cnt) {
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                const float p0 = (m0 == -CUDART_INF_F) ? 0.f : expf(sacc[n][c] - m0);
-                const float p1 = (m1 == -CUDART_INF_F) ? 0.f : expf(sacc[n][2 + c] - m1);
-                sacc[n][c] = p0;
-                sacc[n][2 + c] = p1;
-                l0 += p0;
-                l1 += p1;
+                for (int c = 0; c < 2; ++c) {
+                    const float p0 = exp2f(sacc[n][c] - s0), p1 = exp2f(sacc[n][2 + c] - s1);   // exp2(-inf) = 0
+                    sacc[n][c] = p0;
+                    sacc[n][2 + c] = p1;
+                    l0 += p0;
+                    l1 += p1;
+                }
             }
-        }
         l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
         l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
         l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
         l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
         // ---- O = P V: P (hi + lo) straight from the score fragments, V through transposing ldmatrix ----
-        float oacc[NDT][4];
 #pragma unroll
         for (int n = 0; n < NDT; ++n)
 #pragma unroll
             for (int c = 0; c < 4; ++c) oacc[n][c] = 0.f;
 #pragma unroll
         for (int kk = 0; kk < KT / 16; ++kk) {
-            uint32_t ph[4], pl[4];
-            split2(sacc[2 * kk][0], sacc[2 * kk][1], ph[0], pl[0]);
-            split2(sacc[2 * kk][2], sacc[2 * kk][3], ph[1], pl[1]);
-            split2(sacc[2 * kk + 1][0], sacc[2 * kk + 1][1], ph[2], pl[2]);
-            split2(sacc[2 * kk + 1][2], sacc[2 * kk + 1][3], ph[3], pl[3]);
+            if (kk < cnt) {
+                uint32_t ph[4], pl[4];
+                split2(sacc[2 * kk][0], sacc[2 * kk][1], ph[0], pl[0]);
+                split2(sacc[2 * kk][2], sacc[2 * kk][3], ph[1], pl[1]);
+                split2(sacc[2 * kk + 1][0], sacc[2 * kk + 1][1], ph[2], pl[2]);
+                split2(sacc[2 * kk + 1][2], sacc[2 * kk + 1][3], ph[3], pl[3]);
 #pragma unroll
-            for (int d2 = 0; d2 < HD / 16; ++d2) {
-                const int key = kk * 16 + (lid & 1) * 8 + lrow, c = d2 * 2 + (lid >> 1);
-                uint32_t b0, b1, b2, b3;
-                ldsm4t(vs_base + key * ROWB + ((c ^ (key & 7)) << 4), b0, b1, b2, b3);
-                mma16816(oacc[2 * d2], ph, b0, b1);
-                mma16816(oacc[2 * d2], pl, b0, b1);
-                mma16816(oacc[2 * d2 + 1], ph, b2, b3);
-                mma16816(oacc[2 * d2 + 1], pl, b2, b3);
+                for (int d2 = 0; d2 < HD / 16; ++d2) {
+                    const int key = (kt0 + kk) * 16 + (lid & 1) * 8 + lrow, c = d2 * 2 + (lid >> 1);
+                    uint32_t b0, b1, b2, b3;
+                    ldsm4t(vs_base + key * ROWB + ((c ^ (key & 7)) << 4), b0, b1, b2, b3);
+                    mma16816(oacc[2 * d2], ph, b0, b1);
+                    mma16816(oacc[2 * d2], pl, b0, b1);
+                    mma16816(oacc[2 * d2 + 1], ph, b2, b3);
+                    mma16816(oacc[2 * d2 + 1], pl, b2, b3);
+                }
             }
         }
+        if (kparts > 1) break;                        // one task per warp: merged below
         // ---- partials of the valid rows ----
         if (qi0 < n_q) {
             const int h = g * G + qi0 / nrows, r = qi0 % nrows;
             float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
-            if (tq == 0) { dst[0] = m0; dst[1] = l0; }
+            if (tq == 0) { dst[0] = m0 * LN2; dst[1] = l0; }
 #pragma unroll
             for (int n = 0; n < NDT; ++n)
                 *reinterpret_cast<float2*>(dst + 2 + n * 8 + 2 * tq) = make_float2(oacc[n][0], oacc[n][1]);
@@ -254,10 +269,45 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const float* __restrict__
         if (qi1 < n_q) {
             const int h = g * G + qi1 / nrows, r = qi1 % nrows;
             float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
-            if (tq == 0) { dst[0] = m1; dst[1] = l1; }
+            if (tq == 0) { dst[0] = m1 * LN2; dst[1] = l1; }
 #pragma unroll
             for (int n = 0; n < NDT; ++n)
                 *reinterpret_cast<float2*>(dst + 2 + n * 8 + 2 * tq) = make_float2(oacc[n][2], oacc[n][3]);
+        }
+    }
+    if (kparts > 1) {
+        // ---- key-split tiles: park each warp's (m, l, o) over the K/V/Q area, then merge the parts in key order --
+        __syncthreads();                              // every warp is done reading K, V and the query tiles
+        float* ow = reinterpret_cast<float*>(smem) + warp * 16 * PARK;
+        if (tq == 0) {
+            ml[(warp * 16 + gq) * 2] = m0;     ml[(warp * 16 + gq) * 2 + 1] = l0;
+            ml[(warp * 16 + gq + 8) * 2] = m1; ml[(warp * 16 + gq + 8) * 2 + 1] = l1;
+        }
+#pragma unroll
+        for (int n = 0; n < NDT; ++n) {
+            *reinterpret_cast<float2*>(ow + gq * PARK + n * 8 + 2 * tq) = make_float2(oacc[n][0], oacc[n][1]);
+            *reinterpret_cast<float2*>(ow + (gq + 8) * PARK + n * 8 + 2 * tq) = make_float2(oacc[n][2], oacc[n][3]);
+        }
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < n_mt * 16 * HD; idx += blockDim.x) {
+            const int mtile = idx / (16 * HD), row = (idx / HD) % 16, d = idx % HD;
+            const int qi = mtile * 16 + row;
+            if (qi >= n_q) continue;
+            const int w0 = mtile * kparts;
+            float M = -CUDART_INF_F;
+            for (int q = 0; q < kparts; ++q) M = fmaxf(M, ml[((w0 + q) * 16 + row) * 2]);
+            float acc = 0.f, lsum = 0.f;
+            for (int q = 0; q < kparts; ++q) {
+                const float mq = ml[((w0 + q) * 16 + row) * 2];
+                if (mq == -CUDART_INF_F) continue;
+                const float wgt = exp2f(mq - M);
+                lsum += ml[((w0 + q) * 16 + row) * 2 + 1] * wgt;
+                acc += (reinterpret_cast<const float*>(smem) + (w0 + q) * 16 * PARK)[row * PARK + d] * wgt;
+            }
+            const int h = g * G + qi / nrows, r = qi % nrows;
+            float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
+            dst[2 + d] = acc;
+            if (d == 0) { dst[0] = M * LN2; dst[1] = lsum; }
         }
     }
 }
@@ -265,25 +315,27 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const float* __restrict__
 cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int B, int R,
                                  int nsplit, bool pdl, cudaStream_t st) {
     const int Hq = m.d.n_q_heads, Hkv = m.d.n_kv_heads, hd = m.d.head_dim;
-    const int ldq = (Hq + 2 * Hkv) * hd;
     const __nv_bfloat16* cache = static_cast<const __nv_bfloat16*>(m.d.kv_cache);
     dim3 grid(nsplit, Hkv, B);
+    // query tiles kept in shared memory: all of them (at most two) when the warps split keys, else one per warp
+    const int n_mt_max = ((Hq / Hkv) * R + 15) / 16;
+    const int nslab = n_mt_max <= 2 ? n_mt_max : 4;
+    const size_t smem = (size_t)2 * KT * hd * 2 + (size_t)nslab * 2 * 16 * hd * 2 + 512;
     if (hd == 128) {
-        const size_t smem = 2 * KT * 256 + 4 * 2 * 16 * 256;       // K, V and one query slab per warp
         static bool set128 = false;
         if (!set128) {
             cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 98304);
             if (e != cudaSuccess) return e;
             set128 = true;
         }
-        return launch_pdl(attn_mma_kernel<128>, grid, dim3(128), smem, st, pdl, (const float*)sc.qkv, ldq, cache, rm,
-                          sc.attn_part, layer, m.max_batch, Hq, Hkv, (long long)m.d.kv_capacity, R, nsplit);
+        return launch_pdl(attn_mma_kernel<128>, grid, dim3(128), smem, st, pdl, (const __nv_bfloat16*)sc.q_hi,
+                          (const __nv_bfloat16*)sc.q_lo, cache, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv,
+                          (long long)m.d.kv_capacity, R, nsplit, nslab);
     }
-    if (hd == 64) {
-        const size_t smem = 2 * KT * 128 + 4 * 2 * 16 * 128;
-        return launch_pdl(attn_mma_kernel<64>, grid, dim3(128), smem, st, pdl, (const float*)sc.qkv, ldq, cache, rm,
-                          sc.attn_part, layer, m.max_batch, Hq, Hkv, (long long)m.d.kv_capacity, R, nsplit);
-    }
+    if (hd == 64)
+        return launch_pdl(attn_mma_kernel<64>, grid, dim3(128), smem, st, pdl, (const __nv_bfloat16*)sc.q_hi,
+                          (const __nv_bfloat16*)sc.q_lo, cache, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv,
+                          (long long)m.d.kv_capacity, R, nsplit, nslab);
     return cudaErrorInvalidValue;
 }
 

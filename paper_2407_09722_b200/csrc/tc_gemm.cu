@@ -210,6 +210,12 @@ __device__ __forceinline__ void epi_qkv(const TcGemmParams& p, EpiTile epi, int 
                 float* q = p.q_out + (size_t)t * ldq + head * hd;
                 q[jin] = ra * scale;
                 q[jin + half] = rb * scale;
+                if (p.q_hi) {
+                    // tensor-core attention operands: q * log2(e) / sqrt(hd) as bf16 hi + lo (softmax runs on exp2)
+                    const size_t o = (size_t)t * p.Hq * hd + head * hd;
+                    split_store(ra * scale * 1.4426950408889634f, p.q_hi + o + jin, p.q_lo + o + jin);
+                    split_store(rb * scale * 1.4426950408889634f, p.q_hi + o + jin + half, p.q_lo + o + jin + half);
+                }
             } else {
                 const int sl = p.slot[t];
                 if (sl < 0) continue;

@@ -47,6 +47,7 @@ struct TcGemmParams {
     int seg_k_tile, seg_v_tile;     // first tile of the K rows and of the V rows
     int Hq, Hkv, hd;
     float* q_out;                   // [T, (Hq + 2 Hkv) hd], q part written
+    __nv_bfloat16 *q_hi, *q_lo;     // [T, Hq hd] each, or null: q * log2(e) / sqrt(hd) split for the MMA attention
     const float* rope;              // [T, hd/2, 2]
     __nv_bfloat16* cache;
     const int32_t* slot;
