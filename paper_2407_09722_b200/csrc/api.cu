@@ -318,8 +318,9 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             RUN(MTAD_K_GEMM, wb * (qd + 2.0 * kvd) * d.d_model, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
         }
         if (d.head_dim == 64 || d.head_dim == 128) {
-            const int ns = (int)((total + 63) / 64);
-            RUN(MTAD_K_ATTN, 0, 2, launch_attention_mma(m, l, ctx->rm, sc, B, R, ns, pdl, s));
+            const int nsp = attention_mma_tiles_per_block(m, B, R, total);
+            const int ns = (int)(((total + 63) / 64 + nsp - 1) / nsp);
+            RUN(MTAD_K_ATTN, 0, 2, launch_attention_mma(m, l, ctx->rm, sc, B, R, ns, nsp, pdl, s));
             RUN(MTAD_K_ATTN, 0, 0, launch_attention_combine(m, ctx->rm, sc, B, R, ns, true, pdl, s));
         } else {
             RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, true, pdl, s));

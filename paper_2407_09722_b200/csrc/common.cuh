@@ -128,8 +128,9 @@ cudaError_t launch_rope_append(const ModelView& m, int layer, const RowMeta& rm,
 cudaError_t launch_attention(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int B, int R,
                              int nsplit, int chunk, bool emit_split, bool pdl, cudaStream_t st);
 // tensor-core partial pass (one split per 64 keys) and the combine pass on its own
+int attention_mma_tiles_per_block(const ModelView& m, int B, int R, long long keys);
 cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int B, int R,
-                                 int nsplit, bool pdl, cudaStream_t st);
+                                 int nsplit, int nsp, bool pdl, cudaStream_t st);
 cudaError_t launch_attention_combine(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int nsplit,
                                      bool emit_split, bool pdl, cudaStream_t st);
 cudaError_t launch_lm_merge(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int n_tiles,

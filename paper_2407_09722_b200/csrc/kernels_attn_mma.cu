@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
                                                           const __nv_bfloat16* __restrict__ q_lo,
                                                           const __nv_bfloat16* __restrict__ cache, RowMeta rm,
                                                           float* __restrict__ part, int layer, int max_batch, int Hq,
-                                                          int Hkv, long long cap, int R, int nsplit, int nslab) {
+                                                          int Hkv, long long cap, int R, int nsplit, int nslab, int nsp) {
     constexpr int ROWB = HD * 2;          // bytes of one key row
     constexpr int CPR = HD / 8;           // 16-byte pieces per row
     constexpr int NDT = HD / 8;           // 8-wide output tiles over the head dim
@@ -66,9 +66,8 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
     constexpr int PARK = HD + 8;          // row stride (floats) of a parked output tile
     constexpr float LN2 = 0.6931471805599453f;
     extern __shared__ __align__(128) uint8_t smem[];
-    uint8_t* Ks = smem;                               // [KT][HD] bf16, piece c of row k stored at piece c ^ (k & 7)
-    uint8_t* Vs = smem + KT * ROWB;
-    uint8_t* Qs = smem + 2 * KT * ROWB;               // nslab query tiles, same swizzle
+    // two K/V buffers of [KT][HD] bf16 each (piece c of row k stored at piece c ^ (k & 7)), then the query tiles
+    uint8_t* Qs = smem + 4 * KT * ROWB;               // nslab query tiles, same swizzle
     float* ml = reinterpret_cast<float*>(Qs + nslab * SLAB);           // [4 warps][16 rows][m, l]
 
     const int sp = blockIdx.x, g = blockIdx.y, bi = blockIdx.z;
@@ -79,10 +78,11 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
     if (nrows == 0) return;
     const int L = rm.kv_base[bi];
     const int nkeys = L + nrows;
-    const int k_begin = sp * KT;
+    const int n_tiles = (nkeys + KT - 1) / KT;        // 64-key tiles of this sequence
+    const int tile_begin = sp * nsp, tile_end = min(tile_begin + nsp, n_tiles);
     const int G = Hq / Hkv;
     const int n_q = G * nrows;                        // query rows of this KV head: (head in group, draft row)
-    if (k_begin >= nkeys) {
+    if (tile_begin >= n_tiles) {
         // empty split: leave neutral partials so that the combine pass can read every split
         for (int i = threadIdx.x; i < n_q; i += blockDim.x) {
             const int h = g * G + i / nrows, r = i % nrows;
@@ -114,30 +114,51 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
             cp_async16(s_u32(dst + which * 16 * ROWB + row * ROWB + ((c ^ (row & 7)) << 4)), src, valid);
         }
     };
+    // K and V rows of one 64-key tile -> buffer `buf` (zero-filled past the last key)
+    auto load_kv = [&](int tile, int buf) {
+        const int kb = tile * KT;
+        uint8_t* Kd = smem + buf * (2 * KT * ROWB);
+        uint8_t* Vd = Kd + KT * ROWB;
+        for (int i = threadIdx.x; i < KT * CPR; i += blockDim.x) {
+            const int key = i / CPR, c = i % CPR;
+            const bool valid = kb + key < nkeys;
+            const size_t goff = (size_t)(valid ? kb + key : 0) * HD + c * 8;
+            const uint32_t soff = key * ROWB + ((c ^ (key & 7)) << 4);
+            cp_async16(s_u32(Kd + soff), Kg + goff, valid);
+            cp_async16(s_u32(Vd + soff), Vg + goff, valid);
+        }
+    };
     if (kparts > 1) {
         for (int mt = 0; mt < n_mt; ++mt) stage_q(mt, mt, threadIdx.x, blockDim.x);
     } else if (warp < n_mt) {
         stage_q(warp, warp, lane, 32);
     }
-    // ---- K and V rows of this split -> shared memory (zero-filled past the last key) ----
-    for (int i = threadIdx.x; i < KT * CPR; i += blockDim.x) {
-        const int key = i / CPR, c = i % CPR;
-        const bool valid = k_begin + key < nkeys;
-        const size_t goff = (size_t)(valid ? k_begin + key : 0) * HD + c * 8;
-        const uint32_t soff = key * ROWB + ((c ^ (key & 7)) << 4);
-        cp_async16(s_u32(Ks + soff), Kg + goff, valid);
-        cp_async16(s_u32(Vs + soff), Vg + goff, valid);
-    }
+    load_kv(tile_begin, 0);
     asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_all;" ::: "memory");
-    __syncthreads();
 
     const int gq = lane >> 2, tq = lane & 3;          // fragment coordinates
-    const bool spec = k_begin + KT > L;               // the split reaches into the draft rows: masks apply
-    const uint32_t ks_base = s_u32(Ks), vs_base = s_u32(Vs);
     const int lrow = lane & 7, lid = lane >> 3;       // ldmatrix: row within an 8x8 matrix, matrix id
+    // running softmax state of this thread's two rows (gq and gq + 8), in log2 units
     float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, l0 = 0.f, l1 = 0.f;
     float oacc[NDT][4];
+#pragma unroll
+    for (int n = 0; n < NDT; ++n)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) oacc[n][c] = 0.f;
+
+  for (int tile = tile_begin; tile < tile_end; ++tile) {
+    const int buf = (tile - tile_begin) & 1;
+    if (tile + 1 < tile_end) {                        // prefetch the next tile while this one is computed
+        load_kv(tile + 1, buf ^ 1);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();
+    const int k_begin = tile * KT;
+    const bool spec = k_begin + KT > L;               // the tile reaches into the draft rows: masks apply
+    const uint32_t ks_base = s_u32(smem + buf * (2 * KT * ROWB)), vs_base = ks_base + KT * ROWB;
 
     for (int mt = warp / kparts; mt < n_mt; mt += 4 / kparts) {
         const int slab = kparts > 1 ? mt : warp;
@@ -147,6 +168,13 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
             asm volatile("cp.async.commit_group;" ::: "memory");
             asm volatile("cp.async.wait_all;" ::: "memory");
             __syncwarp();
+        }
+        if (kparts == 1) {                            // whole tiles: one key tile per block, fresh state per query tile
+            m0 = -CUDART_INF_F; m1 = -CUDART_INF_F; l0 = 0.f; l1 = 0.f;
+#pragma unroll
+            for (int n = 0; n < NDT; ++n)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) oacc[n][c] = 0.f;
         }
         const uint32_t qh_base = s_u32(Qs + slab * SLAB), ql_base = qh_base + 16 * ROWB;
         // ---- S = Q K^T over this task's keys: key tiles of 8, accumulated over HD in steps of 16 ----
@@ -201,20 +229,23 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
                     }
                 }
         }
-        // ---- softmax numerators over this task's keys ----
-        m0 = -CUDART_INF_F; m1 = -CUDART_INF_F;
+        // ---- online softmax over this task's keys: new maximum, rescale the running sums, numerators ----
+        float t0 = -CUDART_INF_F, t1 = -CUDART_INF_F;
 #pragma unroll
         for (int n = 0; n < 8; ++n)
             if (n < 2 * cnt) {
-                m0 = fmaxf(m0, fmaxf(sacc[n][0], sacc[n][1]));
-                m1 = fmaxf(m1, fmaxf(sacc[n][2], sacc[n][3]));
+                t0 = fmaxf(t0, fmaxf(sacc[n][0], sacc[n][1]));
+                t1 = fmaxf(t1, fmaxf(sacc[n][2], sacc[n][3]));
             }
-        m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1));
-        m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
-        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1));
-        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
-        l0 = 0.f; l1 = 0.f;
-        const float s0 = (m0 == -CUDART_INF_F) ? 0.f : m0, s1 = (m1 == -CUDART_INF_F) ? 0.f : m1;
+        t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, 1));
+        t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, 2));
+        t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, 1));
+        t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, 2));
+        const float n0 = fmaxf(m0, t0), n1 = fmaxf(m1, t1);
+        const float c0 = (n0 == -CUDART_INF_F) ? 1.f : exp2f(m0 - n0), c1 = (n1 == -CUDART_INF_F) ? 1.f : exp2f(m1 - n1);
+        const float s0 = (n0 == -CUDART_INF_F) ? 0.f : n0, s1 = (n1 == -CUDART_INF_F) ? 0.f : n1;
+        m0 = n0; m1 = n1;
+        float r0 = 0.f, r1 = 0.f;
 #pragma unroll
         for (int n = 0; n < 8; ++n)
             if (n < 2 * cnt) {
@@ -223,19 +254,22 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
                     const float p0 = exp2f(sacc[n][c] - s0), p1 = exp2f(sacc[n][2 + c] - s1);   // exp2(-inf) = 0
                     sacc[n][c] = p0;
                     sacc[n][2 + c] = p1;
-                    l0 += p0;
-                    l1 += p1;
+                    r0 += p0;
+                    r1 += p1;
                 }
             }
-        l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-        l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-        l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-        l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-        // ---- O = P V: P (hi + lo) straight from the score fragments, V through transposing ldmatrix ----
+        r0 += __shfl_xor_sync(0xffffffffu, r0, 1);
+        r0 += __shfl_xor_sync(0xffffffffu, r0, 2);
+        r1 += __shfl_xor_sync(0xffffffffu, r1, 1);
+        r1 += __shfl_xor_sync(0xffffffffu, r1, 2);
+        l0 = l0 * c0 + r0;
+        l1 = l1 * c1 + r1;
 #pragma unroll
-        for (int n = 0; n < NDT; ++n)
-#pragma unroll
-            for (int c = 0; c < 4; ++c) oacc[n][c] = 0.f;
+        for (int n = 0; n < NDT; ++n) {
+            oacc[n][0] *= c0; oacc[n][1] *= c0;
+            oacc[n][2] *= c1; oacc[n][3] *= c1;
+        }
+        // ---- O += P V: P (hi + lo) straight from the score fragments, V through transposing ldmatrix ----
 #pragma unroll
         for (int kk = 0; kk < KT / 16; ++kk) {
             if (kk < cnt) {
@@ -275,9 +309,10 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
                 *reinterpret_cast<float2*>(dst + 2 + n * 8 + 2 * tq) = make_float2(oacc[n][2], oacc[n][3]);
         }
     }
+    __syncthreads();                                  // this tile's buffer may be refilled two iterations on
+  }
     if (kparts > 1) {
         // ---- key-split tiles: park each warp's (m, l, o) over the K/V/Q area, then merge the parts in key order --
-        __syncthreads();                              // every warp is done reading K, V and the query tiles
         float* ow = reinterpret_cast<float*>(smem) + warp * 16 * PARK;
         if (tq == 0) {
             ml[(warp * 16 + gq) * 2] = m0;     ml[(warp * 16 + gq) * 2 + 1] = l0;
@@ -312,30 +347,41 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
     }
 }
 
+int attention_mma_tiles_per_block(const ModelView& m, int B, int R, long long keys) {
+    // with at most two query tiles per KV head a block walks several 64-key tiles (next tile prefetched while the
+    // current one is computed): about three blocks per SM in a single wave; larger trees take one tile per block
+    const int n_mt_max = ((m.d.n_q_heads / m.d.n_kv_heads) * R + 15) / 16;
+    if (n_mt_max > 2) return 1;
+    const long long tiles = (keys + KT - 1) / KT * m.d.n_kv_heads * B;
+    const long long nsp = (tiles + 3 * 148 - 1) / (3 * 148);
+    return (int)(nsp < 1 ? 1 : (nsp > 64 ? 64 : nsp));
+}
+
 cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int B, int R,
-                                 int nsplit, bool pdl, cudaStream_t st) {
+                                 int nsplit, int nsp, bool pdl, cudaStream_t st) {
     const int Hq = m.d.n_q_heads, Hkv = m.d.n_kv_heads, hd = m.d.head_dim;
     const __nv_bfloat16* cache = static_cast<const __nv_bfloat16*>(m.d.kv_cache);
-    dim3 grid(nsplit, Hkv, B);
     // query tiles kept in shared memory: all of them (at most two) when the warps split keys, else one per warp
     const int n_mt_max = ((Hq / Hkv) * R + 15) / 16;
     const int nslab = n_mt_max <= 2 ? n_mt_max : 4;
-    const size_t smem = (size_t)2 * KT * hd * 2 + (size_t)nslab * 2 * 16 * hd * 2 + 512;
-    if (hd == 128) {
-        static bool set128 = false;
-        if (!set128) {
-            cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 98304);
-            if (e != cudaSuccess) return e;
-            set128 = true;
-        }
+    const size_t smem = (size_t)4 * KT * hd * 2 + (size_t)nslab * 2 * 16 * hd * 2 + 512;
+    dim3 grid(nsplit, Hkv, B);
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 102400);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 102400);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    if (hd == 128)
         return launch_pdl(attn_mma_kernel<128>, grid, dim3(128), smem, st, pdl, (const __nv_bfloat16*)sc.q_hi,
                           (const __nv_bfloat16*)sc.q_lo, cache, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv,
-                          (long long)m.d.kv_capacity, R, nsplit, nslab);
-    }
+                          (long long)m.d.kv_capacity, R, nsplit, nslab, nsp);
     if (hd == 64)
         return launch_pdl(attn_mma_kernel<64>, grid, dim3(128), smem, st, pdl, (const __nv_bfloat16*)sc.q_hi,
                           (const __nv_bfloat16*)sc.q_lo, cache, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv,
-                          (long long)m.d.kv_capacity, R, nsplit, nslab);
+                          (long long)m.d.kv_capacity, R, nsplit, nslab, nsp);
     return cudaErrorInvalidValue;
 }
 
