@@ -317,7 +317,8 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             mp.a0 = wm.wq[ix(mq)][l]; mp.a1 = wm.wk[ix(mq)][l]; mp.a2 = wm.wv[ix(mq)][l]; mp.x = xd;
             RUN(MTAD_K_GEMM, wb * (qd + 2.0 * kvd) * d.d_model, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
         }
-        if (d.head_dim == 64 || d.head_dim == 128) {
+        static const bool mma_attn = !(getenv("MTAD_TC_ATTN") && atoi(getenv("MTAD_TC_ATTN")) == 0);
+        if (mma_attn && (d.head_dim == 64 || d.head_dim == 128)) {
             const int nsp = attention_mma_tiles_per_block(m, B, R, total);
             const int ns = (int)(((total + 63) / 64 + nsp - 1) / nsp);
             RUN(MTAD_K_ATTN, 0, 2, launch_attention_mma(m, l, ctx->rm, sc, B, R, ns, nsp, pdl, s));
