@@ -367,13 +367,19 @@ class DraftResult:
     logq: List[float]           # joint log q of the path ending at each node
     best_path: List[int]        # node ids of x** (the final beam with the highest draft likelihood)
     logq_ref: List[float]       # log q(x**_{1:i})
+    min_gap: float = float("inf")   # smallest gap between neighbouring perturbed scores among the b kept and the
+                                    # first one dropped, over all steps (how close any pick was to a tie)
 
 
-def gumbel_top_b(scores: np.ndarray, u: np.ndarray, b: int) -> List[int]:
+def gumbel_top_b(scores: np.ndarray, u: np.ndarray, b: int, with_gap: bool = False):
     """Sample b distinct flat indices without replacement, successive draws proportional to exp(scores):
     the b largest of scores + Gumbel noise, in decreasing order (lowest index first on ties)."""
     y = np.asarray(scores, dtype=np.float64).ravel() - np.log(-np.log(np.asarray(u, dtype=np.float64).ravel()))
     order = sorted(range(y.size), key=lambda i: (-y[i], i))
+    if with_gap:
+        top = [y[i] for i in order[:b + 1]]
+        gap = min((top[k] - top[k + 1] for k in range(len(top) - 1)), default=float("inf"))
+        return order[:b], float(gap)
     return order[:b]
 
 
@@ -402,9 +408,11 @@ def draft_beam(model: OracleModel, cache: np.ndarray, L: int, pending_tok: Seque
     beam_logp = log_softmax(logits[P - 1:P])       # [n_beams, V]
     root_vis = vis[P - 1]
     node_vis = {-1: root_vis}
+    min_gap = float("inf")
     for step in range(gamma):
         scores = beam_logq[:, None] + beam_logp    # joint log-likelihood of every (beam, token) pair
-        picks = gumbel_top_b(scores, u[step, :len(beams), :], b)
+        picks, gap = gumbel_top_b(scores, u[step, :len(beams), :], b, with_gap=True)
+        min_gap = min(min_gap, gap)
         V = scores.shape[1]
         new_nodes = []
         for flat in picks:
@@ -427,4 +435,22 @@ def draft_beam(model: OracleModel, cache: np.ndarray, L: int, pending_tok: Seque
         path.append(n)
         n = parent[n]
     path.reverse()
-    return DraftResult(tok, parent, depth, logq, path, [logq[n] for n in path])
+    return DraftResult(tok, parent, depth, logq, path, [logq[n] for n in path], min_gap)
+
+
+def aux_commit(cache: np.ndarray, L: int, pending_tok: Sequence[int], draft: DraftResult, accepted: Sequence[int],
+               bonus_tok: int, gamma: int):
+    """Roll the auxiliary cache forward after a verification: the pending rows (slots L ..) are already in place;
+    accepted draft node accepted[i] (tree id, depth i + 1, slot L + P + id) moves to position L + P + i if the draft
+    ran it (depth < gamma).  A node of the last layer was never run by the auxiliary model: it stays pending, ahead
+    of the new root.  Returns (new committed length, new pending tokens ending with the new root)."""
+    P = len(pending_tok)
+    base = L + P
+    kept = [n for n in accepted if draft.depth[n] < gamma]
+    for i, n in enumerate(kept):
+        src, dst = base + n, base + i
+        assert src >= dst
+        if src != dst:
+            cache[:, :, :, dst, :] = cache[:, :, :, src, :]
+    pend = [draft.tok[n] for n in accepted if draft.depth[n] >= gamma] + [bonus_tok]
+    return base + len(kept), pend

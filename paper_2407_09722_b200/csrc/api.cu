@@ -32,6 +32,12 @@ struct mtad_ctx {
     RowMeta rm{};
     Scratch sc{};
     std::vector<long long> len_ub;      // host upper bound of each sequence's committed length
+    std::vector<int> npend_ub;          // host upper bound of each sequence's auxiliary pending count
+    DraftState ds{};
+    bool draft_active = false;          // the last mtad_draft's tree has not been committed yet
+    int draft_B = 0, draft_gamma = 0;
+    int32_t draft_seqs[MTAD_MAX_BATCH];
+    bool last_chain = false;            // the last verify call was mtad_verify_chain
     int last_B = 0, last_R = 0, last_D = 0;
     int32_t last_seqs[MTAD_MAX_BATCH];
     int last_cuda = 0;
@@ -111,6 +117,7 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     rm.depth = k.take<int32_t>(T);
     rm.mask = k.take<uint32_t>(T * MTAD_MASK_WORDS);
     rm.n_rows = k.take<int32_t>(max_batch);
+    rm.n_spec = k.take<int32_t>(max_batch);
     rm.kv_base = k.take<int32_t>(max_batch);
     rm.call_seq = k.take<int32_t>(max_batch);
     Scratch sc;
@@ -165,7 +172,18 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     sc.tc_counters = k.take<int32_t>(max_tiles);
     sc.lm_part = k.take<float4>(Tc * lm_tiles);
     sc.node_z = k.take<float>(T);
+    DraftState ds;
+    ds.base_len = k.take<int32_t>(max_batch);
+    ds.npend = k.take<int32_t>(max_batch);
+    ds.gamma = k.take<int32_t>(max_batch);
+    ds.beam = k.take<int32_t>(max_batch);
+    ds.node_tok = k.take<int32_t>((size_t)max_batch * MTAD_DRAFT_NODES);
+    ds.node_parent = k.take<int32_t>((size_t)max_batch * MTAD_DRAFT_NODES);
+    ds.node_logq = k.take<float>((size_t)max_batch * MTAD_DRAFT_NODES);
+    ds.node_mask = k.take<uint32_t>((size_t)max_batch * MTAD_DRAFT_NODES * MTAD_MASK_WORDS);
+    ds.best_path = k.take<int32_t>((size_t)max_batch * MTAD_MAX_DEPTH);
     if (c) {
+        c->ds = ds;
         c->st = st; c->rm = rm; c->sc = sc;
         c->tc_ws_floats = ws_tiles * rpad * TC_TILE_N;
         c->tc_counter_n = max_tiles;
@@ -273,7 +291,7 @@ bool build_weight_maps(const ModelView& m, WeightMaps& w) {
 // epilogue; activations travel between launches as bf16 hi/lo operand rows plus per-row sums of squares, so the
 // RMSNorm is applied as a per-row scale in the consumer's epilogue.  Leaves lm_part / node_z for launch_lm_merge.
 int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int B, int R, long long len_ub,
-                    const float* uniforms, uint32_t* status, cudaStream_t s) {
+                    const float* uniforms, uint32_t* status, bool lm_plain, cudaStream_t s) {
     const int T = B * R;
     const mtad_model_desc& d = m.d;
     const int qd = d.n_q_heads * d.head_dim, kvd = d.n_kv_heads * d.head_dim;
@@ -360,10 +378,11 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
         TcGemmParams p = base; TcMaps mp{};
         tc_decompose(p, up(d.vocab, 128 * mh), d.d_model, T, kCtas);
         p.mh = mh; p.n_rows_total = d.vocab; p.n_tiles128 = up(d.vocab, 128);
-        p.mode = TC_LMHEAD; p.N = d.vocab; p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = dt;
+        p.mode = lm_plain ? TC_PLAIN : TC_LMHEAD; p.N = d.vocab; p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = dt;
+        p.out = sc.logits; p.ldo = d.vocab;                 // draft steps keep the logits for the beam selection
         mp.a0 = wm.lm_head[ix(mh)]; mp.x = xd;
         RUN(MTAD_K_GEMM, wb * d.vocab * d.d_model, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
-        RUN(MTAD_K_LMRED, 0, 2, launch_lm_merge(m, ctx->rm, sc, B, R, p.n_tiles128, uniforms, s));
+        if (!lm_plain) RUN(MTAD_K_LMRED, 0, 2, launch_lm_merge(m, ctx->rm, sc, B, R, p.n_tiles128, uniforms, s));
     }
     return MTAD_OK;
 }
@@ -408,7 +427,7 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
     }
     RUN(MTAD_K_PREPARE, 0, 1, launch_prepare(ctx->target, ctx->st, ctx->rm, ctx->sc, pa, out->status, s));
     if (tc) {
-        int rc = forward_rows_tc(ctx, ctx->target, ctx->tmaps, B, R, ub, bonus_uniform, out->status, s);
+        int rc = forward_rows_tc(ctx, ctx->target, ctx->tmaps, B, R, ub, bonus_uniform, out->status, false, s);
         if (rc != MTAD_OK) return rc;
     } else {
         int rc = forward_rows(ctx, ctx->target, B, R, ub, s);
@@ -419,6 +438,7 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
     AcceptArgs aa{B, R, D, tok, parent, logq_ref, log_tau};
     RUN(MTAD_K_ACCEPT, 0, 1, launch_accept(ctx->rm, ctx->sc, aa, *out, s));
     ctx->last_B = B; ctx->last_R = R; ctx->last_D = D;
+    ctx->last_chain = (parent == nullptr);
     memcpy(ctx->last_seqs, seqs, sizeof(int32_t) * B);
     return MTAD_OK;
 }
@@ -460,6 +480,7 @@ int mtad_create(const mtad_model_desc* target, const mtad_model_desc* aux, int m
     ctx->max_nodes = max_nodes;
     ctx->T_max = max_batch * (max_nodes + 1);
     ctx->len_ub.assign(max_batch, 0);
+    ctx->npend_ub.assign(max_batch, 1);
     carve(ctx, target, aux, max_batch, max_nodes, workspace);
     // tensor-core path unless MTAD_PATH=simt asks for the CUDA-core kernels (or a weight pointer is not 16-byte aligned)
     const char* path = getenv("MTAD_PATH");
@@ -548,6 +569,7 @@ int mtad_seq_set(mtad_ctx* ctx, int seq, int32_t kv_len, int32_t root_token, int
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     RUN(MTAD_K_PREPARE, 0, 1, launch_seq_set(ctx->st, seq, kv_len, root_token, aux_len, npend, pending_tok, s));
     ctx->len_ub[seq] = kv_len;
+    ctx->npend_ub[seq] = npend + 1;
     return MTAD_OK;
 }
 
@@ -567,9 +589,45 @@ int mtad_seq_get(mtad_ctx* ctx, int seq, int32_t* kv_len, int32_t* root_token, v
 int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_width, const float* uniforms,
                int32_t* tok, int32_t* parent, int32_t* depth, float* node_logq, float* logq_ref,
                int32_t* best_path, void* stream) {
-    (void)ctx; (void)B; (void)seqs; (void)gamma; (void)beam_width; (void)uniforms; (void)tok; (void)parent;
-    (void)depth; (void)node_logq; (void)logq_ref; (void)best_path; (void)stream;
-    return MTAD_E_UNIMPLEMENTED;
+    if (!ctx) return MTAD_E_INVALID;
+    if (!ctx->has_aux) return MTAD_E_INVALID;
+    if (!seqs_ok(ctx, B, seqs)) return MTAD_E_INVALID;
+    if (!uniforms || !tok || !parent || !depth || !node_logq || !logq_ref || !best_path) return MTAD_E_INVALID;
+    if (gamma < 1 || beam_width < 1) return MTAD_E_INVALID;
+    if (gamma > MTAD_MAX_DEPTH || beam_width > MTAD_MAX_BEAM || gamma * beam_width > MTAD_DRAFT_NODES - MTAD_MAX_DEPTH - 1 ||
+        gamma * beam_width > MTAD_MAX_NODES)
+        return MTAD_E_CAPACITY;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const ModelView& m = ctx->aux;
+    int R0 = 1;
+    long long ub = 0;
+    for (int i = 0; i < B; ++i) {
+        R0 = std::max(R0, ctx->npend_ub[seqs[i]]);
+        ub = std::max(ub, ctx->len_ub[seqs[i]]);
+    }
+    if (std::max(R0, beam_width) > ctx->max_nodes + 1) return MTAD_E_CAPACITY;    // rows of one step exceed the workspace
+    if (ub + 1 + (long long)gamma * beam_width > m.d.kv_capacity) return MTAD_E_CAPACITY;
+    SeqList sl{};
+    for (int i = 0; i < B; ++i) sl.v[i] = seqs[i];
+    DraftOut out{tok, parent, depth, node_logq, logq_ref, best_path};
+    const bool tc = ctx->use_tc && ctx->amaps.ok;
+    for (int step = 0; step < gamma; ++step) {
+        const int R = step == 0 ? R0 : beam_width;
+        RUN(MTAD_K_PREPARE, 0, 1, launch_draft_prepare(m, ctx->st, ctx->ds, ctx->rm, ctx->sc, sl, B, R, step, beam_width,
+                                                       tc && B * R <= TC_MAX_ROWS, s));
+        // keys of the auxiliary cache: committed ones, the pending rows and every node drafted so far
+        const long long keys_ub = ub + 1 + (long long)step * beam_width;
+        int rc;
+        if (tc && B * R <= TC_MAX_ROWS) rc = forward_rows_tc(ctx, m, ctx->amaps, B, R, keys_ub, nullptr, nullptr, true, s);
+        else rc = forward_rows(ctx, m, B, R, keys_ub, s);
+        if (rc != MTAD_OK) return rc;
+        RUN(MTAD_K_LMRED, 0, 1, launch_draft_select(m, ctx->ds, ctx->sc, sl, B, R, step, gamma, beam_width, uniforms, out, s));
+    }
+    ctx->draft_active = true;
+    ctx->draft_B = B;
+    ctx->draft_gamma = gamma;
+    memcpy(ctx->draft_seqs, seqs, sizeof(int32_t) * B);
+    return MTAD_OK;
 }
 
 int mtad_verify_chain(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, const int32_t* draft_tok,
@@ -593,6 +651,17 @@ int kv_commit(mtad_ctx* ctx, int B, const int32_t* seqs, const mtad_result* res,
     if (!seqs_ok(ctx, B, seqs)) return MTAD_E_INVALID;
     if (B != ctx->last_B || memcmp(seqs, ctx->last_seqs, sizeof(int32_t) * B) != 0) return MTAD_E_INVALID;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (ctx->has_aux) {
+        // auxiliary cache: after a draft its accepted rows are kept; otherwise the accepted tokens wait for replay
+        const bool after_draft = ctx->draft_active && ctx->draft_B == B &&
+                                 memcmp(seqs, ctx->draft_seqs, sizeof(int32_t) * B) == 0;
+        const int mode = after_draft ? (ctx->last_chain ? 0 : 1) : 2;
+        RUN(MTAD_K_COMMIT, 0, 2,
+            launch_aux_commit(ctx->aux, ctx->st, ctx->ds, B, ctx->rm.call_seq, *res, ctx->last_D, mode, s));
+        for (int i = 0; i < B; ++i)
+            ctx->npend_ub[seqs[i]] = after_draft ? 2 : std::min(ctx->npend_ub[seqs[i]] + ctx->last_D + 1, MTAD_MAX_DEPTH + 1);
+        ctx->draft_active = false;
+    }
     RUN(MTAD_K_COMMIT, 0, 1, launch_kv_commit(ctx->target, ctx->st, B, ctx->rm.call_seq, *res, ctx->last_D, s));
     RUN(MTAD_K_COMMIT, 0, 1, launch_seq_advance(ctx->st, B, ctx->rm.call_seq, *res, ctx->last_D, s));
     for (int i = 0; i < B; ++i)

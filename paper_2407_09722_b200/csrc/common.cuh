@@ -24,6 +24,7 @@ struct RowMeta {
     int32_t* depth;      // [T]
     uint32_t* mask;      // [T][MTAD_MASK_WORDS] visible rows of the same sequence (ancestors and self)
     int32_t* n_rows;     // [B] active rows of sequence bi (n_nodes + 1, 0 if the sequence is rejected)
+    int32_t* n_spec;     // [B] cache slots past L that hold draft rows (this call's and, in the draft, earlier steps')
     int32_t* kv_base;    // [B] committed length L seen by this call
     int32_t* call_seq;   // [B] sequence ids of the call
     int32_t* prow;       // [T] global row of a node row's parent, -1 for roots and inactive rows
@@ -44,6 +45,28 @@ struct SeqState {        // device arrays, [max_batch]
     int32_t* aux_len;
     int32_t* aux_npend;
     int32_t* aux_pend;   // [max_batch][MTAD_MAX_DEPTH + 1]
+};
+
+#define MTAD_DRAFT_NODES 256       // nodes of one draft tree kept per sequence
+
+// State of the last draft of every sequence (device arrays indexed by sequence id), kept for the cache roll-forward.
+struct DraftState {
+    int32_t* base_len;     // [max_batch] auxiliary committed length when the draft started
+    int32_t* npend;        // [max_batch] pending tokens replayed by that draft
+    int32_t* gamma;        // [max_batch]
+    int32_t* beam;         // [max_batch]
+    int32_t* node_tok;     // [max_batch][MTAD_DRAFT_NODES]
+    int32_t* node_parent;  // [max_batch][MTAD_DRAFT_NODES]
+    float* node_logq;      // [max_batch][MTAD_DRAFT_NODES]
+    uint32_t* node_mask;   // [max_batch][MTAD_DRAFT_NODES][MTAD_MASK_WORDS] visible virtual rows of each node
+    int32_t* best_path;    // [max_batch][MTAD_MAX_DEPTH]
+};
+
+struct DraftOut {          // caller's device arrays of mtad_draft
+    int32_t *tok, *parent, *depth;
+    float* node_logq;
+    float* logq_ref;
+    int32_t* best_path;
 };
 
 struct Scratch {
@@ -151,6 +174,15 @@ cudaError_t launch_kv_commit(const ModelView& m, const SeqState& s, int B, const
                              const mtad_result& res, int max_depth, cudaStream_t st);
 cudaError_t launch_seq_advance(const SeqState& s, int B, const int32_t* call_seq_dev, const mtad_result& res,
                                int max_depth, cudaStream_t st);
+cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const DraftState& ds, const RowMeta& rm,
+                                 const Scratch& sc, const SeqList& seqs, int B, int R, int step, int beam, bool tc,
+                                 cudaStream_t st);
+cudaError_t launch_draft_select(const ModelView& m, const DraftState& ds, const Scratch& sc, const SeqList& seqs, int B,
+                                int R, int step, int gamma, int beam, const float* uniforms, const DraftOut& out,
+                                cudaStream_t st);
+cudaError_t launch_aux_commit(const ModelView& aux, const SeqState& s, const DraftState& ds, int B,
+                              const int32_t* call_seq_dev, const mtad_result& res, int max_depth, int mode,
+                              cudaStream_t st);
 cudaError_t launch_seq_set(const SeqState& s, int seq, int kv_len, int root, int aux_len, int npend,
                            const int32_t* pend_host, cudaStream_t st);
 

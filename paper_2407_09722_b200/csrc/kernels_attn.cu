@@ -28,7 +28,7 @@ __global__ void __launch_bounds__(128) attn_partial_kernel(const float* __restri
     if (nrows == 0) return;
     const int seq = rm.call_seq[bi];
     const int L = rm.kv_base[bi];
-    const int nkeys = L + nrows;
+    const int nkeys = L + rm.n_spec[bi];
     const int c0 = sp * chunk;
     const int c1 = min(c0 + chunk, nkeys);
     const int g = h / (Hq / Hkv);

@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
     const int nrows = rm.n_rows[bi];
     if (nrows == 0) return;
     const int L = rm.kv_base[bi];
-    const int nkeys = L + nrows;
+    const int nkeys = L + rm.n_spec[bi];
     const int n_tiles = (nkeys + KT - 1) / KT;        // 64-key tiles of this sequence
     const int tile_begin = sp * nsp, tile_end = min(tile_begin + nsp, n_tiles);
     const int G = Hq / Hkv;

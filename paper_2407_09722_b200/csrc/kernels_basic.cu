@@ -56,9 +56,11 @@ __global__ void seq_set_kernel(SeqState s, int seq, int kv_len, int root, int au
 
 cudaError_t launch_seq_set(const SeqState& s, int seq, int kv_len, int root, int aux_len, int npend,
                            const int32_t* pend_host, cudaStream_t st) {
+    // pending list of the auxiliary model: the committed tokens it has not seen yet, then the root
     PendTok p;
     for (int i = 0; i <= MTAD_MAX_DEPTH; ++i) p.v[i] = (i < npend && pend_host) ? pend_host[i] : 0;
-    seq_set_kernel<<<1, 64, 0, st>>>(s, seq, kv_len, root, aux_len, npend, p);
+    p.v[npend] = root;
+    seq_set_kernel<<<1, 64, 0, st>>>(s, seq, kv_len, root, aux_len, npend + 1, p);
     return cudaGetLastError();
 }
 
@@ -122,6 +124,7 @@ __global__ void prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, i
         rm.prow[t] = pr;
         if (r == 0) {
             rm.n_rows[bi] = seq_ok ? nn + 1 : 0;
+            rm.n_spec[bi] = seq_ok ? nn + 1 : 0;
             rm.kv_base[bi] = L;
             rm.call_seq[bi] = seq;
         }

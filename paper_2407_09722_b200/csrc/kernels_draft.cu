@@ -1,0 +1,349 @@
+// Beam-sampling draft with the auxiliary model (Sec. 2.1 of the paper, the p_beam equation; every intermediate
+// beam becomes a node of the candidate tree, Sec. 3.3): row bookkeeping of each draft step, the Gumbel-top-b
+// selection over (beam, token) pairs, and the roll-forward of the auxiliary KV cache after a verification.
+//
+// Virtual rows of one draft: the P pending tokens (not yet in the auxiliary cache, the last one is the root) are
+// rows 0 .. P-1, node n is row P + n; row v lives in cache slot aux_len + v.
+#include <math_constants.h>
+
+#include "common.cuh"
+
+namespace mtad {
+
+namespace {
+
+__device__ __forceinline__ float wsum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float wmax(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+struct Cand {
+    float y;      // perturbed joint score
+    int flat;     // beam * V + token
+};
+__device__ __forceinline__ bool before(const Cand& a, const Cand& b) {     // a ranks ahead of b
+    return a.y > b.y || (a.y == b.y && a.flat < b.flat);
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------------------------
+// rows of one draft step: step 0 runs the pending tokens as a causal chain, step s >= 1 the nodes of layer s
+// ---------------------------------------------------------------------------------------------------------------
+
+__global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, int vocab, int hd,
+                                     double rope_base, SeqState s, DraftState ds, RowMeta rm,
+                                     float* __restrict__ hidden, float* __restrict__ rope, SeqList seqs, int R, int step,
+                                     int beam, const __nv_bfloat16* __restrict__ gain0, __nv_bfloat16* x_hi,
+                                     __nv_bfloat16* x_lo, float* sumsq_out) {
+    const int t = blockIdx.x, bi = t / R, r = t % R;
+    const int seq = seqs.v[bi];
+    __shared__ int sh_tok, sh_pos, sh_ok;
+    if (threadIdx.x == 0) {
+        const int L = step == 0 ? s.aux_len[seq] : ds.base_len[seq];
+        const int P = step == 0 ? s.aux_npend[seq] : ds.npend[seq];
+        if (step == 0 && r == 0) { ds.base_len[seq] = L; ds.npend[seq] = P; }
+        uint32_t mask[MTAD_MASK_WORDS];
+#pragma unroll
+        for (int i = 0; i < MTAD_MASK_WORDS; ++i) mask[i] = 0;
+        int tok = 0, pos = L, vrow = 0;
+        bool active;
+        if (step == 0) {
+            active = r < P;
+            if (active) {
+                tok = s.aux_pend[seq * (MTAD_MAX_DEPTH + 1) + r];
+                vrow = r;
+                pos = L + r;
+                for (int i = 0; i <= r; ++i) mask[i >> 5] |= 1u << (i & 31);        // causal over the pending rows
+            }
+        } else {
+            active = r < beam;
+            if (active) {
+                const int n = (step - 1) * beam + r;
+                tok = ds.node_tok[seq * MTAD_DRAFT_NODES + n];
+                vrow = P + n;
+                pos = L + P - 1 + step;
+#pragma unroll
+                for (int i = 0; i < MTAD_MASK_WORDS; ++i)
+                    mask[i] = ds.node_mask[((size_t)seq * MTAD_DRAFT_NODES + n) * MTAD_MASK_WORDS + i];
+            }
+        }
+        if (tok < 0 || tok >= vocab) tok = 0;
+        rm.tok[t] = tok;
+        rm.depth[t] = step;
+        rm.pos[t] = pos;
+        rm.slot[t] = active ? L + vrow : -1;
+        rm.seq[t] = seq;
+        rm.prow[t] = -1;
+        // the mask is indexed by cache slot minus L: virtual rows
+#pragma unroll
+        for (int i = 0; i < MTAD_MASK_WORDS; ++i) rm.mask[(size_t)t * MTAD_MASK_WORDS + i] = mask[i];
+        if (r == 0) {
+            rm.n_rows[bi] = step == 0 ? P : beam;
+            rm.n_spec[bi] = step == 0 ? P : P + step * beam;
+            rm.kv_base[bi] = L;
+            rm.call_seq[bi] = seq;
+        }
+        sh_tok = tok;
+        sh_pos = pos;
+        sh_ok = active;
+    }
+    __syncthreads();
+    const int tok = sh_tok;
+    const bool ok = sh_ok;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        const float v = ok ? __bfloat162float(embed[(size_t)tok * d + i]) : 0.f;
+        hidden[(size_t)t * d + i] = v;
+        if (x_hi) {
+            const float y = v * __bfloat162float(gain0[i]);
+            const __nv_bfloat16 h = __float2bfloat16_rn(y);
+            x_hi[(size_t)t * 2 * d + i] = h;
+            x_lo[(size_t)t * 2 * d + i] = __float2bfloat16_rn(y - __bfloat162float(h));
+            ss += v * v;
+        }
+    }
+    if (x_hi) {
+        __shared__ float red[32];
+        ss = wsum(ss);
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float a = 0.f;
+            for (int w = 0; w < (int)(blockDim.x >> 5); ++w) a += red[w];
+            sumsq_out[t] = a;
+        }
+    }
+    for (int i = threadIdx.x; i < hd / 2; i += blockDim.x) {
+        const double inv = exp2(-(2.0 * i / hd) * log2(rope_base));
+        double sn, cs;
+        sincos((double)sh_pos * inv, &sn, &cs);
+        rope[((size_t)t * (hd / 2) + i) * 2 + 0] = (float)cs;
+        rope[((size_t)t * (hd / 2) + i) * 2 + 1] = (float)sn;
+    }
+}
+
+cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const DraftState& ds, const RowMeta& rm,
+                                 const Scratch& sc, const SeqList& seqs, int B, int R, int step, int beam, bool tc,
+                                 cudaStream_t st) {
+    draft_prepare_kernel<<<B * R, 128, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(m.d.embed), m.d.d_model, m.d.vocab, m.d.head_dim, (double)m.d.rope_base, s, ds,
+        rm, sc.hidden, sc.rope, seqs, R, step, beam, tc ? m.w(0, 0) : nullptr, tc ? sc.xd_hi : nullptr,
+        tc ? sc.xd_hi + m.d.d_model : nullptr, sc.sumsq_a);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// selection: the `beam` largest of log q(beam) + log q(token | beam) + Gumbel noise over all (beam, token) pairs
+// ---------------------------------------------------------------------------------------------------------------
+
+__global__ void __launch_bounds__(1024) draft_select_kernel(const float* __restrict__ logits, int V, int R, int step,
+                                                            int gamma, int beam, const float* __restrict__ uni,
+                                                            DraftState ds, SeqList seqs, DraftOut out) {
+    const int bi = blockIdx.x, seq = seqs.v[bi];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int P = ds.npend[seq];
+    const int n_beams = step == 0 ? 1 : beam;
+    const int N = gamma * beam;
+    __shared__ float s_red[32];
+    __shared__ float s_lse[MTAD_MAX_BEAM], s_lq[MTAD_MAX_BEAM];
+    __shared__ int s_node[MTAD_MAX_BEAM];
+    __shared__ Cand s_c[1024];
+    // log-sum-exp of every beam's row
+    for (int j = 0; j < n_beams; ++j) {
+        const int row = step == 0 ? P - 1 : j;
+        const float* z = logits + (size_t)(bi * R + row) * V;
+        float m = -CUDART_INF_F;
+        for (int v = tid; v < V; v += blockDim.x) m = fmaxf(m, z[v]);
+        m = wmax(m);
+        if (lane == 0) s_red[warp] = m;
+        __syncthreads();
+        m = s_red[0];
+        for (int w = 1; w < 32; ++w) m = fmaxf(m, s_red[w]);
+        __syncthreads();
+        float sum = 0.f;
+        for (int v = tid; v < V; v += blockDim.x) sum += expf(z[v] - m);
+        sum = wsum(sum);
+        if (lane == 0) s_red[warp] = sum;
+        __syncthreads();
+        if (tid == 0) {
+            float a = 0.f;
+            for (int w = 0; w < 32; ++w) a += s_red[w];           // fixed order
+            s_lse[j] = m + logf(a);
+            const int node = step == 0 ? -1 : (step - 1) * beam + j;
+            s_node[j] = node;
+            s_lq[j] = node < 0 ? 0.f : ds.node_logq[seq * MTAD_DRAFT_NODES + node];
+        }
+        __syncthreads();
+    }
+    // every thread keeps the best `beam` of its share of the (beam, token) pairs, sorted
+    Cand loc[MTAD_MAX_BEAM];
+#pragma unroll
+    for (int k = 0; k < MTAD_MAX_BEAM; ++k) loc[k] = Cand{-CUDART_INF_F, 0x7fffffff};
+    const float* ub = uni + ((size_t)bi * gamma + step) * beam * V;
+    for (int j = 0; j < n_beams; ++j) {
+        const int row = step == 0 ? P - 1 : j;
+        const float* z = logits + (size_t)(bi * R + row) * V;
+        const float add = s_lq[j] - s_lse[j];
+        for (int v = tid; v < V; v += blockDim.x) {
+            Cand c{add + z[v] - logf(-logf(ub[(size_t)j * V + v])), j * V + v};
+            if (before(c, loc[MTAD_MAX_BEAM - 1])) {
+                loc[MTAD_MAX_BEAM - 1] = c;
+#pragma unroll
+                for (int k = MTAD_MAX_BEAM - 1; k > 0; --k)
+                    if (before(loc[k], loc[k - 1])) { const Cand tmp = loc[k]; loc[k] = loc[k - 1]; loc[k - 1] = tmp; }
+            }
+        }
+    }
+    // `beam` rounds: the block's best head-of-list wins, its owner advances
+    int head = 0;
+    for (int k = 0; k < beam; ++k) {
+        Cand c = head < MTAD_MAX_BEAM ? loc[head] : Cand{-CUDART_INF_F, 0x7fffffff};
+        // pick among the 1024 heads
+        s_c[tid] = c;
+        __syncthreads();
+        for (int o = 512; o > 0; o >>= 1) {
+            if (tid < o && before(s_c[tid + o], s_c[tid])) s_c[tid] = s_c[tid + o];
+            __syncthreads();
+        }
+        const Cand win = s_c[0];
+        __syncthreads();
+        if (c.flat == win.flat && c.y == win.y) ++head;      // the owner of the winner (flat indices are unique)
+        if (tid == 0) {
+            const int j = win.flat / V, v = win.flat % V;
+            const int n = step * beam + k;
+            const int row = step == 0 ? P - 1 : j;
+            const float lq = s_lq[j] + logits[(size_t)(bi * R + row) * V + v] - s_lse[j];
+            const int parent = s_node[j];
+            ds.node_tok[seq * MTAD_DRAFT_NODES + n] = v;
+            ds.node_parent[seq * MTAD_DRAFT_NODES + n] = parent;
+            ds.node_logq[seq * MTAD_DRAFT_NODES + n] = lq;
+            uint32_t* mk = ds.node_mask + ((size_t)seq * MTAD_DRAFT_NODES + n) * MTAD_MASK_WORDS;
+            for (int i = 0; i < MTAD_MASK_WORDS; ++i) {
+                uint32_t w;
+                if (parent >= 0) w = ds.node_mask[((size_t)seq * MTAD_DRAFT_NODES + parent) * MTAD_MASK_WORDS + i];
+                else {                                        // child of the root: sees all pending rows
+                    const int lo = i * 32;
+                    w = P >= lo + 32 ? 0xffffffffu : (P > lo ? (1u << (P - lo)) - 1u : 0u);
+                }
+                if (((P + n) >> 5) == i) w |= 1u << ((P + n) & 31);
+                mk[i] = w;
+            }
+            out.tok[bi * N + n] = v;
+            out.parent[bi * N + n] = parent;
+            out.depth[bi * N + n] = step + 1;
+            out.node_logq[bi * N + n] = lq;
+        }
+        __syncthreads();
+    }
+    if (step == gamma - 1 && tid == 0) {
+        // x**: the final beam with the highest draft likelihood (lowest node id on ties), and its prefix likelihoods
+        int best = (gamma - 1) * beam;
+        for (int k = 1; k < beam; ++k) {
+            const int n = (gamma - 1) * beam + k;
+            if (ds.node_logq[seq * MTAD_DRAFT_NODES + n] > ds.node_logq[seq * MTAD_DRAFT_NODES + best]) best = n;
+        }
+        int cur = best;
+        for (int i = gamma - 1; i >= 0 && cur >= 0; --i) {
+            out.best_path[bi * gamma + i] = cur;
+            out.logq_ref[bi * gamma + i] = ds.node_logq[seq * MTAD_DRAFT_NODES + cur];
+            ds.best_path[seq * MTAD_MAX_DEPTH + i] = cur;
+            cur = ds.node_parent[seq * MTAD_DRAFT_NODES + cur];
+        }
+        ds.gamma[seq] = gamma;
+        ds.beam[seq] = beam;
+    }
+}
+
+cudaError_t launch_draft_select(const ModelView& m, const DraftState& ds, const Scratch& sc, const SeqList& seqs, int B,
+                                int R, int step, int gamma, int beam, const float* uniforms, const DraftOut& out,
+                                cudaStream_t st) {
+    draft_select_kernel<<<B, 1024, 0, st>>>(sc.logits, m.d.vocab, R, step, gamma, beam, uniforms, ds, seqs, out);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// auxiliary cache roll-forward after a verification
+// ---------------------------------------------------------------------------------------------------------------
+
+// mode 0: the verified chain was the draft's output sequence (chain node i = draft node best_path[i]);
+// mode 1: the verified tree was the draft's tree (same node ids).  Accepted node i (depth i + 1, slot base + id)
+// moves to position base + i when the draft ran it (depth < gamma).
+__global__ void aux_commit_kernel(__nv_bfloat16* __restrict__ cache, const int32_t* __restrict__ call_seq,
+                                  DraftState ds, mtad_result res, int D, int mode, int max_batch, int Hkv, int hd,
+                                  long long cap) {
+    const int bi = blockIdx.y;
+    if (res.status[bi] != 0) return;
+    const int seq = call_seq[bi];
+    const int gamma = ds.gamma[seq];
+    const int eta = res.eta[bi];
+    const int kept = min(eta, gamma - 1);
+    if (kept <= 0) return;
+    const int base = ds.base_len[seq] + ds.npend[seq];
+    const int head = blockIdx.x % Hkv;
+    const int kv = (blockIdx.x / Hkv) & 1;
+    const int layer = blockIdx.x / (2 * Hkv);
+    __nv_bfloat16* b = cache + (((((size_t)layer * max_batch + seq) * 2 + kv) * Hkv + head) * cap) * hd;
+    extern __shared__ __nv_bfloat16 buf[];
+    for (int i = threadIdx.x; i < kept * hd; i += blockDim.x) {
+        const int r = i / hd, j = i % hd;
+        const int pn = res.path[bi * D + r];
+        const int node = mode == 0 ? ds.best_path[seq * MTAD_MAX_DEPTH + pn] : pn;
+        buf[i] = b[(size_t)(base + node) * hd + j];
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kept * hd; i += blockDim.x) {
+        const int r = i / hd, j = i % hd;
+        b[(size_t)(base + r) * hd + j] = buf[i];
+    }
+}
+
+// New auxiliary state.  mode 0 / 1: after a draft (see above); mode 2: no draft produced the verified rows, the
+// accepted tokens and the new root simply join the pending list (to be replayed by the next draft).
+__global__ void aux_advance_kernel(SeqState s, DraftState ds, const int32_t* __restrict__ call_seq, mtad_result res,
+                                   int D, int mode, int B) {
+    const int bi = blockIdx.x * blockDim.x + threadIdx.x;
+    if (bi >= B || res.status[bi] != 0) return;
+    const int seq = call_seq[bi];
+    const int eta = res.eta[bi];
+    int32_t* pend = s.aux_pend + seq * (MTAD_MAX_DEPTH + 1);
+    const int bonus = res.out_tok[bi * (D + 1) + eta];
+    if (mode == 2) {
+        int np = s.aux_npend[seq];
+        if (np + eta + 1 > MTAD_MAX_DEPTH + 1) { atomicOr(&res.status[bi], MTAD_ST_AUX_PENDING); return; }
+        for (int i = 0; i <= eta; ++i) pend[np + i] = res.out_tok[bi * (D + 1) + i];
+        s.aux_npend[seq] = np + eta + 1;
+        return;
+    }
+    const int gamma = ds.gamma[seq];
+    const int kept = min(eta, gamma - 1);
+    s.aux_len[seq] = ds.base_len[seq] + ds.npend[seq] + kept;
+    int np = 0;
+    if (eta >= gamma) pend[np++] = res.out_tok[bi * (D + 1) + eta - 1];   // last layer's node: never run by the aux model
+    pend[np++] = bonus;
+    s.aux_npend[seq] = np;
+}
+
+cudaError_t launch_aux_commit(const ModelView& aux, const SeqState& s, const DraftState& ds, int B,
+                              const int32_t* call_seq_dev, const mtad_result& res, int max_depth, int mode,
+                              cudaStream_t st) {
+    if (mode != 2) {
+        dim3 grid(aux.d.layers * 2 * aux.d.n_kv_heads, B);
+        const size_t smem = (size_t)(max_depth > 0 ? max_depth : 1) * aux.d.head_dim * sizeof(__nv_bfloat16);
+        aux_commit_kernel<<<grid, 128, smem, st>>>(static_cast<__nv_bfloat16*>(aux.d.kv_cache), call_seq_dev, ds, res,
+                                                   max_depth, mode, aux.max_batch, aux.d.n_kv_heads, aux.d.head_dim,
+                                                   (long long)aux.d.kv_capacity);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    aux_advance_kernel<<<1, 64, 0, st>>>(s, ds, call_seq_dev, res, max_depth, mode, B);
+    return cudaGetLastError();
+}
+
+}  // namespace mtad

@@ -35,6 +35,21 @@ class GpuModel(DeviceModel):
                 layer_maker=lambda l: w["layers"][l])
         return self._oracle
 
+    def oracle_aux(self) -> O.OracleModel:
+        if getattr(self, "_oracle_aux", None) is None:
+            self._oracle_aux = oracle_model(self.aux_weights)
+        return self._oracle_aux
+
+    def inject_aux(self, seq: int, length: int):
+        S.fill_kv_cache(self.aux_cache, 1, seq, length, self.seed)
+
+    def aux_cache_bits(self, seq: int, upto: int) -> np.ndarray:
+        s = self.aux_shape
+        cap = self.aux_cache.shape[4]
+        out = np.zeros((s.layers, 2, s.n_kv_heads, cap, s.head_dim), np.uint16)
+        out[:, :, :, :upto] = bits(self.aux_cache[:, seq, :, :, :upto].contiguous())
+        return out
+
     def cache_bits(self, seq: int, upto: int) -> np.ndarray:
         """Host copy of one sequence's cache [layers, 2, Hkv, capacity, hd] as bf16 bits (only [0, upto) filled)."""
         out = np.zeros((self.shape.layers, 2, self.shape.n_kv_heads, self.capacity, self.shape.head_dim), np.uint16)

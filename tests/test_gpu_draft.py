@@ -1,0 +1,102 @@
+"""mtad_draft (beam sampling with the auxiliary model) and the auxiliary cache roll-forward against the oracle's
+draft_beam / aux_commit, through whole draft -> verify -> commit iterations."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import mtad_synth as S
+import paper_2407_09722_b200 as M
+from oracle import mtad_oracle as O
+from tests.parity import GpuModel, LP_TOL
+
+pytestmark = pytest.mark.gpu
+W = S.WORKLOADS["tiny"]
+
+
+def _draft_gpu(gm, seq, gamma, b, u):
+    N = gamma * b
+    i32 = dict(dtype=torch.int32, device="cuda")
+    f32 = dict(dtype=torch.float32, device="cuda")
+    out = {"tok": torch.zeros(1, N, **i32), "parent": torch.zeros(1, N, **i32), "depth": torch.zeros(1, N, **i32),
+           "node_logq": torch.zeros(1, N, **f32), "logq_ref": torch.zeros(1, gamma, **f32),
+           "best_path": torch.zeros(1, gamma, **i32)}
+    gm.ctx.mtad_draft([seq], gamma, b, u, out["tok"], out["parent"], out["depth"], out["node_logq"], out["logq_ref"],
+                      out["best_path"])
+    torch.cuda.synchronize()
+    return out
+
+
+@pytest.mark.parametrize("gamma,b,chain", [(4, 4, False), (3, 2, True), (4, 1, True), (2, 8, False)])
+def test_draft_verify_commit_iterations(gamma, b, chain):
+    gm = GpuModel(W.target, max_batch=2, max_nodes=40, capacity=256, aux=W.aux, aux_capacity=256)
+    seq, L = 1, 24
+    gm.inject(seq, L)
+    gm.inject_aux(seq, L)
+    root = 5
+    gm.ctx.mtad_seq_set(seq, L, root, aux_len=L)
+    tcache = gm.cache_bits(seq, L)
+    acache = gm.aux_cache_bits(seq, L)
+    La, pend = L, [root]
+    V = W.target.vocab
+    skipped = 0
+    for it in range(6):
+        u = S.uniforms(0, (31 << 40) | (it * 16 + gamma), gamma * b * V, "cuda").view(1, gamma, b, V)
+        g = _draft_gpu(gm, seq, gamma, b, u)
+        dr = O.draft_beam(gm.oracle_aux(), acache, La, pend, gamma, b, u[0].cpu().numpy())
+        near = dr.min_gap < 1e-3
+        if not near:
+            assert g["tok"][0].tolist() == dr.tok and g["parent"][0].tolist() == dr.parent
+            assert g["depth"][0].tolist() == dr.depth and g["best_path"][0].tolist() == dr.best_path
+            assert np.max(np.abs(g["node_logq"][0].cpu().numpy() - np.asarray(dr.logq))) < LP_TOL
+            assert np.max(np.abs(g["logq_ref"][0].cpu().numpy() - np.asarray(dr.logq_ref))) < LP_TOL
+        else:
+            skipped += 1
+        # verify what the oracle drafted (teacher forcing keeps both sides on one trajectory)
+        bu = S.bonus_uniforms(9, it, 1, V, "cuda")
+        log_tau = math.log(0.3)
+        ref = np.asarray(dr.logq_ref, np.float32)
+        if chain:
+            toks = [dr.tok[n] for n in dr.best_path]
+            res = M.ResultBuffers(1, gamma, gamma)
+            gm.ctx.mtad_verify_chain([seq], gamma, torch.tensor(toks, dtype=torch.int32, device="cuda"),
+                                     torch.tensor(ref, device="cuda"), log_tau, bu, res)
+            r = O.verify_chain(gm.oracle(), tcache, L, root, toks, ref.astype(np.float64), log_tau, bu[0].cpu().numpy())
+            accepted = [dr.best_path[i] for i in r.path]
+        else:
+            res = M.ResultBuffers(1, gamma * b, gamma)
+            gm.ctx.mtad_verify_tree([seq], None, gamma * b, gamma, torch.tensor(dr.tok, dtype=torch.int32, device="cuda"),
+                                    torch.tensor(dr.parent, dtype=torch.int32, device="cuda"),
+                                    torch.tensor(ref, device="cuda"), log_tau, bu, res)
+            r = O.verify_tree(gm.oracle(), tcache, L, root, dr.tok, dr.parent, ref.astype(np.float64), log_tau,
+                              bu[0].cpu().numpy())
+            accepted = list(r.path)
+        gm.ctx.kv_commit([seq], res)
+        h = res.host()
+        assert int(h["status"][0]) == 0
+        tie = min(r.margin_accept, r.margin_tie, r.margin_bonus) < 1e-3
+        if near or tie:
+            pytest.skip("near tie on the trajectory")          # vanishingly rare with these seeds
+        assert int(h["eta"][0]) == r.eta and h["out_tok"][0, :r.eta + 1].tolist() == r.out_tok
+        L = O.kv_commit(tcache, L, r.path)
+        La, pend = O.aux_commit(acache, La, pend, dr, accepted, r.out_tok[-1], gamma)
+        root = r.out_tok[-1]
+        assert gm.ctx.mtad_seq_get(seq) == (L, root)
+    assert skipped == 0
+
+
+def test_draft_rejects_bad_arguments():
+    gm = GpuModel(W.target, max_batch=1, max_nodes=40, capacity=128, aux=W.aux, aux_capacity=128)
+    V = W.target.vocab
+    u = torch.full((1, 4, 4, V), 0.5, device="cuda")
+    i32 = dict(dtype=torch.int32, device="cuda")
+    t = torch.zeros(1, 64, **i32)
+    f = torch.zeros(1, 64, device="cuda")
+    c = gm.ctx
+    assert c.mtad_draft([0], 0, 4, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_INVALID
+    assert c.mtad_draft([0], 4, 9, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_CAPACITY
+    assert c.mtad_draft([0], 33, 1, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_CAPACITY
+    assert c.mtad_draft([3], 4, 4, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_INVALID
+    no_aux = GpuModel(W.target, max_batch=1, max_nodes=8, capacity=64)
+    assert no_aux.ctx.mtad_draft([0], 4, 4, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_INVALID

@@ -304,3 +304,34 @@ def test_draft_beam_bookkeeping():
         lg = O.decoder_rows(model, c3, pos, [cur], [pos], [pos], [[pos]])[0]
         cur, _ = O.gumbel_argmax(lg, u[step, 0]); pos += 1
         assert cur == d1.tok[step]
+
+
+def test_aux_commit_equals_rerunning_the_accepted_tokens():
+    """After a draft and the roll-forward of the auxiliary cache, the next draft step must see exactly what causal
+    decoding of the committed tokens would have produced, whether or not the last drafted layer was accepted."""
+    from oracle.adapters import oracle_model
+    shape = S.WORKLOADS["tiny"].aux
+    model = oracle_model(S.make_model(shape, 1))
+    gamma, b, cap = 3, 3, 64
+    for accept_len in (0, 2, 3):
+        cache = np.zeros((shape.layers, 2, shape.n_kv_heads, cap, shape.head_dim), dtype=np.uint16)
+        ctx = S.token_ids(0, 41, 6, shape.vocab).tolist()
+        for i, t in enumerate(ctx[:-1]):
+            O.decoder_rows(model, cache, i, [t], [i], [i], [[i]])
+        L, pend = len(ctx) - 1, [ctx[-1]]
+        u = S.uniforms(0, 42 + accept_len, gamma * b * shape.vocab).view(gamma, b, shape.vocab).numpy()
+        dr = O.draft_beam(model, cache, L, pend, gamma, b, u)
+        accepted = dr.best_path[:accept_len]
+        bonus = 77
+        L2, pend2 = O.aux_commit(cache, L, pend, dr, accepted, bonus, gamma)
+        committed = ctx + [dr.tok[n] for n in accepted] + [bonus]
+        assert L2 + len(pend2) == len(committed) and pend2[-1] == bonus
+        assert committed[L2:] == pend2
+        # next step through the rolled-forward cache vs from scratch
+        vis = [[L2 + i for i in range(r + 1)] for r in range(len(pend2))]
+        got = O.decoder_rows(model, cache, L2, pend2, [L2 + i for i in range(len(pend2))],
+                             [L2 + i for i in range(len(pend2))], vis)[-1]
+        c2 = np.zeros_like(cache)
+        for i, t in enumerate(committed):
+            ref = O.decoder_rows(model, c2, i, [t], [i], [i], [[i]])[0]
+        assert np.max(np.abs(ref - got)) < 1e-10
