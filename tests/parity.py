@@ -50,6 +50,15 @@ class GpuModel(DeviceModel):
         out[:, :, :, :upto] = bits(self.aux_cache[:, seq, :, :, :upto].contiguous())
         return out
 
+    def upload(self, seq: int, target_bits: np.ndarray = None, aux_bits: np.ndarray = None):
+        """Overwrite one sequence's device caches with host bit arrays [layers, 2, Hkv, cap, hd]."""
+        if target_bits is not None:
+            t = torch.from_numpy(target_bits.view(np.int16)).view(torch.bfloat16).cuda()
+            self.cache[:, seq] = t
+        if aux_bits is not None:
+            t = torch.from_numpy(aux_bits.view(np.int16)).view(torch.bfloat16).cuda()
+            self.aux_cache[:, seq] = t
+
     def cache_bits(self, seq: int, upto: int) -> np.ndarray:
         """Host copy of one sequence's cache [layers, 2, Hkv, capacity, hd] as bf16 bits (only [0, upto) filled)."""
         out = np.zeros((self.shape.layers, 2, self.shape.n_kv_heads, self.capacity, self.shape.head_dim), np.uint16)
