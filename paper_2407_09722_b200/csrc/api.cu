@@ -24,7 +24,7 @@ struct WeightMaps {                      // index 0, 1, 2: tiles of 128, 256, 51
 struct mtad_ctx {
     WeightMaps tmaps, amaps;
     bool use_tc = false, use_pdl = false;
-    size_t tc_ws_floats = 0, tc_counter_n = 0, xf_elems = 0;
+    size_t tc_ws_floats = 0, tc_counter_n = 0, tc_flag_n = 0, xf_elems = 0;
     ModelView target, aux;
     bool has_aux = false;
     int max_batch = 0, max_nodes = 0, T_max = 0;
@@ -168,8 +168,13 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     };
     shape_ws(t);
     if (a) shape_ws(a);
-    sc.tc_ws = k.take<float>(ws_tiles * rpad * TC_TILE_N);
-    sc.tc_counters = k.take<int32_t>(max_tiles);
+    // the phases of a chained launch work side by side: one fix-up region and one set of counters per phase
+    sc.tc_ws = k.take<float>(ws_tiles * rpad * TC_TILE_N * TC_MAX_PHASES);
+    sc.tc_counters = k.take<int32_t>(max_tiles * TC_MAX_PHASES);
+    size_t layers_max = t->layers;
+    if (a) layers_max = std::max<size_t>(layers_max, a->layers);
+    const size_t flag_n = (layers_max + 1) * TC_MAX_PHASES * (max_tiles + 1);
+    sc.tc_flags = k.take<int32_t>(flag_n);
     sc.lm_part = k.take<float4>(Tc * lm_tiles);
     sc.node_z = k.take<float>(T);
     DraftState ds;
@@ -185,7 +190,8 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     if (c) {
         c->ds = ds;
         c->st = st; c->rm = rm; c->sc = sc;
-        c->tc_ws_floats = ws_tiles * rpad * TC_TILE_N;
+        c->tc_ws_floats = ws_tiles * rpad * TC_TILE_N * TC_MAX_PHASES;
+        c->tc_flag_n = flag_n;
         c->tc_counter_n = max_tiles;
         c->xf_elems = (size_t)2 * TC_X_ROWS * F;
     }
@@ -287,6 +293,11 @@ bool build_weight_maps(const ModelView& m, WeightMaps& w) {
     return ok;
 }
 
+bool mma_attention(const mtad_model_desc& d) {
+    static const bool on = !(getenv("MTAD_TC_ATTN") && atoi(getenv("MTAD_TC_ATTN")) == 0);
+    return on && (d.head_dim == 64 || d.head_dim == 128);
+}
+
 // The same forward on the tensor-core path: every projection is one launch of the TMA + tcgen05 GEMM with a fused
 // epilogue; activations travel between launches as bf16 hi/lo operand rows plus per-row sums of squares, so the
 // RMSNorm is applied as a per-row scale in the consumer's epilogue.  Leaves lm_part / node_z for launch_lm_merge.
@@ -324,6 +335,11 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
     base.hidden = sc.hidden; base.R = R; base.prow = ctx->rm.prow; base.tok = ctx->rm.tok; base.node_z = sc.node_z;
     base.lm_part = sc.lm_part; base.uniforms = uniforms;
     const double wb = 2.0;
+    // Every GEMM of the step is described first; then the projections that feed one another without attention in
+    // between (O, gate/up, down, and the next layer's QKV or the LM head) are chained as phases of one launch.
+    struct GemmDesc { TcMaps mp; TcGemmParams p; double bytes; };
+    std::vector<GemmDesc> g;           // per layer: QKV, O, gate/up, down; then the LM head
+    g.reserve((size_t)d.layers * 4 + 1);
     for (int l = 0; l < d.layers; ++l) {
         {   // QKV + rotary + append
             TcGemmParams p = base; TcMaps mp{};
@@ -333,16 +349,7 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             p.mode = TC_QKV; p.N = qd; p.seg_k_tile = qt; p.seg_v_tile = qt + kt; p.layer = l;
             p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = (l == 0) ? 1 : dt;
             mp.a0 = wm.wq[ix(mq)][l]; mp.a1 = wm.wk[ix(mq)][l]; mp.a2 = wm.wv[ix(mq)][l]; mp.x = xd;
-            RUN(MTAD_K_GEMM, wb * (qd + 2.0 * kvd) * d.d_model, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
-        }
-        static const bool mma_attn = !(getenv("MTAD_TC_ATTN") && atoi(getenv("MTAD_TC_ATTN")) == 0);
-        if (mma_attn && (d.head_dim == 64 || d.head_dim == 128)) {
-            const int nsp = attention_mma_tiles_per_block(m, B, R, total);
-            const int ns = (int)(((total + 63) / 64 + nsp - 1) / nsp);
-            RUN(MTAD_K_ATTN, 0, 2, launch_attention_mma(m, l, ctx->rm, sc, B, R, ns, nsp, pdl, s));
-            RUN(MTAD_K_ATTN, 0, 0, launch_attention_combine(m, ctx->rm, sc, B, R, ns, true, pdl, s));
-        } else {
-            RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, true, pdl, s));
+            g.push_back({mp, p, wb * (qd + 2.0 * kvd) * d.d_model});
         }
         {   // O projection + residual, emits the FFN norm's operand rows
             TcGemmParams p = base; TcMaps mp{};
@@ -352,7 +359,7 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             p.gain = m.w(l, 5); p.x_hi = sc.xd_hi; p.x_lo = sc.xd_hi + d.d_model; p.ldx = 2 * d.d_model;
             p.sumsq_out = sc.sumsq_b;
             mp.a0 = wm.wo[ix(mh)][l]; mp.x = xa;
-            RUN(MTAD_K_GEMM, wb * d.d_model * qd, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
+            g.push_back({mp, p, wb * d.d_model * qd});
         }
         {   // gate / up + SwiGLU
             TcGemmParams p = base; TcMaps mp{};
@@ -361,7 +368,7 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             p.mode = TC_SWIGLU; p.N = d.d_ffn; p.sumsq_in = sc.sumsq_b; p.sumsq_in_parts = dt;
             p.x_hi = sc.xf_hi; p.x_lo = sc.xf_hi + d.d_ffn; p.ldx = 2 * d.d_ffn;
             mp.a0 = wm.gate[ix(mh)][l]; mp.a1 = wm.up[ix(mh)][l]; mp.x = xd;
-            RUN(MTAD_K_GEMM, wb * 2.0 * d.d_ffn * d.d_model, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
+            g.push_back({mp, p, wb * 2.0 * d.d_ffn * d.d_model});
         }
         {   // down projection + residual, emits the next norm's operand rows
             TcGemmParams p = base; TcMaps mp{};
@@ -371,19 +378,72 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             p.gain = (l + 1 < d.layers) ? m.w(l + 1, 0) : static_cast<const __nv_bfloat16*>(d.final_norm);
             p.x_hi = sc.xd_hi; p.x_lo = sc.xd_hi + d.d_model; p.ldx = 2 * d.d_model; p.sumsq_out = sc.sumsq_a;
             mp.a0 = wm.down[ix(mh)][l]; mp.x = xf;
-            RUN(MTAD_K_GEMM, wb * d.d_model * d.d_ffn, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
+            g.push_back({mp, p, wb * d.d_model * d.d_ffn});
         }
     }
-    {   // LM head + per-tile log-softmax / Gumbel-argmax partials + gather of the drafted tokens' logits
+    int lm_tiles128 = 0;
+    {   // LM head: per-tile log-softmax / Gumbel-argmax partials + gather of the drafted tokens' logits, or plain
+        // logits for the draft's beam selection
         TcGemmParams p = base; TcMaps mp{};
         tc_decompose(p, up(d.vocab, 128 * mh), d.d_model, T, kCtas);
         p.mh = mh; p.n_rows_total = d.vocab; p.n_tiles128 = up(d.vocab, 128);
         p.mode = lm_plain ? TC_PLAIN : TC_LMHEAD; p.N = d.vocab; p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = dt;
-        p.out = sc.logits; p.ldo = d.vocab;                 // draft steps keep the logits for the beam selection
+        p.out = sc.logits; p.ldo = d.vocab;
         mp.a0 = wm.lm_head[ix(mh)]; mp.x = xd;
-        RUN(MTAD_K_GEMM, wb * d.vocab * d.d_model, 1, launch_tc_gemm(mp, p, kCtas, pdl, s));
-        if (!lm_plain) RUN(MTAD_K_LMRED, 0, 2, launch_lm_merge(m, ctx->rm, sc, B, R, p.n_tiles128, uniforms, s));
+        lm_tiles128 = p.n_tiles128;
+        g.push_back({mp, p, wb * d.vocab * d.d_model});
     }
+    // chained launches are available but off by default: with stream-K every tile of a phase finishes at the end of
+    // the phase, so a chained phase starts no earlier than a separately launched kernel with its weights prefetched
+    static const bool use_chain = getenv("MTAD_TC_CHAIN") && atoi(getenv("MTAD_TC_CHAIN")) != 0;
+    const size_t flag_stride = ctx->tc_counter_n + 1;      // per (launch, phase): tile flags, then the finished-tile count
+    const bool chain = use_chain && mq == mh && (size_t)(d.layers + 1) * TC_MAX_PHASES * flag_stride <= ctx->tc_flag_n;
+    if (chain) CU(cudaMemsetAsync(sc.tc_flags, 0, sizeof(int32_t) * (size_t)(d.layers + 1) * TC_MAX_PHASES * flag_stride, s));
+    int launch_no = 0;
+    // launches descriptors [i0, i0 + n) as one kernel
+    auto launch = [&](size_t i0, int n) -> int {
+        TcChain ch{};
+        ch.n_phases = n;
+        double bytes = 0;
+        for (int k = 0; k < n; ++k) {
+            ch.maps[k] = g[i0 + k].mp;
+            ch.p[k] = g[i0 + k].p;
+            bytes += g[i0 + k].bytes;
+            ch.p[k].ws = sc.tc_ws + (size_t)k * (ctx->tc_ws_floats / TC_MAX_PHASES);
+            ch.p[k].counters = sc.tc_counters + (size_t)k * ctx->tc_counter_n;
+            if (n > 1) {
+                int32_t* fl = sc.tc_flags + ((size_t)launch_no * TC_MAX_PHASES + k) * flag_stride;
+                ch.p[k].tile_done = fl;
+                ch.p[k].phase_done = fl + ctx->tc_counter_n;
+                if (k > 0) {
+                    const TcGemmParams& prev = g[i0 + k - 1].p;
+                    ch.p[k].dep_feat = (prev.mode == TC_SWIGLU ? 64 : 128) * prev.mh;
+                }
+            }
+        }
+        ++launch_no;
+        RUN(MTAD_K_GEMM, bytes, 1, launch_tc_chain(ch, pdl, s));
+        return MTAD_OK;
+    };
+    if (int rc = launch(0, 1)) return rc;                       // QKV of layer 0
+    for (int l = 0; l < d.layers; ++l) {
+        if (mma_attention(d)) {
+            const int nsp = attention_mma_tiles_per_block(m, B, R, total);
+            const int ns = (int)(((total + 63) / 64 + nsp - 1) / nsp);
+            RUN(MTAD_K_ATTN, 0, 2, launch_attention_mma(m, l, ctx->rm, sc, B, R, ns, nsp, pdl, s));
+            RUN(MTAD_K_ATTN, 0, 0, launch_attention_combine(m, ctx->rm, sc, B, R, ns, true, pdl, s));
+        } else {
+            RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, true, pdl, s));
+        }
+        const size_t o = (size_t)l * 4 + 1;                     // O, gate/up, down of this layer, then what follows
+        if (chain) {
+            if (int rc = launch(o, 4)) return rc;
+        } else {
+            for (int k = 0; k < 4; ++k)
+                if (int rc = launch(o + k, 1)) return rc;
+        }
+    }
+    if (!lm_plain) RUN(MTAD_K_LMRED, 0, 2, launch_lm_merge(m, ctx->rm, sc, B, R, lm_tiles128, uniforms, s));
     return MTAD_OK;
 }
 

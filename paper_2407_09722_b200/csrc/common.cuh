@@ -91,6 +91,7 @@ struct Scratch {
     float* sumsq_b;      // [tiles(d)][256] the same after the O projection
     float* tc_ws;        // split-K partial tiles
     int32_t* tc_counters;
+    int32_t* tc_flags;   // finished-tile flags and counts of the phases of chained GEMM launches, zeroed per forward
     float4* lm_part;     // [T][tiles(V)]
     float* node_z;       // [T]
 };

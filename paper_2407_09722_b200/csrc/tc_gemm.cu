@@ -9,11 +9,14 @@
 // evenly to the CTAs (one per SM); a tile whose k-range spans several CTAs is completed by whichever of them
 // arrives last, which sums the partial tiles in CTA order (deterministic) and runs the fused epilogue.
 //
-// Warp roles: 0 = TMA producer, 1..4 = MMA issuers (one per 128-row half of a stage; a single thread cannot issue
-// the many small MMAs of a skinny problem fast enough), 5..8 = epilogue (one TMEM lane quadrant each).
+// Warp roles: 0 = weight producer (TMA), 1 = operand-row producer (TMA, waits for the rows to exist), 2..5 = MMA
+// issuers (one per 128-row half of a stage; a single thread cannot issue the many small MMAs of a skinny problem
+// fast enough), 6..9 = epilogue (one TMEM lane quadrant each).
 // Every wait on an mbarrier is bounded; on a time-out the kernel raises MTAD_ST_TIMEOUT, waits (bounded) for its
 // own copies in flight, frees its tensor memory and returns.
 #include <math_constants.h>
+
+#include <algorithm>
 #include <stdlib.h>
 
 #include "tc_gemm.cuh"
@@ -26,7 +29,7 @@ constexpr int MAX_STAGES = 12;
 constexpr int EPI_THREADS = 128;
 constexpr int EPI_ROWS = 8;                       // draft rows finished per epilogue pass
 constexpr int MAX_HALVES = 4;                     // 128-row weight halves per stage, one MMA-issuing warp each
-constexpr int TC_THREADS = 32 * (1 + MAX_HALVES + 4);
+constexpr int TC_THREADS = 32 * (2 + MAX_HALVES + 4);
 constexpr uint64_t HINT_STREAM = 0x12F0000000000000ull;   // evict-first: weights are read once
 constexpr uint64_t HINT_KEEP = 0x14F0000000000000ull;     // evict-last: activation operands are re-read by every CTA
 
@@ -55,6 +58,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
         if (mbar_test(bar, parity)) return true;
         if (it > 64) __nanosleep(32);
+        if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+// Bounded wait until a counter written by other CTAs of this launch reaches `want` (acquire at gpu scope).
+__device__ __forceinline__ bool flag_wait(const int* flag, int want, volatile int* abort_flag) {
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+        if (v >= want) return true;
+        __nanosleep(64);
         if ((it & 255u) == 255u && *abort_flag) return false;
     }
     *abort_flag = 1;
@@ -114,16 +130,29 @@ __device__ __forceinline__ void split_store(float y, __nv_bfloat16* hi, __nv_bfl
     *lo = __float2bfloat16_rn(y - __bfloat162float(h));
 }
 
-#ifdef MTAD_TC_TRACE
-__device__ unsigned long long g_trace[1024 * 8];
-__device__ __forceinline__ void trace(int k) {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    g_trace[blockIdx.x * 8 + k] = t;
+
+// Weight boxes of one stage: how many, and for box b of a tile which map (0..2), which row coordinate and which
+// row offset inside the stage.  SwiGLU tiles take their first half from the gate matrix and their second half
+// from the up matrix; QKV tiles lie in the q, k or v matrix; a 512-row tile is fetched as two 256-row boxes.
+__device__ __forceinline__ int a_boxes(int mode, int mh) { return (mode == TC_SWIGLU || mh == 4) ? 2 : 1; }
+__device__ __forceinline__ void a_box(int mode, int mh, int seg_k, int seg_v, int tile, int b, int& which, int& y,
+                                      int& row_off) {
+    if (mode == TC_SWIGLU) {
+        const int rows = 64 * mh;
+        which = b;
+        y = tile * rows;
+        row_off = b * rows;
+    } else if (mode == TC_QKV) {
+        const int t128 = tile * mh;
+        which = t128 < seg_k ? 0 : (t128 < seg_v ? 1 : 2);
+        y = (t128 < seg_k ? t128 : (t128 < seg_v ? t128 - seg_k : t128 - seg_v)) * TC_TILE_N + b * 256;
+        row_off = b * 256;
+    } else {
+        which = 0;
+        y = tile * mh * TC_TILE_N + b * 256;
+        row_off = b * 256;
+    }
 }
-#else
-__device__ __forceinline__ void trace(int) {}
-#endif
 
 struct Smem {
     uint8_t* ring;
@@ -238,7 +267,7 @@ __device__ __forceinline__ void epi_resid(const TcGemmParams& p, const Smem& s, 
         const int t = r0 + j;
         float y = 0.f;
         if (ok && t < p.T) {
-            y = p.hidden[(size_t)t * p.N + n] + epi[j][e];
+            y = __ldcg(p.hidden + (size_t)t * p.N + n) + epi[j][e];
             p.hidden[(size_t)t * p.N + n] = y;
             split_store(y * g, p.x_hi + (size_t)t * p.ldx + n, p.x_lo + (size_t)t * p.ldx + n);
         }
@@ -337,36 +366,28 @@ __device__ __forceinline__ void epi_lmhead(const TcGemmParams& p, const Smem& s,
 // kernel
 // ---------------------------------------------------------------------------------------------------------------
 
-__global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_constant__ TcMaps maps, const TcGemmParams p) {
+__global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_constant__ TcChain ch) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int mh = p.mh;                               // 128-row weight halves per stage (1, 2 or 4)
+    const TcGemmParams& p0 = ch.p[0];
+    const int mh = p0.mh;                              // 128-row weight halves per stage (1, 2 or 4), same in every phase
     const int a_bytes = mh * TC_TILE_N * 128;
-    const int acc_cols = 2 * p.rpad;                   // one column per operand row: hi and lo of a draft row are neighbours
+    const int acc_cols = 2 * p0.rpad;                  // one column per operand row: hi and lo of a draft row are neighbours
     const int n_bbox = acc_cols > 256 ? 2 : 1;         // TMA boxes (and MMAs per k step and half) that cover the operand rows
     const int bbox_rows = acc_cols / n_bbox;
     const int stage_bytes = a_bytes + acc_cols * 128;
-    const Smem s = carve(smem_base, p.stages, stage_bytes);
+    const int stages = p0.stages, nbuf = p0.nbuf, T = p0.T;
+    const Smem s = carve(smem_base, stages, stage_bytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        trace(0);
-        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps.a0)) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps.x)) : "memory");
-        if (p.mode == TC_QKV || p.mode == TC_SWIGLU)
-            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps.a1)) : "memory");
-        if (p.mode == TC_QKV)
-            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps.a2)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&ch.maps[0].a0)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&ch.maps[0].x)) : "memory");
     }
-    const int u_begin = blockIdx.x * p.units_per_cta;
-    const int u_end = min(u_begin + p.units_per_cta, p.total_units);
-    const int n_units = max(u_end - u_begin, 0);
-    const int KB = p.k_blocks;
-    const int nbuf = p.nbuf;
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < nbuf * mh * acc_cols) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < p.stages; ++i) {
+        for (int i = 0; i < stages; ++i) {
             mbar_init(smem_u32(&s.full[i]), 1);
             mbar_init(smem_u32(&s.empty[i]), mh);        // one commit per MMA-issuing warp
         }
@@ -378,7 +399,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {
+    if (warp == 2) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s.tmem_ptr)),
                      "r"(tmem_cols)
                      : "memory");
@@ -388,279 +409,287 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *s.tmem_ptr;
-    if (threadIdx.x == 0) trace(1);
     // let the next kernel in the stream start its own prologue (it waits for this grid before it reads our output)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     volatile int* abort_flag = s.abort_flag;
+    // this CTA's share of a phase: units [first, first + count)
+    auto share = [&](const TcGemmParams& p, int& first, int& count) {
+        first = (int)blockIdx.x * p.units_per_cta;
+        count = max(min(first + p.units_per_cta, p.total_units) - first, 0);
+    };
 
     if (warp == 0) {
-        // ---------------- TMA producer: the whole warp walks the units, lane l issues the l-th copy of a stage ------
-        if (n_units > 0) {
-            // copies of one stage: weight boxes first (gate|up, or two 256-row boxes of a 512-row tile), then the
-            // operand-row boxes
-            const int n_a = (p.mode == TC_SWIGLU || mh == 4) ? 2 : 1;
-            auto issue = [&](int i, bool do_a, bool do_b) {
-                const int u = u_begin + i, tile = u / KB, kb = u % KB, st = i % p.stages;
-                const uint32_t bar = smem_u32(&s.full[st]);
-                const uint32_t base = smem_u32(s.ring + (size_t)st * stage_bytes);
-                if (do_a && lane == 0) mbar_expect_tx(bar, (uint32_t)stage_bytes);
-                __syncwarp();
-                const CUtensorMap* m = nullptr;
-                uint32_t dst = 0;
-                int y = 0;
-                uint64_t hint = HINT_STREAM;
-                if (lane < n_a) {
-                    if (!do_a) return;
-                    if (p.mode == TC_SWIGLU) {
-                        // gate rows fill the first half of the stage's weight rows, up rows the second half
-                        const int rows = 64 * mh;
-                        m = lane == 0 ? &maps.a0 : &maps.a1;
-                        dst = base + lane * rows * 128;
-                        y = tile * rows;
-                    } else if (p.mode == TC_QKV) {
-                        const int t128 = tile * mh;
-                        m = t128 < p.seg_k_tile ? &maps.a0 : (t128 < p.seg_v_tile ? &maps.a1 : &maps.a2);
-                        y = (t128 < p.seg_k_tile ? t128 : (t128 < p.seg_v_tile ? t128 - p.seg_k_tile
-                                                                               : t128 - p.seg_v_tile)) * TC_TILE_N +
-                            lane * 256;
-                        dst = base + lane * 256 * 128;
-                    } else {
-                        m = &maps.a0;
-                        y = tile * mh * TC_TILE_N + lane * 256;
-                        dst = base + lane * 256 * 128;
-                    }
-                } else if (lane < n_a + n_bbox) {
-                    if (!do_b) return;
-                    const int b = lane - n_a;
-                    m = &maps.x;
-                    dst = base + a_bytes + b * bbox_rows * 128;
-                    y = b * bbox_rows;
-                    hint = HINT_KEEP;
-                } else {
-                    return;
-                }
-                tma_load_2d(dst, m, bar, kb * TC_TILE_K, y, hint);
-            };
-            // weights do not depend on the previous kernel: start streaming them before waiting for it
-            const int pre = min(p.stages, n_units);
-            for (int i = 0; i < pre; ++i) issue(i, true, false);
-            asm volatile("griddepcontrol.wait;" ::: "memory");
-            for (int i = 0; i < pre; ++i) issue(i, false, true);
-            if (lane == 0) trace(2);
+        // ---------------- weight producer (one thread) -------------------------------------------------------------
+        // Weights never depend on an earlier step: their copies go out as soon as a stage is free, across phase
+        // boundaries too.  The operand rows of the same stage are brought by the next warp once they exist.
+        if (lane == 0) {
+            int g = 0;
             bool ok = true;
-#ifdef MTAD_TC_TRACE
-            unsigned long long t_wait = 0, t_all0 = clock64();
-#endif
-            for (int i = pre; i < n_units; ++i) {
-                const int st = i % p.stages;
-                const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-#ifdef MTAD_TC_TRACE
-                unsigned long long c0 = clock64();
-                if (lane == 0) ok = mbar_wait(smem_u32(&s.empty[st]), ph ^ 1u, abort_flag);
-                t_wait += clock64() - c0;
-                if (lane == 0 && i == n_units - 1)
-                    g_trace[blockIdx.x * 8 + 7] = (t_wait << 32) | ((clock64() - t_all0) & 0xffffffffull);
-#else
-                if (lane == 0) ok = mbar_wait(smem_u32(&s.empty[st]), ph ^ 1u, abort_flag);
-#endif
-                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-                if (!ok) break;
-                issue(i, true, true);
-            }
-            if (lane == 0 && *abort_flag) {
-                // give our own copies in flight a bounded chance to land before the CTA exits
-                const int first = max(0, n_units - p.stages);
-                for (int i = first; i < n_units; ++i) {
-                    const uint32_t bar = smem_u32(&s.full[i % p.stages]);
-                    const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-                    for (uint32_t it = 0; it < (1u << 16) && !mbar_test(bar, ph); ++it) __nanosleep(64);
+            for (int ph = 0; ph < ch.n_phases && ok; ++ph) {
+                const TcGemmParams& p = ch.p[ph];
+                const TcMaps& mp = ch.maps[ph];
+                int first, n_units;
+                share(p, first, n_units);
+                const int nb = a_boxes(p.mode, mh);
+                int tile = n_units > 0 ? first / p.k_blocks : 0, kb = n_units > 0 ? first % p.k_blocks : 0;
+                for (int i = 0; i < n_units; ++i, ++g) {
+                    const int st = g % stages;
+                    if (g >= stages) {
+                        ok = mbar_wait(smem_u32(&s.empty[st]), (((uint32_t)(g / stages)) & 1u) ^ 1u, abort_flag);
+                        if (!ok) break;
+                    }
+                    const uint32_t bar = smem_u32(&s.full[st]);
+                    const uint32_t base = smem_u32(s.ring + (size_t)st * stage_bytes);
+                    mbar_expect_tx(bar, (uint32_t)stage_bytes);
+                    for (int b = 0; b < nb; ++b) {
+                        int which, y, row_off;
+                        a_box(p.mode, mh, p.seg_k_tile, p.seg_v_tile, tile, b, which, y, row_off);
+                        const CUtensorMap* m = which == 0 ? &mp.a0 : (which == 1 ? &mp.a1 : &mp.a2);
+                        tma_load_2d(base + row_off * 128, m, bar, kb * TC_TILE_K, y, HINT_STREAM);
+                    }
+                    if (++kb == p.k_blocks) { kb = 0; ++tile; }
                 }
             }
         }
-    } else if (warp <= MAX_HALVES) {
-        // ---------------- MMA issuers: warp 1 + h owns the 128-row half h of every stage and its accumulator --------
-        const int h = warp - 1;
-        if (lane == 0 && n_units > 0 && h < mh) {
+    } else if (warp == 1) {
+        // ---------------- operand-row producer (one thread) --------------------------------------------------------
+        // The rows of a k-block exist once their producer is finished: the previous kernel for phase 0, the tile of
+        // the previous phase that wrote those 64 columns otherwise.
+        if (lane == 0) {
+            int g = 0;
+            bool ok = true;
+            for (int ph = 0; ph < ch.n_phases && ok; ++ph) {
+                const TcGemmParams& p = ch.p[ph];
+                int first, n_units;
+                share(p, first, n_units);
+                if (ph == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
+                int kb = n_units > 0 ? first % p.k_blocks : 0;
+                int ready_tile = -1;                   // tile of the previous phase known to be finished
+                for (int i = 0; i < n_units && ok; ++i, ++g) {
+                    const int st = g % stages;
+                    if (g >= stages) {
+                        ok = mbar_wait(smem_u32(&s.empty[st]), (((uint32_t)(g / stages)) & 1u) ^ 1u, abort_flag);
+                        if (!ok) break;
+                    }
+                    if (ph > 0) {
+                        const int need = (kb * TC_TILE_K) / p.dep_feat;
+                        if (need != ready_tile) {
+                            ok = flag_wait(ch.p[ph - 1].tile_done + need, 1, abort_flag);
+                            if (!ok) break;
+                            ready_tile = need;
+                            asm volatile("fence.proxy.async;" ::: "memory");    // the rows are read by TMA next
+                        }
+                    }
+                    const uint32_t bar = smem_u32(&s.full[st]);
+                    const uint32_t base = smem_u32(s.ring + (size_t)st * stage_bytes) + a_bytes;
+                    for (int b = 0; b < n_bbox; ++b)
+                        tma_load_2d(base + b * bbox_rows * 128, &ch.maps[ph].x, bar, kb * TC_TILE_K, b * bbox_rows,
+                                    HINT_KEEP);
+                    if (++kb == p.k_blocks) kb = 0;
+                }
+            }
+            if (*abort_flag) {
+                // give the copies in flight a bounded chance to land before the CTA exits
+                for (int i = max(0, g - stages); i < g; ++i) {
+                    const uint32_t bar = smem_u32(&s.full[i % stages]);
+                    const uint32_t phs = (uint32_t)(i / stages) & 1u;
+                    for (uint32_t it = 0; it < (1u << 16) && !mbar_test(bar, phs); ++it) __nanosleep(64);
+                }
+            }
+        }
+    } else if (warp < 2 + MAX_HALVES) {
+        // ---------------- MMA issuers: warp 2 + h owns the 128-row half h of every stage and its accumulator --------
+        const int h = warp - 2;
+        if (lane == 0 && h < mh) {
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bbox_rows >> 3) << 17) |
                                    ((uint32_t)(TC_TILE_N >> 4) << 24);
-            int i = 0, seg = 0;
+            int g = 0, seg = 0;                        // running unit and segment counters over all phases
             bool ok = true;
-#ifdef MTAD_TC_TRACE
-            unsigned long long mma_wait = 0, mma_t0 = clock64(), mma_issue = 0, mma_commit = 0;
-#endif
-            while (i < n_units && ok) {
-                const int u = u_begin + i;
-                const int kb0 = u % KB;
-                const int len = min(KB - kb0, n_units - i);
-                const int buf = seg % nbuf;
-                const uint32_t aph = (uint32_t)(seg / nbuf) & 1u;
-                ok = mbar_wait(smem_u32(&s.tempty[buf]), aph ^ 1u, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * mh * acc_cols);
-                for (int k = 0; k < len && ok; ++k, ++i) {
-                    const int st = i % p.stages;
-                    const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-#ifdef MTAD_TC_TRACE
-                    unsigned long long c0 = clock64();
-                    ok = mbar_wait(smem_u32(&s.full[st]), ph, abort_flag);
-                    if (i > 0) mma_wait += clock64() - c0;
-#else
-                    ok = mbar_wait(smem_u32(&s.full[st]), ph, abort_flag);
-#endif
+            for (int ph = 0; ph < ch.n_phases && ok; ++ph) {
+                const TcGemmParams& p = ch.p[ph];
+                int first, n_units;
+                share(p, first, n_units);
+                const int KB = p.k_blocks;
+                int i = 0;
+                while (i < n_units && ok) {
+                    const int kb0 = (first + i) % KB;
+                    const int len = min(KB - kb0, n_units - i);
+                    const int buf = seg % nbuf;
+                    const uint32_t aph = (uint32_t)(seg / nbuf) & 1u;
+                    ok = mbar_wait(smem_u32(&s.tempty[buf]), aph ^ 1u, abort_flag);
                     if (!ok) break;
-                    if (i == 0 && h == 0) trace(3);
                     tc_fence_after();
-                    const uint32_t a_addr = smem_u32(s.ring + (size_t)st * stage_bytes);
-                    const uint32_t b_addr = a_addr + a_bytes;
-#ifdef MTAD_TC_TRACE
-                    unsigned long long ci0 = clock64();
-#endif
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(buf * mh * acc_cols);
+                    for (int k = 0; k < len && ok; ++k, ++i, ++g) {
+                        const int st = g % stages;
+                        const uint32_t sph = (uint32_t)(g / stages) & 1u;
+                        ok = mbar_wait(smem_u32(&s.full[st]), sph, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t a_addr = smem_u32(s.ring + (size_t)st * stage_bytes);
+                        const uint32_t b_addr = a_addr + a_bytes;
 #pragma unroll
-                    for (int k4 = 0; k4 < TC_TILE_K / 16; ++k4) {
-                        const uint32_t acc = (k > 0 || k4 > 0) ? 1u : 0u;
-                        const uint64_t ad = smem_desc(a_addr + h * TC_TILE_N * 128 + k4 * 32);
-                        for (int b = 0; b < n_bbox; ++b)
-                            tc_mma(d_tmem + (uint32_t)(h * acc_cols + b * bbox_rows), ad,
-                                   smem_desc(b_addr + b * bbox_rows * 128 + k4 * 32), idesc, acc);
+                        for (int k4 = 0; k4 < TC_TILE_K / 16; ++k4) {
+                            const uint32_t acc = (k > 0 || k4 > 0) ? 1u : 0u;
+                            const uint64_t ad = smem_desc(a_addr + h * TC_TILE_N * 128 + k4 * 32);
+                            for (int b = 0; b < n_bbox; ++b)
+                                tc_mma(d_tmem + (uint32_t)(h * acc_cols + b * bbox_rows), ad,
+                                       smem_desc(b_addr + b * bbox_rows * 128 + k4 * 32), idesc, acc);
+                        }
+                        tc_commit(smem_u32(&s.empty[st]));      // frees the smem stage once these MMAs have read it
                     }
-#ifdef MTAD_TC_TRACE
-                    unsigned long long ci1 = clock64();
-#endif
-                    tc_commit(smem_u32(&s.empty[st]));      // frees the smem stage once these MMAs have read it
-#ifdef MTAD_TC_TRACE
-                    mma_issue += ci1 - ci0; mma_commit += clock64() - ci1;
-#endif
+                    if (ok) tc_commit(smem_u32(&s.tfull[buf]));  // accumulator of this segment complete
+                    ++seg;
                 }
-                if (ok) tc_commit(smem_u32(&s.tfull[buf]));  // accumulator of this segment complete
-                ++seg;
             }
-            if (h == 0) trace(4);
-#ifdef MTAD_TC_TRACE
-            if (h == 0) g_trace[blockIdx.x * 8 + 5] = (mma_wait << 32) | ((clock64() - mma_t0) & 0xffffffffull);
-            if (h == 0) g_trace[blockIdx.x * 8 + 6] = (mma_issue << 32) | (mma_commit & 0xffffffffull);
-#endif
         }
     } else {
         // ---------------- epilogue ----------------
-        const int e = threadIdx.x - 32 * (1 + MAX_HALVES);   // 0..127
+        const int e = threadIdx.x - 32 * (2 + MAX_HALVES);   // 0..127
         const int quad = warp & 3;                      // TMEM lane quadrant this warp may read
         const int feat = quad * 32 + lane;              // feature (TMEM lane) within a 128-row half
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        // deferred RMSNorm scale of every row
-        for (int r = e; r < TC_MAX_ROWS; r += EPI_THREADS) {
-            float v = 1.f;
-            if (r < p.T && p.sumsq_in_parts > 0) {
-                float acc = 0.f;
-                for (int q = 0; q < p.sumsq_in_parts; ++q) acc += p.sumsq_in[(size_t)q * TC_X_ROWS + r];
-                v = rsqrtf(acc * p.inv_dim + p.eps);
-            }
-            s.rstd[r] = v;
-        }
-        epi_bar();
-        const size_t half_floats = (size_t)p.rpad * TC_TILE_N;
+        const size_t half_floats = (size_t)p0.rpad * TC_TILE_N;
         const size_t part_floats = (size_t)mh * half_floats;
-        int i = 0, seg = 0;
-        while (i < n_units) {
-            const int u = u_begin + i;
-            const int tile = u / KB, kb0 = u % KB;
-            const int len = min(KB - kb0, n_units - i);
-            const int buf = seg % nbuf;
-            const uint32_t aph = (uint32_t)(seg / nbuf) & 1u;
-            bool ok = true;
-            if (lane == 0) ok = mbar_wait(smem_u32(&s.tfull[buf]), aph, abort_flag);
-            if (lane == 0) s.flags[1 + (warp - 1 - MAX_HALVES)] = ok ? 1 : 0;
+        int seg = 0;
+        bool alive = true;
+        for (int ph = 0; ph < ch.n_phases && alive; ++ph) {
+            const TcGemmParams& p = ch.p[ph];
+            int first, n_units;
+            share(p, first, n_units);
+            const int KB = p.k_blocks;
+            // everything this phase reads besides its operand rows (row statistics, the residual stream) is final once
+            // the previous kernel (phase 0) or the whole previous phase has finished
+            if (ph == 0) {
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+            } else {
+                if (e == 0) s.flags[0] = flag_wait(ch.p[ph - 1].phase_done, ch.p[ph - 1].n_tiles, abort_flag) ? 1 : 0;
+                epi_bar();
+                alive = s.flags[0] != 0;
+                epi_bar();
+                if (!alive) break;
+            }
+            // deferred RMSNorm scale of every row
+            for (int r = e; r < TC_MAX_ROWS; r += EPI_THREADS) {
+                float v = 1.f;
+                if (r < T && p.sumsq_in_parts > 0) {
+                    float acc = 0.f;
+                    for (int q = 0; q < p.sumsq_in_parts; ++q) acc += __ldcg(p.sumsq_in + (size_t)q * TC_X_ROWS + r);
+                    v = rsqrtf(acc * p.inv_dim + p.eps);
+                }
+                s.rstd[r] = v;
+            }
             epi_bar();
-            if (!(s.flags[1] && s.flags[2] && s.flags[3] && s.flags[4])) break;   // uniform over the 128 threads
-            tc_fence_after();
-            // contributors of this tile, in CTA order
-            const int c_first = (tile * KB) / p.units_per_cta;
-            const int c_last = ((tile + 1) * KB - 1) / p.units_per_cta;
-            const int n_contrib = c_last - c_first + 1;
-            const int slot_idx = (int)blockIdx.x - c_first;
-            float* part = p.ws + ((size_t)tile * p.max_contrib + slot_idx) * part_floats;
-            for (int h = 0; h < mh; ++h) {
-                for (int c0 = 0; c0 < 2 * p.T; c0 += 16) {
-                    float v[16];
-                    tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) +
-                                (uint32_t)(buf * mh * acc_cols + h * acc_cols + c0), v);
+            int i = 0;
+            while (i < n_units) {
+                const int u = first + i;
+                const int tile = u / KB, kb0 = u % KB;
+                const int len = min(KB - kb0, n_units - i);
+                const int buf = seg % nbuf;
+                const uint32_t aph = (uint32_t)(seg / nbuf) & 1u;
+                bool ok = true;
+                if (lane == 0) ok = mbar_wait(smem_u32(&s.tfull[buf]), aph, abort_flag);
+                if (lane == 0) s.flags[1 + (warp - 2 - MAX_HALVES)] = ok ? 1 : 0;
+                epi_bar();
+                if (!(s.flags[1] && s.flags[2] && s.flags[3] && s.flags[4])) { alive = false; break; }
+                tc_fence_after();
+                // contributors of this tile, in CTA order
+                const int c_first = (tile * KB) / p.units_per_cta;
+                const int c_last = ((tile + 1) * KB - 1) / p.units_per_cta;
+                const int n_contrib = c_last - c_first + 1;
+                const int slot_idx = (int)blockIdx.x - c_first;
+                float* part = p.ws + ((size_t)tile * p.max_contrib + slot_idx) * part_floats;
+                for (int h = 0; h < mh; ++h) {
+                    for (int c0 = 0; c0 < 2 * T; c0 += 16) {
+                        float v[16];
+                        tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) +
+                                    (uint32_t)(buf * mh * acc_cols + h * acc_cols + c0), v);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int r = (c0 >> 1) + j;
-                        if (r < p.T) part[h * half_floats + (size_t)r * TC_TILE_N + feat] = v[2 * j] + v[2 * j + 1];
+                        for (int j = 0; j < 8; ++j) {
+                            const int r = (c0 >> 1) + j;
+                            if (r < T) part[h * half_floats + (size_t)r * TC_TILE_N + feat] = v[2 * j] + v[2 * j + 1];
+                        }
                     }
                 }
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&s.tempty[buf]));   // MMA may reuse this accumulator
-            __threadfence();
-            epi_bar();
-            if (e == 0) {
-                const int old = atomicAdd(&p.counters[tile], 1);
-                s.flags[0] = (old + 1 == n_contrib);
-            }
-            epi_bar();
-            if (s.flags[0]) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&s.tempty[buf]));   // MMA may reuse this accumulator
                 __threadfence();
-                const float* tile_ws = p.ws + (size_t)tile * p.max_contrib * part_floats;
-                for (int r0 = 0; r0 < p.T; r0 += EPI_ROWS) {
-                    for (int h = 0; h < mh; ++h) {
-                        float acc[EPI_ROWS];
-#pragma unroll
-                        for (int j = 0; j < EPI_ROWS; ++j) acc[j] = 0.f;
-                        // partials are added in CTA order (deterministic); four contributors' loads are issued
-                        // together so that the L2 latency is paid once per group, not once per contributor
-                        for (int c = 0; c < n_contrib; c += 4) {
-                            float v[4][EPI_ROWS];
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const float* src = tile_ws + (size_t)(c + q) * part_floats + h * half_floats + e;
-#pragma unroll
-                                for (int j = 0; j < EPI_ROWS; ++j)
-                                    v[q][j] = (c + q < n_contrib && r0 + j < p.T)
-                                                  ? __ldcg(src + (size_t)(r0 + j) * TC_TILE_N) : 0.f;
-                            }
-#pragma unroll
-                            for (int q = 0; q < 4; ++q)
-#pragma unroll
-                                for (int j = 0; j < EPI_ROWS; ++j) acc[j] += v[q][j];
-                        }
-#pragma unroll
-                        for (int j = 0; j < EPI_ROWS; ++j) s.epi[h][j][e] = (r0 + j < p.T) ? acc[j] * s.rstd[r0 + j] : 0.f;
-                    }
-                    epi_bar();
-                    if (p.mode == TC_SWIGLU) {
-                        epi_swiglu(p, s, tile, r0, e);
-                    } else {
-                        for (int h = 0; h < mh; ++h) {
-                            const int t128 = tile * mh + h;
-                            if (t128 * TC_TILE_N >= p.n_rows_total) break;      // half beyond the last weight row
-                            switch (p.mode) {
-                                case TC_PLAIN: epi_plain(p, s.epi[h], t128, r0, e); break;
-                                case TC_QKV: epi_qkv(p, s.epi[h], t128, r0, e); break;
-                                case TC_RESID: epi_resid(p, s, s.epi[h], t128, r0, e); break;
-                                default: epi_lmhead(p, s, s.epi[h], t128, r0, e); break;
-                            }
-                        }
-                    }
-                    epi_bar();
+                epi_bar();
+                if (e == 0) {
+                    const int old = atomicAdd(&p.counters[tile], 1);
+                    s.flags[0] = (old + 1 == n_contrib);
                 }
-                if (e == 0) p.counters[tile] = 0;          // ready for the next launch
+                epi_bar();
+                if (s.flags[0]) {
+                    __threadfence();
+                    const float* tile_ws = p.ws + (size_t)tile * p.max_contrib * part_floats;
+                    for (int r0 = 0; r0 < T; r0 += EPI_ROWS) {
+                        for (int h = 0; h < mh; ++h) {
+                            float acc[EPI_ROWS];
+#pragma unroll
+                            for (int j = 0; j < EPI_ROWS; ++j) acc[j] = 0.f;
+                            // partials are added in CTA order (deterministic); four contributors' loads are issued
+                            // together so that the L2 latency is paid once per group, not once per contributor
+                            for (int c = 0; c < n_contrib; c += 4) {
+                                float v[4][EPI_ROWS];
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    const float* src = tile_ws + (size_t)(c + q) * part_floats + h * half_floats + e;
+#pragma unroll
+                                    for (int j = 0; j < EPI_ROWS; ++j)
+                                        v[q][j] = (c + q < n_contrib && r0 + j < T)
+                                                      ? __ldcg(src + (size_t)(r0 + j) * TC_TILE_N) : 0.f;
+                                }
+#pragma unroll
+                                for (int q = 0; q < 4; ++q)
+#pragma unroll
+                                    for (int j = 0; j < EPI_ROWS; ++j) acc[j] += v[q][j];
+                            }
+#pragma unroll
+                            for (int j = 0; j < EPI_ROWS; ++j) s.epi[h][j][e] = (r0 + j < T) ? acc[j] * s.rstd[r0 + j] : 0.f;
+                        }
+                        epi_bar();
+                        if (p.mode == TC_SWIGLU) {
+                            epi_swiglu(p, s, tile, r0, e);
+                        } else {
+                            for (int h = 0; h < mh; ++h) {
+                                const int t128 = tile * mh + h;
+                                if (t128 * TC_TILE_N >= p.n_rows_total) break;      // half beyond the last weight row
+                                switch (p.mode) {
+                                    case TC_PLAIN: epi_plain(p, s.epi[h], t128, r0, e); break;
+                                    case TC_QKV: epi_qkv(p, s.epi[h], t128, r0, e); break;
+                                    case TC_RESID: epi_resid(p, s, s.epi[h], t128, r0, e); break;
+                                    default: epi_lmhead(p, s, s.epi[h], t128, r0, e); break;
+                                }
+                            }
+                        }
+                        epi_bar();
+                    }
+                    if (e == 0) p.counters[tile] = 0;          // ready for the next launch
+                    if (p.tile_done) {
+                        // publish the finished tile to the phase that reads it as operand rows
+                        __threadfence();
+                        epi_bar();
+                        if (e == 0) {
+                            asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p.tile_done + tile), "r"(1) : "memory");
+                            atomicAdd(p.phase_done, 1);
+                        }
+                    }
+                }
+                i += len;
+                ++seg;
             }
-            i += len;
-            ++seg;
         }
     }
     // ---------------- teardown ----------------
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == 2) {
         __syncwarp();
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
-    if (threadIdx.x == 0 && *abort_flag && p.status) atomicOr(p.status, MTAD_ST_TIMEOUT);
+    if (threadIdx.x == 0 && *abort_flag && p0.status) atomicOr(p0.status, MTAD_ST_TIMEOUT);
 }
 
 __global__ void split_rows_kernel(const float* __restrict__ x, int ldx_in, __nv_bfloat16* __restrict__ hi,
@@ -688,11 +717,6 @@ EncodeTiledFn encode_fn() {
 
 }  // namespace
 
-#ifdef MTAD_TC_TRACE
-extern "C" int mtad_debug_trace(unsigned long long* out, int n) {
-    return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(unsigned long long) * n);
-}
-#endif
 
 int tc_make_map(CUtensorMap* out, const void* base, long long rows, long long cols, int box_rows) {
     EncodeTiledFn fn = encode_fn();
@@ -732,18 +756,27 @@ size_t tc_workspace_floats(int n_tiles_max, int max_contrib_max, int rpad_max) {
     return (size_t)n_tiles_max * max_contrib_max * rpad_max * TC_TILE_N;
 }
 
-cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p_in, int ctas, bool pdl, cudaStream_t st) {
-    TcGemmParams p = p_in;
-    if (p.mh != 1 && p.mh != 2 && p.mh != 4) return cudaErrorInvalidValue;
-    p.nbuf = (2 * p.mh * 2 * p.rpad <= 512) ? 2 : 1;
-    if (p.mh * 2 * p.rpad > 512) return cudaErrorInvalidValue;
-    const int stage_bytes = p.mh * TC_TILE_N * 128 + 2 * p.rpad * 128;
+cudaError_t launch_tc_chain(const TcChain& chain_in, bool pdl, cudaStream_t st) {
+    TcChain ch = chain_in;
+    if (ch.n_phases < 1 || ch.n_phases > TC_MAX_PHASES) return cudaErrorInvalidValue;
+    const TcGemmParams& f = ch.p[0];
+    if (f.mh != 1 && f.mh != 2 && f.mh != 4) return cudaErrorInvalidValue;
+    if (f.mh * 2 * f.rpad > 512) return cudaErrorInvalidValue;
+    const int nbuf = (2 * f.mh * 2 * f.rpad <= 512) ? 2 : 1;
+    const int stage_bytes = f.mh * TC_TILE_N * 128 + 2 * f.rpad * 128;
     static const int budget_kb_env = getenv("MTAD_TC_SMEM_KB") ? atoi(getenv("MTAD_TC_SMEM_KB")) : 0;
     const size_t budget = (size_t)(budget_kb_env > 0 ? budget_kb_env : 226) * 1024;
     int stages = (int)((budget - SMEM_TAIL - 1024) / stage_bytes);
     stages = stages > MAX_STAGES ? MAX_STAGES : stages;
     if (stages < 2) return cudaErrorInvalidValue;
-    p.stages = stages;
+    int grid = 1;
+    for (int i = 0; i < ch.n_phases; ++i) {
+        TcGemmParams& p = ch.p[i];
+        if (p.mh != f.mh || p.rpad != f.rpad || p.T != f.T) return cudaErrorInvalidValue;   // one ring, one TMEM layout
+        p.nbuf = nbuf;
+        p.stages = stages;
+        grid = std::max(grid, (p.total_units + p.units_per_cta - 1) / p.units_per_cta);
+    }
     const size_t smem = (size_t)stages * stage_bytes + SMEM_TAIL + 1024;
     static bool attr_set = false;
     if (!attr_set) {
@@ -751,7 +784,6 @@ cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p_in, int cta
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    const int grid = (p.total_units + p.units_per_cta - 1) / p.units_per_cta;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(TC_THREADS);
@@ -762,8 +794,18 @@ cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p_in, int cta
     at[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
     cfg.attrs = at;
     cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, tc_gemm_kernel, ch);
+}
+
+cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p, int ctas, bool pdl, cudaStream_t st) {
     (void)ctas;
-    return cudaLaunchKernelEx(&cfg, tc_gemm_kernel, maps, p);
+    TcChain ch{};
+    ch.n_phases = 1;
+    ch.maps[0] = maps;
+    ch.p[0] = p;
+    ch.p[0].tile_done = nullptr;
+    ch.p[0].phase_done = nullptr;
+    return launch_tc_chain(ch, pdl, st);
 }
 
 cudaError_t launch_split_rows(const float* x, int ldx_in, __nv_bfloat16* hi, __nv_bfloat16* lo, int ld, int T, int K,

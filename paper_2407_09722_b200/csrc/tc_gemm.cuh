@@ -32,6 +32,12 @@ struct TcGemmParams {
     int stages;            // smem ring depth
     int mode;
     int N;                 // output features (bound for stores)
+    // Chained phases of one launch: a phase whose operand rows are written by the phase before it reads, per k-block,
+    // the flag of the tile that wrote those 64 columns (dep_feat = output features per tile of that phase); every
+    // finished tile sets tile_done[tile] and bumps *phase_done.  Null in a launch of a single phase.
+    int* tile_done;
+    int* phase_done;
+    int dep_feat;
     // split-K fix-up
     float* ws;             // [n_tiles][max_contrib][mh][rpad][128] partial tiles
     int* counters;         // [n_tiles], zero between launches
@@ -74,6 +80,17 @@ struct TcMaps {
     CUtensorMap a0, a1, a2;         // weight maps (QKV: wq, wk, wv; SwiGLU: gate, up; else a0)
     CUtensorMap x;                  // operand rows [2 * TC_X_ROWS, K]: row 2t = hi(t), row 2t + 1 = lo(t)
 };
+
+// Up to four GEMMs that feed one another (O projection, gate/up, down, next layer's QKV) run as phases of one launch:
+// the weight stream never stops at a phase boundary, and a phase starts on a k-block as soon as the tile that
+// produced those operand columns is final.
+constexpr int TC_MAX_PHASES = 4;
+struct TcChain {
+    int n_phases;
+    TcMaps maps[TC_MAX_PHASES];
+    TcGemmParams p[TC_MAX_PHASES];
+};
+cudaError_t launch_tc_chain(const TcChain& chain, bool pdl, cudaStream_t st);
 
 // Encodes a 2-D bf16 tensor map (row-major [rows, cols], 128-byte swizzle, box [box_rows, 64]).
 int tc_make_map(CUtensorMap* out, const void* base, long long rows, long long cols, int box_rows);
