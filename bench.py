@@ -184,7 +184,7 @@ def run_reference(args, w: S.Workload):
 
 
 def cpu_baseline(w: S.Workload):
-    n_layers = 2
+    n_layers = min(8, w.target.layers)
     smp = OracleSampler(w, n_layers)
     est, acc, ts = smp.step(0)
     return {"value": acc / est, "unit": "tokens/s", "cores": _blas_threads(), "kind": "oracle",
@@ -373,7 +373,7 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=32)
+    ap.add_argument("--steps", type=int, default=128)
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--workload", default="7b_chain", choices=sorted(S.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
