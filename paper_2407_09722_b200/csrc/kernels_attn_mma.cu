@@ -324,25 +324,35 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
             *reinterpret_cast<float2*>(ow + (gq + 8) * PARK + n * 8 + 2 * tq) = make_float2(oacc[n][2], oacc[n][3]);
         }
         __syncthreads();
-        for (int idx = threadIdx.x; idx < n_mt * 16 * HD; idx += blockDim.x) {
-            const int mtile = idx / (16 * HD), row = (idx / HD) % 16, d = idx % HD;
-            const int qi = mtile * 16 + row;
-            if (qi >= n_q) continue;
-            const int w0 = mtile * kparts;
+        // per (row, part) weight exp2(m_part - M) and the row's sum first, then the outputs of the valid rows only
+        float* wq = ml + 4 * 16 * 2;                  // [32 rows][4 parts] weights, then [32] maxima and [32] sums
+        float* wM = wq + 2 * 16 * 4;
+        float* wl = wM + 2 * 16;
+        for (int qi = threadIdx.x; qi < n_q; qi += blockDim.x) {
+            const int w0 = (qi >> 4) * kparts, row = qi & 15;
             float M = -CUDART_INF_F;
             for (int q = 0; q < kparts; ++q) M = fmaxf(M, ml[((w0 + q) * 16 + row) * 2]);
-            float acc = 0.f, lsum = 0.f;
-            for (int q = 0; q < kparts; ++q) {
+            float lsum = 0.f;
+            for (int q = 0; q < kparts; ++q) {                       // key order: deterministic
                 const float mq = ml[((w0 + q) * 16 + row) * 2];
-                if (mq == -CUDART_INF_F) continue;
-                const float wgt = exp2f(mq - M);
+                const float wgt = (mq == -CUDART_INF_F) ? 0.f : exp2f(mq - M);
+                wq[qi * 4 + q] = wgt;
                 lsum += ml[((w0 + q) * 16 + row) * 2 + 1] * wgt;
-                acc += (reinterpret_cast<const float*>(smem) + (w0 + q) * 16 * PARK)[row * PARK + d] * wgt;
             }
+            wM[qi] = M;
+            wl[qi] = lsum;
+        }
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < n_q * HD; idx += blockDim.x) {
+            const int qi = idx / HD, d = idx % HD;
+            const int w0 = (qi >> 4) * kparts, row = qi & 15;
+            float acc = 0.f;
+            for (int q = 0; q < kparts; ++q)
+                acc += (reinterpret_cast<const float*>(smem) + (w0 + q) * 16 * PARK)[row * PARK + d] * wq[qi * 4 + q];
             const int h = g * G + qi / nrows, r = qi % nrows;
             float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
             dst[2 + d] = acc;
-            if (d == 0) { dst[0] = M * LN2; dst[1] = lsum; }
+            if (d == 0) { dst[0] = wM[qi] * LN2; dst[1] = wl[qi]; }
         }
     }
 }
@@ -364,7 +374,7 @@ cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& r
     // query tiles kept in shared memory: all of them (at most two) when the warps split keys, else one per warp
     const int n_mt_max = ((Hq / Hkv) * R + 15) / 16;
     const int nslab = n_mt_max <= 2 ? n_mt_max : 4;
-    const size_t smem = (size_t)4 * KT * hd * 2 + (size_t)nslab * 2 * 16 * hd * 2 + 512;
+    const size_t smem = (size_t)4 * KT * hd * 2 + (size_t)nslab * 2 * 16 * hd * 2 + 2048;
     dim3 grid(nsplit, Hkv, B);
     static bool attr_set = false;
     if (!attr_set) {
