@@ -140,10 +140,9 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     const size_t Tc = std::min<size_t>(T, TC_MAX_ROWS);
     const size_t rpad = (Tc + 15) / 16 * 16;
     // operand rows, hi and lo interleaved: row 2t = hi(t), row 2t + 1 = lo(t)
-    sc.xd_hi = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * d);
-    sc.xa_hi = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * qd);
-    sc.xf_hi = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * F);
-    sc.xd_lo = sc.xa_lo = sc.xf_lo = nullptr;
+    sc.xd = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * d);
+    sc.xa = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * qd);
+    sc.xf = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * F);
     const size_t dt = (d + TC_TILE_N - 1) / TC_TILE_N;
     sc.sumsq_a = k.take<float>(dt * TC_X_ROWS);
     sc.sumsq_b = k.take<float>(dt * TC_X_ROWS);
@@ -320,11 +319,12 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
     while (mq > 1 && (qd % (128 * mq) || kvd % (128 * mq))) mq /= 2;
     auto ix = [](int halves) { return halves == 1 ? 0 : (halves == 2 ? 1 : 2); };
     auto up = [](int a, int b) { return (a + b - 1) / b; };
-    // operand-row maps for this call's row count: box = all 2 * rpad interleaved rows (two boxes beyond 256)
-    const int xbox = 2 * rpad > 256 ? rpad : 2 * rpad;
+    // operand-row maps for this call's row count: box = all terms * rpad interleaved rows (two boxes beyond 256)
+    const int terms = tc_terms(T);
+    const int xbox = terms * rpad > 256 ? terms * rpad / 2 : terms * rpad;
     CUtensorMap xd, xa, xf;
-    if (tc_make_map(&xd, sc.xd_hi, 2 * TC_X_ROWS, d.d_model, xbox) || tc_make_map(&xa, sc.xa_hi, 2 * TC_X_ROWS, qd, xbox) ||
-        tc_make_map(&xf, sc.xf_hi, 2 * TC_X_ROWS, d.d_ffn, xbox))
+    if (tc_make_map(&xd, sc.xd, 2 * TC_X_ROWS, d.d_model, xbox) || tc_make_map(&xa, sc.xa, 2 * TC_X_ROWS, qd, xbox) ||
+        tc_make_map(&xf, sc.xf, 2 * TC_X_ROWS, d.d_ffn, xbox))
         return MTAD_E_CUDA;
     TcGemmParams base{};
     base.ws = sc.tc_ws; base.counters = sc.tc_counters; base.status = status;
@@ -356,7 +356,7 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             tc_decompose(p, up(d.d_model, 128 * mh), qd, T, kCtas);
             p.mh = mh; p.n_rows_total = d.d_model;
             p.mode = TC_RESID; p.N = d.d_model; p.sumsq_in_parts = 0;
-            p.gain = m.w(l, 5); p.x_hi = sc.xd_hi; p.x_lo = sc.xd_hi + d.d_model; p.ldx = 2 * d.d_model;
+            p.gain = m.w(l, 5); p.x_out = sc.xd; p.xk = d.d_model;
             p.sumsq_out = sc.sumsq_b;
             mp.a0 = wm.wo[ix(mh)][l]; mp.x = xa;
             g.push_back({mp, p, wb * d.d_model * qd});
@@ -366,7 +366,7 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             tc_decompose(p, up(d.d_ffn, 64 * mh), d.d_model, T, kCtas);
             p.mh = mh; p.n_rows_total = d.d_ffn;
             p.mode = TC_SWIGLU; p.N = d.d_ffn; p.sumsq_in = sc.sumsq_b; p.sumsq_in_parts = dt;
-            p.x_hi = sc.xf_hi; p.x_lo = sc.xf_hi + d.d_ffn; p.ldx = 2 * d.d_ffn;
+            p.x_out = sc.xf; p.xk = d.d_ffn;
             mp.a0 = wm.gate[ix(mh)][l]; mp.a1 = wm.up[ix(mh)][l]; mp.x = xd;
             g.push_back({mp, p, wb * 2.0 * d.d_ffn * d.d_model});
         }
@@ -376,7 +376,7 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             p.mh = mh; p.n_rows_total = d.d_model;
             p.mode = TC_RESID; p.N = d.d_model; p.sumsq_in_parts = 0;
             p.gain = (l + 1 < d.layers) ? m.w(l + 1, 0) : static_cast<const __nv_bfloat16*>(d.final_norm);
-            p.x_hi = sc.xd_hi; p.x_lo = sc.xd_hi + d.d_model; p.ldx = 2 * d.d_model; p.sumsq_out = sc.sumsq_a;
+            p.x_out = sc.xd; p.xk = d.d_model; p.sumsq_out = sc.sumsq_a;
             mp.a0 = wm.down[ix(mh)][l]; mp.x = xf;
             g.push_back({mp, p, wb * d.d_model * d.d_ffn});
         }
@@ -482,7 +482,7 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
     pa.B = B; pa.R = R; pa.max_depth = D; pa.n_nodes = n_nodes; pa.tok = tok; pa.parent = parent;
     const bool tc = ctx->use_tc && ctx->tmaps.ok && B * R <= TC_MAX_ROWS;
     if (tc) {
-        pa.gain0 = ctx->target.w(0, 0); pa.x_hi = ctx->sc.xd_hi; pa.x_lo = ctx->sc.xd_hi + ctx->target.d.d_model;
+        pa.gain0 = ctx->target.w(0, 0); pa.x = ctx->sc.xd; pa.terms = tc_terms(B * R);
         pa.sumsq_out = ctx->sc.sumsq_a;
     }
     RUN(MTAD_K_PREPARE, 0, 1, launch_prepare(ctx->target, ctx->st, ctx->rm, ctx->sc, pa, out->status, s));
@@ -607,12 +607,12 @@ int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, 
         (size_t)p.n_tiles > ctx->tc_counter_n)
         return MTAD_E_WORKSPACE;
     TcMaps mp{};
-    const int xbox = 2 * p.rpad > 256 ? p.rpad : 2 * p.rpad;
-    if (tc_make_map(&mp.a0, W, N, K, mh == 1 ? 128 : 256) || tc_make_map(&mp.x, ctx->sc.xf_hi, 2 * TC_X_ROWS, K, xbox))
+    const int xbox = p.terms * p.rpad > 256 ? p.terms * p.rpad / 2 : p.terms * p.rpad;
+    if (tc_make_map(&mp.a0, W, N, K, mh == 1 ? 128 : 256) || tc_make_map(&mp.x, ctx->sc.xf, 2 * TC_X_ROWS, K, xbox))
         return MTAD_E_CUDA;
     p.mode = TC_PLAIN; p.N = N; p.out = y; p.ldo = N;
     p.ws = ctx->sc.tc_ws; p.counters = ctx->sc.tc_counters; p.status = nullptr;
-    RUN(MTAD_K_PREPARE, 0, 1, launch_split_rows(x, K, ctx->sc.xf_hi, ctx->sc.xf_hi + K, 2 * K, T, K, s));
+    RUN(MTAD_K_PREPARE, 0, 1, launch_split_rows(x, K, ctx->sc.xf, p.terms, T, K, s));
     RUN(MTAD_K_GEMM, 2.0 * N * K, 1, launch_tc_gemm(mp, p, kCtas, false, s));
     return MTAD_OK;
 }

@@ -83,10 +83,11 @@ struct Scratch {
     float* row_lse;      // [T]
     int32_t* row_cand;   // [T]
     float* row_cand_lp;  // [T]
-    // tensor-core path: bf16 hi/lo operand rows, deferred-norm statistics, split-K workspace, LM-head partials
-    __nv_bfloat16 *xd_hi, *xd_lo;      // [256, d]   input of QKV / gate-up / LM head (un-normalised hidden * gain)
-    __nv_bfloat16 *xa_hi, *xa_lo;      // [256, Hq hd] attention output
-    __nv_bfloat16 *xf_hi, *xf_lo;      // [256, F]   SwiGLU output
+    // tensor-core path: bf16 operand rows (see store_terms), deferred-norm statistics, split-K workspace, LM-head
+    // partials
+    __nv_bfloat16* xd;   // [512, d]     input of QKV / gate-up / LM head (un-normalised hidden * gain)
+    __nv_bfloat16* xa;   // [512, Hq hd] attention output
+    __nv_bfloat16* xf;   // [512, F]     SwiGLU output
     float* sumsq_a;      // [tiles(d)][256] sums of squares of the hidden rows (after down proj / embedding)
     float* sumsq_b;      // [tiles(d)][256] the same after the O projection
     float* tc_ws;        // split-K partial tiles
@@ -119,6 +120,19 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// An fp32 activation enters the tensor-core GEMM as `terms` bf16 values whose sum is the activation to ~2^-17
+// relative (two terms) or to fp32 rounding (three).  The terms of row t are neighbouring rows of the operand
+// buffer: term j of element k lives at x[(t * terms + j) * K + k].
+int tc_terms(int T);       // terms used for a call of T rows: 3 while the three accumulators fit tensor memory twice
+__device__ __forceinline__ void store_terms(float y, __nv_bfloat16* x, size_t K, int terms) {
+    const __nv_bfloat16 h = __float2bfloat16_rn(y);
+    x[0] = h;
+    const float r = y - __bfloat162float(h);
+    const __nv_bfloat16 l = __float2bfloat16_rn(r);
+    x[K] = l;
+    if (terms == 3) x[2 * K] = __float2bfloat16_rn(r - __bfloat162float(l));
+}
+
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
@@ -136,7 +150,8 @@ struct PrepareArgs {
     const int32_t* parent;     // device [B, R-1] or nullptr (chain)
     // tensor-core path (null otherwise): first layer's norm gains, operand rows and row statistics to emit
     const __nv_bfloat16* gain0;
-    __nv_bfloat16 *x_hi, *x_lo;
+    __nv_bfloat16* x;
+    int terms;
     float* sumsq_out;
 };
 

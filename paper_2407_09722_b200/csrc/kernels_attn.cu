@@ -139,17 +139,17 @@ __global__ void __launch_bounds__(128) attn_partial_kernel(const float* __restri
 // the block, then every thread sums its output dimension over the splits with independent loads
 template <int HD>
 __global__ void attn_combine_kernel(const float* __restrict__ part, float* __restrict__ out, const int32_t* slot,
-                                    int Hq, int nsplit, __nv_bfloat16* __restrict__ x_hi,
-                                    __nv_bfloat16* __restrict__ x_lo) {
+                                    int Hq, int nsplit, __nv_bfloat16* __restrict__ x, int terms) {
     const int t = blockIdx.x, h = blockIdx.y, d = threadIdx.x;
     pdl_wait();
     pdl_trigger();
     const size_t idx = ((size_t)t * Hq + h) * HD + d;
-    const size_t xidx = ((size_t)2 * t * Hq + h) * HD + d;     // interleaved operand rows: hi at row 2t, lo at 2t + 1
+    const size_t xk = (size_t)Hq * HD;                          // operand rows of the O projection: see store_terms
+    const size_t xidx = (size_t)t * terms * xk + (size_t)h * HD + d;
     float* dst = out + idx;
     if (slot[t] < 0) {
         *dst = 0.f;
-        if (x_hi) { x_hi[xidx] = __float2bfloat16_rn(0.f); x_lo[xidx] = __float2bfloat16_rn(0.f); }
+        if (x) store_terms(0.f, x + xidx, xk, terms);
         return;
     }
     extern __shared__ float wsm[];                  // [nsplit] weights, then [1] the normaliser
@@ -180,11 +180,7 @@ __global__ void attn_combine_kernel(const float* __restrict__ part, float* __res
     __syncthreads();
     const float y = acc / wsm[nsplit];
     *dst = y;
-    if (x_hi) {      // operand rows of the O projection: bf16 hi + lo
-        const __nv_bfloat16 hb = __float2bfloat16_rn(y);
-        x_hi[xidx] = hb;
-        x_lo[xidx] = __float2bfloat16_rn(y - __bfloat162float(hb));
-    }
+    if (x) store_terms(y, x + xidx, xk, terms);
 }
 
 cudaError_t launch_attention(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int B, int R,
@@ -195,8 +191,8 @@ cudaError_t launch_attention(const ModelView& m, int layer, const RowMeta& rm, c
     const __nv_bfloat16* cache = static_cast<const __nv_bfloat16*>(m.d.kv_cache);
     dim3 cgrid(B * R, Hq);
     cudaError_t e = cudaSuccess;
-    __nv_bfloat16* xh = emit_split ? sc.xa_hi : nullptr;
-    __nv_bfloat16* xl = emit_split ? sc.xa_hi + (size_t)Hq * hd : nullptr;
+    __nv_bfloat16* xh = emit_split ? sc.xa : nullptr;
+    const int xl = tc_terms(B * R);
     if (hd == 128) {
         e = launch_pdl(attn_partial_kernel<128>, grid, dim3(128), 0, st, pdl, sc.qkv, ldq, cache, rm, sc.attn_part, layer, m.max_batch, Hq,
                                                        Hkv, (long long)m.d.kv_capacity, R, nsplit, chunk);
@@ -225,8 +221,8 @@ cudaError_t launch_attention_combine(const ModelView& m, const RowMeta& rm, cons
                                      bool emit_split, bool pdl, cudaStream_t st) {
     const int Hq = m.d.n_q_heads, hd = m.d.head_dim;
     dim3 cgrid(B * R, Hq);
-    __nv_bfloat16* xh = emit_split ? sc.xa_hi : nullptr;
-    __nv_bfloat16* xl = emit_split ? sc.xa_hi + (size_t)Hq * hd : nullptr;
+    __nv_bfloat16* xh = emit_split ? sc.xa : nullptr;
+    const int xl = tc_terms(B * R);
     if (hd == 128)
         return launch_pdl(attn_combine_kernel<128>, cgrid, dim3(128), (nsplit + 1) * sizeof(float), st, pdl, (const float*)sc.attn_part, sc.attn,
                           (const int32_t*)rm.slot, Hq, nsplit, xh, xl);

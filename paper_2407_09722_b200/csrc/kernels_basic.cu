@@ -139,15 +139,12 @@ __global__ void prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, i
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
         const float v = ok ? __bfloat162float(embed[(size_t)tok * d + i]) : 0.f;
         hidden[(size_t)t * d + i] = v;
-        if (a.x_hi) {
-            const float y = v * __bfloat162float(a.gain0[i]);
-            const __nv_bfloat16 h = __float2bfloat16_rn(y);
-            a.x_hi[(size_t)t * 2 * d + i] = h;                      // interleaved operand rows: stride 2 d
-            a.x_lo[(size_t)t * 2 * d + i] = __float2bfloat16_rn(y - __bfloat162float(h));
+        if (a.x) {
+            store_terms(v * __bfloat162float(a.gain0[i]), a.x + (size_t)t * a.terms * d + i, d, a.terms);
             ss += v * v;
         }
     }
-    if (a.x_hi) {
+    if (a.x) {
         __shared__ float red[32];
         ss = block_sum(ss, red);
         if (threadIdx.x == 0) a.sumsq_out[t] = ss;

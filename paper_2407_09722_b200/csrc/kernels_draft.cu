@@ -40,8 +40,8 @@ __device__ __forceinline__ bool before(const Cand& a, const Cand& b) {     // a 
 __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, int vocab, int hd,
                                      double rope_base, SeqState s, DraftState ds, RowMeta rm,
                                      float* __restrict__ hidden, float* __restrict__ rope, SeqList seqs, int R, int step,
-                                     int beam, const __nv_bfloat16* __restrict__ gain0, __nv_bfloat16* x_hi,
-                                     __nv_bfloat16* x_lo, float* sumsq_out) {
+                                     int beam, const __nv_bfloat16* __restrict__ gain0, __nv_bfloat16* x, int terms,
+                                     float* sumsq_out) {
     const int t = blockIdx.x, bi = t / R, r = t % R;
     const int seq = seqs.v[bi];
     __shared__ int sh_tok, sh_pos, sh_ok;
@@ -101,15 +101,12 @@ __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, in
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
         const float v = ok ? __bfloat162float(embed[(size_t)tok * d + i]) : 0.f;
         hidden[(size_t)t * d + i] = v;
-        if (x_hi) {
-            const float y = v * __bfloat162float(gain0[i]);
-            const __nv_bfloat16 h = __float2bfloat16_rn(y);
-            x_hi[(size_t)t * 2 * d + i] = h;
-            x_lo[(size_t)t * 2 * d + i] = __float2bfloat16_rn(y - __bfloat162float(h));
+        if (x) {
+            store_terms(v * __bfloat162float(gain0[i]), x + (size_t)t * terms * d + i, d, terms);
             ss += v * v;
         }
     }
-    if (x_hi) {
+    if (x) {
         __shared__ float red[32];
         ss = wsum(ss);
         if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
@@ -134,8 +131,8 @@ cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const Dr
                                  cudaStream_t st) {
     draft_prepare_kernel<<<B * R, 128, 0, st>>>(
         static_cast<const __nv_bfloat16*>(m.d.embed), m.d.d_model, m.d.vocab, m.d.head_dim, (double)m.d.rope_base, s, ds,
-        rm, sc.hidden, sc.rope, seqs, R, step, beam, tc ? m.w(0, 0) : nullptr, tc ? sc.xd_hi : nullptr,
-        tc ? sc.xd_hi + m.d.d_model : nullptr, sc.sumsq_a);
+        rm, sc.hidden, sc.rope, seqs, R, step, beam, tc ? m.w(0, 0) : nullptr, tc ? sc.xd : nullptr,
+        tc_terms(B * R), sc.sumsq_a);
     return cudaGetLastError();
 }
 

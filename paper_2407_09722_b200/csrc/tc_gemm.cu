@@ -1,11 +1,13 @@
 // Tensor-core weight-streaming GEMM for the skinny projections of the verification step.
 //
-//   acc[n, r] = sum_k W[n, k] * (x_hi[r, k] + x_lo[r, k])          n: output feature, r: draft row
+//   acc[n, r] = sum_k W[n, k] * (x_0[r, k] + x_1[r, k] (+ x_2[r, k]))      n: output feature, r: draft row
 //
 // The weight matrix is the 128-row MMA operand (A), the draft rows are the MMA N dimension (B), both K-major bf16
 // tiles of 64 elements (one 128-byte swizzled row) brought in by TMA; fp32 accumulators live in tensor memory.
-// The fp32 activations arrive split into bf16 hi + lo rows, so the tensor cores see them to ~2^-17 relative;
-// the two products accumulate into the same TMEM columns.  Work is cut into (tile, k-block) units dealt out
+// The fp32 activations arrive split into two or three bf16 terms (x_0 = bf16(x), x_1 = bf16(x - x_0), ...): with
+// three the tensor cores see the fp32 value itself, with two (row counts whose three accumulators would not fit
+// tensor memory) ~2^-17 relative.  Every term is a row of the MMA's N dimension with an fp32 accumulator column
+// of its own; the drain adds a row's columns.  Work is cut into (tile, k-block) units dealt out
 // evenly to the CTAs (one per SM); a tile whose k-range spans several CTAs is completed by whichever of them
 // arrives last, which sums the partial tiles in CTA order (deterministic) and runs the fused epilogue.
 //
@@ -124,12 +126,12 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
+// two-term split of the query rows for the tensor-core attention
 __device__ __forceinline__ void split_store(float y, __nv_bfloat16* hi, __nv_bfloat16* lo) {
     const __nv_bfloat16 h = __float2bfloat16_rn(y);
     *hi = h;
     *lo = __float2bfloat16_rn(y - __bfloat162float(h));
 }
-
 
 // Weight boxes of one stage: how many, and for box b of a tile which map (0..2), which row coordinate and which
 // row offset inside the stage.  SwiGLU tiles take their first half from the gate matrix and their second half
@@ -269,7 +271,7 @@ __device__ __forceinline__ void epi_resid(const TcGemmParams& p, const Smem& s, 
         if (ok && t < p.T) {
             y = __ldcg(p.hidden + (size_t)t * p.N + n) + epi[j][e];
             p.hidden[(size_t)t * p.N + n] = y;
-            split_store(y * g, p.x_hi + (size_t)t * p.ldx + n, p.x_lo + (size_t)t * p.ldx + n);
+            store_terms(y * g, p.x_out + (size_t)t * p.terms * p.xk + n, p.xk, p.terms);
         }
         float sq = y * y;
 #pragma unroll
@@ -291,8 +293,7 @@ __device__ __forceinline__ void epi_swiglu(const TcGemmParams& p, const Smem& s,
         if (f >= p.N) return;
         for (int j = 0; j < EPI_ROWS && r0 + j < p.T; ++j) {
             const float g = s.epi[0][j][e], u = s.epi[0][j][e + 64];
-            split_store(g / (1.f + expf(-g)) * u, p.x_hi + (size_t)(r0 + j) * p.ldx + f,
-                        p.x_lo + (size_t)(r0 + j) * p.ldx + f);
+            store_terms(g / (1.f + expf(-g)) * u, p.x_out + (size_t)(r0 + j) * p.terms * p.xk + f, p.xk, p.terms);
         }
         return;
     }
@@ -302,8 +303,7 @@ __device__ __forceinline__ void epi_swiglu(const TcGemmParams& p, const Smem& s,
         if (f >= p.N) break;
         for (int j = 0; j < EPI_ROWS && r0 + j < p.T; ++j) {
             const float g = s.epi[h][j][e], u = s.epi[h + hh][j][e];
-            split_store(g / (1.f + expf(-g)) * u, p.x_hi + (size_t)(r0 + j) * p.ldx + f,
-                        p.x_lo + (size_t)(r0 + j) * p.ldx + f);
+            store_terms(g / (1.f + expf(-g)) * u, p.x_out + (size_t)(r0 + j) * p.terms * p.xk + f, p.xk, p.terms);
         }
     }
 }
@@ -372,7 +372,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
     const TcGemmParams& p0 = ch.p[0];
     const int mh = p0.mh;                              // 128-row weight halves per stage (1, 2 or 4), same in every phase
     const int a_bytes = mh * TC_TILE_N * 128;
-    const int acc_cols = 2 * p0.rpad;                  // one column per operand row: hi and lo of a draft row are neighbours
+    const int terms = p0.terms;
+    const int acc_cols = terms * p0.rpad;              // one column per operand row: the terms of a draft row are neighbours
     const int n_bbox = acc_cols > 256 ? 2 : 1;         // TMA boxes (and MMAs per k step and half) that cover the operand rows
     const int bbox_rows = acc_cols / n_bbox;
     const int stage_bytes = a_bytes + acc_cols * 128;
@@ -599,14 +600,29 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                 const int slot_idx = (int)blockIdx.x - c_first;
                 float* part = p.ws + ((size_t)tile * p.max_contrib + slot_idx) * part_floats;
                 for (int h = 0; h < mh; ++h) {
-                    for (int c0 = 0; c0 < 2 * T; c0 += 16) {
-                        float v[16];
-                        tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) +
-                                    (uint32_t)(buf * mh * acc_cols + h * acc_cols + c0), v);
+                    const uint32_t t_acc = tmem_base + ((uint32_t)(quad * 32) << 16) +
+                                           (uint32_t)(buf * mh * acc_cols + h * acc_cols);
+                    float* dst = part + h * half_floats + feat;
+                    if (terms == 3) {
+                        for (int rb = 0; rb < T; rb += 16) {           // 16 rows = 48 accumulator columns
+                            float v[48];
+                            tc_ld16(t_acc + 3 * rb, v);
+                            tc_ld16(t_acc + 3 * rb + 16, v + 16);
+                            tc_ld16(t_acc + 3 * rb + 32, v + 32);
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const int r = (c0 >> 1) + j;
-                            if (r < T) part[h * half_floats + (size_t)r * TC_TILE_N + feat] = v[2 * j] + v[2 * j + 1];
+                            for (int j = 0; j < 16; ++j)
+                                if (rb + j < T)
+                                    dst[(size_t)(rb + j) * TC_TILE_N] = v[3 * j] + (v[3 * j + 1] + v[3 * j + 2]);
+                        }
+                    } else {
+                        for (int c0 = 0; c0 < 2 * T; c0 += 16) {
+                            float v[16];
+                            tc_ld16(t_acc + c0, v);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const int r = (c0 >> 1) + j;
+                                if (r < T) dst[(size_t)r * TC_TILE_N] = v[2 * j] + v[2 * j + 1];
+                            }
                         }
                     }
                 }
@@ -692,11 +708,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
     if (threadIdx.x == 0 && *abort_flag && p0.status) atomicOr(p0.status, MTAD_ST_TIMEOUT);
 }
 
-__global__ void split_rows_kernel(const float* __restrict__ x, int ldx_in, __nv_bfloat16* __restrict__ hi,
-                                  __nv_bfloat16* __restrict__ lo, int ld, int K) {
+__global__ void split_rows_kernel(const float* __restrict__ x, int ldx_in, __nv_bfloat16* __restrict__ out, int terms,
+                                  int K) {
     const int t = blockIdx.x;
     for (int k = threadIdx.x; k < K; k += blockDim.x)
-        split_store(x[(size_t)t * ldx_in + k], hi + (size_t)t * ld + k, lo + (size_t)t * ld + k);
+        store_terms(x[(size_t)t * ldx_in + k], out + (size_t)t * terms * K + k, K, terms);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -741,14 +757,23 @@ void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int ctas) {
     p.max_contrib = (p.k_blocks + p.units_per_cta - 1) / p.units_per_cta + 1;
     p.T = T;
     p.rpad = (T + 15) / 16 * 16;
+    p.terms = tc_terms(T);
+}
+
+int tc_terms(int T) {
+    // three terms while two accumulator buffers of 3 * rpad columns fit the 512 columns of tensor memory and the
+    // operand tile stays one TMA box / one MMA (N <= 256); MTAD_TC_TERMS=2 keeps two everywhere
+    static const int cap = getenv("MTAD_TC_TERMS") ? atoi(getenv("MTAD_TC_TERMS")) : 3;
+    const int rpad = (T + 15) / 16 * 16;
+    return (cap >= 3 && rpad <= 80) ? 3 : 2;
 }
 
 int tc_halves(int T) {
-    // TMEM holds 2 buffers x halves x 2 * rpad columns <= 512; two halves (two MMA-issuing warps) already keep the
-    // tensor pipe ahead of HBM, and smaller stages fill and drain faster than 512-row ones
+    // TMEM holds 2 buffers x halves x terms * rpad columns <= 512; two halves (two MMA-issuing warps) already keep
+    // the tensor pipe ahead of HBM, and smaller stages fill and drain faster than 512-row ones
     static const int cap = getenv("MTAD_TC_MH") ? atoi(getenv("MTAD_TC_MH")) : 2;
-    const int rpad = (T + 15) / 16 * 16;
-    const int fit = rpad <= 32 ? 4 : (rpad <= 64 ? 2 : 1);
+    const int cols = tc_terms(T) * ((T + 15) / 16 * 16);
+    const int fit = cols <= 64 ? 4 : (cols <= 128 ? 2 : 1);
     return fit < cap ? fit : cap;
 }
 
@@ -761,9 +786,11 @@ cudaError_t launch_tc_chain(const TcChain& chain_in, bool pdl, cudaStream_t st) 
     if (ch.n_phases < 1 || ch.n_phases > TC_MAX_PHASES) return cudaErrorInvalidValue;
     const TcGemmParams& f = ch.p[0];
     if (f.mh != 1 && f.mh != 2 && f.mh != 4) return cudaErrorInvalidValue;
-    if (f.mh * 2 * f.rpad > 512) return cudaErrorInvalidValue;
-    const int nbuf = (2 * f.mh * 2 * f.rpad <= 512) ? 2 : 1;
-    const int stage_bytes = f.mh * TC_TILE_N * 128 + 2 * f.rpad * 128;
+    if (f.terms != 2 && f.terms != 3) return cudaErrorInvalidValue;
+    const int acc_cols = f.terms * f.rpad;
+    if (f.mh * acc_cols > 512 || (acc_cols > 256 && acc_cols % 32)) return cudaErrorInvalidValue;
+    const int nbuf = (2 * f.mh * acc_cols <= 512) ? 2 : 1;
+    const int stage_bytes = f.mh * TC_TILE_N * 128 + acc_cols * 128;
     static const int budget_kb_env = getenv("MTAD_TC_SMEM_KB") ? atoi(getenv("MTAD_TC_SMEM_KB")) : 0;
     const size_t budget = (size_t)(budget_kb_env > 0 ? budget_kb_env : 226) * 1024;
     int stages = (int)((budget - SMEM_TAIL - 1024) / stage_bytes);
@@ -772,7 +799,7 @@ cudaError_t launch_tc_chain(const TcChain& chain_in, bool pdl, cudaStream_t st) 
     int grid = 1;
     for (int i = 0; i < ch.n_phases; ++i) {
         TcGemmParams& p = ch.p[i];
-        if (p.mh != f.mh || p.rpad != f.rpad || p.T != f.T) return cudaErrorInvalidValue;   // one ring, one TMEM layout
+        if (p.mh != f.mh || p.rpad != f.rpad || p.T != f.T || p.terms != f.terms) return cudaErrorInvalidValue;   // one ring, one TMEM layout
         p.nbuf = nbuf;
         p.stages = stages;
         grid = std::max(grid, (p.total_units + p.units_per_cta - 1) / p.units_per_cta);
@@ -808,9 +835,8 @@ cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p, int ctas, 
     return launch_tc_chain(ch, pdl, st);
 }
 
-cudaError_t launch_split_rows(const float* x, int ldx_in, __nv_bfloat16* hi, __nv_bfloat16* lo, int ld, int T, int K,
-                              cudaStream_t st) {
-    split_rows_kernel<<<T, 256, 0, st>>>(x, ldx_in, hi, lo, ld, K);
+cudaError_t launch_split_rows(const float* x, int ldx_in, __nv_bfloat16* out, int terms, int T, int K, cudaStream_t st) {
+    split_rows_kernel<<<T, 256, 0, st>>>(x, ldx_in, out, terms, K);
     return cudaGetLastError();
 }
 

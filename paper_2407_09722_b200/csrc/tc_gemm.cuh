@@ -24,7 +24,8 @@ struct TcGemmParams {
     // decomposition
     int n_tiles, k_blocks, total_units, units_per_cta, max_contrib;
     int T;                 // valid activation rows
-    int rpad;              // T rounded up to 16; the operand tile has 2 * rpad rows (hi and lo of a row are neighbours)
+    int rpad;              // T rounded up to 16; the operand tile has terms * rpad rows (the terms of a row are neighbours)
+    int terms;             // bf16 terms per activation row (2 or 3), the same for the rows read and the rows emitted
     int mh;                // 128-row weight halves per tile and stage (1 or 2); a tile is mh * 128 output features
     int nbuf;              // TMEM accumulator buffers (set by the launcher)
     int n_rows_total;      // weight rows, for skipping a half that lies beyond them
@@ -39,7 +40,7 @@ struct TcGemmParams {
     int* phase_done;
     int dep_feat;
     // split-K fix-up
-    float* ws;             // [n_tiles][max_contrib][mh][rpad][128] partial tiles
+    float* ws;             // [n_tiles][max_contrib][mh][rpad][128] partial tiles (terms already summed)
     int* counters;         // [n_tiles], zero between launches
     uint32_t* status;      // device status word for time-outs (may be null)
     // deferred RMSNorm of the input: rstd[r] = rsqrt(sum_parts / dim + eps); parts == 0 -> 1
@@ -63,9 +64,8 @@ struct TcGemmParams {
     // TC_RESID / TC_SWIGLU outputs
     float* hidden;                  // [T, N]
     const __nv_bfloat16* gain;      // [N] gains of the norm that follows (TC_RESID)
-    __nv_bfloat16* x_hi;            // operand rows for the next GEMM: row t of the hi part at x_hi + t * ldx,
-    __nv_bfloat16* x_lo;            // of the lo part at x_lo + t * ldx (interleaved buffer: x_lo = x_hi + K, ldx = 2 K)
-    int ldx;
+    __nv_bfloat16* x_out;           // operand rows for the next GEMM (layout of store_terms)
+    int xk;                         // their row length: the next GEMM's K
     float* sumsq_out;               // [n_tiles][TC_X_ROWS]
     // TC_LMHEAD
     float4* lm_part;                // [T][n_tiles] (max, sumexp, best value, best index bits)
@@ -78,7 +78,7 @@ struct TcGemmParams {
 
 struct TcMaps {
     CUtensorMap a0, a1, a2;         // weight maps (QKV: wq, wk, wv; SwiGLU: gate, up; else a0)
-    CUtensorMap x;                  // operand rows [2 * TC_X_ROWS, K]: row 2t = hi(t), row 2t + 1 = lo(t)
+    CUtensorMap x;                  // operand rows [2 * TC_X_ROWS, K]: row terms * t + j = term j of activation row t
 };
 
 // Up to four GEMMs that feed one another (O projection, gate/up, down, next layer's QKV) run as phases of one launch:
@@ -95,16 +95,15 @@ cudaError_t launch_tc_chain(const TcChain& chain, bool pdl, cudaStream_t st);
 // Encodes a 2-D bf16 tensor map (row-major [rows, cols], 128-byte swizzle, box [box_rows, 64]).
 int tc_make_map(CUtensorMap* out, const void* base, long long rows, long long cols, int box_rows);
 
-// Fills the decomposition fields of p for a problem of n_tiles x k_blocks on `ctas` CTAs.
+// Fills the decomposition fields of p (and p.terms = tc_terms(T)) for a problem of n_tiles x k_blocks on `ctas` CTAs.
 void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int ctas);
-// Weight halves per tile that fit tensor memory for T rows (2 up to 64 rows, else 1).
+// Weight halves per tile that fit tensor memory for T rows, given tc_terms(T) accumulator columns per row.
 int tc_halves(int T);
 size_t tc_workspace_floats(int n_tiles_max, int max_contrib_max, int rpad_max);
 
 cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p, int ctas, bool pdl, cudaStream_t st);
 
-// Splits fp32 rows into bf16 hi + lo operand rows (hi = bf16(x), lo = bf16(x - hi)).
-cudaError_t launch_split_rows(const float* x, int ldx_in, __nv_bfloat16* hi, __nv_bfloat16* lo, int ld, int T, int K,
-                              cudaStream_t st);
+// Splits fp32 rows [T, K] into operand rows of `terms` bf16 terms (layout of store_terms).
+cudaError_t launch_split_rows(const float* x, int ldx_in, __nv_bfloat16* out, int terms, int T, int K, cudaStream_t st);
 
 }  // namespace mtad
