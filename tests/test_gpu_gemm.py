@@ -24,7 +24,10 @@ def _check(dm, N, K, T, seed):
     ref = x.double() @ W.double().t()
     err = (y.double() - ref).abs().max().item()
     scale = ref.abs().max().item()
-    assert err <= 2e-5 * max(scale, 1.0), (N, K, T, err, scale)
+    # up to 80 rows the activations enter as three bf16 terms (exact): only fp32 accumulation error is left; beyond,
+    # two terms (~2^-17 relative per element)
+    tol = 4e-6 if T <= 80 else 2e-5
+    assert err <= tol * max(scale, 1.0), (N, K, T, err, scale)
 
 
 @pytest.mark.parametrize("N,K,T", [(128, 64, 1), (128, 256, 5), (256, 256, 16), (384, 688, 17), (200, 136, 3),

@@ -51,10 +51,21 @@ def test_13b_ragged_batch_four_layers():
     assert st.n_seq == 8
 
 
-@pytest.mark.xfail(strict=False, reason="decisions (eta, path, tokens) match, but at d = 8192 a handful of K/V elements "
-                   "round to the neighbouring bf16 value on one side only (the tensor-core path sees activations "
-                   "as bf16 hi + lo, ~2^-17 relative) and peaked attention over the draft rows amplifies them: "
-                   "max |d log p| is 5e-3 here against the 2e-3 bound")
+def test_70b_shape_chain_two_layers():
+    """The 8192-wide GQA model itself is inside the bound: same weights and cache length as the 70B tree case, with a
+    5-row chain instead of the 129-row tree."""
+    w = S.WORKLOADS["70b_gqa_tree"]
+    c = dataclasses.replace(S.WORKLOADS["7b_chain"], target=w.target, kv_len=w.kv_len)
+    shape = dataclasses.replace(w.target, layers=2)
+    st = _run(c, shape, max(w.kv_len) + 256, [0.1])
+    assert st.max_lp_err < 5e-4
+
+
+@pytest.mark.xfail(strict=False, reason="decisions (eta, path, tokens) match, but at d = 8192 a few K/V elements round "
+                   "to the neighbouring bf16 value (fp32 against fp64 accumulation) and the peaked attention over the "
+                   "draft rows at this width amplifies a flip to ~1e-3 in a row's output; the second layer cascades: "
+                   "max |d log p| is 5e-3 here against the 2e-3 bound (CUDA-core path: 5e-4; the same model with a "
+                   "5-row chain: 1e-4)")
 def test_70b_gqa_tree_two_layers():
     w = S.WORKLOADS["70b_gqa_tree"]
     shape = dataclasses.replace(w.target, layers=2)
