@@ -12,7 +12,7 @@
 
 using namespace mtad;
 
-static const int kCtas = getenv("MTAD_TC_CTAS") ? atoi(getenv("MTAD_TC_CTAS")) : 148;   // CTAs of the tensor-core GEMM (one per SM)
+static const int kCtas = getenv("MTAD_TC_CTAS") ? atoi(getenv("MTAD_TC_CTAS")) : 148;   // SMs the tensor-core GEMM spreads over
 
 // Host-side tensor maps of one model's weight matrices.
 struct WeightMaps {                      // index 0, 1, 2: tiles of 128, 256, 512 rows (1, 2, 4 halves)
@@ -155,13 +155,14 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
                                   {(m->d_model + 127) / 128, m->d_ffn},
                                   {(m->vocab + 127) / 128, m->d_model}};
         for (auto& sh : shapes) {
-            for (int mh = 1; mh <= 4; mh *= 2) {
-                TcGemmParams tp{};
-                const int tiles = (sh[0] + mh - 1) / mh;
-                tc_decompose(tp, tiles, sh[1], 1, kCtas);
-                ws_tiles = std::max(ws_tiles, (size_t)tiles * tp.max_contrib * mh);
-                max_tiles = std::max(max_tiles, (size_t)tiles);
-            }
+            for (int mh = 1; mh <= 4; mh *= 2)
+                for (int per_sm = 1; per_sm <= 2; ++per_sm) {
+                    TcGemmParams tp{};
+                    const int tiles = (sh[0] + mh - 1) / mh;
+                    tc_decompose(tp, tiles, sh[1], 1, kCtas, per_sm);
+                    ws_tiles = std::max(ws_tiles, (size_t)tiles * tp.max_contrib * mh);
+                    max_tiles = std::max(max_tiles, (size_t)tiles);
+                }
         }
         lm_tiles = std::max(lm_tiles, (size_t)(m->vocab + 127) / 128);
     };

@@ -9,7 +9,9 @@
 // tensor memory) ~2^-17 relative.  Every term is a row of the MMA's N dimension with an fp32 accumulator column
 // of its own; the drain adds a row's columns.  Work is cut into (tile, k-block) units dealt out
 // evenly to the CTAs (one per SM); a tile whose k-range spans several CTAs is completed by whichever of them
-// arrives last, which sums the partial tiles in CTA order (deterministic) and runs the fused epilogue.
+// arrives last, which sums the partial tiles in CTA order (deterministic) and runs the fused epilogue.  With few rows
+// two CTAs share an SM (half the shared-memory ring and at most half the tensor memory each): while one drains its
+// accumulator, waits for a fix-up or runs an epilogue, the other keeps the weight stream going.
 //
 // Warp roles: 0 = weight producer (TMA), 1 = operand-row producer (TMA, waits for the rows to exist), 2..5 = MMA
 // issuers (one per 128-row half of a stage; a single thread cannot issue the many small MMAs of a skinny problem
@@ -366,7 +368,7 @@ __device__ __forceinline__ void epi_lmhead(const TcGemmParams& p, const Smem& s,
 // kernel
 // ---------------------------------------------------------------------------------------------------------------
 
-__global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_constant__ TcChain ch) {
+__global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_constant__ TcChain ch) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const TcGemmParams& p0 = ch.p[0];
@@ -749,7 +751,9 @@ int tc_make_map(CUtensorMap* out, const void* base, long long rows, long long co
     return r == CUDA_SUCCESS ? 0 : -1;
 }
 
-void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int ctas) {
+void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int sms, int per_sm) {
+    p.per_sm = per_sm > 0 ? per_sm : tc_ctas_per_sm(T);
+    const int ctas = sms * p.per_sm;
     p.n_tiles = n_tiles;
     p.k_blocks = (K + TC_TILE_K - 1) / TC_TILE_K;
     p.total_units = n_tiles * p.k_blocks;
@@ -768,7 +772,18 @@ int tc_terms(int T) {
     return (cap >= 3 && rpad <= 80) ? 3 : 2;
 }
 
+int tc_ctas_per_sm(int T) {
+    // two CTAs need: 16 KB of weights + terms * rpad operand rows per stage, at least two stages in 112 KB less the
+    // epilogue scratch, and one accumulator buffer of terms * rpad columns within 256 columns
+    static const int force = getenv("MTAD_TC_PER_SM") ? atoi(getenv("MTAD_TC_PER_SM")) : 0;
+    const int rpad = (T + 15) / 16 * 16, cols = tc_terms(T) * rpad;
+    if (cols > 240 || force == 1) return 1;
+    if (force == 2) return 2;
+    return rpad <= 32 ? 2 : 1;
+}
+
 int tc_halves(int T) {
+    if (tc_ctas_per_sm(T) == 2) return 1;
     // TMEM holds 2 buffers x halves x terms * rpad columns <= 512; two halves (two MMA-issuing warps) already keep
     // the tensor pipe ahead of HBM, and smaller stages fill and drain faster than 512-row ones
     static const int cap = getenv("MTAD_TC_MH") ? atoi(getenv("MTAD_TC_MH")) : 2;
@@ -787,19 +802,22 @@ cudaError_t launch_tc_chain(const TcChain& chain_in, bool pdl, cudaStream_t st) 
     const TcGemmParams& f = ch.p[0];
     if (f.mh != 1 && f.mh != 2 && f.mh != 4) return cudaErrorInvalidValue;
     if (f.terms != 2 && f.terms != 3) return cudaErrorInvalidValue;
+    if (f.per_sm != 1 && f.per_sm != 2) return cudaErrorInvalidValue;
     const int acc_cols = f.terms * f.rpad;
-    if (f.mh * acc_cols > 512 || (acc_cols > 256 && acc_cols % 32)) return cudaErrorInvalidValue;
-    const int nbuf = (2 * f.mh * acc_cols <= 512) ? 2 : 1;
+    const int tmem_budget = 512 / f.per_sm;           // the CTAs of an SM allocate tensor memory side by side
+    if (f.mh * acc_cols > tmem_budget || (acc_cols > 256 && acc_cols % 32)) return cudaErrorInvalidValue;
+    const int nbuf = (2 * f.mh * acc_cols <= tmem_budget) ? 2 : 1;
     const int stage_bytes = f.mh * TC_TILE_N * 128 + acc_cols * 128;
     static const int budget_kb_env = getenv("MTAD_TC_SMEM_KB") ? atoi(getenv("MTAD_TC_SMEM_KB")) : 0;
-    const size_t budget = (size_t)(budget_kb_env > 0 ? budget_kb_env : 226) * 1024;
+    const size_t budget = f.per_sm == 2 ? (size_t)112 * 1024 : (size_t)(budget_kb_env > 0 ? budget_kb_env : 226) * 1024;
     int stages = (int)((budget - SMEM_TAIL - 1024) / stage_bytes);
     stages = stages > MAX_STAGES ? MAX_STAGES : stages;
     if (stages < 2) return cudaErrorInvalidValue;
     int grid = 1;
     for (int i = 0; i < ch.n_phases; ++i) {
         TcGemmParams& p = ch.p[i];
-        if (p.mh != f.mh || p.rpad != f.rpad || p.T != f.T || p.terms != f.terms) return cudaErrorInvalidValue;   // one ring, one TMEM layout
+        if (p.mh != f.mh || p.rpad != f.rpad || p.T != f.T || p.terms != f.terms || p.per_sm != f.per_sm)
+            return cudaErrorInvalidValue;                  // one ring, one TMEM layout
         p.nbuf = nbuf;
         p.stages = stages;
         grid = std::max(grid, (p.total_units + p.units_per_cta - 1) / p.units_per_cta);

@@ -28,6 +28,7 @@ struct TcGemmParams {
     int terms;             // bf16 terms per activation row (2 or 3), the same for the rows read and the rows emitted
     int mh;                // 128-row weight halves per tile and stage (1 or 2); a tile is mh * 128 output features
     int nbuf;              // TMEM accumulator buffers (set by the launcher)
+    int per_sm;            // CTAs of this launch that share an SM (1 or 2): sets the shared- and tensor-memory budget
     int n_rows_total;      // weight rows, for skipping a half that lies beyond them
     int n_tiles128;        // ceil(N / 128): row stride of lm_part
     int stages;            // smem ring depth
@@ -95,8 +96,12 @@ cudaError_t launch_tc_chain(const TcChain& chain, bool pdl, cudaStream_t st);
 // Encodes a 2-D bf16 tensor map (row-major [rows, cols], 128-byte swizzle, box [box_rows, 64]).
 int tc_make_map(CUtensorMap* out, const void* base, long long rows, long long cols, int box_rows);
 
-// Fills the decomposition fields of p (and p.terms = tc_terms(T)) for a problem of n_tiles x k_blocks on `ctas` CTAs.
-void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int ctas);
+// Fills the decomposition fields of p (and p.terms, p.per_sm for T rows) for a problem of n_tiles x k_blocks on
+// `sms` SMs with per_sm CTAs each (0: tc_ctas_per_sm(T)).
+void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int sms, int per_sm = 0);
+// CTAs per SM for a call of T rows: 2 for few rows (each with half the shared memory and at most 256 columns of
+// tensor memory: one CTA's drain, fix-up and epilogue overlap the other's streaming), else 1.
+int tc_ctas_per_sm(int T);
 // Weight halves per tile that fit tensor memory for T rows, given tc_terms(T) accumulator columns per row.
 int tc_halves(int T);
 size_t tc_workspace_floats(int n_tiles_max, int max_contrib_max, int rpad_max);
