@@ -1,7 +1,8 @@
 // Tree-masked attention of the draft rows against the KV cache on tensor cores (warp-level mma.sync, bf16 x bf16
 // -> fp32): the partial pass of the split-KV scheme.  One block owns (sequence, KV head, split of 64 keys): its K
 // and V rows arrive in shared memory with cp.async (16-byte pieces, XOR-swizzled so that ldmatrix is conflict
-// free) and every query row of the KV head's group - the draft rows of all its query heads, 16 per MMA tile - is
+// free; a block that walks several tiles keeps up to three in flight, and the tiles that hold only committed
+// positions are requested before the block waits for the kernel in front of it) and every query row of the KV head's group - the draft rows of all its query heads, 16 per MMA tile - is
 // run against them by one of the four warps.  fp32 queries and probabilities enter the tensor cores as bf16
 // hi + lo pairs (two MMAs), so only the cache's own bf16 rounding remains.  A row sees the committed positions
 // [0, L) and the draft rows among its ancestors and itself (Sec. 3.3 of the paper: tree attention).
@@ -58,7 +59,8 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
                                                           const __nv_bfloat16* __restrict__ q_lo,
                                                           const __nv_bfloat16* __restrict__ cache, RowMeta rm,
                                                           float* __restrict__ part, int layer, int max_batch, int Hq,
-                                                          int Hkv, long long cap, int R, int nsplit, int nslab, int nsp) {
+                                                          int Hkv, long long cap, int R, int nsplit, int nslab, int nsp,
+                                                          int nb, int early) {
     constexpr int ROWB = HD * 2;          // bytes of one key row
     constexpr int CPR = HD / 8;           // 16-byte pieces per row
     constexpr int NDT = HD / 8;           // 8-wide output tiles over the head dim
@@ -66,14 +68,15 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
     constexpr int PARK = HD + 8;          // row stride (floats) of a parked output tile
     constexpr float LN2 = 0.6931471805599453f;
     extern __shared__ __align__(128) uint8_t smem[];
-    // two K/V buffers of [KT][HD] bf16 each (piece c of row k stored at piece c ^ (k & 7)), then the query tiles
-    uint8_t* Qs = smem + 4 * KT * ROWB;               // nslab query tiles, same swizzle
+    // nb K/V buffers of [KT][HD] bf16 each (piece c of row k stored at piece c ^ (k & 7)), then the query tiles
+    uint8_t* Qs = smem + nb * 2 * KT * ROWB;          // nslab query tiles, same swizzle
     float* ml = reinterpret_cast<float*>(Qs + nslab * SLAB);           // [4 warps][16 rows][m, l]
 
     const int sp = blockIdx.x, g = blockIdx.y, bi = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    pdl_wait();          // q, the appended K/V rows and the row metadata come from the kernels before
-    pdl_trigger();
+    // q and the appended K/V rows come from the kernel before; with `early` the row metadata is older than that
+    // (any layer but the first), so the committed part of the cache can be requested before waiting for it
+    if (!early) { pdl_wait(); pdl_trigger(); }
     const int nrows = rm.n_rows[bi];
     if (nrows == 0) return;
     const int L = rm.kv_base[bi];
@@ -84,6 +87,7 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
     const int n_q = G * nrows;                        // query rows of this KV head: (head in group, draft row)
     if (tile_begin >= n_tiles) {
         // empty split: leave neutral partials so that the combine pass can read every split
+        if (early) { pdl_wait(); pdl_trigger(); }
         for (int i = threadIdx.x; i < n_q; i += blockDim.x) {
             const int h = g * G + i / nrows, r = i % nrows;
             float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
@@ -128,12 +132,27 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
             cp_async16(s_u32(Vd + soff), Vg + goff, valid);
         }
     };
+    // prologue: the first tiles of the block (one, or as many as the prefetch distance nb - 1)
+    const int pd = nb - 1;
+    const int n_pro = min(max(pd, 1), tile_end - tile_begin);
+    uint32_t asked = 0;
+    if (early) {
+        for (int j = 0; j < n_pro; ++j)
+            if ((tile_begin + j + 1) * KT <= L) {          // committed positions only
+                load_kv(tile_begin + j, j);
+                asked |= 1u << j;
+            }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        pdl_wait();
+        pdl_trigger();
+    }
     if (kparts > 1) {
         for (int mt = 0; mt < n_mt; ++mt) stage_q(mt, mt, threadIdx.x, blockDim.x);
     } else if (warp < n_mt) {
         stage_q(warp, warp, lane, 32);
     }
-    load_kv(tile_begin, 0);
+    for (int j = 0; j < n_pro; ++j)
+        if (!((asked >> j) & 1u)) load_kv(tile_begin + j, j);
     asm volatile("cp.async.commit_group;" ::: "memory");
 
     const int gq = lane >> 2, tq = lane & 3;          // fragment coordinates
@@ -147,11 +166,14 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
         for (int c = 0; c < 4; ++c) oacc[n][c] = 0.f;
 
   for (int tile = tile_begin; tile < tile_end; ++tile) {
-    const int buf = (tile - tile_begin) & 1;
-    if (tile + 1 < tile_end) {                        // prefetch the next tile while this one is computed
-        load_kv(tile + 1, buf ^ 1);
+    const int t = tile - tile_begin, buf = t % nb;
+    if (pd > 0) {
+        // request tile t + pd into the buffer tile t - 1 has left; one group per iteration (empty past the end), so
+        // that "all but the latest pd groups" always means "up to tile t"
+        if (tile + pd < tile_end) load_kv(tile + pd, (t + pd) % nb);
         asm volatile("cp.async.commit_group;" ::: "memory");
-        asm volatile("cp.async.wait_group 1;" ::: "memory");
+        if (t == 0 || pd == 1) asm volatile("cp.async.wait_group 1;" ::: "memory");   // t == 0: the whole prologue
+        else asm volatile("cp.async.wait_group 2;" ::: "memory");
     } else {
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
@@ -309,7 +331,7 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
                 *reinterpret_cast<float2*>(dst + 2 + n * 8 + 2 * tq) = make_float2(oacc[n][2], oacc[n][3]);
         }
     }
-    __syncthreads();                                  // this tile's buffer may be refilled two iterations on
+    __syncthreads();                                  // this tile's buffer is refilled by the next iteration's request
   }
     if (kparts > 1) {
         // ---- key-split tiles: park each warp's (m, l, o) over the K/V/Q area, then merge the parts in key order --
@@ -357,13 +379,23 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
     }
 }
 
+namespace {
+size_t attn_smem(int hd, int nslab, int nb) {
+    return (size_t)nb * 2 * KT * hd * 2 + (size_t)nslab * 2 * 16 * hd * 2 + 2048;
+}
+// K/V buffers of a block that walks several tiles: three (two tiles in flight behind the one being computed) when
+// two such blocks fit an SM, else two
+int attn_ring(int hd, int nslab) { return 2 * (attn_smem(hd, nslab, 3) + 1024) <= 228 * 1024 ? 3 : 2; }
+}  // namespace
+
 int attention_mma_tiles_per_block(const ModelView& m, int B, int R, long long keys) {
-    // with at most two query tiles per KV head a block walks several 64-key tiles (next tile prefetched while the
-    // current one is computed): about three blocks per SM in a single wave; larger trees take one tile per block
+    // with at most two query tiles per KV head a block walks several 64-key tiles, all blocks resident in a single
+    // wave (two per SM with a ring of three buffers at head_dim 128, else three); larger trees take one tile per block
     const int n_mt_max = ((m.d.n_q_heads / m.d.n_kv_heads) * R + 15) / 16;
     if (n_mt_max > 2) return 1;
+    const int per_sm = (attn_ring(m.d.head_dim, n_mt_max) == 3 && m.d.head_dim == 128) ? 2 : 3;
     const long long tiles = (keys + KT - 1) / KT * m.d.n_kv_heads * B;
-    const long long nsp = (tiles + 3 * 148 - 1) / (3 * 148);
+    const long long nsp = (tiles + per_sm * 148 - 1) / (per_sm * 148);
     return (int)(nsp < 1 ? 1 : (nsp > 64 ? 64 : nsp));
 }
 
@@ -374,24 +406,26 @@ cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& r
     // query tiles kept in shared memory: all of them (at most two) when the warps split keys, else one per warp
     const int n_mt_max = ((Hq / Hkv) * R + 15) / 16;
     const int nslab = n_mt_max <= 2 ? n_mt_max : 4;
-    const size_t smem = (size_t)4 * KT * hd * 2 + (size_t)nslab * 2 * 16 * hd * 2 + 2048;
+    const int nb = nsp == 1 ? 1 : (nsp == 2 ? 2 : attn_ring(hd, nslab));
+    const size_t smem = attn_smem(hd, nslab, nb);
+    const int early = layer > 0 ? 1 : 0;              // the row metadata was final before the previous kernel started
     dim3 grid(nsplit, Hkv, B);
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 102400);
+        cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 116 * 1024);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 102400);
+            e = cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 116 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     if (hd == 128)
         return launch_pdl(attn_mma_kernel<128>, grid, dim3(128), smem, st, pdl, (const __nv_bfloat16*)sc.q_hi,
                           (const __nv_bfloat16*)sc.q_lo, cache, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv,
-                          (long long)m.d.kv_capacity, R, nsplit, nslab, nsp);
+                          (long long)m.d.kv_capacity, R, nsplit, nslab, nsp, nb, early);
     if (hd == 64)
         return launch_pdl(attn_mma_kernel<64>, grid, dim3(128), smem, st, pdl, (const __nv_bfloat16*)sc.q_hi,
                           (const __nv_bfloat16*)sc.q_lo, cache, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv,
-                          (long long)m.d.kv_capacity, R, nsplit, nslab, nsp);
+                          (long long)m.d.kv_capacity, R, nsplit, nslab, nsp, nb, early);
     return cudaErrorInvalidValue;
 }
 
