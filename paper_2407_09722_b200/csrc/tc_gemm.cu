@@ -216,6 +216,8 @@ __device__ __forceinline__ void epi_plain(const TcGemmParams& p, EpiTile epi, in
     for (int j = 0; j < EPI_ROWS && r0 + j < p.T; ++j) p.out[(size_t)(r0 + j) * p.ldo + n] = epi[j][e];
 }
 
+// The epilogues below first issue the global loads of all EPI_ROWS rows, then compute: a finished tile is the end of
+// a dependency chain (the next kernel waits for it), so one L2 round trip per pass instead of one per row matters.
 __device__ __forceinline__ void epi_qkv(const TcGemmParams& p, EpiTile epi, int tile, int r0, int e) {
     const int hd = p.hd, half = hd >> 1;
     int seg, tin;
@@ -228,35 +230,45 @@ __device__ __forceinline__ void epi_qkv(const TcGemmParams& p, EpiTile epi, int 
     if (head >= heads) return;
     const int ldq = (p.Hq + 2 * p.Hkv) * hd;
     const float scale = rsqrtf((float)hd);
-    for (int j = 0; j < EPI_ROWS && r0 + j < p.T; ++j) {
+    const bool rot = seg != 2 && jin < half;          // this thread rotates the pair (jin, jin + half)
+    if (seg != 2 && !rot) return;
+    int sl[EPI_ROWS], sq[EPI_ROWS];
+    float2 cs[EPI_ROWS];
+#pragma unroll
+    for (int j = 0; j < EPI_ROWS; ++j) {
         const int t = r0 + j;
+        const bool valid = t < p.T;
+        sl[j] = (valid && seg != 0) ? p.slot[t] : (valid ? 0 : -1);
+        sq[j] = (valid && seg != 0) ? p.seq[t] : 0;
+        cs[j] = (valid && rot) ? *reinterpret_cast<const float2*>(p.rope + ((size_t)t * half + jin) * 2)
+                               : make_float2(1.f, 0.f);
+    }
+#pragma unroll
+    for (int j = 0; j < EPI_ROWS; ++j) {
+        const int t = r0 + j;
+        if (sl[j] < 0) continue;                      // row beyond T, or an inactive row (no cache slot)
         if (seg == 2) {
-            const int sl = p.slot[t];
-            if (sl < 0) continue;
-            const size_t base = (((((size_t)p.layer * p.max_batch + p.seq[t]) * 2 + 1) * p.Hkv + head) * p.cap + sl) * hd;
+            const size_t base = (((((size_t)p.layer * p.max_batch + sq[j]) * 2 + 1) * p.Hkv + head) * p.cap + sl[j]) * hd;
             p.cache[base + jin] = __float2bfloat16_rn(epi[j][e]);
-        } else if (jin < half) {
-            const float c = p.rope[((size_t)t * half + jin) * 2], sn = p.rope[((size_t)t * half + jin) * 2 + 1];
-            const float a = epi[j][e], b = epi[j][e + half];
-            const float ra = a * c - b * sn, rb = b * c + a * sn;
-            if (seg == 0) {
-                float* q = p.q_out + (size_t)t * ldq + head * hd;
-                q[jin] = ra * scale;
-                q[jin + half] = rb * scale;
-                if (p.q_hi) {
-                    // tensor-core attention operands: q * log2(e) / sqrt(hd) as bf16 hi + lo (softmax runs on exp2)
-                    const size_t o = (size_t)t * p.Hq * hd + head * hd;
-                    split_store(ra * scale * 1.4426950408889634f, p.q_hi + o + jin, p.q_lo + o + jin);
-                    split_store(rb * scale * 1.4426950408889634f, p.q_hi + o + jin + half, p.q_lo + o + jin + half);
-                }
-            } else {
-                const int sl = p.slot[t];
-                if (sl < 0) continue;
-                const size_t base =
-                    (((((size_t)p.layer * p.max_batch + p.seq[t]) * 2 + 0) * p.Hkv + head) * p.cap + sl) * hd;
-                p.cache[base + jin] = __float2bfloat16_rn(ra);
-                p.cache[base + jin + half] = __float2bfloat16_rn(rb);
+            continue;
+        }
+        const float c = cs[j].x, sn = cs[j].y;
+        const float a = epi[j][e], b = epi[j][e + half];
+        const float ra = a * c - b * sn, rb = b * c + a * sn;
+        if (seg == 0) {
+            float* q = p.q_out + (size_t)t * ldq + head * hd;
+            q[jin] = ra * scale;
+            q[jin + half] = rb * scale;
+            if (p.q_hi) {
+                // tensor-core attention operands: q * log2(e) / sqrt(hd) as bf16 hi + lo (softmax runs on exp2)
+                const size_t o = (size_t)t * p.Hq * hd + head * hd;
+                split_store(ra * scale * 1.4426950408889634f, p.q_hi + o + jin, p.q_lo + o + jin);
+                split_store(rb * scale * 1.4426950408889634f, p.q_hi + o + jin + half, p.q_lo + o + jin + half);
             }
+        } else {
+            const size_t base = (((((size_t)p.layer * p.max_batch + sq[j]) * 2 + 0) * p.Hkv + head) * p.cap + sl[j]) * hd;
+            p.cache[base + jin] = __float2bfloat16_rn(ra);
+            p.cache[base + jin + half] = __float2bfloat16_rn(rb);
         }
     }
 }
@@ -267,18 +279,27 @@ __device__ __forceinline__ void epi_resid(const TcGemmParams& p, const Smem& s, 
     const bool ok = n < p.N;
     const float g = ok ? __bfloat162float(p.gain[n]) : 0.f;
     const int warp = e >> 5, lane = e & 31;
+    float y[EPI_ROWS];
+#pragma unroll
+    for (int j = 0; j < EPI_ROWS; ++j)
+        y[j] = (ok && r0 + j < p.T) ? __ldcg(p.hidden + (size_t)(r0 + j) * p.N + n) : 0.f;
+#pragma unroll
     for (int j = 0; j < EPI_ROWS; ++j) {
         const int t = r0 + j;
-        float y = 0.f;
         if (ok && t < p.T) {
-            y = __ldcg(p.hidden + (size_t)t * p.N + n) + epi[j][e];
-            p.hidden[(size_t)t * p.N + n] = y;
-            store_terms(y * g, p.x_out + (size_t)t * p.terms * p.xk + n, p.xk, p.terms);
+            y[j] += epi[j][e];
+            p.hidden[(size_t)t * p.N + n] = y[j];
+            store_terms(y[j] * g, p.x_out + (size_t)t * p.terms * p.xk + n, p.xk, p.terms);
         }
-        float sq = y * y;
+        y[j] *= y[j];
+    }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-        if (lane == 0) s.red[warp * EPI_ROWS + j] = sq;
+    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+        for (int j = 0; j < EPI_ROWS; ++j) y[j] += __shfl_xor_sync(0xffffffffu, y[j], o);
+    if (lane == 0) {
+#pragma unroll
+        for (int j = 0; j < EPI_ROWS; ++j) s.red[warp * EPI_ROWS + j] = y[j];
     }
     epi_bar();
     if (e < EPI_ROWS && r0 + e < p.T)
@@ -315,29 +336,42 @@ __device__ __forceinline__ void epi_lmhead(const TcGemmParams& p, const Smem& s,
     const int v = tile * TC_TILE_N + e;
     const bool ok = v < p.N;
     const int warp = e >> 5, lane = e & 31;
+    float m[EPI_ROWS], sum[EPI_ROWS], bv[EPI_ROWS];
+    int bi[EPI_ROWS];
+#pragma unroll
+    for (int j = 0; j < EPI_ROWS; ++j) {              // the uniforms of all rows first
+        const int t = r0 + j;
+        bv[j] = (ok && t < p.T) ? p.uniforms[(size_t)(t / p.R) * p.N + v] : 0.5f;
+    }
+#pragma unroll
     for (int j = 0; j < EPI_ROWS; ++j) {
         const int t = r0 + j;
-        float m = -CUDART_INF_F, sum = 0.f, bv = -CUDART_INF_F;
-        int bi = 0x7fffffff;
         if (ok && t < p.T) {
             const float z = epi[j][e];
-            m = z;
-            sum = 1.f;
-            const float u = p.uniforms[(size_t)(t / p.R) * p.N + v];
-            bv = z - logf(-logf(u));
-            bi = v;
+            m[j] = z;
+            sum[j] = 1.f;
+            bv[j] = z - logf(-logf(bv[j]));
+            bi[j] = v;
+        } else {
+            m[j] = -CUDART_INF_F; sum[j] = 0.f; bv[j] = -CUDART_INF_F; bi[j] = 0x7fffffff;
         }
+    }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, sum, o);
-            const float v2 = __shfl_xor_sync(0xffffffffu, bv, o);
-            const int i2 = __shfl_xor_sync(0xffffffffu, bi, o);
-            const float mm = fmaxf(m, m2);
-            sum = (m == -CUDART_INF_F ? 0.f : sum * expf(m - mm)) + (m2 == -CUDART_INF_F ? 0.f : s2 * expf(m2 - mm));
-            m = mm;
-            if (v2 > bv || (v2 == bv && i2 < bi)) { bv = v2; bi = i2; }
+    for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+        for (int j = 0; j < EPI_ROWS; ++j) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, m[j], o), s2 = __shfl_xor_sync(0xffffffffu, sum[j], o);
+            const float v2 = __shfl_xor_sync(0xffffffffu, bv[j], o);
+            const int i2 = __shfl_xor_sync(0xffffffffu, bi[j], o);
+            const float mm = fmaxf(m[j], m2);
+            sum[j] = (m[j] == -CUDART_INF_F ? 0.f : sum[j] * expf(m[j] - mm)) + (m2 == -CUDART_INF_F ? 0.f : s2 * expf(m2 - mm));
+            m[j] = mm;
+            if (v2 > bv[j] || (v2 == bv[j] && i2 < bi[j])) { bv[j] = v2; bi[j] = i2; }
         }
-        if (lane == 0) s.red4[warp * EPI_ROWS + j] = make_float4(m, sum, bv, __int_as_float(bi));
+    }
+    if (lane == 0) {
+#pragma unroll
+        for (int j = 0; j < EPI_ROWS; ++j) s.red4[warp * EPI_ROWS + j] = make_float4(m[j], sum[j], bv[j], __int_as_float(bi[j]));
     }
     epi_bar();
     if (e < EPI_ROWS && r0 + e < p.T) {
