@@ -68,6 +68,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
+// Bounded wait until the arrival count of a tile (low 16 bits of its counter) reaches `want` (acquire at gpu scope).
+__device__ __forceinline__ bool arrivals_wait(const int* counter, int want, volatile int* abort_flag) {
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+        if ((v & 0xFFFF) >= want) return true;
+        __nanosleep(64);
+        if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
 // Bounded wait until a counter written by other CTAs of this launch reaches `want` (acquire at gpu scope).
 __device__ __forceinline__ bool flag_wait(const int* flag, int want, volatile int* abort_flag) {
     for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
@@ -667,15 +680,33 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
                 if (lane == 0) mbar_arrive(smem_u32(&s.tempty[buf]));   // MMA may reuse this accumulator
                 __threadfence();
                 epi_bar();
+                // Who finishes the tile.  Few rows (one pass): whoever arrives last.  More rows: the contributors for
+                // which this tile is the last of their run - all of them but, possibly, the last in CTA order, which
+                // met the tile at the start of its run - arrive within microseconds of one another at the end of the
+                // launch; each waits for the full count and takes every n_late-th pass of eight rows, so the passes
+                // (each a chain of L2 round trips) run side by side on several SMs.  Counter: arrivals in the low
+                // 16 bits, finished late contributors in the high 16.
+                const int run_end = min(((int)blockIdx.x + 1) * p.units_per_cta, p.total_units);
+                const bool c_last_late = min((c_last + 1) * p.units_per_cta, p.total_units) == (tile + 1) * KB;
+                const int n_late = (c_last - c_first) + (c_last_late ? 1 : 0);
+                const bool sliced = p.sliced && n_contrib > 1;
+                const bool late = u + len == run_end;
+                int pass0 = 0, pass_step = 1;
                 if (e == 0) {
                     const int old = atomicAdd(&p.counters[tile], 1);
-                    s.flags[0] = (old + 1 == n_contrib);
+                    int fin = (old + 1 == n_contrib) ? 1 : 0;
+                    if (sliced) fin = !late ? 0 : (arrivals_wait(&p.counters[tile], n_contrib, abort_flag) ? 1 : 2);
+                    s.flags[0] = fin;
                 }
                 epi_bar();
-                if (s.flags[0]) {
+                const int fin = s.flags[0];
+                epi_bar();                                  // flags[0] is rewritten by the next segment
+                if (fin == 2) { alive = false; break; }
+                if (sliced) { pass0 = slot_idx; pass_step = n_late; }
+                if (fin == 1) {
                     __threadfence();
                     const float* tile_ws = p.ws + (size_t)tile * p.max_contrib * part_floats;
-                    for (int r0 = 0; r0 < T; r0 += EPI_ROWS) {
+                    for (int r0 = pass0 * EPI_ROWS; r0 < T; r0 += pass_step * EPI_ROWS) {
                         for (int h = 0; h < mh; ++h) {
                             float acc[EPI_ROWS];
 #pragma unroll
@@ -717,8 +748,20 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
                         }
                         epi_bar();
                     }
-                    if (e == 0) p.counters[tile] = 0;          // ready for the next launch
-                    if (p.tile_done) {
+                    bool closer = true;                         // the one that leaves the tile's counter at zero
+                    if (sliced) {
+                        __threadfence();
+                        epi_bar();
+                        if (e == 0) {
+                            const int old = atomicAdd(&p.counters[tile], 0x10000);
+                            s.flags[0] = ((old >> 16) + 1 == n_late) ? 1 : 0;
+                        }
+                        epi_bar();
+                        closer = s.flags[0] != 0;
+                        epi_bar();
+                    }
+                    if (e == 0 && closer) p.counters[tile] = 0;          // ready for the next launch
+                    if (p.tile_done && closer) {
                         // publish the finished tile to the phase that reads it as operand rows
                         __threadfence();
                         epi_bar();
@@ -796,6 +839,10 @@ void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int sms, int per_s
     p.T = T;
     p.rpad = (T + 15) / 16 * 16;
     p.terms = tc_terms(T);
+    // more than one pass of eight rows: the passes of a tile are shared out among its contributors, which wait for
+    // one another - every CTA of the launch must be resident, i.e. at most one per SM slot
+    static const bool no_slice = getenv("MTAD_TC_SLICED") && atoi(getenv("MTAD_TC_SLICED")) == 0;
+    p.sliced = (T > EPI_ROWS && sms <= 148 && !no_slice) ? 1 : 0;
 }
 
 int tc_terms(int T) {

@@ -29,6 +29,7 @@ struct TcGemmParams {
     int mh;                // 128-row weight halves per tile and stage (1 or 2); a tile is mh * 128 output features
     int nbuf;              // TMEM accumulator buffers (set by the launcher)
     int per_sm;            // CTAs of this launch that share an SM (1 or 2): sets the shared- and tensor-memory budget
+    int sliced;            // 1: the passes of a finished tile are shared out among its contributors (more than 8 rows)
     int n_rows_total;      // weight rows, for skipping a half that lies beyond them
     int n_tiles128;        // ceil(N / 128): row stride of lm_part
     int stages;            // smem ring depth
