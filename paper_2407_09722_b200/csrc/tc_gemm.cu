@@ -349,39 +349,42 @@ __device__ __forceinline__ void epi_lmhead(const TcGemmParams& p, const Smem& s,
     const int v = tile * TC_TILE_N + e;
     const bool ok = v < p.N;
     const int warp = e >> 5, lane = e & 31;
-    float m[EPI_ROWS], sum[EPI_ROWS], bv[EPI_ROWS];
-    int bi[EPI_ROWS];
-#pragma unroll
-    for (int j = 0; j < EPI_ROWS; ++j) {              // the uniforms of all rows first
-        const int t = r0 + j;
-        bv[j] = (ok && t < p.T) ? p.uniforms[(size_t)(t / p.R) * p.N + v] : 0.5f;
-    }
+    // Gumbel noise of this token: one draw per sequence, shared by all its rows
+    float u[EPI_ROWS];
 #pragma unroll
     for (int j = 0; j < EPI_ROWS; ++j) {
         const int t = r0 + j;
-        if (ok && t < p.T) {
-            const float z = epi[j][e];
-            m[j] = z;
-            sum[j] = 1.f;
-            bv[j] = z - logf(-logf(bv[j]));
-            bi[j] = v;
-        } else {
-            m[j] = -CUDART_INF_F; sum[j] = 0.f; bv[j] = -CUDART_INF_F; bi[j] = 0x7fffffff;
-        }
+        const bool fresh = j == 0 || t / p.R != (t - 1) / p.R;
+        u[j] = (ok && t < p.T && fresh) ? p.uniforms[(size_t)(t / p.R) * p.N + v] : -1.f;
     }
+    float m[EPI_ROWS], sum[EPI_ROWS], bv[EPI_ROWS];
+    int bi[EPI_ROWS];
+    float gum = 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
+    for (int j = 0; j < EPI_ROWS; ++j) {
+        if (u[j] >= 0.f) gum = -logf(-logf(u[j]));
+        const bool valid = ok && r0 + j < p.T;
+        m[j] = valid ? epi[j][e] : -CUDART_INF_F;
+        bv[j] = valid ? m[j] + gum : -CUDART_INF_F;
+        bi[j] = valid ? v : 0x7fffffff;
+        sum[j] = m[j];                                // this thread's logit, kept for the sum below
+    }
+    // per row: maximum over the warp, then one exponential per thread and a sum; arg-max of the perturbed logits
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
         for (int j = 0; j < EPI_ROWS; ++j) {
-            const float m2 = __shfl_xor_sync(0xffffffffu, m[j], o), s2 = __shfl_xor_sync(0xffffffffu, sum[j], o);
+            m[j] = fmaxf(m[j], __shfl_xor_sync(0xffffffffu, m[j], o));
             const float v2 = __shfl_xor_sync(0xffffffffu, bv[j], o);
             const int i2 = __shfl_xor_sync(0xffffffffu, bi[j], o);
-            const float mm = fmaxf(m[j], m2);
-            sum[j] = (m[j] == -CUDART_INF_F ? 0.f : sum[j] * expf(m[j] - mm)) + (m2 == -CUDART_INF_F ? 0.f : s2 * expf(m2 - mm));
-            m[j] = mm;
             if (v2 > bv[j] || (v2 == bv[j] && i2 < bi[j])) { bv[j] = v2; bi[j] = i2; }
         }
-    }
+#pragma unroll
+    for (int j = 0; j < EPI_ROWS; ++j) sum[j] = (sum[j] == -CUDART_INF_F) ? 0.f : expf(sum[j] - m[j]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+        for (int j = 0; j < EPI_ROWS; ++j) sum[j] += __shfl_xor_sync(0xffffffffu, sum[j], o);
     if (lane == 0) {
 #pragma unroll
         for (int j = 0; j < EPI_ROWS; ++j) s.red4[warp * EPI_ROWS + j] = make_float4(m[j], sum[j], bv[j], __int_as_float(bi[j]));
