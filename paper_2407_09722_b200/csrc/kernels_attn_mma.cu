@@ -118,18 +118,30 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
             cp_async16(s_u32(dst + which * 16 * ROWB + row * ROWB + ((c ^ (row & 7)) << 4)), src, valid);
         }
     };
-    // K and V rows of one 64-key tile -> buffer `buf` (zero-filled past the last key)
+    // K and V rows of one 64-key tile -> buffer `buf` (zero-filled past the last key).  Thread i copies piece
+    // i % CPR of the keys i / CPR + k * (128 / CPR): its swizzled piece index is the same for all of them.
+    constexpr int KSTEP = 128 / CPR;                  // keys between two copies of a thread
+    const int ld_key = threadIdx.x / CPR, ld_c = threadIdx.x % CPR;
+    const uint32_t ld_soff = ld_key * ROWB + ((ld_c ^ (ld_key & 7)) << 4);
+    static_assert(KSTEP % 8 == 0, "the swizzle of a thread's pieces must not change from copy to copy");
     auto load_kv = [&](int tile, int buf) {
         const int kb = tile * KT;
-        uint8_t* Kd = smem + buf * (2 * KT * ROWB);
-        uint8_t* Vd = Kd + KT * ROWB;
-        for (int i = threadIdx.x; i < KT * CPR; i += blockDim.x) {
-            const int key = i / CPR, c = i % CPR;
-            const bool valid = kb + key < nkeys;
-            const size_t goff = (size_t)(valid ? kb + key : 0) * HD + c * 8;
-            const uint32_t soff = key * ROWB + ((c ^ (key & 7)) << 4);
-            cp_async16(s_u32(Kd + soff), Kg + goff, valid);
-            cp_async16(s_u32(Vd + soff), Vg + goff, valid);
+        const uint32_t Kd = s_u32(smem + buf * (2 * KT * ROWB)) + ld_soff, Vd = Kd + KT * ROWB;
+        const __nv_bfloat16* kg = Kg + (size_t)(kb + ld_key) * HD + ld_c * 8;
+        const __nv_bfloat16* vg = Vg + (size_t)(kb + ld_key) * HD + ld_c * 8;
+        if (kb + KT <= nkeys) {                       // whole tile valid
+#pragma unroll
+            for (int k = 0; k < KT / KSTEP; ++k) {
+                cp_async16(Kd + k * KSTEP * ROWB, kg + (size_t)k * KSTEP * HD, true);
+                cp_async16(Vd + k * KSTEP * ROWB, vg + (size_t)k * KSTEP * HD, true);
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < KT / KSTEP; ++k) {
+                const bool valid = kb + ld_key + k * KSTEP < nkeys;
+                cp_async16(Kd + k * KSTEP * ROWB, valid ? kg + (size_t)k * KSTEP * HD : Kg, valid);
+                cp_async16(Vd + k * KSTEP * ROWB, valid ? vg + (size_t)k * KSTEP * HD : Vg, valid);
+            }
         }
     };
     // prologue: the first tiles of the block (one, or as many as the prefetch distance nb - 1)
