@@ -8,15 +8,16 @@
 // three the tensor cores see the fp32 value itself, with two (row counts whose three accumulators would not fit
 // tensor memory) ~2^-17 relative.  Every term is a row of the MMA's N dimension with an fp32 accumulator column
 // of its own; the drain adds a row's columns.  Work is cut into (tile, k-block) units dealt out
-// evenly to the CTAs (one per SM); a tile whose k-range spans several CTAs is completed by whichever of them
-// arrives last, which sums the partial tiles in CTA order (deterministic) and runs the fused epilogue.  With few rows
+// evenly to the CTAs; a tile whose k-range spans several CTAs is completed by whichever of them arrives last, which
+// sums the partial tiles in CTA order (deterministic) and runs the fused epilogue - with more than eight rows by all
+// the contributors whose run ends in the tile, each taking every n-th pass of eight rows.  With few rows
 // two CTAs share an SM (half the shared-memory ring and at most half the tensor memory each): while one drains its
 // accumulator, waits for a fix-up or runs an epilogue, the other keeps the weight stream going.
 //
 // Warp roles: 0 = weight producer (TMA), 1 = operand-row producer (TMA, waits for the rows to exist), 2..5 = MMA
 // issuers (one per 128-row half of a stage; a single thread cannot issue the many small MMAs of a skinny problem
 // fast enough), 6..9 = epilogue (one TMEM lane quadrant each).
-// Every wait on an mbarrier is bounded; on a time-out the kernel raises MTAD_ST_TIMEOUT, waits (bounded) for its
+// Every wait on an mbarrier or on another CTA's counter is bounded; on a time-out the kernel raises MTAD_ST_TIMEOUT, waits (bounded) for its
 // own copies in flight, frees its tensor memory and returns.
 #include <math_constants.h>
 
