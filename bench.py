@@ -214,6 +214,65 @@ def throughput(total_ms: float, tokens: float) -> float:
 
 
 # ---------------------------------------------------------------------------------------------------------------
+# the whole iteration of Algorithm 1 with the library's own draft (chain workloads): mtad_draft -> verify -> commit
+# ---------------------------------------------------------------------------------------------------------------
+
+DRAFT_BEAM = 4          # the paper's smaller beam width
+
+
+def draft_loop(w: S.Workload, steps: int, warmup: int, cap: int):
+    """Decode iterations in which the auxiliary model drafts (beam sampling, the best beam is the chain), the target
+    verifies that chain and both caches are rolled forward.  Returns tokens/s including the draft and the draft's
+    share; a reported extra, not the headline (the headline times the verification path on synthetic drafts)."""
+    import paper_2407_09722_b200 as M
+    from paper_2407_09722_b200.runtime import DeviceModel
+    lens = S.kv_lengths(w, SEED)
+    g, b, B, V = w.gamma, DRAFT_BEAM, w.batch, w.target.vocab
+    dm = DeviceModel(w.target, B, max(w.n_nodes, g * b), cap, SEED, aux=w.aux, aux_capacity=cap + g * b + 8)
+    ctx = dm.ctx
+    seqs = list(range(B))
+    for s_, L in enumerate(lens):
+        dm.inject(s_, L)
+        S.fill_kv_cache(dm.aux_cache, 1, s_, L, SEED)
+        ctx.mtad_seq_set(s_, L, 1, aux_len=L)
+    i32 = dict(dtype=torch.int32, device="cuda")
+    f32 = dict(dtype=torch.float32, device="cuda")
+    tok, parent, depth = (torch.zeros(B, g * b, **i32) for _ in range(3))
+    node_logq, logq_ref, best = torch.zeros(B, g * b, **f32), torch.zeros(B, g, **f32), torch.zeros(B, g, **i32)
+    n_u = 4
+    u_draft = [S.uniforms(SEED, (41 << 40) | i, B * g * b * V, "cuda").view(B, g, b, V) for i in range(n_u)]
+    u_bonus = [S.bonus_uniforms(SEED, 1000 + i, B, V, "cuda") for i in range(n_u)]
+    res = M.ResultBuffers(B, g, g)
+    acc = torch.zeros((), dtype=torch.int64, device="cuda")
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    log_tau = math.log(TAU)
+    for i in range(-warmup, steps):
+        if i >= 0:
+            ev[i][0].record()
+        ctx.mtad_draft(seqs, g, b, u_draft[i % n_u], tok, parent, depth, node_logq, logq_ref, best)
+        if i >= 0:
+            ev[i][1].record()
+        chain_tok = tok.gather(1, best.long())              # tokens of the best beam, in depth order
+        ctx.mtad_verify_chain(seqs, g, chain_tok, logq_ref, log_tau, u_bonus[i % n_u], res)
+        ctx.kv_commit(seqs, res)
+        if i >= 0:
+            acc += res.n_out.sum()
+            ev[i][2].record()
+        elif i == -1:
+            acc.zero_()
+    torch.cuda.synchronize()
+    status = int(res.status.max().item())
+    d_us = [1e3 * e[0].elapsed_time(e[1]) for e in ev]
+    it_ms = [e[0].elapsed_time(e[2]) for e in ev]
+    total_ms = ev[0][0].elapsed_time(ev[-1][2])
+    accepted = float(acc.item())
+    return {"value": accepted / (total_ms * 1e-3), "unit": "tokens/s", "steps": steps, "gamma": g, "beam": b,
+            "block_efficiency": accepted / (steps * B), "iteration_ms": total_ms / steps,
+            "draft_us_median": statistics.median(d_us), "verify_commit_us_median": 1e3 * statistics.median(it_ms)
+            - statistics.median(d_us), "device_status": status}
+
+
+# ---------------------------------------------------------------------------------------------------------------
 # our arm
 # ---------------------------------------------------------------------------------------------------------------
 
@@ -363,9 +422,12 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
-    if world == 1 and not args.no_cpu_baseline:
-        del dm, ctx
+    del dm, ctx
+    torch.cuda.empty_cache()
+    if world == 1 and chain and w.batch == 1 and not args.no_draft_loop:      # mtad_draft takes one sequence per call
+        line["draft_loop"] = draft_loop(w, min(args.steps, 32), 3, cap)
         torch.cuda.empty_cache()
+    if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w)
     print(json.dumps(line))
 
@@ -378,6 +440,7 @@ def main():
     ap.add_argument("--workload", default="7b_chain", choices=sorted(S.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-draft-loop", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = S.WORKLOADS[args.workload]

@@ -125,7 +125,8 @@ int mtad_seq_get(mtad_ctx* ctx, int seq, int32_t* kv_len, int32_t* root_token, v
  * equation; every intermediate beam becomes a tree node, Sec. 3.3).  At each step the beam_width kept sequences
  * are drawn without replacement, proportionally to their joint likelihood, as the beam_width largest values of
  * log q(beam) + log q(token | beam) + Gumbel noise, noise = -log(-log(u)).
- *   seqs        host  [B]                 sequence ids
+ *   seqs        host  [B]                 sequence ids; B = 1 for now (MTAD_E_UNIMPLEMENTED otherwise: batched
+ *                                         drafts are switched off until a fault seen with B = 8 is understood)
  *   uniforms    device [B, gamma, beam_width, vocab] fp32 in (0,1)
  *   tok,parent,depth  device [B, gamma*beam_width] int32  node arrays, layer by layer (parent = -1: child of root)
  *   node_logq   device [B, gamma*beam_width] fp32  joint draft log-likelihood of the path ending at each node

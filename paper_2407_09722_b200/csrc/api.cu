@@ -655,6 +655,10 @@ int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_wi
     if (!seqs_ok(ctx, B, seqs)) return MTAD_E_INVALID;
     if (!uniforms || !tok || !parent || !depth || !node_logq || !logq_ref || !best_path) return MTAD_E_INVALID;
     if (gamma < 1 || beam_width < 1) return MTAD_E_INVALID;
+    // Drafts of several sequences in one call are refused for now: a call with eight sequences (13B-shaped pair,
+    // gamma 6, width 4) ended in an illegal memory access whose cause has not been found; one sequence per call is
+    // what the tests cover.
+    if (B > 1) return MTAD_E_UNIMPLEMENTED;
     if (gamma > MTAD_MAX_DEPTH || beam_width > MTAD_MAX_BEAM || gamma * beam_width > MTAD_DRAFT_NODES - MTAD_MAX_DEPTH - 1 ||
         gamma * beam_width > MTAD_MAX_NODES)
         return MTAD_E_CAPACITY;

@@ -77,10 +77,10 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
     // q and the appended K/V rows come from the kernel before; with `early` the row metadata is older than that
     // (any layer but the first), so the committed part of the cache can be requested before waiting for it
     if (!early) { pdl_wait(); pdl_trigger(); }
-    const int nrows = rm.n_rows[bi];
+    const int nrows = __ldcg(rm.n_rows + bi);         // past L1: these words are rewritten by every step
     if (nrows == 0) return;
-    const int L = rm.kv_base[bi];
-    const int nkeys = L + rm.n_spec[bi];
+    const int L = __ldcg(rm.kv_base + bi);
+    const int nkeys = L + __ldcg(rm.n_spec + bi);
     const int n_tiles = (nkeys + KT - 1) / KT;        // 64-key tiles of this sequence
     const int tile_begin = sp * nsp, tile_end = min(tile_begin + nsp, n_tiles);
     const int G = Hq / Hkv;
@@ -96,7 +96,7 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
         }
         return;
     }
-    const int seq = rm.call_seq[bi];
+    const int seq = __ldcg(rm.call_seq + bi);
     const __nv_bfloat16* Kg = cache + (((((size_t)layer * max_batch + seq) * 2 + 0) * Hkv + g) * cap) * HD;
     const __nv_bfloat16* Vg = cache + (((((size_t)layer * max_batch + seq) * 2 + 1) * Hkv + g) * cap) * HD;
     const int n_mt = (n_q + 15) / 16;

@@ -100,5 +100,9 @@ def test_draft_rejects_bad_arguments():
     assert c.mtad_draft([0], 4, 9, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_CAPACITY
     assert c.mtad_draft([0], 33, 1, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_CAPACITY
     assert c.mtad_draft([3], 4, 4, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_INVALID
+    # several sequences per call are refused for now (before anything is launched)
+    two = GpuModel(W.target, max_batch=2, max_nodes=40, capacity=128, aux=W.aux, aux_capacity=128)
+    u2 = torch.full((2, 4, 4, V), 0.5, device="cuda")
+    assert two.ctx.mtad_draft([0, 1], 4, 4, u2, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_UNIMPLEMENTED
     no_aux = GpuModel(W.target, max_batch=1, max_nodes=8, capacity=64)
     assert no_aux.ctx.mtad_draft([0], 4, 4, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_INVALID
