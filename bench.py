@@ -313,6 +313,7 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
     reset()
     sampler = ClockSampler(local_rank)       # started before the warm-up: nvidia-smi needs a moment to come up
     acc_dev = torch.zeros((), dtype=torch.int64, device="cuda")
+    bad_dev = torch.zeros((), dtype=torch.int32, device="cuda")      # OR of the per-sequence device status words
     for i in range(args.warmup):
         inputs[i].verify(ctx, seqs, log_tau, unis[i], res)
         ctx.kv_commit(seqs, res)
@@ -328,7 +329,12 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
         ctx.kv_commit(seqs, res)
         acc_dev += res.n_out.sum()
         ev[k + 1].record()
+        if k % 16 == 15 or k == args.steps - 1:      # outside the per-step events' critical path most of the time
+            bad_dev |= res.status.max()
     barrier()
+    device_status = int(bad_dev.item())
+    if device_status != 0:
+        raise RuntimeError(f"device status {device_status:#x} during the timed steps (see MTAD_ST_* in mtad.h)")
     launches = M.mtad_kernel_launches() - launches0
     clocks = sampler.stop()
     total_ms, accepted = combine_ranks(ev[0].elapsed_time(ev[-1]), float(acc_dev.item()), world)
@@ -419,7 +425,7 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
         "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / args.steps},
-        "gpu_launches": int(launches),
+        "gpu_launches": int(launches), "device_status": device_status,
         "clocks": clocks,
     }
     del dm, ctx
