@@ -123,7 +123,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // An fp32 activation enters the tensor-core GEMM as `terms` bf16 values whose sum is the activation to ~2^-17
 // relative (two terms) or to fp32 rounding (three).  The terms of row t are neighbouring rows of the operand
 // buffer: term j of element k lives at x[(t * terms + j) * K + k].
-int tc_terms(int T);       // terms used for a call of T rows: 3 while the three accumulators fit tensor memory twice
+int tc_terms(int T);       // terms used for a call of T rows: 3 up to 32 rows, else 2
 __device__ __forceinline__ void store_terms(float y, __nv_bfloat16* x, size_t K, int terms) {
     const __nv_bfloat16 h = __float2bfloat16_rn(y);
     x[0] = h;

@@ -5,8 +5,7 @@
 // The weight matrix is the 128-row MMA operand (A), the draft rows are the MMA N dimension (B), both K-major bf16
 // tiles of 64 elements (one 128-byte swizzled row) brought in by TMA; fp32 accumulators live in tensor memory.
 // The fp32 activations arrive split into two or three bf16 terms (x_0 = bf16(x), x_1 = bf16(x - x_0), ...): with
-// three the tensor cores see the fp32 value itself, with two (row counts whose three accumulators would not fit
-// tensor memory) ~2^-17 relative.  Every term is a row of the MMA's N dimension with an fp32 accumulator column
+// three (up to 32 rows) the tensor cores see the fp32 value itself, with two ~2^-17 relative.  Every term is a row of the MMA's N dimension with an fp32 accumulator column
 // of its own; the drain adds a row's columns.  Work is cut into (tile, k-block) units dealt out
 // evenly to the CTAs; a tile whose k-range spans several CTAs is completed by whichever of them arrives last, which
 // sums the partial tiles in CTA order (deterministic) and runs the fused epilogue - with more than eight rows by all
@@ -850,11 +849,16 @@ void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int sms, int per_s
 }
 
 int tc_terms(int T) {
-    // three terms while two accumulator buffers of 3 * rpad columns fit the 512 columns of tensor memory and the
-    // operand tile stays one TMA box / one MMA (N <= 256); MTAD_TC_TERMS=2 keeps two everywhere
-    static const int cap = getenv("MTAD_TC_TERMS") ? atoi(getenv("MTAD_TC_TERMS")) : 3;
+    // Three terms up to 32 rows, where the third costs nothing measurable; two beyond.  With more rows the operand
+    // rows (terms * rows * 128 B per k-block, re-read from L2 by every CTA) outweigh the 16 KB of weights they meet,
+    // two terms leave room in tensor memory for two weight halves per stage up to 64 rows, and at the level of the
+    // whole model the third term changes nothing (the error there is set by bf16 K/V rounding).  MTAD_TC_TERMS=2 /
+    // =3 force a count (3 only up to 80 rows: three accumulators must fit tensor memory twice).
+    static const int force = getenv("MTAD_TC_TERMS") ? atoi(getenv("MTAD_TC_TERMS")) : 0;
     const int rpad = (T + 15) / 16 * 16;
-    return (cap >= 3 && rpad <= 80) ? 3 : 2;
+    if (force == 2) return 2;
+    if (force == 3) return rpad <= 80 ? 3 : 2;
+    return rpad <= 32 ? 3 : 2;
 }
 
 int tc_ctas_per_sm(int T) {
