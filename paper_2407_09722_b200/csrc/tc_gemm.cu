@@ -873,11 +873,13 @@ int tc_ctas_per_sm(int T) {
 
 int tc_halves(int T) {
     if (tc_ctas_per_sm(T) == 2) return 1;
-    // TMEM holds 2 buffers x halves x terms * rpad columns <= 512; two halves (two MMA-issuing warps) already keep
-    // the tensor pipe ahead of HBM, and smaller stages fill and drain faster than 512-row ones
+    // TMEM holds buffers x halves x terms * rpad columns <= 512.  Two halves (two MMA-issuing warps, 32 KB of weights
+    // per stage against the same operand rows) are worth more than a second accumulator buffer: with 129..256
+    // columns a stage has two halves and the launch a single buffer (7B tree 8.7 -> 8.0 ms).  Four halves fit the
+    // smallest row counts but fill and drain slower than two.
     static const int cap = getenv("MTAD_TC_MH") ? atoi(getenv("MTAD_TC_MH")) : 2;
     const int cols = tc_terms(T) * ((T + 15) / 16 * 16);
-    const int fit = cols <= 64 ? 4 : (cols <= 128 ? 2 : 1);
+    const int fit = cols <= 64 ? 4 : (cols <= 256 ? 2 : 1);
     return fit < cap ? fit : cap;
 }
 
