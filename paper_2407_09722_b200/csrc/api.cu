@@ -293,9 +293,17 @@ bool build_weight_maps(const ModelView& m, WeightMaps& w) {
     return ok;
 }
 
-bool mma_attention(const mtad_model_desc& d) {
+bool mma_attention(const ModelView& m) {
     static const bool on = !(getenv("MTAD_TC_ATTN") && atoi(getenv("MTAD_TC_ATTN")) == 0);
-    return on && (d.head_dim == 64 || d.head_dim == 128);
+    return on && m.kv_map_ok && (m.d.head_dim == 64 || m.d.head_dim == 128);
+}
+
+// K/V tiles of the tensor-core attention arrive by TMA: one map over the whole cache of a model
+void build_kv_map(ModelView& m) {
+    const mtad_model_desc& d = m.d;
+    m.kv_map_ok = (d.head_dim == 64 || d.head_dim == 128) && (reinterpret_cast<uintptr_t>(d.kv_cache) & 15) == 0 &&
+                  tc_make_kv_map(&m.kv_map, d.kv_cache, d.head_dim, d.kv_capacity,
+                                 (long long)d.layers * m.max_batch * 2 * d.n_kv_heads) == 0;
 }
 
 // The same forward on the tensor-core path: every projection is one launch of the TMA + tcgen05 GEMM with a fused
@@ -428,10 +436,10 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
     };
     if (int rc = launch(0, 1)) return rc;                       // QKV of layer 0
     for (int l = 0; l < d.layers; ++l) {
-        if (mma_attention(d)) {
+        if (mma_attention(m)) {
             const int nsp = attention_mma_tiles_per_block(m, B, R, total);
             const int ns = (int)(((total + 63) / 64 + nsp - 1) / nsp);
-            RUN(MTAD_K_ATTN, 0, 2, launch_attention_mma(m, l, ctx->rm, sc, B, R, ns, nsp, pdl, s));
+            RUN(MTAD_K_ATTN, 0, 2, launch_attention_mma(m, l, ctx->rm, sc, B, R, ns, nsp, status, pdl, s));
             RUN(MTAD_K_ATTN, 0, 0, launch_attention_combine(m, ctx->rm, sc, B, R, ns, true, pdl, s));
         } else {
             RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, true, pdl, s));
@@ -547,6 +555,10 @@ int mtad_create(const mtad_model_desc* target, const mtad_model_desc* aux, int m
     const char* path = getenv("MTAD_PATH");
     ctx->use_tc = !(path && strcmp(path, "simt") == 0) && build_weight_maps(ctx->target, ctx->tmaps);
     if (ctx->use_tc && aux) build_weight_maps(ctx->aux, ctx->amaps);
+    if (ctx->use_tc) {
+        build_kv_map(ctx->target);
+        if (aux) build_kv_map(ctx->aux);
+    }
     const char* pdl = getenv("MTAD_PDL");
     ctx->use_pdl = !(pdl && strcmp(pdl, "0") == 0);        // programmatic dependent launch unless MTAD_PDL=0
     cudaError_t e = cudaMemset(workspace, 0, need);

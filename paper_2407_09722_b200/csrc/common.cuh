@@ -1,6 +1,7 @@
 // Internal declarations shared by the host dispatcher and the kernel translation units.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -34,6 +35,8 @@ struct ModelView {
     mtad_model_desc d;
     std::vector<const void*> lw;   // layers * 9 device pointers
     int max_batch;
+    CUtensorMap kv_map;            // KV cache as (head_dim, position, plane = ((layer, sequence), K|V, KV head)), boxes of 64 x 64
+    bool kv_map_ok = false;
     const __nv_bfloat16* w(int layer, int which) const {
         return static_cast<const __nv_bfloat16*>(lw[(size_t)layer * MTAD_LAYER_TENSORS + which]);
     }
@@ -169,7 +172,7 @@ cudaError_t launch_attention(const ModelView& m, int layer, const RowMeta& rm, c
 // tensor-core partial pass (one split per 64 keys) and the combine pass on its own
 int attention_mma_tiles_per_block(const ModelView& m, int B, int R, long long keys);
 cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int B, int R,
-                                 int nsplit, int nsp, bool pdl, cudaStream_t st);
+                                 int nsplit, int nsp, uint32_t* status, bool pdl, cudaStream_t st);
 cudaError_t launch_attention_combine(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int nsplit,
                                      bool emit_split, bool pdl, cudaStream_t st);
 cudaError_t launch_lm_merge(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int n_tiles,

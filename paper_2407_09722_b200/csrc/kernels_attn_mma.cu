@@ -1,8 +1,8 @@
 // Tree-masked attention of the draft rows against the KV cache on tensor cores (warp-level mma.sync, bf16 x bf16
 // -> fp32): the partial pass of the split-KV scheme.  One block owns (sequence, KV head, split of 64 keys): its K
-// and V rows arrive in shared memory with cp.async (16-byte pieces, XOR-swizzled so that ldmatrix is conflict
-// free; a block that walks several tiles keeps up to three in flight, and the tiles that hold only committed
-// positions are requested before the block waits for the kernel in front of it) and every query row of the KV head's group - the draft rows of all its query heads, 16 per MMA tile - is
+// and V rows arrive in shared memory by TMA (64 x 64 boxes of a map over the whole cache, 128-byte swizzle so that
+// ldmatrix is conflict free; a block that walks several tiles keeps up to three in flight, and the tiles that hold
+// only committed positions are requested before the block waits for the kernel in front of it) and every query row of the KV head's group - the draft rows of all its query heads, 16 per MMA tile - is
 // run against them by one of the four warps.  fp32 queries and probabilities enter the tensor cores as bf16
 // hi + lo pairs (two MMAs), so only the cache's own bf16 rounding remains.  A row sees the committed positions
 // [0, L) and the draft rows among its ancestors and itself (Sec. 3.3 of the paper: tree attention).
@@ -20,6 +20,38 @@ __device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cv
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
     const int n = valid ? 16 : 0;                      // src-size 0: the 16 bytes are zero-filled
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+
+// ---- TMA + mbarrier (K/V tiles) ----
+constexpr uint32_t ATTN_WAIT_LIMIT = 1u << 22;
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded: false when the limit ran out
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < ATTN_WAIT_LIMIT; ++it) {
+        if (mbar_test(bar, parity)) return true;
+        if (it > 64) __nanosleep(32);
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y), "r"(z)
+        : "memory");
 }
 
 __device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
@@ -55,22 +87,30 @@ __device__ __forceinline__ void split2(float x, float y, uint32_t& hi, uint32_t&
 // keys of the split; attn_combine_kernel merges the splits in order.  q_hi / q_lo hold the query rows times
 // log2(e) / sqrt(HD), so the softmax numerators are exp2(s - m); m is stored back in natural-log units.
 template <int HD>
-__global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* __restrict__ q_hi,
-                                                          const __nv_bfloat16* __restrict__ q_lo,
-                                                          const __nv_bfloat16* __restrict__ cache, RowMeta rm,
+__global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __grid_constant__ CUtensorMap kvmap,
+                                                          const __nv_bfloat16* __restrict__ q_hi,
+                                                          const __nv_bfloat16* __restrict__ q_lo, RowMeta rm,
                                                           float* __restrict__ part, int layer, int max_batch, int Hq,
-                                                          int Hkv, long long cap, int R, int nsplit, int nslab, int nsp,
-                                                          int nb, int early) {
+                                                          int Hkv, int R, int nsplit, int nslab, int nsp, int nb,
+                                                          int early, uint32_t* status) {
     constexpr int ROWB = HD * 2;          // bytes of one key row
     constexpr int CPR = HD / 8;           // 16-byte pieces per row
     constexpr int NDT = HD / 8;           // 8-wide output tiles over the head dim
     constexpr int SLAB = 2 * 16 * ROWB;   // one query tile: 16 rows hi, then 16 rows lo
     constexpr int PARK = HD + 8;          // row stride (floats) of a parked output tile
     constexpr float LN2 = 0.6931471805599453f;
-    extern __shared__ __align__(128) uint8_t smem[];
-    // nb K/V buffers of [KT][HD] bf16 each (piece c of row k stored at piece c ^ (k & 7)), then the query tiles
-    uint8_t* Qs = smem + nb * 2 * KT * ROWB;          // nslab query tiles, same swizzle
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // nb K/V buffers, each K then V as TMA boxes of [KT keys][64 elements = 128 bytes] (two per tensor at head_dim
+    // 128), 128-byte swizzle: 16-byte piece c of key k sits at piece c ^ (k & 7) of its row; then the query tiles
+    uint8_t* Qs = smem + nb * 2 * KT * ROWB;          // nslab query tiles, [16 rows][HD], same XOR on the piece index
     float* ml = reinterpret_cast<float*>(Qs + nslab * SLAB);           // [4 warps][16 rows][m, l]
+    uint64_t* full = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(ml) + 1536);   // one barrier per buffer
+    if (threadIdx.x == 0) {
+        for (int b = 0; b < nb; ++b) mbar_init(s_u32(&full[b]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
 
     const int sp = blockIdx.x, g = blockIdx.y, bi = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -97,8 +137,7 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
         return;
     }
     const int seq = __ldcg(rm.call_seq + bi);
-    const __nv_bfloat16* Kg = cache + (((((size_t)layer * max_batch + seq) * 2 + 0) * Hkv + g) * cap) * HD;
-    const __nv_bfloat16* Vg = cache + (((((size_t)layer * max_batch + seq) * 2 + 1) * Hkv + g) * cap) * HD;
+    const int plane_k = ((layer * max_batch + seq) * 2 + 0) * Hkv + g, plane_v = plane_k + Hkv;
     const int n_mt = (n_q + 15) / 16;
     // With fewer than three query tiles the warps share a tile and split its 64 keys instead (kparts warps per
     // tile, merged through shared memory below); otherwise every warp runs whole tiles against all 64 keys.
@@ -118,43 +157,36 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
             cp_async16(s_u32(dst + which * 16 * ROWB + row * ROWB + ((c ^ (row & 7)) << 4)), src, valid);
         }
     };
-    // K and V rows of one 64-key tile -> buffer `buf` (zero-filled past the last key).  Thread i copies piece
-    // i % CPR of the keys i / CPR + k * (128 / CPR): its swizzled piece index is the same for all of them.
-    constexpr int KSTEP = 128 / CPR;                  // keys between two copies of a thread
-    const int ld_key = threadIdx.x / CPR, ld_c = threadIdx.x % CPR;
-    const uint32_t ld_soff = ld_key * ROWB + ((ld_c ^ (ld_key & 7)) << 4);
-    static_assert(KSTEP % 8 == 0, "the swizzle of a thread's pieces must not change from copy to copy");
+    // K and V rows of one 64-key tile -> buffer `buf`, by TMA (one thread): positions past the cache capacity come
+    // back as zeros, positions between the last key and the tile's end hold whatever the cache holds there
+    constexpr uint32_t TILE_BYTES = 2 * KT * ROWB;
     auto load_kv = [&](int tile, int buf) {
-        const int kb = tile * KT;
-        const uint32_t Kd = s_u32(smem + buf * (2 * KT * ROWB)) + ld_soff, Vd = Kd + KT * ROWB;
-        const __nv_bfloat16* kg = Kg + (size_t)(kb + ld_key) * HD + ld_c * 8;
-        const __nv_bfloat16* vg = Vg + (size_t)(kb + ld_key) * HD + ld_c * 8;
-        if (kb + KT <= nkeys) {                       // whole tile valid
+        const uint32_t bar = s_u32(&full[buf]);
+        const uint32_t dst = s_u32(smem + buf * TILE_BYTES);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the buffer's last readers were ldmatrix
+        mbar_expect_tx(bar, TILE_BYTES);
 #pragma unroll
-            for (int k = 0; k < KT / KSTEP; ++k) {
-                cp_async16(Kd + k * KSTEP * ROWB, kg + (size_t)k * KSTEP * HD, true);
-                cp_async16(Vd + k * KSTEP * ROWB, vg + (size_t)k * KSTEP * HD, true);
-            }
-        } else {
-#pragma unroll
-            for (int k = 0; k < KT / KSTEP; ++k) {
-                const bool valid = kb + ld_key + k * KSTEP < nkeys;
-                cp_async16(Kd + k * KSTEP * ROWB, valid ? kg + (size_t)k * KSTEP * HD : Kg, valid);
-                cp_async16(Vd + k * KSTEP * ROWB, valid ? vg + (size_t)k * KSTEP * HD : Vg, valid);
-            }
+        for (int h = 0; h < HD / 64; ++h) {
+            tma_load_3d(dst + h * (KT * 128), &kvmap, bar, h * 64, tile * KT, plane_k);
+            tma_load_3d(dst + KT * ROWB + h * (KT * 128), &kvmap, bar, h * 64, tile * KT, plane_v);
         }
     };
+    // byte offset of 16-byte piece c of key `key` inside a K or V tile
+    auto kv_off = [](int key, int c) -> uint32_t {
+        return (uint32_t)((c >> 3) * (KT * 128) + key * 128 + (((c & 7) ^ (key & 7)) << 4));
+    };
+    int n_issued = 0;                                 // tiles requested so far (thread 0)
     // prologue: the first tiles of the block (one, or as many as the prefetch distance nb - 1)
     const int pd = nb - 1;
     const int n_pro = min(max(pd, 1), tile_end - tile_begin);
     uint32_t asked = 0;
     if (early) {
-        for (int j = 0; j < n_pro; ++j)
-            if ((tile_begin + j + 1) * KT <= L) {          // committed positions only
-                load_kv(tile_begin + j, j);
-                asked |= 1u << j;
-            }
-        asm volatile("cp.async.commit_group;" ::: "memory");
+        if (threadIdx.x == 0)
+            for (int j = 0; j < n_pro; ++j)
+                if ((tile_begin + j + 1) * KT <= L) {      // committed positions only
+                    load_kv(tile_begin + j, j);
+                    asked |= 1u << j;
+                }
         pdl_wait();
         pdl_trigger();
     }
@@ -163,9 +195,12 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
     } else if (warp < n_mt) {
         stage_q(warp, warp, lane, 32);
     }
-    for (int j = 0; j < n_pro; ++j)
-        if (!((asked >> j) & 1u)) load_kv(tile_begin + j, j);
     asm volatile("cp.async.commit_group;" ::: "memory");
+    if (threadIdx.x == 0) {
+        for (int j = 0; j < n_pro; ++j)
+            if (!((asked >> j) & 1u)) load_kv(tile_begin + j, j);
+        n_issued = n_pro;
+    }
 
     const int gq = lane >> 2, tq = lane & 3;          // fragment coordinates
     const int lrow = lane & 7, lid = lane >> 3;       // ldmatrix: row within an 8x8 matrix, matrix id
@@ -179,20 +214,41 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
 
   for (int tile = tile_begin; tile < tile_end; ++tile) {
     const int t = tile - tile_begin, buf = t % nb;
-    if (pd > 0) {
-        // request tile t + pd into the buffer tile t - 1 has left; one group per iteration (empty past the end), so
-        // that "all but the latest pd groups" always means "up to tile t"
-        if (tile + pd < tile_end) load_kv(tile + pd, (t + pd) % nb);
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        if (t == 0 || pd == 1) asm volatile("cp.async.wait_group 1;" ::: "memory");   // t == 0: the whole prologue
-        else asm volatile("cp.async.wait_group 2;" ::: "memory");
-    } else {
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
+    // request tile t + pd into the buffer that tile t - 1 has left (all warps passed the barrier that ends it)
+    if (pd > 0 && tile + pd < tile_end && threadIdx.x == 0) {
+        load_kv(tile + pd, (t + pd) % nb);
+        n_issued = t + pd + 1;
     }
-    __syncthreads();
+    if (t == 0) asm volatile("cp.async.wait_group 0;" ::: "memory");      // this thread's query pieces
+    bool ok = mbar_wait(s_u32(&full[buf]), (uint32_t)(t / nb) & 1u);
+    if (ok && tile * KT + KT > nkeys) {
+        // rows past the last key: their scores are masked below, but 0 x (stale V) must not make a NaN
+        const int first = max(nkeys - tile * KT, 0);
+        uint8_t* Vs = smem + buf * TILE_BYTES + KT * ROWB;
+        for (int i = threadIdx.x; i < (KT - first) * CPR; i += blockDim.x) {
+            const int key = first + i / CPR, c = i % CPR;
+            *reinterpret_cast<uint4*>(Vs + kv_off(key, c)) = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+    if (__syncthreads_or(ok ? 0 : 1)) {
+        // a tile did not arrive within the limit: flag it, let the copies in flight land (bounded), leave neutral
+        // partials so that the combine pass reads defined values
+        if (threadIdx.x == 0) {
+            if (status) atomicOr(status + bi, MTAD_ST_TIMEOUT);
+            for (int tt = t; tt < n_issued; ++tt) mbar_wait(s_u32(&full[tt % nb]), (uint32_t)(tt / nb) & 1u);
+        }
+        for (int i = threadIdx.x; i < n_q; i += blockDim.x) {
+            const int h = g * G + i / nrows, r = i % nrows;
+            float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
+            dst[0] = -CUDART_INF_F;
+            dst[1] = 0.f;
+        }
+        __syncthreads();
+        return;
+    }
     const int k_begin = tile * KT;
     const bool spec = k_begin + KT > L;               // the tile reaches into the draft rows: masks apply
-    const uint32_t ks_base = s_u32(smem + buf * (2 * KT * ROWB)), vs_base = ks_base + KT * ROWB;
+    const uint32_t ks_base = s_u32(smem + buf * TILE_BYTES), vs_base = ks_base + KT * ROWB;
 
     for (int mt = warp / kparts; mt < n_mt; mt += 4 / kparts) {
         const int slab = kparts > 1 ? mt : warp;
@@ -231,7 +287,7 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
                 if (n2 < cnt) {                       // sacc[2 * n2 ..] covers keys (kt0 + n2) * 16 ..
                     const int key = (kt0 + n2) * 16 + (lid >> 1) * 8 + lrow, c = ks * 2 + (lid & 1);
                     uint32_t b0, b1, b2, b3;
-                    ldsm4(ks_base + key * ROWB + ((c ^ (key & 7)) << 4), b0, b1, b2, b3);
+                    ldsm4(ks_base + kv_off(key, c), b0, b1, b2, b3);
                     mma16816(sacc[2 * n2], ah, b0, b1);
                     mma16816(sacc[2 * n2], al, b0, b1);
                     mma16816(sacc[2 * n2 + 1], ah, b2, b3);
@@ -316,7 +372,7 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
                 for (int d2 = 0; d2 < HD / 16; ++d2) {
                     const int key = (kt0 + kk) * 16 + (lid & 1) * 8 + lrow, c = d2 * 2 + (lid >> 1);
                     uint32_t b0, b1, b2, b3;
-                    ldsm4t(vs_base + key * ROWB + ((c ^ (key & 7)) << 4), b0, b1, b2, b3);
+                    ldsm4t(vs_base + kv_off(key, c), b0, b1, b2, b3);
                     mma16816(oacc[2 * d2], ph, b0, b1);
                     mma16816(oacc[2 * d2], pl, b0, b1);
                     mma16816(oacc[2 * d2 + 1], ph, b2, b3);
@@ -393,7 +449,8 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __nv_bfloat16* _
 
 namespace {
 size_t attn_smem(int hd, int nslab, int nb) {
-    return (size_t)nb * 2 * KT * hd * 2 + (size_t)nslab * 2 * 16 * hd * 2 + 2048;
+    // K/V ring, query tiles, merge scratch and barriers, and room to align the ring to 1024 bytes (TMA swizzle)
+    return (size_t)nb * 2 * KT * hd * 2 + (size_t)nslab * 2 * 16 * hd * 2 + 2048 + 1024;
 }
 // K/V buffers of a block that walks several tiles: three (two tiles in flight behind the one being computed) when
 // two such blocks fit an SM, else two
@@ -412,9 +469,9 @@ int attention_mma_tiles_per_block(const ModelView& m, int B, int R, long long ke
 }
 
 cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& rm, const Scratch& sc, int B, int R,
-                                 int nsplit, int nsp, bool pdl, cudaStream_t st) {
+                                 int nsplit, int nsp, uint32_t* status, bool pdl, cudaStream_t st) {
     const int Hq = m.d.n_q_heads, Hkv = m.d.n_kv_heads, hd = m.d.head_dim;
-    const __nv_bfloat16* cache = static_cast<const __nv_bfloat16*>(m.d.kv_cache);
+    if (!m.kv_map_ok) return cudaErrorInvalidValue;
     // query tiles kept in shared memory: all of them (at most two) when the warps split keys, else one per warp
     const int n_mt_max = ((Hq / Hkv) * R + 15) / 16;
     const int nslab = n_mt_max <= 2 ? n_mt_max : 4;
@@ -431,13 +488,13 @@ cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& r
         attr_set = true;
     }
     if (hd == 128)
-        return launch_pdl(attn_mma_kernel<128>, grid, dim3(128), smem, st, pdl, (const __nv_bfloat16*)sc.q_hi,
-                          (const __nv_bfloat16*)sc.q_lo, cache, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv,
-                          (long long)m.d.kv_capacity, R, nsplit, nslab, nsp, nb, early);
+        return launch_pdl(attn_mma_kernel<128>, grid, dim3(128), smem, st, pdl, m.kv_map, (const __nv_bfloat16*)sc.q_hi,
+                          (const __nv_bfloat16*)sc.q_lo, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv, R, nsplit,
+                          nslab, nsp, nb, early, status);
     if (hd == 64)
-        return launch_pdl(attn_mma_kernel<64>, grid, dim3(128), smem, st, pdl, (const __nv_bfloat16*)sc.q_hi,
-                          (const __nv_bfloat16*)sc.q_lo, cache, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv,
-                          (long long)m.d.kv_capacity, R, nsplit, nslab, nsp, nb, early);
+        return launch_pdl(attn_mma_kernel<64>, grid, dim3(128), smem, st, pdl, m.kv_map, (const __nv_bfloat16*)sc.q_hi,
+                          (const __nv_bfloat16*)sc.q_lo, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv, R, nsplit,
+                          nslab, nsp, nb, early, status);
     return cudaErrorInvalidValue;
 }
 

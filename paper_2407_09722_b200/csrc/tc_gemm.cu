@@ -831,6 +831,19 @@ int tc_make_map(CUtensorMap* out, const void* base, long long rows, long long co
     return r == CUDA_SUCCESS ? 0 : -1;
 }
 
+int tc_make_kv_map(CUtensorMap* out, const void* cache, int hd, long long cap, long long planes) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || (hd != 64 && hd != 128) || cap < 1 || planes < 1) return -1;
+    const cuuint64_t dims[3] = {(cuuint64_t)hd, (cuuint64_t)cap, (cuuint64_t)planes};
+    const cuuint64_t strides[2] = {(cuuint64_t)hd * 2, (cuuint64_t)cap * hd * 2};
+    const cuuint32_t box[3] = {64, 64, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(cache), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : -1;
+}
+
 void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int sms, int per_sm) {
     p.per_sm = per_sm > 0 ? per_sm : tc_ctas_per_sm(T);
     const int ctas = sms * p.per_sm;

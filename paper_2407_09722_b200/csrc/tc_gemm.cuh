@@ -96,6 +96,9 @@ cudaError_t launch_tc_chain(const TcChain& chain, bool pdl, cudaStream_t st);
 
 // Encodes a 2-D bf16 tensor map (row-major [rows, cols], 128-byte swizzle, box [box_rows, 64]).
 int tc_make_map(CUtensorMap* out, const void* base, long long rows, long long cols, int box_rows);
+// KV cache [planes][cap][hd] bf16 as a 3-D map (hd, cap, planes) with boxes of 64 elements x 64 positions, 128-byte
+// swizzle (hd = 64 or 128).
+int tc_make_kv_map(CUtensorMap* out, const void* cache, int hd, long long cap, long long planes);
 
 // Fills the decomposition fields of p (and p.terms, p.per_sm for T rows) for a problem of n_tiles x k_blocks on
 // `sms` SMs with per_sm CTAs each (0: tc_ctas_per_sm(T)).
