@@ -86,8 +86,8 @@ __device__ __forceinline__ void split2(float x, float y, uint32_t& hi, uint32_t&
 // part[(t * Hq + h) * nsplit + split] = (running max m, sum l, unnormalised output o[HD]) of row t, head h over the
 // keys of the split; attn_combine_kernel merges the splits in order.  q_hi / q_lo hold the query rows times
 // log2(e) / sqrt(HD), so the softmax numerators are exp2(s - m); m is stored back in natural-log units.
-template <int HD>
-__global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __grid_constant__ CUtensorMap kvmap,
+template <int HD, int CNT>
+__global__ void __launch_bounds__(128, CNT == 1 ? 4 : 3) attn_mma_kernel(const __grid_constant__ CUtensorMap kvmap,
                                                           const __nv_bfloat16* __restrict__ q_hi,
                                                           const __nv_bfloat16* __restrict__ q_lo, RowMeta rm,
                                                           float* __restrict__ part, int layer, int max_batch, int Hq,
@@ -141,8 +141,10 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __grid_constant_
     const int n_mt = (n_q + 15) / 16;
     // With fewer than three query tiles the warps share a tile and split its 64 keys instead (kparts warps per
     // tile, merged through shared memory below); otherwise every warp runs whole tiles against all 64 keys.
-    const int kparts = n_mt >= 3 ? 1 : (n_mt == 2 ? 2 : 4);
-    const int cnt = 4 / kparts;                       // 16-key groups per task
+    // (compile-time: the launch picks CNT from its largest sequence; with CNT = 1 the kernel needs 126 registers
+    // instead of 168 and its unrolled loops carry no dead iterations)
+    constexpr int cnt = CNT;                          // 16-key groups per task
+    constexpr int kparts = 4 / CNT;
     const int kt0 = (warp % kparts) * cnt;            // first 16-key group of this warp's tasks
 
     // query tile mt -> slab (16-byte async copies by `nthr` threads; rows past the last query are zero-filled)
@@ -218,6 +220,10 @@ __global__ void __launch_bounds__(128, 3) attn_mma_kernel(const __grid_constant_
     if (pd > 0 && tile + pd < tile_end && threadIdx.x == 0) {
         load_kv(tile + pd, (t + pd) % nb);
         n_issued = t + pd + 1;
+    }
+    if (pd == 0 && t > 0 && threadIdx.x == 0) {       // single buffer: the tile is requested when its turn comes
+        load_kv(tile, 0);
+        n_issued = t + 1;
     }
     if (t == 0) asm volatile("cp.async.wait_group 0;" ::: "memory");      // this thread's query pieces
     bool ok = mbar_wait(s_u32(&full[buf]), (uint32_t)(t / nb) & 1u);
@@ -466,7 +472,8 @@ int attention_mma_tiles_per_block(const ModelView& m, int B, int R, long long ke
     // wave (two per SM with a ring of three buffers at head_dim 128, else three); larger trees take one tile per block
     const int n_mt_max = ((m.d.n_q_heads / m.d.n_kv_heads) * R + 15) / 16;
     if (n_mt_max > 2) return 1;
-    const int per_sm = (attn_ring(m.d.head_dim, n_mt_max, (long long)m.d.n_kv_heads * B) == 3 && m.d.head_dim == 128) ? 2 : 3;
+    const int ring = attn_ring(m.d.head_dim, n_mt_max, (long long)m.d.n_kv_heads * B);
+    const int per_sm = (ring == 3 && m.d.head_dim == 128) ? 2 : 3;
     const long long tiles = (keys + KT - 1) / KT * m.d.n_kv_heads * B;
     const long long nsp = (tiles + per_sm * 148 - 1) / (per_sm * 148);
     return (int)(nsp < 1 ? 1 : (nsp > 64 ? 64 : nsp));
@@ -479,26 +486,21 @@ cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& r
     // query tiles kept in shared memory: all of them (at most two) when the warps split keys, else one per warp
     const int n_mt_max = ((Hq / Hkv) * R + 15) / 16;
     const int nslab = n_mt_max <= 2 ? n_mt_max : 4;
-    const int nb = nsp == 1 ? 1 : (nsp == 2 ? 2 : attn_ring(hd, nslab, (long long)Hkv * B));
+    const int ring = attn_ring(hd, nslab, (long long)Hkv * B);
+    const int nb = nsp == 1 ? 1 : (nsp == 2 ? 2 : ring);
     const size_t smem = attn_smem(hd, nslab, nb);
     const int early = layer > 0 ? 1 : 0;              // the row metadata was final before the previous kernel started
     dim3 grid(nsplit, Hkv, B);
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 116 * 1024);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 116 * 1024);
+    const int cnt = n_mt_max >= 3 ? 4 : (n_mt_max == 2 ? 2 : 1);     // 16-key groups per warp task (template parameter)
+    auto go = [&](auto kernel) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 116 * 1024);
         if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
-    if (hd == 128)
-        return launch_pdl(attn_mma_kernel<128>, grid, dim3(128), smem, st, pdl, m.kv_map, (const __nv_bfloat16*)sc.q_hi,
+        return launch_pdl(kernel, grid, dim3(128), smem, st, pdl, m.kv_map, (const __nv_bfloat16*)sc.q_hi,
                           (const __nv_bfloat16*)sc.q_lo, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv, R, nsplit,
                           nslab, nsp, nb, early, status);
-    if (hd == 64)
-        return launch_pdl(attn_mma_kernel<64>, grid, dim3(128), smem, st, pdl, m.kv_map, (const __nv_bfloat16*)sc.q_hi,
-                          (const __nv_bfloat16*)sc.q_lo, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv, R, nsplit,
-                          nslab, nsp, nb, early, status);
+    };
+    if (hd == 128) return cnt == 1 ? go(attn_mma_kernel<128, 1>) : (cnt == 2 ? go(attn_mma_kernel<128, 2>) : go(attn_mma_kernel<128, 4>));
+    if (hd == 64) return cnt == 1 ? go(attn_mma_kernel<64, 1>) : (cnt == 2 ? go(attn_mma_kernel<64, 2>) : go(attn_mma_kernel<64, 4>));
     return cudaErrorInvalidValue;
 }
 
