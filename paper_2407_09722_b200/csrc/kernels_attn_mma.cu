@@ -86,7 +86,7 @@ __device__ __forceinline__ void split2(float x, float y, uint32_t& hi, uint32_t&
 // part[(t * Hq + h) * nsplit + split] = (running max m, sum l, unnormalised output o[HD]) of row t, head h over the
 // keys of the split; attn_combine_kernel merges the splits in order.  q_hi / q_lo hold the query rows times
 // log2(e) / sqrt(HD), so the softmax numerators are exp2(s - m); m is stored back in natural-log units.
-template <int HD, int CNT>
+template <int HD, int CNT, bool PACK>
 __global__ void __launch_bounds__(128, CNT == 1 ? 4 : 3) attn_mma_kernel(const __grid_constant__ CUtensorMap kvmap,
                                                           const __nv_bfloat16* __restrict__ q_hi,
                                                           const __nv_bfloat16* __restrict__ q_lo, RowMeta rm,
@@ -145,6 +145,10 @@ __global__ void __launch_bounds__(128, CNT == 1 ? 4 : 3) attn_mma_kernel(const _
     // instead of 168 and its unrolled loops carry no dead iterations)
     constexpr int cnt = CNT;                          // 16-key groups per task
     constexpr int kparts = 4 / CNT;
+    // PACK (at most eight query rows per KV head in the whole launch): the hi parts take rows 0..7 of the 16-row MMA
+    // tile and the lo parts rows 8..15, so one MMA multiplies both and a thread (which holds rows g and g + 8) adds
+    // the two products of its query row: half the MMAs, one softmax row per thread
+    constexpr bool packed = PACK;
     const int kt0 = (warp % kparts) * cnt;            // first 16-key group of this warp's tasks
 
     // query tile mt -> slab (16-byte async copies by `nthr` threads; rows past the last query are zero-filled)
@@ -156,6 +160,11 @@ __global__ void __launch_bounds__(128, CNT == 1 ? 4 : 3) attn_mma_kernel(const _
             const bool valid = qi < n_q;
             const int hg = valid ? qi / nrows : 0, r = valid ? qi % nrows : 0;
             const __nv_bfloat16* src = (which ? q_lo : q_hi) + ((size_t)(bi * R + r) * Hq + g * G + hg) * HD + c * 8;
+            if (packed) {                             // query row `row` < 8: hi -> tile row `row`, lo -> tile row 8 + row
+                if (row < 8)
+                    cp_async16(s_u32(dst + (which * 8 + row) * ROWB + ((c ^ (row & 7)) << 4)), src, valid);
+                continue;
+            }
             cp_async16(s_u32(dst + which * 16 * ROWB + row * ROWB + ((c ^ (row & 7)) << 4)), src, valid);
         }
     };
@@ -286,7 +295,7 @@ __global__ void __launch_bounds__(128, CNT == 1 ? 4 : 3) attn_mma_kernel(const _
                 const int row = (lid & 1) * 8 + lrow, c = ks * 2 + (lid >> 1);
                 const uint32_t off = row * ROWB + ((c ^ (row & 7)) << 4);
                 ldsm4(qh_base + off, ah[0], ah[1], ah[2], ah[3]);
-                ldsm4(ql_base + off, al[0], al[1], al[2], al[3]);
+                if (!packed) ldsm4(ql_base + off, al[0], al[1], al[2], al[3]);
             }
 #pragma unroll
             for (int n2 = 0; n2 < 4; ++n2) {
@@ -295,10 +304,22 @@ __global__ void __launch_bounds__(128, CNT == 1 ? 4 : 3) attn_mma_kernel(const _
                     uint32_t b0, b1, b2, b3;
                     ldsm4(ks_base + kv_off(key, c), b0, b1, b2, b3);
                     mma16816(sacc[2 * n2], ah, b0, b1);
-                    mma16816(sacc[2 * n2], al, b0, b1);
                     mma16816(sacc[2 * n2 + 1], ah, b2, b3);
-                    mma16816(sacc[2 * n2 + 1], al, b2, b3);
+                    if (!packed) {
+                        mma16816(sacc[2 * n2], al, b0, b1);
+                        mma16816(sacc[2 * n2 + 1], al, b2, b3);
+                    }
                 }
+            }
+        }
+        if (packed) {
+            // hi product (row g) + lo product (row g + 8) = the score of query row g; the second row is no query
+#pragma unroll
+            for (int n = 0; n < 8; ++n) {
+                sacc[n][0] += sacc[n][2];
+                sacc[n][1] += sacc[n][3];
+                sacc[n][2] = -CUDART_INF_F;
+                sacc[n][3] = -CUDART_INF_F;
             }
         }
         // ---- visibility: keys past the last one, and draft rows that are not ancestors-or-self ----
@@ -338,7 +359,8 @@ __global__ void __launch_bounds__(128, CNT == 1 ? 4 : 3) attn_mma_kernel(const _
         t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, 1));
         t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, 2));
         const float n0 = fmaxf(m0, t0), n1 = fmaxf(m1, t1);
-        const float c0 = (n0 == -CUDART_INF_F) ? 1.f : exp2f(m0 - n0), c1 = (n1 == -CUDART_INF_F) ? 1.f : exp2f(m1 - n1);
+        const float c0 = (n0 == -CUDART_INF_F) ? 1.f : exp2f(m0 - n0);
+        const float c1 = packed ? c0 : ((n1 == -CUDART_INF_F) ? 1.f : exp2f(m1 - n1));   // packed: both rows are one query
         const float s0 = (n0 == -CUDART_INF_F) ? 0.f : n0, s1 = (n1 == -CUDART_INF_F) ? 0.f : n1;
         m0 = n0; m1 = n1;
         float r0 = 0.f, r1 = 0.f;
@@ -371,18 +393,25 @@ __global__ void __launch_bounds__(128, CNT == 1 ? 4 : 3) attn_mma_kernel(const _
             if (kk < cnt) {
                 uint32_t ph[4], pl[4];
                 split2(sacc[2 * kk][0], sacc[2 * kk][1], ph[0], pl[0]);
-                split2(sacc[2 * kk][2], sacc[2 * kk][3], ph[1], pl[1]);
                 split2(sacc[2 * kk + 1][0], sacc[2 * kk + 1][1], ph[2], pl[2]);
-                split2(sacc[2 * kk + 1][2], sacc[2 * kk + 1][3], ph[3], pl[3]);
+                if (packed) {                         // rows 8..15 of the probability tile carry the lo parts
+                    ph[1] = pl[0];
+                    ph[3] = pl[2];
+                } else {
+                    split2(sacc[2 * kk][2], sacc[2 * kk][3], ph[1], pl[1]);
+                    split2(sacc[2 * kk + 1][2], sacc[2 * kk + 1][3], ph[3], pl[3]);
+                }
 #pragma unroll
                 for (int d2 = 0; d2 < HD / 16; ++d2) {
                     const int key = (kt0 + kk) * 16 + (lid & 1) * 8 + lrow, c = d2 * 2 + (lid >> 1);
                     uint32_t b0, b1, b2, b3;
                     ldsm4t(vs_base + kv_off(key, c), b0, b1, b2, b3);
                     mma16816(oacc[2 * d2], ph, b0, b1);
-                    mma16816(oacc[2 * d2], pl, b0, b1);
                     mma16816(oacc[2 * d2 + 1], ph, b2, b3);
-                    mma16816(oacc[2 * d2 + 1], pl, b2, b3);
+                    if (!packed) {
+                        mma16816(oacc[2 * d2], pl, b0, b1);
+                        mma16816(oacc[2 * d2 + 1], pl, b2, b3);
+                    }
                 }
             }
         }
@@ -416,6 +445,11 @@ __global__ void __launch_bounds__(128, CNT == 1 ? 4 : 3) attn_mma_kernel(const _
         }
 #pragma unroll
         for (int n = 0; n < NDT; ++n) {
+            if (packed) {                             // hi-part sums (row g) + lo-part sums (row g + 8)
+                *reinterpret_cast<float2*>(ow + gq * PARK + n * 8 + 2 * tq) =
+                    make_float2(oacc[n][0] + oacc[n][2], oacc[n][1] + oacc[n][3]);
+                continue;
+            }
             *reinterpret_cast<float2*>(ow + gq * PARK + n * 8 + 2 * tq) = make_float2(oacc[n][0], oacc[n][1]);
             *reinterpret_cast<float2*>(ow + (gq + 8) * PARK + n * 8 + 2 * tq) = make_float2(oacc[n][2], oacc[n][3]);
         }
@@ -499,8 +533,13 @@ cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& r
                           (const __nv_bfloat16*)sc.q_lo, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv, R, nsplit,
                           nslab, nsp, nb, early, status);
     };
-    if (hd == 128) return cnt == 1 ? go(attn_mma_kernel<128, 1>) : (cnt == 2 ? go(attn_mma_kernel<128, 2>) : go(attn_mma_kernel<128, 4>));
-    if (hd == 64) return cnt == 1 ? go(attn_mma_kernel<64, 1>) : (cnt == 2 ? go(attn_mma_kernel<64, 2>) : go(attn_mma_kernel<64, 4>));
+    const bool pack = (Hq / Hkv) * R <= 8;            // every sequence of the launch has at most eight query rows per KV head
+    if (hd == 128)
+        return cnt == 1 ? (pack ? go(attn_mma_kernel<128, 1, true>) : go(attn_mma_kernel<128, 1, false>))
+                        : (cnt == 2 ? go(attn_mma_kernel<128, 2, false>) : go(attn_mma_kernel<128, 4, false>));
+    if (hd == 64)
+        return cnt == 1 ? (pack ? go(attn_mma_kernel<64, 1, true>) : go(attn_mma_kernel<64, 1, false>))
+                        : (cnt == 2 ? go(attn_mma_kernel<64, 2, false>) : go(attn_mma_kernel<64, 4, false>));
     return cudaErrorInvalidValue;
 }
 
