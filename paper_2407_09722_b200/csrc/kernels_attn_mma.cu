@@ -1,11 +1,13 @@
 // Tree-masked attention of the draft rows against the KV cache on tensor cores (warp-level mma.sync, bf16 x bf16
-// -> fp32): the partial pass of the split-KV scheme.  One block owns (sequence, KV head, split of 64 keys): its K
+// -> fp32): the partial pass of the split-KV scheme.  One block owns (sequence, KV head, run of 64-key tiles): its K
 // and V rows arrive in shared memory by TMA (64 x 64 boxes of a map over the whole cache, 128-byte swizzle so that
 // ldmatrix is conflict free; a block that walks several tiles keeps up to three in flight, and the tiles that hold
-// only committed positions are requested before the block waits for the kernel in front of it) and every query row of the KV head's group - the draft rows of all its query heads, 16 per MMA tile - is
-// run against them by one of the four warps.  fp32 queries and probabilities enter the tensor cores as bf16
-// hi + lo pairs (two MMAs), so only the cache's own bf16 rounding remains.  A row sees the committed positions
-// [0, L) and the draft rows among its ancestors and itself (Sec. 3.3 of the paper: tree attention).
+// only committed positions are requested before the block waits for the kernel in front of it), and every query
+// row of the KV head's group - the draft rows of all its query heads, 16 per MMA tile - is run against them by one
+// of the four warps.  fp32 queries and probabilities enter the tensor cores as bf16 hi + lo pairs (two MMAs, or one
+// MMA tile that carries both when the group has at most eight query rows), so only the cache's own bf16 rounding
+// remains.  A row sees the committed positions [0, L) and the draft rows among its ancestors and itself (Sec. 3.3
+// of the paper: tree attention).  Waits on the tile barriers are bounded and end in MTAD_ST_TIMEOUT.
 #include <math_constants.h>
 
 #include "common.cuh"
