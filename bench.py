@@ -74,7 +74,7 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
             out, _ = self.proc.communicate()
-        sm, mx, reasons = [], [], set()
+        sm, mx, watts, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in (self.first + out).strip().splitlines():
             f = [x.strip() for x in line.split(",")]
@@ -84,11 +84,16 @@ class ClockSampler:
                 sm.append(float(f[0])); mx.append(float(f[1]))
             except ValueError:
                 continue
+            try:
+                watts.append(float(f[2]))
+            except ValueError:
+                pass
             for n, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons),
+                "power_w_mean": sum(watts) / len(watts) if watts else None}
 
 
 # ---------------------------------------------------------------------------------------------------------------
@@ -388,10 +393,16 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
         for n, t in out_host.items():
             t.copy_(getattr(res, n), non_blocking=True)
         torch.cuda.synchronize()
-        return int(out_host["n_out"].sum())
+        # log-likelihood of the emitted tokens under the target, for the output perplexity (Eq. 1)
+        n = out_host["n_out"].long()
+        emitted = torch.arange(out_host["out_lp"].shape[1])[None, :] < n[:, None]
+        lp_sum[0] += float(out_host["out_lp"].double()[emitted].sum())
+        return int(n.sum())
 
+    lp_sum = [0.0]
     for i in range(args.warmup):
         e2e_step(i)
+    lp_sum[0] = 0.0
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0 = time.perf_counter()
@@ -427,6 +438,14 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
                 "ms_per_step": e2e_ms / args.steps},
         "gpu_launches": int(launches), "device_status": device_status,
         "clocks": clocks,
+        # what the paper reports around the path (Eq. 1; Sec. 5 and App. D), on synthetic random-init models:
+        # perplexity of the emitted tokens under the target, tokens per iteration, energy per token from the
+        # sampled board power over the device-timed steps
+        "metrics": {"output_ppl": math.exp(-lp_sum[0] / acc_e2e) if acc_e2e else None,
+                    "tokens_per_iteration": accepted / (args.steps * w.batch * world),
+                    "power_w_mean": clocks.get("power_w_mean"),
+                    "joules_per_token": (clocks["power_w_mean"] * total_ms * 1e-3 * world / accepted
+                                         if clocks.get("power_w_mean") and accepted else None)},
     }
     del dm, ctx
     torch.cuda.empty_cache()
