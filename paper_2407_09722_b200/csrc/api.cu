@@ -177,6 +177,7 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     sc.tc_flags = k.take<int32_t>(flag_n);
     sc.lm_part = k.take<float4>(Tc * lm_tiles);
     sc.node_z = k.take<float>(T);
+    sc.draft_part = a ? k.take<DraftPart>((size_t)max_batch * MTAD_MAX_BEAM * MTAD_DRAFT_CHUNKS) : nullptr;
     DraftState ds;
     ds.base_len = k.take<int32_t>(max_batch);
     ds.npend = k.take<int32_t>(max_batch);
@@ -698,7 +699,7 @@ int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_wi
         if (tc && B * R <= TC_MAX_ROWS) rc = forward_rows_tc(ctx, m, ctx->amaps, B, R, keys_ub, nullptr, nullptr, true, s);
         else rc = forward_rows(ctx, m, B, R, keys_ub, s);
         if (rc != MTAD_OK) return rc;
-        RUN(MTAD_K_LMRED, 0, 1, launch_draft_select(m, ctx->ds, ctx->sc, sl, B, R, step, gamma, beam_width, uniforms, out, s));
+        RUN(MTAD_K_LMRED, 0, 2, launch_draft_select(m, ctx->ds, ctx->sc, sl, B, R, step, gamma, beam_width, uniforms, out, s));
     }
     ctx->draft_active = true;
     ctx->draft_B = B;

@@ -72,6 +72,16 @@ struct DraftOut {          // caller's device arrays of mtad_draft
     int32_t* best_path;
 };
 
+#define MTAD_DRAFT_CHUNKS 32       // vocabulary chunks of one beam row in the draft's selection (at most)
+
+// What one chunk of a beam row hands to the draft's selection: its share of the row's log-sum-exp and its largest
+// perturbed logits (token -1: none).
+struct DraftPart {
+    float m, s;
+    float t[MTAD_MAX_BEAM];
+    int32_t v[MTAD_MAX_BEAM];
+};
+
 struct Scratch {
     float* hidden;       // [T, d]
     float* xn;           // [T, d]
@@ -98,6 +108,7 @@ struct Scratch {
     int32_t* tc_flags;   // finished-tile flags and counts of the phases of chained GEMM launches, zeroed per forward
     float4* lm_part;     // [T][tiles(V)]
     float* node_z;       // [T]
+    DraftPart* draft_part;   // [max_batch][MTAD_MAX_BEAM][MTAD_DRAFT_CHUNKS], only with an auxiliary model
 };
 
 inline int attn_split_cap(int n_q_heads) {

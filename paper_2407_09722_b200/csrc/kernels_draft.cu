@@ -17,11 +17,6 @@ __device__ __forceinline__ float wsum(float v) {
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
 }
-__device__ __forceinline__ float wmax(float v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
-}
 
 struct Cand {
     float y;      // perturbed joint score
@@ -138,82 +133,139 @@ cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const Dr
 
 // ---------------------------------------------------------------------------------------------------------------
 // selection: the `beam` largest of log q(beam) + log q(token | beam) + Gumbel noise over all (beam, token) pairs
+//
+// Two passes.  draft_scan_kernel, one block per (chunk of the vocabulary, beam row, sequence): the chunk's share of
+// the row's log-sum-exp (running maximum and sum) and its `beam` largest perturbed logits t = z - log(-log u).  The
+// joint score of a pair is t + (log q(beam) - lse(row)), a per-row constant added in fp32 (monotone), so a pair
+// among the overall `beam` largest is among the `beam` largest of its chunk.  draft_pick_kernel, one block per
+// sequence: merges the chunks of every row in chunk order, scores the surviving pairs and takes the `beam` largest
+// (ties to the lower flat index beam * V + token), then writes the new layer of the tree.
 // ---------------------------------------------------------------------------------------------------------------
 
-__global__ void __launch_bounds__(1024) draft_select_kernel(const float* __restrict__ logits, int V, int R, int step,
-                                                            int gamma, int beam, const float* __restrict__ uni,
-                                                            DraftState ds, SeqList seqs, DraftOut out) {
-    const int bi = blockIdx.x, seq = seqs.v[bi];
+__global__ void __launch_bounds__(256) draft_scan_kernel(const float* __restrict__ logits, int V, int R, int step,
+                                                         int gamma, int beam, const float* __restrict__ uni,
+                                                         DraftState ds, SeqList seqs, DraftPart* __restrict__ part,
+                                                         int nch) {
+    const int c = blockIdx.x, j = blockIdx.y, bi = blockIdx.z, seq = seqs.v[bi];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int P = ds.npend[seq];
-    const int n_beams = step == 0 ? 1 : beam;
-    const int N = gamma * beam;
-    __shared__ float s_red[32];
-    __shared__ float s_lse[MTAD_MAX_BEAM], s_lq[MTAD_MAX_BEAM];
-    __shared__ int s_node[MTAD_MAX_BEAM];
-    __shared__ Cand s_c[1024];
-    // log-sum-exp of every beam's row
-    for (int j = 0; j < n_beams; ++j) {
-        const int row = step == 0 ? P - 1 : j;
-        const float* z = logits + (size_t)(bi * R + row) * V;
-        float m = -CUDART_INF_F;
-        for (int v = tid; v < V; v += blockDim.x) m = fmaxf(m, z[v]);
-        m = wmax(m);
-        if (lane == 0) s_red[warp] = m;
-        __syncthreads();
-        m = s_red[0];
-        for (int w = 1; w < 32; ++w) m = fmaxf(m, s_red[w]);
-        __syncthreads();
-        float sum = 0.f;
-        for (int v = tid; v < V; v += blockDim.x) sum += expf(z[v] - m);
-        sum = wsum(sum);
-        if (lane == 0) s_red[warp] = sum;
-        __syncthreads();
-        if (tid == 0) {
-            float a = 0.f;
-            for (int w = 0; w < 32; ++w) a += s_red[w];           // fixed order
-            s_lse[j] = m + logf(a);
-            const int node = step == 0 ? -1 : (step - 1) * beam + j;
-            s_node[j] = node;
-            s_lq[j] = node < 0 ? 0.f : ds.node_logq[seq * MTAD_DRAFT_NODES + node];
-        }
-        __syncthreads();
-    }
-    // every thread keeps the best `beam` of its share of the (beam, token) pairs, sorted
+    const int row = step == 0 ? P - 1 : j;
+    const float* z = logits + (size_t)(bi * R + row) * V;
+    const float* ub = uni + (((size_t)bi * gamma + step) * beam + j) * V;
+    const int len = (V + nch - 1) / nch, v0 = c * len, v1 = min(V, v0 + len);
+    __shared__ float s_m[8], s_s[8];
+    __shared__ Cand s_c[256];
+    float m = -CUDART_INF_F, sum = 0.f;
     Cand loc[MTAD_MAX_BEAM];
 #pragma unroll
     for (int k = 0; k < MTAD_MAX_BEAM; ++k) loc[k] = Cand{-CUDART_INF_F, 0x7fffffff};
-    const float* ub = uni + ((size_t)bi * gamma + step) * beam * V;
-    for (int j = 0; j < n_beams; ++j) {
-        const int row = step == 0 ? P - 1 : j;
-        const float* z = logits + (size_t)(bi * R + row) * V;
-        const float add = s_lq[j] - s_lse[j];
-        for (int v = tid; v < V; v += blockDim.x) {
-            Cand c{add + z[v] - logf(-logf(ub[(size_t)j * V + v])), j * V + v};
-            if (before(c, loc[MTAD_MAX_BEAM - 1])) {
-                loc[MTAD_MAX_BEAM - 1] = c;
+    for (int v = v0 + tid; v < v1; v += 256) {
+        const float zv = z[v];
+        if (zv > m) { sum = sum * expf(m - zv) + 1.f; m = zv; }
+        else sum += expf(zv - m);
+        const Cand cd{zv - logf(-logf(ub[v])), v};
+        if (before(cd, loc[MTAD_MAX_BEAM - 1])) {
+            loc[MTAD_MAX_BEAM - 1] = cd;
 #pragma unroll
-                for (int k = MTAD_MAX_BEAM - 1; k > 0; --k)
-                    if (before(loc[k], loc[k - 1])) { const Cand tmp = loc[k]; loc[k] = loc[k - 1]; loc[k - 1] = tmp; }
-            }
+            for (int k = MTAD_MAX_BEAM - 1; k > 0; --k)
+                if (before(loc[k], loc[k - 1])) { const Cand tmp = loc[k]; loc[k] = loc[k - 1]; loc[k - 1] = tmp; }
         }
     }
+    // the chunk's maximum and sum of exponentials (fixed combination order: butterfly, then warps in order)
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, sum, o);
+        const float M = fmaxf(m, m2);
+        sum = (M == -CUDART_INF_F) ? 0.f : sum * expf(m - M) + s2 * expf(m2 - M);
+        m = M;
+    }
+    if (lane == 0) { s_m[warp] = m; s_s[warp] = sum; }
+    DraftPart* dst = part + ((size_t)(bi * MTAD_MAX_BEAM + j)) * nch + c;
     // `beam` rounds: the block's best head-of-list wins, its owner advances
     int head = 0;
     for (int k = 0; k < beam; ++k) {
-        Cand c = head < MTAD_MAX_BEAM ? loc[head] : Cand{-CUDART_INF_F, 0x7fffffff};
-        // pick among the 1024 heads
-        s_c[tid] = c;
+        const Cand cd = head < MTAD_MAX_BEAM ? loc[head] : Cand{-CUDART_INF_F, 0x7fffffff};
+        s_c[tid] = cd;
         __syncthreads();
-        for (int o = 512; o > 0; o >>= 1) {
+        for (int o = 128; o > 0; o >>= 1) {
             if (tid < o && before(s_c[tid + o], s_c[tid])) s_c[tid] = s_c[tid + o];
             __syncthreads();
         }
         const Cand win = s_c[0];
         __syncthreads();
-        if (c.flat == win.flat && c.y == win.y) ++head;      // the owner of the winner (flat indices are unique)
+        if (cd.flat == win.flat && win.flat != 0x7fffffff) ++head;      // the owner of the winner (tokens are unique)
         if (tid == 0) {
-            const int j = win.flat / V, v = win.flat % V;
+            dst->t[k] = win.y;
+            dst->v[k] = win.flat == 0x7fffffff ? -1 : win.flat;
+        }
+    }
+    if (tid == 0) {
+        float M = -CUDART_INF_F;
+        for (int w = 0; w < 8; ++w) M = fmaxf(M, s_m[w]);
+        float a = 0.f;
+        for (int w = 0; w < 8; ++w) a += (s_m[w] == -CUDART_INF_F) ? 0.f : s_s[w] * expf(s_m[w] - M);
+        dst->m = M;
+        dst->s = a;
+    }
+}
+
+__global__ void __launch_bounds__(256) draft_pick_kernel(const float* __restrict__ logits, int V, int R, int step,
+                                                         int gamma, int beam, DraftState ds, SeqList seqs,
+                                                         const DraftPart* __restrict__ part, int nch, DraftOut out) {
+    const int bi = blockIdx.x, seq = seqs.v[bi];
+    const int tid = threadIdx.x;
+    const int P = ds.npend[seq];
+    const int n_beams = step == 0 ? 1 : beam;
+    const int N = gamma * beam;
+    __shared__ float s_lse[MTAD_MAX_BEAM], s_lq[MTAD_MAX_BEAM];
+    __shared__ int s_node[MTAD_MAX_BEAM];
+    __shared__ float s_y[MTAD_MAX_BEAM * MTAD_DRAFT_CHUNKS * MTAD_MAX_BEAM];
+    __shared__ int s_flat[MTAD_MAX_BEAM * MTAD_DRAFT_CHUNKS * MTAD_MAX_BEAM];
+    __shared__ Cand s_c[256];
+    __shared__ int s_i[256];
+    const DraftPart* pp = part + (size_t)bi * MTAD_MAX_BEAM * nch;
+    if (tid < n_beams) {
+        // log-sum-exp of beam row tid: chunks in order
+        const DraftPart* pj = pp + (size_t)tid * nch;
+        float M = -CUDART_INF_F;
+        for (int c = 0; c < nch; ++c) M = fmaxf(M, pj[c].m);
+        float a = 0.f;
+        for (int c = 0; c < nch; ++c) a += (pj[c].m == -CUDART_INF_F) ? 0.f : pj[c].s * expf(pj[c].m - M);
+        s_lse[tid] = M + logf(a);
+        const int node = step == 0 ? -1 : (step - 1) * beam + tid;
+        s_node[tid] = node;
+        s_lq[tid] = node < 0 ? 0.f : ds.node_logq[seq * MTAD_DRAFT_NODES + node];
+    }
+    __syncthreads();
+    const int n_cand = n_beams * nch * MTAD_MAX_BEAM;
+    for (int i = tid; i < n_cand; i += 256) {
+        const int j = i / (nch * MTAD_MAX_BEAM), c = (i / MTAD_MAX_BEAM) % nch, k = i % MTAD_MAX_BEAM;
+        const DraftPart& d = pp[(size_t)j * nch + c];
+        const bool ok = k < beam && d.v[k] >= 0;
+        s_y[i] = ok ? d.t[k] + (s_lq[j] - s_lse[j]) : -CUDART_INF_F;
+        s_flat[i] = ok ? j * V + d.v[k] : 0x7fffffff;
+    }
+    __syncthreads();
+    for (int k = 0; k < beam; ++k) {
+        Cand best{-CUDART_INF_F, 0x7fffffff};
+        int bidx = -1;
+        for (int i = tid; i < n_cand; i += 256) {
+            const Cand cd{s_y[i], s_flat[i]};
+            if (cd.flat != 0x7fffffff && before(cd, best)) { best = cd; bidx = i; }
+        }
+        s_c[tid] = best;
+        s_i[tid] = bidx;
+        __syncthreads();
+        for (int o = 128; o > 0; o >>= 1) {
+            if (tid < o && before(s_c[tid + o], s_c[tid])) { s_c[tid] = s_c[tid + o]; s_i[tid] = s_i[tid + o]; }
+            __syncthreads();
+        }
+        if (tid == 0) {
+            const Cand win = s_c[0];
+            const int widx = s_i[0];
+            // a vocabulary of at least `beam` tokens always leaves a pair to take
+            const int j = widx >= 0 ? win.flat / V : 0, v = widx >= 0 ? win.flat % V : 0;
+            if (widx >= 0) { s_y[widx] = -CUDART_INF_F; s_flat[widx] = 0x7fffffff; }
             const int n = step * beam + k;
             const int row = step == 0 ? P - 1 : j;
             const float lq = s_lq[j] + logits[(size_t)(bi * R + row) * V + v] - s_lse[j];
@@ -261,7 +313,15 @@ __global__ void __launch_bounds__(1024) draft_select_kernel(const float* __restr
 cudaError_t launch_draft_select(const ModelView& m, const DraftState& ds, const Scratch& sc, const SeqList& seqs, int B,
                                 int R, int step, int gamma, int beam, const float* uniforms, const DraftOut& out,
                                 cudaStream_t st) {
-    draft_select_kernel<<<B, 1024, 0, st>>>(sc.logits, m.d.vocab, R, step, gamma, beam, uniforms, ds, seqs, out);
+    const int V = m.d.vocab;
+    int nch = (V + 1023) / 1024;
+    nch = nch < 1 ? 1 : (nch > MTAD_DRAFT_CHUNKS ? MTAD_DRAFT_CHUNKS : nch);
+    const int n_beams = step == 0 ? 1 : beam;
+    draft_scan_kernel<<<dim3(nch, n_beams, B), 256, 0, st>>>(sc.logits, V, R, step, gamma, beam, uniforms, ds, seqs,
+                                                             sc.draft_part, nch);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    draft_pick_kernel<<<B, 256, 0, st>>>(sc.logits, V, R, step, gamma, beam, ds, seqs, sc.draft_part, nch, out);
     return cudaGetLastError();
 }
 
