@@ -851,6 +851,10 @@ void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int sms, int per_s
     p.k_blocks = (K + TC_TILE_K - 1) / TC_TILE_K;
     p.total_units = n_tiles * p.k_blocks;
     p.units_per_cta = (p.total_units + ctas - 1) / ctas;
+    // small matrices (the auxiliary model's): fewer CTAs with longer runs, so that a tile is not cut into one
+    // contributor per k-block whose partial tiles the last arriver has to add up
+    static const int min_units = getenv("MTAD_TC_MIN_UNITS") ? atoi(getenv("MTAD_TC_MIN_UNITS")) : 2;
+    if (p.units_per_cta < min_units) p.units_per_cta = min_units;
     p.max_contrib = (p.k_blocks + p.units_per_cta - 1) / p.units_per_cta + 1;
     p.T = T;
     p.rpad = (T + 15) / 16 * 16;
