@@ -692,14 +692,15 @@ int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_wi
     for (int step = 0; step < gamma; ++step) {
         const int R = step == 0 ? R0 : beam_width;
         RUN(MTAD_K_PREPARE, 0, 1, launch_draft_prepare(m, ctx->st, ctx->ds, ctx->rm, ctx->sc, sl, B, R, step, beam_width,
-                                                       tc && B * R <= TC_MAX_ROWS, s));
+                                                       tc && B * R <= TC_MAX_ROWS, ctx->use_pdl, s));
         // keys of the auxiliary cache: committed ones, the pending rows and every node drafted so far
         const long long keys_ub = ub + 1 + (long long)step * beam_width;
         int rc;
         if (tc && B * R <= TC_MAX_ROWS) rc = forward_rows_tc(ctx, m, ctx->amaps, B, R, keys_ub, nullptr, nullptr, true, s);
         else rc = forward_rows(ctx, m, B, R, keys_ub, s);
         if (rc != MTAD_OK) return rc;
-        RUN(MTAD_K_LMRED, 0, 2, launch_draft_select(m, ctx->ds, ctx->sc, sl, B, R, step, gamma, beam_width, uniforms, out, s));
+        RUN(MTAD_K_LMRED, 0, 2, launch_draft_select(m, ctx->ds, ctx->sc, sl, B, R, step, gamma, beam_width, uniforms, out,
+                                                     ctx->use_pdl, s));
     }
     ctx->draft_active = true;
     ctx->draft_B = B;

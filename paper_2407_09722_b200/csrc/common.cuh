@@ -206,10 +206,10 @@ cudaError_t launch_seq_advance(const SeqState& s, int B, const int32_t* call_seq
                                int max_depth, cudaStream_t st);
 cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const DraftState& ds, const RowMeta& rm,
                                  const Scratch& sc, const SeqList& seqs, int B, int R, int step, int beam, bool tc,
-                                 cudaStream_t st);
+                                 bool pdl, cudaStream_t st);
 cudaError_t launch_draft_select(const ModelView& m, const DraftState& ds, const Scratch& sc, const SeqList& seqs, int B,
                                 int R, int step, int gamma, int beam, const float* uniforms, const DraftOut& out,
-                                cudaStream_t st);
+                                bool pdl, cudaStream_t st);
 cudaError_t launch_aux_commit(const ModelView& aux, const SeqState& s, const DraftState& ds, int B,
                               const int32_t* call_seq_dev, const mtad_result& res, int max_depth, int mode,
                               cudaStream_t st);

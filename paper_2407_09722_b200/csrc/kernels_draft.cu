@@ -40,6 +40,8 @@ __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, in
     const int t = blockIdx.x, bi = t / R, r = t % R;
     const int seq = seqs.v[bi];
     __shared__ int sh_tok, sh_pos, sh_ok;
+    pdl_wait();               // the sequence and draft state, and every buffer written here, belong to earlier kernels
+    pdl_trigger();
     if (threadIdx.x == 0) {
         const int L = step == 0 ? s.aux_len[seq] : ds.base_len[seq];
         const int P = step == 0 ? s.aux_npend[seq] : ds.npend[seq];
@@ -123,12 +125,12 @@ __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, in
 
 cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const DraftState& ds, const RowMeta& rm,
                                  const Scratch& sc, const SeqList& seqs, int B, int R, int step, int beam, bool tc,
-                                 cudaStream_t st) {
-    draft_prepare_kernel<<<B * R, 128, 0, st>>>(
-        static_cast<const __nv_bfloat16*>(m.d.embed), m.d.d_model, m.d.vocab, m.d.head_dim, (double)m.d.rope_base, s, ds,
-        rm, sc.hidden, sc.rope, seqs, R, step, beam, tc ? m.w(0, 0) : nullptr, tc ? sc.xd : nullptr,
-        tc_terms(B * R), sc.sumsq_a);
-    return cudaGetLastError();
+                                 bool pdl, cudaStream_t st) {
+    return launch_pdl(draft_prepare_kernel, dim3(B * R), dim3(128), 0, st, pdl,
+                      static_cast<const __nv_bfloat16*>(m.d.embed), m.d.d_model, m.d.vocab, m.d.head_dim,
+                      (double)m.d.rope_base, s, ds, rm, sc.hidden, sc.rope, seqs, R, step, beam,
+                      tc ? m.w(0, 0) : (const __nv_bfloat16*)nullptr, tc ? sc.xd : (__nv_bfloat16*)nullptr,
+                      tc_terms(B * R), sc.sumsq_a);
 }
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -148,6 +150,8 @@ __global__ void __launch_bounds__(256) draft_scan_kernel(const float* __restrict
                                                          int nch) {
     const int c = blockIdx.x, j = blockIdx.y, bi = blockIdx.z, seq = seqs.v[bi];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_wait();               // the logits come from the kernel before
+    pdl_trigger();
     const int P = ds.npend[seq];
     const int row = step == 0 ? P - 1 : j;
     const float* z = logits + (size_t)(bi * R + row) * V;
@@ -214,6 +218,8 @@ __global__ void __launch_bounds__(256) draft_pick_kernel(const float* __restrict
                                                          const DraftPart* __restrict__ part, int nch, DraftOut out) {
     const int bi = blockIdx.x, seq = seqs.v[bi];
     const int tid = threadIdx.x;
+    pdl_wait();               // the chunk results come from the kernel before
+    pdl_trigger();
     const int P = ds.npend[seq];
     const int n_beams = step == 0 ? 1 : beam;
     const int N = gamma * beam;
@@ -312,17 +318,16 @@ __global__ void __launch_bounds__(256) draft_pick_kernel(const float* __restrict
 
 cudaError_t launch_draft_select(const ModelView& m, const DraftState& ds, const Scratch& sc, const SeqList& seqs, int B,
                                 int R, int step, int gamma, int beam, const float* uniforms, const DraftOut& out,
-                                cudaStream_t st) {
+                                bool pdl, cudaStream_t st) {
     const int V = m.d.vocab;
     int nch = (V + 1023) / 1024;
     nch = nch < 1 ? 1 : (nch > MTAD_DRAFT_CHUNKS ? MTAD_DRAFT_CHUNKS : nch);
     const int n_beams = step == 0 ? 1 : beam;
-    draft_scan_kernel<<<dim3(nch, n_beams, B), 256, 0, st>>>(sc.logits, V, R, step, gamma, beam, uniforms, ds, seqs,
-                                                             sc.draft_part, nch);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_pdl(draft_scan_kernel, dim3(nch, n_beams, B), dim3(256), 0, st, pdl, (const float*)sc.logits,
+                               V, R, step, gamma, beam, uniforms, ds, seqs, sc.draft_part, nch);
     if (e != cudaSuccess) return e;
-    draft_pick_kernel<<<B, 256, 0, st>>>(sc.logits, V, R, step, gamma, beam, ds, seqs, sc.draft_part, nch, out);
-    return cudaGetLastError();
+    return launch_pdl(draft_pick_kernel, dim3(B), dim3(256), 0, st, pdl, (const float*)sc.logits, V, R, step, gamma,
+                      beam, ds, seqs, (const DraftPart*)sc.draft_part, nch, out);
 }
 
 // ---------------------------------------------------------------------------------------------------------------
