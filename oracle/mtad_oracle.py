@@ -21,7 +21,9 @@ What follows the paper, and where:
     (Algorithm 1, "t ~ p'"), drawn with the Gumbel-max identity from caller
     supplied uniforms so that the draw is a pure function of its inputs;
   * beam sampling draft with the auxiliary model (Sec. 2.1, the p_beam
-    equation), sampled without replacement with Gumbel-top-b.
+    equation), sampled without replacement with Gumbel-top-b;
+  * optionally, the warping of the paper's experiments on every target row
+    before the rule (App. F: top-k, renormalise, top-p).
 
 The decoder itself is only named by the paper (Llama / OPT families); the
 definition used is the Llama one: pre-RMSNorm, rotary embedding with
@@ -33,7 +35,8 @@ Parity pins (tests/test_oracle_*.py): chain-shaped tree == token-by-token
 causal decoding; every tree node == the chain of its own path; cross-check
 against stock torch fp64 ops; log-softmax normalisation; prefix sums vs
 products of probabilities; hand-built accept cases incl. the non-monotone
-one; exhaustive enumeration at vocab 8, gamma 3; sampler frequencies.
+one; exhaustive enumeration at vocab 8, gamma 3; sampler frequencies;
+hand-computed warped rows, and brute-force subset search for top-p.
 The *distribution* of the beam-sampling draft is pinned only through the
 Gumbel-top-b inclusion probabilities at vocab 8: beyond that it is
 "parity unpinned".
@@ -282,6 +285,48 @@ def inverse_cdf_sample(p: np.ndarray, u: float) -> int:
 
 
 # ----------------------------------------------------------------------------
+# warped distributions (App. F: top-k, renormalise, then top-p)
+# ----------------------------------------------------------------------------
+
+def warp_row(z: np.ndarray, top_k: int, top_p: float):
+    """The warping of the paper's experiments applied to one row of logits (App. F): keep the top_k most likely
+    tokens and renormalise; sort them by probability, descending (lower token id first among equals), and keep the
+    first K whose cumulative probability is larger than top_p (all of them if it never is); the rest get
+    probability 0.  The kept tokens are renormalised so that the row is a distribution to sample from (Sec. 2.1:
+    tokens are sampled from that smallest subset).  Returns (log-probabilities with -inf for dropped tokens,
+    margin), margin = how close any of the decisions was to going the other way: the logit gap across the top_k
+    boundary and the distance of every partial cumulative sum from top_p."""
+    z = np.asarray(z, dtype=np.float64)
+    V = z.size
+    order = sorted(range(V), key=lambda i: (-z[i], i))
+    k = min(top_k, V)
+    top = order[:k]
+    margin = float(z[order[k - 1]] - z[order[k]]) if k < V else float("inf")
+    zt = z[top]
+    pt = np.exp(zt - zt[0])
+    pt = pt / pt.sum()
+    keep = k
+    c = 0.0
+    for i in range(k):
+        c += pt[i]
+        if i + 1 < k or c > top_p:
+            margin = min(margin, abs(c - top_p))
+        if c > top_p:
+            keep = i + 1
+            break
+    kept = top[:keep]
+    out = np.full(V, NEG_INF, dtype=np.float64)
+    zk = z[kept]
+    out[kept] = zk - (zk[0] + np.log(np.sum(np.exp(zk - zk[0]))))
+    return out, margin
+
+
+def warp_rows(logits: np.ndarray, top_k: int, top_p: float):
+    rows, margins = zip(*(warp_row(r, top_k, top_p) for r in logits))
+    return np.stack(rows), float(min(margins))
+
+
+# ----------------------------------------------------------------------------
 # one verification step and the cache commit
 # ----------------------------------------------------------------------------
 
@@ -301,10 +346,16 @@ class VerifyResult:
     margin_tie: float
     margin_bonus: float
     logits: Optional[np.ndarray] = None
+    margin_warp: float = float("inf")   # closest warping decision (warp_row) over all rows; inf without warping
 
 
 def verify_from_logits(logits: np.ndarray, tok, parent, logq_or_ref, log_tau: float, u: np.ndarray,
-                       chain: bool) -> VerifyResult:
+                       chain: bool, warp=None) -> VerifyResult:
+    """warp = (top_k, top_p): every row of P is warped first (the paper's footnote to Sec. 3.2: the method is
+    equally valid on warped distributions); a drafted token outside a row's kept set has probability 0."""
+    m_warp = float("inf")
+    if warp is not None:
+        logits, m_warp = warp_rows(logits, warp[0], warp[1])
     lp, lse = node_logprobs(logits, tok, parent)
     LP = path_prefix_sums(lp, parent)
     if chain:
@@ -323,25 +374,25 @@ def verify_from_logits(logits: np.ndarray, tok, parent, logq_or_ref, log_tau: fl
     out_tok = [int(tok[n]) for n in path] + [int(cand[wrow])]
     out_lp = [float(lp[n]) for n in path] + [float(cand_lp[wrow])]
     return VerifyResult(eta, winner, path, out_tok, out_lp, lp, LP, lse, cand, cand_lp, m_acc, m_tie,
-                        float(gaps[wrow]), logits)
+                        float(gaps[wrow]), logits, m_warp)
 
 
 def verify_chain(model: OracleModel, cache: np.ndarray, L: int, root_tok: int, draft_tok, draft_logq,
-                 log_tau: float, u: np.ndarray) -> VerifyResult:
+                 log_tau: float, u: np.ndarray, warp=None) -> VerifyResult:
     """Algorithm 1 from "P <- M_p(input, X)" to the return: draft_logq[i] = log q(x_{1:i+1} | input)."""
     parent = list(range(-1, len(draft_tok) - 1))
     rows = tree_rows(L, root_tok, draft_tok, parent)
     logits = decoder_rows(model, cache, L, *rows)
-    return verify_from_logits(logits, draft_tok, parent, draft_logq, log_tau, u, chain=True)
+    return verify_from_logits(logits, draft_tok, parent, draft_logq, log_tau, u, chain=True, warp=warp)
 
 
 def verify_tree(model: OracleModel, cache: np.ndarray, L: int, root_tok: int, tok, parent, logq_ref,
-                log_tau: float, u: np.ndarray) -> VerifyResult:
+                log_tau: float, u: np.ndarray, warp=None) -> VerifyResult:
     """Sec. 3.3: all candidates in one forward under the tree mask, normalised by the output beam's likelihood."""
     assert max(node_depths(parent), default=0) <= len(logq_ref)
     rows = tree_rows(L, root_tok, tok, parent)
     logits = decoder_rows(model, cache, L, *rows)
-    return verify_from_logits(logits, tok, parent, logq_ref, log_tau, u, chain=False)
+    return verify_from_logits(logits, tok, parent, logq_ref, log_tau, u, chain=False, warp=warp)
 
 
 def kv_commit(cache: np.ndarray, L: int, path: Sequence[int]) -> int:

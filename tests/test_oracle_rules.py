@@ -335,3 +335,89 @@ def test_aux_commit_equals_rerunning_the_accepted_tokens():
         for i, t in enumerate(committed):
             ref = O.decoder_rows(model, c2, i, [t], [i], [i], [[i]])[0]
         assert np.max(np.abs(ref - got)) < 1e-10
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# warped rows (App. F: top-k, renormalise, then top-p)
+# ----------------------------------------------------------------------------------------------------------------
+
+def test_warp_row_hand_computed():
+    z = np.log(np.array([0.5, 0.3, 0.15, 0.05]))
+    # top-3 -> (0.5, 0.3, 0.15) / 0.95; cumulative 0.526, 0.842 > 0.8 -> two tokens, 5/8 and 3/8
+    out, _ = O.warp_row(z, 3, 0.8)
+    assert np.allclose(np.exp(out), [5 / 8, 3 / 8, 0, 0], atol=1e-12)
+    # top-4 keeps everything; cumulative 0.5, 0.8, 0.95 > 0.9 -> three tokens, 10/19, 6/19, 3/19
+    out, margin = O.warp_row(z, 4, 0.9)
+    assert np.allclose(np.exp(out), [10 / 19, 6 / 19, 3 / 19, 0], atol=1e-12)
+    assert abs(margin - 0.05) < 1e-12
+    # k = 1 is greedy decoding (Sec. 2.1)
+    out, _ = O.warp_row(np.array([0.1, 2.0, -1.0, 1.9]), 1, 0.9)
+    assert np.exp(out).tolist() == [0, 1, 0, 0]
+    # the order of the tokens in the row does not matter
+    perm = [2, 0, 3, 1]
+    out_p, _ = O.warp_row(z[perm], 3, 0.8)
+    assert np.allclose(np.exp(out_p), np.array([5 / 8, 3 / 8, 0, 0])[perm], atol=1e-12)
+
+
+def test_warp_row_without_limits_is_log_softmax():
+    rng = np.random.default_rng(5)
+    z = rng.normal(size=37)
+    out, margin = O.warp_row(z, 37, 1.0)
+    assert np.allclose(out, O.log_softmax(z[None])[0], atol=1e-12)
+    out, _ = O.warp_row(z, 1000, 1.0)
+    assert np.allclose(out, O.log_softmax(z[None])[0], atol=1e-12)
+
+
+def test_warp_row_is_the_smallest_subset_above_top_p():
+    """Brute force over all subsets of a 7-token row: the kept set is a smallest subset of the top-k tokens whose
+    renormalised mass is larger than top_p, and the heaviest among those; kept probabilities keep their ratios."""
+    import itertools
+    rng = np.random.default_rng(11)
+    for trial in range(40):
+        z = rng.normal(scale=1.5, size=7)
+        k = int(rng.integers(2, 8))
+        top_p = float(rng.uniform(0.3, 0.97))
+        out, margin = O.warp_row(z, k, top_p)
+        kept = [i for i in range(7) if np.isfinite(out[i])]
+        assert abs(np.exp(out[kept]).sum() - 1) < 1e-12
+        topk = sorted(range(7), key=lambda i: -z[i])[:k]
+        assert set(kept) <= set(topk)
+        p = np.exp(z[topk]) / np.exp(z[topk]).sum()
+        mass = dict(zip(topk, p))
+        best = None
+        for n in range(1, k + 1):
+            ok = [s for s in itertools.combinations(topk, n) if sum(mass[i] for i in s) > top_p]
+            if ok:
+                best = max(ok, key=lambda s: sum(mass[i] for i in s))
+                break
+        if best is None:
+            best = tuple(topk)
+        if margin > 1e-9:
+            assert set(kept) == set(best)
+        ref = kept[0]
+        for i in kept:
+            assert abs((out[i] - out[ref]) - (z[i] - z[ref])) < 1e-12
+
+
+def test_warped_verification_drops_tokens_outside_the_kept_set():
+    rng = np.random.default_rng(3)
+    V, g = 12, 3
+    logits = rng.normal(scale=2.0, size=(g + 1, V))
+    warped, _ = O.warp_rows(logits, 4, 0.9)
+    u = rng.uniform(0.01, 0.99, size=V)
+    # a draft whose first token lies outside the first row's kept set can never be accepted, however unlikely q
+    dropped = int(np.argmin(logits[0]))
+    kept_next = [int(np.argmax(logits[i])) for i in range(1, g)]
+    r = O.verify_from_logits(logits, [dropped] + kept_next, list(range(-1, g - 1)), [-50.0] * g, np.log(0.1), u,
+                             chain=True, warp=(4, 0.9))
+    assert r.eta == 0 and np.isfinite(warped[0, r.out_tok[0]])
+    # the most likely token of every row is always kept: that draft passes against a small enough q
+    best = [int(np.argmax(logits[i])) for i in range(g)]
+    r = O.verify_from_logits(logits, best, list(range(-1, g - 1)), [-50.0] * g, np.log(0.1), u, chain=True,
+                             warp=(4, 0.9))
+    assert r.eta == g and np.isfinite(warped[g, r.out_tok[-1]])
+    # warping that keeps everything changes nothing
+    a = O.verify_from_logits(logits, best, list(range(-1, g - 1)), [-3.0, -6.0, -9.0], np.log(0.3), u, chain=True)
+    b = O.verify_from_logits(logits, best, list(range(-1, g - 1)), [-3.0, -6.0, -9.0], np.log(0.3), u, chain=True,
+                             warp=(V, 1.0))
+    assert a.eta == b.eta and a.out_tok == b.out_tok and np.allclose(a.out_lp, b.out_lp, atol=1e-12)
