@@ -121,6 +121,18 @@ int mtad_seq_set(mtad_ctx* ctx, int seq, int32_t kv_len, int32_t root_token, int
 /* Read back the committed length and root token of a sequence.  Synchronises the stream. */
 int mtad_seq_get(mtad_ctx* ctx, int seq, int32_t* kv_len, int32_t* root_token, void* stream);
 
+/* Warp the target's distributions before the verification rule and the extra token, as in the paper's experiments
+ * (App. F; the footnote to Sec. 3.2 states that the method is equally valid on warped distributions): every row of
+ * P keeps its top_k most likely tokens, renormalised; of these, in descending order of probability (lower token id
+ * first among equals), the first ones whose cumulative probability is larger than top_p are kept and renormalised,
+ * the rest get probability 0.  A drafted token outside its row's kept set has probability 0 and cannot be accepted;
+ * the extra token is drawn from the kept set.  The verify calls that follow then compute plain logits [rows, vocab]
+ * into the workspace and derive the warped rows from them (row_lse of mtad_result is the log-sum-exp over the kept
+ * tokens).  top_k = 0 switches warping off (the default); top_k <= 16 (MTAD_E_CAPACITY beyond), 0 < top_p <= 1
+ * (MTAD_E_INVALID otherwise).  Host-side setting of the context, no launch.  The draft log-likelihoods passed to
+ * the verify calls are the caller's: mtad_draft itself samples from the unwarped auxiliary distribution. */
+int mtad_set_warp(mtad_ctx* ctx, int top_k, float top_p);
+
 /* Draft with the auxiliary model: beam sampling of width beam_width for gamma steps (Sec. 2.1, the p_beam
  * equation; every intermediate beam becomes a tree node, Sec. 3.3).  At each step the beam_width kept sequences
  * are drawn without replacement, proportionally to their joint likelihood, as the beam_width largest values of

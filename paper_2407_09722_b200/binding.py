@@ -40,7 +40,7 @@ class Result(C.Structure):
 EXPORTS = ("mtad_workspace_bytes", "mtad_create", "mtad_destroy", "mtad_seq_set", "mtad_seq_get", "mtad_draft",
            "mtad_verify_chain", "mtad_verify_tree", "kv_commit", "mtad_status_str", "mtad_last_cuda_error",
            "mtad_profile_begin", "mtad_profile_end", "mtad_kernel_launches", "mtad_verify_chain_static",
-           "mtad_debug_gemm")
+           "mtad_debug_gemm", "mtad_set_warp")
 MTAD_STATIC_SCRATCH_BYTES = 16 << 20
 KERNEL_CLASSES = ("prepare", "norm", "gemm", "rope_append", "attention", "lm_reduce", "accept", "commit")
 
@@ -64,6 +64,7 @@ def load_library() -> C.CDLL:
     lib.mtad_destroy.argtypes = [P]
     lib.mtad_seq_set.argtypes = [P, I, C.c_int32, C.c_int32, C.c_int32, I32P, P]
     lib.mtad_seq_get.argtypes = [P, I, I32P, I32P, P]
+    lib.mtad_set_warp.argtypes = [P, I, C.c_float]
     lib.mtad_draft.argtypes = [P, I, I32P, I, I, P, P, P, P, P, P, P, P]
     lib.mtad_verify_chain.argtypes = [P, I, I32P, I, P, P, F, P, RS, P]
     lib.mtad_verify_tree.argtypes = [P, I, I32P, P, I, I, P, P, P, F, P, RS, P]
@@ -202,6 +203,12 @@ class Context:
         pend = (C.c_int32 * len(pending_tok))(*pending_tok) if pending_tok else None
         self._check(self._lib.mtad_seq_set(self.handle, seq, kv_len, root_token, aux_len, pend, _stream(stream)),
                     "mtad_seq_set")
+
+    def mtad_set_warp(self, top_k: int, top_p: float = 1.0, check=True) -> int:
+        rc = self._lib.mtad_set_warp(self.handle, top_k, top_p)
+        if check:
+            self._check(rc, "mtad_set_warp")
+        return rc
 
     def mtad_seq_get(self, seq: int, stream=None):
         a, b = C.c_int32(), C.c_int32()

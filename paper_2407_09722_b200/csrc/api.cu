@@ -41,6 +41,8 @@ struct mtad_ctx {
     int last_B = 0, last_R = 0, last_D = 0;
     int32_t last_seqs[MTAD_MAX_BATCH];
     int last_cuda = 0;
+    int warp_k = 0;                     // 0: unwarped target rows
+    float warp_p = 1.f;
     // optional per-kernel-class timing (cudaEvent pairs around each launch)
     bool prof_on = false;
     std::vector<cudaEvent_t> prof_ev;        // pool, used pairwise
@@ -178,6 +180,8 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     sc.lm_part = k.take<float4>(Tc * lm_tiles);
     sc.node_z = k.take<float>(T);
     sc.draft_part = a ? k.take<DraftPart>((size_t)max_batch * MTAD_MAX_BEAM * MTAD_DRAFT_CHUNKS) : nullptr;
+    sc.warp_part = k.take<WarpPart>(T * MTAD_DRAFT_CHUNKS);
+    sc.warp_row = k.take<WarpRow>(T);
     DraftState ds;
     ds.base_len = k.take<int32_t>(max_batch);
     ds.npend = k.take<int32_t>(max_batch);
@@ -496,15 +500,20 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
         pa.sumsq_out = ctx->sc.sumsq_a;
     }
     RUN(MTAD_K_PREPARE, 0, 1, launch_prepare(ctx->target, ctx->st, ctx->rm, ctx->sc, pa, out->status, s));
+    const bool warped = ctx->warp_k > 0;       // warped rows are made from plain logits, after the forward
     if (tc) {
-        int rc = forward_rows_tc(ctx, ctx->target, ctx->tmaps, B, R, ub, bonus_uniform, out->status, false, s);
+        int rc = forward_rows_tc(ctx, ctx->target, ctx->tmaps, B, R, ub, bonus_uniform, out->status, warped, s);
         if (rc != MTAD_OK) return rc;
     } else {
         int rc = forward_rows(ctx, ctx->target, B, R, ub, s);
         if (rc != MTAD_OK) return rc;
-        RUN(MTAD_K_LMRED, 0, R > 1 ? 2 : 1,
-            launch_lm_reduce(ctx->target, ctx->rm, ctx->sc, B, R, bonus_uniform, tok, parent, s));
+        if (!warped)
+            RUN(MTAD_K_LMRED, 0, R > 1 ? 2 : 1,
+                launch_lm_reduce(ctx->target, ctx->rm, ctx->sc, B, R, bonus_uniform, tok, parent, s));
     }
+    if (warped)
+        RUN(MTAD_K_LMRED, 0, 3,
+            launch_warp_rows(ctx->target, ctx->rm, ctx->sc, B, R, ctx->warp_k, ctx->warp_p, bonus_uniform, s));
     AcceptArgs aa{B, R, D, tok, parent, logq_ref, log_tau};
     RUN(MTAD_K_ACCEPT, 0, 1, launch_accept(ctx->rm, ctx->sc, aa, *out, s));
     ctx->last_B = B; ctx->last_R = R; ctx->last_D = D;
@@ -644,6 +653,14 @@ int mtad_seq_set(mtad_ctx* ctx, int seq, int32_t kv_len, int32_t root_token, int
     RUN(MTAD_K_PREPARE, 0, 1, launch_seq_set(ctx->st, seq, kv_len, root_token, aux_len, npend, pending_tok, s));
     ctx->len_ub[seq] = kv_len;
     ctx->npend_ub[seq] = npend + 1;
+    return MTAD_OK;
+}
+
+int mtad_set_warp(mtad_ctx* ctx, int top_k, float top_p) {
+    if (!ctx || top_k < 0 || isnan(top_p) || !(top_p > 0.f) || top_p > 1.f) return MTAD_E_INVALID;
+    if (top_k > MTAD_MAX_TOPK) return MTAD_E_CAPACITY;
+    ctx->warp_k = top_k;
+    ctx->warp_p = top_p;
     return MTAD_OK;
 }
 

@@ -82,6 +82,19 @@ struct DraftPart {
     int32_t v[MTAD_MAX_BEAM];
 };
 
+#define MTAD_MAX_TOPK 16           // largest top-k of the warped rows
+
+// Warped rows: a chunk's largest logits (token -1: none), and a row's kept tokens with their log-probabilities
+struct WarpPart {
+    float z[MTAD_MAX_TOPK];
+    int32_t v[MTAD_MAX_TOPK];
+};
+struct WarpRow {
+    int32_t n;
+    int32_t idx[MTAD_MAX_TOPK];
+    float lp[MTAD_MAX_TOPK];
+};
+
 struct Scratch {
     float* hidden;       // [T, d]
     float* xn;           // [T, d]
@@ -109,6 +122,8 @@ struct Scratch {
     float4* lm_part;     // [T][tiles(V)]
     float* node_z;       // [T]
     DraftPart* draft_part;   // [max_batch][MTAD_MAX_BEAM][MTAD_DRAFT_CHUNKS], only with an auxiliary model
+    WarpPart* warp_part;     // [T][MTAD_DRAFT_CHUNKS]
+    WarpRow* warp_row;       // [T]
 };
 
 inline int attn_split_cap(int n_q_heads) {
@@ -191,6 +206,9 @@ cudaError_t launch_lm_merge(const ModelView& m, const RowMeta& rm, const Scratch
 cudaError_t launch_lm_reduce(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R,
                              const float* bonus_uniform, const int32_t* tok, const int32_t* parent,
                              cudaStream_t st);
+// Warped target rows from sc.logits: fills row_lse (over the kept tokens), row_cand, row_cand_lp and node_lp.
+cudaError_t launch_warp_rows(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int top_k,
+                             float top_p, const float* bonus_uniform, cudaStream_t st);
 struct AcceptArgs {
     int B, R, max_depth;
     const int32_t* tok;        // [B, R-1]
