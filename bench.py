@@ -296,6 +296,8 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
     for b, L in enumerate(lens):
         dm.inject(b, L)
     ctx = dm.ctx
+    if args.top_k > 0:
+        ctx.mtad_set_warp(args.top_k, args.top_p)      # the warping of the paper's experiments (App. F) on the target rows
     seqs = list(range(w.batch))
     V = w.target.vocab
     log_tau = math.log(TAU)
@@ -427,7 +429,8 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "tau": TAU, "batch": w.batch, "rows_per_seq": rows, "kv_len_start": lens,
                    "replicas": world, "l2": "inputs larger than L2 (weights streamed once per step)",
-                   "block_efficiency": accepted / (args.steps * w.batch * world)},
+                   "block_efficiency": accepted / (args.steps * w.batch * world),
+                   "warp": {"top_k": args.top_k, "top_p": args.top_p} if args.top_k > 0 else None},
         "verify_step_us": {"median": 1e3 * statistics.median(step_ms), "min": 1e3 * min(step_ms),
                            "max": 1e3 * max(step_ms)},
         "step_hbm": {"algorithmic_gb": step_bytes / 1e9, "achieved_gbs": step_bytes / (ms_per_step * 1e-3) / 1e9,
@@ -466,6 +469,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-draft-loop", action="store_true")
+    ap.add_argument("--top-k", type=int, default=0, help="warp the target rows: top-k (0 = off, the default)")
+    ap.add_argument("--top-p", type=float, default=0.9)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = S.WORKLOADS[args.workload]
