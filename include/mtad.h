@@ -209,6 +209,11 @@ enum { MTAD_K_PREPARE = 0, MTAD_K_NORM, MTAD_K_GEMM, MTAD_K_ROPE, MTAD_K_ATTN, M
 /* Start bracketing every kernel launch of this context with a pair of CUDA events on the launching stream (room
  * for max_launches launches; later launches go unrecorded).  Creates events, no device memory. */
 int mtad_profile_begin(mtad_ctx* ctx, int max_launches);
+/* Grouped bracketing (call before mtad_profile_begin; on != 0): one event pair around every run of consecutive
+ * launches of the same class instead of one per launch.  An event between two launches keeps the second from
+ * starting before the first has drained, so per-launch brackets time every kernel as if it stood alone; a run's
+ * bracket times its launches as they overlap in the real step.  MTAD_E_INVALID while profiling is on. */
+int mtad_profile_grouped(mtad_ctx* ctx, int on);
 /* Stop, synchronise the device and sum per kernel class: elapsed milliseconds, algorithmic bytes (bf16 weight
  * bytes of the GEMM launches; 0 for the other classes) and launch count.  Arrays of MTAD_K_CLASSES, host. */
 int mtad_profile_end(mtad_ctx* ctx, double* ms, double* bytes, int64_t* launches);

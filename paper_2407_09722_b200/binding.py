@@ -40,7 +40,7 @@ class Result(C.Structure):
 EXPORTS = ("mtad_workspace_bytes", "mtad_create", "mtad_destroy", "mtad_seq_set", "mtad_seq_get", "mtad_draft",
            "mtad_verify_chain", "mtad_verify_tree", "kv_commit", "mtad_status_str", "mtad_last_cuda_error",
            "mtad_profile_begin", "mtad_profile_end", "mtad_kernel_launches", "mtad_verify_chain_static",
-           "mtad_debug_gemm", "mtad_set_warp")
+           "mtad_debug_gemm", "mtad_set_warp", "mtad_profile_grouped")
 MTAD_STATIC_SCRATCH_BYTES = 16 << 20
 KERNEL_CLASSES = ("prepare", "norm", "gemm", "rope_append", "attention", "lm_reduce", "accept", "commit")
 
@@ -65,6 +65,7 @@ def load_library() -> C.CDLL:
     lib.mtad_seq_set.argtypes = [P, I, C.c_int32, C.c_int32, C.c_int32, I32P, P]
     lib.mtad_seq_get.argtypes = [P, I, I32P, I32P, P]
     lib.mtad_set_warp.argtypes = [P, I, C.c_float]
+    lib.mtad_profile_grouped.argtypes = [P, I]
     lib.mtad_draft.argtypes = [P, I, I32P, I, I, P, P, P, P, P, P, P, P]
     lib.mtad_verify_chain.argtypes = [P, I, I32P, I, P, P, F, P, RS, P]
     lib.mtad_verify_tree.argtypes = [P, I, I32P, P, I, I, P, P, P, F, P, RS, P]
@@ -251,6 +252,9 @@ class Context:
 
     def mtad_profile_begin(self, max_launches: int = 8192):
         self._check(self._lib.mtad_profile_begin(self.handle, max_launches), "mtad_profile_begin")
+
+    def mtad_profile_grouped(self, on: bool):
+        self._check(self._lib.mtad_profile_grouped(self.handle, 1 if on else 0), "mtad_profile_grouped")
 
     def mtad_profile_end(self) -> Dict[str, dict]:
         n = len(KERNEL_CLASSES)

@@ -48,7 +48,11 @@ struct mtad_ctx {
     std::vector<cudaEvent_t> prof_ev;        // pool, used pairwise
     std::vector<int> prof_cls;               // class of each recorded pair
     std::vector<double> prof_bytes;          // algorithmic bytes of each recorded pair
+    std::vector<int> prof_n;                 // launches inside each recorded pair
     size_t prof_used = 0;
+    bool prof_grouped = false;               // one pair around every run of consecutive launches of a class
+    int prof_open = -1;                      // class of the run whose closing event is still to be recorded
+    cudaStream_t prof_stream = nullptr;
 };
 
 unsigned long long g_kernel_launches = 0;    // kernels of this library enqueued since load
@@ -209,18 +213,35 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
         if (e__ != cudaSuccess) { ctx->last_cuda = (int)e__; return MTAD_E_CUDA; } \
     } while (0)
 
-// Enqueue one launcher; when profiling is on, bracket it with an event pair on the same stream.
+// Enqueue one launcher; when profiling is on, bracket it with an event pair on the same stream - or, in grouped mode,
+// bracket every run of consecutive launches of one class with a single pair, so that the launches inside a run keep
+// their programmatic overlap (an event between two launches serialises them).
 template <class F>
 int timed(mtad_ctx* ctx, int cls, double bytes, int kernels, cudaStream_t s, F&& f) {
-    const bool rec = ctx->prof_on && ctx->prof_used + 2 <= ctx->prof_ev.size();
-    if (rec) CU(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s));
+    if (ctx->prof_on) {
+        if (ctx->prof_open >= 0 && !(ctx->prof_grouped && ctx->prof_open == cls)) {
+            CU(cudaEventRecord(ctx->prof_ev[2 * (ctx->prof_cls.size() - 1) + 1], ctx->prof_stream));
+            ctx->prof_open = -1;
+        }
+        if (ctx->prof_open < 0 && ctx->prof_used + 2 <= ctx->prof_ev.size()) {
+            CU(cudaEventRecord(ctx->prof_ev[ctx->prof_used], s));
+            ctx->prof_cls.push_back(cls);
+            ctx->prof_bytes.push_back(0.0);
+            ctx->prof_n.push_back(0);
+            ctx->prof_used += 2;
+            ctx->prof_open = cls;
+            ctx->prof_stream = s;
+        }
+    }
     CU(f());
     g_kernel_launches += kernels;
-    if (rec) {
-        CU(cudaEventRecord(ctx->prof_ev[ctx->prof_used + 1], s));
-        ctx->prof_cls.push_back(cls);
-        ctx->prof_bytes.push_back(bytes);
-        ctx->prof_used += 2;
+    if (ctx->prof_on && ctx->prof_open >= 0) {
+        ctx->prof_bytes.back() += bytes;
+        ctx->prof_n.back() += 1;
+        if (!ctx->prof_grouped) {
+            CU(cudaEventRecord(ctx->prof_ev[2 * (ctx->prof_cls.size() - 1) + 1], s));
+            ctx->prof_open = -1;
+        }
     }
     return MTAD_OK;
 }
@@ -594,14 +615,26 @@ int mtad_profile_begin(mtad_ctx* ctx, int max_launches) {
     }
     ctx->prof_cls.clear();
     ctx->prof_bytes.clear();
+    ctx->prof_n.clear();
     ctx->prof_used = 0;
+    ctx->prof_open = -1;
     ctx->prof_on = true;
+    return MTAD_OK;
+}
+
+int mtad_profile_grouped(mtad_ctx* ctx, int on) {
+    if (!ctx || ctx->prof_on) return MTAD_E_INVALID;
+    ctx->prof_grouped = on != 0;
     return MTAD_OK;
 }
 
 int mtad_profile_end(mtad_ctx* ctx, double* ms, double* bytes, int64_t* launches) {
     if (!ctx || !ms || !bytes || !launches) return MTAD_E_INVALID;
     ctx->prof_on = false;
+    if (ctx->prof_open >= 0) {
+        CU(cudaEventRecord(ctx->prof_ev[2 * (ctx->prof_cls.size() - 1) + 1], ctx->prof_stream));
+        ctx->prof_open = -1;
+    }
     for (int c = 0; c < MTAD_K_CLASSES; ++c) { ms[c] = 0; bytes[c] = 0; launches[c] = 0; }
     CU(cudaDeviceSynchronize());
     for (size_t i = 0; i < ctx->prof_cls.size(); ++i) {
@@ -610,7 +643,7 @@ int mtad_profile_end(mtad_ctx* ctx, double* ms, double* bytes, int64_t* launches
         const int c = ctx->prof_cls[i];
         ms[c] += t;
         bytes[c] += ctx->prof_bytes[i];
-        launches[c] += 1;
+        launches[c] += ctx->prof_n[i];
     }
     ctx->prof_used = 0;
     return MTAD_OK;
