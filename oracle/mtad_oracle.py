@@ -23,7 +23,10 @@ What follows the paper, and where:
   * beam sampling draft with the auxiliary model (Sec. 2.1, the p_beam
     equation), sampled without replacement with Gumbel-top-b;
   * optionally, the warping of the paper's experiments on every target row
-    before the rule (App. F: top-k, renormalise, top-p).
+    before the rule (App. F: top-k, renormalise, top-p);
+  * the rule of vanilla speculative decoding as a second accept mode
+    (Sec. 2.2: per-token ratio test against a uniform, stop at the first
+    rejection, resample from the normalised positive part of p - q).
 
 The decoder itself is only named by the paper (Llama / OPT families); the
 definition used is the Llama one: pre-RMSNorm, rotary embedding with
@@ -36,7 +39,9 @@ causal decoding; every tree node == the chain of its own path; cross-check
 against stock torch fp64 ops; log-softmax normalisation; prefix sums vs
 products of probabilities; hand-built accept cases incl. the non-monotone
 one; exhaustive enumeration at vocab 8, gamma 3; sampler frequencies;
-hand-computed warped rows, and brute-force subset search for top-p.
+hand-computed warped rows, and brute-force subset search for top-p;
+for speculative decoding the closed form "accept + residual == target
+distribution" at vocab 8, its threshold in u, and p == q accepting all.
 The *distribution* of the beam-sampling draft is pinned only through the
 Gumbel-top-b inclusion probabilities at vocab 8: beyond that it is
 "parity unpinned".
@@ -393,6 +398,73 @@ def verify_tree(model: OracleModel, cache: np.ndarray, L: int, root_tok: int, to
     rows = tree_rows(L, root_tok, tok, parent)
     logits = decoder_rows(model, cache, L, *rows)
     return verify_from_logits(logits, tok, parent, logq_ref, log_tau, u, chain=False, warp=warp)
+
+
+# ----------------------------------------------------------------------------
+# vanilla speculative decoding (Sec. 2.2), the rule MTAD is measured against
+# ----------------------------------------------------------------------------
+
+def spd_residual(logp_row: np.ndarray, logq_row: np.ndarray) -> np.ndarray:
+    """Unnormalised residual weights max(0, p - q) of Sec. 2.2, step 4 (the distribution a rejected position is
+    resampled from, norm(max(0, p - q)))."""
+    return np.maximum(0.0, np.exp(np.asarray(logp_row, np.float64)) - np.exp(np.asarray(logq_row, np.float64)))
+
+
+@dataclass
+class SpdResult:
+    eta: int
+    path: List[int]
+    out_tok: List[int]
+    out_lp: List[float]             # target log-probabilities of the emitted tokens
+    margin_accept: float            # smallest |log u_i - min(0, log p_i - log q_i)| over the tested positions
+    margin_bonus: float             # gap between the two largest perturbed values of the last draw
+    margin_bonus_robust: float      # the same gap when every log p may be off by +-tol against the winner
+    logits: Optional[np.ndarray] = None
+
+
+def spd_from_logits(logits: np.ndarray, tok: Sequence[int], logq_rows: np.ndarray, u_acc: Sequence[float],
+                    u_res: np.ndarray, tol: float = 2e-3) -> SpdResult:
+    """Sec. 2.2, steps 2-4: draft token i (drawn from q_i) is accepted with probability min(1, p_i(x_i) / q_i(x_i)),
+    i.e. iff u_i < that ratio; verification stops at the first rejection, whose position is resampled from
+    norm(max(0, p_i - q_i)); with every token accepted one more is drawn from the target's next row.
+    logits: [gamma + 1, V] target rows; logq_rows: [gamma, V] the auxiliary model's normalised log-distributions
+    at the draft positions; u_acc: [gamma] uniforms of the accept tests; u_res: [V] uniforms of the final draw
+    (Gumbel-argmax, as for the extra token of Algorithm 1)."""
+    logp = log_softmax(logits)
+    g = len(tok)
+    eta, margin = g, float("inf")
+    for i in range(g):
+        ratio = min(0.0, float(logp[i, tok[i]] - logq_rows[i, tok[i]]))
+        lu = math.log(u_acc[i])
+        margin = min(margin, abs(lu - ratio))
+        if not lu < ratio:
+            eta = i
+            break
+    if eta == g:
+        z = logp[g]
+        z_lo, z_hi = z - tol, z + tol
+    else:
+        p_row, q_row = np.exp(logp[eta]), np.exp(np.asarray(logq_rows[eta], np.float64))
+        with np.errstate(divide="ignore"):
+            z = np.log(np.maximum(0.0, p_row - q_row))
+            z_lo = np.log(np.maximum(0.0, p_row * math.exp(-tol) - q_row))
+            z_hi = np.log(np.maximum(0.0, p_row * math.exp(tol) - q_row))
+    t, gap = gumbel_argmax(z, u_res)
+    noise = -np.log(-np.log(np.asarray(u_res, dtype=np.float64)))
+    others = np.delete(z_hi + noise, t)
+    robust = float(z_lo[t] + noise[t] - (np.max(others) if others.size else NEG_INF))
+    path = list(range(eta))
+    out_tok = [int(tok[i]) for i in path] + [t]
+    out_lp = [float(logp[i, tok[i]]) for i in path] + [float(logp[eta, t])]
+    return SpdResult(eta, path, out_tok, out_lp, margin, gap, robust, logits)
+
+
+def verify_chain_spd(model: OracleModel, cache: np.ndarray, L: int, root_tok: int, draft_tok, logq_rows,
+                     u_acc, u_res) -> SpdResult:
+    parent = list(range(-1, len(draft_tok) - 1))
+    rows = tree_rows(L, root_tok, draft_tok, parent)
+    logits = decoder_rows(model, cache, L, *rows)
+    return spd_from_logits(logits, draft_tok, logq_rows, u_acc, u_res)
 
 
 def kv_commit(cache: np.ndarray, L: int, path: Sequence[int]) -> int:

@@ -421,3 +421,64 @@ def test_warped_verification_drops_tokens_outside_the_kept_set():
     b = O.verify_from_logits(logits, best, list(range(-1, g - 1)), [-3.0, -6.0, -9.0], np.log(0.3), u, chain=True,
                              warp=(V, 1.0))
     assert a.eta == b.eta and a.out_tok == b.out_tok and np.allclose(a.out_lp, b.out_lp, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# vanilla speculative decoding (Sec. 2.2)
+# ----------------------------------------------------------------------------------------------------------------
+
+def test_spd_accept_plus_residual_is_the_target_distribution():
+    """The identity that makes the rule lossless, from the oracle's own pieces at vocab 8:
+    q(y) min(1, p(y)/q(y)) + (1 - sum_x q(x) min(1, p(x)/q(x))) * res(y) / sum(res) = p(y)."""
+    p, q = _tables(21, 0.8)
+    for ctx in [(), (3,), (1, 6)]:
+        lp, lq = np.log(p[ctx]), np.log(q[ctx])
+        res = O.spd_residual(lp, lq)
+        acc = q[ctx] * np.minimum(1.0, p[ctx] / q[ctx])
+        out = acc + (1.0 - acc.sum()) * res / res.sum()
+        assert np.allclose(out, p[ctx], atol=1e-12)
+        assert np.all(res[p[ctx] <= q[ctx]] == 0) and np.all(res >= 0)
+
+
+def test_spd_threshold_stop_and_identical_models():
+    p, q = _tables(22, 1.0)
+    x = [2, 5, 1]
+    logits, _ = _chain_inputs(p, q, x)
+    logq_rows = np.stack([np.log(q[tuple(x[:i])]) for i in range(len(x))])
+    u_res = np.random.default_rng(0).uniform(0.01, 0.99, size=V)
+    ratio = [min(1.0, p[tuple(x[:i])][x[i]] / q[tuple(x[:i])][x[i]]) for i in range(3)]
+    # every u below its ratio: all accepted, the extra token is a draw from the row after the chain
+    r = O.spd_from_logits(logits, x, logq_rows, [0.999 * a for a in ratio], u_res)
+    assert r.eta == 3 and r.out_tok[:3] == x
+    assert r.out_tok[3] == O.gumbel_argmax(logits[3], u_res)[0]
+    # the threshold in u at a position with ratio < 1, and the stop at the first rejection
+    k = next(i for i in range(3) if ratio[i] < 1.0)
+    u = [0.999 * a for a in ratio]
+    u[k] = min(0.999999, ratio[k] * 1.001)
+    r = O.spd_from_logits(logits, x, logq_rows, u, u_res)
+    assert r.eta == k and len(r.out_tok) == k + 1
+    res = O.spd_residual(np.log(p[tuple(x[:k])]), logq_rows[k])
+    assert res[r.out_tok[-1]] > 0                                  # resampled where p exceeds q
+    with np.errstate(divide="ignore"):
+        assert r.out_tok[-1] == O.gumbel_argmax(np.log(res), u_res)[0]
+    # identical models: the ratio is 1 everywhere, every draft is accepted whatever u
+    lp_rows = np.stack([np.log(p[tuple(x[:i])]) for i in range(len(x))])
+    r = O.spd_from_logits(logits, x, lp_rows, [0.999999, 0.5, 1e-9], u_res)
+    assert r.eta == 3
+
+
+def test_spd_first_token_frequencies_follow_the_target():
+    """Monte-Carlo over seeded uniforms at vocab 8: the first emitted token (accepted draft or resampled) is
+    distributed as the target's first row (chi-square, 7 degrees of freedom)."""
+    p, q = _tables(23, 1.2)
+    rng = np.random.default_rng(1)
+    n = 6000
+    logits = np.log(p[()])[None].repeat(2, axis=0)
+    counts = np.zeros(V)
+    for _ in range(n):
+        x0 = int(rng.choice(V, p=q[()]))
+        r = O.spd_from_logits(np.stack([np.log(p[()]), np.log(p[(x0,)])]), [x0], np.log(q[()])[None],
+                              [float(rng.uniform(1e-12, 1))], rng.uniform(1e-12, 1, size=V))
+        counts[r.out_tok[0]] += 1
+    chi2 = float(np.sum((counts - n * p[()]) ** 2 / (n * p[()])))
+    assert chi2 < 24.3          # 99.9 % quantile of chi-square with 7 degrees of freedom
