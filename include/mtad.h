@@ -162,6 +162,22 @@ int mtad_verify_chain(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, cons
                       const float* draft_logq, float log_tau, const float* bonus_uniform,
                       const mtad_result* out, void* stream);
 
+/* The rule of vanilla speculative decoding (Sec. 2.2, steps 2-4) on a draft chain, as a second accept mode on the
+ * same target forward: token i is accepted iff accept_uniform[i] < min(1, p_i(x_i) / q_i(x_i)); the scan stops at
+ * the first rejection, whose position is resampled from norm(max(0, p_i - q_i)); with every token accepted one more
+ * token is drawn from the target's next row.  The last draw is a Gumbel-argmax over log of those weights with noise
+ * from resample_uniform (lowest token id on ties).
+ *   draft_tok        device [B, gamma] int32
+ *   draft_logq_rows  device [B, gamma, vocab] fp32  the auxiliary model's normalised log-distribution at every
+ *                    draft position (the whole row: the residual needs q at every token)
+ *   accept_uniform   device [B, gamma] fp32 in (0,1);  resample_uniform  device [B, vocab] fp32 in (0,1)
+ * Outputs as for mtad_verify_chain (path[i] = i; margin[0] = smallest |log u - log ratio| over the tested
+ * positions); kv_commit follows as usual.  The verify forward computes plain logits [rows, vocab] into the
+ * workspace; a warping set by mtad_set_warp is not applied in this mode.  gamma >= 1. */
+int mtad_verify_chain_spd(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, const int32_t* draft_tok,
+                          const float* draft_logq_rows, const float* accept_uniform, const float* resample_uniform,
+                          const mtad_result* out, void* stream);
+
 /* Verify a candidate tree (Sec. 3.3).  Node n of sequence b has token tok[b,n] and parent parent[b,n] (< n, or
  * -1 for a child of the root); n_nodes[b] <= max_nodes nodes are valid (n_nodes NULL: all max_nodes).
  * Candidate n at depth i passes iff log p(path to n) - logq_ref[b, i-1] > log_tau with

@@ -40,7 +40,8 @@ class Result(C.Structure):
 EXPORTS = ("mtad_workspace_bytes", "mtad_create", "mtad_destroy", "mtad_seq_set", "mtad_seq_get", "mtad_draft",
            "mtad_verify_chain", "mtad_verify_tree", "kv_commit", "mtad_status_str", "mtad_last_cuda_error",
            "mtad_profile_begin", "mtad_profile_end", "mtad_kernel_launches", "mtad_verify_chain_static",
-           "mtad_debug_gemm", "mtad_set_warp", "mtad_profile_grouped")
+           "mtad_debug_gemm", "mtad_set_warp", "mtad_profile_grouped",
+           "mtad_verify_chain_spd")
 MTAD_STATIC_SCRATCH_BYTES = 16 << 20
 KERNEL_CLASSES = ("prepare", "norm", "gemm", "rope_append", "attention", "lm_reduce", "accept", "commit")
 
@@ -69,6 +70,7 @@ def load_library() -> C.CDLL:
     lib.mtad_draft.argtypes = [P, I, I32P, I, I, P, P, P, P, P, P, P, P]
     lib.mtad_verify_chain.argtypes = [P, I, I32P, I, P, P, F, P, RS, P]
     lib.mtad_verify_tree.argtypes = [P, I, I32P, P, I, I, P, P, P, F, P, RS, P]
+    lib.mtad_verify_chain_spd.argtypes = [P, I, I32P, I, P, P, P, P, RS, P]
     lib.kv_commit.argtypes = [P, I, I32P, RS, P]
     lib.mtad_status_str.argtypes = [I]
     lib.mtad_status_str.restype = C.c_char_p
@@ -223,6 +225,17 @@ class Context:
                                          _ptr(bonus_uniform, torch.float32), C.byref(out.struct), _stream(stream))
         if check:
             self._check(rc, "mtad_verify_chain")
+        return rc
+
+    def mtad_verify_chain_spd(self, seqs, gamma: int, draft_tok, draft_logq_rows, accept_uniform, resample_uniform,
+                              out: ResultBuffers, stream=None, check=True) -> int:
+        rc = self._lib.mtad_verify_chain_spd(self.handle, len(seqs), _seqs(seqs), gamma,
+                                             _ptr(draft_tok, torch.int32), _ptr(draft_logq_rows, torch.float32),
+                                             _ptr(accept_uniform, torch.float32),
+                                             _ptr(resample_uniform, torch.float32), C.byref(out.struct),
+                                             _stream(stream))
+        if check:
+            self._check(rc, "mtad_verify_chain_spd")
         return rc
 
     def mtad_verify_tree(self, seqs, n_nodes, max_nodes: int, max_depth: int, tok, parent, logq_ref, log_tau: float,

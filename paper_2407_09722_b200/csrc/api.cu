@@ -498,7 +498,10 @@ bool result_ok(const mtad_result* r) {
 
 int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_nodes, int N, int D,
                   const int32_t* tok, const int32_t* parent, const float* logq_ref, float log_tau,
-                  const float* bonus_uniform, const mtad_result* out, void* stream) {
+                  const float* bonus_uniform, const mtad_result* out, void* stream,
+                  const float* spd_accept_uniform = nullptr) {
+    // spd_accept_uniform set: the rule of vanilla speculative decoding on a chain; logq_ref then holds the auxiliary
+    // model's log-distributions [B, gamma, V] and bonus_uniform the uniforms of the final draw
     if (!ctx) return MTAD_E_INVALID;
     if (!seqs_ok(ctx, B, seqs)) return B > (ctx ? ctx->max_batch : 0) ? MTAD_E_CAPACITY : MTAD_E_INVALID;
     if (N < 0 || D < 0) return MTAD_E_INVALID;
@@ -521,22 +524,28 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
         pa.sumsq_out = ctx->sc.sumsq_a;
     }
     RUN(MTAD_K_PREPARE, 0, 1, launch_prepare(ctx->target, ctx->st, ctx->rm, ctx->sc, pa, out->status, s));
-    const bool warped = ctx->warp_k > 0;       // warped rows are made from plain logits, after the forward
+    const bool spd = spd_accept_uniform != nullptr;
+    const bool warped = ctx->warp_k > 0 && !spd;   // warped rows are made from plain logits, after the forward
     if (tc) {
-        int rc = forward_rows_tc(ctx, ctx->target, ctx->tmaps, B, R, ub, bonus_uniform, out->status, warped, s);
+        int rc = forward_rows_tc(ctx, ctx->target, ctx->tmaps, B, R, ub, bonus_uniform, out->status, warped || spd, s);
         if (rc != MTAD_OK) return rc;
     } else {
         int rc = forward_rows(ctx, ctx->target, B, R, ub, s);
         if (rc != MTAD_OK) return rc;
-        if (!warped)
+        if (!warped && !spd)
             RUN(MTAD_K_LMRED, 0, R > 1 ? 2 : 1,
                 launch_lm_reduce(ctx->target, ctx->rm, ctx->sc, B, R, bonus_uniform, tok, parent, s));
     }
     if (warped)
         RUN(MTAD_K_LMRED, 0, 3,
             launch_warp_rows(ctx->target, ctx->rm, ctx->sc, B, R, ctx->warp_k, ctx->warp_p, bonus_uniform, s));
-    AcceptArgs aa{B, R, D, tok, parent, logq_ref, log_tau};
-    RUN(MTAD_K_ACCEPT, 0, 1, launch_accept(ctx->rm, ctx->sc, aa, *out, s));
+    if (spd) {
+        SpdArgs sa{B, R, D, tok, logq_ref, spd_accept_uniform, bonus_uniform};
+        RUN(MTAD_K_ACCEPT, 0, 1, launch_spd_accept(ctx->target, ctx->rm, ctx->sc, sa, *out, s));
+    } else {
+        AcceptArgs aa{B, R, D, tok, parent, logq_ref, log_tau};
+        RUN(MTAD_K_ACCEPT, 0, 1, launch_accept(ctx->rm, ctx->sc, aa, *out, s));
+    }
     ctx->last_B = B; ctx->last_R = R; ctx->last_D = D;
     ctx->last_chain = (parent == nullptr);
     memcpy(ctx->last_seqs, seqs, sizeof(int32_t) * B);
@@ -765,6 +774,14 @@ int mtad_verify_chain(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, cons
     // a chain is the tree parent[n] = n - 1; node j has depth j + 1, so log q(x**_{1:j+1}) = draft_logq[j]
     return verify_common(ctx, B, seqs, nullptr, gamma, gamma, draft_tok, nullptr, draft_logq, log_tau,
                          bonus_uniform, out, stream);
+}
+
+int mtad_verify_chain_spd(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, const int32_t* draft_tok,
+                          const float* draft_logq_rows, const float* accept_uniform, const float* resample_uniform,
+                          const mtad_result* out, void* stream) {
+    if (gamma < 1 || !accept_uniform || !draft_logq_rows) return MTAD_E_INVALID;
+    return verify_common(ctx, B, seqs, nullptr, gamma, gamma, draft_tok, nullptr, draft_logq_rows, -1.f,
+                         resample_uniform, out, stream, accept_uniform);
 }
 
 int mtad_verify_tree(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_nodes, int max_nodes,

@@ -216,6 +216,15 @@ struct AcceptArgs {
     const float* logq_ref;     // [B, max_depth]
     float log_tau;
 };
+struct SpdArgs {
+    int B, R, max_depth;
+    const int32_t* tok;             // [B, R-1]
+    const float* logq_rows;         // [B, R-1, V] the auxiliary model's log-distributions at the draft positions
+    const float* accept_uniform;    // [B, R-1]
+    const float* resample_uniform;  // [B, V]
+};
+cudaError_t launch_spd_accept(const ModelView& m, const RowMeta& rm, const Scratch& sc, const SpdArgs& a,
+                              const mtad_result& out, cudaStream_t st);
 cudaError_t launch_accept(const RowMeta& rm, const Scratch& sc, const AcceptArgs& a, const mtad_result& out,
                           cudaStream_t st);
 cudaError_t launch_kv_commit(const ModelView& m, const SeqState& s, int B, const int32_t* call_seq_dev,
