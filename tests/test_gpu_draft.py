@@ -88,6 +88,32 @@ def test_draft_verify_commit_iterations(gamma, b, chain):
     assert skipped <= 3
 
 
+def test_draft_wide_vocabulary():
+    """Vocabulary 32000: the selection runs over 32 chunks per beam row, as at full size."""
+    target = S.ModelShape(1, 128, 2, 2, 64, 344, 32000)
+    aux = S.ModelShape(1, 128, 2, 2, 64, 512, 32000)
+    gm = GpuModel(target, max_batch=1, max_nodes=16, capacity=128, aux=aux, aux_capacity=128)
+    L, root, gamma, b = 20, 7, 3, 4
+    gm.inject(0, L)
+    gm.inject_aux(0, L)
+    gm.ctx.mtad_seq_set(0, L, root, aux_len=L)
+    acache = gm.aux_cache_bits(0, L)
+    skipped = 0
+    for it in range(3):
+        u = S.uniforms(0, (33 << 40) | it, gamma * b * 32000, "cuda").view(1, gamma, b, 32000)
+        g = _draft_gpu(gm, 0, gamma, b, u)
+        dr = O.draft_beam(gm.oracle_aux(), acache, L, [root], gamma, b, u[0].cpu().numpy())
+        if dr.min_gap < 1e-3:
+            skipped += 1
+        else:
+            assert g["tok"][0].tolist() == dr.tok and g["parent"][0].tolist() == dr.parent
+            assert g["best_path"][0].tolist() == dr.best_path
+            assert np.max(np.abs(g["node_logq"][0].cpu().numpy() - np.asarray(dr.logq))) < LP_TOL
+            assert np.max(np.abs(g["logq_ref"][0].cpu().numpy() - np.asarray(dr.logq_ref))) < LP_TOL
+        gm.ctx.mtad_seq_set(0, L, root, aux_len=L)          # the same state again: only the noise changes
+    assert skipped <= 1
+
+
 def test_draft_rejects_bad_arguments():
     gm = GpuModel(W.target, max_batch=1, max_nodes=40, capacity=128, aux=W.aux, aux_capacity=128)
     V = W.target.vocab

@@ -15,6 +15,7 @@ pytestmark = pytest.mark.gpu
 
 TINY = S.WORKLOADS["tiny"].target
 GQA64 = S.ModelShape(3, 192, 6, 2, 64, 328, 500)
+WIDE_VOCAB = S.ModelShape(1, 128, 2, 2, 64, 344, 32000)     # 32 chunks of the vocabulary per row, as at full size
 
 
 def _likely_tree(gm, seq, L, root, parent, ranks, dq):
@@ -48,7 +49,8 @@ def _likely_tree(gm, seq, L, root, parent, ranks, dq):
     return S.DraftTree(tok, list(parent), depth, lq, path, [lq[n] for n in path])
 
 
-@pytest.mark.parametrize("shape,warp", [(TINY, (10, 0.9)), (TINY, (4, 0.6)), (GQA64, (16, 0.95)), (TINY, (1, 0.9))])
+@pytest.mark.parametrize("shape,warp", [(TINY, (10, 0.9)), (TINY, (4, 0.6)), (GQA64, (16, 0.95)), (TINY, (1, 0.9)),
+                                        (WIDE_VOCAB, (10, 0.9))])
 def test_warped_chain_matches_oracle(shape, warp):
     gm = GpuModel(shape, max_batch=2, max_nodes=16, capacity=160)
     rng = np.random.default_rng(warp[0])
