@@ -58,6 +58,7 @@ enum {
 #define MTAD_ST_BAD_COUNT   16u  /* n_nodes[b] outside [0, max_nodes] */
 #define MTAD_ST_TIMEOUT     32u  /* a bounded wait inside a kernel gave up */
 #define MTAD_ST_AUX_PENDING 64u  /* more than MTAD_MAX_DEPTH + 1 tokens wait to be replayed by the auxiliary model */
+#define MTAD_ST_NONFINITE  128u  /* a row of target logits was not finite (NaN or infinite weights, cache or input) */
 #define MTAD_MAX_BEAM 8          /* beam width of mtad_draft */
 
 /* A Llama-style decoder (pre-RMSNorm, rotary embedding with half-split pairing (i, i + head_dim/2), grouped-

@@ -43,6 +43,7 @@ EXPORTS = ("mtad_workspace_bytes", "mtad_create", "mtad_destroy", "mtad_seq_set"
            "mtad_debug_gemm", "mtad_set_warp", "mtad_profile_grouped",
            "mtad_verify_chain_spd")
 MTAD_STATIC_SCRATCH_BYTES = 16 << 20
+MTAD_ST_TIMEOUT, MTAD_ST_AUX_PENDING, MTAD_ST_NONFINITE = 32, 64, 128      # device status bits (mtad.h)
 KERNEL_CLASSES = ("prepare", "norm", "gemm", "rope_append", "attention", "lm_reduce", "accept", "commit")
 
 _lib = None

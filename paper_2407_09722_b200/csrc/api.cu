@@ -478,7 +478,7 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
                 if (int rc = launch(o + k, 1)) return rc;
         }
     }
-    if (!lm_plain) RUN(MTAD_K_LMRED, 0, 2, launch_lm_merge(m, ctx->rm, sc, B, R, lm_tiles128, uniforms, s));
+    if (!lm_plain) RUN(MTAD_K_LMRED, 0, 2, launch_lm_merge(m, ctx->rm, sc, B, R, lm_tiles128, uniforms, status, s));
     return MTAD_OK;
 }
 
@@ -534,7 +534,7 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
         if (rc != MTAD_OK) return rc;
         if (!warped && !spd)
             RUN(MTAD_K_LMRED, 0, R > 1 ? 2 : 1,
-                launch_lm_reduce(ctx->target, ctx->rm, ctx->sc, B, R, bonus_uniform, tok, parent, s));
+                launch_lm_reduce(ctx->target, ctx->rm, ctx->sc, B, R, bonus_uniform, tok, parent, out->status, s));
     }
     if (warped)
         RUN(MTAD_K_LMRED, 0, 3,

@@ -202,10 +202,10 @@ cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& r
 cudaError_t launch_attention_combine(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int nsplit,
                                      bool emit_split, bool pdl, cudaStream_t st);
 cudaError_t launch_lm_merge(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int n_tiles,
-                            const float* bonus_uniform, cudaStream_t st);
+                            const float* bonus_uniform, uint32_t* status, cudaStream_t st);
 cudaError_t launch_lm_reduce(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R,
                              const float* bonus_uniform, const int32_t* tok, const int32_t* parent,
-                             cudaStream_t st);
+                             uint32_t* status, cudaStream_t st);
 // Warped target rows from sc.logits: fills row_lse (over the kept tokens), row_cand, row_cand_lp and node_lp.
 cudaError_t launch_warp_rows(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int top_k,
                              float top_p, const float* bonus_uniform, cudaStream_t st);

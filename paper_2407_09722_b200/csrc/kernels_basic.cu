@@ -360,7 +360,7 @@ __global__ void __launch_bounds__(1024) lm_reduce_kernel(const float* __restrict
                                                          const float* __restrict__ uni,
                                                          const int32_t* __restrict__ slot,
                                                          float* __restrict__ row_lse, int32_t* __restrict__ row_cand,
-                                                         float* __restrict__ row_cand_lp) {
+                                                         float* __restrict__ row_cand_lp, uint32_t* status) {
     const int t = blockIdx.x, bi = t / R;
     if (slot[t] < 0) {
         if (threadIdx.x == 0) { row_lse[t] = 0.f; row_cand[t] = 0; row_cand_lp[t] = 0.f; }
@@ -396,9 +396,13 @@ __global__ void __launch_bounds__(1024) lm_reduce_kernel(const float* __restrict
     }
     if (threadIdx.x == 0) {
         const float lse = sm[0] + logf(ss[0]);
+        // a row of NaN logits wins no comparison and leaves no candidate: flag it instead of indexing with it
+        const bool none = (unsigned)si[0] >= (unsigned)V;
+        if (none || !isfinite(lse)) atomicOr(&status[bi], MTAD_ST_NONFINITE);
+        const int c = none ? 0 : si[0];
         row_lse[t] = lse;
-        row_cand[t] = si[0];
-        row_cand_lp[t] = z[si[0]] - lse;
+        row_cand[t] = c;
+        row_cand_lp[t] = z[c] - lse;
     }
 }
 
@@ -424,9 +428,9 @@ __global__ void node_lp_kernel(const float* __restrict__ logits, int V, int B, i
 
 cudaError_t launch_lm_reduce(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R,
                              const float* bonus_uniform, const int32_t* tok, const int32_t* parent,
-                             cudaStream_t st) {
+                             uint32_t* status, cudaStream_t st) {
     lm_reduce_kernel<<<B * R, 1024, 0, st>>>(sc.logits, m.d.vocab, R, bonus_uniform, rm.slot, sc.row_lse, sc.row_cand,
-                                             sc.row_cand_lp);
+                                             sc.row_cand_lp, status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (R > 1) {
@@ -443,7 +447,7 @@ cudaError_t launch_lm_reduce(const ModelView& m, const RowMeta& rm, const Scratc
 __global__ void lm_merge_kernel(const float4* __restrict__ part, int n_tiles, int V, int R,
                                 const float* __restrict__ uni, const int32_t* __restrict__ slot,
                                 float* __restrict__ row_lse, int32_t* __restrict__ row_cand,
-                                float* __restrict__ row_cand_lp) {
+                                float* __restrict__ row_cand_lp, uint32_t* status) {
     const int t = blockIdx.x, bi = t / R;
     if (slot[t] < 0) {
         if (threadIdx.x == 0) { row_lse[t] = 0.f; row_cand[t] = 0; row_cand_lp[t] = 0.f; }
@@ -477,7 +481,10 @@ __global__ void lm_merge_kernel(const float4* __restrict__ part, int n_tiles, in
     }
     if (threadIdx.x == 0) {
         const float lse = sm[0] + logf(ss[0]);
-        const int c = si[0];
+        // a row of NaN logits wins no comparison and leaves no candidate: flag it instead of indexing with it
+        const bool none = (unsigned)si[0] >= (unsigned)V;
+        if (none || !isfinite(lse)) atomicOr(&status[bi], MTAD_ST_NONFINITE);
+        const int c = none ? 0 : si[0];
         row_lse[t] = lse;
         row_cand[t] = c;
         // the partial keeps logit + noise; take the noise off again to get the candidate's logit
@@ -495,9 +502,9 @@ __global__ void node_lp_from_z_kernel(const float* __restrict__ node_z, const in
 }
 
 cudaError_t launch_lm_merge(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int n_tiles,
-                            const float* bonus_uniform, cudaStream_t st) {
+                            const float* bonus_uniform, uint32_t* status, cudaStream_t st) {
     lm_merge_kernel<<<B * R, 256, 0, st>>>(sc.lm_part, n_tiles, m.d.vocab, R, bonus_uniform, rm.slot, sc.row_lse,
-                                           sc.row_cand, sc.row_cand_lp);
+                                           sc.row_cand, sc.row_cand_lp, status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     node_lp_from_z_kernel<<<(B * R + 127) / 128, 128, 0, st>>>(sc.node_z, rm.prow, sc.row_lse, sc.node_lp, B * R);
