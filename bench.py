@@ -397,21 +397,35 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
 
     # ---- end to end: host buffers in, host results out, every step --------------------------------------------------
     reset()
-    stage = {k: torch.empty_like(v, device="cuda") for k, v in inputs[0].host.items()}
-    u_stage = torch.empty_like(unis[0])
-    out_host = {n: torch.empty_like(getattr(res, n), device="cpu").pin_memory()
-                for n in ("eta", "n_out", "out_tok", "out_lp", "status")}
-    h2d = sum(v.numel() * v.element_size() for v in inputs[0].host.values()) + u_stage.numel() * 4
-    d2h = sum(v.numel() * v.element_size() for v in out_host.values())
+    # per step: ONE host-to-device copy of a pinned block (uniforms, then the draft arrays) and ONE device-to-host
+    # copy of the result head (eta, n_out, status, out_tok, out_lp)
+    names = list(inputs[0].host.keys())
+
+    def pack(i):
+        parts = [unis_host[i].view(torch.int32).flatten()]
+        parts += [inputs[i].host[k].view(torch.int32).flatten() for k in names]
+        return torch.cat(parts).pin_memory()
+
+    packed = [pack(i) for i in range(total_steps)]
+    stage_buf = torch.empty_like(packed[0], device="cuda")
+    off = unis_host[0].numel()
+    u_stage = stage_buf[:off].view(torch.float32).view_as(unis[0])
+    stage = {}
+    for k in names:
+        v = inputs[0].host[k]
+        piece = stage_buf[off:off + v.numel()]
+        stage[k] = (piece if v.dtype == torch.int32 else piece.view(v.dtype)).view_as(v)
+        off += v.numel()
+    head_host = torch.empty_like(res.head, device="cpu").pin_memory()
+    out_host = res.head_views(head_host)
+    h2d = packed[0].numel() * 4
+    d2h = head_host.numel() * 4
 
     def e2e_step(i):
-        for k, v in inputs[i].host.items():
-            stage[k].copy_(v, non_blocking=True)
-        u_stage.copy_(unis_host[i], non_blocking=True)
+        stage_buf.copy_(packed[i], non_blocking=True)
         inputs[i].verify(ctx, seqs, log_tau, u_stage, res, dev=stage)
         ctx.kv_commit(seqs, res)
-        for n, t in out_host.items():
-            t.copy_(getattr(res, n), non_blocking=True)
+        head_host.copy_(res.head, non_blocking=True)
         torch.cuda.synchronize()
         # log-likelihood of the emitted tokens under the target, for the output perplexity (Eq. 1)
         n = out_host["n_out"].long()

@@ -150,23 +150,36 @@ class ResultBuffers:
         i32 = dict(dtype=torch.int32, device=device)
         f32 = dict(dtype=torch.float32, device=device)
         self.B, self.N, self.D = B, N, D
-        self.eta = torch.zeros(B, **i32)
-        self.winner = torch.zeros(B, **i32)
-        self.path = torch.zeros(B, max(D, 1), **i32)
-        self.n_out = torch.zeros(B, **i32)
-        self.out_tok = torch.zeros(B, D + 1, **i32)
-        self.out_lp = torch.zeros(B, D + 1, **f32)
-        self.node_lp = torch.zeros(B, max(N, 1), **f32)
-        self.node_LP = torch.zeros(B, max(N, 1), **f32)
-        self.row_lse = torch.zeros(B, N + 1, **f32)
-        self.row_cand = torch.zeros(B, N + 1, **i32)
-        self.row_cand_lp = torch.zeros(B, N + 1, **f32)
-        self.margin = torch.zeros(B, 2, **f32)
-        self.status = torch.zeros(B, **i32)
+        # one allocation, the members are views: `head` (eta, n_out, status, out_tok, out_lp - what a decode loop reads
+        # back every step) is contiguous, so that a caller can fetch it with a single device-to-host copy
+        shapes = [("eta", (B,), torch.int32), ("n_out", (B,), torch.int32), ("status", (B,), torch.int32),
+                  ("out_tok", (B, D + 1), torch.int32), ("out_lp", (B, D + 1), torch.float32),
+                  ("winner", (B,), torch.int32), ("path", (B, max(D, 1)), torch.int32),
+                  ("node_lp", (B, max(N, 1)), torch.float32), ("node_LP", (B, max(N, 1)), torch.float32),
+                  ("row_lse", (B, N + 1), torch.float32), ("row_cand", (B, N + 1), torch.int32),
+                  ("row_cand_lp", (B, N + 1), torch.float32), ("margin", (B, 2), torch.float32)]
+        words = [int(math.prod(sh)) for _, sh, _ in shapes]
+        self.buf = torch.zeros(sum(words), **i32)
+        self.head_fields, off = {}, 0
+        for (name, sh, dt), n in zip(shapes, words):
+            v = self.buf[off:off + n]
+            setattr(self, name, (v if dt == torch.int32 else v.view(torch.float32)).view(*sh))
+            if name in ("eta", "n_out", "status", "out_tok", "out_lp"):
+                self.head_fields[name] = (off, sh, dt)
+            off += n
+        self.head = self.buf[:sum(words[:5])]
         self.struct = Result(*[getattr(self, n).data_ptr() for n, _ in Result._fields_])
 
     def host(self) -> Dict[str, torch.Tensor]:
         return {n: getattr(self, n).cpu() for n, _ in Result._fields_}
+
+    def head_views(self, host_head: torch.Tensor) -> Dict[str, torch.Tensor]:
+        """Views of a host copy of `head` (an int32 tensor of the same length) under the members' names."""
+        out = {}
+        for name, (off, sh, dt) in self.head_fields.items():
+            v = host_head[off:off + int(math.prod(sh))]
+            out[name] = (v if dt == torch.int32 else v.view(torch.float32)).view(*sh)
+        return out
 
 
 class Context:
