@@ -538,7 +538,8 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
     }
     if (warped)
         RUN(MTAD_K_LMRED, 0, 3,
-            launch_warp_rows(ctx->target, ctx->rm, ctx->sc, B, R, ctx->warp_k, ctx->warp_p, bonus_uniform, s));
+            launch_warp_rows(ctx->target, ctx->rm, ctx->sc, B, R, ctx->warp_k, ctx->warp_p, bonus_uniform,
+                             out->status, s));
     if (spd) {
         SpdArgs sa{B, R, D, tok, logq_ref, spd_accept_uniform, bonus_uniform};
         RUN(MTAD_K_ACCEPT, 0, 1, launch_spd_accept(ctx->target, ctx->rm, ctx->sc, sa, *out, s));

@@ -208,7 +208,7 @@ cudaError_t launch_lm_reduce(const ModelView& m, const RowMeta& rm, const Scratc
                              uint32_t* status, cudaStream_t st);
 // Warped target rows from sc.logits: fills row_lse (over the kept tokens), row_cand, row_cand_lp and node_lp.
 cudaError_t launch_warp_rows(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int top_k,
-                             float top_p, const float* bonus_uniform, cudaStream_t st);
+                             float top_p, const float* bonus_uniform, uint32_t* status, cudaStream_t st);
 struct AcceptArgs {
     int B, R, max_depth;
     const int32_t* tok;        // [B, R-1]

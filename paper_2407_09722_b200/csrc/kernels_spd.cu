@@ -58,6 +58,16 @@ __global__ void __launch_bounds__(1024) spd_accept_kernel(const float* __restric
         }
         __syncthreads();
     }
+    // rows of NaN logits: flag the sequence and accept nothing, as the other modes do
+    bool finite = true;
+    for (int r = 0; r < R; ++r) finite = finite && isfinite(s_lse[r]);
+    if (!finite) {
+        if (tid == 0) {
+            atomicOr(&out.status[bi], MTAD_ST_NONFINITE);
+            out.eta[bi] = 0; out.winner[bi] = -1; out.n_out[bi] = 0;
+        }
+        return;
+    }
     // the accept scan: stops at the first rejection
     if (tid == 0) {
         int eta = g;

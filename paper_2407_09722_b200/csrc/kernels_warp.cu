@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(32) warp_merge_kernel(const WarpPart* __restri
                                                         int V, int R, const float* __restrict__ uni,
                                                         const int32_t* __restrict__ slot, WarpRow* __restrict__ rows,
                                                         float* __restrict__ row_lse, int32_t* __restrict__ row_cand,
-                                                        float* __restrict__ row_cand_lp) {
+                                                        float* __restrict__ row_cand_lp, uint32_t* status) {
     const int t = blockIdx.x, bi = t / R, lane = threadIdx.x;
     WarpRow* row = rows + t;
     if (slot[t] < 0) {
@@ -133,6 +133,8 @@ __global__ void __launch_bounds__(32) warp_merge_kernel(const WarpPart* __restri
             const float y = s_tz[i] - logf(-logf(uni[(size_t)bi * V + s_tv[i]]));
             if (y > by || (y == by && s_tv[i] < bv)) { by = y; bv = s_tv[i]; blp = lp; }
         }
+        // a row of NaN logits ranks no token: flag the sequence, as the unwarped path does
+        if (found == 0 || bv == NONE || !isfinite(lse)) atomicOr(&status[bi], MTAD_ST_NONFINITE);
         row_lse[t] = lse;
         row_cand[t] = bv == NONE ? 0 : bv;
         row_cand_lp[t] = blp;
@@ -156,7 +158,7 @@ __global__ void warp_node_lp_kernel(const WarpRow* __restrict__ rows, const int3
 }
 
 cudaError_t launch_warp_rows(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int top_k,
-                             float top_p, const float* bonus_uniform, cudaStream_t st) {
+                             float top_p, const float* bonus_uniform, uint32_t* status, cudaStream_t st) {
     const int V = m.d.vocab, T = B * R;
     int nch = (V + 1023) / 1024;
     nch = nch < 1 ? 1 : (nch > MTAD_DRAFT_CHUNKS ? MTAD_DRAFT_CHUNKS : nch);
@@ -164,7 +166,7 @@ cudaError_t launch_warp_rows(const ModelView& m, const RowMeta& rm, const Scratc
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     warp_merge_kernel<<<T, 32, 0, st>>>(sc.warp_part, nch, top_k, top_p, V, R, bonus_uniform, rm.slot, sc.warp_row,
-                                        sc.row_lse, sc.row_cand, sc.row_cand_lp);
+                                        sc.row_lse, sc.row_cand, sc.row_cand_lp, status);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     warp_node_lp_kernel<<<(T + 127) / 128, 128, 0, st>>>(sc.warp_row, rm.prow, rm.tok, sc.node_lp, T);

@@ -218,7 +218,7 @@ def test_host_side_rejections(tiny):
         c.mtad_seq_set(0, tiny.capacity + 1, 0)
 
 
-@pytest.mark.parametrize("path", ["tc", "simt"])
+@pytest.mark.parametrize("path", ["tc", "simt", "warped"])
 def test_non_finite_logits_set_a_status_bit(path, monkeypatch):
     """A NaN in the committed cache makes every logit of the sequence NaN: no arg-max candidate exists.  The call
     must report MTAD_ST_NONFINITE for that sequence (and leave the other one alone), not index with the missing
@@ -230,7 +230,8 @@ def test_non_finite_logits_set_a_status_bit(path, monkeypatch):
         gm.inject(seq, 40)
     gm.cache[0, 1, 0, 0, 3, 5] = float("nan")           # layer 0, sequence 1, K, head 0, position 3
     cases = [SeqCase(seq, 40, 3 + seq, S.chain_tree(4, TINY.vocab, stream=90 + seq)) for seq in range(2)]
-    res = run_gpu(gm, cases, math.log(0.1), _u(6, 0, 2, TINY.vocab), chain=True)
+    res = run_gpu(gm, cases, math.log(0.1), _u(6, 0, 2, TINY.vocab), chain=True,
+                  warp=(10, 0.9) if path == "warped" else None)
     h = res.host()
     assert int(h["status"][0]) == 0 and int(h["n_out"][0]) >= 1
     assert int(h["status"][1]) & Bn.MTAD_ST_NONFINITE and int(h["n_out"][1]) == 0

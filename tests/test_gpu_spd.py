@@ -69,6 +69,26 @@ def test_spd_chain_matches_oracle(shape, scale):
     assert min(etas) < max(etas)            # both rejections and longer acceptances occurred
 
 
+def test_spd_non_finite_logits_set_a_status_bit():
+    gm = GpuModel(TINY, max_batch=2, max_nodes=8, capacity=96)
+    V, g = TINY.vocab, 4
+    for seq in range(2):
+        gm.inject(seq, 40)
+        gm.ctx.mtad_seq_set(seq, 40, 3 + seq)
+    gm.cache[0, 1, 0, 0, 3, 5] = float("nan")           # layer 0, sequence 1, K, head 0, position 3
+    rng = np.random.default_rng(2)
+    rows, toks = zip(*(_draft(rng, g, V, 0.5) for _ in range(2)))
+    res = M.ResultBuffers(2, g, g)
+    gm.ctx.mtad_verify_chain_spd([0, 1], g, torch.tensor(toks, dtype=torch.int32, device="cuda"),
+                                 torch.tensor(np.asarray(rows, np.float32), device="cuda"),
+                                 torch.full((2, g), 0.5, device="cuda"), S.bonus_uniforms(1, 0, 2, V, "cuda"), res)
+    gm.ctx.kv_commit([0, 1], res)
+    h = res.host()
+    assert int(h["status"][0]) == 0 and int(h["n_out"][0]) >= 1
+    assert int(h["status"][1]) & M.binding.MTAD_ST_NONFINITE and int(h["n_out"][1]) == 0
+    assert gm.ctx.mtad_seq_get(1) == (40, 4)
+
+
 def test_spd_rejects_bad_arguments():
     gm = GpuModel(TINY, max_batch=1, max_nodes=8, capacity=96)
     V = TINY.vocab
