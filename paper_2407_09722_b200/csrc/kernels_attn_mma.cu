@@ -89,7 +89,7 @@ __device__ __forceinline__ void split2(float x, float y, uint32_t& hi, uint32_t&
 // keys of the split; attn_combine_kernel merges the splits in order.  q_hi / q_lo hold the query rows times
 // log2(e) / sqrt(HD), so the softmax numerators are exp2(s - m); m is stored back in natural-log units.
 template <int HD, int CNT, bool PACK>
-__global__ void __launch_bounds__(128, CNT == 1 ? 4 : 3) attn_mma_kernel(const __grid_constant__ CUtensorMap kvmap,
+__global__ void __launch_bounds__(CNT == 4 ? 192 : 128, CNT == 1 ? 4 : (CNT == 4 ? 2 : 3)) attn_mma_kernel(const __grid_constant__ CUtensorMap kvmap,
                                                           const __nv_bfloat16* __restrict__ q_hi,
                                                           const __nv_bfloat16* __restrict__ q_lo, RowMeta rm,
                                                           float* __restrict__ part, int layer, int max_batch, int Hq,
@@ -267,7 +267,9 @@ __global__ void __launch_bounds__(128, CNT == 1 ? 4 : 3) attn_mma_kernel(const _
     const bool spec = k_begin + KT > L;               // the tile reaches into the draft rows: masks apply
     const uint32_t ks_base = s_u32(smem + buf * TILE_BYTES), vs_base = ks_base + KT * ROWB;
 
-    for (int mt = warp / kparts; mt < n_mt; mt += 4 / kparts) {
+    // (whole-tile mode: the block has four to six warps, one query tile per warp and round)
+    const int mt_step = kparts > 1 ? 4 / kparts : (int)(blockDim.x >> 5);
+    for (int mt = warp / kparts; mt < n_mt; mt += mt_step) {
         const int slab = kparts > 1 ? mt : warp;
         if (kparts == 1 && mt != warp) {
             __syncwarp();                             // the previous tile's fragments have been read
@@ -521,7 +523,10 @@ cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& r
     if (!m.kv_map_ok) return cudaErrorInvalidValue;
     // query tiles kept in shared memory: all of them (at most two) when the warps split keys, else one per warp
     const int n_mt_max = ((Hq / Hkv) * R + 15) / 16;
-    const int nslab = n_mt_max <= 2 ? n_mt_max : 4;
+    // whole-tile mode with five or six query tiles per KV head: one warp per tile instead of four warps in two rounds
+    // (a 64-node tree plus its root is five tiles)
+    const int n_warps = (n_mt_max == 5 || n_mt_max == 6) ? n_mt_max : 4;
+    const int nslab = n_mt_max <= 2 ? n_mt_max : n_warps;
     const int ring = attn_ring(hd, nslab, (long long)Hkv * B);
     const int nb = nsp == 1 ? 1 : (nsp == 2 ? 2 : ring);
     const size_t smem = attn_smem(hd, nslab, nb);
@@ -531,7 +536,7 @@ cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& r
     auto go = [&](auto kernel) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 116 * 1024);
         if (e != cudaSuccess) return e;
-        return launch_pdl(kernel, grid, dim3(128), smem, st, pdl, m.kv_map, (const __nv_bfloat16*)sc.q_hi,
+        return launch_pdl(kernel, grid, dim3(32 * n_warps), smem, st, pdl, m.kv_map, (const __nv_bfloat16*)sc.q_hi,
                           (const __nv_bfloat16*)sc.q_lo, rm, sc.attn_part, layer, m.max_batch, Hq, Hkv, R, nsplit,
                           nslab, nsp, nb, early, status);
     };
