@@ -148,7 +148,6 @@ class ResultBuffers:
 
     def __init__(self, B: int, N: int, D: int, device="cuda"):
         i32 = dict(dtype=torch.int32, device=device)
-        f32 = dict(dtype=torch.float32, device=device)
         self.B, self.N, self.D = B, N, D
         # one allocation, the members are views: `head` (eta, n_out, status, out_tok, out_lp - what a decode loop reads
         # back every step) is contiguous, so that a caller can fetch it with a single device-to-host copy

@@ -236,3 +236,16 @@ def test_non_finite_logits_set_a_status_bit(path, monkeypatch):
     assert int(h["status"][0]) == 0 and int(h["n_out"][0]) >= 1
     assert int(h["status"][1]) & Bn.MTAD_ST_NONFINITE and int(h["n_out"][1]) == 0
     assert gm.ctx.mtad_seq_get(1) == (40, 4)              # nothing committed for the flagged sequence
+
+
+def test_result_head_is_one_contiguous_copy(tiny):
+    """The members a decode loop reads back every step (eta, n_out, status, out_tok, out_lp) lie in one block: a
+    single device-to-host copy of `head` gives the same values as the member-by-member copies."""
+    tiny.inject(0, 50)
+    res = run_gpu(tiny, [SeqCase(0, 50, 8, S.chain_tree(5, TINY.vocab, stream=123))], math.log(0.1),
+                  _u(7, 0, 1, TINY.vocab), chain=True)
+    h = res.host()
+    hv = res.head_views(res.head.cpu())
+    assert set(hv) == {"eta", "n_out", "status", "out_tok", "out_lp"}
+    for name, v in hv.items():
+        assert torch.equal(v, h[name]), name
