@@ -162,6 +162,86 @@ __device__ __forceinline__ void store_terms(float y, __nv_bfloat16* x, size_t K,
     if (terms == 3) x[2 * K] = __float2bfloat16_rn(r - __bfloat162float(l));
 }
 
+// One embedding row -> the fp32 hidden row and (tensor-core path) its bf16 operand terms times the first norm's gain;
+// returns this thread's share of the row's sum of squares.  16-byte loads, four in flight per thread: a scalar loop
+// whose loads wait behind the previous iteration's stores pays one DRAM latency per element (32 us for a 4096-wide
+// row).  d is a multiple of 8; rows that are not 16-byte aligned take the scalar loop.
+__device__ __forceinline__ float embed_row(const __nv_bfloat16* __restrict__ src_row, bool ok, int d,
+                                           float* __restrict__ hidden_row, const __nv_bfloat16* __restrict__ gain,
+                                           __nv_bfloat16* x_row, int terms) {
+    float ss = 0.f;
+    const bool vec = ((reinterpret_cast<uintptr_t>(src_row) | reinterpret_cast<uintptr_t>(hidden_row) |
+                       reinterpret_cast<uintptr_t>(gain) | reinterpret_cast<uintptr_t>(x_row)) & 15) == 0;
+    if (!vec) {
+        for (int i = threadIdx.x; i < d; i += blockDim.x) {
+            const float v = ok ? __bfloat162float(src_row[i]) : 0.f;
+            hidden_row[i] = v;
+            if (x_row) {
+                store_terms(v * __bfloat162float(gain[i]), x_row + i, d, terms);
+                ss += v * v;
+            }
+        }
+        return ss;
+    }
+    const int nv = d >> 3;
+    const uint4* src = reinterpret_cast<const uint4*>(src_row);
+    const uint4* gsrc = reinterpret_cast<const uint4*>(gain);
+    for (int c0 = threadIdx.x; c0 < nv; c0 += 4 * blockDim.x) {
+        uint4 q[4], gq[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int c = c0 + k * blockDim.x;
+            q[k] = (ok && c < nv) ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+            gq[k] = (x_row && c < nv) ? __ldg(gsrc + c) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int c = c0 + k * blockDim.x;
+            if (c >= nv) continue;
+            const uint32_t w[4] = {q[k].x, q[k].y, q[k].z, q[k].w}, gw[4] = {gq[k].x, gq[k].y, gq[k].z, gq[k].w};
+            float v[8];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                v[2 * e] = __uint_as_float(w[e] << 16);
+                v[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+            }
+            float4* h4 = reinterpret_cast<float4*>(hidden_row + (size_t)c * 8);
+            h4[0] = make_float4(v[0], v[1], v[2], v[3]);
+            h4[1] = make_float4(v[4], v[5], v[6], v[7]);
+            if (x_row) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    store_terms(v[2 * e] * __uint_as_float(gw[e] << 16), x_row + (size_t)c * 8 + 2 * e, d, terms);
+                    store_terms(v[2 * e + 1] * __uint_as_float(gw[e] & 0xffff0000u), x_row + (size_t)c * 8 + 2 * e + 1, d,
+                                terms);
+                    ss += v[2 * e] * v[2 * e] + v[2 * e + 1] * v[2 * e + 1];
+                }
+            }
+        }
+    }
+    return ss;
+}
+
+// Rotary frequencies base^(-2i/hd), i < hd/2, computed once on the host in double and passed to the kernels that
+// build a call's rotary table; the angle pos * frequency is reduced to [-pi, pi] in double (a few fused
+// multiply-adds) and its sine and cosine taken in fp32: double-precision sincos of an unreduced angle was most of
+// the row-preparation kernels' time.
+struct RopeInv {
+    double v[64];
+};
+inline RopeInv rope_inv(double base, int hd) {
+    RopeInv r{};
+    for (int i = 0; i < hd / 2 && i < 64; ++i) r.v[i] = exp2(-(2.0 * i / hd) * log2(base));
+    return r;
+}
+__device__ __forceinline__ void rope_cs(double pos, double inv, float& cs, float& sn) {
+    const double x = pos * inv;
+    const double k = rint(x * 0.15915494309189535);
+    double r = fma(-k, 6.283185307179586, x);
+    r = fma(-k, 2.4492935982947064e-16, r);
+    sincosf((float)r, &sn, &cs);
+}
+
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 

@@ -68,7 +68,7 @@ cudaError_t launch_seq_set(const SeqState& s, int seq, int kv_len, int root, int
 // prepare: rows of the verify forward (root + draft nodes), validation, embedding gather, rotary table
 // ---------------------------------------------------------------------------------------------------------------
 
-__global__ void prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, int vocab, int hd, double rope_base,
+__global__ void prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, int vocab, int hd, RopeInv rinv,
                                long long kv_capacity, SeqState s, RowMeta rm, float* __restrict__ hidden,
                                float* __restrict__ rope, PrepareArgs a, uint32_t* status) {
     const int t = blockIdx.x, bi = t / a.R, r = t % a.R;
@@ -135,34 +135,27 @@ __global__ void prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, i
     __syncthreads();
     const int tok = sh_tok;
     const bool ok = sh_ok;
-    float ss = 0.f;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        const float v = ok ? __bfloat162float(embed[(size_t)tok * d + i]) : 0.f;
-        hidden[(size_t)t * d + i] = v;
-        if (a.x) {
-            store_terms(v * __bfloat162float(a.gain0[i]), a.x + (size_t)t * a.terms * d + i, d, a.terms);
-            ss += v * v;
-        }
-    }
+    float ss = embed_row(embed + (size_t)tok * d, ok, d, hidden + (size_t)t * d, a.gain0,
+                         a.x ? a.x + (size_t)t * a.terms * d : nullptr, a.terms);
     if (a.x) {
         __shared__ float red[32];
         ss = block_sum(ss, red);
         if (threadIdx.x == 0) a.sumsq_out[t] = ss;
     }
-    // rotary table in double: angle = pos * base^(-2i/hd)
+    // rotary table: angle = pos * base^(-2i/hd)
     for (int i = threadIdx.x; i < hd / 2; i += blockDim.x) {
-        const double inv = exp2(-(2.0 * i / hd) * log2(rope_base));
-        double sn, cs;
-        sincos((double)sh_pos * inv, &sn, &cs);
-        rope[((size_t)t * (hd / 2) + i) * 2 + 0] = (float)cs;
-        rope[((size_t)t * (hd / 2) + i) * 2 + 1] = (float)sn;
+        float cs, sn;
+        rope_cs((double)sh_pos, rinv.v[i], cs, sn);
+        rope[((size_t)t * (hd / 2) + i) * 2 + 0] = cs;
+        rope[((size_t)t * (hd / 2) + i) * 2 + 1] = sn;
     }
 }
 
 cudaError_t launch_prepare(const ModelView& m, const SeqState& s, const RowMeta& rm, const Scratch& sc,
                            const PrepareArgs& a, uint32_t* status, cudaStream_t st) {
     prepare_kernel<<<a.B * a.R, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(m.d.embed), m.d.d_model, m.d.vocab,
-                                              m.d.head_dim, (double)m.d.rope_base, (long long)m.d.kv_capacity, s, rm,
+                                              m.d.head_dim, rope_inv((double)m.d.rope_base, m.d.head_dim),
+                                              (long long)m.d.kv_capacity, s, rm,
                                               sc.hidden, sc.rope, a, status);
     return cudaGetLastError();
 }

@@ -33,7 +33,7 @@ __device__ __forceinline__ bool before(const Cand& a, const Cand& b) {     // a 
 // ---------------------------------------------------------------------------------------------------------------
 
 __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, int vocab, int hd,
-                                     double rope_base, SeqState s, DraftState ds, RowMeta rm,
+                                     RopeInv rinv, SeqState s, DraftState ds, RowMeta rm,
                                      float* __restrict__ hidden, float* __restrict__ rope, SeqList seqs, int R, int step,
                                      int beam, const __nv_bfloat16* __restrict__ gain0, __nv_bfloat16* x, int terms,
                                      float* sumsq_out) {
@@ -94,15 +94,8 @@ __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, in
     __syncthreads();
     const int tok = sh_tok;
     const bool ok = sh_ok;
-    float ss = 0.f;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        const float v = ok ? __bfloat162float(embed[(size_t)tok * d + i]) : 0.f;
-        hidden[(size_t)t * d + i] = v;
-        if (x) {
-            store_terms(v * __bfloat162float(gain0[i]), x + (size_t)t * terms * d + i, d, terms);
-            ss += v * v;
-        }
-    }
+    float ss = embed_row(embed + (size_t)tok * d, ok, d, hidden + (size_t)t * d, gain0,
+                         x ? x + (size_t)t * terms * d : nullptr, terms);
     if (x) {
         __shared__ float red[32];
         ss = wsum(ss);
@@ -115,11 +108,10 @@ __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, in
         }
     }
     for (int i = threadIdx.x; i < hd / 2; i += blockDim.x) {
-        const double inv = exp2(-(2.0 * i / hd) * log2(rope_base));
-        double sn, cs;
-        sincos((double)sh_pos * inv, &sn, &cs);
-        rope[((size_t)t * (hd / 2) + i) * 2 + 0] = (float)cs;
-        rope[((size_t)t * (hd / 2) + i) * 2 + 1] = (float)sn;
+        float cs, sn;
+        rope_cs((double)sh_pos, rinv.v[i], cs, sn);
+        rope[((size_t)t * (hd / 2) + i) * 2 + 0] = cs;
+        rope[((size_t)t * (hd / 2) + i) * 2 + 1] = sn;
     }
 }
 
@@ -128,7 +120,7 @@ cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const Dr
                                  bool pdl, cudaStream_t st) {
     return launch_pdl(draft_prepare_kernel, dim3(B * R), dim3(128), 0, st, pdl,
                       static_cast<const __nv_bfloat16*>(m.d.embed), m.d.d_model, m.d.vocab, m.d.head_dim,
-                      (double)m.d.rope_base, s, ds, rm, sc.hidden, sc.rope, seqs, R, step, beam,
+                      rope_inv((double)m.d.rope_base, m.d.head_dim), s, ds, rm, sc.hidden, sc.rope, seqs, R, step, beam,
                       tc ? m.w(0, 0) : (const __nv_bfloat16*)nullptr, tc ? sc.xd : (__nv_bfloat16*)nullptr,
                       tc_terms(B * R), sc.sumsq_a);
 }
