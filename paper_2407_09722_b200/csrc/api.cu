@@ -57,6 +57,37 @@ struct mtad_ctx {
 
 unsigned long long g_kernel_launches = 0;    // kernels of this library enqueued since load
 
+#ifdef MTAD_TRACE
+// Trace builds only: global-timer stamps of every CTA of the GEMM launches made while tracing is on
+constexpr int kTraceLaunches = 320, kTraceCtas = 320;
+static __device__ unsigned long long g_trace[kTraceLaunches][kTraceCtas][8];
+static unsigned long long* g_trace_dev = nullptr;
+static int g_trace_n = -1;                   // launches recorded so far, -1: off
+static int g_trace_meta[kTraceLaunches][4];  // cluster?, mode, grid, csize
+static unsigned long long* trace_slot(bool cluster, int mode, int grid, int csize) {
+    if (g_trace_n < 0 || g_trace_n >= kTraceLaunches || grid > kTraceCtas) return nullptr;
+    g_trace_meta[g_trace_n][0] = cluster; g_trace_meta[g_trace_n][1] = mode;
+    g_trace_meta[g_trace_n][2] = grid; g_trace_meta[g_trace_n][3] = csize;
+    return g_trace_dev + (size_t)(g_trace_n++) * kTraceCtas * 8;
+}
+extern "C" int mtad_trace_begin(void) {
+    if (!g_trace_dev && cudaGetSymbolAddress((void**)&g_trace_dev, g_trace) != cudaSuccess) return -1;
+    cudaMemset(g_trace_dev, 0, sizeof(unsigned long long) * kTraceLaunches * kTraceCtas * 8);
+    g_trace_n = 0;
+    return 0;
+}
+extern "C" int mtad_trace_end(unsigned long long* host, int* meta, int max_launches) {
+    cudaDeviceSynchronize();
+    const int n = g_trace_n < max_launches ? g_trace_n : max_launches;
+    g_trace_n = -1;
+    if (n > 0) {
+        cudaMemcpy(host, g_trace_dev, sizeof(unsigned long long) * (size_t)n * kTraceCtas * 8, cudaMemcpyDeviceToHost);
+        memcpy(meta, g_trace_meta, sizeof(int) * 4 * n);
+    }
+    return n;
+}
+#endif
+
 namespace {
 
 struct Carver {
@@ -372,7 +403,17 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
     const double wb = 2.0;
     // Every GEMM of the step is described first; then the projections that feed one another without attention in
     // between (O, gate/up, down, and the next layer's QKV or the LM head) are chained as phases of one launch.
-    struct GemmDesc { TcMaps mp; TcGemmParams p; double bytes; };
+    struct GemmDesc { TcMaps mp; TcGemmParams p; double bytes; bool cluster; };
+    // Calls of up to 32 rows run the projections whose tiles fill the CTA slots as clusters that reduce over
+    // distributed shared memory (tc_gemm_cluster.cu); bit k of the mask: QKV, O, gate/up, down, LM head
+    static const int cluster_mask = getenv("MTAD_TC_CLUSTER") ? atoi(getenv("MTAD_TC_CLUSTER")) : 27;
+    auto clusterize = [&](TcGemmParams& p, int n_tiles, int K, int bit) -> bool {
+        if (!((cluster_mask >> bit) & 1)) return false;
+        TcGemmParams q = p;
+        if (!tc_cluster_plan(q, n_tiles, K, T, 2 * kCtas)) return false;
+        p = q;
+        return true;
+    };
     std::vector<GemmDesc> g;           // per layer: QKV, O, gate/up, down; then the LM head
     g.reserve((size_t)d.layers * 4 + 1);
     for (int l = 0; l < d.layers; ++l) {
@@ -384,7 +425,8 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             p.mode = TC_QKV; p.N = qd; p.seg_k_tile = qt; p.seg_v_tile = qt + kt; p.layer = l;
             p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = (l == 0) ? 1 : dt;
             mp.a0 = wm.wq[ix(mq)][l]; mp.a1 = wm.wk[ix(mq)][l]; mp.a2 = wm.wv[ix(mq)][l]; mp.x = xd;
-            g.push_back({mp, p, wb * (qd + 2.0 * kvd) * d.d_model});
+            const bool cl = mq == 1 && clusterize(p, qt + 2 * kt, d.d_model, 0);
+            g.push_back({mp, p, wb * (qd + 2.0 * kvd) * d.d_model, cl});
         }
         {   // O projection + residual, emits the FFN norm's operand rows
             TcGemmParams p = base; TcMaps mp{};
@@ -394,7 +436,8 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             p.gain = m.w(l, 5); p.x_out = sc.xd; p.xk = d.d_model;
             p.sumsq_out = sc.sumsq_b;
             mp.a0 = wm.wo[ix(mh)][l]; mp.x = xa;
-            g.push_back({mp, p, wb * d.d_model * qd});
+            const bool cl = mh == 1 && clusterize(p, up(d.d_model, 128), qd, 1);
+            g.push_back({mp, p, wb * d.d_model * qd, cl});
         }
         {   // gate / up + SwiGLU
             TcGemmParams p = base; TcMaps mp{};
@@ -403,7 +446,8 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             p.mode = TC_SWIGLU; p.N = d.d_ffn; p.sumsq_in = sc.sumsq_b; p.sumsq_in_parts = dt;
             p.x_out = sc.xf; p.xk = d.d_ffn;
             mp.a0 = wm.gate[ix(mh)][l]; mp.a1 = wm.up[ix(mh)][l]; mp.x = xd;
-            g.push_back({mp, p, wb * 2.0 * d.d_ffn * d.d_model});
+            const bool cl = mh == 1 && clusterize(p, up(d.d_ffn, 64), d.d_model, 2);
+            g.push_back({mp, p, wb * 2.0 * d.d_ffn * d.d_model, cl});
         }
         {   // down projection + residual, emits the next norm's operand rows
             TcGemmParams p = base; TcMaps mp{};
@@ -413,7 +457,8 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             p.gain = (l + 1 < d.layers) ? m.w(l + 1, 0) : static_cast<const __nv_bfloat16*>(d.final_norm);
             p.x_out = sc.xd; p.xk = d.d_model; p.sumsq_out = sc.sumsq_a;
             mp.a0 = wm.down[ix(mh)][l]; mp.x = xf;
-            g.push_back({mp, p, wb * d.d_model * d.d_ffn});
+            const bool cl = mh == 1 && clusterize(p, up(d.d_model, 128), d.d_ffn, 3);
+            g.push_back({mp, p, wb * d.d_model * d.d_ffn, cl});
         }
     }
     int lm_tiles128 = 0;
@@ -426,17 +471,27 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
         p.out = sc.logits; p.ldo = d.vocab;
         mp.a0 = wm.lm_head[ix(mh)]; mp.x = xd;
         lm_tiles128 = p.n_tiles128;
-        g.push_back({mp, p, wb * d.vocab * d.d_model});
+        const bool cl = mh == 1 && clusterize(p, up(d.vocab, 128), d.d_model, 4);
+        g.push_back({mp, p, wb * d.vocab * d.d_model, cl});
     }
     // chained launches are available but off by default: with stream-K every tile of a phase finishes at the end of
     // the phase, so a chained phase starts no earlier than a separately launched kernel with its weights prefetched
     static const bool use_chain = getenv("MTAD_TC_CHAIN") && atoi(getenv("MTAD_TC_CHAIN")) != 0;
     const size_t flag_stride = ctx->tc_counter_n + 1;      // per (launch, phase): tile flags, then the finished-tile count
-    const bool chain = use_chain && mq == mh && (size_t)(d.layers + 1) * TC_MAX_PHASES * flag_stride <= ctx->tc_flag_n;
+    bool any_cluster = false;
+    for (const GemmDesc& gd : g) any_cluster = any_cluster || gd.cluster;
+    const bool chain = use_chain && !any_cluster && mq == mh && (size_t)(d.layers + 1) * TC_MAX_PHASES * flag_stride <= ctx->tc_flag_n;
     if (chain) CU(cudaMemsetAsync(sc.tc_flags, 0, sizeof(int32_t) * (size_t)(d.layers + 1) * TC_MAX_PHASES * flag_stride, s));
     int launch_no = 0;
     // launches descriptors [i0, i0 + n) as one kernel
     auto launch = [&](size_t i0, int n) -> int {
+        if (n == 1 && g[i0].cluster) {
+#ifdef MTAD_TRACE
+            g[i0].p.trace = trace_slot(true, g[i0].p.mode, g[i0].p.n_tiles * g[i0].p.csize, g[i0].p.csize);
+#endif
+            RUN(MTAD_K_GEMM, g[i0].bytes, 1, launch_tc_cluster(g[i0].mp, g[i0].p, pdl, s));
+            return MTAD_OK;
+        }
         TcChain ch{};
         ch.n_phases = n;
         double bytes = 0;
@@ -457,6 +512,9 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             }
         }
         ++launch_no;
+#ifdef MTAD_TRACE
+        ch.p[0].trace = trace_slot(false, ch.p[0].mode, (ch.p[0].total_units + ch.p[0].units_per_cta - 1) / ch.p[0].units_per_cta, 0);
+#endif
         RUN(MTAD_K_GEMM, bytes, 1, launch_tc_chain(ch, pdl, s));
         return MTAD_OK;
     };
@@ -679,6 +737,12 @@ int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, 
     p.mode = TC_PLAIN; p.N = N; p.out = y; p.ldo = N;
     p.ws = ctx->sc.tc_ws; p.counters = ctx->sc.tc_counters; p.status = nullptr;
     RUN(MTAD_K_PREPARE, 0, 1, launch_split_rows(x, K, ctx->sc.xf, p.terms, T, K, s));
+    static const int cluster_mask = getenv("MTAD_TC_CLUSTER") ? atoi(getenv("MTAD_TC_CLUSTER")) : 27;
+    TcGemmParams q = p;
+    if (mh == 1 && ((cluster_mask >> 5) & 1) && tc_cluster_plan(q, p.n_tiles, K, T, 2 * kCtas)) {
+        RUN(MTAD_K_GEMM, 2.0 * N * K, 1, launch_tc_cluster(mp, q, false, s));
+        return MTAD_OK;
+    }
     RUN(MTAD_K_GEMM, 2.0 * N * K, 1, launch_tc_gemm(mp, p, kCtas, false, s));
     return MTAD_OK;
 }

@@ -126,6 +126,30 @@ struct Scratch {
     WarpRow* warp_row;       // [T]
 };
 
+// ---- index arithmetic used by the kernels and, on the host, by the extent audit (mtad_audit_extents) -----------
+// first element of position `pos` of (layer, sequence, K|V, KV head) in a cache [layer][max_batch][2][Hkv][cap][hd]
+__host__ __device__ inline size_t idx_cache(long long layer, long long max_batch, long long seq, int kv, long long Hkv,
+                                            long long head, long long cap, long long pos, long long hd) {
+    return (size_t)((((((layer * max_batch + seq) * 2 + kv) * Hkv + head) * cap) + pos) * hd);
+}
+// split-KV partial (m, l, o[hd]) of row t, head h, split sp
+__host__ __device__ inline size_t idx_attn_part(long long t, long long Hq, long long h, long long nsplit, long long sp,
+                                                long long hd) {
+    return (size_t)((((t * Hq + h) * nsplit) + sp) * (hd + 2));
+}
+// term j of element k of activation row t in an operand-row buffer of row length K
+__host__ __device__ inline size_t idx_xrow(long long t, long long terms, long long j, long long K, long long k) {
+    return (size_t)((t * terms + j) * K + k);
+}
+// LM-head partial of (row t, 128-token tile)
+__host__ __device__ inline size_t idx_lm_part(long long t, long long n_tiles, long long tile) {
+    return (size_t)(t * n_tiles + tile);
+}
+// split-K partial tile of (tile, contributor): part_floats floats each
+__host__ __device__ inline size_t idx_tc_ws(long long tile, long long max_contrib, long long contrib, long long part_floats) {
+    return (size_t)((tile * max_contrib + contrib) * part_floats);
+}
+
 inline int attn_split_cap(int n_q_heads) {
     int s = (4 * 148 + n_q_heads - 1) / n_q_heads;
     return s < 1 ? 1 : (s > 32 ? 32 : s);

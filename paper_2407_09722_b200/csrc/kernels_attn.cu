@@ -32,8 +32,8 @@ __global__ void __launch_bounds__(128) attn_partial_kernel(const float* __restri
     const int c0 = sp * chunk;
     const int c1 = min(c0 + chunk, nkeys);
     const int g = h / (Hq / Hkv);
-    const __nv_bfloat16* Kg = cache + (((((size_t)layer * max_batch + seq) * 2 + 0) * Hkv + g) * cap) * HD;
-    const __nv_bfloat16* Vg = cache + (((((size_t)layer * max_batch + seq) * 2 + 1) * Hkv + g) * cap) * HD;
+    const __nv_bfloat16* Kg = cache + idx_cache(layer, max_batch, seq, 0, Hkv, g, cap, 0, HD);
+    const __nv_bfloat16* Vg = cache + idx_cache(layer, max_batch, seq, 1, Hkv, g, cap, 0, HD);
 
     for (int rc = 0; rc < nrows; rc += MTAD_ROW_CHUNK) {
         __syncthreads();
@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(128) attn_partial_kernel(const float* __restri
         for (int a = 0; a < 2; ++a) {
             const int r = rc + warp * 2 + a;
             if (r >= nrows) continue;
-            float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
+            float* dst = part + idx_attn_part(bi * R + r, Hq, h, nsplit, sp, HD);
             if (lane == 0) { dst[0] = m[a]; dst[1] = l[a]; }
 #pragma unroll
             for (int d = 0; d < DPL; ++d) dst[2 + lane * DPL + d] = o[a][d];
@@ -153,7 +153,7 @@ __global__ void attn_combine_kernel(const float* __restrict__ part, float* __res
         return;
     }
     extern __shared__ float wsm[];                  // [nsplit] weights, then [1] the normaliser
-    const float* p = part + (((size_t)t * Hq + h) * nsplit) * (HD + 2);
+    const float* p = part + idx_attn_part(t, Hq, h, nsplit, 0, HD);
     __shared__ float s_max;
     if (threadIdx.x < 32) {
         float M = -CUDART_INF_F;

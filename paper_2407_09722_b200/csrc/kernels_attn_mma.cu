@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(CNT == 4 ? 192 : 128, CNT == 1 ? 4 : (CNT == 4
         if (early) { pdl_wait(); pdl_trigger(); }
         for (int i = threadIdx.x; i < n_q; i += blockDim.x) {
             const int h = g * G + i / nrows, r = i % nrows;
-            float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
+            float* dst = part + idx_attn_part(bi * R + r, Hq, h, nsplit, sp, HD);
             dst[0] = -CUDART_INF_F;
             dst[1] = 0.f;
         }
@@ -256,7 +256,7 @@ __global__ void __launch_bounds__(CNT == 4 ? 192 : 128, CNT == 1 ? 4 : (CNT == 4
         }
         for (int i = threadIdx.x; i < n_q; i += blockDim.x) {
             const int h = g * G + i / nrows, r = i % nrows;
-            float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
+            float* dst = part + idx_attn_part(bi * R + r, Hq, h, nsplit, sp, HD);
             dst[0] = -CUDART_INF_F;
             dst[1] = 0.f;
         }
@@ -423,7 +423,7 @@ __global__ void __launch_bounds__(CNT == 4 ? 192 : 128, CNT == 1 ? 4 : (CNT == 4
         // ---- partials of the valid rows ----
         if (qi0 < n_q) {
             const int h = g * G + qi0 / nrows, r = qi0 % nrows;
-            float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
+            float* dst = part + idx_attn_part(bi * R + r, Hq, h, nsplit, sp, HD);
             if (tq == 0) { dst[0] = m0 * LN2; dst[1] = l0; }
 #pragma unroll
             for (int n = 0; n < NDT; ++n)
@@ -431,7 +431,7 @@ __global__ void __launch_bounds__(CNT == 4 ? 192 : 128, CNT == 1 ? 4 : (CNT == 4
         }
         if (qi1 < n_q) {
             const int h = g * G + qi1 / nrows, r = qi1 % nrows;
-            float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
+            float* dst = part + idx_attn_part(bi * R + r, Hq, h, nsplit, sp, HD);
             if (tq == 0) { dst[0] = m1 * LN2; dst[1] = l1; }
 #pragma unroll
             for (int n = 0; n < NDT; ++n)
@@ -484,7 +484,7 @@ __global__ void __launch_bounds__(CNT == 4 ? 192 : 128, CNT == 1 ? 4 : (CNT == 4
             for (int q = 0; q < kparts; ++q)
                 acc += (reinterpret_cast<const float*>(smem) + (w0 + q) * 16 * PARK)[row * PARK + d] * wq[qi * 4 + q];
             const int h = g * G + qi / nrows, r = qi % nrows;
-            float* dst = part + (((size_t)(bi * R + r) * Hq + h) * nsplit + sp) * (HD + 2);
+            float* dst = part + idx_attn_part(bi * R + r, Hq, h, nsplit, sp, HD);
             dst[2 + d] = acc;
             if (d == 0) { dst[0] = wM[qi] * LN2; dst[1] = wl[qi]; }
         }

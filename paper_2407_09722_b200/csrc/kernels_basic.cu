@@ -449,7 +449,7 @@ __global__ void lm_merge_kernel(const float4* __restrict__ part, int n_tiles, in
     float m = -CUDART_INF_F, s = 0.f;
     Best best{-CUDART_INF_F, 0x7fffffff};
     for (int j = threadIdx.x; j < n_tiles; j += blockDim.x) {
-        const float4 q = part[(size_t)t * n_tiles + j];
+        const float4 q = part[idx_lm_part(t, n_tiles, j)];
         const float mm = fmaxf(m, q.x);
         s = (m == -CUDART_INF_F ? 0.f : s * expf(m - mm)) + (q.x == -CUDART_INF_F ? 0.f : q.y * expf(q.x - mm));
         m = mm;
@@ -608,7 +608,7 @@ __global__ void kv_commit_kernel(__nv_bfloat16* __restrict__ cache, const int32_
     const int head = blockIdx.x % Hkv;
     const int kv = (blockIdx.x / Hkv) & 1;
     const int layer = blockIdx.x / (2 * Hkv);
-    __nv_bfloat16* base = cache + (((((size_t)layer * max_batch + seq) * 2 + kv) * Hkv + head) * cap) * hd;
+    __nv_bfloat16* base = cache + idx_cache(layer, max_batch, seq, kv, Hkv, head, cap, 0, hd);
     extern __shared__ __nv_bfloat16 buf[];
     for (int i = threadIdx.x; i < eta * hd; i += blockDim.x) {
         const int r = i / hd, j = i % hd;

@@ -343,7 +343,7 @@ __global__ void aux_commit_kernel(__nv_bfloat16* __restrict__ cache, const int32
     const int head = blockIdx.x % Hkv;
     const int kv = (blockIdx.x / Hkv) & 1;
     const int layer = blockIdx.x / (2 * Hkv);
-    __nv_bfloat16* b = cache + (((((size_t)layer * max_batch + seq) * 2 + kv) * Hkv + head) * cap) * hd;
+    __nv_bfloat16* b = cache + idx_cache(layer, max_batch, seq, kv, Hkv, head, cap, 0, hd);
     extern __shared__ __nv_bfloat16 buf[];
     for (int i = threadIdx.x; i < kept * hd; i += blockDim.x) {
         const int r = i / hd, j = i % hd;

@@ -33,6 +33,9 @@ struct TcGemmParams {
     int n_rows_total;      // weight rows, for skipping a half that lies beyond them
     int n_tiles128;        // ceil(N / 128): row stride of lm_part
     int stages;            // smem ring depth
+    unsigned long long* trace;   // MTAD_TRACE builds: [CTA][8] global-timer stamps of this launch, else null
+    int csize;             // cluster kernel: CTAs that share a tile's k-range (1..8)
+    int rpr;               // cluster kernel: rows per epilogue pass (1..8); pass q is finished by rank q % csize
     int mode;
     int N;                 // output features (bound for stores)
     // Chained phases of one launch: a phase whose operand rows are written by the phase before it reads, per k-block,
@@ -109,6 +112,13 @@ int tc_ctas_per_sm(int T);
 // Weight halves per tile that fit tensor memory for T rows, given tc_terms(T) accumulator columns per row.
 int tc_halves(int T);
 size_t tc_workspace_floats(int n_tiles_max, int max_contrib_max, int rpad_max);
+
+// Cluster variant (tc_gemm_cluster.cu) for calls of up to 32 rows: a cluster of p.csize CTAs per 128-feature tile,
+// partial rows exchanged through distributed shared memory.  tc_cluster_plan fills the decomposition for n_tiles
+// tiles on `slots` co-resident CTAs and returns false when the shape does not suit it (too many rows, more tiles
+// than slots).
+bool tc_cluster_plan(TcGemmParams& p, int n_tiles, int K, int T, int slots);
+cudaError_t launch_tc_cluster(const TcMaps& maps, const TcGemmParams& p, bool pdl, cudaStream_t st);
 
 cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p, int ctas, bool pdl, cudaStream_t st);
 

@@ -24,9 +24,10 @@ def _check(dm, N, K, T, seed):
     ref = x.double() @ W.double().t()
     err = (y.double() - ref).abs().max().item()
     scale = ref.abs().max().item()
-    # up to 32 rows the activations enter as three bf16 terms (exact): only fp32 accumulation error is left; beyond,
-    # two terms (~2^-17 relative per element)
-    tol = 4e-6 if T <= 32 else 2e-5
+    # up to 32 rows the activations enter as three bf16 terms (exact): only the tensor cores' fp32 accumulation error
+    # is left, which grows with the number of k-blocks summed in one accumulator (all of K when a tile is not split);
+    # beyond 32 rows, two terms (~2^-17 relative per element)
+    tol = (4e-6 if K <= 2048 else 8e-6) if T <= 32 else 2e-5
     assert err <= tol * max(scale, 1.0), (N, K, T, err, scale)
 
 
