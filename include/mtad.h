@@ -122,6 +122,14 @@ int mtad_seq_set(mtad_ctx* ctx, int seq, int32_t kv_len, int32_t root_token, int
 /* Read back the committed length and root token of a sequence.  Synchronises the stream. */
 int mtad_seq_get(mtad_ctx* ctx, int seq, int32_t* kv_len, int32_t* root_token, void* stream);
 
+/* The context keeps, on the host, an upper bound of every sequence's committed length (it sizes the attention
+ * launch and the capacity checks of mtad_draft without reading device memory).  kv_commit can only add the largest
+ * possible advance (max_depth + 1) to it, so over a long decode loop the bound drifts above the true length.  A
+ * caller that reads eta back anyway hands the true length in here (host-side, no launch, no synchronisation);
+ * mtad_seq_get also refreshes the bound.  Without either, mtad_draft may report MTAD_E_CAPACITY early and the
+ * attention launches carry blocks for keys that do not exist (harmless, slower). */
+int mtad_seq_hint(mtad_ctx* ctx, int seq, int32_t kv_len);
+
 /* Warp the target's distributions before the verification rule and the extra token, as in the paper's experiments
  * (App. F; the footnote to Sec. 3.2 states that the method is equally valid on warped distributions): every row of
  * P keeps its top_k most likely tokens, renormalised; of these, in descending order of probability (lower token id
@@ -209,8 +217,9 @@ int kv_commit(mtad_ctx* ctx, int B, const int32_t* seqs, const mtad_result* res,
  * mtad_verify_chain; there is no commit step, the caller keeps the rows it accepts.
  * Limits and sharing: returns MTAD_E_WORKSPACE when the model shape or gamma needs more scratch than the array
  * holds (mtad_workspace_bytes(target, NULL, 1, gamma) tells how much).  All calls on a device share the one array,
- * which still contains the previous call's data: the library re-zeroes the parts that must start at zero whenever
- * the model or gamma changes, but two calls whose GPU work overlaps (different streams, different threads) race
+ * which still contains the previous call's data: the library re-zeroes the whole array whenever the model or gamma
+ * changes (after synchronising the device, so that earlier calls still running on any stream are over) and the
+ * split-K counters at the start of every call, but two calls whose GPU work overlaps (different streams, different threads) race
  * on it - issue them on one stream or synchronise in between.  The first call on a device (and any call that
  * changes the model or gamma) looks up the array's device address, zeroes it and synchronises the device; make
  * that call before starting a stream capture. */
@@ -240,6 +249,12 @@ uint64_t mtad_kernel_launches(void);
  * (bf16, device, 16-byte aligned), T <= 256, K a multiple of 8 and at most the context's largest FFN width.
  * For unit tests and kernel timing; uses the context's workspace. */
 int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, int T, float* y, void* stream);
+
+/* Test hook for the time-out path: wait_limit = iterations a bounded wait inside the GEMM kernels may poll (0: the
+ * default); no_operands != 0 makes the GEMM kernels leave out their operand-row copies, so the waits on them run out
+ * and every sequence of the call reports MTAD_ST_TIMEOUT.  The kernels return normally; a later call with the hook
+ * switched off is unaffected. */
+int mtad_debug_set_wait(mtad_ctx* ctx, unsigned int wait_limit, int no_operands);
 
 const char* mtad_status_str(int status);
 int mtad_last_cuda_error(const mtad_ctx* ctx);

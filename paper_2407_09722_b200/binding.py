@@ -41,7 +41,7 @@ EXPORTS = ("mtad_workspace_bytes", "mtad_create", "mtad_destroy", "mtad_seq_set"
            "mtad_verify_chain", "mtad_verify_tree", "kv_commit", "mtad_status_str", "mtad_last_cuda_error",
            "mtad_profile_begin", "mtad_profile_end", "mtad_kernel_launches", "mtad_verify_chain_static",
            "mtad_debug_gemm", "mtad_set_warp", "mtad_profile_grouped",
-           "mtad_verify_chain_spd")
+           "mtad_verify_chain_spd", "mtad_seq_hint", "mtad_debug_set_wait")
 MTAD_STATIC_SCRATCH_BYTES = 16 << 20
 MTAD_ST_TIMEOUT, MTAD_ST_AUX_PENDING, MTAD_ST_NONFINITE = 32, 64, 128      # device status bits (mtad.h)
 KERNEL_CLASSES = ("prepare", "norm", "gemm", "rope_append", "attention", "lm_reduce", "accept", "commit")
@@ -67,6 +67,8 @@ def load_library() -> C.CDLL:
     lib.mtad_seq_set.argtypes = [P, I, C.c_int32, C.c_int32, C.c_int32, I32P, P]
     lib.mtad_seq_get.argtypes = [P, I, I32P, I32P, P]
     lib.mtad_set_warp.argtypes = [P, I, C.c_float]
+    lib.mtad_seq_hint.argtypes = [P, I, C.c_int32]
+    lib.mtad_debug_set_wait.argtypes = [P, C.c_uint, I]
     lib.mtad_profile_grouped.argtypes = [P, I]
     lib.mtad_draft.argtypes = [P, I, I32P, I, I, P, P, P, P, P, P, P, P]
     lib.mtad_verify_chain.argtypes = [P, I, I32P, I, P, P, F, P, RS, P]
@@ -225,6 +227,13 @@ class Context:
         if check:
             self._check(rc, "mtad_set_warp")
         return rc
+
+    def mtad_seq_hint(self, seq: int, kv_len: int):
+        self._check(self._lib.mtad_seq_hint(self.handle, seq, kv_len), "mtad_seq_hint")
+
+    def mtad_debug_set_wait(self, wait_limit: int, no_operands: bool):
+        self._check(self._lib.mtad_debug_set_wait(self.handle, wait_limit, 1 if no_operands else 0),
+                    "mtad_debug_set_wait")
 
     def mtad_seq_get(self, seq: int, stream=None):
         a, b = C.c_int32(), C.c_int32()

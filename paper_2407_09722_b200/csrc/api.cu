@@ -41,6 +41,8 @@ struct mtad_ctx {
     int last_B = 0, last_R = 0, last_D = 0;
     int32_t last_seqs[MTAD_MAX_BATCH];
     int last_cuda = 0;
+    unsigned int wait_limit = 0;        // debug: iteration limit of the GEMM kernels' bounded waits (0: default)
+    int debug_no_operands = 0;          // debug: the GEMM kernels' operand-row copies are left out (waits run out)
     int warp_k = 0;                     // 0: unwarped target rows
     float warp_p = 1.f;
     // optional per-kernel-class timing (cudaEvent pairs around each launch)
@@ -400,6 +402,7 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
     base.slot = ctx->rm.slot; base.seq = ctx->rm.seq; base.max_batch = m.max_batch; base.cap = d.kv_capacity;
     base.hidden = sc.hidden; base.R = R; base.prow = ctx->rm.prow; base.tok = ctx->rm.tok; base.node_z = sc.node_z;
     base.lm_part = sc.lm_part; base.uniforms = uniforms;
+    base.wait_limit = ctx->wait_limit; base.debug_no_operands = ctx->debug_no_operands;
     const double wb = 2.0;
     // Every GEMM of the step is described first; then the projections that feed one another without attention in
     // between (O, gate/up, down, and the next layer's QKV or the LM head) are chained as phases of one launch.
@@ -573,6 +576,8 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
     for (int i = 0; i < B; ++i) ub = std::max(ub, ctx->len_ub[seqs[i]]);
 
     CU(cudaMemsetAsync(out->status, 0, sizeof(uint32_t) * B, s));
+    // a launch that gave up on a wait leaves split-K arrival counters behind: every call starts from zero
+    CU(cudaMemsetAsync(ctx->sc.tc_counters, 0, sizeof(int32_t) * ctx->tc_counter_n * TC_MAX_PHASES, s));
     PrepareArgs pa{};
     for (int i = 0; i < B; ++i) pa.seqs.v[i] = seqs[i];
     pa.B = B; pa.R = R; pa.max_depth = D; pa.n_nodes = n_nodes; pa.tok = tok; pa.parent = parent;
@@ -771,6 +776,20 @@ int mtad_set_warp(mtad_ctx* ctx, int top_k, float top_p) {
     return MTAD_OK;
 }
 
+int mtad_seq_hint(mtad_ctx* ctx, int seq, int32_t kv_len) {
+    if (!ctx || seq < 0 || seq >= ctx->max_batch || kv_len < 0) return MTAD_E_INVALID;
+    if (kv_len > ctx->target.d.kv_capacity) return MTAD_E_CAPACITY;
+    ctx->len_ub[seq] = kv_len;
+    return MTAD_OK;
+}
+
+int mtad_debug_set_wait(mtad_ctx* ctx, unsigned int wait_limit, int no_operands) {
+    if (!ctx) return MTAD_E_INVALID;
+    ctx->wait_limit = wait_limit;
+    ctx->debug_no_operands = no_operands ? 1 : 0;
+    return MTAD_OK;
+}
+
 int mtad_seq_get(mtad_ctx* ctx, int seq, int32_t* kv_len, int32_t* root_token, void* stream) {
     if (!ctx || seq < 0 || seq >= ctx->max_batch) return MTAD_E_INVALID;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -813,6 +832,7 @@ int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_wi
     for (int i = 0; i < B; ++i) sl.v[i] = seqs[i];
     DraftOut out{tok, parent, depth, node_logq, logq_ref, best_path};
     const bool tc = ctx->use_tc && ctx->amaps.ok;
+    CU(cudaMemsetAsync(ctx->sc.tc_counters, 0, sizeof(int32_t) * ctx->tc_counter_n * TC_MAX_PHASES, s));
     for (int step = 0; step < gamma; ++step) {
         const int R = step == 0 ? R0 : beam_width;
         RUN(MTAD_K_PREPARE, 0, 1, launch_draft_prepare(m, ctx->st, ctx->ds, ctx->rm, ctx->sc, sl, B, R, step, beam_width,

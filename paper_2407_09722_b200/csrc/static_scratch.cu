@@ -59,6 +59,9 @@ extern "C" int mtad_verify_chain_static(const mtad_model_desc* target, int32_t k
         p.scratch = ptr;
     }
     if (!same_model(p, target, gamma)) {
+        // The array is about to be laid out afresh and zeroed: work of earlier calls that still runs on the caller's
+        // stream (a non-blocking stream does not wait for the zeroing on the default stream) must be over first.
+        if (cudaDeviceSynchronize() != cudaSuccess) return MTAD_E_CUDA;
         if (p.ctx) { mtad_destroy(p.ctx); p.ctx = nullptr; }
         // mtad_create lays the step's scratch out inside the array and zeroes it (the array still holds the
         // previous caller's data); it allocates no device memory itself.

@@ -51,9 +51,11 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false when the limit ran out here or another role already gave up.
+// Bounded wait.  Returns false when the limit ran out here or another role already gave up.  abort_flag[0] is the
+// CTA's give-up flag, abort_flag[1] the iteration limit of every wait of this launch.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    const uint32_t limit = (uint32_t)abort_flag[1];
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_test(bar, parity)) return true;
         if (it > 64) __nanosleep(32);
         if ((it & 255u) == 255u && *abort_flag) return false;
@@ -64,7 +66,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 
 // Bounded wait until the arrival count of a tile (low 16 bits of its counter) reaches `want` (acquire at gpu scope).
 __device__ __forceinline__ bool arrivals_wait(const int* counter, int want, volatile int* abort_flag) {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    const uint32_t limit = (uint32_t)abort_flag[1];
+    for (uint32_t it = 0; it < limit; ++it) {
         int v;
         asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
         if ((v & 0xFFFF) >= want) return true;
@@ -77,7 +80,8 @@ __device__ __forceinline__ bool arrivals_wait(const int* counter, int want, vola
 
 // Bounded wait until a counter written by other CTAs of this launch reaches `want` (acquire at gpu scope).
 __device__ __forceinline__ bool flag_wait(const int* flag, int want, volatile int* abort_flag) {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    const uint32_t limit = (uint32_t)abort_flag[1];
+    for (uint32_t it = 0; it < limit; ++it) {
         int v;
         asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
         if (v >= want) return true;

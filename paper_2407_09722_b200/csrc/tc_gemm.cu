@@ -64,7 +64,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
             mbar_init(smem_u32(&s.tfull[i]), mh);
             mbar_init(smem_u32(&s.tempty[i]), 4);
         }
-        *s.abort_flag = 0;
+        s.abort_flag[0] = 0;
+        s.abort_flag[1] = (int)(p0.wait_limit ? p0.wait_limit : WAIT_LIMIT);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -153,7 +154,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
                     }
                     const uint32_t bar = smem_u32(&s.full[st]);
                     const uint32_t base = smem_u32(s.ring + (size_t)st * stage_bytes) + a_bytes;
-                    for (int b = 0; b < n_bbox; ++b)
+                    for (int b = 0; b < n_bbox && !p0.debug_no_operands; ++b)
                         tma_load_2d(base + b * bbox_rows * 128, &ch.maps[ph].x, bar, kb * TC_TILE_K, b * bbox_rows,
                                     HINT_KEEP);
                     if (++kb == p.k_blocks) kb = 0;
@@ -411,7 +412,11 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
-    if (threadIdx.x == 0 && *abort_flag && p0.status) atomicOr(p0.status, MTAD_ST_TIMEOUT);
+    if (threadIdx.x == 0 && *abort_flag && p0.status) {
+        // every sequence of the call carries the bit: the rows of all of them went through this launch
+        const int nseq = p0.R > 0 ? (T + p0.R - 1) / p0.R : 1;
+        for (int b = 0; b < nseq; ++b) atomicOr(p0.status + b, MTAD_ST_TIMEOUT);
+    }
 }
 
 __global__ void split_rows_kernel(const float* __restrict__ x, int ldx_in, __nv_bfloat16* __restrict__ out, int terms,

@@ -33,6 +33,8 @@ struct TcGemmParams {
     int n_rows_total;      // weight rows, for skipping a half that lies beyond them
     int n_tiles128;        // ceil(N / 128): row stride of lm_part
     int stages;            // smem ring depth
+    unsigned int wait_limit;     // iterations a bounded wait may poll (0: the default, 2^22)
+    int debug_no_operands;       // test hook: the operand-row producer issues no copies, so the waits on them run out
     unsigned long long* trace;   // MTAD_TRACE builds: [CTA][8] global-timer stamps of this launch, else null
     int csize;             // cluster kernel: CTAs that share a tile's k-range (1..8)
     int rpr;               // cluster kernel: rows per epilogue pass (1..8); pass q is finished by rank q % csize

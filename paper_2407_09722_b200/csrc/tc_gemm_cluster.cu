@@ -121,7 +121,8 @@ __global__ void __launch_bounds__(CL_THREADS, 2) tc_gemm_cluster_kernel(const __
             mbar_init(smem_u32(&s.empty[i]), 1);
         }
         mbar_init(smem_u32(s.tfull), 1);
-        *s.abort_flag = 0;
+        s.abort_flag[0] = 0;
+        s.abort_flag[1] = (int)(p.wait_limit ? p.wait_limit : WAIT_LIMIT);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -175,7 +176,7 @@ __global__ void __launch_bounds__(CL_THREADS, 2) tc_gemm_cluster_kernel(const __
                     break;
                 const uint32_t bar = smem_u32(&s.full[st]);
                 const uint32_t base = smem_u32(s.ring + (size_t)st * stage_bytes) + a_bytes;
-                tma_load_2d(base, &mp.x, bar, (kb0 + i) * TC_TILE_K, 0, HINT_KEEP);
+                if (!p.debug_no_operands) tma_load_2d(base, &mp.x, bar, (kb0 + i) * TC_TILE_K, 0, HINT_KEEP);
             }
             if (*abort_flag) {
                 // give the copies in flight a bounded chance to land before the CTA exits
