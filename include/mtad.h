@@ -59,6 +59,8 @@ enum {
 #define MTAD_ST_TIMEOUT     32u  /* a bounded wait inside a kernel gave up */
 #define MTAD_ST_AUX_PENDING 64u  /* more than MTAD_MAX_DEPTH + 1 tokens wait to be replayed by the auxiliary model */
 #define MTAD_ST_NONFINITE  128u  /* a row of target logits was not finite (NaN or infinite weights, cache or input) */
+#define MTAD_ST_RANGE     256u  /* an index derived from device-resident state (length, slot, node id, path) fell
+                                    outside its array: the access was skipped (corrupted state or a library bug) */
 #define MTAD_MAX_BEAM 8          /* beam width of mtad_draft */
 
 /* A Llama-style decoder (pre-RMSNorm, rotary embedding with half-split pairing (i, i + head_dim/2), grouped-
@@ -146,8 +148,7 @@ int mtad_set_warp(mtad_ctx* ctx, int top_k, float top_p);
  * equation; every intermediate beam becomes a tree node, Sec. 3.3).  At each step the beam_width kept sequences
  * are drawn without replacement, proportionally to their joint likelihood, as the beam_width largest values of
  * log q(beam) + log q(token | beam) + Gumbel noise, noise = -log(-log(u)).
- *   seqs        host  [B]                 sequence ids; B = 1 for now (MTAD_E_UNIMPLEMENTED otherwise: batched
- *                                         drafts are switched off until a fault seen with B = 8 is understood)
+ *   seqs        host  [B]                 sequence ids (distinct)
  *   uniforms    device [B, gamma, beam_width, vocab] fp32 in (0,1)
  *   tok,parent,depth  device [B, gamma*beam_width] int32  node arrays, layer by layer (parent = -1: child of root)
  *   node_logq   device [B, gamma*beam_width] fp32  joint draft log-likelihood of the path ending at each node
@@ -249,6 +250,24 @@ uint64_t mtad_kernel_launches(void);
  * (bf16, device, 16-byte aligned), T <= 256, K a multiple of 8 and at most the context's largest FFN width.
  * For unit tests and kernel timing; uses the context's workspace. */
 int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, int T, float* y, void* stream);
+
+/* Extent audit (host arithmetic only: no device, no driver, descriptors may carry null pointers).  For one call on a
+ * context created with (target, aux, max_batch, max_nodes) it lists, per array the call's kernels touch - every region
+ * of the workspace, the KV caches, the caller's arrays - `reach`, one past the largest element index the kernels form
+ * into it, and `extent`, the elements it holds; reach <= extent must hold everywhere.  call: MTAD_AUDIT_VERIFY (B
+ * sequences of nodes + 1 rows, depth gamma), MTAD_AUDIT_DRAFT (mtad_draft with gamma, beam; every step), or
+ * MTAD_AUDIT_COMMIT (kv_commit after such a verify).  len_ub: largest committed length of the sequences.  Writes at
+ * most max_out records, *n_out = records there are; `what` points at static strings. */
+typedef struct mtad_extent { const char* what; int64_t reach; int64_t extent; } mtad_extent;
+enum { MTAD_AUDIT_VERIFY = 0, MTAD_AUDIT_DRAFT = 1, MTAD_AUDIT_COMMIT = 2 };
+int mtad_audit_extents(const mtad_model_desc* target, const mtad_model_desc* aux, int max_batch, int max_nodes,
+                       int call, int B, int nodes, int gamma, int beam, int64_t len_ub, mtad_extent* out,
+                       int max_out, int* n_out);
+
+/* Every array of the workspace is followed by 64 guard bytes written at mtad_create.  Synchronises the stream, reads
+ * them back and returns how many arrays have damaged guards (0: none; *damaged, if given, names the first one) - a
+ * write past the end of a workspace array that happened to land in mapped memory shows up here.  For tests. */
+int mtad_debug_check_canaries(mtad_ctx* ctx, void* stream, const char** damaged);
 
 /* Test hook for the time-out path: wait_limit = iterations a bounded wait inside the GEMM kernels may poll (0: the
  * default); no_operands != 0 makes the GEMM kernels leave out their operand-row copies, so the waits on them run out

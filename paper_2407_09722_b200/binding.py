@@ -37,13 +37,20 @@ class Result(C.Structure):
                                            "node_LP", "row_lse", "row_cand", "row_cand_lp", "margin", "status")]
 
 
+class Extent(C.Structure):
+    _fields_ = [("what", C.c_char_p), ("reach", C.c_int64), ("extent", C.c_int64)]
+
+
+AUDIT_VERIFY, AUDIT_DRAFT, AUDIT_COMMIT = 0, 1, 2
+
 EXPORTS = ("mtad_workspace_bytes", "mtad_create", "mtad_destroy", "mtad_seq_set", "mtad_seq_get", "mtad_draft",
            "mtad_verify_chain", "mtad_verify_tree", "kv_commit", "mtad_status_str", "mtad_last_cuda_error",
            "mtad_profile_begin", "mtad_profile_end", "mtad_kernel_launches", "mtad_verify_chain_static",
            "mtad_debug_gemm", "mtad_set_warp", "mtad_profile_grouped",
-           "mtad_verify_chain_spd", "mtad_seq_hint", "mtad_debug_set_wait")
+           "mtad_verify_chain_spd", "mtad_seq_hint", "mtad_debug_set_wait", "mtad_audit_extents",
+           "mtad_debug_check_canaries")
 MTAD_STATIC_SCRATCH_BYTES = 16 << 20
-MTAD_ST_TIMEOUT, MTAD_ST_AUX_PENDING, MTAD_ST_NONFINITE = 32, 64, 128      # device status bits (mtad.h)
+MTAD_ST_TIMEOUT, MTAD_ST_AUX_PENDING, MTAD_ST_NONFINITE, MTAD_ST_RANGE = 32, 64, 128, 256      # device status bits (mtad.h)
 KERNEL_CLASSES = ("prepare", "norm", "gemm", "rope_append", "attention", "lm_reduce", "accept", "commit")
 
 _lib = None
@@ -68,7 +75,9 @@ def load_library() -> C.CDLL:
     lib.mtad_seq_get.argtypes = [P, I, I32P, I32P, P]
     lib.mtad_set_warp.argtypes = [P, I, C.c_float]
     lib.mtad_seq_hint.argtypes = [P, I, C.c_int32]
+    lib.mtad_audit_extents.argtypes = [MD, MD, I, I, I, I, I, I, I, C.c_int64, C.POINTER(Extent), I, C.POINTER(I)]
     lib.mtad_debug_set_wait.argtypes = [P, C.c_uint, I]
+    lib.mtad_debug_check_canaries.argtypes = [P, P, C.POINTER(C.c_char_p)]
     lib.mtad_profile_grouped.argtypes = [P, I]
     lib.mtad_draft.argtypes = [P, I, I32P, I, I, P, P, P, P, P, P, P, P]
     lib.mtad_verify_chain.argtypes = [P, I, I32P, I, P, P, F, P, RS, P]
@@ -235,6 +244,14 @@ class Context:
         self._check(self._lib.mtad_debug_set_wait(self.handle, wait_limit, 1 if no_operands else 0),
                     "mtad_debug_set_wait")
 
+    def mtad_debug_check_canaries(self, stream=None) -> str:
+        """Name of the first workspace array whose guard bytes are damaged, '' if all are intact."""
+        name = C.c_char_p(None)
+        n = self._lib.mtad_debug_check_canaries(self.handle, _stream(stream), C.byref(name))
+        if n < 0:
+            raise MtadError(n, "mtad_debug_check_canaries", self._lib.mtad_last_cuda_error(self.handle))
+        return name.value.decode() if n > 0 and name.value else ""
+
     def mtad_seq_get(self, seq: int, stream=None):
         a, b = C.c_int32(), C.c_int32()
         self._check(self._lib.mtad_seq_get(self.handle, seq, C.byref(a), C.byref(b), _stream(stream)), "mtad_seq_get")
@@ -315,6 +332,24 @@ def mtad_verify_chain_static(target: ModelDesc, kv_len: int, root_token: int, ga
     return load_library().mtad_verify_chain_static(
         C.byref(target), kv_len, root_token, gamma, _ptr(draft_tok, torch.int32), _ptr(draft_logq, torch.float32),
         log_tau, _ptr(bonus_uniform, torch.float32), C.byref(out.struct), _stream(stream))
+
+
+def shape_desc(shape, capacity: int) -> ModelDesc:
+    """Descriptor of a model shape without any memory behind it (for the host-only extent audit)."""
+    return ModelDesc(shape.layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.d_ffn,
+                     shape.vocab, shape.rope_base, shape.rms_eps, None, None, None, None, None, capacity)
+
+
+def mtad_audit_extents(target: ModelDesc, aux: Optional[ModelDesc], max_batch: int, max_nodes: int, call: int, B: int,
+                       nodes: int, gamma: int, beam: int, len_ub: int):
+    """[(what, reach, extent)] of one call shape: see mtad_audit_extents in mtad.h.  Host arithmetic only."""
+    out = (Extent * 4096)()
+    n = C.c_int(0)
+    rc = load_library().mtad_audit_extents(C.byref(target), C.byref(aux) if aux is not None else None, max_batch,
+                                           max_nodes, call, B, nodes, gamma, beam, len_ub, out, 4096, C.byref(n))
+    if rc != MTAD_OK:
+        raise MtadError(rc, "mtad_audit_extents")
+    return [(out[i].what.decode(), out[i].reach, out[i].extent) for i in range(min(n.value, 4096))]
 
 
 def mtad_kernel_launches() -> int:

@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <map>
 #include <new>
 
 #include "common.cuh"
@@ -21,10 +22,29 @@ struct WeightMaps {                      // index 0, 1, 2: tiles of 128, 256, 51
     bool ok = false;
 };
 
+constexpr size_t kCanaryBytes = 64;
+struct Region {                 // one array of the workspace: where it starts and how many elements it holds
+    const char* name;
+    size_t off, count, elem;
+};
+
+// One GEMM launch of the tensor-core forward, and the plan of a whole forward: everything about the launches that
+// depends only on (model, sequences per call, rows per sequence, LM-head mode).  Plans are built once per shape and
+// kept in the context; a call patches in what changes from call to call (status words, uniforms, debug fields).
+struct GemmDesc { TcMaps mp; TcGemmParams p; double bytes; bool cluster; };
+struct ForwardPlan {
+    std::vector<GemmDesc> g;           // per layer: QKV, O, gate/up, down; then the LM head
+    int lm_tiles128 = 0;
+    bool maps = false;                 // tensor maps encoded (false: decomposition only, for the extent audit)
+};
+
 struct mtad_ctx {
+    std::vector<Region> regions;        // the workspace's arrays, each followed by kCanaryBytes of guard pattern
+    char* ws_base = nullptr;
+    std::map<uint64_t, ForwardPlan> plans;   // by (model, sequences, rows per sequence, LM-head mode)
     WeightMaps tmaps, amaps;
     bool use_tc = false, use_pdl = false;
-    size_t tc_ws_floats = 0, tc_counter_n = 0, tc_flag_n = 0, xf_elems = 0;
+    size_t tc_ws_floats = 0, tc_counter_n = 0, xf_elems = 0;
     ModelView target, aux;
     bool has_aux = false;
     int max_batch = 0, max_nodes = 0, T_max = 0;
@@ -95,12 +115,14 @@ namespace {
 struct Carver {
     char* base;
     size_t off = 0;
+    std::vector<Region>* log = nullptr;
     explicit Carver(void* b) : base(static_cast<char*>(b)) {}
     template <typename T>
-    T* take(size_t count) {
+    T* take(size_t count, const char* name) {
         off = (off + 255) & ~size_t(255);
         T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
-        off += count * sizeof(T);
+        if (log) log->push_back({name, off, count, sizeof(T)});
+        off += count * sizeof(T) + kCanaryBytes;          // guard words behind every array (mtad_debug_check_canaries)
         return p;
     }
 };
@@ -126,8 +148,9 @@ bool model_ptrs_ok(const mtad_model_desc* m) {
 
 // Lays out the workspace; with base == nullptr only measures it.
 size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, int max_batch, int max_nodes,
-             void* base) {
+             void* base, std::vector<Region>* log = nullptr) {
     Carver k(base);
+    k.log = log;
     const size_t T = (size_t)max_batch * (max_nodes + 1);
     auto mx = [&](auto f) { size_t v = f(t); if (a) v = std::max(v, (size_t)f(a)); return v; };
     const size_t d = mx([](const mtad_model_desc* m) { return (size_t)m->d_model; });
@@ -143,48 +166,48 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
         return (size_t)m->n_q_heads * splits * (m->head_dim + 2);
     });
     SeqState st;
-    st.kv_len = k.take<int32_t>(max_batch);
-    st.root_tok = k.take<int32_t>(max_batch);
-    st.aux_len = k.take<int32_t>(max_batch);
-    st.aux_npend = k.take<int32_t>(max_batch);
-    st.aux_pend = k.take<int32_t>((size_t)max_batch * (MTAD_MAX_DEPTH + 1));
+    st.kv_len = k.take<int32_t>(max_batch, "st_kv_len");
+    st.root_tok = k.take<int32_t>(max_batch, "st_root_tok");
+    st.aux_len = k.take<int32_t>(max_batch, "st_aux_len");
+    st.aux_npend = k.take<int32_t>(max_batch, "st_aux_npend");
+    st.aux_pend = k.take<int32_t>((size_t)max_batch * (MTAD_MAX_DEPTH + 1), "st_aux_pend");
     RowMeta rm;
-    rm.tok = k.take<int32_t>(T);
-    rm.pos = k.take<int32_t>(T);
-    rm.slot = k.take<int32_t>(T);
-    rm.seq = k.take<int32_t>(T);
-    rm.depth = k.take<int32_t>(T);
-    rm.mask = k.take<uint32_t>(T * MTAD_MASK_WORDS);
-    rm.n_rows = k.take<int32_t>(max_batch);
-    rm.n_spec = k.take<int32_t>(max_batch);
-    rm.kv_base = k.take<int32_t>(max_batch);
-    rm.call_seq = k.take<int32_t>(max_batch);
+    rm.tok = k.take<int32_t>(T, "rm_tok");
+    rm.pos = k.take<int32_t>(T, "rm_pos");
+    rm.slot = k.take<int32_t>(T, "rm_slot");
+    rm.seq = k.take<int32_t>(T, "rm_seq");
+    rm.depth = k.take<int32_t>(T, "rm_depth");
+    rm.mask = k.take<uint32_t>(T * MTAD_MASK_WORDS, "rm_mask");
+    rm.n_rows = k.take<int32_t>(max_batch, "rm_n_rows");
+    rm.n_spec = k.take<int32_t>(max_batch, "rm_n_spec");
+    rm.kv_base = k.take<int32_t>(max_batch, "rm_kv_base");
+    rm.call_seq = k.take<int32_t>(max_batch, "rm_call_seq");
     Scratch sc;
-    sc.hidden = k.take<float>(T * d);
-    sc.xn = k.take<float>(T * d);
-    sc.qkv = k.take<float>(T * qkv);
-    sc.attn = k.take<float>(T * qd);
-    sc.act = k.take<float>(T * F);
-    sc.rope = k.take<float>(T * hh * 2);
-    sc.attn_part = k.take<float>(T * part);
-    sc.q_hi = k.take<__nv_bfloat16>(T * qd);
-    sc.q_lo = k.take<__nv_bfloat16>(T * qd);
-    sc.logits = k.take<float>(T * V);
-    sc.node_lp = k.take<float>(T);
-    sc.row_lse = k.take<float>(T);
-    sc.row_cand = k.take<int32_t>(T);
-    sc.row_cand_lp = k.take<float>(T);
-    rm.prow = k.take<int32_t>(T);
+    sc.hidden = k.take<float>(T * d, "hidden");
+    sc.xn = k.take<float>(T * d, "xn");
+    sc.qkv = k.take<float>(T * qkv, "qkv");
+    sc.attn = k.take<float>(T * qd, "attn");
+    sc.act = k.take<float>(T * F, "act");
+    sc.rope = k.take<float>(T * hh * 2, "rope");
+    sc.attn_part = k.take<float>(T * part, "attn_part");
+    sc.q_hi = k.take<__nv_bfloat16>(T * qd, "q_hi");
+    sc.q_lo = k.take<__nv_bfloat16>(T * qd, "q_lo");
+    sc.logits = k.take<float>(T * V, "logits");
+    sc.node_lp = k.take<float>(T, "node_lp");
+    sc.row_lse = k.take<float>(T, "row_lse");
+    sc.row_cand = k.take<int32_t>(T, "row_cand");
+    sc.row_cand_lp = k.take<float>(T, "row_cand_lp");
+    rm.prow = k.take<int32_t>(T, "rm_prow");
     // tensor-core path buffers (operand rows are always TC_X_ROWS high so that the TMA box never leaves them)
     const size_t Tc = std::min<size_t>(T, TC_MAX_ROWS);
     const size_t rpad = (Tc + 15) / 16 * 16;
     // operand rows, hi and lo interleaved: row 2t = hi(t), row 2t + 1 = lo(t)
-    sc.xd = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * d);
-    sc.xa = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * qd);
-    sc.xf = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * F);
+    sc.xd = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * d, "xd");
+    sc.xa = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * qd, "xa");
+    sc.xf = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * F, "xf");
     const size_t dt = (d + TC_TILE_N - 1) / TC_TILE_N;
-    sc.sumsq_a = k.take<float>(dt * TC_X_ROWS);
-    sc.sumsq_b = k.take<float>(dt * TC_X_ROWS);
+    sc.sumsq_a = k.take<float>(dt * TC_X_ROWS, "sumsq_a");
+    sc.sumsq_b = k.take<float>(dt * TC_X_ROWS, "sumsq_b");
     size_t ws_tiles = 0, max_tiles = 0, lm_tiles = 0;
     auto shape_ws = [&](const mtad_model_desc* m) {
         const int qdm = m->n_q_heads * m->head_dim, kvm = m->n_kv_heads * m->head_dim;
@@ -207,33 +230,27 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     };
     shape_ws(t);
     if (a) shape_ws(a);
-    // the phases of a chained launch work side by side: one fix-up region and one set of counters per phase
-    sc.tc_ws = k.take<float>(ws_tiles * rpad * TC_TILE_N * TC_MAX_PHASES);
-    sc.tc_counters = k.take<int32_t>(max_tiles * TC_MAX_PHASES);
-    size_t layers_max = t->layers;
-    if (a) layers_max = std::max<size_t>(layers_max, a->layers);
-    const size_t flag_n = (layers_max + 1) * TC_MAX_PHASES * (max_tiles + 1);
-    sc.tc_flags = k.take<int32_t>(flag_n);
-    sc.lm_part = k.take<float4>(Tc * lm_tiles);
-    sc.node_z = k.take<float>(T);
-    sc.draft_part = a ? k.take<DraftPart>((size_t)max_batch * MTAD_MAX_BEAM * MTAD_DRAFT_CHUNKS) : nullptr;
-    sc.warp_part = k.take<WarpPart>(T * MTAD_DRAFT_CHUNKS);
-    sc.warp_row = k.take<WarpRow>(T);
+    sc.tc_ws = k.take<float>(ws_tiles * rpad * TC_TILE_N, "tc_ws");
+    sc.tc_counters = k.take<int32_t>(max_tiles, "tc_counters");
+    sc.lm_part = k.take<float4>(Tc * lm_tiles, "lm_part");
+    sc.node_z = k.take<float>(T, "node_z");
+    sc.draft_part = a ? k.take<DraftPart>((size_t)max_batch * MTAD_MAX_BEAM * MTAD_DRAFT_CHUNKS, "draft_part") : nullptr;
+    sc.warp_part = k.take<WarpPart>(T * MTAD_DRAFT_CHUNKS, "warp_part");
+    sc.warp_row = k.take<WarpRow>(T, "warp_row");
     DraftState ds;
-    ds.base_len = k.take<int32_t>(max_batch);
-    ds.npend = k.take<int32_t>(max_batch);
-    ds.gamma = k.take<int32_t>(max_batch);
-    ds.beam = k.take<int32_t>(max_batch);
-    ds.node_tok = k.take<int32_t>((size_t)max_batch * MTAD_DRAFT_NODES);
-    ds.node_parent = k.take<int32_t>((size_t)max_batch * MTAD_DRAFT_NODES);
-    ds.node_logq = k.take<float>((size_t)max_batch * MTAD_DRAFT_NODES);
-    ds.node_mask = k.take<uint32_t>((size_t)max_batch * MTAD_DRAFT_NODES * MTAD_MASK_WORDS);
-    ds.best_path = k.take<int32_t>((size_t)max_batch * MTAD_MAX_DEPTH);
+    ds.base_len = k.take<int32_t>(max_batch, "ds_base_len");
+    ds.npend = k.take<int32_t>(max_batch, "ds_npend");
+    ds.gamma = k.take<int32_t>(max_batch, "ds_gamma");
+    ds.beam = k.take<int32_t>(max_batch, "ds_beam");
+    ds.node_tok = k.take<int32_t>((size_t)max_batch * MTAD_DRAFT_NODES, "ds_node_tok");
+    ds.node_parent = k.take<int32_t>((size_t)max_batch * MTAD_DRAFT_NODES, "ds_node_parent");
+    ds.node_logq = k.take<float>((size_t)max_batch * MTAD_DRAFT_NODES, "ds_node_logq");
+    ds.node_mask = k.take<uint32_t>((size_t)max_batch * MTAD_DRAFT_NODES * MTAD_MASK_WORDS, "ds_node_mask");
+    ds.best_path = k.take<int32_t>((size_t)max_batch * MTAD_MAX_DEPTH, "ds_best_path");
     if (c) {
         c->ds = ds;
         c->st = st; c->rm = rm; c->sc = sc;
-        c->tc_ws_floats = ws_tiles * rpad * TC_TILE_N * TC_MAX_PHASES;
-        c->tc_flag_n = flag_n;
+        c->tc_ws_floats = ws_tiles * rpad * TC_TILE_N;
         c->tc_counter_n = max_tiles;
         c->xf_elems = (size_t)2 * TC_X_ROWS * F;
     }
@@ -365,60 +382,55 @@ void build_kv_map(ModelView& m) {
                                  (long long)d.layers * m.max_batch * 2 * d.n_kv_heads) == 0;
 }
 
-// The same forward on the tensor-core path: every projection is one launch of the TMA + tcgen05 GEMM with a fused
-// epilogue; activations travel between launches as bf16 hi/lo operand rows plus per-row sums of squares, so the
-// RMSNorm is applied as a per-row scale in the consumer's epilogue.  Leaves lm_part / node_z for launch_lm_merge.
-int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int B, int R, long long len_ub,
-                    const float* uniforms, uint32_t* status, bool lm_plain, cudaStream_t s) {
+// Builds the plan.  with_maps = false leaves out everything that needs the driver (the operand-row tensor maps) and
+// the weight maps: what is left is the index arithmetic of the launches.
+int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const ModelView& m, const WeightMaps* wm, int B,
+               int R, bool lm_plain, bool with_maps) {
     const int T = B * R;
     const mtad_model_desc& d = m.d;
     const int qd = d.n_q_heads * d.head_dim, kvd = d.n_kv_heads * d.head_dim;
-    const Scratch& sc = ctx->sc;
-    const long long total = std::min<long long>(len_ub, d.kv_capacity) + R;
-    int nsplit = (int)std::min<long long>(attn_split_cap(d.n_q_heads), (total + MTAD_ATTN_TILE - 1) / MTAD_ATTN_TILE);
-    nsplit = std::max(1, std::min(nsplit, (4 * 148 + d.n_q_heads * B - 1) / (d.n_q_heads * B)));
-    long long chunk = (total + nsplit - 1) / nsplit;
-    chunk = (chunk + MTAD_ATTN_TILE - 1) / MTAD_ATTN_TILE * MTAD_ATTN_TILE;
     const int rpad = (T + 15) / 16 * 16;
     const int dt = (d.d_model + TC_TILE_N - 1) / TC_TILE_N;
-    const bool pdl = ctx->use_pdl;
     const int mh = tc_halves(T);                          // weight halves per tile, as many as tensor memory allows
     int mq = mh;                                          // QKV tiles must not straddle q | k | v
     while (mq > 1 && (qd % (128 * mq) || kvd % (128 * mq))) mq /= 2;
     auto ix = [](int halves) { return halves == 1 ? 0 : (halves == 2 ? 1 : 2); };
     auto up = [](int a, int b) { return (a + b - 1) / b; };
-    // operand-row maps for this call's row count: box = all terms * rpad interleaved rows (two boxes beyond 256)
+    // operand-row maps for this row count: box = all terms * rpad interleaved rows (two boxes beyond 256)
     const int terms = tc_terms(T);
     const int xbox = terms * rpad > 256 ? terms * rpad / 2 : terms * rpad;
-    CUtensorMap xd, xa, xf;
-    if (tc_make_map(&xd, sc.xd, 2 * TC_X_ROWS, d.d_model, xbox) || tc_make_map(&xa, sc.xa, 2 * TC_X_ROWS, qd, xbox) ||
-        tc_make_map(&xf, sc.xf, 2 * TC_X_ROWS, d.d_ffn, xbox))
+    CUtensorMap xd{}, xa{}, xf{};
+    if (with_maps &&
+        (tc_make_map(&xd, sc.xd, 2 * TC_X_ROWS, d.d_model, xbox) || tc_make_map(&xa, sc.xa, 2 * TC_X_ROWS, qd, xbox) ||
+         tc_make_map(&xf, sc.xf, 2 * TC_X_ROWS, d.d_ffn, xbox)))
         return MTAD_E_CUDA;
     TcGemmParams base{};
-    base.ws = sc.tc_ws; base.counters = sc.tc_counters; base.status = status;
+    base.ws = sc.tc_ws; base.counters = sc.tc_counters;
     base.inv_dim = 1.f / (float)d.d_model; base.eps = d.rms_eps;
     base.Hq = d.n_q_heads; base.Hkv = d.n_kv_heads; base.hd = d.head_dim;
-    base.q_out = sc.qkv; base.q_hi = sc.q_hi; base.q_lo = sc.q_lo; base.rope = sc.rope; base.cache = static_cast<__nv_bfloat16*>(d.kv_cache);
-    base.slot = ctx->rm.slot; base.seq = ctx->rm.seq; base.max_batch = m.max_batch; base.cap = d.kv_capacity;
-    base.hidden = sc.hidden; base.R = R; base.prow = ctx->rm.prow; base.tok = ctx->rm.tok; base.node_z = sc.node_z;
-    base.lm_part = sc.lm_part; base.uniforms = uniforms;
-    base.wait_limit = ctx->wait_limit; base.debug_no_operands = ctx->debug_no_operands;
+    base.q_out = sc.qkv; base.q_hi = sc.q_hi; base.q_lo = sc.q_lo; base.rope = sc.rope;
+    base.cache = static_cast<__nv_bfloat16*>(d.kv_cache);
+    base.slot = rm.slot; base.seq = rm.seq; base.max_batch = m.max_batch; base.cap = d.kv_capacity;
+    base.hidden = sc.hidden; base.R = R; base.prow = rm.prow; base.tok = rm.tok; base.node_z = sc.node_z;
+    base.lm_part = sc.lm_part;
     const double wb = 2.0;
-    // Every GEMM of the step is described first; then the projections that feed one another without attention in
-    // between (O, gate/up, down, and the next layer's QKV or the LM head) are chained as phases of one launch.
-    struct GemmDesc { TcMaps mp; TcGemmParams p; double bytes; bool cluster; };
     // Calls of up to 32 rows run the projections whose tiles fill the CTA slots as clusters that reduce over
-    // distributed shared memory (tc_gemm_cluster.cu); bit k of the mask: QKV, O, gate/up, down, LM head
-    static const int cluster_mask = getenv("MTAD_TC_CLUSTER") ? atoi(getenv("MTAD_TC_CLUSTER")) : 27;
-    auto clusterize = [&](TcGemmParams& p, int n_tiles, int K, int bit) -> bool {
-        if (!((cluster_mask >> bit) & 1)) return false;
+    // distributed shared memory (tc_gemm_cluster.cu): QKV, O, down and the LM head; gate / up, with more tiles than
+    // half the CTA slots, keeps the stream-K decomposition, which balances it better.
+    auto clusterize = [&](TcGemmParams& p, int n_tiles, int K, bool want) -> bool {
+        if (!want || mh != 1) return false;
         TcGemmParams q = p;
         if (!tc_cluster_plan(q, n_tiles, K, T, 2 * kCtas)) return false;
         p = q;
         return true;
     };
-    std::vector<GemmDesc> g;           // per layer: QKV, O, gate/up, down; then the LM head
+    std::vector<GemmDesc>& g = fp.g;
+    g.clear();
     g.reserve((size_t)d.layers * 4 + 1);
+    const CUtensorMap none{};
+    auto wmap = [&](const std::vector<CUtensorMap> (&v)[3], int halves, int l) -> const CUtensorMap& {
+        return with_maps ? v[ix(halves)][l] : none;
+    };
     for (int l = 0; l < d.layers; ++l) {
         {   // QKV + rotary + append
             TcGemmParams p = base; TcMaps mp{};
@@ -427,8 +439,9 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             p.mh = mq; p.n_rows_total = (qt + 2 * kt) * 128;
             p.mode = TC_QKV; p.N = qd; p.seg_k_tile = qt; p.seg_v_tile = qt + kt; p.layer = l;
             p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = (l == 0) ? 1 : dt;
-            mp.a0 = wm.wq[ix(mq)][l]; mp.a1 = wm.wk[ix(mq)][l]; mp.a2 = wm.wv[ix(mq)][l]; mp.x = xd;
-            const bool cl = mq == 1 && clusterize(p, qt + 2 * kt, d.d_model, 0);
+            if (with_maps) { mp.a0 = wmap(wm->wq, mq, l); mp.a1 = wmap(wm->wk, mq, l); mp.a2 = wmap(wm->wv, mq, l); }
+            mp.x = xd;
+            const bool cl = mq == 1 && clusterize(p, qt + 2 * kt, d.d_model, true);
             g.push_back({mp, p, wb * (qd + 2.0 * kvd) * d.d_model, cl});
         }
         {   // O projection + residual, emits the FFN norm's operand rows
@@ -438,8 +451,9 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             p.mode = TC_RESID; p.N = d.d_model; p.sumsq_in_parts = 0;
             p.gain = m.w(l, 5); p.x_out = sc.xd; p.xk = d.d_model;
             p.sumsq_out = sc.sumsq_b;
-            mp.a0 = wm.wo[ix(mh)][l]; mp.x = xa;
-            const bool cl = mh == 1 && clusterize(p, up(d.d_model, 128), qd, 1);
+            if (with_maps) mp.a0 = wmap(wm->wo, mh, l);
+            mp.x = xa;
+            const bool cl = clusterize(p, up(d.d_model, 128), qd, true);
             g.push_back({mp, p, wb * d.d_model * qd, cl});
         }
         {   // gate / up + SwiGLU
@@ -448,9 +462,9 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             p.mh = mh; p.n_rows_total = d.d_ffn;
             p.mode = TC_SWIGLU; p.N = d.d_ffn; p.sumsq_in = sc.sumsq_b; p.sumsq_in_parts = dt;
             p.x_out = sc.xf; p.xk = d.d_ffn;
-            mp.a0 = wm.gate[ix(mh)][l]; mp.a1 = wm.up[ix(mh)][l]; mp.x = xd;
-            const bool cl = mh == 1 && clusterize(p, up(d.d_ffn, 64), d.d_model, 2);
-            g.push_back({mp, p, wb * 2.0 * d.d_ffn * d.d_model, cl});
+            if (with_maps) { mp.a0 = wmap(wm->gate, mh, l); mp.a1 = wmap(wm->up, mh, l); }
+            mp.x = xd;
+            g.push_back({mp, p, wb * 2.0 * d.d_ffn * d.d_model, false});
         }
         {   // down projection + residual, emits the next norm's operand rows
             TcGemmParams p = base; TcMaps mp{};
@@ -459,87 +473,85 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
             p.mode = TC_RESID; p.N = d.d_model; p.sumsq_in_parts = 0;
             p.gain = (l + 1 < d.layers) ? m.w(l + 1, 0) : static_cast<const __nv_bfloat16*>(d.final_norm);
             p.x_out = sc.xd; p.xk = d.d_model; p.sumsq_out = sc.sumsq_a;
-            mp.a0 = wm.down[ix(mh)][l]; mp.x = xf;
-            const bool cl = mh == 1 && clusterize(p, up(d.d_model, 128), d.d_ffn, 3);
+            if (with_maps) mp.a0 = wmap(wm->down, mh, l);
+            mp.x = xf;
+            const bool cl = clusterize(p, up(d.d_model, 128), d.d_ffn, true);
             g.push_back({mp, p, wb * d.d_model * d.d_ffn, cl});
         }
     }
-    int lm_tiles128 = 0;
     {   // LM head: per-tile log-softmax / Gumbel-argmax partials + gather of the drafted tokens' logits, or plain
-        // logits for the draft's beam selection
+        // logits for the draft's beam selection and the warped rows
         TcGemmParams p = base; TcMaps mp{};
         tc_decompose(p, up(d.vocab, 128 * mh), d.d_model, T, kCtas);
         p.mh = mh; p.n_rows_total = d.vocab; p.n_tiles128 = up(d.vocab, 128);
         p.mode = lm_plain ? TC_PLAIN : TC_LMHEAD; p.N = d.vocab; p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = dt;
         p.out = sc.logits; p.ldo = d.vocab;
-        mp.a0 = wm.lm_head[ix(mh)]; mp.x = xd;
-        lm_tiles128 = p.n_tiles128;
-        const bool cl = mh == 1 && clusterize(p, up(d.vocab, 128), d.d_model, 4);
+        if (with_maps) mp.a0 = wm->lm_head[ix(mh)];
+        mp.x = xd;
+        fp.lm_tiles128 = p.n_tiles128;
+        const bool cl = clusterize(p, up(d.vocab, 128), d.d_model, true);
         g.push_back({mp, p, wb * d.vocab * d.d_model, cl});
     }
-    // chained launches are available but off by default: with stream-K every tile of a phase finishes at the end of
-    // the phase, so a chained phase starts no earlier than a separately launched kernel with its weights prefetched
-    static const bool use_chain = getenv("MTAD_TC_CHAIN") && atoi(getenv("MTAD_TC_CHAIN")) != 0;
-    const size_t flag_stride = ctx->tc_counter_n + 1;      // per (launch, phase): tile flags, then the finished-tile count
-    bool any_cluster = false;
-    for (const GemmDesc& gd : g) any_cluster = any_cluster || gd.cluster;
-    const bool chain = use_chain && !any_cluster && mq == mh && (size_t)(d.layers + 1) * TC_MAX_PHASES * flag_stride <= ctx->tc_flag_n;
-    if (chain) CU(cudaMemsetAsync(sc.tc_flags, 0, sizeof(int32_t) * (size_t)(d.layers + 1) * TC_MAX_PHASES * flag_stride, s));
-    int launch_no = 0;
-    // launches descriptors [i0, i0 + n) as one kernel
-    auto launch = [&](size_t i0, int n) -> int {
-        if (n == 1 && g[i0].cluster) {
+    fp.maps = with_maps;
+    return MTAD_OK;
+}
+
+// Split of the keys [0, total) of the attention pass on the tensor-core path: tiles per block and blocks per head
+struct AttnSplit { int nsp, ns; };
+AttnSplit attn_split(const ModelView& m, int B, int R, long long total) {
+    const int nsp = attention_mma_tiles_per_block(m, B, R, total);
+    return {nsp, (int)(((total + 63) / 64 + nsp - 1) / nsp)};
+}
+
+// The forward on the tensor-core path: every projection is one launch of the TMA + tcgen05 GEMM with a fused
+// epilogue; activations travel between launches as bf16 operand rows plus per-row sums of squares, so the RMSNorm is
+// applied as a per-row scale in the consumer's epilogue.  Leaves lm_part / node_z for launch_lm_merge.
+int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int B, int R, long long len_ub,
+                    const float* uniforms, uint32_t* status, bool lm_plain, cudaStream_t s) {
+    const mtad_model_desc& d = m.d;
+    const Scratch& sc = ctx->sc;
+    const long long total = std::min<long long>(len_ub, d.kv_capacity) + R;
+    const bool pdl = ctx->use_pdl;
+    const uint64_t key = ((uint64_t)(&m == &ctx->aux ? 1 : 0) << 40) | ((uint64_t)B << 24) | ((uint64_t)R << 8) |
+                         (lm_plain ? 1u : 0u);
+    auto it = ctx->plans.find(key);
+    if (it == ctx->plans.end()) {
+        ForwardPlan fp;
+        if (int rc = build_plan(fp, sc, ctx->rm, m, &wm, B, R, lm_plain, true)) return rc;
+        it = ctx->plans.emplace(key, std::move(fp)).first;
+    }
+    ForwardPlan& fp = it->second;
+    auto launch = [&](size_t i) -> int {
+        GemmDesc& gd = fp.g[i];
+        TcGemmParams& p = gd.p;
+        p.status = status; p.uniforms = uniforms;
+        p.wait_limit = ctx->wait_limit; p.debug_no_operands = ctx->debug_no_operands;
 #ifdef MTAD_TRACE
-            g[i0].p.trace = trace_slot(true, g[i0].p.mode, g[i0].p.n_tiles * g[i0].p.csize, g[i0].p.csize);
+        p.trace = trace_slot(gd.cluster, p.mode,
+                             gd.cluster ? p.n_tiles * p.csize : (p.total_units + p.units_per_cta - 1) / p.units_per_cta,
+                             gd.cluster ? p.csize : 0);
 #endif
-            RUN(MTAD_K_GEMM, g[i0].bytes, 1, launch_tc_cluster(g[i0].mp, g[i0].p, pdl, s));
-            return MTAD_OK;
-        }
-        TcChain ch{};
-        ch.n_phases = n;
-        double bytes = 0;
-        for (int k = 0; k < n; ++k) {
-            ch.maps[k] = g[i0 + k].mp;
-            ch.p[k] = g[i0 + k].p;
-            bytes += g[i0 + k].bytes;
-            ch.p[k].ws = sc.tc_ws + (size_t)k * (ctx->tc_ws_floats / TC_MAX_PHASES);
-            ch.p[k].counters = sc.tc_counters + (size_t)k * ctx->tc_counter_n;
-            if (n > 1) {
-                int32_t* fl = sc.tc_flags + ((size_t)launch_no * TC_MAX_PHASES + k) * flag_stride;
-                ch.p[k].tile_done = fl;
-                ch.p[k].phase_done = fl + ctx->tc_counter_n;
-                if (k > 0) {
-                    const TcGemmParams& prev = g[i0 + k - 1].p;
-                    ch.p[k].dep_feat = (prev.mode == TC_SWIGLU ? 64 : 128) * prev.mh;
-                }
-            }
-        }
-        ++launch_no;
-#ifdef MTAD_TRACE
-        ch.p[0].trace = trace_slot(false, ch.p[0].mode, (ch.p[0].total_units + ch.p[0].units_per_cta - 1) / ch.p[0].units_per_cta, 0);
-#endif
-        RUN(MTAD_K_GEMM, bytes, 1, launch_tc_chain(ch, pdl, s));
+        if (gd.cluster) RUN(MTAD_K_GEMM, gd.bytes, 1, launch_tc_cluster(gd.mp, p, pdl, s));
+        else RUN(MTAD_K_GEMM, gd.bytes, 1, launch_tc_gemm(gd.mp, p, kCtas, pdl, s));
         return MTAD_OK;
     };
-    if (int rc = launch(0, 1)) return rc;                       // QKV of layer 0
+    if (int rc = launch(0)) return rc;                          // QKV of layer 0
     for (int l = 0; l < d.layers; ++l) {
         if (mma_attention(m)) {
-            const int nsp = attention_mma_tiles_per_block(m, B, R, total);
-            const int ns = (int)(((total + 63) / 64 + nsp - 1) / nsp);
-            RUN(MTAD_K_ATTN, 0, 2, launch_attention_mma(m, l, ctx->rm, sc, B, R, ns, nsp, status, pdl, s));
-            RUN(MTAD_K_ATTN, 0, 0, launch_attention_combine(m, ctx->rm, sc, B, R, ns, true, pdl, s));
+            const AttnSplit as = attn_split(m, B, R, total);
+            RUN(MTAD_K_ATTN, 0, 2, launch_attention_mma(m, l, ctx->rm, sc, B, R, as.ns, as.nsp, status, pdl, s));
+            RUN(MTAD_K_ATTN, 0, 0, launch_attention_combine(m, ctx->rm, sc, B, R, as.ns, true, pdl, s));
         } else {
+            int nsplit = (int)std::min<long long>(attn_split_cap(d.n_q_heads), (total + MTAD_ATTN_TILE - 1) / MTAD_ATTN_TILE);
+            nsplit = std::max(1, std::min(nsplit, (4 * 148 + d.n_q_heads * B - 1) / (d.n_q_heads * B)));
+            long long chunk = (total + nsplit - 1) / nsplit;
+            chunk = (chunk + MTAD_ATTN_TILE - 1) / MTAD_ATTN_TILE * MTAD_ATTN_TILE;
             RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, true, pdl, s));
         }
-        const size_t o = (size_t)l * 4 + 1;                     // O, gate/up, down of this layer, then what follows
-        if (chain) {
-            if (int rc = launch(o, 4)) return rc;
-        } else {
-            for (int k = 0; k < 4; ++k)
-                if (int rc = launch(o + k, 1)) return rc;
-        }
+        for (int k = 0; k < 4; ++k)                              // O, gate/up, down of this layer, then what follows
+            if (int rc = launch((size_t)l * 4 + 1 + k)) return rc;
     }
-    if (!lm_plain) RUN(MTAD_K_LMRED, 0, 2, launch_lm_merge(m, ctx->rm, sc, B, R, lm_tiles128, uniforms, status, s));
+    if (!lm_plain) RUN(MTAD_K_LMRED, 0, 2, launch_lm_merge(m, ctx->rm, sc, B, R, fp.lm_tiles128, uniforms, status, s));
     return MTAD_OK;
 }
 
@@ -577,7 +589,7 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
 
     CU(cudaMemsetAsync(out->status, 0, sizeof(uint32_t) * B, s));
     // a launch that gave up on a wait leaves split-K arrival counters behind: every call starts from zero
-    CU(cudaMemsetAsync(ctx->sc.tc_counters, 0, sizeof(int32_t) * ctx->tc_counter_n * TC_MAX_PHASES, s));
+    CU(cudaMemsetAsync(ctx->sc.tc_counters, 0, sizeof(int32_t) * ctx->tc_counter_n, s));
     PrepareArgs pa{};
     for (int i = 0; i < B; ++i) pa.seqs.v[i] = seqs[i];
     pa.B = B; pa.R = R; pa.max_depth = D; pa.n_nodes = n_nodes; pa.tok = tok; pa.parent = parent;
@@ -654,7 +666,8 @@ int mtad_create(const mtad_model_desc* target, const mtad_model_desc* aux, int m
     ctx->T_max = max_batch * (max_nodes + 1);
     ctx->len_ub.assign(max_batch, 0);
     ctx->npend_ub.assign(max_batch, 1);
-    carve(ctx, target, aux, max_batch, max_nodes, workspace);
+    carve(ctx, target, aux, max_batch, max_nodes, workspace, &ctx->regions);
+    ctx->ws_base = static_cast<char*>(workspace);
     // tensor-core path unless MTAD_PATH=simt asks for the CUDA-core kernels (or a weight pointer is not 16-byte aligned)
     const char* path = getenv("MTAD_PATH");
     ctx->use_tc = !(path && strcmp(path, "simt") == 0) && build_weight_maps(ctx->target, ctx->tmaps);
@@ -666,6 +679,8 @@ int mtad_create(const mtad_model_desc* target, const mtad_model_desc* aux, int m
     const char* pdl = getenv("MTAD_PDL");
     ctx->use_pdl = !(pdl && strcmp(pdl, "0") == 0);        // programmatic dependent launch unless MTAD_PDL=0
     cudaError_t e = cudaMemset(workspace, 0, need);
+    for (const Region& r : ctx->regions)
+        if (e == cudaSuccess) e = cudaMemset(ctx->ws_base + r.off + r.count * r.elem, 0xC5, kCanaryBytes);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete ctx; return MTAD_E_CUDA; }
     *out = ctx;
@@ -783,6 +798,25 @@ int mtad_seq_hint(mtad_ctx* ctx, int seq, int32_t kv_len) {
     return MTAD_OK;
 }
 
+int mtad_debug_check_canaries(mtad_ctx* ctx, void* stream, const char** damaged) {
+    if (!ctx) return MTAD_E_INVALID;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CU(cudaStreamSynchronize(s));
+    unsigned char buf[kCanaryBytes];
+    int bad = 0;
+    for (size_t i = 0; i < ctx->regions.size(); ++i) {
+        const Region& r = ctx->regions[i];
+        CU(cudaMemcpy(buf, ctx->ws_base + r.off + r.count * r.elem, kCanaryBytes, cudaMemcpyDeviceToHost));
+        for (size_t k = 0; k < kCanaryBytes; ++k)
+            if (buf[k] != 0xC5) {
+                if (!bad && damaged) *damaged = r.name;
+                ++bad;
+                break;
+            }
+    }
+    return bad;
+}
+
 int mtad_debug_set_wait(mtad_ctx* ctx, unsigned int wait_limit, int no_operands) {
     if (!ctx) return MTAD_E_INVALID;
     ctx->wait_limit = wait_limit;
@@ -811,10 +845,6 @@ int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_wi
     if (!seqs_ok(ctx, B, seqs)) return MTAD_E_INVALID;
     if (!uniforms || !tok || !parent || !depth || !node_logq || !logq_ref || !best_path) return MTAD_E_INVALID;
     if (gamma < 1 || beam_width < 1) return MTAD_E_INVALID;
-    // Drafts of several sequences in one call are refused for now: a call with eight sequences (13B-shaped pair,
-    // gamma 6, width 4) ended in an illegal memory access whose cause has not been found; one sequence per call is
-    // what the tests cover.
-    if (B > 1) return MTAD_E_UNIMPLEMENTED;
     if (gamma > MTAD_MAX_DEPTH || beam_width > MTAD_MAX_BEAM || gamma * beam_width > MTAD_DRAFT_NODES - MTAD_MAX_DEPTH - 1 ||
         gamma * beam_width > MTAD_MAX_NODES)
         return MTAD_E_CAPACITY;
@@ -832,7 +862,7 @@ int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_wi
     for (int i = 0; i < B; ++i) sl.v[i] = seqs[i];
     DraftOut out{tok, parent, depth, node_logq, logq_ref, best_path};
     const bool tc = ctx->use_tc && ctx->amaps.ok;
-    CU(cudaMemsetAsync(ctx->sc.tc_counters, 0, sizeof(int32_t) * ctx->tc_counter_n * TC_MAX_PHASES, s));
+    CU(cudaMemsetAsync(ctx->sc.tc_counters, 0, sizeof(int32_t) * ctx->tc_counter_n, s));
     for (int step = 0; step < gamma; ++step) {
         const int R = step == 0 ? R0 : beam_width;
         RUN(MTAD_K_PREPARE, 0, 1, launch_draft_prepare(m, ctx->st, ctx->ds, ctx->rm, ctx->sc, sl, B, R, step, beam_width,
@@ -894,10 +924,193 @@ int kv_commit(mtad_ctx* ctx, int B, const int32_t* seqs, const mtad_result* res,
         ctx->draft_active = false;
     }
     RUN(MTAD_K_COMMIT, 0, 1, launch_kv_commit(ctx->target, ctx->st, B, ctx->rm.call_seq, *res, ctx->last_D, s));
-    RUN(MTAD_K_COMMIT, 0, 1, launch_seq_advance(ctx->st, B, ctx->rm.call_seq, *res, ctx->last_D, s));
+    RUN(MTAD_K_COMMIT, 0, 1, launch_seq_advance(ctx->st, B, ctx->rm.call_seq, *res, ctx->last_D, ctx->max_batch,
+                                              (long long)ctx->target.d.kv_capacity, s));
     for (int i = 0; i < B; ++i)
         ctx->len_ub[seqs[i]] = std::min<long long>(ctx->len_ub[seqs[i]] + ctx->last_D + 1, ctx->target.d.kv_capacity);
     ctx->last_B = 0;
+    return MTAD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Extent audit: for one call shape, the largest element index that the call's kernels form into every array of the
+// workspace, into the KV caches and into the caller's arrays, next to how many elements the array holds.  Host
+// arithmetic only (no device, no driver): the launch plans are the ones the calls use, the index expressions are the
+// kernels' own helpers (idx_*), evaluated at the largest row, head, tile and split of the launch.
+// ---------------------------------------------------------------------------------------------------------------
+namespace {
+
+struct Audit {
+    std::vector<Region> regions;
+    std::vector<mtad_extent> out;
+    size_t region_count(const char* name) const {
+        for (const Region& r : regions)
+            if (strcmp(r.name, name) == 0) return r.count;
+        return 0;
+    }
+    void ws(const char* name, size_t reach) { out.push_back({name, (int64_t)reach, (int64_t)region_count(name)}); }
+    void ext(const char* name, size_t reach, size_t extent) { out.push_back({name, (int64_t)reach, (int64_t)extent}); }
+};
+
+// one decoder forward of B * R rows of model m on the tensor-core path: the prepared rows, every GEMM launch of the
+// plan, the attention passes and the LM-head reductions
+void audit_forward(Audit& au, const mtad_ctx& c, const ModelView& m, int B, int R, long long len_ub, bool lm_plain,
+                   const char* cache_name) {
+    const mtad_model_desc& d = m.d;
+    const int T = B * R, hd = d.head_dim, Hq = d.n_q_heads, Hkv = d.n_kv_heads;
+    const size_t qd = (size_t)Hq * hd;
+    const int terms = tc_terms(T);
+    // row preparation: row metadata, residual stream, rotary table, first operand rows and their statistics
+    for (const char* n : {"rm_tok", "rm_pos", "rm_slot", "rm_seq", "rm_depth", "rm_prow", "node_lp", "row_lse", "row_cand",
+                          "row_cand_lp", "node_z"})
+        au.ws(n, T);
+    au.ws("rm_mask", (size_t)T * MTAD_MASK_WORDS);
+    for (const char* n : {"rm_n_rows", "rm_n_spec", "rm_kv_base", "rm_call_seq"}) au.ws(n, B);
+    au.ws("hidden", (size_t)T * d.d_model);
+    au.ws("rope", ((size_t)(T - 1) * (hd / 2) + (hd / 2 - 1)) * 2 + 2);
+    au.ws("xd", idx_xrow(T - 1, terms, terms - 1, d.d_model, d.d_model - 1) + 1);
+    au.ws("sumsq_a", T);
+    ForwardPlan fp;
+    build_plan(fp, c.sc, c.rm, m, nullptr, B, R, lm_plain, false);
+    const long long cap = d.kv_capacity;
+    const long long slot_max = std::min<long long>(len_ub + R - 1, cap - 1);     // prepare refuses rows past the capacity
+    const size_t cache_elems = (size_t)d.layers * m.max_batch * 2 * Hkv * cap * hd;
+    for (const GemmDesc& gd : fp.g) {
+        const TcGemmParams& p = gd.p;
+        if (!gd.cluster) {
+            // split-K partial tiles: the last tile's last contributor, last half, last row, last feature
+            const size_t part_floats = (size_t)p.mh * p.rpad * TC_TILE_N;
+            au.ws("tc_ws", idx_tc_ws(p.n_tiles - 1, p.max_contrib, p.max_contrib - 1, part_floats) + part_floats);
+            au.ws("tc_counters", p.n_tiles);
+        }
+        const int t128_last = p.mode == TC_SWIGLU ? 0 : (p.n_rows_total + TC_TILE_N - 1) / TC_TILE_N - 1;
+        switch (p.mode) {
+            case TC_QKV:
+                au.ws("qkv", (size_t)(T - 1) * (Hq + 2 * Hkv) * hd + qd);
+                au.ws("q_hi", (size_t)T * qd);
+                au.ws("q_lo", (size_t)T * qd);
+                au.ext(cache_name, idx_cache(p.layer, m.max_batch, m.max_batch - 1, 1, Hkv, Hkv - 1, cap, slot_max, hd) + hd,
+                       cache_elems);
+                break;
+            case TC_RESID:
+                au.ws("hidden", (size_t)(T - 1) * p.N + p.N);
+                au.ws(p.x_out == c.sc.xd ? "xd" : "xf", idx_xrow(T - 1, terms, terms - 1, p.xk, p.N - 1) + 1);
+                au.ws(p.sumsq_out == c.sc.sumsq_a ? "sumsq_a" : "sumsq_b", (size_t)t128_last * TC_X_ROWS + T);
+                break;
+            case TC_SWIGLU:
+                au.ws("xf", idx_xrow(T - 1, terms, terms - 1, p.xk, p.N - 1) + 1);
+                break;
+            case TC_PLAIN:
+                au.ws("logits", (size_t)(T - 1) * p.ldo + p.N);
+                break;
+            default:
+                au.ws("lm_part", idx_lm_part(T - 1, p.n_tiles128, p.n_tiles128 - 1) + 1);
+                break;
+        }
+        if (p.sumsq_in_parts > 0)
+            au.ws(p.sumsq_in == c.sc.sumsq_a ? "sumsq_a" : "sumsq_b", (size_t)(p.sumsq_in_parts - 1) * TC_X_ROWS + T);
+    }
+    // attention: split-KV partials of the last row, head and split; combined rows and the O projection's operand rows
+    const long long total = std::min<long long>(len_ub, cap) + R;
+    const AttnSplit as = attn_split(m, B, R, total);
+    au.ws("attn_part", idx_attn_part(T - 1, Hq, Hq - 1, as.ns, as.ns - 1, hd) + hd + 2);
+    au.ws("attn", (size_t)T * qd);
+    au.ws("xa", idx_xrow(T - 1, terms, terms - 1, qd, qd - 1) + 1);
+    // the K/V tiles come by TMA from a map over [layers * max_batch * 2 * Hkv planes][cap][hd]: the last plane asked for
+    au.ext("kv_map_planes", (size_t)((d.layers - 1) * m.max_batch + (m.max_batch - 1)) * 2 * Hkv + 2 * Hkv,
+           (size_t)d.layers * m.max_batch * 2 * Hkv);
+}
+
+}  // namespace
+
+int mtad_audit_extents(const mtad_model_desc* target, const mtad_model_desc* aux, int max_batch, int max_nodes,
+                       int call, int B, int nodes, int gamma, int beam, int64_t len_ub, mtad_extent* out,
+                       int max_out, int* n_out) {
+    if (!out || !n_out || max_out < 0 || !model_ok(target) || (aux && !model_ok(aux))) return MTAD_E_INVALID;
+    if (max_batch < 1 || max_batch > MTAD_MAX_BATCH || max_nodes < 0 || max_nodes > MTAD_MAX_NODES) return MTAD_E_INVALID;
+    if (B < 1 || B > max_batch || nodes < 0 || nodes > max_nodes || len_ub < 0) return MTAD_E_INVALID;
+    if ((call == MTAD_AUDIT_DRAFT || (call == MTAD_AUDIT_COMMIT && aux)) && (gamma < 1 || beam < 1)) return MTAD_E_INVALID;
+    if (call == MTAD_AUDIT_DRAFT && !aux) return MTAD_E_INVALID;
+    mtad_ctx c;
+    Audit au;
+    auto fill = [&](ModelView& v, const mtad_model_desc* m) {
+        v.d = *m;
+        v.lw.assign((size_t)m->layers * MTAD_LAYER_TENSORS, nullptr);
+        v.d.layer_weights = v.lw.data();
+        v.max_batch = max_batch;
+    };
+    fill(c.target, target);
+    if (aux) { fill(c.aux, aux); c.has_aux = true; }
+    c.max_batch = max_batch; c.max_nodes = max_nodes;
+    carve(&c, target, aux, max_batch, max_nodes, nullptr, &au.regions);
+    const int D = gamma > 0 ? gamma : 1;
+    if (call == MTAD_AUDIT_VERIFY) {
+        const int R = nodes + 1;
+        if (B * R > TC_MAX_ROWS) return MTAD_E_CAPACITY;
+        audit_forward(au, c, c.target, B, R, len_ub, false, "target_cache");
+        // caller's arrays: inputs [B, nodes], logq_ref [B, D], uniforms [B, V], results as documented in mtad_result
+        au.ext("tok/parent (caller)", (size_t)(B - 1) * nodes + nodes, (size_t)B * nodes);
+        au.ext("logq_ref (caller)", (size_t)(B - 1) * D + D, (size_t)B * D);
+        au.ext("bonus_uniform (caller)", (size_t)(B - 1) * target->vocab + target->vocab, (size_t)B * target->vocab);
+        au.ext("result.path", (size_t)(B - 1) * D + D, (size_t)B * D);
+        au.ext("result.out_tok/out_lp", (size_t)(B - 1) * (D + 1) + D + 1, (size_t)B * (D + 1));
+        au.ext("result.node_lp/node_LP", (size_t)(B - 1) * nodes + nodes, (size_t)B * nodes);
+        au.ext("result.row_*", (size_t)(B - 1) * R + R, (size_t)B * R);
+        au.ext("embed rows (target)", (size_t)(target->vocab - 1) * target->d_model + target->d_model,
+               (size_t)target->vocab * target->d_model);
+    } else if (call == MTAD_AUDIT_DRAFT) {
+        if (gamma > MTAD_MAX_DEPTH || beam > MTAD_MAX_BEAM || gamma * beam > MTAD_DRAFT_NODES - MTAD_MAX_DEPTH - 1)
+            return MTAD_E_CAPACITY;
+        const int V = aux->vocab;
+        int nch = (V + 1023) / 1024;
+        nch = nch < 1 ? 1 : (nch > MTAD_DRAFT_CHUNKS ? MTAD_DRAFT_CHUNKS : nch);
+        const int P_max = MTAD_MAX_DEPTH + 1;
+        for (int step = 0; step < gamma; ++step) {
+            // step 0 replays up to `nodes + 1` pending rows (the caller's bound of the pending list), later steps run
+            // the beam nodes of a layer
+            const int R = step == 0 ? std::min(nodes + 1, P_max) : beam;
+            if (B * R > TC_MAX_ROWS) return MTAD_E_CAPACITY;
+            audit_forward(au, c, c.aux, B, R, len_ub + 1 + (long long)step * beam, true, "aux_cache");
+            // selection: per-chunk parts of every beam row, the draft state of the sequence with the largest id
+            au.ws("draft_part", ((size_t)((B - 1) * MTAD_MAX_BEAM + (step == 0 ? 0 : beam - 1))) * nch + nch);
+            const size_t n_last = (size_t)step * beam + beam - 1;
+            au.ws("ds_node_tok", (size_t)(max_batch - 1) * MTAD_DRAFT_NODES + n_last + 1);
+            au.ws("ds_node_parent", (size_t)(max_batch - 1) * MTAD_DRAFT_NODES + n_last + 1);
+            au.ws("ds_node_logq", (size_t)(max_batch - 1) * MTAD_DRAFT_NODES + n_last + 1);
+            au.ws("ds_node_mask", ((size_t)(max_batch - 1) * MTAD_DRAFT_NODES + n_last) * MTAD_MASK_WORDS + MTAD_MASK_WORDS);
+            // a node's mask bit: virtual row P + n, below MTAD_MASK_WORDS * 32
+            au.ext("mask bits (virtual rows)", (size_t)R + n_last + 1 + (step == 0 ? 0 : P_max), (size_t)MTAD_MASK_WORDS * 32);
+            au.ext("uniforms (caller)", (((size_t)(B - 1) * gamma + step) * beam + (step == 0 ? 0 : beam - 1)) * V + V,
+                   (size_t)B * gamma * beam * V);
+        }
+        au.ws("ds_best_path", (size_t)(max_batch - 1) * MTAD_MAX_DEPTH + gamma);
+        au.ws("st_aux_pend", (size_t)(max_batch - 1) * (MTAD_MAX_DEPTH + 1) + P_max);
+        au.ext("tok/parent/depth/node_logq (caller)", (size_t)(B - 1) * gamma * beam + gamma * beam, (size_t)B * gamma * beam);
+        au.ext("logq_ref/best_path (caller)", (size_t)(B - 1) * gamma + gamma, (size_t)B * gamma);
+        // auxiliary cache slots: committed length + pending rows + every node
+        au.ext("aux cache slots", (size_t)len_ub + 1 + (size_t)gamma * beam, (size_t)aux->kv_capacity);
+    } else if (call == MTAD_AUDIT_COMMIT) {
+        const mtad_model_desc& t = *target;
+        const long long L1 = std::min<long long>(len_ub + 1 + nodes, t.kv_capacity);     // one past the last row moved
+        au.ext("target_cache", idx_cache(t.layers - 1, max_batch, max_batch - 1, 1, t.n_kv_heads, t.n_kv_heads - 1,
+                                         t.kv_capacity, L1 - 1, t.head_dim) + t.head_dim,
+               (size_t)t.layers * max_batch * 2 * t.n_kv_heads * t.kv_capacity * t.head_dim);
+        au.ext("commit staging (shared memory, bf16)", (size_t)D * t.head_dim, (size_t)D * t.head_dim);
+        au.ext("result.path", (size_t)(B - 1) * D + D, (size_t)B * D);
+        if (aux) {
+            const mtad_model_desc& a = *aux;
+            const long long last = len_ub + 1 + (long long)gamma * beam - 1;               // slot of the last draft node
+            au.ext("aux_cache", idx_cache(a.layers - 1, max_batch, max_batch - 1, 1, a.n_kv_heads, a.n_kv_heads - 1,
+                                          a.kv_capacity, last, a.head_dim) + a.head_dim,
+                   (size_t)a.layers * max_batch * 2 * a.n_kv_heads * a.kv_capacity * a.head_dim);
+            au.ws("ds_best_path", (size_t)(max_batch - 1) * MTAD_MAX_DEPTH + gamma);
+            au.ws("st_aux_pend", (size_t)(max_batch - 1) * (MTAD_MAX_DEPTH + 1) + 2);
+        }
+    } else {
+        return MTAD_E_INVALID;
+    }
+    *n_out = (int)au.out.size();
+    for (int i = 0; i < *n_out && i < max_out; ++i) out[i] = au.out[i];
     return MTAD_OK;
 }
 

@@ -118,7 +118,6 @@ struct Scratch {
     float* sumsq_b;      // [tiles(d)][256] the same after the O projection
     float* tc_ws;        // split-K partial tiles
     int32_t* tc_counters;
-    int32_t* tc_flags;   // finished-tile flags and counts of the phases of chained GEMM launches, zeroed per forward
     float4* lm_part;     // [T][tiles(V)]
     float* node_z;       // [T]
     DraftPart* draft_part;   // [max_batch][MTAD_MAX_BEAM][MTAD_DRAFT_CHUNKS], only with an auxiliary model
@@ -334,7 +333,7 @@ cudaError_t launch_accept(const RowMeta& rm, const Scratch& sc, const AcceptArgs
 cudaError_t launch_kv_commit(const ModelView& m, const SeqState& s, int B, const int32_t* call_seq_dev,
                              const mtad_result& res, int max_depth, cudaStream_t st);
 cudaError_t launch_seq_advance(const SeqState& s, int B, const int32_t* call_seq_dev, const mtad_result& res,
-                               int max_depth, cudaStream_t st);
+                               int max_depth, int max_batch, long long cap, cudaStream_t st);
 cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const DraftState& ds, const RowMeta& rm,
                                  const Scratch& sc, const SeqList& seqs, int B, int R, int step, int beam, bool tc,
                                  bool pdl, cudaStream_t st);

@@ -80,7 +80,7 @@ __global__ void prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, i
     if (threadIdx.x == 0) {
         uint32_t st = 0;
         if (nn < 0 || nn > N) { st |= MTAD_ST_BAD_COUNT; nn = 0; }
-        if ((long long)L + nn + 1 > kv_capacity) st |= MTAD_ST_KV_OVERFLOW;
+        if (L < 0 || (long long)L + nn + 1 > kv_capacity) st |= MTAD_ST_KV_OVERFLOW;
         const bool seq_ok = (st == 0);
         int tok = 0, depth = 0;
         uint32_t mask[MTAD_MASK_WORDS];
@@ -310,7 +310,7 @@ __global__ void rope_append_kernel(float* __restrict__ qkv, const float* __restr
         row[h * hd + j] = (a * c - b * sn) * scale;
         row[h * hd + j + half] = (b * c + a * sn) * scale;
     }
-    if (sl < 0) return;
+    if (sl < 0 || sl >= cap || (unsigned)seq[t] >= (unsigned)max_batch) return;
     const size_t kbase = ((((size_t)layer * max_batch + seq[t]) * 2 + 0) * Hkv) * cap * hd;
     const size_t vbase = ((((size_t)layer * max_batch + seq[t]) * 2 + 1) * Hkv) * cap * hd;
     const float* kr = row + Hq * hd;
@@ -604,7 +604,14 @@ __global__ void kv_commit_kernel(__nv_bfloat16* __restrict__ cache, const int32_
     const int eta = res.eta[bi];
     if (eta <= 0) return;
     const int seq = call_seq[bi];
+    if ((unsigned)seq >= (unsigned)max_batch) return;
     const int L = kv_len[seq];
+    // every source and destination row inside the cache, or nothing moves (seq_advance_kernel flags the sequence)
+    if (eta > D || L < 0 || (long long)L + 1 + eta > cap) return;
+    for (int r = 0; r < eta; ++r) {
+        const int pn = res.path[bi * D + r];
+        if (pn < 0 || (long long)L + 1 + pn >= cap) return;
+    }
     const int head = blockIdx.x % Hkv;
     const int kv = (blockIdx.x / Hkv) & 1;
     const int layer = blockIdx.x / (2 * Hkv);
@@ -621,11 +628,22 @@ __global__ void kv_commit_kernel(__nv_bfloat16* __restrict__ cache, const int32_
     }
 }
 
-__global__ void seq_advance_kernel(SeqState s, const int32_t* __restrict__ call_seq, mtad_result res, int D, int B) {
+__global__ void seq_advance_kernel(SeqState s, const int32_t* __restrict__ call_seq, mtad_result res, int D, int B,
+                                   int max_batch, long long cap) {
     const int bi = blockIdx.x * blockDim.x + threadIdx.x;
     if (bi >= B || res.status[bi] != 0) return;
     const int seq = call_seq[bi];
     const int eta = res.eta[bi];
+    bool ok = (unsigned)seq < (unsigned)max_batch && eta >= 0 && eta <= D;
+    if (ok) {
+        const long long L = s.kv_len[seq];
+        ok = L >= 0 && L + 1 + eta <= cap;
+        for (int r = 0; r < eta && ok; ++r) {
+            const int pn = res.path[bi * D + r];
+            ok = pn >= 0 && L + 1 + pn < cap;
+        }
+    }
+    if (!ok) { atomicOr(&res.status[bi], MTAD_ST_RANGE); return; }
     s.kv_len[seq] += eta + 1;
     s.root_tok[seq] = res.out_tok[bi * (D + 1) + eta];
 }
@@ -641,8 +659,8 @@ cudaError_t launch_kv_commit(const ModelView& m, const SeqState& s, int B, const
 }
 
 cudaError_t launch_seq_advance(const SeqState& s, int B, const int32_t* call_seq_dev, const mtad_result& res,
-                               int max_depth, cudaStream_t st) {
-    seq_advance_kernel<<<1, 64, 0, st>>>(s, call_seq_dev, res, max_depth, B);
+                               int max_depth, int max_batch, long long cap, cudaStream_t st) {
+    seq_advance_kernel<<<1, 64, 0, st>>>(s, call_seq_dev, res, max_depth, B, max_batch, cap);
     return cudaGetLastError();
 }
 

@@ -33,7 +33,7 @@ __device__ __forceinline__ bool before(const Cand& a, const Cand& b) {     // a 
 // ---------------------------------------------------------------------------------------------------------------
 
 __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, int vocab, int hd,
-                                     RopeInv rinv, SeqState s, DraftState ds, RowMeta rm,
+                                     RopeInv rinv, long long kv_capacity, SeqState s, DraftState ds, RowMeta rm,
                                      float* __restrict__ hidden, float* __restrict__ rope, SeqList seqs, int R, int step,
                                      int beam, const __nv_bfloat16* __restrict__ gain0, __nv_bfloat16* x, int terms,
                                      float* sumsq_out) {
@@ -75,6 +75,7 @@ __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, in
         rm.tok[t] = tok;
         rm.depth[t] = step;
         rm.pos[t] = pos;
+        if (L < 0 || P < 1 || P > MTAD_MAX_DEPTH + 1 || (long long)L + vrow >= kv_capacity) active = false;
         rm.slot[t] = active ? L + vrow : -1;
         rm.seq[t] = seq;
         rm.prow[t] = -1;
@@ -82,8 +83,10 @@ __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, in
 #pragma unroll
         for (int i = 0; i < MTAD_MASK_WORDS; ++i) rm.mask[(size_t)t * MTAD_MASK_WORDS + i] = mask[i];
         if (r == 0) {
-            rm.n_rows[bi] = step == 0 ? P : beam;
-            rm.n_spec[bi] = step == 0 ? P : P + step * beam;
+            const bool state_ok = L >= 0 && P >= 1 && P <= MTAD_MAX_DEPTH + 1 && P <= (step == 0 ? R : MTAD_MAX_DEPTH + 1) &&
+                                  (long long)L + P + (long long)step * beam <= kv_capacity;
+            rm.n_rows[bi] = !state_ok ? 0 : (step == 0 ? P : beam);
+            rm.n_spec[bi] = !state_ok ? 0 : (step == 0 ? P : P + step * beam);
             rm.kv_base[bi] = L;
             rm.call_seq[bi] = seq;
         }
@@ -120,7 +123,8 @@ cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const Dr
                                  bool pdl, cudaStream_t st) {
     return launch_pdl(draft_prepare_kernel, dim3(B * R), dim3(128), 0, st, pdl,
                       static_cast<const __nv_bfloat16*>(m.d.embed), m.d.d_model, m.d.vocab, m.d.head_dim,
-                      rope_inv((double)m.d.rope_base, m.d.head_dim), s, ds, rm, sc.hidden, sc.rope, seqs, R, step, beam,
+                      rope_inv((double)m.d.rope_base, m.d.head_dim), (long long)m.d.kv_capacity, s, ds, rm, sc.hidden,
+                      sc.rope, seqs, R, step, beam,
                       tc ? m.w(0, 0) : (const __nv_bfloat16*)nullptr, tc ? sc.xd : (__nv_bfloat16*)nullptr,
                       tc_terms(B * R), sc.sumsq_a);
 }
@@ -144,7 +148,7 @@ __global__ void __launch_bounds__(256) draft_scan_kernel(const float* __restrict
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     pdl_wait();               // the logits come from the kernel before
     pdl_trigger();
-    const int P = ds.npend[seq];
+    const int P = min(max(ds.npend[seq], 1), step == 0 ? R : MTAD_MAX_DEPTH + 1);   // in range whatever the state holds
     const int row = step == 0 ? P - 1 : j;
     const float* z = logits + (size_t)(bi * R + row) * V;
     const float* ub = uni + (((size_t)bi * gamma + step) * beam + j) * V;
@@ -212,7 +216,7 @@ __global__ void __launch_bounds__(256) draft_pick_kernel(const float* __restrict
     const int tid = threadIdx.x;
     pdl_wait();               // the chunk results come from the kernel before
     pdl_trigger();
-    const int P = ds.npend[seq];
+    const int P = min(max(ds.npend[seq], 1), step == 0 ? R : MTAD_MAX_DEPTH + 1);   // in range whatever the state holds
     const int n_beams = step == 0 ? 1 : beam;
     const int N = gamma * beam;
     __shared__ float s_lse[MTAD_MAX_BEAM], s_lq[MTAD_MAX_BEAM];
@@ -326,6 +330,20 @@ cudaError_t launch_draft_select(const ModelView& m, const DraftState& ds, const 
 // auxiliary cache roll-forward after a verification
 // ---------------------------------------------------------------------------------------------------------------
 
+// The rows that the roll-forward would touch: accepted node r (r < kept) is read from slot base + node id and written
+// to slot base + r; all of them inside [0, cap), the path entries inside the draft's node arrays.
+__device__ __forceinline__ bool aux_commit_in_range(const DraftState& ds, const mtad_result& res, int bi, int seq, int D,
+                                                    int mode, int kept, int base, long long cap) {
+    if (kept > D || kept > MTAD_MAX_DEPTH || base < 0 || (long long)base + kept > cap) return false;
+    for (int r = 0; r < kept; ++r) {
+        const int pn = res.path[bi * D + r];
+        if (pn < 0 || pn >= (mode == 0 ? MTAD_MAX_DEPTH : MTAD_DRAFT_NODES)) return false;
+        const int node = mode == 0 ? ds.best_path[seq * MTAD_MAX_DEPTH + pn] : pn;
+        if (node < 0 || node >= MTAD_DRAFT_NODES || (long long)base + node >= cap) return false;
+    }
+    return true;
+}
+
 // mode 0: the verified chain was the draft's output sequence (chain node i = draft node best_path[i]);
 // mode 1: the verified tree was the draft's tree (same node ids).  Accepted node i (depth i + 1, slot base + id)
 // moves to position base + i when the draft ran it (depth < gamma).
@@ -335,11 +353,14 @@ __global__ void aux_commit_kernel(__nv_bfloat16* __restrict__ cache, const int32
     const int bi = blockIdx.y;
     if (res.status[bi] != 0) return;
     const int seq = call_seq[bi];
+    if ((unsigned)seq >= (unsigned)max_batch) return;
     const int gamma = ds.gamma[seq];
     const int eta = res.eta[bi];
     const int kept = min(eta, gamma - 1);
     if (kept <= 0) return;
     const int base = ds.base_len[seq] + ds.npend[seq];
+    // every row read or written lies inside the cache, or nothing moves (aux_advance_kernel flags the sequence)
+    if (!aux_commit_in_range(ds, res, bi, seq, D, mode, kept, base, cap)) return;
     const int head = blockIdx.x % Hkv;
     const int kv = (blockIdx.x / Hkv) & 1;
     const int layer = blockIdx.x / (2 * Hkv);
@@ -361,11 +382,12 @@ __global__ void aux_commit_kernel(__nv_bfloat16* __restrict__ cache, const int32
 // New auxiliary state.  mode 0 / 1: after a draft (see above); mode 2: no draft produced the verified rows, the
 // accepted tokens and the new root simply join the pending list (to be replayed by the next draft).
 __global__ void aux_advance_kernel(SeqState s, DraftState ds, const int32_t* __restrict__ call_seq, mtad_result res,
-                                   int D, int mode, int B) {
+                                   int D, int mode, int B, int max_batch, long long cap) {
     const int bi = blockIdx.x * blockDim.x + threadIdx.x;
     if (bi >= B || res.status[bi] != 0) return;
     const int seq = call_seq[bi];
     const int eta = res.eta[bi];
+    if ((unsigned)seq >= (unsigned)max_batch || eta < 0 || eta > D) { atomicOr(&res.status[bi], MTAD_ST_RANGE); return; }
     int32_t* pend = s.aux_pend + seq * (MTAD_MAX_DEPTH + 1);
     const int bonus = res.out_tok[bi * (D + 1) + eta];
     if (mode == 2) {
@@ -377,6 +399,10 @@ __global__ void aux_advance_kernel(SeqState s, DraftState ds, const int32_t* __r
     }
     const int gamma = ds.gamma[seq];
     const int kept = min(eta, gamma - 1);
+    if (kept > 0 && !aux_commit_in_range(ds, res, bi, seq, D, mode, kept, ds.base_len[seq] + ds.npend[seq], cap)) {
+        atomicOr(&res.status[bi], MTAD_ST_RANGE);
+        return;
+    }
     s.aux_len[seq] = ds.base_len[seq] + ds.npend[seq] + kept;
     int np = 0;
     if (eta >= gamma) pend[np++] = res.out_tok[bi * (D + 1) + eta - 1];   // last layer's node: never run by the aux model
@@ -396,7 +422,8 @@ cudaError_t launch_aux_commit(const ModelView& aux, const SeqState& s, const Dra
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    aux_advance_kernel<<<1, 64, 0, st>>>(s, ds, call_seq_dev, res, max_depth, mode, B);
+    aux_advance_kernel<<<1, 64, 0, st>>>(s, ds, call_seq_dev, res, max_depth, mode, B, aux.max_batch,
+                                         (long long)aux.d.kv_capacity);
     return cudaGetLastError();
 }
 

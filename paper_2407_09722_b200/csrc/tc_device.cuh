@@ -258,6 +258,7 @@ __device__ __forceinline__ void epi_qkv(const TcGemmParams& p, EpiTile epi, int 
     for (int j = 0; j < EPI_ROWS; ++j) {
         const int t = r0 + j;
         if (sl[j] < 0) continue;                      // row beyond T, or an inactive row (no cache slot)
+        if (seg != 0 && (sl[j] >= p.cap || (unsigned)sq[j] >= (unsigned)p.max_batch)) continue;   // never past the cache
         if (seg == 2) {
             const size_t base = idx_cache(p.layer, p.max_batch, sq[j], 1, p.Hkv, head, p.cap, sl[j], hd);
             p.cache[base + jin] = __float2bfloat16_rn(epi[j][e]);

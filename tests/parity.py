@@ -217,4 +217,6 @@ def compare(gm: GpuModel, cases: Sequence[SeqCase], log_tau: float, u: torch.Ten
             # fp32 accumulation error: report the excess over one step
             excess = np.abs(got - want) - 2.0 ** -7 * np.abs(want)
             stats.cache_max_excess = max(stats.cache_max_excess, float(np.max(excess)))
+    damaged = gm.ctx.mtad_debug_check_canaries()
+    assert damaged == "", f"write past the end of workspace array {damaged}"
     return stats

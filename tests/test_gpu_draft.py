@@ -126,9 +126,79 @@ def test_draft_rejects_bad_arguments():
     assert c.mtad_draft([0], 4, 9, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_CAPACITY
     assert c.mtad_draft([0], 33, 1, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_CAPACITY
     assert c.mtad_draft([3], 4, 4, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_INVALID
-    # several sequences per call are refused for now (before anything is launched)
-    two = GpuModel(W.target, max_batch=2, max_nodes=40, capacity=128, aux=W.aux, aux_capacity=128)
-    u2 = torch.full((2, 4, 4, V), 0.5, device="cuda")
-    assert two.ctx.mtad_draft([0, 1], 4, 4, u2, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_UNIMPLEMENTED
     no_aux = GpuModel(W.target, max_batch=1, max_nodes=8, capacity=64)
     assert no_aux.ctx.mtad_draft([0], 4, 4, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_INVALID
+
+
+def _draft_gpu_batch(gm, seqs, gamma, b, u):
+    B, N = len(seqs), gamma * b
+    i32 = dict(dtype=torch.int32, device="cuda")
+    f32 = dict(dtype=torch.float32, device="cuda")
+    out = {"tok": torch.zeros(B, N, **i32), "parent": torch.zeros(B, N, **i32), "depth": torch.zeros(B, N, **i32),
+           "node_logq": torch.zeros(B, N, **f32), "logq_ref": torch.zeros(B, gamma, **f32),
+           "best_path": torch.zeros(B, gamma, **i32)}
+    gm.ctx.mtad_draft(seqs, gamma, b, u, out["tok"], out["parent"], out["depth"], out["node_logq"], out["logq_ref"],
+                      out["best_path"])
+    torch.cuda.synchronize()
+    return out
+
+
+@pytest.mark.parametrize("B,gamma,b", [(2, 4, 4), (3, 3, 2), (8, 4, 4), (8, 6, 4)])
+def test_batched_draft_verify_commit_iterations(B, gamma, b):
+    """Several ragged sequences per mtad_draft call, each followed by a chain verification and a commit of all of
+    them (Algorithm 1 for a batch), teacher-forced on the oracle's draft_beam / verify_chain / aux_commit per
+    sequence; the guard bytes behind every workspace array must be intact afterwards."""
+    gm = GpuModel(W.target, max_batch=B, max_nodes=max(gamma * b, gamma), capacity=256, aux=W.aux, aux_capacity=256)
+    V = W.target.vocab
+    seqs = list(range(B))
+    state = []
+    for s in seqs:
+        L = 10 + 7 * s
+        gm.inject(s, L)
+        gm.inject_aux(s, L)
+        root = 5 + s
+        gm.ctx.mtad_seq_set(s, L, root, aux_len=L)
+        state.append({"L": L, "La": L, "pend": [root], "root": root, "tc": gm.cache_bits(s, L),
+                      "ac": gm.aux_cache_bits(s, L)})
+    skipped = 0
+    log_tau = math.log(0.3)
+    for it in range(4):
+        u = S.uniforms(0, (35 << 40) | (it * 64 + B), B * gamma * b * V, "cuda").view(B, gamma, b, V)
+        g = _draft_gpu_batch(gm, seqs, gamma, b, u)
+        bu = S.bonus_uniforms(11, it, B, V, "cuda")
+        drafts, near = [], []
+        for s in seqs:
+            st = state[s]
+            dr = O.draft_beam(gm.oracle_aux(), st["ac"], st["La"], st["pend"], gamma, b, u[s].cpu().numpy())
+            drafts.append(dr)
+            near.append(dr.min_gap < 1e-3)
+            if not near[-1]:
+                assert g["tok"][s].tolist() == dr.tok and g["parent"][s].tolist() == dr.parent, (it, s)
+                assert g["best_path"][s].tolist() == dr.best_path
+                assert np.max(np.abs(g["node_logq"][s].cpu().numpy() - np.asarray(dr.logq))) < LP_TOL
+                assert np.max(np.abs(g["logq_ref"][s].cpu().numpy() - np.asarray(dr.logq_ref))) < LP_TOL
+        toks = torch.tensor([[dr.tok[n] for n in dr.best_path] for dr in drafts], dtype=torch.int32, device="cuda")
+        ref = torch.tensor([dr.logq_ref for dr in drafts], dtype=torch.float32, device="cuda")
+        res = M.ResultBuffers(B, gamma, gamma)
+        gm.ctx.mtad_verify_chain(seqs, gamma, toks, ref, log_tau, bu, res)
+        gm.ctx.kv_commit(seqs, res)
+        h = res.host()
+        for s in seqs:
+            st, dr = state[s], drafts[s]
+            assert int(h["status"][s]) == 0
+            r = O.verify_chain(gm.oracle(), st["tc"], st["L"], st["root"], [dr.tok[n] for n in dr.best_path],
+                               np.asarray(dr.logq_ref, np.float32).astype(np.float64), log_tau, bu[s].cpu().numpy())
+            tie = min(r.margin_accept, r.margin_tie, r.margin_bonus) < 1e-3
+            accepted = [dr.best_path[i] for i in r.path]
+            st["L"] = O.kv_commit(st["tc"], st["L"], r.path)
+            st["La"], st["pend"] = O.aux_commit(st["ac"], st["La"], st["pend"], dr, accepted, r.out_tok[-1], gamma)
+            st["root"] = r.out_tok[-1]
+            if near[s] or tie:
+                skipped += 1
+                gm.upload(s, st["tc"], st["ac"])
+                gm.ctx.mtad_seq_set(s, st["L"], st["root"], aux_len=st["La"], pending_tok=st["pend"][:-1])
+                continue
+            assert int(h["eta"][s]) == r.eta and h["out_tok"][s, :r.eta + 1].tolist() == r.out_tok, (it, s)
+            assert gm.ctx.mtad_seq_get(s) == (st["L"], st["root"])
+    assert skipped <= B
+    assert gm.ctx.mtad_debug_check_canaries() == ""
