@@ -484,7 +484,7 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
     }
     del dm, ctx
     torch.cuda.empty_cache()
-    if world == 1 and chain and w.batch == 1 and not args.no_draft_loop:      # mtad_draft takes one sequence per call
+    if world == 1 and chain and not args.no_draft_loop:
         line["draft_loop"] = draft_loop(w, min(args.steps, 32), 3, cap)
         torch.cuda.empty_cache()
     if world == 1 and not args.no_cpu_baseline:

@@ -269,6 +269,10 @@ int mtad_audit_extents(const mtad_model_desc* target, const mtad_model_desc* aux
  * write past the end of a workspace array that happened to land in mapped memory shows up here.  For tests. */
 int mtad_debug_check_canaries(mtad_ctx* ctx, void* stream, const char** damaged);
 
+/* Where the workspace array `name` (the names the extent audit reports) lies: byte offset from the workspace base,
+ * element count and element size.  For tests that inspect intermediate results. */
+int mtad_debug_region(const mtad_ctx* ctx, const char* name, size_t* offset, size_t* count, size_t* elem_bytes);
+
 /* Test hook for the time-out path: wait_limit = iterations a bounded wait inside the GEMM kernels may poll (0: the
  * default); no_operands != 0 makes the GEMM kernels leave out their operand-row copies, so the waits on them run out
  * and every sequence of the call reports MTAD_ST_TIMEOUT.  The kernels return normally; a later call with the hook

@@ -48,7 +48,7 @@ EXPORTS = ("mtad_workspace_bytes", "mtad_create", "mtad_destroy", "mtad_seq_set"
            "mtad_profile_begin", "mtad_profile_end", "mtad_kernel_launches", "mtad_verify_chain_static",
            "mtad_debug_gemm", "mtad_set_warp", "mtad_profile_grouped",
            "mtad_verify_chain_spd", "mtad_seq_hint", "mtad_debug_set_wait", "mtad_audit_extents",
-           "mtad_debug_check_canaries")
+           "mtad_debug_check_canaries", "mtad_debug_region")
 MTAD_STATIC_SCRATCH_BYTES = 16 << 20
 MTAD_ST_TIMEOUT, MTAD_ST_AUX_PENDING, MTAD_ST_NONFINITE, MTAD_ST_RANGE = 32, 64, 128, 256      # device status bits (mtad.h)
 KERNEL_CLASSES = ("prepare", "norm", "gemm", "rope_append", "attention", "lm_reduce", "accept", "commit")
@@ -77,6 +77,7 @@ def load_library() -> C.CDLL:
     lib.mtad_seq_hint.argtypes = [P, I, C.c_int32]
     lib.mtad_audit_extents.argtypes = [MD, MD, I, I, I, I, I, I, I, C.c_int64, C.POINTER(Extent), I, C.POINTER(I)]
     lib.mtad_debug_set_wait.argtypes = [P, C.c_uint, I]
+    lib.mtad_debug_region.argtypes = [P, C.c_char_p, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     lib.mtad_debug_check_canaries.argtypes = [P, P, C.POINTER(C.c_char_p)]
     lib.mtad_profile_grouped.argtypes = [P, I]
     lib.mtad_draft.argtypes = [P, I, I32P, I, I, P, P, P, P, P, P, P, P]
@@ -243,6 +244,15 @@ class Context:
     def mtad_debug_set_wait(self, wait_limit: int, no_operands: bool):
         self._check(self._lib.mtad_debug_set_wait(self.handle, wait_limit, 1 if no_operands else 0),
                     "mtad_debug_set_wait")
+
+    def region(self, name: str, dtype) -> torch.Tensor:
+        """View of the workspace array `name` (a live view of device memory, for tests)."""
+        off, cnt, el = C.c_size_t(0), C.c_size_t(0), C.c_size_t(0)
+        self._check(self._lib.mtad_debug_region(self.handle, name.encode(), C.byref(off), C.byref(cnt), C.byref(el)),
+                    "mtad_debug_region")
+        base = ((self.workspace.data_ptr() + 255) & ~255) - self.workspace.data_ptr()
+        raw = self.workspace[base + off.value: base + off.value + cnt.value * el.value]
+        return raw.view(dtype)
 
     def mtad_debug_check_canaries(self, stream=None) -> str:
         """Name of the first workspace array whose guard bytes are damaged, '' if all are intact."""

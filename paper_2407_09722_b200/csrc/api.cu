@@ -817,6 +817,16 @@ int mtad_debug_check_canaries(mtad_ctx* ctx, void* stream, const char** damaged)
     return bad;
 }
 
+int mtad_debug_region(const mtad_ctx* ctx, const char* name, size_t* offset, size_t* count, size_t* elem_bytes) {
+    if (!ctx || !name || !offset || !count || !elem_bytes) return MTAD_E_INVALID;
+    for (const Region& r : ctx->regions)
+        if (strcmp(r.name, name) == 0) {
+            *offset = r.off; *count = r.count; *elem_bytes = r.elem;
+            return MTAD_OK;
+        }
+    return MTAD_E_INVALID;
+}
+
 int mtad_debug_set_wait(mtad_ctx* ctx, unsigned int wait_limit, int no_operands) {
     if (!ctx) return MTAD_E_INVALID;
     ctx->wait_limit = wait_limit;

@@ -169,14 +169,21 @@ __global__ void attn_combine_kernel(const float* __restrict__ part, float* __res
         wsm[s] = (ms == -CUDART_INF_F) ? 0.f : expf(ms - M);
     }
     __syncthreads();
+    // A split without keys (a sequence shorter than its neighbours in the call) carries m = -inf, l = 0 and an
+    // output part that nobody wrote: whatever an earlier call left there, possibly not finite, so it must not even be
+    // multiplied by its zero weight.
     if (threadIdx.x == 0) {                          // fixed order: deterministic
         float lsum = 0.f;
-        for (int s = 0; s < nsplit; ++s) lsum += p[(size_t)s * (HD + 2) + 1] * wsm[s];
+        for (int s = 0; s < nsplit; ++s)
+            if (wsm[s] != 0.f) lsum += p[(size_t)s * (HD + 2) + 1] * wsm[s];
         wsm[nsplit] = lsum;
     }
     float acc = 0.f;
 #pragma unroll 8
-    for (int s = 0; s < nsplit; ++s) acc += p[(size_t)s * (HD + 2) + 2 + d] * wsm[s];
+    for (int s = 0; s < nsplit; ++s) {
+        const float wgt = wsm[s];
+        if (wgt != 0.f) acc += p[(size_t)s * (HD + 2) + 2 + d] * wgt;
+    }
     __syncthreads();
     const float y = acc / wsm[nsplit];
     *dst = y;

@@ -145,15 +145,21 @@ def _draft_gpu_batch(gm, seqs, gamma, b, u):
 
 @pytest.mark.parametrize("B,gamma,b", [(2, 4, 4), (3, 3, 2), (8, 4, 4), (8, 6, 4)])
 def test_batched_draft_verify_commit_iterations(B, gamma, b):
+    batched_iterations(W.target, W.aux, [10 + 7 * s for s in range(B)], gamma, b, 256, 256, 4)
+
+
+def batched_iterations(target, aux, lens, gamma, b, capacity, aux_capacity, iters):
     """Several ragged sequences per mtad_draft call, each followed by a chain verification and a commit of all of
     them (Algorithm 1 for a batch), teacher-forced on the oracle's draft_beam / verify_chain / aux_commit per
     sequence; the guard bytes behind every workspace array must be intact afterwards."""
-    gm = GpuModel(W.target, max_batch=B, max_nodes=max(gamma * b, gamma), capacity=256, aux=W.aux, aux_capacity=256)
-    V = W.target.vocab
+    B = len(lens)
+    gm = GpuModel(target, max_batch=B, max_nodes=max(gamma * b, gamma), capacity=capacity, aux=aux,
+                  aux_capacity=aux_capacity)
+    V = target.vocab
     seqs = list(range(B))
     state = []
     for s in seqs:
-        L = 10 + 7 * s
+        L = lens[s]
         gm.inject(s, L)
         gm.inject_aux(s, L)
         root = 5 + s
@@ -162,7 +168,7 @@ def test_batched_draft_verify_commit_iterations(B, gamma, b):
                       "ac": gm.aux_cache_bits(s, L)})
     skipped = 0
     log_tau = math.log(0.3)
-    for it in range(4):
+    for it in range(iters):
         u = S.uniforms(0, (35 << 40) | (it * 64 + B), B * gamma * b * V, "cuda").view(B, gamma, b, V)
         g = _draft_gpu_batch(gm, seqs, gamma, b, u)
         bu = S.bonus_uniforms(11, it, B, V, "cuda")

@@ -249,3 +249,19 @@ def test_result_head_is_one_contiguous_copy(tiny):
     assert set(hv) == {"eta", "n_out", "status", "out_tok", "out_lp"}
     for name, v in hv.items():
         assert torch.equal(v, h[name]), name
+
+
+def test_empty_attention_splits_ignore_stale_partials():
+    """A ragged batch in which the short sequence leaves whole key splits without keys: their partial outputs are
+    never written, so whatever an earlier call (of another shape, for instance a draft) left in that scratch must not
+    reach the result - here the scratch is filled with NaN beforehand."""
+    gm = GpuModel(TINY, max_batch=2, max_nodes=8, capacity=256)
+    stats = ParityStats()
+    for it, (La, Lb) in enumerate([(200, 5), (3, 190)]):
+        gm.inject(0, La)
+        gm.inject(1, Lb)
+        gm.ctx.region("attn_part", torch.float32).fill_(float("nan"))
+        cases = [SeqCase(0, La, _root(3, it, TINY.vocab), S.chain_tree(4, TINY.vocab, stream=300 + it)),
+                 SeqCase(1, Lb, _root(4, it, TINY.vocab), S.chain_tree(4, TINY.vocab, stream=310 + it))]
+        compare(gm, cases, Bn.log_tau(0.2), _u(7, it, 2, TINY.vocab), chain=True, stats=stats)
+    assert stats.ok() and stats.near_ties <= 1, stats

@@ -70,3 +70,14 @@ def test_70b_gqa_tree_two_layers():
     w = S.WORKLOADS["70b_gqa_tree"]
     shape = dataclasses.replace(w.target, layers=2)
     _run(w, shape, 1024 + 256, [0.1])
+
+
+def test_13b_pair_batched_draft_two_layers():
+    """The batched iteration of Algorithm 1 at the 13B-shaped pair: eight ragged sequences of 1024..4096 committed
+    tokens, the full-size auxiliary model (2 layers, 1024 wide, 16 heads of 64), gamma 6, beam width 4, the target cut
+    to two layers so that the oracle stays affordable: mtad_draft of all eight, mtad_verify_chain of the eight output
+    sequences, kv_commit of both caches, twice, against the oracle sequence by sequence."""
+    from tests.test_gpu_draft import batched_iterations
+    w = S.WORKLOADS["13b_batched_chain"]
+    shape = dataclasses.replace(w.target, layers=2)
+    batched_iterations(shape, w.aux, S.kv_lengths(w), w.gamma, 4, 4160, 4160, 2)
