@@ -112,7 +112,8 @@ def _blas_threads() -> int:
 class OracleSampler:
     """Times the oracle's verify step on a model truncated to `n_layers` layers (same shapes and inputs) and on the
     same model with no layers (embedding, final norm, LM head, accept rule); the full-depth time is extrapolated
-    as t0 + layers * (tn - t0) / n.  Accepted tokens are those of the truncated model's own decision."""
+    as t0 + layers * (tn - t0) / n.  Accepted tokens are always those decided by the model truncated to ONE layer,
+    whatever n_layers is, so that two samples of the same step count the same tokens."""
 
     def __init__(self, w: S.Workload, n_layers: int):
         from oracle import mtad_oracle as O
@@ -126,7 +127,7 @@ class OracleSampler:
                 "final_norm": S.make_tensor(s, 0, "final_norm", seed=SEED, device=dev)}
         layers = [{k: bits(v) for k, v in S.make_layer(s, 0, l, SEED, dev).items()} for l in range(n_layers)]
         self.models = {}
-        for n in (0, n_layers):
+        for n in sorted({0, 1, n_layers}):
             m = oracle_model(head, layer_maker=lambda l: None)
             m.layers = layers
             m.n_layers = n
@@ -148,7 +149,7 @@ class OracleSampler:
         ref = np.asarray(tree.logq_ref, np.float32).astype(np.float64)
         ts = {}
         acc = 0
-        for n in (0, self.n):
+        for n in sorted({0, 1, self.n}):
             cache = self.cache.copy()
             t0 = time.perf_counter()
             if w.kind == "chain":
@@ -156,7 +157,8 @@ class OracleSampler:
             else:
                 r = O.verify_tree(self.models[n], cache, self.lens[0], 1, tree.tok, tree.parent, ref, math.log(TAU), u)
             ts[n] = time.perf_counter() - t0
-            acc = r.eta + 1
+            if n == 1:
+                acc = r.eta + 1
         per_layer = max(ts[self.n] - ts[0], 0.0) / self.n
         est = (ts[0] + w.target.layers * per_layer) * w.batch
         return est, acc * w.batch, ts
@@ -181,21 +183,25 @@ def run_reference(args, w: S.Workload):
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": 1e3 * tot_t / max(args.steps, 1), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "tau": TAU},
+            "config": {"workload": w.name, "tau": TAU, "batch": w.batch, "rows_per_seq": w.n_nodes + 1,
+                       "kv_len_start": smp.lens, "replicas": 1,
+                       "l2": "inputs larger than L2 (weights streamed once per step)",
+                       "block_efficiency": tot_a / max(args.steps * w.batch, 1), "warp": None},
             "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
 
 
-def cpu_baseline(w: S.Workload):
+def cpu_baseline(w: S.Workload, it: int = 0):
     n_layers = min(8, w.target.layers)
     smp = OracleSampler(w, n_layers)
-    est, acc, ts = smp.step(0)
+    est, acc, ts = smp.step(it)
     return {"value": acc / est, "unit": "tokens/s", "cores": _blas_threads(), "kind": "oracle",
             "sample": (f"one oracle verify step of sequence 0 truncated to {n_layers} of {w.target.layers} layers "
                        f"({ts[n_layers]:.1f} s) and to 0 layers ({ts[0]:.1f} s); full depth extrapolated linearly, "
-                       f"times batch {w.batch}: {est:.1f} s per step"),
+                       f"times batch {w.batch}: {est:.1f} s per step; tokens: the decision of the 1-layer model on "
+                       f"step {it}, as in the --impl reference arm"),
             "est_step_s": est}
 
 
@@ -275,6 +281,123 @@ def draft_loop(w: S.Workload, steps: int, warmup: int, cap: int):
             "block_efficiency": accepted / (steps * B), "iteration_ms": total_ms / steps,
             "draft_us_median": statistics.median(d_us), "verify_commit_us_median": 1e3 * statistics.median(it_ms)
             - statistics.median(d_us), "device_status": status}
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# extra records of the default run: the other configuration the 70 % target is stated on, the rows sweep, the
+# read-only streaming rate
+# ---------------------------------------------------------------------------------------------------------------
+
+def quantiles(xs):
+    s = sorted(xs)
+    q = lambda f: s[min(len(s) - 1, max(0, int(round(f * (len(s) - 1)))))]
+    return {"median": statistics.median(s), "p10": q(0.1), "p90": q(0.9), "min": s[0], "max": s[-1]}
+
+
+def quick_time(w: S.Workload, steps: int, warmup: int, profile: bool = True, dm=None):
+    """Device-timed verify + commit steps of one workload (synthetic drafts, inputs resident): step-time quantiles,
+    achieved share of the HBM roofline on the step's algorithmic bytes and, optionally, per-class event times."""
+    import paper_2407_09722_b200 as M
+    from paper_2407_09722_b200.runtime import DeviceModel, StepInputs
+    lens = S.kv_lengths(w, SEED)
+    chain = w.kind == "chain"
+    total = warmup + steps
+    cap = (max(lens) + (total + 2) * (w.gamma + 1) + w.n_nodes + 9 + 63) // 64 * 64
+    own = dm is None
+    if own:
+        dm = DeviceModel(w.target, w.batch, w.n_nodes, cap, SEED)
+    for b_, L in enumerate(lens):
+        dm.inject(b_, L)
+    ctx = dm.ctx
+    seqs = list(range(w.batch))
+    inputs = [StepInputs(step_trees(w, i), chain) for i in range(total)]
+    unis = [S.bonus_uniforms(SEED, i, w.batch, w.target.vocab, "cuda") for i in range(min(total, 4))]
+    res = M.ResultBuffers(w.batch, inputs[0].N, inputs[0].D)
+    log_tau = math.log(TAU)
+
+    def reset():
+        for b_, L in enumerate(lens):
+            ctx.mtad_seq_set(b_, L, 1)
+
+    reset()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    acc = torch.zeros((), dtype=torch.int64, device="cuda")
+    bad = torch.zeros((), dtype=torch.int32, device="cuda")
+    for i in range(total):
+        if i == warmup:
+            torch.cuda.synchronize()
+            acc.zero_()
+            ev[0].record()
+        inputs[i].verify(ctx, seqs, log_tau, unis[i % len(unis)], res)
+        ctx.kv_commit(seqs, res)
+        acc += res.n_out.sum()
+        if i >= warmup:
+            ev[i - warmup + 1].record()
+    bad |= res.status.max()
+    torch.cuda.synchronize()
+    step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(steps)]
+    final = [ctx.mtad_seq_get(b_)[0] for b_ in seqs]
+    peak, _ = measured_peaks()
+    step_bytes = algorithmic_bytes(w, [(a + c) / 2 for a, c in zip(lens, final)])
+    med = statistics.median(step_ms)
+    out = {"workload": w.name, "batch": w.batch, "rows_per_seq": w.n_nodes + 1, "steps": steps,
+           "step_us": {k: 1e3 * v for k, v in quantiles(step_ms).items()},
+           "accepted_tokens_per_s": float(acc.item()) / (sum(step_ms) * 1e-3),
+           "algorithmic_gb": step_bytes / 1e9, "achieved_gbs": step_bytes / (med * 1e-3) / 1e9,
+           "frac_of_measured_copy": step_bytes / (med * 1e-3) / 1e9 / peak,
+           "frac_of_8000": step_bytes / (med * 1e-3) / 1e9 / 8000.0, "device_status": int(bad.item())}
+    if profile:
+        reset()
+        n = min(steps, 4)
+        ctx.mtad_profile_grouped(True)
+        ctx.mtad_profile_begin(n * (w.target.layers * 16 + 32))
+        for i in range(n):
+            inputs[i].verify(ctx, seqs, log_tau, unis[i % len(unis)], res)
+            ctx.kv_commit(seqs, res)
+        prof = ctx.mtad_profile_end()
+        ctx.mtad_profile_grouped(False)
+        out["per_class_ms_per_step"] = {k: v["ms"] / n for k, v in prof.items()}
+        g = prof["gemm"]
+        out["gemm_gbs"] = g["bytes"] / (g["ms"] * 1e-3) / 1e9 if g["ms"] > 0 else None
+    if own:
+        del dm, ctx
+        torch.cuda.empty_cache()
+    return out
+
+
+def rows_sweep(steps: int, warmup: int):
+    """Rows per forward R in {1, 2, 4, 8, 16} at the 13B shape on one set of weights: what the paper's batch-size
+    table (Sec. 4) varies - the step time is nearly flat while the weights dominate the bytes."""
+    from paper_2407_09722_b200.runtime import DeviceModel
+    base = S.WORKLOADS["13b_batched_chain"]
+    dm = DeviceModel(base.target, 1, 16, 2048 + 64 * 17, SEED)
+    out = []
+    for rows in (1, 2, 4, 8, 16):
+        w = S.Workload(f"13b_rows{rows}", base.target, base.aux, batch=1, kind="chain", gamma=rows - 1, n_nodes=rows - 1,
+                       kv_len=(2048, 2048))
+        r = quick_time(w, steps, warmup, profile=False, dm=dm)
+        out.append({"rows": rows, "step_us_median": r["step_us"]["median"], "frac_of_measured_copy": r["frac_of_measured_copy"]})
+    del dm
+    torch.cuda.empty_cache()
+    return out
+
+
+def read_only_peak(gb: float = 8.0):
+    """Read-only streaming rate of this GPU: a sum over `gb` GB of fp32 (the path is read-dominated; the copy figure
+    of MEASURED_PEAKS.json counts read + write)."""
+    n = int(gb * 1e9 / 4)
+    x = torch.ones(n, dtype=torch.float32, device="cuda")
+    best = 0.0
+    for _ in range(4):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        x.sum()
+        e1.record()
+        torch.cuda.synchronize()
+        best = max(best, n * 4 / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    del x
+    torch.cuda.empty_cache()
+    return best
 
 
 # ---------------------------------------------------------------------------------------------------------------
@@ -463,8 +586,9 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
                    "replicas": world, "l2": "inputs larger than L2 (weights streamed once per step)",
                    "block_efficiency": accepted / (args.steps * w.batch * world),
                    "warp": {"top_k": args.top_k, "top_p": args.top_p} if args.top_k > 0 else None},
-        "verify_step_us": {"median": 1e3 * statistics.median(step_ms), "min": 1e3 * min(step_ms),
-                           "max": 1e3 * max(step_ms)},
+        "verify_step_us": {k: 1e3 * v for k, v in quantiles(step_ms).items()},
+        "value_note": "verify + commit steps on synthetic drafts with synthetic draft likelihoods (no auxiliary model in "
+                      "the timed region); draft_loop.value is accepted tokens/s of whole iterations with mtad_draft",
         "step_hbm": {"algorithmic_gb": step_bytes / 1e9, "achieved_gbs": step_bytes / (ms_per_step * 1e-3) / 1e9,
                      "frac_of_measured_copy": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
                      "frac_of_8000": step_bytes / (ms_per_step * 1e-3) / 1e9 / 8000.0},
@@ -487,8 +611,13 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
     if world == 1 and chain and not args.no_draft_loop:
         line["draft_loop"] = draft_loop(w, min(args.steps, 32), 3, cap)
         torch.cuda.empty_cache()
+    if world == 1 and not args.no_extras:
+        line["read_only_peak_gbs"] = read_only_peak()
+        if w.name != "7b_tree":
+            line["tree"] = quick_time(S.WORKLOADS["7b_tree"], min(args.steps, 16), 3)
+        line["rows_sweep_13b"] = rows_sweep(8, 3)
     if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(w)
+        line["cpu_baseline"] = cpu_baseline(w, args.warmup)
     print(json.dumps(line))
 
 
@@ -501,6 +630,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-draft-loop", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the tree record, the rows sweep and the read-only rate")
     ap.add_argument("--top-k", type=int, default=0, help="warp the target rows: top-k (0 = off, the default)")
     ap.add_argument("--top-p", type=float, default=0.9)
     args = ap.parse_args()

@@ -1,6 +1,7 @@
 // Host dispatcher behind the C ABI: argument validation, workspace carving, and the launch sequence of one
 // verification step.  No device memory is allocated here; everything lives in the caller's workspace.
 #include <math.h>
+#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -13,6 +14,9 @@
 
 using namespace mtad;
 
+// K and V are rounded to bf16 for the cache: their projection accumulates at most this many k-blocks (512 elements)
+// per tensor-memory accumulator, the pieces being added in fp32 (relative error about 4e-7 instead of 4e-6 at K = 8192)
+static const int kQkvSegCap = 8;
 static const int kCtas = getenv("MTAD_TC_CTAS") ? atoi(getenv("MTAD_TC_CTAS")) : 148;   // SMs the tensor-core GEMM spreads over
 
 // Host-side tensor maps of one model's weight matrices.
@@ -393,17 +397,22 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
     const int dt = (d.d_model + TC_TILE_N - 1) / TC_TILE_N;
     const int mh = tc_halves(T);                          // weight halves per tile, as many as tensor memory allows
     int mq = mh;                                          // QKV tiles must not straddle q | k | v
-    while (mq > 1 && (qd % (128 * mq) || kvd % (128 * mq))) mq /= 2;
+    while (mq > 1 && (qd % (128 * mq) || kvd % (128 * mq) || mq * tc_qkv_terms(T) * rpad > 512)) mq /= 2;
     auto ix = [](int halves) { return halves == 1 ? 0 : (halves == 2 ? 1 : 2); };
     auto up = [](int a, int b) { return (a + b - 1) / b; };
-    // operand-row maps for this row count: box = all terms * rpad interleaved rows (two boxes beyond 256)
-    const int terms = tc_terms(T);
-    const int xbox = terms * rpad > 256 ? terms * rpad / 2 : terms * rpad;
-    CUtensorMap xd{}, xa{}, xf{};
+    // Operand rows: `terms` bf16 terms per activation row in general, `tq` for the rows that feed the Q/K/V
+    // projection and the LM head (written by the row preparation and by the down projection).  One TMA box covers
+    // all terms * rpad interleaved rows, or they are cut into two or three boxes of at most 256 rows.
+    const int terms = tc_terms(T), tq = tc_qkv_terms(T);
+    const int xbox = terms * rpad / tc_boxes(terms * rpad), qbox = tq * rpad / tc_boxes(tq * rpad);
+    CUtensorMap xd{}, xq{}, xa{}, xf{};
     if (with_maps &&
-        (tc_make_map(&xd, sc.xd, 2 * TC_X_ROWS, d.d_model, xbox) || tc_make_map(&xa, sc.xa, 2 * TC_X_ROWS, qd, xbox) ||
-         tc_make_map(&xf, sc.xf, 2 * TC_X_ROWS, d.d_ffn, xbox)))
+        (tc_make_map(&xd, sc.xd, 2 * TC_X_ROWS, d.d_model, xbox) || tc_make_map(&xq, sc.xd, 2 * TC_X_ROWS, d.d_model, qbox) ||
+         tc_make_map(&xa, sc.xa, 2 * TC_X_ROWS, qd, xbox) || tc_make_map(&xf, sc.xf, 2 * TC_X_ROWS, d.d_ffn, xbox)))
         return MTAD_E_CUDA;
+    // weight halves per tile of the launches that read tq terms: their accumulators must fit tensor memory too
+    int mhq = mh;
+    while (mhq > 1 && mhq * tq * rpad > 512) mhq /= 2;
     TcGemmParams base{};
     base.ws = sc.tc_ws; base.counters = sc.tc_counters;
     base.inv_dim = 1.f / (float)d.d_model; base.eps = d.rms_eps;
@@ -435,12 +444,13 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
         {   // QKV + rotary + append
             TcGemmParams p = base; TcMaps mp{};
             const int qt = up(qd, 128), kt = up(kvd, 128);
-            tc_decompose(p, (qt + 2 * kt) / mq, d.d_model, T, kCtas);
+            tc_decompose(p, (qt + 2 * kt) / mq, d.d_model, T, kCtas, 0, tq);
             p.mh = mq; p.n_rows_total = (qt + 2 * kt) * 128;
+            p.seg_cap = kQkvSegCap;
             p.mode = TC_QKV; p.N = qd; p.seg_k_tile = qt; p.seg_v_tile = qt + kt; p.layer = l;
             p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = (l == 0) ? 1 : dt;
             if (with_maps) { mp.a0 = wmap(wm->wq, mq, l); mp.a1 = wmap(wm->wk, mq, l); mp.a2 = wmap(wm->wv, mq, l); }
-            mp.x = xd;
+            mp.x = xq;
             const bool cl = mq == 1 && clusterize(p, qt + 2 * kt, d.d_model, true);
             g.push_back({mp, p, wb * (qd + 2.0 * kvd) * d.d_model, cl});
         }
@@ -472,7 +482,7 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
             p.mh = mh; p.n_rows_total = d.d_model;
             p.mode = TC_RESID; p.N = d.d_model; p.sumsq_in_parts = 0;
             p.gain = (l + 1 < d.layers) ? m.w(l + 1, 0) : static_cast<const __nv_bfloat16*>(d.final_norm);
-            p.x_out = sc.xd; p.xk = d.d_model; p.sumsq_out = sc.sumsq_a;
+            p.x_out = sc.xd; p.xk = d.d_model; p.sumsq_out = sc.sumsq_a; p.out_terms = tq;
             if (with_maps) mp.a0 = wmap(wm->down, mh, l);
             mp.x = xf;
             const bool cl = clusterize(p, up(d.d_model, 128), d.d_ffn, true);
@@ -482,12 +492,12 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
     {   // LM head: per-tile log-softmax / Gumbel-argmax partials + gather of the drafted tokens' logits, or plain
         // logits for the draft's beam selection and the warped rows
         TcGemmParams p = base; TcMaps mp{};
-        tc_decompose(p, up(d.vocab, 128 * mh), d.d_model, T, kCtas);
-        p.mh = mh; p.n_rows_total = d.vocab; p.n_tiles128 = up(d.vocab, 128);
+        tc_decompose(p, up(d.vocab, 128 * mhq), d.d_model, T, kCtas, 0, tq);
+        p.mh = mhq; p.n_rows_total = d.vocab; p.n_tiles128 = up(d.vocab, 128);
         p.mode = lm_plain ? TC_PLAIN : TC_LMHEAD; p.N = d.vocab; p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = dt;
         p.out = sc.logits; p.ldo = d.vocab;
-        if (with_maps) mp.a0 = wm->lm_head[ix(mh)];
-        mp.x = xd;
+        if (with_maps) mp.a0 = wm->lm_head[ix(mhq)];
+        mp.x = xq;
         fp.lm_tiles128 = p.n_tiles128;
         const bool cl = clusterize(p, up(d.vocab, 128), d.d_model, true);
         g.push_back({mp, p, wb * d.vocab * d.d_model, cl});
@@ -595,7 +605,7 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
     pa.B = B; pa.R = R; pa.max_depth = D; pa.n_nodes = n_nodes; pa.tok = tok; pa.parent = parent;
     const bool tc = ctx->use_tc && ctx->tmaps.ok && B * R <= TC_MAX_ROWS;
     if (tc) {
-        pa.gain0 = ctx->target.w(0, 0); pa.x = ctx->sc.xd; pa.terms = tc_terms(B * R);
+        pa.gain0 = ctx->target.w(0, 0); pa.x = ctx->sc.xd; pa.terms = tc_qkv_terms(B * R);
         pa.sumsq_out = ctx->sc.sumsq_a;
     }
     RUN(MTAD_K_PREPARE, 0, 1, launch_prepare(ctx->target, ctx->st, ctx->rm, ctx->sc, pa, out->status, s));
@@ -751,7 +761,7 @@ int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, 
         (size_t)p.n_tiles > ctx->tc_counter_n)
         return MTAD_E_WORKSPACE;
     TcMaps mp{};
-    const int xbox = p.terms * p.rpad > 256 ? p.terms * p.rpad / 2 : p.terms * p.rpad;
+    const int xbox = p.terms * p.rpad / tc_boxes(p.terms * p.rpad);
     if (tc_make_map(&mp.a0, W, N, K, mh == 1 ? 128 : 256) || tc_make_map(&mp.x, ctx->sc.xf, 2 * TC_X_ROWS, K, xbox))
         return MTAD_E_CUDA;
     p.mode = TC_PLAIN; p.N = N; p.out = y; p.ldo = N;
@@ -978,7 +988,8 @@ void audit_forward(Audit& au, const mtad_ctx& c, const ModelView& m, int B, int 
     for (const char* n : {"rm_n_rows", "rm_n_spec", "rm_kv_base", "rm_call_seq"}) au.ws(n, B);
     au.ws("hidden", (size_t)T * d.d_model);
     au.ws("rope", ((size_t)(T - 1) * (hd / 2) + (hd / 2 - 1)) * 2 + 2);
-    au.ws("xd", idx_xrow(T - 1, terms, terms - 1, d.d_model, d.d_model - 1) + 1);
+    const int tq = tc_qkv_terms(T);
+    au.ws("xd", idx_xrow(T - 1, tq, tq - 1, d.d_model, d.d_model - 1) + 1);
     au.ws("sumsq_a", T);
     ForwardPlan fp;
     build_plan(fp, c.sc, c.rm, m, nullptr, B, R, lm_plain, false);
@@ -1004,7 +1015,7 @@ void audit_forward(Audit& au, const mtad_ctx& c, const ModelView& m, int B, int 
                 break;
             case TC_RESID:
                 au.ws("hidden", (size_t)(T - 1) * p.N + p.N);
-                au.ws(p.x_out == c.sc.xd ? "xd" : "xf", idx_xrow(T - 1, terms, terms - 1, p.xk, p.N - 1) + 1);
+                au.ws(p.x_out == c.sc.xd ? "xd" : "xf", idx_xrow(T - 1, p.out_terms, p.out_terms - 1, p.xk, p.N - 1) + 1);
                 au.ws(p.sumsq_out == c.sc.sumsq_a ? "sumsq_a" : "sumsq_b", (size_t)t128_last * TC_X_ROWS + T);
                 break;
             case TC_SWIGLU:

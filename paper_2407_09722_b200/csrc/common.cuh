@@ -176,6 +176,11 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // relative (two terms) or to fp32 rounding (three).  The terms of row t are neighbouring rows of the operand
 // buffer: term j of element k lives at x[(t * terms + j) * K + k].
 int tc_terms(int T);       // terms used for a call of T rows: 3 up to 32 rows, else 2
+// Terms of the rows that feed the Q/K/V projection (and the LM head): three whenever their accumulator columns fit
+// tensor memory (up to 160 rows).  K and V are rounded to bf16 for the cache, and every element that rounds the other
+// way than the exact value would shifts attention scores of later rows; with two terms (2.5e-6 relative error) a few
+// tenths of a percent of the elements do, with three (2.5e-7) ten times fewer.
+int tc_qkv_terms(int T);
 __device__ __forceinline__ void store_terms(float y, __nv_bfloat16* x, size_t K, int terms) {
     const __nv_bfloat16 h = __float2bfloat16_rn(y);
     x[0] = h;

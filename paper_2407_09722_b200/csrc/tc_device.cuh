@@ -301,7 +301,7 @@ __device__ __forceinline__ void epi_resid(const TcGemmParams& p, float* red, Epi
         if (ok && t < t_end) {
             y[j] += epi[j][e];
             p.hidden[(size_t)t * p.N + n] = y[j];
-            store_terms(y[j] * g, p.x_out + (size_t)t * p.terms * p.xk + n, p.xk, p.terms);
+            store_terms(y[j] * g, p.x_out + (size_t)t * p.out_terms * p.xk + n, p.xk, p.out_terms);
         }
         y[j] *= y[j];
     }
@@ -329,7 +329,7 @@ __device__ __forceinline__ void epi_swiglu(const TcGemmParams& p, float (*epi)[E
         if (f >= p.N) return;
         for (int j = 0; j < EPI_ROWS && r0 + j < t_end; ++j) {
             const float g = epi[0][j][e], u = epi[0][j][e + 64];
-            store_terms(g / (1.f + expf(-g)) * u, p.x_out + (size_t)(r0 + j) * p.terms * p.xk + f, p.xk, p.terms);
+            store_terms(g / (1.f + expf(-g)) * u, p.x_out + (size_t)(r0 + j) * p.out_terms * p.xk + f, p.xk, p.out_terms);
         }
         return;
     }
@@ -339,7 +339,7 @@ __device__ __forceinline__ void epi_swiglu(const TcGemmParams& p, float (*epi)[E
         if (f >= p.N) break;
         for (int j = 0; j < EPI_ROWS && r0 + j < t_end; ++j) {
             const float g = epi[h][j][e], u = epi[h + hh][j][e];
-            store_terms(g / (1.f + expf(-g)) * u, p.x_out + (size_t)(r0 + j) * p.terms * p.xk + f, p.xk, p.terms);
+            store_terms(g / (1.f + expf(-g)) * u, p.x_out + (size_t)(r0 + j) * p.out_terms * p.xk + f, p.xk, p.out_terms);
         }
     }
 }

@@ -42,7 +42,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
     const int a_bytes = mh * TC_TILE_N * 128;
     const int terms = p0.terms;
     const int acc_cols = terms * p0.rpad;              // one column per operand row: the terms of a draft row are neighbours
-    const int n_bbox = acc_cols > 256 ? 2 : 1;         // TMA boxes (and MMAs per k step and half) that cover the operand rows
+    const int n_bbox = p0.n_bbox;                      // TMA boxes (and MMAs per k step and half) that cover the operand rows
     const int bbox_rows = acc_cols / n_bbox;
     const int stage_bytes = a_bytes + acc_cols * 128;
     const int stages = p0.stages, nbuf = p0.nbuf, T = p0.T;
@@ -185,7 +185,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
                 int i = 0;
                 while (i < n_units && ok) {
                     const int kb0 = (first + i) % KB;
-                    const int len = min(KB - kb0, n_units - i);
+                    const int len = min(min(KB - kb0, n_units - i), p.seg_cap);
                     const int buf = seg % nbuf;
                     const uint32_t aph = (uint32_t)(seg / nbuf) & 1u;
                     ok = mbar_wait(smem_u32(&s.tempty[buf]), aph ^ 1u, abort_flag);
@@ -257,7 +257,12 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
             while (i < n_units) {
                 const int u = first + i;
                 const int tile = u / KB, kb0 = u % KB;
-                const int len = min(KB - kb0, n_units - i);
+                // A run of this CTA inside one tile is accumulated in pieces of at most seg_cap k-blocks: the tensor
+                // cores truncate every partial sum, so a long chain drifts (about -6e-8 relative per k-block); the
+                // pieces are added up in fp32 in this CTA's partial tile
+                const int len_all = min(KB - kb0, n_units - i);
+                const int len = min(len_all, p.seg_cap);
+                const bool first_piece = (i == 0 || kb0 == 0), last_piece = (len == len_all);
                 const int buf = seg % nbuf;
                 const uint32_t aph = (uint32_t)(seg / nbuf) & 1u;
                 bool ok = true;
@@ -285,8 +290,11 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
                             tc_ld16(t_acc + 3 * rb + 32, v + 32);
 #pragma unroll
                             for (int j = 0; j < 16; ++j)
-                                if (rb + j < T)
-                                    dst[(size_t)(rb + j) * TC_TILE_N] = v[3 * j] + (v[3 * j + 1] + v[3 * j + 2]);
+                                if (rb + j < T) {
+                                    const float y = v[3 * j] + (v[3 * j + 1] + v[3 * j + 2]);
+                                    float* q = dst + (size_t)(rb + j) * TC_TILE_N;
+                                    *q = first_piece ? y : *q + y;
+                                }
                         }
                     } else {
                         for (int c0 = 0; c0 < 2 * T; c0 += 16) {
@@ -295,7 +303,11 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
                                 const int r = (c0 >> 1) + j;
-                                if (r < T) dst[(size_t)r * TC_TILE_N] = v[2 * j] + v[2 * j + 1];
+                                if (r < T) {
+                                    const float y = v[2 * j] + v[2 * j + 1];
+                                    float* q = dst + (size_t)r * TC_TILE_N;
+                                    *q = first_piece ? y : *q + y;
+                                }
                             }
                         }
                     }
@@ -303,6 +315,11 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&s.tempty[buf]));   // MMA may reuse this accumulator
+                if (!last_piece) {                                      // more of this run in this tile to come
+                    i += len;
+                    ++seg;
+                    continue;
+                }
                 __threadfence();
                 epi_bar();
                 // Who finishes the tile.  Few rows (one pass): whoever arrives last.  More rows: the contributors for
@@ -315,7 +332,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
                 const bool c_last_late = min((c_last + 1) * p.units_per_cta, p.total_units) == (tile + 1) * KB;
                 const int n_late = (c_last - c_first) + (c_last_late ? 1 : 0);
                 const bool sliced = p.sliced && n_contrib > 1;
-                const bool late = u + len == run_end;
+                const bool late = u + len == run_end;          // (last piece: u + len is the end of the run in this tile)
                 int pass0 = 0, pass_step = 1;
                 if (e == 0) {
                     const int old = atomicAdd(&p.counters[tile], 1);
@@ -473,7 +490,18 @@ int tc_make_kv_map(CUtensorMap* out, const void* cache, int hd, long long cap, l
     return r == CUDA_SUCCESS ? 0 : -1;
 }
 
-void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int sms, int per_sm) {
+int tc_boxes(int acc_cols) {
+    for (int n = 1; n <= 3; ++n)
+        if (acc_cols % n == 0 && acc_cols / n <= 256 && (acc_cols / n) % 16 == 0) return n;
+    return 0;
+}
+
+int tc_qkv_terms(int T) {
+    const int rpad = (T + 15) / 16 * 16;
+    return 3 * rpad <= 512 ? 3 : tc_terms(T);
+}
+
+void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int sms, int per_sm, int terms) {
     p.per_sm = per_sm > 0 ? per_sm : tc_ctas_per_sm(T);
     const int ctas = sms * p.per_sm;
     p.n_tiles = n_tiles;
@@ -487,11 +515,14 @@ void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int sms, int per_s
     p.max_contrib = (p.k_blocks + p.units_per_cta - 1) / p.units_per_cta + 1;
     p.T = T;
     p.rpad = (T + 15) / 16 * 16;
-    p.terms = tc_terms(T);
+    p.terms = terms > 0 ? terms : tc_terms(T);
+    p.out_terms = p.terms;
+    p.n_bbox = tc_boxes(p.terms * p.rpad);
     // more than one pass of eight rows: the passes of a tile are shared out among its contributors, which wait for
     // one another - every CTA of the launch must be resident, i.e. at most one per SM slot
     static const bool no_slice = getenv("MTAD_TC_SLICED") && atoi(getenv("MTAD_TC_SLICED")) == 0;
     p.sliced = (T > EPI_ROWS && sms <= 148 && !no_slice) ? 1 : 0;
+    p.seg_cap = 1 << 20;
 }
 
 int tc_terms(int T) {
@@ -542,7 +573,7 @@ cudaError_t launch_tc_chain(const TcChain& chain_in, bool pdl, cudaStream_t st) 
     if (f.per_sm != 1 && f.per_sm != 2) return cudaErrorInvalidValue;
     const int acc_cols = f.terms * f.rpad;
     const int tmem_budget = 512 / f.per_sm;           // the CTAs of an SM allocate tensor memory side by side
-    if (f.mh * acc_cols > tmem_budget || (acc_cols > 256 && acc_cols % 32)) return cudaErrorInvalidValue;
+    if (f.mh * acc_cols > tmem_budget || f.n_bbox < 1 || f.n_bbox != tc_boxes(acc_cols)) return cudaErrorInvalidValue;
     const int nbuf = (2 * f.mh * acc_cols <= tmem_budget) ? 2 : 1;
     const int stage_bytes = f.mh * TC_TILE_N * 128 + acc_cols * 128;
     static const int budget_kb_env = getenv("MTAD_TC_SMEM_KB") ? atoi(getenv("MTAD_TC_SMEM_KB")) : 0;
@@ -553,7 +584,8 @@ cudaError_t launch_tc_chain(const TcChain& chain_in, bool pdl, cudaStream_t st) 
     int grid = 1;
     for (int i = 0; i < ch.n_phases; ++i) {
         TcGemmParams& p = ch.p[i];
-        if (p.mh != f.mh || p.rpad != f.rpad || p.T != f.T || p.terms != f.terms || p.per_sm != f.per_sm)
+        if (p.mh != f.mh || p.rpad != f.rpad || p.T != f.T || p.terms != f.terms || p.per_sm != f.per_sm ||
+            p.n_bbox != f.n_bbox)
             return cudaErrorInvalidValue;                  // one ring, one TMEM layout
         p.nbuf = nbuf;
         p.stages = stages;

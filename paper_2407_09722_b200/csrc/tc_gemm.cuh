@@ -25,7 +25,10 @@ struct TcGemmParams {
     int n_tiles, k_blocks, total_units, units_per_cta, max_contrib;
     int T;                 // valid activation rows
     int rpad;              // T rounded up to 16; the operand tile has terms * rpad rows (the terms of a row are neighbours)
-    int terms;             // bf16 terms per activation row (2 or 3), the same for the rows read and the rows emitted
+    int terms;             // bf16 terms per activation row read (2 or 3)
+    int out_terms;         // bf16 terms per activation row emitted (what the GEMM that reads x_out expects)
+    int seg_cap;           // stream-K kernel: k-blocks accumulated in tensor memory before the accumulator is drained
+    int n_bbox;            // TMA boxes (and MMAs per k step and half) that cover the operand rows: 1, 2 or 3
     int mh;                // 128-row weight halves per tile and stage (1 or 2); a tile is mh * 128 output features
     int nbuf;              // TMEM accumulator buffers (set by the launcher)
     int per_sm;            // CTAs of this launch that share an SM (1 or 2): sets the shared- and tensor-memory budget
@@ -107,7 +110,9 @@ int tc_make_kv_map(CUtensorMap* out, const void* cache, int hd, long long cap, l
 
 // Fills the decomposition fields of p (and p.terms, p.per_sm for T rows) for a problem of n_tiles x k_blocks on
 // `sms` SMs with per_sm CTAs each (0: tc_ctas_per_sm(T)).
-void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int sms, int per_sm = 0);
+void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int sms, int per_sm = 0, int terms = 0);
+// Operand-row boxes for acc_cols accumulator columns: each at most 256 rows and a multiple of 16
+int tc_boxes(int acc_cols);
 // CTAs per SM for a call of T rows: 2 for few rows (each with half the shared memory and at most 256 columns of
 // tensor memory: one CTA's drain, fix-up and epilogue overlap the other's streaming), else 1.
 int tc_ctas_per_sm(int T);

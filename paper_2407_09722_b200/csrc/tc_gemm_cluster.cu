@@ -389,6 +389,8 @@ bool tc_cluster_plan(TcGemmParams& p, int n_tiles, int K, int T, int slots) {
     p.T = T;
     p.rpad = (T + 15) / 16 * 16;
     p.terms = tc_terms(T);
+    p.out_terms = p.terms;
+    p.n_bbox = 1;
     p.mh = 1;
     p.per_sm = 2;
     p.nbuf = 1;

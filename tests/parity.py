@@ -170,17 +170,20 @@ def _max_abs_diff(got: np.ndarray, want: np.ndarray) -> float:
 
 
 def compare(gm: GpuModel, cases: Sequence[SeqCase], log_tau: float, u: torch.Tensor, chain: bool,
-            stats: Optional[ParityStats] = None, check_cache: bool = True, warp=None) -> ParityStats:
+            stats: Optional[ParityStats] = None, check_cache: bool = True, warp=None,
+            only: Optional[Sequence[int]] = None) -> ParityStats:
     """Run both sides on the same inputs and accumulate the comparison.  warp = (top_k, top_p): warped target rows on
     both sides; a sequence with a warping decision within WARP_MARGIN of going the other way counts as a near tie
     and only its decisions-independent outputs are skipped."""
     stats = stats or ParityStats()
-    before = [gm.cache_bits(c.seq, c.L) for c in cases]
+    before = [gm.cache_bits(c.seq, c.L) if (only is None or i in only) else None for i, c in enumerate(cases)]
     res = run_gpu(gm, cases, log_tau, u, chain, warp=warp)
     h = res.host()
     u_host = u.cpu().numpy()
     for i, c in enumerate(cases):
         assert int(h["status"][i]) == 0, f"device status {int(h['status'][i])}"
+        if only is not None and i not in only:      # the device ran the whole batch; the oracle follows a part of it
+            continue
         r, ocache, newL = run_oracle(gm, c, before[i], log_tau, u_host[i], chain, warp=warp)
         n = len(r.node_lp)
         warp_tie = r.margin_warp < WARP_MARGIN

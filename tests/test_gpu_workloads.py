@@ -1,5 +1,5 @@
-"""Parity at the shapes of the benchmark workloads (same launch configuration as bench.py): the 7B chain and the 7B
-tree at full depth, the 13B ragged batch and the 70B GQA tree at reduced depth (the oracle widens every weight to
+"""Parity at the shapes of the benchmark workloads (same launch configuration as bench.py): the 7B chain, the 7B
+tree and the 13B ragged batch at full depth, the 70B GQA tree at reduced depth (the oracle widens every weight to
 fp64 on the host, so depth is what bounds its run time; width, row count, cache length and tree shape are the
 workload's own)."""
 import dataclasses
@@ -61,15 +61,32 @@ def test_70b_shape_chain_two_layers():
     assert st.max_lp_err < 5e-4
 
 
-@pytest.mark.xfail(strict=False, reason="decisions (eta, path, tokens) match, but at d = 8192 a few K/V elements round "
-                   "to the neighbouring bf16 value (fp32 against fp64 accumulation) and the peaked attention over the "
-                   "draft rows at this width amplifies a flip to ~1e-3 in a row's output; the second layer cascades: "
-                   "max |d log p| is 5e-3 here against the 2e-3 bound (CUDA-core path: 5e-4; the same model with a "
-                   "5-row chain: 1e-4)")
-def test_70b_gqa_tree_two_layers():
+@pytest.mark.parametrize("layers", [2, 8])
+def test_70b_gqa_tree(layers):
+    """129 rows at width 8192.  K and V are rounded to bf16 for the cache; an element that rounds the other way than
+    the exact value shifts the scores of the rows that attend to it, and the peaked attention over draft rows at this
+    width amplifies that by two orders of magnitude into the next layer.  The Q/K/V projection therefore keeps its
+    relative error near 5e-7 (three operand terms, accumulation chains of at most eight k-blocks), which holds the
+    log-probabilities inside the bound with room to spare at two and at eight layers."""
     w = S.WORKLOADS["70b_gqa_tree"]
-    shape = dataclasses.replace(w.target, layers=2)
-    _run(w, shape, 1024 + 256, [0.1])
+    shape = dataclasses.replace(w.target, layers=layers)
+    st = _run(w, shape, 1024 + 256, [0.1])
+    assert st.max_lp_err < 1.5e-3 and st.near_ties <= 1, st
+
+
+def test_13b_ragged_batch_full_depth():
+    """All 40 layers of the 13B-shaped batch (eight ragged sequences, seven rows each) on the device; the oracle, which
+    widens every weight to fp64 on the host, follows two of the eight sequences (the longest and the shortest)."""
+    w = S.WORKLOADS["13b_batched_chain"]
+    lens = S.kv_lengths(w)
+    gm = GpuModel(w.target, max_batch=w.batch, max_nodes=w.n_nodes, capacity=4096 + 16)
+    for b, L in enumerate(lens):
+        gm.inject(b, L)
+    u = S.bonus_uniforms(0, 0, w.batch, w.target.vocab, "cuda")
+    pick = [max(range(w.batch), key=lambda b: lens[b]), min(range(w.batch), key=lambda b: lens[b])]
+    st = compare(gm, _cases(w, lens, 0), math.log(0.1), u, chain=True, only=pick)
+    assert st.n_seq == 2 and st.ok() and st.near_ties <= 1, st
+    assert st.max_lp_err < 2e-3
 
 
 def test_13b_pair_batched_draft_two_layers():
