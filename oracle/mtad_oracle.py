@@ -49,7 +49,7 @@ Gumbel-top-b inclusion probabilities at vocab 8: beyond that it is
 from __future__ import annotations
 
 import math
-from dataclasses import dataclass
+from dataclasses import dataclass, field
 from typing import List, Optional, Sequence
 
 import numpy as np
@@ -492,6 +492,9 @@ class DraftResult:
     logq_ref: List[float]       # log q(x**_{1:i})
     min_gap: float = float("inf")   # smallest gap between neighbouring perturbed scores among the b kept and the
                                     # first one dropped, over all steps (how close any pick was to a tie)
+    slot: List[int] = field(default_factory=list)   # per node: its row in the auxiliary cache is base + slot (the
+                                                    # k-th beam of layer s has slot s * b + k); -1 for a candidate
+                                                    # that was recorded but not kept as a beam (never run)
 
 
 def gumbel_top_b(scores: np.ndarray, u: np.ndarray, b: int, with_gap: bool = False):
@@ -507,14 +510,20 @@ def gumbel_top_b(scores: np.ndarray, u: np.ndarray, b: int, with_gap: bool = Fal
 
 
 def draft_beam(model: OracleModel, cache: np.ndarray, L: int, pending_tok: Sequence[int], gamma: int, b: int,
-               u: np.ndarray) -> DraftResult:
+               u: np.ndarray, keep_all: bool = False) -> DraftResult:
     """Beam sampling of width b for gamma steps (Sec. 2.1): at each step the b kept sequences are drawn without
     replacement from p_beam over (beam, token) pairs, i.e. proportionally to the joint likelihood
     q(beam) * q(token | beam).  Every intermediate beam becomes a tree node (Sec. 3.3).
 
     pending_tok: tokens not yet in the auxiliary cache, oldest first, ending with the root (last emitted token);
     they occupy positions L .. L+len-1 and are run causally in the first step.  u: [gamma, b, vocab] uniforms.
-    Speculative node n uses cache slot L + len(pending) + n.
+    The k-th beam of layer s uses cache slot L + len(pending) + s * b + k (DraftResult.slot).
+
+    keep_all: the tree also records the candidates that the sampling looked at but did not keep - every layer
+    holds b * b nodes: the b * b best perturbed tokens of the context in the first layer, the b best perturbed tokens
+    of each of the b beams afterwards, beam by beam, best first.  The beams kept for the next step are, as before,
+    the b best of all (beam, token) pairs, which are among those; the others are leaves (slot -1).  Without keep_all a
+    layer holds just its b beams, best first (the paper's tree).
     """
     P = len(pending_tok)
     base = L + P
@@ -532,24 +541,40 @@ def draft_beam(model: OracleModel, cache: np.ndarray, L: int, pending_tok: Seque
     root_vis = vis[P - 1]
     node_vis = {-1: root_vis}
     min_gap = float("inf")
+    slot: List[int] = []
     for step in range(gamma):
         scores = beam_logq[:, None] + beam_logp    # joint log-likelihood of every (beam, token) pair
         picks, gap = gumbel_top_b(scores, u[step, :len(beams), :], b, with_gap=True)
         min_gap = min(min_gap, gap)
         V = scores.shape[1]
-        new_nodes = []
-        for flat in picks:
+        if keep_all:
+            # the layer's nodes: per beam its best perturbed tokens (b * b of the single beam of the first step)
+            per_beam = (b * b) // len(beams)
+            layer = []
+            for j in range(len(beams)):
+                own, gap_j = gumbel_top_b(scores[j:j + 1], u[step, j:j + 1, :], per_beam, with_gap=True)
+                min_gap = min(min_gap, gap_j)
+                layer += [j * V + int(v) for v in own]
+        else:
+            layer = list(picks)
+        new_nodes = [None] * len(picks)
+        for flat in layer:
             j, v = divmod(flat, V)
             n = len(tok)
             tok.append(int(v)); parent.append(beams[j]); depth.append(step + 1)
             logq.append(float(scores[j, v]))
-            node_vis[n] = node_vis[beams[j]] + [base + n]
-            new_nodes.append(n)
+            if flat in picks:                      # kept as the k-th beam of this layer: gets a row of the cache
+                k = list(picks).index(flat)
+                slot.append(step * b + k)
+                node_vis[n] = node_vis[beams[j]] + [base + step * b + k]
+                new_nodes[k] = n
+            else:
+                slot.append(-1)
         beams = new_nodes
         beam_logq = np.array([logq[n] for n in beams])
         if step + 1 < gamma:
             logits = decoder_rows(model, cache, L, [tok[n] for n in beams], [base - 1 + depth[n] for n in beams],
-                                  [base + n for n in beams], [node_vis[n] for n in beams])
+                                  [base + slot[n] for n in beams], [node_vis[n] for n in beams])
             beam_logp = log_softmax(logits)
     best = max(beams, key=lambda n: (logq[n], -n))
     path = []
@@ -558,22 +583,27 @@ def draft_beam(model: OracleModel, cache: np.ndarray, L: int, pending_tok: Seque
         path.append(n)
         n = parent[n]
     path.reverse()
-    return DraftResult(tok, parent, depth, logq, path, [logq[n] for n in path], min_gap)
+    return DraftResult(tok, parent, depth, logq, path, [logq[n] for n in path], min_gap, slot)
 
 
 def aux_commit(cache: np.ndarray, L: int, pending_tok: Sequence[int], draft: DraftResult, accepted: Sequence[int],
                bonus_tok: int, gamma: int):
     """Roll the auxiliary cache forward after a verification: the pending rows (slots L ..) are already in place;
-    accepted draft node accepted[i] (tree id, depth i + 1, slot L + P + id) moves to position L + P + i if the draft
-    ran it (depth < gamma).  A node of the last layer was never run by the auxiliary model: it stays pending, ahead
-    of the new root.  Returns (new committed length, new pending tokens ending with the new root)."""
+    accepted draft node accepted[i] (tree id, depth i + 1, row L + P + slot) moves to position L + P + i if the draft
+    ran it (a beam of a layer before the last).  A node of the last layer, or a recorded candidate that was not kept
+    as a beam, was never run by the auxiliary model: it stays pending, ahead of the new root (it can only be the last
+    node of the path: neither has children).  Returns (new committed length, new pending tokens ending with the new
+    root)."""
     P = len(pending_tok)
     base = L + P
-    kept = [n for n in accepted if draft.depth[n] < gamma]
+    slot = draft.slot if draft.slot else list(range(len(draft.tok)))
+    ran = lambda n: draft.depth[n] < gamma and slot[n] >= 0
+    kept = [n for n in accepted if ran(n)]
+    assert kept == list(accepted[:len(kept)])
     for i, n in enumerate(kept):
-        src, dst = base + n, base + i
+        src, dst = base + slot[n], base + i
         assert src >= dst
         if src != dst:
             cache[:, :, :, dst, :] = cache[:, :, :, src, :]
-    pend = [draft.tok[n] for n in accepted if draft.depth[n] >= gamma] + [bonus_tok]
+    pend = [draft.tok[n] for n in accepted if not ran(n)] + [bonus_tok]
     return base + len(kept), pend

@@ -482,3 +482,78 @@ def test_spd_first_token_frequencies_follow_the_target():
         counts[r.out_tok[0]] += 1
     chi2 = float(np.sum((counts - n * p[()]) ** 2 / (n * p[()])))
     assert chi2 < 24.3          # 99.9 % quantile of chi-square with 7 degrees of freedom
+
+
+def test_draft_beam_keep_all_candidates():
+    """The wider tree (every layer records b * b candidates) contains the paper's tree: its kept beams are the same
+    nodes with the same likelihoods and the same x**; the extra candidates are leaves without a cache row whose
+    joint log q is the parent's plus the auxiliary log-probability of their token, and a beam's children come in
+    decreasing order of perturbed score."""
+    from oracle.adapters import oracle_model
+    shape = S.WORKLOADS["tiny"].aux
+    model = oracle_model(S.make_model(shape, 1))
+    gamma, b, L, cap = 3, 3, 0, 48
+    pend = S.token_ids(0, 51, 4, shape.vocab).tolist()
+    u = S.uniforms(0, 52, gamma * b * shape.vocab).view(gamma, b, shape.vocab).numpy()
+    mk = lambda: np.zeros((shape.layers, 2, shape.n_kv_heads, cap, shape.head_dim), dtype=np.uint16)
+    base = O.draft_beam(model, mk(), L, pend, gamma, b, u)
+    wide = O.draft_beam(model, mk(), L, pend, gamma, b, u, keep_all=True)
+    assert len(wide.tok) == gamma * b * b and wide.depth == sum(([s + 1] * (b * b) for s in range(gamma)), [])
+    kept = [n for n in range(len(wide.tok)) if wide.slot[n] >= 0]
+    assert len(kept) == gamma * b and sorted(wide.slot[n] for n in kept) == list(range(gamma * b))
+    by_slot = {wide.slot[n]: n for n in kept}
+    for k in range(gamma * b):                      # beam k of the plain tree == the kept node with slot k
+        n = by_slot[k]
+        assert wide.tok[n] == base.tok[k] and abs(wide.logq[n] - base.logq[k]) < 1e-12
+        assert (wide.parent[n] == -1) == (base.parent[k] == -1)
+        if base.parent[k] >= 0:
+            assert wide.slot[wide.parent[n]] == base.parent[k]
+    assert [wide.slot[n] for n in wide.best_path] == base.best_path and np.allclose(wide.logq_ref, base.logq_ref)
+    # leaves: never parents, no cache row; parents are kept nodes of the layer before
+    for n in range(len(wide.tok)):
+        p = wide.parent[n]
+        assert p < n and (p == -1 or (wide.slot[p] >= 0 and wide.depth[p] == wide.depth[n] - 1))
+    # children of one beam: distinct tokens, and log q(child) - log q(parent) is the aux log-softmax of the token after
+    # the parent's path (causal decoding from scratch)
+    n = max(i for i in range(len(wide.tok)) if wide.slot[i] < 0)          # a leaf of the last layer
+    path = []
+    c = n
+    while c >= 0:
+        path.append(c); c = wide.parent[c]
+    path.reverse()
+    seq = pend + [wide.tok[i] for i in path]
+    c2 = mk()
+    for i, t in enumerate(seq[:-1]):
+        lg = O.decoder_rows(model, c2, i, [t], [i], [i], [[i]])
+    want = O.log_softmax(lg)[0, seq[-1]]
+    parent_lq = wide.logq[wide.parent[n]] if wide.parent[n] >= 0 else 0.0
+    assert abs((wide.logq[n] - parent_lq) - want) < 1e-10
+    sib = [i for i in range(len(wide.tok)) if wide.parent[i] == wide.parent[n] and wide.depth[i] == wide.depth[n]]
+    assert len({wide.tok[i] for i in sib}) == len(sib) == b
+
+
+def test_aux_commit_with_an_accepted_leaf():
+    """A recorded candidate that was not kept as a beam has no row in the auxiliary cache: when the verification
+    accepts it (as the last node of the path) it must wait, like a node of the last layer, to be replayed."""
+    from oracle.adapters import oracle_model
+    shape = S.WORKLOADS["tiny"].aux
+    model = oracle_model(S.make_model(shape, 1))
+    gamma, b, cap = 3, 2, 64
+    cache = np.zeros((shape.layers, 2, shape.n_kv_heads, cap, shape.head_dim), dtype=np.uint16)
+    ctx = S.token_ids(0, 61, 5, shape.vocab).tolist()
+    for i, t in enumerate(ctx[:-1]):
+        O.decoder_rows(model, cache, i, [t], [i], [i], [[i]])
+    L, pend = len(ctx) - 1, [ctx[-1]]
+    u = S.uniforms(0, 62, gamma * b * shape.vocab).view(gamma, b, shape.vocab).numpy()
+    dr = O.draft_beam(model, cache, L, pend, gamma, b, u, keep_all=True)
+    leaf = next(n for n in range(len(dr.tok)) if dr.slot[n] < 0 and dr.depth[n] == 2)
+    accepted = [dr.parent[leaf], leaf]
+    L2, pend2 = O.aux_commit(cache, L, pend, dr, accepted, 9, gamma)
+    committed = ctx + [dr.tok[n] for n in accepted] + [9]
+    assert committed[L2:] == pend2 and pend2 == [dr.tok[leaf], 9] and L2 == L + 1 + 1
+    vis = [[L2 + i for i in range(r + 1)] for r in range(len(pend2))]
+    got = O.decoder_rows(model, cache, L2, pend2, [L2 + i for i in range(2)], [L2 + i for i in range(2)], vis)[-1]
+    c2 = np.zeros_like(cache)
+    for i, t in enumerate(committed):
+        want = O.decoder_rows(model, c2, i, [t], [i], [i], [[i]])[0]
+    assert np.max(np.abs(got - want)) < 1e-9
