@@ -35,10 +35,13 @@ struct Region {                 // one array of the workspace: where it starts a
 // One GEMM launch of the tensor-core forward, and the plan of a whole forward: everything about the launches that
 // depends only on (model, sequences per call, rows per sequence, LM-head mode).  Plans are built once per shape and
 // kept in the context; a call patches in what changes from call to call (status words, uniforms, debug fields).
-struct GemmDesc { TcMaps mp; TcGemmParams p; double bytes; bool cluster; };
+struct GemmDesc { TcMaps mp; TcGemmParams p; double bytes; bool cluster; bool attn_before; };
 struct ForwardPlan {
-    std::vector<GemmDesc> g;           // per layer: QKV, O, gate/up, down; then the LM head
+    std::vector<GemmDesc> g;           // per layer: QKV (or Q, then K/V), O (the attention pass runs before it),
+                                       // gate/up, down; then the LM head
     int lm_tiles128 = 0;
+    bool split_kv = false;             // K and V have a launch of their own, fed by sc.xkv with kv_terms terms
+    int kv_terms = 0;
     bool maps = false;                 // tensor maps encoded (false: decomposition only, for the extent audit)
 };
 
@@ -209,6 +212,7 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     sc.xd = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * d, "xd");
     sc.xa = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * qd, "xa");
     sc.xf = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * F, "xf");
+    sc.xkv = k.take<__nv_bfloat16>((size_t)2 * TC_X_ROWS * d, "xkv");
     const size_t dt = (d + TC_TILE_N - 1) / TC_TILE_N;
     sc.sumsq_a = k.take<float>(dt * TC_X_ROWS, "sumsq_a");
     sc.sumsq_b = k.take<float>(dt * TC_X_ROWS, "sumsq_b");
@@ -389,30 +393,33 @@ void build_kv_map(ModelView& m) {
 // Builds the plan.  with_maps = false leaves out everything that needs the driver (the operand-row tensor maps) and
 // the weight maps: what is left is the index arithmetic of the launches.
 int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const ModelView& m, const WeightMaps* wm, int B,
-               int R, bool lm_plain, bool with_maps) {
+               int R, bool lm_plain, bool with_maps, bool split_kv_ok) {
     const int T = B * R;
     const mtad_model_desc& d = m.d;
     const int qd = d.n_q_heads * d.head_dim, kvd = d.n_kv_heads * d.head_dim;
     const int rpad = (T + 15) / 16 * 16;
     const int dt = (d.d_model + TC_TILE_N - 1) / TC_TILE_N;
     const int mh = tc_halves(T);                          // weight halves per tile, as many as tensor memory allows
-    int mq = mh;                                          // QKV tiles must not straddle q | k | v
-    while (mq > 1 && (qd % (128 * mq) || kvd % (128 * mq) || mq * tc_qkv_terms(T) * rpad > 512)) mq /= 2;
     auto ix = [](int halves) { return halves == 1 ? 0 : (halves == 2 ? 1 : 2); };
     auto up = [](int a, int b) { return (a + b - 1) / b; };
-    // Operand rows: `terms` bf16 terms per activation row in general, `tq` for the rows that feed the Q/K/V
-    // projection and the LM head (written by the row preparation and by the down projection).  One TMA box covers
-    // all terms * rpad interleaved rows, or they are cut into two or three boxes of at most 256 rows.
-    const int terms = tc_terms(T), tq = tc_qkv_terms(T);
-    const int xbox = terms * rpad / tc_boxes(terms * rpad), qbox = tq * rpad / tc_boxes(tq * rpad);
-    CUtensorMap xd{}, xq{}, xa{}, xf{};
+    // Operand rows: `terms` bf16 terms per activation row.  One TMA box covers all terms * rpad interleaved rows, or
+    // they are cut into two or three boxes of at most 256 rows.
+    // From width 8192 on the K/V rounding decides the accuracy of the whole step (a bf16 element that rounds the
+    // other way shifts attention scores that are sharply peaked at that width).  There, with more than 32 rows (up to
+    // 32 every row has three terms anyway), the K and V rows get a launch of their own: its input rows carry three
+    // terms (a second copy written by the row preparation and the down projection) and its tensor-memory accumulation
+    // runs in short chains (tc_gemm.cu), which holds the relative error near 5e-7; Q, which is never rounded to
+    // bf16, keeps two terms and whole runs (about 2.5e-6) like every other projection.
+    const int terms = tc_terms(T), tkv = tc_qkv_terms(T);
+    const bool split_kv = split_kv_ok && d.d_model >= 8192 && T > 32 && tkv > terms;
+    int mq = mh;                                          // QKV tiles must not straddle q | k | v
+    while (mq > 1 && (qd % (128 * mq) || (!split_kv && kvd % (128 * mq)))) mq /= 2;
+    const int xbox = terms * rpad / tc_boxes(terms * rpad), kvbox = tkv * rpad / tc_boxes(tkv * rpad);
+    CUtensorMap xd{}, xkv{}, xa{}, xf{};
     if (with_maps &&
-        (tc_make_map(&xd, sc.xd, 2 * TC_X_ROWS, d.d_model, xbox) || tc_make_map(&xq, sc.xd, 2 * TC_X_ROWS, d.d_model, qbox) ||
+        (tc_make_map(&xd, sc.xd, 2 * TC_X_ROWS, d.d_model, xbox) || tc_make_map(&xkv, sc.xkv, 2 * TC_X_ROWS, d.d_model, kvbox) ||
          tc_make_map(&xa, sc.xa, 2 * TC_X_ROWS, qd, xbox) || tc_make_map(&xf, sc.xf, 2 * TC_X_ROWS, d.d_ffn, xbox)))
         return MTAD_E_CUDA;
-    // weight halves per tile of the launches that read tq terms: their accumulators must fit tensor memory too
-    int mhq = mh;
-    while (mhq > 1 && mhq * tq * rpad > 512) mhq /= 2;
     TcGemmParams base{};
     base.ws = sc.tc_ws; base.counters = sc.tc_counters;
     base.inv_dim = 1.f / (float)d.d_model; base.eps = d.rms_eps;
@@ -441,18 +448,29 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
         return with_maps ? v[ix(halves)][l] : none;
     };
     for (int l = 0; l < d.layers; ++l) {
-        {   // QKV + rotary + append
+        {   // QKV + rotary + append (Q alone when K and V have their own launch)
             TcGemmParams p = base; TcMaps mp{};
             const int qt = up(qd, 128), kt = up(kvd, 128);
-            tc_decompose(p, (qt + 2 * kt) / mq, d.d_model, T, kCtas, 0, tq);
-            p.mh = mq; p.n_rows_total = (qt + 2 * kt) * 128;
-            p.seg_cap = kQkvSegCap;
+            const int n128 = split_kv ? qt : qt + 2 * kt;
+            tc_decompose(p, n128 / mq, d.d_model, T, kCtas);
+            p.mh = mq; p.n_rows_total = n128 * 128;
             p.mode = TC_QKV; p.N = qd; p.seg_k_tile = qt; p.seg_v_tile = qt + kt; p.layer = l;
             p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = (l == 0) ? 1 : dt;
             if (with_maps) { mp.a0 = wmap(wm->wq, mq, l); mp.a1 = wmap(wm->wk, mq, l); mp.a2 = wmap(wm->wv, mq, l); }
-            mp.x = xq;
-            const bool cl = mq == 1 && clusterize(p, qt + 2 * kt, d.d_model, true);
-            g.push_back({mp, p, wb * (qd + 2.0 * kvd) * d.d_model, cl});
+            mp.x = xd;
+            const bool cl = mq == 1 && clusterize(p, n128, d.d_model, true);
+            g.push_back({mp, p, wb * (qd + (split_kv ? 0.0 : 2.0 * kvd)) * d.d_model, cl, false});
+        }
+        if (split_kv) {   // K and V rows: three-term input, short accumulation chains
+            TcGemmParams p = base; TcMaps mp{};
+            const int kt = up(kvd, 128);
+            tc_decompose(p, 2 * kt, d.d_model, T, kCtas, 0, tkv);
+            p.mh = 1; p.n_rows_total = 2 * kt * 128; p.seg_cap = kQkvSegCap;
+            p.mode = TC_QKV; p.N = qd; p.seg_k_tile = 0; p.seg_v_tile = kt; p.layer = l;
+            p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = (l == 0) ? 1 : dt;
+            if (with_maps) { mp.a0 = wmap(wm->wk, 1, l); mp.a1 = wmap(wm->wk, 1, l); mp.a2 = wmap(wm->wv, 1, l); }
+            mp.x = xkv;
+            g.push_back({mp, p, wb * 2.0 * kvd * d.d_model, false, false});
         }
         {   // O projection + residual, emits the FFN norm's operand rows
             TcGemmParams p = base; TcMaps mp{};
@@ -464,7 +482,7 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
             if (with_maps) mp.a0 = wmap(wm->wo, mh, l);
             mp.x = xa;
             const bool cl = clusterize(p, up(d.d_model, 128), qd, true);
-            g.push_back({mp, p, wb * d.d_model * qd, cl});
+            g.push_back({mp, p, wb * d.d_model * qd, cl, true});
         }
         {   // gate / up + SwiGLU
             TcGemmParams p = base; TcMaps mp{};
@@ -474,7 +492,7 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
             p.x_out = sc.xf; p.xk = d.d_ffn;
             if (with_maps) { mp.a0 = wmap(wm->gate, mh, l); mp.a1 = wmap(wm->up, mh, l); }
             mp.x = xd;
-            g.push_back({mp, p, wb * 2.0 * d.d_ffn * d.d_model, false});
+            g.push_back({mp, p, wb * 2.0 * d.d_ffn * d.d_model, false, false});
         }
         {   // down projection + residual, emits the next norm's operand rows
             TcGemmParams p = base; TcMaps mp{};
@@ -482,27 +500,30 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
             p.mh = mh; p.n_rows_total = d.d_model;
             p.mode = TC_RESID; p.N = d.d_model; p.sumsq_in_parts = 0;
             p.gain = (l + 1 < d.layers) ? m.w(l + 1, 0) : static_cast<const __nv_bfloat16*>(d.final_norm);
-            p.x_out = sc.xd; p.xk = d.d_model; p.sumsq_out = sc.sumsq_a; p.out_terms = tq;
+            p.x_out = sc.xd; p.xk = d.d_model; p.sumsq_out = sc.sumsq_a;
+            if (split_kv && l + 1 < d.layers) { p.x_out2 = sc.xkv; p.out_terms2 = tkv; }
             if (with_maps) mp.a0 = wmap(wm->down, mh, l);
             mp.x = xf;
             const bool cl = clusterize(p, up(d.d_model, 128), d.d_ffn, true);
-            g.push_back({mp, p, wb * d.d_model * d.d_ffn, cl});
+            g.push_back({mp, p, wb * d.d_model * d.d_ffn, cl, false});
         }
     }
     {   // LM head: per-tile log-softmax / Gumbel-argmax partials + gather of the drafted tokens' logits, or plain
         // logits for the draft's beam selection and the warped rows
         TcGemmParams p = base; TcMaps mp{};
-        tc_decompose(p, up(d.vocab, 128 * mhq), d.d_model, T, kCtas, 0, tq);
-        p.mh = mhq; p.n_rows_total = d.vocab; p.n_tiles128 = up(d.vocab, 128);
+        tc_decompose(p, up(d.vocab, 128 * mh), d.d_model, T, kCtas);
+        p.mh = mh; p.n_rows_total = d.vocab; p.n_tiles128 = up(d.vocab, 128);
         p.mode = lm_plain ? TC_PLAIN : TC_LMHEAD; p.N = d.vocab; p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = dt;
         p.out = sc.logits; p.ldo = d.vocab;
-        if (with_maps) mp.a0 = wm->lm_head[ix(mhq)];
-        mp.x = xq;
+        if (with_maps) mp.a0 = wm->lm_head[ix(mh)];
+        mp.x = xd;
         fp.lm_tiles128 = p.n_tiles128;
         const bool cl = clusterize(p, up(d.vocab, 128), d.d_model, true);
-        g.push_back({mp, p, wb * d.vocab * d.d_model, cl});
+        g.push_back({mp, p, wb * d.vocab * d.d_model, cl, false});
     }
     fp.maps = with_maps;
+    fp.split_kv = split_kv;
+    fp.kv_terms = tkv;
     return MTAD_OK;
 }
 
@@ -527,7 +548,7 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
     auto it = ctx->plans.find(key);
     if (it == ctx->plans.end()) {
         ForwardPlan fp;
-        if (int rc = build_plan(fp, sc, ctx->rm, m, &wm, B, R, lm_plain, true)) return rc;
+        if (int rc = build_plan(fp, sc, ctx->rm, m, &wm, B, R, lm_plain, true, &m == &ctx->target)) return rc;
         it = ctx->plans.emplace(key, std::move(fp)).first;
     }
     ForwardPlan& fp = it->second;
@@ -545,21 +566,23 @@ int forward_rows_tc(mtad_ctx* ctx, const ModelView& m, const WeightMaps& wm, int
         else RUN(MTAD_K_GEMM, gd.bytes, 1, launch_tc_gemm(gd.mp, p, kCtas, pdl, s));
         return MTAD_OK;
     };
-    if (int rc = launch(0)) return rc;                          // QKV of layer 0
-    for (int l = 0; l < d.layers; ++l) {
-        if (mma_attention(m)) {
-            const AttnSplit as = attn_split(m, B, R, total);
-            RUN(MTAD_K_ATTN, 0, 2, launch_attention_mma(m, l, ctx->rm, sc, B, R, as.ns, as.nsp, status, pdl, s));
-            RUN(MTAD_K_ATTN, 0, 0, launch_attention_combine(m, ctx->rm, sc, B, R, as.ns, true, pdl, s));
-        } else {
-            int nsplit = (int)std::min<long long>(attn_split_cap(d.n_q_heads), (total + MTAD_ATTN_TILE - 1) / MTAD_ATTN_TILE);
-            nsplit = std::max(1, std::min(nsplit, (4 * 148 + d.n_q_heads * B - 1) / (d.n_q_heads * B)));
-            long long chunk = (total + nsplit - 1) / nsplit;
-            chunk = (chunk + MTAD_ATTN_TILE - 1) / MTAD_ATTN_TILE * MTAD_ATTN_TILE;
-            RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, true, pdl, s));
+    int layer = 0;
+    for (size_t i = 0; i < fp.g.size(); ++i) {
+        if (fp.g[i].attn_before) {                               // the O projection: the attention pass feeds it
+            const int l = layer++;
+            if (mma_attention(m)) {
+                const AttnSplit as = attn_split(m, B, R, total);
+                RUN(MTAD_K_ATTN, 0, 2, launch_attention_mma(m, l, ctx->rm, sc, B, R, as.ns, as.nsp, status, pdl, s));
+                RUN(MTAD_K_ATTN, 0, 0, launch_attention_combine(m, ctx->rm, sc, B, R, as.ns, true, pdl, s));
+            } else {
+                int nsplit = (int)std::min<long long>(attn_split_cap(d.n_q_heads), (total + MTAD_ATTN_TILE - 1) / MTAD_ATTN_TILE);
+                nsplit = std::max(1, std::min(nsplit, (4 * 148 + d.n_q_heads * B - 1) / (d.n_q_heads * B)));
+                long long chunk = (total + nsplit - 1) / nsplit;
+                chunk = (chunk + MTAD_ATTN_TILE - 1) / MTAD_ATTN_TILE * MTAD_ATTN_TILE;
+                RUN(MTAD_K_ATTN, 0, 2, launch_attention(m, l, ctx->rm, sc, B, R, nsplit, (int)chunk, true, pdl, s));
+            }
         }
-        for (int k = 0; k < 4; ++k)                              // O, gate/up, down of this layer, then what follows
-            if (int rc = launch((size_t)l * 4 + 1 + k)) return rc;
+        if (int rc = launch(i)) return rc;
     }
     if (!lm_plain) RUN(MTAD_K_LMRED, 0, 2, launch_lm_merge(m, ctx->rm, sc, B, R, fp.lm_tiles128, uniforms, status, s));
     return MTAD_OK;
@@ -605,7 +628,10 @@ int verify_common(mtad_ctx* ctx, int B, const int32_t* seqs, const int32_t* n_no
     pa.B = B; pa.R = R; pa.max_depth = D; pa.n_nodes = n_nodes; pa.tok = tok; pa.parent = parent;
     const bool tc = ctx->use_tc && ctx->tmaps.ok && B * R <= TC_MAX_ROWS;
     if (tc) {
-        pa.gain0 = ctx->target.w(0, 0); pa.x = ctx->sc.xd; pa.terms = tc_qkv_terms(B * R);
+        pa.gain0 = ctx->target.w(0, 0); pa.x = ctx->sc.xd; pa.terms = tc_terms(B * R);
+        if (ctx->target.d.d_model >= 8192 && B * R > 32 && tc_qkv_terms(B * R) > pa.terms) {
+            pa.x2 = ctx->sc.xkv; pa.terms2 = tc_qkv_terms(B * R);     // rows of the separate K/V launch (build_plan)
+        }
         pa.sumsq_out = ctx->sc.sumsq_a;
     }
     RUN(MTAD_K_PREPARE, 0, 1, launch_prepare(ctx->target, ctx->st, ctx->rm, ctx->sc, pa, out->status, s));
@@ -988,11 +1014,11 @@ void audit_forward(Audit& au, const mtad_ctx& c, const ModelView& m, int B, int 
     for (const char* n : {"rm_n_rows", "rm_n_spec", "rm_kv_base", "rm_call_seq"}) au.ws(n, B);
     au.ws("hidden", (size_t)T * d.d_model);
     au.ws("rope", ((size_t)(T - 1) * (hd / 2) + (hd / 2 - 1)) * 2 + 2);
-    const int tq = tc_qkv_terms(T);
-    au.ws("xd", idx_xrow(T - 1, tq, tq - 1, d.d_model, d.d_model - 1) + 1);
+    au.ws("xd", idx_xrow(T - 1, terms, terms - 1, d.d_model, d.d_model - 1) + 1);
     au.ws("sumsq_a", T);
     ForwardPlan fp;
-    build_plan(fp, c.sc, c.rm, m, nullptr, B, R, lm_plain, false);
+    build_plan(fp, c.sc, c.rm, m, nullptr, B, R, lm_plain, false, &m == &c.target);
+    if (fp.split_kv) au.ws("xkv", idx_xrow(T - 1, fp.kv_terms, fp.kv_terms - 1, d.d_model, d.d_model - 1) + 1);
     const long long cap = d.kv_capacity;
     const long long slot_max = std::min<long long>(len_ub + R - 1, cap - 1);     // prepare refuses rows past the capacity
     const size_t cache_elems = (size_t)d.layers * m.max_batch * 2 * Hkv * cap * hd;

@@ -114,6 +114,7 @@ struct Scratch {
     __nv_bfloat16* xd;   // [512, d]     input of QKV / gate-up / LM head (un-normalised hidden * gain)
     __nv_bfloat16* xa;   // [512, Hq hd] attention output
     __nv_bfloat16* xf;   // [512, F]     SwiGLU output
+    __nv_bfloat16* xkv;  // [512, d]     input of a separate K/V projection (three terms), see build_plan
     float* sumsq_a;      // [tiles(d)][256] sums of squares of the hidden rows (after down proj / embedding)
     float* sumsq_b;      // [tiles(d)][256] the same after the O projection
     float* tc_ws;        // split-K partial tiles
@@ -289,6 +290,8 @@ struct PrepareArgs {
     const __nv_bfloat16* gain0;
     __nv_bfloat16* x;
     int terms;
+    __nv_bfloat16* x2;         // second copy of the operand rows with terms2 terms, or null
+    int terms2;
     float* sumsq_out;
 };
 

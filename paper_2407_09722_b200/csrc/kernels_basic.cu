@@ -139,8 +139,12 @@ __global__ void prepare_kernel(const __nv_bfloat16* __restrict__ embed, int d, i
                          a.x ? a.x + (size_t)t * a.terms * d : nullptr, a.terms);
     if (a.x) {
         __shared__ float red[32];
-        ss = block_sum(ss, red);
+        ss = block_sum(ss, red);                     // (also orders the hidden row's stores before the loop below)
         if (threadIdx.x == 0) a.sumsq_out[t] = ss;
+        if (a.x2)
+            for (int i = threadIdx.x; i < d; i += blockDim.x)
+                store_terms(hidden[(size_t)t * d + i] * __bfloat162float(a.gain0[i]),
+                            a.x2 + (size_t)t * a.terms2 * d + i, d, a.terms2);
     }
     // rotary table: angle = pos * base^(-2i/hd)
     for (int i = threadIdx.x; i < hd / 2; i += blockDim.x) {

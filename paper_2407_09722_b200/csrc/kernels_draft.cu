@@ -126,7 +126,7 @@ cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const Dr
                       rope_inv((double)m.d.rope_base, m.d.head_dim), (long long)m.d.kv_capacity, s, ds, rm, sc.hidden,
                       sc.rope, seqs, R, step, beam,
                       tc ? m.w(0, 0) : (const __nv_bfloat16*)nullptr, tc ? sc.xd : (__nv_bfloat16*)nullptr,
-                      tc_qkv_terms(B * R), sc.sumsq_a);
+                      tc_terms(B * R), sc.sumsq_a);
 }
 
 // ---------------------------------------------------------------------------------------------------------------

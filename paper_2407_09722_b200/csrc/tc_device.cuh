@@ -302,6 +302,7 @@ __device__ __forceinline__ void epi_resid(const TcGemmParams& p, float* red, Epi
             y[j] += epi[j][e];
             p.hidden[(size_t)t * p.N + n] = y[j];
             store_terms(y[j] * g, p.x_out + (size_t)t * p.out_terms * p.xk + n, p.xk, p.out_terms);
+            if (p.x_out2) store_terms(y[j] * g, p.x_out2 + (size_t)t * p.out_terms2 * p.xk + n, p.xk, p.out_terms2);
         }
         y[j] *= y[j];
     }

@@ -21,6 +21,7 @@
 #include <math_constants.h>
 
 #include <algorithm>
+#include <type_traits>
 #include <stdlib.h>
 
 #include "tc_device.cuh"
@@ -185,7 +186,9 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
                 int i = 0;
                 while (i < n_units && ok) {
                     const int kb0 = (first + i) % KB;
-                    const int len = min(min(KB - kb0, n_units - i), p.seg_cap);
+                    // (only tiles of the K and V rows are accumulated in capped pieces: Q is never rounded to bf16)
+                    const int cap = ((first + i) / KB) * mh < p.seg_k_tile ? (1 << 20) : p.seg_cap;
+                    const int len = min(min(KB - kb0, n_units - i), cap);
                     const int buf = seg % nbuf;
                     const uint32_t aph = (uint32_t)(seg / nbuf) & 1u;
                     ok = mbar_wait(smem_u32(&s.tempty[buf]), aph ^ 1u, abort_flag);
@@ -257,11 +260,11 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
             while (i < n_units) {
                 const int u = first + i;
                 const int tile = u / KB, kb0 = u % KB;
-                // A run of this CTA inside one tile is accumulated in pieces of at most seg_cap k-blocks: the tensor
-                // cores truncate every partial sum, so a long chain drifts (about -6e-8 relative per k-block); the
-                // pieces are added up in fp32 in this CTA's partial tile
+                // A run of this CTA inside one tile of K or V rows is accumulated in pieces of at most seg_cap k-blocks:
+                // the tensor cores truncate every partial sum, so a long chain drifts (about -6e-8 relative per
+                // k-block); the pieces are added up in fp32 in this CTA's partial tile
                 const int len_all = min(KB - kb0, n_units - i);
-                const int len = min(len_all, p.seg_cap);
+                const int len = min(len_all, tile * mh < p.seg_k_tile ? (1 << 20) : p.seg_cap);
                 const bool first_piece = (i == 0 || kb0 == 0), last_piece = (len == len_all);
                 const int buf = seg % nbuf;
                 const uint32_t aph = (uint32_t)(seg / nbuf) & 1u;
@@ -278,40 +281,47 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
                 const int n_contrib = c_last - c_first + 1;
                 const int slot_idx = (int)blockIdx.x - c_first;
                 float* part = p.ws + idx_tc_ws(tile, p.max_contrib, slot_idx, part_floats);
-                for (int h = 0; h < mh; ++h) {
-                    const uint32_t t_acc = tmem_base + ((uint32_t)(quad * 32) << 16) +
-                                           (uint32_t)(buf * mh * acc_cols + h * acc_cols);
-                    float* dst = part + h * half_floats + feat;
-                    if (terms == 3) {
-                        for (int rb = 0; rb < T; rb += 16) {           // 16 rows = 48 accumulator columns
-                            float v[48];
-                            tc_ld16(t_acc + 3 * rb, v);
-                            tc_ld16(t_acc + 3 * rb + 16, v + 16);
-                            tc_ld16(t_acc + 3 * rb + 32, v + 32);
+                // (two copies of the loops, chosen once per piece: a per-element choice between storing and adding
+                // would make every store wait for a load)
+                auto drain = [&](auto accumulate) {
+                    constexpr bool ADD = decltype(accumulate)::value;
+                    for (int h = 0; h < mh; ++h) {
+                        const uint32_t t_acc = tmem_base + ((uint32_t)(quad * 32) << 16) +
+                                               (uint32_t)(buf * mh * acc_cols + h * acc_cols);
+                        float* dst = part + h * half_floats + feat;
+                        if (terms == 3) {
+                            for (int rb = 0; rb < T; rb += 16) {           // 16 rows = 48 accumulator columns
+                                float v[48];
+                                tc_ld16(t_acc + 3 * rb, v);
+                                tc_ld16(t_acc + 3 * rb + 16, v + 16);
+                                tc_ld16(t_acc + 3 * rb + 32, v + 32);
 #pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (rb + j < T) {
-                                    const float y = v[3 * j] + (v[3 * j + 1] + v[3 * j + 2]);
-                                    float* q = dst + (size_t)(rb + j) * TC_TILE_N;
-                                    *q = first_piece ? y : *q + y;
-                                }
-                        }
-                    } else {
-                        for (int c0 = 0; c0 < 2 * T; c0 += 16) {
-                            float v[16];
-                            tc_ld16(t_acc + c0, v);
+                                for (int j = 0; j < 16; ++j)
+                                    if (rb + j < T) {
+                                        const float y = v[3 * j] + (v[3 * j + 1] + v[3 * j + 2]);
+                                        float* q = dst + (size_t)(rb + j) * TC_TILE_N;
+                                        if (ADD) *q += y; else *q = y;
+                                    }
+                            }
+                        } else {
+                            for (int c0 = 0; c0 < 2 * T; c0 += 16) {
+                                float v[16];
+                                tc_ld16(t_acc + c0, v);
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                const int r = (c0 >> 1) + j;
-                                if (r < T) {
-                                    const float y = v[2 * j] + v[2 * j + 1];
-                                    float* q = dst + (size_t)r * TC_TILE_N;
-                                    *q = first_piece ? y : *q + y;
+                                for (int j = 0; j < 8; ++j) {
+                                    const int r = (c0 >> 1) + j;
+                                    if (r < T) {
+                                        const float y = v[2 * j] + v[2 * j + 1];
+                                        float* q = dst + (size_t)r * TC_TILE_N;
+                                        if (ADD) *q += y; else *q = y;
+                                    }
                                 }
                             }
                         }
                     }
-                }
+                };
+                if (first_piece) drain(std::false_type{});
+                else drain(std::true_type{});
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&s.tempty[buf]));   // MMA may reuse this accumulator

@@ -75,6 +75,8 @@ struct TcGemmParams {
     float* hidden;                  // [T, N]
     const __nv_bfloat16* gain;      // [N] gains of the norm that follows (TC_RESID)
     __nv_bfloat16* x_out;           // operand rows for the next GEMM (layout of store_terms)
+    __nv_bfloat16* x_out2;          // TC_RESID: a second copy with out_terms2 terms (rows of the K/V projection), or null
+    int out_terms2;
     int xk;                         // their row length: the next GEMM's K
     float* sumsq_out;               // [n_tiles][TC_X_ROWS]
     // TC_LMHEAD
