@@ -232,14 +232,21 @@ DRAFT_BEAM = 4          # the paper's smaller beam width
 
 
 def draft_loop(w: S.Workload, steps: int, warmup: int, cap: int):
-    """Decode iterations in which the auxiliary model drafts (beam sampling, the best beam is the chain), the target
-    verifies that chain and both caches are rolled forward.  Returns tokens/s including the draft and the draft's
-    share; a reported extra, not the headline (the headline times the verification path on synthetic drafts)."""
+    """Decode iterations in which the auxiliary model drafts by beam sampling, the target verifies and both caches are
+    rolled forward.  Chain workloads verify the best beam (Algorithm 1); tree workloads keep every candidate of the
+    beam sampling (beam * beam nodes a layer, the workload's tree size) and verify that tree as mtad_draft left it on
+    the device (Sec. 3.3).  Returns tokens/s including the draft and the draft's share; a reported extra, not the
+    headline (the headline times the verification path on synthetic drafts)."""
     import paper_2407_09722_b200 as M
     from paper_2407_09722_b200.runtime import DeviceModel
     lens = S.kv_lengths(w, SEED)
-    g, b, B, V = w.gamma, DRAFT_BEAM, w.batch, w.target.vocab
-    dm = DeviceModel(w.target, B, max(w.n_nodes, g * b), cap, SEED, aux=w.aux, aux_capacity=cap + g * b + 8)
+    tree = w.kind == "tree"
+    g, B, V = w.gamma, w.batch, w.target.vocab
+    b = DRAFT_BEAM
+    if tree:                                   # the beam width whose candidates fill the workload's tree
+        b = max(1, int(round(math.sqrt(w.n_nodes / g))))
+    N = g * b * b if tree else g * b
+    dm = DeviceModel(w.target, B, max(w.n_nodes, N), cap, SEED, aux=w.aux, aux_capacity=cap + g * b + 8)
     ctx = dm.ctx
     seqs = list(range(B))
     for s_, L in enumerate(lens):
@@ -248,23 +255,28 @@ def draft_loop(w: S.Workload, steps: int, warmup: int, cap: int):
         ctx.mtad_seq_set(s_, L, 1, aux_len=L)
     i32 = dict(dtype=torch.int32, device="cuda")
     f32 = dict(dtype=torch.float32, device="cuda")
-    tok, parent, depth = (torch.zeros(B, g * b, **i32) for _ in range(3))
-    node_logq, logq_ref, best = torch.zeros(B, g * b, **f32), torch.zeros(B, g, **f32), torch.zeros(B, g, **i32)
+    tok, parent, depth = (torch.zeros(B, N, **i32) for _ in range(3))
+    node_logq, logq_ref, best = torch.zeros(B, N, **f32), torch.zeros(B, g, **f32), torch.zeros(B, g, **i32)
+    n_nodes = torch.zeros(B, **i32)
     n_u = 4
     u_draft = [S.uniforms(SEED, (41 << 40) | i, B * g * b * V, "cuda").view(B, g, b, V) for i in range(n_u)]
     u_bonus = [S.bonus_uniforms(SEED, 1000 + i, B, V, "cuda") for i in range(n_u)]
-    res = M.ResultBuffers(B, g, g)
+    res = M.ResultBuffers(B, N, g) if tree else M.ResultBuffers(B, g, g)
     acc = torch.zeros((), dtype=torch.int64, device="cuda")
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
     log_tau = math.log(TAU)
     for i in range(-warmup, steps):
         if i >= 0:
             ev[i][0].record()
-        ctx.mtad_draft(seqs, g, b, u_draft[i % n_u], tok, parent, depth, node_logq, logq_ref, best)
+        ctx.mtad_draft(seqs, g, b, u_draft[i % n_u], tok, parent, depth, node_logq, logq_ref, best,
+                       keep_all_candidates=tree, n_nodes=n_nodes)
         if i >= 0:
             ev[i][1].record()
-        chain_tok = tok.gather(1, best.long())              # tokens of the best beam, in depth order
-        ctx.mtad_verify_chain(seqs, g, chain_tok, logq_ref, log_tau, u_bonus[i % n_u], res)
+        if tree:
+            ctx.mtad_verify_tree(seqs, n_nodes, N, g, tok, parent, logq_ref, log_tau, u_bonus[i % n_u], res)
+        else:
+            chain_tok = tok.gather(1, best.long())              # tokens of the best beam, in depth order
+            ctx.mtad_verify_chain(seqs, g, chain_tok, logq_ref, log_tau, u_bonus[i % n_u], res)
         ctx.kv_commit(seqs, res)
         if i >= 0:
             acc += res.n_out.sum()
@@ -278,6 +290,7 @@ def draft_loop(w: S.Workload, steps: int, warmup: int, cap: int):
     total_ms = ev[0][0].elapsed_time(ev[-1][2])
     accepted = float(acc.item())
     return {"value": accepted / (total_ms * 1e-3), "unit": "tokens/s", "steps": steps, "gamma": g, "beam": b,
+            "nodes": N, "verified_as": "tree" if tree else "chain",
             "block_efficiency": accepted / (steps * B), "iteration_ms": total_ms / steps,
             "draft_us_median": statistics.median(d_us), "verify_commit_us_median": 1e3 * statistics.median(it_ms)
             - statistics.median(d_us), "device_status": status}
@@ -608,13 +621,19 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
     }
     del dm, ctx
     torch.cuda.empty_cache()
-    if world == 1 and chain and not args.no_draft_loop:
+    if world == 1 and not args.no_draft_loop:
         line["draft_loop"] = draft_loop(w, min(args.steps, 32), 3, cap)
         torch.cuda.empty_cache()
     if world == 1 and not args.no_extras:
         line["read_only_peak_gbs"] = read_only_peak()
         if w.name != "7b_tree":
-            line["tree"] = quick_time(S.WORKLOADS["7b_tree"], min(args.steps, 16), 3)
+            wt = S.WORKLOADS["7b_tree"]
+            line["tree"] = quick_time(wt, min(args.steps, 16), 3)
+            if not args.no_draft_loop:
+                n_it = min(args.steps, 16)
+                line["tree"]["draft_loop"] = draft_loop(wt, n_it, 3, max(S.kv_lengths(wt, SEED)) + (n_it + 5) *
+                                                        (wt.gamma + 1) + wt.n_nodes + 64)
+            torch.cuda.empty_cache()
         line["rows_sweep_13b"] = rows_sweep(8, 3)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, args.warmup)

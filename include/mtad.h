@@ -149,15 +149,26 @@ int mtad_set_warp(mtad_ctx* ctx, int top_k, float top_p);
  * are drawn without replacement, proportionally to their joint likelihood, as the beam_width largest values of
  * log q(beam) + log q(token | beam) + Gumbel noise, noise = -log(-log(u)).
  *   seqs        host  [B]                 sequence ids (distinct)
+ *   keep_all_candidates  0: the tree holds the kept beams, W = beam_width nodes a layer, best first (the paper's
+ *               tree).  Non-zero: a layer also records the candidates that the selection looked at and did not
+ *               keep, as leaves: W = beam_width^2 nodes a layer - the beam_width^2 best perturbed tokens of the
+ *               single beam of step 1, afterwards beam by beam (in the order of the previous layer's kept beams)
+ *               its beam_width best perturbed tokens, best first.  The kept beams are the beam_width best of the
+ *               layer; only they have children.  Needs gamma * beam_width^2 <= MTAD_MAX_NODES and a vocabulary of
+ *               at least beam_width^2 tokens (MTAD_E_CAPACITY otherwise).
  *   uniforms    device [B, gamma, beam_width, vocab] fp32 in (0,1)
- *   tok,parent,depth  device [B, gamma*beam_width] int32  node arrays, layer by layer (parent = -1: child of root)
- *   node_logq   device [B, gamma*beam_width] fp32  joint draft log-likelihood of the path ending at each node
+ *   n_nodes     device [B] int32, may be NULL   gamma * W, for the mtad_verify_tree call that follows
+ *   tok,parent,depth  device [B, gamma * W] int32  node arrays, layer by layer (parent = -1: child of root)
+ *   node_logq   device [B, gamma * W] fp32  joint draft log-likelihood of the path ending at each node
  *   logq_ref    device [B, gamma] fp32   log q(x**_{1:i}), x** = final beam with the highest likelihood
  *   best_path   device [B, gamma] int32  node ids of x**
- * The chain of Algorithm 1 is best_path with logq_ref. */
-int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_width, const float* uniforms,
-               int32_t* tok, int32_t* parent, int32_t* depth, float* node_logq, float* logq_ref,
-               int32_t* best_path, void* stream);
+ * The chain of Algorithm 1 is best_path with logq_ref.  kv_commit after a verification of this tree (or of that
+ * chain) also rolls the auxiliary cache forward: accepted nodes that were beams of a layer before the last keep
+ * their keys and values, an accepted node that the auxiliary model never ran (last layer, or a candidate that was
+ * not kept) is replayed by the next draft together with the extra token. */
+int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_width, int keep_all_candidates,
+               const float* uniforms, int32_t* n_nodes, int32_t* tok, int32_t* parent, int32_t* depth,
+               float* node_logq, float* logq_ref, int32_t* best_path, void* stream);
 
 /* Verify a draft chain x_1..x_gamma (Algorithm 1 from "P <- M_p(input, X)" to the return).
  *   seqs         host   [B]

@@ -80,7 +80,7 @@ def load_library() -> C.CDLL:
     lib.mtad_debug_region.argtypes = [P, C.c_char_p, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     lib.mtad_debug_check_canaries.argtypes = [P, P, C.POINTER(C.c_char_p)]
     lib.mtad_profile_grouped.argtypes = [P, I]
-    lib.mtad_draft.argtypes = [P, I, I32P, I, I, P, P, P, P, P, P, P, P]
+    lib.mtad_draft.argtypes = [P, I, I32P, I, I, I, P, P, P, P, P, P, P, P, P]
     lib.mtad_verify_chain.argtypes = [P, I, I32P, I, P, P, F, P, RS, P]
     lib.mtad_verify_tree.argtypes = [P, I, I32P, P, I, I, P, P, P, F, P, RS, P]
     lib.mtad_verify_chain_spd.argtypes = [P, I, I32P, I, P, P, P, P, RS, P]
@@ -325,9 +325,12 @@ class Context:
         return {k: {"ms": ms[i], "bytes": by[i], "launches": cnt[i]} for i, k in enumerate(KERNEL_CLASSES)}
 
     def mtad_draft(self, seqs, gamma: int, beam_width: int, uniforms, tok, parent, depth, node_logq, logq_ref,
-                   best_path, stream=None, check=True) -> int:
+                   best_path, stream=None, check=True, keep_all_candidates=False, n_nodes=None) -> int:
+        """Node arrays hold gamma * beam_width entries per sequence, gamma * beam_width**2 with keep_all_candidates."""
         rc = self._lib.mtad_draft(self.handle, len(seqs), _seqs(seqs), gamma, beam_width,
-                                  _ptr(uniforms, torch.float32), _ptr(tok, torch.int32), _ptr(parent, torch.int32),
+                                  1 if keep_all_candidates else 0, _ptr(uniforms, torch.float32),
+                                  None if n_nodes is None else _ptr(n_nodes, torch.int32),
+                                  _ptr(tok, torch.int32), _ptr(parent, torch.int32),
                                   _ptr(depth, torch.int32), _ptr(node_logq, torch.float32),
                                   _ptr(logq_ref, torch.float32), _ptr(best_path, torch.int32), _stream(stream))
         if check:

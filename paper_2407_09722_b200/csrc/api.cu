@@ -255,6 +255,8 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     ds.node_logq = k.take<float>((size_t)max_batch * MTAD_DRAFT_NODES, "ds_node_logq");
     ds.node_mask = k.take<uint32_t>((size_t)max_batch * MTAD_DRAFT_NODES * MTAD_MASK_WORDS, "ds_node_mask");
     ds.best_path = k.take<int32_t>((size_t)max_batch * MTAD_MAX_DEPTH, "ds_best_path");
+    ds.tree_id = k.take<int32_t>((size_t)max_batch * MTAD_DRAFT_NODES, "ds_tree_id");
+    ds.tree2slot = k.take<int32_t>((size_t)max_batch * MTAD_DRAFT_NODES, "ds_tree2slot");
     if (c) {
         c->ds = ds;
         c->st = st; c->rm = rm; c->sc = sc;
@@ -883,9 +885,9 @@ int mtad_seq_get(mtad_ctx* ctx, int seq, int32_t* kv_len, int32_t* root_token, v
     return MTAD_OK;
 }
 
-int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_width, const float* uniforms,
-               int32_t* tok, int32_t* parent, int32_t* depth, float* node_logq, float* logq_ref,
-               int32_t* best_path, void* stream) {
+int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_width, int keep_all_candidates,
+               const float* uniforms, int32_t* n_nodes, int32_t* tok, int32_t* parent, int32_t* depth, float* node_logq,
+               float* logq_ref, int32_t* best_path, void* stream) {
     if (!ctx) return MTAD_E_INVALID;
     if (!ctx->has_aux) return MTAD_E_INVALID;
     if (!seqs_ok(ctx, B, seqs)) return MTAD_E_INVALID;
@@ -893,6 +895,11 @@ int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_wi
     if (gamma < 1 || beam_width < 1) return MTAD_E_INVALID;
     if (gamma > MTAD_MAX_DEPTH || beam_width > MTAD_MAX_BEAM || gamma * beam_width > MTAD_DRAFT_NODES - MTAD_MAX_DEPTH - 1 ||
         gamma * beam_width > MTAD_MAX_NODES)
+        return MTAD_E_CAPACITY;
+    const int keep_all = keep_all_candidates ? 1 : 0;
+    // the caller's tree: beam_width * beam_width nodes a layer with every candidate kept (a verify call takes
+    // MTAD_MAX_NODES at most), and a layer can only be filled from a vocabulary that large
+    if (keep_all && (gamma * beam_width * beam_width > MTAD_MAX_NODES || ctx->aux.d.vocab < beam_width * beam_width))
         return MTAD_E_CAPACITY;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const ModelView& m = ctx->aux;
@@ -906,7 +913,7 @@ int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_wi
     if (ub + 1 + (long long)gamma * beam_width > m.d.kv_capacity) return MTAD_E_CAPACITY;
     SeqList sl{};
     for (int i = 0; i < B; ++i) sl.v[i] = seqs[i];
-    DraftOut out{tok, parent, depth, node_logq, logq_ref, best_path};
+    DraftOut out{n_nodes, tok, parent, depth, node_logq, logq_ref, best_path};
     const bool tc = ctx->use_tc && ctx->amaps.ok;
     CU(cudaMemsetAsync(ctx->sc.tc_counters, 0, sizeof(int32_t) * ctx->tc_counter_n, s));
     for (int step = 0; step < gamma; ++step) {
@@ -919,7 +926,7 @@ int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_wi
         if (tc && B * R <= TC_MAX_ROWS) rc = forward_rows_tc(ctx, m, ctx->amaps, B, R, keys_ub, nullptr, nullptr, true, s);
         else rc = forward_rows(ctx, m, B, R, keys_ub, s);
         if (rc != MTAD_OK) return rc;
-        RUN(MTAD_K_LMRED, 0, 2, launch_draft_select(m, ctx->ds, ctx->sc, sl, B, R, step, gamma, beam_width, uniforms, out,
+        RUN(MTAD_K_LMRED, 0, 2, launch_draft_select(m, ctx->ds, ctx->sc, sl, B, R, step, gamma, beam_width, keep_all, uniforms, out,
                                                      ctx->use_pdl, s));
     }
     ctx->draft_active = true;
@@ -1125,6 +1132,14 @@ int mtad_audit_extents(const mtad_model_desc* target, const mtad_model_desc* aux
             au.ws("ds_node_parent", (size_t)(max_batch - 1) * MTAD_DRAFT_NODES + n_last + 1);
             au.ws("ds_node_logq", (size_t)(max_batch - 1) * MTAD_DRAFT_NODES + n_last + 1);
             au.ws("ds_node_mask", ((size_t)(max_batch - 1) * MTAD_DRAFT_NODES + n_last) * MTAD_MASK_WORDS + MTAD_MASK_WORDS);
+            au.ws("ds_tree_id", (size_t)(max_batch - 1) * MTAD_DRAFT_NODES + n_last + 1);
+            // node ids of the caller's tree: beam per layer, or beam * beam with every candidate kept (when that fits a
+            // verify call); the selection holds the chunks' candidates of all beam rows in shared memory
+            const size_t per_layer = gamma * beam * beam <= MTAD_MAX_NODES ? (size_t)beam * beam : (size_t)beam;
+            au.ws("ds_tree2slot", (size_t)(max_batch - 1) * MTAD_DRAFT_NODES + step * per_layer + per_layer);
+            au.ext("selection candidates (shared memory)",
+                   (size_t)(step == 0 ? 1 : beam) * nch * (step == 0 ? per_layer : (size_t)beam),
+                   (size_t)MTAD_MAX_BEAM * MTAD_DRAFT_CHUNKS * MTAD_MAX_BEAM);
             // a node's mask bit: virtual row P + n, below MTAD_MASK_WORDS * 32
             au.ext("mask bits (virtual rows)", (size_t)R + n_last + 1 + (step == 0 ? 0 : P_max), (size_t)MTAD_MASK_WORDS * 32);
             au.ext("uniforms (caller)", (((size_t)(B - 1) * gamma + step) * beam + (step == 0 ? 0 : beam - 1)) * V + V,

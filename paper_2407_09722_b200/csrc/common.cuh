@@ -62,10 +62,15 @@ struct DraftState {
     int32_t* node_parent;  // [max_batch][MTAD_DRAFT_NODES]
     float* node_logq;      // [max_batch][MTAD_DRAFT_NODES]
     uint32_t* node_mask;   // [max_batch][MTAD_DRAFT_NODES][MTAD_MASK_WORDS] visible virtual rows of each node
-    int32_t* best_path;    // [max_batch][MTAD_MAX_DEPTH]
+    int32_t* best_path;    // [max_batch][MTAD_MAX_DEPTH] beam slots of x** (slot = layer * beam + rank)
+    // The nodes above are the beams (the rows the auxiliary model runs), indexed by beam slot.  The tree handed to the
+    // caller may hold more (mtad_draft with keep_all_candidates): these map between the two numberings.
+    int32_t* tree_id;      // [max_batch][MTAD_DRAFT_NODES] beam slot -> node id in the caller's tree
+    int32_t* tree2slot;    // [max_batch][MTAD_DRAFT_NODES] node id in the caller's tree -> beam slot, -1: not a beam
 };
 
 struct DraftOut {          // caller's device arrays of mtad_draft
+    int32_t* n_nodes;      // [B] or null
     int32_t *tok, *parent, *depth;
     float* node_logq;
     float* logq_ref;
@@ -76,10 +81,11 @@ struct DraftOut {          // caller's device arrays of mtad_draft
 
 // What one chunk of a beam row hands to the draft's selection: its share of the row's log-sum-exp and its largest
 // perturbed logits (token -1: none).
+#define MTAD_MAX_CAND (MTAD_MAX_BEAM * MTAD_MAX_BEAM)   // candidates of one beam row kept per chunk (at most)
 struct DraftPart {
     float m, s;
-    float t[MTAD_MAX_BEAM];
-    int32_t v[MTAD_MAX_BEAM];
+    float t[MTAD_MAX_CAND];
+    int32_t v[MTAD_MAX_CAND];
 };
 
 #define MTAD_MAX_TOPK 16           // largest top-k of the warped rows
@@ -346,8 +352,8 @@ cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const Dr
                                  const Scratch& sc, const SeqList& seqs, int B, int R, int step, int beam, bool tc,
                                  bool pdl, cudaStream_t st);
 cudaError_t launch_draft_select(const ModelView& m, const DraftState& ds, const Scratch& sc, const SeqList& seqs, int B,
-                                int R, int step, int gamma, int beam, const float* uniforms, const DraftOut& out,
-                                bool pdl, cudaStream_t st);
+                                int R, int step, int gamma, int beam, int keep_all, const float* uniforms,
+                                const DraftOut& out, bool pdl, cudaStream_t st);
 cudaError_t launch_aux_commit(const ModelView& aux, const SeqState& s, const DraftState& ds, int B,
                               const int32_t* call_seq_dev, const mtad_result& res, int max_depth, int mode,
                               cudaStream_t st);

@@ -26,6 +26,24 @@ __device__ __forceinline__ bool before(const Cand& a, const Cand& b) {     // a 
     return a.y > b.y || (a.y == b.y && a.flat < b.flat);
 }
 
+// The best candidate of a block of 256 threads, returned to every thread: butterfly inside each warp, then the eight
+// warp winners through shared memory (two barriers a call; s_w is free again on return).
+__device__ __forceinline__ Cand block_best(Cand c, Cand* s_w, int tid) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const Cand c2{__shfl_xor_sync(0xffffffffu, c.y, o), __shfl_xor_sync(0xffffffffu, c.flat, o)};
+        if (before(c2, c)) c = c2;
+    }
+    if ((tid & 31) == 0) s_w[tid >> 5] = c;
+    __syncthreads();
+    Cand best = s_w[0];
+#pragma unroll
+    for (int w = 1; w < 8; ++w)
+        if (before(s_w[w], best)) best = s_w[w];
+    __syncthreads();
+    return best;
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -141,9 +159,11 @@ cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const Dr
 // ---------------------------------------------------------------------------------------------------------------
 
 __global__ void __launch_bounds__(256) draft_scan_kernel(const float* __restrict__ logits, int V, int R, int step,
-                                                         int gamma, int beam, const float* __restrict__ uni,
+                                                         int gamma, int beam, int kpb, const float* __restrict__ uni,
                                                          DraftState ds, SeqList seqs, DraftPart* __restrict__ part,
                                                          int nch) {
+    // kpb: perturbed logits of this chunk to hand on (the beam width, or with all candidates kept the candidates
+    // recorded per beam: beam * beam of the single beam of step 0, beam afterwards)
     const int c = blockIdx.x, j = blockIdx.y, bi = blockIdx.z, seq = seqs.v[bi];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     pdl_wait();               // the logits come from the kernel before
@@ -154,8 +174,10 @@ __global__ void __launch_bounds__(256) draft_scan_kernel(const float* __restrict
     const float* ub = uni + (((size_t)bi * gamma + step) * beam + j) * V;
     const int len = (V + nch - 1) / nch, v0 = c * len, v1 = min(V, v0 + len);
     __shared__ float s_m[8], s_s[8];
-    __shared__ Cand s_c[256];
+    __shared__ Cand s_w[8];
     float m = -CUDART_INF_F, sum = 0.f;
+    // a thread sees at most MTAD_MAX_BEAM tokens of the chunk (the host keeps chunks within 256 * MTAD_MAX_BEAM), so
+    // its sorted list holds all of them and the rounds below find the chunk's exact order
     Cand loc[MTAD_MAX_BEAM];
 #pragma unroll
     for (int k = 0; k < MTAD_MAX_BEAM; ++k) loc[k] = Cand{-CUDART_INF_F, 0x7fffffff};
@@ -181,18 +203,14 @@ __global__ void __launch_bounds__(256) draft_scan_kernel(const float* __restrict
     }
     if (lane == 0) { s_m[warp] = m; s_s[warp] = sum; }
     DraftPart* dst = part + ((size_t)(bi * MTAD_MAX_BEAM + j)) * nch + c;
-    // `beam` rounds: the block's best head-of-list wins, its owner advances
+    // kpb rounds: the block's best head-of-list wins, its owner advances
     int head = 0;
-    for (int k = 0; k < beam; ++k) {
-        const Cand cd = head < MTAD_MAX_BEAM ? loc[head] : Cand{-CUDART_INF_F, 0x7fffffff};
-        s_c[tid] = cd;
-        __syncthreads();
-        for (int o = 128; o > 0; o >>= 1) {
-            if (tid < o && before(s_c[tid + o], s_c[tid])) s_c[tid] = s_c[tid + o];
-            __syncthreads();
-        }
-        const Cand win = s_c[0];
-        __syncthreads();
+    for (int k = 0; k < kpb; ++k) {
+        Cand cd{-CUDART_INF_F, 0x7fffffff};
+#pragma unroll
+        for (int q = 0; q < MTAD_MAX_BEAM; ++q)
+            if (q == head) cd = loc[q];
+        const Cand win = block_best(cd, s_w, tid);
         if (cd.flat == win.flat && win.flat != 0x7fffffff) ++head;      // the owner of the winner (tokens are unique)
         if (tid == 0) {
             dst->t[k] = win.y;
@@ -210,21 +228,24 @@ __global__ void __launch_bounds__(256) draft_scan_kernel(const float* __restrict
 }
 
 __global__ void __launch_bounds__(256) draft_pick_kernel(const float* __restrict__ logits, int V, int R, int step,
-                                                         int gamma, int beam, DraftState ds, SeqList seqs,
-                                                         const DraftPart* __restrict__ part, int nch, DraftOut out) {
+                                                         int gamma, int beam, int keep_all, int kpb, DraftState ds,
+                                                         SeqList seqs, const DraftPart* __restrict__ part, int nch,
+                                                         DraftOut out) {
     const int bi = blockIdx.x, seq = seqs.v[bi];
     const int tid = threadIdx.x;
     pdl_wait();               // the chunk results come from the kernel before
     pdl_trigger();
     const int P = min(max(ds.npend[seq], 1), step == 0 ? R : MTAD_MAX_DEPTH + 1);   // in range whatever the state holds
     const int n_beams = step == 0 ? 1 : beam;
-    const int N = gamma * beam;
+    const int per_layer = keep_all ? beam * beam : beam;          // nodes of a layer of the caller's tree
+    const int N = gamma * per_layer;
     __shared__ float s_lse[MTAD_MAX_BEAM], s_lq[MTAD_MAX_BEAM];
-    __shared__ int s_node[MTAD_MAX_BEAM];
+    __shared__ int s_slot[MTAD_MAX_BEAM], s_tree[MTAD_MAX_BEAM];   // the current beams: beam slot and tree id (-1: the context)
     __shared__ float s_y[MTAD_MAX_BEAM * MTAD_DRAFT_CHUNKS * MTAD_MAX_BEAM];
     __shared__ int s_flat[MTAD_MAX_BEAM * MTAD_DRAFT_CHUNKS * MTAD_MAX_BEAM];
-    __shared__ Cand s_c[256];
-    __shared__ int s_i[256];
+    __shared__ Cand s_w[8];
+    __shared__ float l_y[MTAD_MAX_CAND];                           // the layer's nodes: perturbed score, flat pair,
+    __shared__ int l_flat[MTAD_MAX_CAND], l_rank[MTAD_MAX_CAND];   // rank among the kept beams (-1: not kept)
     const DraftPart* pp = part + (size_t)bi * MTAD_MAX_BEAM * nch;
     if (tid < n_beams) {
         // log-sum-exp of beam row tid: chunks in order
@@ -234,48 +255,82 @@ __global__ void __launch_bounds__(256) draft_pick_kernel(const float* __restrict
         float a = 0.f;
         for (int c = 0; c < nch; ++c) a += (pj[c].m == -CUDART_INF_F) ? 0.f : pj[c].s * expf(pj[c].m - M);
         s_lse[tid] = M + logf(a);
-        const int node = step == 0 ? -1 : (step - 1) * beam + tid;
-        s_node[tid] = node;
-        s_lq[tid] = node < 0 ? 0.f : ds.node_logq[seq * MTAD_DRAFT_NODES + node];
+        const int slot = step == 0 ? -1 : (step - 1) * beam + tid;
+        s_slot[tid] = slot;
+        s_tree[tid] = slot < 0 ? -1 : ds.tree_id[seq * MTAD_DRAFT_NODES + slot];
+        s_lq[tid] = slot < 0 ? 0.f : ds.node_logq[seq * MTAD_DRAFT_NODES + slot];
     }
     __syncthreads();
-    const int n_cand = n_beams * nch * MTAD_MAX_BEAM;
+    const int per_beam = nch * kpb;                                // candidates of one beam row
+    const int n_cand = n_beams * per_beam;
     for (int i = tid; i < n_cand; i += 256) {
-        const int j = i / (nch * MTAD_MAX_BEAM), c = (i / MTAD_MAX_BEAM) % nch, k = i % MTAD_MAX_BEAM;
+        const int j = i / per_beam, c = (i / kpb) % nch, k = i % kpb;
         const DraftPart& d = pp[(size_t)j * nch + c];
-        const bool ok = k < beam && d.v[k] >= 0;
+        const bool ok = d.v[k] >= 0;
         s_y[i] = ok ? d.t[k] + (s_lq[j] - s_lse[j]) : -CUDART_INF_F;
         s_flat[i] = ok ? j * V + d.v[k] : 0x7fffffff;
     }
     __syncthreads();
-    for (int k = 0; k < beam; ++k) {
-        Cand best{-CUDART_INF_F, 0x7fffffff};
-        int bidx = -1;
-        for (int i = tid; i < n_cand; i += 256) {
-            const Cand cd{s_y[i], s_flat[i]};
-            if (cd.flat != 0x7fffffff && before(cd, best)) { best = cd; bidx = i; }
-        }
-        s_c[tid] = best;
-        s_i[tid] = bidx;
-        __syncthreads();
-        for (int o = 128; o > 0; o >>= 1) {
-            if (tid < o && before(s_c[tid + o], s_c[tid])) { s_c[tid] = s_c[tid + o]; s_i[tid] = s_i[tid + o]; }
+    // The layer's nodes.  Plain tree: the `beam` best pairs of all, best first.  All candidates kept: beam by beam its
+    // kpb best pairs, best first.  Every round is a block-wide arg-max over a range of the candidates; the winner is
+    // struck out.
+    const int n_groups = keep_all ? n_beams : 1, rounds = keep_all ? kpb : beam;
+    for (int gidx = 0; gidx < n_groups; ++gidx) {
+        const int lo = keep_all ? gidx * per_beam : 0, hi = keep_all ? lo + per_beam : n_cand;
+        for (int k = 0; k < rounds; ++k) {
+            Cand best{-CUDART_INF_F, 0x7fffffff};
+            int bidx = -1;
+            for (int i = lo + tid; i < hi; i += 256) {
+                const Cand cd{s_y[i], s_flat[i]};
+                if (cd.flat != 0x7fffffff && before(cd, best)) { best = cd; bidx = i; }
+            }
+            const Cand win = block_best(best, s_w, tid);
+            const bool found = win.flat != 0x7fffffff;
+            if (found && bidx >= 0 && best.flat == win.flat) {       // the owner strikes the winner out (pairs are unique)
+                s_y[bidx] = -CUDART_INF_F;
+                s_flat[bidx] = 0x7fffffff;
+            }
+            if (tid == 0) {
+                const int m = gidx * rounds + k;
+                l_y[m] = found ? win.y : -CUDART_INF_F;
+                l_flat[m] = win.flat;
+                l_rank[m] = keep_all ? -1 : k;
+            }
             __syncthreads();
         }
-        if (tid == 0) {
-            const Cand win = s_c[0];
-            const int widx = s_i[0];
-            // a vocabulary of at least `beam` tokens always leaves a pair to take
-            const int j = widx >= 0 ? win.flat / V : 0, v = widx >= 0 ? win.flat % V : 0;
-            if (widx >= 0) { s_y[widx] = -CUDART_INF_F; s_flat[widx] = 0x7fffffff; }
-            const int n = step * beam + k;
-            const int row = step == 0 ? P - 1 : j;
-            const float lq = s_lq[j] + logits[(size_t)(bi * R + row) * V + v] - s_lse[j];
-            const int parent = s_node[j];
-            ds.node_tok[seq * MTAD_DRAFT_NODES + n] = v;
-            ds.node_parent[seq * MTAD_DRAFT_NODES + n] = parent;
-            ds.node_logq[seq * MTAD_DRAFT_NODES + n] = lq;
-            uint32_t* mk = ds.node_mask + ((size_t)seq * MTAD_DRAFT_NODES + n) * MTAD_MASK_WORDS;
+    }
+    if (keep_all && tid == 0) {
+        // the beams kept for the next step: the `beam` best of the layer's nodes (they are the best of all pairs)
+        for (int k = 0; k < beam; ++k) {
+            int bm = -1;
+            for (int m = 0; m < per_layer; ++m)
+                if (l_rank[m] < 0 && l_flat[m] != 0x7fffffff &&
+                    (bm < 0 || before(Cand{l_y[m], l_flat[m]}, Cand{l_y[bm], l_flat[bm]})))
+                    bm = m;
+            if (bm >= 0) l_rank[bm] = k;
+        }
+    }
+    __syncthreads();
+    // every node of the layer, one thread each: the caller's tree, and for a kept node the beam state of the next step
+    for (int m = tid; m < per_layer; m += 256) {
+        const bool valid = l_flat[m] != 0x7fffffff;        // a vocabulary of at least per_layer tokens always fills the layer
+        const int j = valid ? l_flat[m] / V : 0, v = valid ? l_flat[m] % V : 0;
+        const int n = step * per_layer + m;
+        const int row = step == 0 ? P - 1 : j;
+        const float lq = s_lq[j] + logits[(size_t)(bi * R + row) * V + v] - s_lse[j];
+        out.tok[bi * N + n] = v;
+        out.parent[bi * N + n] = s_tree[j];
+        out.depth[bi * N + n] = step + 1;
+        out.node_logq[bi * N + n] = lq;
+        const int k = l_rank[m];
+        if (n < MTAD_DRAFT_NODES) ds.tree2slot[seq * MTAD_DRAFT_NODES + n] = k >= 0 ? step * beam + k : -1;
+        if (k >= 0) {
+            const int slot = step * beam + k, parent = s_slot[j];
+            ds.node_tok[seq * MTAD_DRAFT_NODES + slot] = v;
+            ds.node_parent[seq * MTAD_DRAFT_NODES + slot] = parent;
+            ds.node_logq[seq * MTAD_DRAFT_NODES + slot] = lq;
+            ds.tree_id[seq * MTAD_DRAFT_NODES + slot] = n;
+            uint32_t* mk = ds.node_mask + ((size_t)seq * MTAD_DRAFT_NODES + slot) * MTAD_MASK_WORDS;
             for (int i = 0; i < MTAD_MASK_WORDS; ++i) {
                 uint32_t w;
                 if (parent >= 0) w = ds.node_mask[((size_t)seq * MTAD_DRAFT_NODES + parent) * MTAD_MASK_WORDS + i];
@@ -283,70 +338,86 @@ __global__ void __launch_bounds__(256) draft_pick_kernel(const float* __restrict
                     const int lo = i * 32;
                     w = P >= lo + 32 ? 0xffffffffu : (P > lo ? (1u << (P - lo)) - 1u : 0u);
                 }
-                if (((P + n) >> 5) == i) w |= 1u << ((P + n) & 31);
+                if (((P + slot) >> 5) == i) w |= 1u << ((P + slot) & 31);
                 mk[i] = w;
             }
-            out.tok[bi * N + n] = v;
-            out.parent[bi * N + n] = parent;
-            out.depth[bi * N + n] = step + 1;
-            out.node_logq[bi * N + n] = lq;
         }
-        __syncthreads();
     }
+    __syncthreads();
     if (step == gamma - 1 && tid == 0) {
-        // x**: the final beam with the highest draft likelihood (lowest node id on ties), and its prefix likelihoods
+        // x**: the final beam with the highest draft likelihood (lowest tree id on ties), and its prefix likelihoods
+        __threadfence_block();
         int best = (gamma - 1) * beam;
         for (int k = 1; k < beam; ++k) {
-            const int n = (gamma - 1) * beam + k;
-            if (ds.node_logq[seq * MTAD_DRAFT_NODES + n] > ds.node_logq[seq * MTAD_DRAFT_NODES + best]) best = n;
+            const int sl = (gamma - 1) * beam + k;
+            const float a = ds.node_logq[seq * MTAD_DRAFT_NODES + sl], b0 = ds.node_logq[seq * MTAD_DRAFT_NODES + best];
+            if (a > b0 || (a == b0 && ds.tree_id[seq * MTAD_DRAFT_NODES + sl] < ds.tree_id[seq * MTAD_DRAFT_NODES + best]))
+                best = sl;
         }
         int cur = best;
         for (int i = gamma - 1; i >= 0 && cur >= 0; --i) {
-            out.best_path[bi * gamma + i] = cur;
+            out.best_path[bi * gamma + i] = ds.tree_id[seq * MTAD_DRAFT_NODES + cur];
             out.logq_ref[bi * gamma + i] = ds.node_logq[seq * MTAD_DRAFT_NODES + cur];
             ds.best_path[seq * MTAD_MAX_DEPTH + i] = cur;
             cur = ds.node_parent[seq * MTAD_DRAFT_NODES + cur];
         }
         ds.gamma[seq] = gamma;
         ds.beam[seq] = beam;
+        if (out.n_nodes) out.n_nodes[bi] = N;
     }
 }
 
 cudaError_t launch_draft_select(const ModelView& m, const DraftState& ds, const Scratch& sc, const SeqList& seqs, int B,
-                                int R, int step, int gamma, int beam, const float* uniforms, const DraftOut& out,
-                                bool pdl, cudaStream_t st) {
+                                int R, int step, int gamma, int beam, int keep_all, const float* uniforms,
+                                const DraftOut& out, bool pdl, cudaStream_t st) {
     const int V = m.d.vocab;
     int nch = (V + 1023) / 1024;
     nch = nch < 1 ? 1 : (nch > MTAD_DRAFT_CHUNKS ? MTAD_DRAFT_CHUNKS : nch);
     const int n_beams = step == 0 ? 1 : beam;
+    const int kpb = (keep_all && step == 0) ? beam * beam : beam;
     cudaError_t e = launch_pdl(draft_scan_kernel, dim3(nch, n_beams, B), dim3(256), 0, st, pdl, (const float*)sc.logits,
-                               V, R, step, gamma, beam, uniforms, ds, seqs, sc.draft_part, nch);
+                               V, R, step, gamma, beam, kpb, uniforms, ds, seqs, sc.draft_part, nch);
     if (e != cudaSuccess) return e;
     return launch_pdl(draft_pick_kernel, dim3(B), dim3(256), 0, st, pdl, (const float*)sc.logits, V, R, step, gamma,
-                      beam, ds, seqs, (const DraftPart*)sc.draft_part, nch, out);
+                      beam, keep_all, kpb, ds, seqs, (const DraftPart*)sc.draft_part, nch, out);
 }
 
 // ---------------------------------------------------------------------------------------------------------------
 // auxiliary cache roll-forward after a verification
 // ---------------------------------------------------------------------------------------------------------------
 
-// The rows that the roll-forward would touch: accepted node r (r < kept) is read from slot base + node id and written
-// to slot base + r; all of them inside [0, cap), the path entries inside the draft's node arrays.
-__device__ __forceinline__ bool aux_commit_in_range(const DraftState& ds, const mtad_result& res, int bi, int seq, int D,
-                                                    int mode, int kept, int base, long long cap) {
-    if (kept > D || kept > MTAD_MAX_DEPTH || base < 0 || (long long)base + kept > cap) return false;
-    for (int r = 0; r < kept; ++r) {
-        const int pn = res.path[bi * D + r];
-        if (pn < 0 || pn >= (mode == 0 ? MTAD_MAX_DEPTH : MTAD_DRAFT_NODES)) return false;
-        const int node = mode == 0 ? ds.best_path[seq * MTAD_MAX_DEPTH + pn] : pn;
-        if (node < 0 || node >= MTAD_DRAFT_NODES || (long long)base + node >= cap) return false;
-    }
-    return true;
+// Beam slot of accepted node r of a verified draft.  mode 0: the verified chain was the draft's output sequence (chain
+// node i = beam slot best_path[i]); mode 1: the verified tree was the draft's tree (node ids of that tree; a node that
+// was recorded as a candidate only has no slot).  -1: no slot, -2: the path entry itself is out of range.
+__device__ __forceinline__ int aux_slot_of(const DraftState& ds, const mtad_result& res, int bi, int seq, int D, int mode,
+                                           int r) {
+    const int pn = res.path[bi * D + r];
+    if (pn < 0 || pn >= (mode == 0 ? MTAD_MAX_DEPTH : MTAD_DRAFT_NODES)) return -2;
+    const int slot = mode == 0 ? ds.best_path[seq * MTAD_MAX_DEPTH + pn] : ds.tree2slot[seq * MTAD_DRAFT_NODES + pn];
+    return slot >= MTAD_DRAFT_NODES ? -2 : (slot < 0 ? -1 : slot);
 }
 
-// mode 0: the verified chain was the draft's output sequence (chain node i = draft node best_path[i]);
-// mode 1: the verified tree was the draft's tree (same node ids).  Accepted node i (depth i + 1, slot base + id)
-// moves to position base + i when the draft ran it (depth < gamma).
+// Accepted nodes whose keys and values the draft left in the auxiliary cache: the leading ones that were beams of a
+// layer before the last (the last layer, and candidates that were not kept, never ran).  At most one accepted token
+// can follow them (such a node is a leaf of the tree).  Returns -1 when the path, the state or a cache row that the
+// roll-forward would touch is out of range: accepted node r (r < kept) is read from slot base + beam slot and written
+// to slot base + r, all inside [0, cap).
+__device__ __forceinline__ int aux_kept_rows(const DraftState& ds, const mtad_result& res, int bi, int seq, int D, int mode,
+                                             int eta, int base, long long cap) {
+    const int gamma = ds.gamma[seq], beam = ds.beam[seq];
+    if (gamma < 1 || gamma > MTAD_MAX_DEPTH || beam < 1 || beam > MTAD_MAX_BEAM || eta > D || base < 0) return -1;
+    int kept = 0;
+    for (; kept < eta; ++kept) {
+        const int slot = aux_slot_of(ds, res, bi, seq, D, mode, kept);
+        if (slot == -2) return -1;
+        if (slot < 0 || slot >= (gamma - 1) * beam) break;
+        if ((long long)base + slot >= cap) return -1;
+    }
+    if (eta - kept > 1 || kept > MTAD_MAX_DEPTH || (long long)base + kept > cap) return -1;
+    return kept;
+}
+
+// Accepted node i (depth i + 1, slot base + beam slot) moves to position base + i when the draft ran it.
 __global__ void aux_commit_kernel(__nv_bfloat16* __restrict__ cache, const int32_t* __restrict__ call_seq,
                                   DraftState ds, mtad_result res, int D, int mode, int max_batch, int Hkv, int hd,
                                   long long cap) {
@@ -354,13 +425,12 @@ __global__ void aux_commit_kernel(__nv_bfloat16* __restrict__ cache, const int32
     if (res.status[bi] != 0) return;
     const int seq = call_seq[bi];
     if ((unsigned)seq >= (unsigned)max_batch) return;
-    const int gamma = ds.gamma[seq];
     const int eta = res.eta[bi];
-    const int kept = min(eta, gamma - 1);
-    if (kept <= 0) return;
+    if (eta <= 0) return;
     const int base = ds.base_len[seq] + ds.npend[seq];
     // every row read or written lies inside the cache, or nothing moves (aux_advance_kernel flags the sequence)
-    if (!aux_commit_in_range(ds, res, bi, seq, D, mode, kept, base, cap)) return;
+    const int kept = aux_kept_rows(ds, res, bi, seq, D, mode, eta, base, cap);
+    if (kept <= 0) return;
     const int head = blockIdx.x % Hkv;
     const int kv = (blockIdx.x / Hkv) & 1;
     const int layer = blockIdx.x / (2 * Hkv);
@@ -368,8 +438,7 @@ __global__ void aux_commit_kernel(__nv_bfloat16* __restrict__ cache, const int32
     extern __shared__ __nv_bfloat16 buf[];
     for (int i = threadIdx.x; i < kept * hd; i += blockDim.x) {
         const int r = i / hd, j = i % hd;
-        const int pn = res.path[bi * D + r];
-        const int node = mode == 0 ? ds.best_path[seq * MTAD_MAX_DEPTH + pn] : pn;
+        const int node = aux_slot_of(ds, res, bi, seq, D, mode, r);
         buf[i] = b[(size_t)(base + node) * hd + j];
     }
     __syncthreads();
@@ -397,15 +466,12 @@ __global__ void aux_advance_kernel(SeqState s, DraftState ds, const int32_t* __r
         s.aux_npend[seq] = np + eta + 1;
         return;
     }
-    const int gamma = ds.gamma[seq];
-    const int kept = min(eta, gamma - 1);
-    if (kept > 0 && !aux_commit_in_range(ds, res, bi, seq, D, mode, kept, ds.base_len[seq] + ds.npend[seq], cap)) {
-        atomicOr(&res.status[bi], MTAD_ST_RANGE);
-        return;
-    }
-    s.aux_len[seq] = ds.base_len[seq] + ds.npend[seq] + kept;
+    const int base = ds.base_len[seq] + ds.npend[seq];
+    const int kept = aux_kept_rows(ds, res, bi, seq, D, mode, eta, base, cap);
+    if (kept < 0) { atomicOr(&res.status[bi], MTAD_ST_RANGE); return; }
+    s.aux_len[seq] = base + kept;
     int np = 0;
-    if (eta >= gamma) pend[np++] = res.out_tok[bi * (D + 1) + eta - 1];   // last layer's node: never run by the aux model
+    if (eta > kept) pend[np++] = res.out_tok[bi * (D + 1) + eta - 1];   // accepted, but never run by the auxiliary model
     pend[np++] = bonus;
     s.aux_npend[seq] = np;
 }

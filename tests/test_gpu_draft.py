@@ -15,22 +15,39 @@ pytestmark = pytest.mark.gpu
 W = S.WORKLOADS["tiny"]
 
 
-def _draft_gpu(gm, seq, gamma, b, u):
-    N = gamma * b
+def draft_gap(keep_all: bool) -> float:
+    """Smallest gap between two consecutive perturbed scores of the oracle's draft below which the device's order of
+    them is not compared.  The plain tree orders b pairs a layer: 1e-3, the margin of every other decision.  With
+    every candidate kept a layer orders b * b of them, and the k-th and (k+1)-th largest of V Gumbel-perturbed scores
+    lie about 1/k apart, so some gap among gamma * b * b falls below 1e-3 in most drafts and that margin would skip
+    nearly every case.  The device's error on one perturbed score is that of an fp32 logit of the auxiliary model
+    (one narrow layer here: the node_logq comparison below measures at most 5e-6 against the fp64 oracle and asserts 2e-5
+    on it), so 1e-4 still leaves a factor of five."""
+    return 1e-4 if keep_all else 1e-3
+
+
+def _draft_gpu(gm, seq, gamma, b, u, keep_all=False):
+    N = gamma * (b * b if keep_all else b)
     i32 = dict(dtype=torch.int32, device="cuda")
     f32 = dict(dtype=torch.float32, device="cuda")
     out = {"tok": torch.zeros(1, N, **i32), "parent": torch.zeros(1, N, **i32), "depth": torch.zeros(1, N, **i32),
            "node_logq": torch.zeros(1, N, **f32), "logq_ref": torch.zeros(1, gamma, **f32),
-           "best_path": torch.zeros(1, gamma, **i32)}
+           "best_path": torch.zeros(1, gamma, **i32), "n_nodes": torch.full((1,), -7, **i32)}
     gm.ctx.mtad_draft([seq], gamma, b, u, out["tok"], out["parent"], out["depth"], out["node_logq"], out["logq_ref"],
-                      out["best_path"])
+                      out["best_path"], keep_all_candidates=keep_all, n_nodes=out["n_nodes"])
     torch.cuda.synchronize()
+    assert out["n_nodes"].tolist() == [N]
     return out
 
 
-@pytest.mark.parametrize("gamma,b,chain", [(4, 4, False), (3, 2, True), (4, 1, True), (2, 8, False)])
-def test_draft_verify_commit_iterations(gamma, b, chain):
-    gm = GpuModel(W.target, max_batch=2, max_nodes=40, capacity=256, aux=W.aux, aux_capacity=256)
+# the last four keep every candidate of the beam sampling: 64-, 12- and 128-node trees (Sec. 3.3 with the tree sizes
+# of the full-size workloads), and the output sequence of such a draft verified as a chain
+@pytest.mark.parametrize("gamma,b,chain,keep_all", [(4, 4, False, False), (3, 2, True, False), (4, 1, True, False),
+                                                    (2, 8, False, False), (4, 4, False, True), (3, 2, False, True),
+                                                    (2, 8, False, True), (3, 3, True, True)])
+def test_draft_verify_commit_iterations(gamma, b, chain, keep_all):
+    N = gamma * (b * b if keep_all else b)
+    gm = GpuModel(W.target, max_batch=2, max_nodes=max(40, N), capacity=320, aux=W.aux, aux_capacity=320)
     seq, L = 1, 24
     gm.inject(seq, L)
     gm.inject_aux(seq, L)
@@ -41,32 +58,38 @@ def test_draft_verify_commit_iterations(gamma, b, chain):
     La, pend = L, [root]
     V = W.target.vocab
     skipped = 0
+    leaves = 0                  # accepted paths that end in a node the auxiliary model never ran
+    lq_err = 0.0
     for it in range(6):
         u = S.uniforms(0, (31 << 40) | (it * 16 + gamma), gamma * b * V, "cuda").view(1, gamma, b, V)
-        g = _draft_gpu(gm, seq, gamma, b, u)
-        dr = O.draft_beam(gm.oracle_aux(), acache, La, pend, gamma, b, u[0].cpu().numpy())
-        near = dr.min_gap < 1e-3
+        g = _draft_gpu(gm, seq, gamma, b, u, keep_all)
+        dr = O.draft_beam(gm.oracle_aux(), acache, La, pend, gamma, b, u[0].cpu().numpy(), keep_all=keep_all)
+        assert len(dr.tok) == N
+        near = dr.min_gap < draft_gap(keep_all)
         if not near:
             assert g["tok"][0].tolist() == dr.tok and g["parent"][0].tolist() == dr.parent
             assert g["depth"][0].tolist() == dr.depth and g["best_path"][0].tolist() == dr.best_path
+            lq_err = max(lq_err, float(np.max(np.abs(g["node_logq"][0].cpu().numpy() - np.asarray(dr.logq)))))
             assert np.max(np.abs(g["node_logq"][0].cpu().numpy() - np.asarray(dr.logq))) < LP_TOL
             assert np.max(np.abs(g["logq_ref"][0].cpu().numpy() - np.asarray(dr.logq_ref))) < LP_TOL
-        # verify what the oracle drafted (teacher forcing keeps both sides on one trajectory)
+        # The device verifies its own draft, straight from the arrays mtad_draft wrote; next to a tie of the draft
+        # it gets the oracle's instead (and its caches are put back on the oracle's trajectory afterwards).
         bu = S.bonus_uniforms(9, it, 1, V, "cuda")
         log_tau = math.log(0.3)
         ref = np.asarray(dr.logq_ref, np.float32)
+        d_ref = g["logq_ref"] if not near else torch.tensor(ref, device="cuda").view(1, -1)
         if chain:
             toks = [dr.tok[n] for n in dr.best_path]
             res = M.ResultBuffers(1, gamma, gamma)
-            gm.ctx.mtad_verify_chain([seq], gamma, torch.tensor(toks, dtype=torch.int32, device="cuda"),
-                                     torch.tensor(ref, device="cuda"), log_tau, bu, res)
+            gm.ctx.mtad_verify_chain([seq], gamma, torch.tensor(toks, dtype=torch.int32, device="cuda"), d_ref,
+                                     log_tau, bu, res)
             r = O.verify_chain(gm.oracle(), tcache, L, root, toks, ref.astype(np.float64), log_tau, bu[0].cpu().numpy())
             accepted = [dr.best_path[i] for i in r.path]
         else:
-            res = M.ResultBuffers(1, gamma * b, gamma)
-            gm.ctx.mtad_verify_tree([seq], None, gamma * b, gamma, torch.tensor(dr.tok, dtype=torch.int32, device="cuda"),
-                                    torch.tensor(dr.parent, dtype=torch.int32, device="cuda"),
-                                    torch.tensor(ref, device="cuda"), log_tau, bu, res)
+            res = M.ResultBuffers(1, N, gamma)
+            d_tok = g["tok"] if not near else torch.tensor(dr.tok, dtype=torch.int32, device="cuda")
+            d_par = g["parent"] if not near else torch.tensor(dr.parent, dtype=torch.int32, device="cuda")
+            gm.ctx.mtad_verify_tree([seq], g["n_nodes"], N, gamma, d_tok, d_par, d_ref, log_tau, bu, res)
             r = O.verify_tree(gm.oracle(), tcache, L, root, dr.tok, dr.parent, ref.astype(np.float64), log_tau,
                               bu[0].cpu().numpy())
             accepted = list(r.path)
@@ -76,6 +99,7 @@ def test_draft_verify_commit_iterations(gamma, b, chain):
         tie = min(r.margin_accept, r.margin_tie, r.margin_bonus) < 1e-3
         L = O.kv_commit(tcache, L, r.path)
         La, pend = O.aux_commit(acache, La, pend, dr, accepted, r.out_tok[-1], gamma)
+        leaves += len(pend) == 2
         root = r.out_tok[-1]
         if near or tie:
             # a decision within 1e-3 of a tie may legitimately differ: put the device back on the oracle's trajectory
@@ -85,7 +109,10 @@ def test_draft_verify_commit_iterations(gamma, b, chain):
             continue
         assert int(h["eta"][0]) == r.eta and h["out_tok"][0, :r.eta + 1].tolist() == r.out_tok
         assert gm.ctx.mtad_seq_get(seq) == (L, root)
-    assert skipped <= 3
+    print(f"keep_all={keep_all} gamma={gamma} b={b}: skipped {skipped}, paths ending in a not-run node {leaves}, "
+          f"largest node_logq error {lq_err:.2e}")
+    assert skipped <= 3 and lq_err < 2e-5
+    assert gm.ctx.mtad_debug_check_canaries() == ""
 
 
 def test_draft_wide_vocabulary():
@@ -126,19 +153,21 @@ def test_draft_rejects_bad_arguments():
     assert c.mtad_draft([0], 4, 9, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_CAPACITY
     assert c.mtad_draft([0], 33, 1, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_CAPACITY
     assert c.mtad_draft([3], 4, 4, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_INVALID
+    # every candidate kept: gamma * b * b nodes must fit a verify call
+    assert c.mtad_draft([0], 4, 8, u, t, t, t, f, f, t, check=False, keep_all_candidates=True) == M.binding.MTAD_E_CAPACITY
     no_aux = GpuModel(W.target, max_batch=1, max_nodes=8, capacity=64)
     assert no_aux.ctx.mtad_draft([0], 4, 4, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_INVALID
 
 
-def _draft_gpu_batch(gm, seqs, gamma, b, u):
-    B, N = len(seqs), gamma * b
+def _draft_gpu_batch(gm, seqs, gamma, b, u, keep_all=False):
+    B, N = len(seqs), gamma * (b * b if keep_all else b)
     i32 = dict(dtype=torch.int32, device="cuda")
     f32 = dict(dtype=torch.float32, device="cuda")
     out = {"tok": torch.zeros(B, N, **i32), "parent": torch.zeros(B, N, **i32), "depth": torch.zeros(B, N, **i32),
            "node_logq": torch.zeros(B, N, **f32), "logq_ref": torch.zeros(B, gamma, **f32),
-           "best_path": torch.zeros(B, gamma, **i32)}
+           "best_path": torch.zeros(B, gamma, **i32), "n_nodes": torch.zeros(B, **i32)}
     gm.ctx.mtad_draft(seqs, gamma, b, u, out["tok"], out["parent"], out["depth"], out["node_logq"], out["logq_ref"],
-                      out["best_path"])
+                      out["best_path"], keep_all_candidates=keep_all, n_nodes=out["n_nodes"])
     torch.cuda.synchronize()
     return out
 
@@ -148,12 +177,21 @@ def test_batched_draft_verify_commit_iterations(B, gamma, b):
     batched_iterations(W.target, W.aux, [10 + 7 * s for s in range(B)], gamma, b, 256, 256, 4)
 
 
-def batched_iterations(target, aux, lens, gamma, b, capacity, aux_capacity, iters):
-    """Several ragged sequences per mtad_draft call, each followed by a chain verification and a commit of all of
-    them (Algorithm 1 for a batch), teacher-forced on the oracle's draft_beam / verify_chain / aux_commit per
-    sequence; the guard bytes behind every workspace array must be intact afterwards."""
+@pytest.mark.parametrize("B,gamma,b,keep_all", [(2, 3, 3, False), (3, 4, 4, True), (2, 3, 2, True)])
+def test_batched_draft_tree_verify_commit_iterations(B, gamma, b, keep_all):
+    """MMTAD for a batch (Sec. 3.3): the tree that mtad_draft wrote goes to mtad_verify_tree as it lies on the device."""
+    batched_iterations(W.target, W.aux, [10 + 7 * s for s in range(B)], gamma, b, 320, 320, 4, tree=True,
+                       keep_all=keep_all)
+
+
+def batched_iterations(target, aux, lens, gamma, b, capacity, aux_capacity, iters, tree=False, keep_all=False):
+    """Several ragged sequences per mtad_draft call, each followed by a verification (of the output sequences as
+    chains: Algorithm 1 for a batch; with `tree` of the whole draft trees, read from the arrays mtad_draft wrote) and
+    a commit of all of them, teacher-forced on the oracle's draft_beam / verify / aux_commit per sequence; the guard
+    bytes behind every workspace array must be intact afterwards."""
     B = len(lens)
-    gm = GpuModel(target, max_batch=B, max_nodes=max(gamma * b, gamma), capacity=capacity, aux=aux,
+    N = gamma * (b * b if keep_all else b)
+    gm = GpuModel(target, max_batch=B, max_nodes=max(N, gamma), capacity=capacity, aux=aux,
                   aux_capacity=aux_capacity)
     V = target.vocab
     seqs = list(range(B))
@@ -170,32 +208,48 @@ def batched_iterations(target, aux, lens, gamma, b, capacity, aux_capacity, iter
     log_tau = math.log(0.3)
     for it in range(iters):
         u = S.uniforms(0, (35 << 40) | (it * 64 + B), B * gamma * b * V, "cuda").view(B, gamma, b, V)
-        g = _draft_gpu_batch(gm, seqs, gamma, b, u)
+        g = _draft_gpu_batch(gm, seqs, gamma, b, u, keep_all)
         bu = S.bonus_uniforms(11, it, B, V, "cuda")
         drafts, near = [], []
         for s in seqs:
             st = state[s]
-            dr = O.draft_beam(gm.oracle_aux(), st["ac"], st["La"], st["pend"], gamma, b, u[s].cpu().numpy())
+            dr = O.draft_beam(gm.oracle_aux(), st["ac"], st["La"], st["pend"], gamma, b, u[s].cpu().numpy(),
+                              keep_all=keep_all)
             drafts.append(dr)
-            near.append(dr.min_gap < 1e-3)
+            near.append(dr.min_gap < draft_gap(keep_all))
             if not near[-1]:
                 assert g["tok"][s].tolist() == dr.tok and g["parent"][s].tolist() == dr.parent, (it, s)
                 assert g["best_path"][s].tolist() == dr.best_path
                 assert np.max(np.abs(g["node_logq"][s].cpu().numpy() - np.asarray(dr.logq))) < LP_TOL
                 assert np.max(np.abs(g["logq_ref"][s].cpu().numpy() - np.asarray(dr.logq_ref))) < LP_TOL
-        toks = torch.tensor([[dr.tok[n] for n in dr.best_path] for dr in drafts], dtype=torch.int32, device="cuda")
         ref = torch.tensor([dr.logq_ref for dr in drafts], dtype=torch.float32, device="cuda")
-        res = M.ResultBuffers(B, gamma, gamma)
-        gm.ctx.mtad_verify_chain(seqs, gamma, toks, ref, log_tau, bu, res)
+        if tree:
+            # sequences next to a tie of the draft get the oracle's tree (they are put back on its trajectory below)
+            for s in seqs:
+                if near[s]:
+                    g["tok"][s] = torch.tensor(drafts[s].tok, dtype=torch.int32, device="cuda")
+                    g["parent"][s] = torch.tensor(drafts[s].parent, dtype=torch.int32, device="cuda")
+            res = M.ResultBuffers(B, N, gamma)
+            gm.ctx.mtad_verify_tree(seqs, g["n_nodes"], N, gamma, g["tok"], g["parent"], ref, log_tau, bu, res)
+        else:
+            toks = torch.tensor([[dr.tok[n] for n in dr.best_path] for dr in drafts], dtype=torch.int32, device="cuda")
+            res = M.ResultBuffers(B, gamma, gamma)
+            gm.ctx.mtad_verify_chain(seqs, gamma, toks, ref, log_tau, bu, res)
         gm.ctx.kv_commit(seqs, res)
         h = res.host()
         for s in seqs:
             st, dr = state[s], drafts[s]
             assert int(h["status"][s]) == 0
-            r = O.verify_chain(gm.oracle(), st["tc"], st["L"], st["root"], [dr.tok[n] for n in dr.best_path],
-                               np.asarray(dr.logq_ref, np.float32).astype(np.float64), log_tau, bu[s].cpu().numpy())
+            ref64 = np.asarray(dr.logq_ref, np.float32).astype(np.float64)
+            if tree:
+                r = O.verify_tree(gm.oracle(), st["tc"], st["L"], st["root"], dr.tok, dr.parent, ref64, log_tau,
+                                  bu[s].cpu().numpy())
+                accepted = list(r.path)
+            else:
+                r = O.verify_chain(gm.oracle(), st["tc"], st["L"], st["root"], [dr.tok[n] for n in dr.best_path],
+                                   ref64, log_tau, bu[s].cpu().numpy())
+                accepted = [dr.best_path[i] for i in r.path]
             tie = min(r.margin_accept, r.margin_tie, r.margin_bonus) < 1e-3
-            accepted = [dr.best_path[i] for i in r.path]
             st["L"] = O.kv_commit(st["tc"], st["L"], r.path)
             st["La"], st["pend"] = O.aux_commit(st["ac"], st["La"], st["pend"], dr, accepted, r.out_tok[-1], gamma)
             st["root"] = r.out_tok[-1]

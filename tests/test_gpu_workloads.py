@@ -98,3 +98,14 @@ def test_13b_pair_batched_draft_two_layers():
     w = S.WORKLOADS["13b_batched_chain"]
     shape = dataclasses.replace(w.target, layers=2)
     batched_iterations(shape, w.aux, S.kv_lengths(w), w.gamma, 4, 4160, 4160, 2)
+
+
+def test_7b_pair_drafted_tree_two_layers():
+    """MMTAD end to end at the 7B-shaped pair (Sec. 3.3): the full-size auxiliary model (2 layers, 768 wide) drafts
+    with beam width 4 for gamma 4 and keeps every candidate - the 64-node tree of the tree workload -, the target (cut
+    to two layers so that the oracle stays affordable) verifies that tree from the arrays mtad_draft wrote, kv_commit
+    rolls both caches forward; two iterations at 2048 committed tokens, against the oracle."""
+    from tests.test_gpu_draft import batched_iterations
+    w = S.WORKLOADS["7b_tree"]
+    shape = dataclasses.replace(w.target, layers=2)
+    batched_iterations(shape, w.aux, [2048], w.gamma, 4, 2048 + 160, 2048 + 160, 2, tree=True, keep_all=True)
