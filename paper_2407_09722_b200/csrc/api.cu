@@ -432,13 +432,18 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
     base.hidden = sc.hidden; base.R = R; base.prow = rm.prow; base.tok = rm.tok; base.node_z = sc.node_z;
     base.lm_part = sc.lm_part;
     const double wb = 2.0;
-    // Calls of up to 32 rows run the projections whose tiles fill the CTA slots as clusters that reduce over
-    // distributed shared memory (tc_gemm_cluster.cu): QKV, O, down and the LM head; gate / up, with more tiles than
-    // half the CTA slots, keeps the stream-K decomposition, which balances it better.
-    auto clusterize = [&](TcGemmParams& p, int n_tiles, int K, bool want) -> bool {
-        if (!want || mh != 1) return false;
+    // The projections whose tiles fit the co-resident CTAs run as clusters that reduce over distributed shared memory
+    // (tc_gemm_cluster.cu): QKV, O, down and, with few rows, the LM head; gate / up, with more tiles than half the CTA
+    // slots, keeps the stream-K decomposition, which balances it better.  The plan picks the halves per tile itself.
+    auto clusterize = [&](TcGemmParams& p, int n_tiles128, int K, bool want) -> bool {
+        if (!want) return false;
         TcGemmParams q = p;
-        if (!tc_cluster_plan(q, n_tiles, K, T, 2 * kCtas)) return false;
+        if (!tc_cluster_plan(q, n_tiles128, K, T, kCtas)) return false;
+        static const int big_mask = getenv("MTAD_TC_CLBIG") ? atoi(getenv("MTAD_TC_CLBIG")) : 31;   // experiment knob
+        if (q.per_sm == 1) {
+            const int bit = p.mode == TC_QKV ? 1 : (p.mode == TC_RESID ? (K == d.d_ffn ? 8 : 2) : 16);
+            if (!(big_mask & bit)) return false;
+        }
         p = q;
         return true;
     };
@@ -458,9 +463,9 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
             p.mh = mq; p.n_rows_total = n128 * 128;
             p.mode = TC_QKV; p.N = qd; p.seg_k_tile = qt; p.seg_v_tile = qt + kt; p.layer = l;
             p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = (l == 0) ? 1 : dt;
-            if (with_maps) { mp.a0 = wmap(wm->wq, mq, l); mp.a1 = wmap(wm->wk, mq, l); mp.a2 = wmap(wm->wv, mq, l); }
+            const bool cl = clusterize(p, n128, d.d_model, true);
+            if (with_maps) { mp.a0 = wmap(wm->wq, p.mh, l); mp.a1 = wmap(wm->wk, p.mh, l); mp.a2 = wmap(wm->wv, p.mh, l); }
             mp.x = xd;
-            const bool cl = mq == 1 && clusterize(p, n128, d.d_model, true);
             g.push_back({mp, p, wb * (qd + (split_kv ? 0.0 : 2.0 * kvd)) * d.d_model, cl, false});
         }
         if (split_kv) {   // K and V rows: three-term input, short accumulation chains
@@ -481,9 +486,9 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
             p.mode = TC_RESID; p.N = d.d_model; p.sumsq_in_parts = 0;
             p.gain = m.w(l, 5); p.x_out = sc.xd; p.xk = d.d_model;
             p.sumsq_out = sc.sumsq_b;
-            if (with_maps) mp.a0 = wmap(wm->wo, mh, l);
-            mp.x = xa;
             const bool cl = clusterize(p, up(d.d_model, 128), qd, true);
+            if (with_maps) mp.a0 = wmap(wm->wo, p.mh, l);
+            mp.x = xa;
             g.push_back({mp, p, wb * d.d_model * qd, cl, true});
         }
         {   // gate / up + SwiGLU
@@ -504,9 +509,9 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
             p.gain = (l + 1 < d.layers) ? m.w(l + 1, 0) : static_cast<const __nv_bfloat16*>(d.final_norm);
             p.x_out = sc.xd; p.xk = d.d_model; p.sumsq_out = sc.sumsq_a;
             if (split_kv && l + 1 < d.layers) { p.x_out2 = sc.xkv; p.out_terms2 = tkv; }
-            if (with_maps) mp.a0 = wmap(wm->down, mh, l);
-            mp.x = xf;
             const bool cl = clusterize(p, up(d.d_model, 128), d.d_ffn, true);
+            if (with_maps) mp.a0 = wmap(wm->down, p.mh, l);
+            mp.x = xf;
             g.push_back({mp, p, wb * d.d_model * d.d_ffn, cl, false});
         }
     }
@@ -517,10 +522,10 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
         p.mh = mh; p.n_rows_total = d.vocab; p.n_tiles128 = up(d.vocab, 128);
         p.mode = lm_plain ? TC_PLAIN : TC_LMHEAD; p.N = d.vocab; p.sumsq_in = sc.sumsq_a; p.sumsq_in_parts = dt;
         p.out = sc.logits; p.ldo = d.vocab;
-        if (with_maps) mp.a0 = wm->lm_head[ix(mh)];
-        mp.x = xd;
         fp.lm_tiles128 = p.n_tiles128;
         const bool cl = clusterize(p, up(d.vocab, 128), d.d_model, true);
+        if (with_maps) mp.a0 = wm->lm_head[ix(p.mh)];
+        mp.x = xd;
         g.push_back({mp, p, wb * d.vocab * d.d_model, cl, false});
     }
     fp.maps = with_maps;
@@ -797,7 +802,8 @@ int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, 
     RUN(MTAD_K_PREPARE, 0, 1, launch_split_rows(x, K, ctx->sc.xf, p.terms, T, K, s));
     static const int cluster_mask = getenv("MTAD_TC_CLUSTER") ? atoi(getenv("MTAD_TC_CLUSTER")) : 27;
     TcGemmParams q = p;
-    if (mh == 1 && ((cluster_mask >> 5) & 1) && tc_cluster_plan(q, p.n_tiles, K, T, 2 * kCtas)) {
+    if (((cluster_mask >> 5) & 1) && tc_cluster_plan(q, (N + TC_TILE_N - 1) / TC_TILE_N, K, T, kCtas)) {
+        if (q.mh != mh && tc_make_map(&mp.a0, W, N, K, q.mh == 1 ? 128 : 256)) return MTAD_E_CUDA;
         RUN(MTAD_K_GEMM, 2.0 * N * K, 1, launch_tc_cluster(mp, q, false, s));
         return MTAD_OK;
     }

@@ -152,6 +152,10 @@ __global__ void __launch_bounds__(CNT == 4 ? 192 : 128, CNT == 1 ? 4 : (CNT == 4
     // the two products of its query row: half the MMAs, one softmax row per thread
     constexpr bool packed = PACK;
     const int kt0 = (warp % kparts) * cnt;            // first 16-key group of this warp's tasks
+    // whole-tile mode with a warp for every query tile: the warp keeps its tile's running softmax state and output in
+    // registers over all key tiles of the block and writes one partial at the end; with more query tiles than warps
+    // the block owns a single key tile (the launch sets nsp = 1) and every (query tile, key tile) is a partial
+    const bool persist = kparts == 1 && n_mt <= (int)(blockDim.x >> 5);
 
     // query tile mt -> slab (16-byte async copies by `nthr` threads; rows past the last query are zero-filled)
     auto stage_q = [&](int mt, int slab, int tid, int nthr) {
@@ -278,7 +282,7 @@ __global__ void __launch_bounds__(CNT == 4 ? 192 : 128, CNT == 1 ? 4 : (CNT == 4
             asm volatile("cp.async.wait_all;" ::: "memory");
             __syncwarp();
         }
-        if (kparts == 1) {                            // whole tiles: one key tile per block, fresh state per query tile
+        if (kparts == 1 && (t == 0 || !persist)) {    // whole tiles: fresh state, unless this warp keeps its one query tile
             m0 = -CUDART_INF_F; m1 = -CUDART_INF_F; l0 = 0.f; l1 = 0.f;
 #pragma unroll
             for (int n = 0; n < NDT; ++n)
@@ -420,6 +424,7 @@ __global__ void __launch_bounds__(CNT == 4 ? 192 : 128, CNT == 1 ? 4 : (CNT == 4
             }
         }
         if (kparts > 1) break;                        // one task per warp: merged below
+        if (persist && tile + 1 < tile_end) break;    // the warp's query tile goes on to the block's next key tile
         // ---- partials of the valid rows ----
         if (qi0 < n_q) {
             const int h = g * G + qi0 / nrows, r = qi0 % nrows;
@@ -509,7 +514,13 @@ int attention_mma_tiles_per_block(const ModelView& m, int B, int R, long long ke
     // with at most two query tiles per KV head a block walks several 64-key tiles, all blocks resident in a single
     // wave (two per SM with a ring of three buffers at head_dim 128, else three); larger trees take one tile per block
     const int n_mt_max = ((m.d.n_q_heads / m.d.n_kv_heads) * R + 15) / 16;
-    if (n_mt_max > 2) return 1;
+    if (n_mt_max > 6) return 1;
+    if (n_mt_max > 2) {
+        // three to six query tiles: a warp per tile, two K/V buffers, two blocks per SM, all blocks in one wave
+        const long long tiles = (keys + KT - 1) / KT * m.d.n_kv_heads * B;
+        const long long nsp = (tiles + 2 * 148 - 1) / (2 * 148);
+        return (int)(nsp < 1 ? 1 : (nsp > 64 ? 64 : nsp));
+    }
     const int ring = attn_ring(m.d.head_dim, n_mt_max, (long long)m.d.n_kv_heads * B);
     const int per_sm = (ring == 3 && m.d.head_dim == 128) ? 2 : 3;
     const long long tiles = (keys + KT - 1) / KT * m.d.n_kv_heads * B;
@@ -527,7 +538,8 @@ cudaError_t launch_attention_mma(const ModelView& m, int layer, const RowMeta& r
     // (a 64-node tree plus its root is five tiles)
     const int n_warps = (n_mt_max == 5 || n_mt_max == 6) ? n_mt_max : 4;
     const int nslab = n_mt_max <= 2 ? n_mt_max : n_warps;
-    const int ring = attn_ring(hd, nslab, (long long)Hkv * B);
+    if (n_mt_max > n_warps && nsp != 1) return cudaErrorInvalidValue;     // query tiles in rounds: one key tile per block
+    const int ring = n_mt_max > 2 ? 2 : attn_ring(hd, nslab, (long long)Hkv * B);
     const int nb = nsp == 1 ? 1 : (nsp == 2 ? 2 : ring);
     const size_t smem = attn_smem(hd, nslab, nb);
     const int early = layer > 0 ? 1 : 0;              // the row metadata was final before the previous kernel started

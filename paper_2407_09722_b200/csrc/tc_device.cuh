@@ -137,7 +137,44 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// 32 consecutive columns of this warp's TMEM lanes
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// ---- thread-block clusters ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_arrive_release() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait_acquire() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// fp32 store into the shared memory of CTA `rank` of this cluster, at the address that `local_addr` has in this CTA
+__device__ __forceinline__ void st_cluster_f32(uint32_t local_addr, uint32_t rank, float v) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+
+// barrier of one group of 128 epilogue threads (id 1, or 1 and 2 where a kernel has two groups)
+__device__ __forceinline__ void epi_bar(int id = 1) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
 
 // two-term split of the query rows for the tensor-core attention
 __device__ __forceinline__ void split_store(float y, __nv_bfloat16* hi, __nv_bfloat16* lo) {
@@ -216,19 +253,22 @@ constexpr size_t SMEM_TAIL = sizeof(float) * MAX_HALVES * EPI_ROWS * (TC_TILE_N 
                              sizeof(float4) * 4 * EPI_ROWS * 2 + 8 * MAX_STAGES * 2 + 16 + 16 + 8 + 8 + 32;
 
 // ---------------------------------------------------------------------------------------------------------------
-// epilogues: called by the 128 epilogue threads for a block of EPI_ROWS finished rows of one 128-feature tile held
-// in epi[j][i] (j: row r0 + j, i: feature tile * 128 + i).  e = epilogue thread index 0..127.
+// epilogues: called by the 128 epilogue threads for a block of ROWS finished rows (a template parameter: 8, or 16 where
+// shared memory allows and there are many rows) of one 128-feature tile held in epi[j][i] (j: row r0 + j, i: feature
+// tile * 128 + i).  e = epilogue thread index 0..127.
 typedef float (*EpiTile)[TC_TILE_N + 1];
 // ---------------------------------------------------------------------------------------------------------------
 
+template <int ROWS>
 __device__ __forceinline__ void epi_plain(const TcGemmParams& p, EpiTile epi, int tile, int r0, int t_end, int e) {
     const int n = tile * TC_TILE_N + e;
     if (n >= p.N) return;
-    for (int j = 0; j < EPI_ROWS && r0 + j < t_end; ++j) p.out[(size_t)(r0 + j) * p.ldo + n] = epi[j][e];
+    for (int j = 0; j < ROWS && r0 + j < t_end; ++j) p.out[(size_t)(r0 + j) * p.ldo + n] = epi[j][e];
 }
 
-// The epilogues below first issue the global loads of all EPI_ROWS rows, then compute: a finished tile is the end of
+// The epilogues below first issue the global loads of all ROWS rows, then compute: a finished tile is the end of
 // a dependency chain (the next kernel waits for it), so one L2 round trip per pass instead of one per row matters.
+template <int ROWS>
 __device__ __forceinline__ void epi_qkv(const TcGemmParams& p, EpiTile epi, int tile, int r0, int t_end, int e) {
     const int hd = p.hd, half = hd >> 1;
     int seg, tin;
@@ -243,10 +283,10 @@ __device__ __forceinline__ void epi_qkv(const TcGemmParams& p, EpiTile epi, int 
     const float scale = rsqrtf((float)hd);
     const bool rot = seg != 2 && jin < half;          // this thread rotates the pair (jin, jin + half)
     if (seg != 2 && !rot) return;
-    int sl[EPI_ROWS], sq[EPI_ROWS];
-    float2 cs[EPI_ROWS];
+    int sl[ROWS], sq[ROWS];
+    float2 cs[ROWS];
 #pragma unroll
-    for (int j = 0; j < EPI_ROWS; ++j) {
+    for (int j = 0; j < ROWS; ++j) {
         const int t = r0 + j;
         const bool valid = t < t_end;
         sl[j] = (valid && seg != 0) ? p.slot[t] : (valid ? 0 : -1);
@@ -255,7 +295,7 @@ __device__ __forceinline__ void epi_qkv(const TcGemmParams& p, EpiTile epi, int 
                                : make_float2(1.f, 0.f);
     }
 #pragma unroll
-    for (int j = 0; j < EPI_ROWS; ++j) {
+    for (int j = 0; j < ROWS; ++j) {
         const int t = r0 + j;
         if (sl[j] < 0) continue;                      // row beyond T, or an inactive row (no cache slot)
         if (seg != 0 && (sl[j] >= p.cap || (unsigned)sq[j] >= (unsigned)p.max_batch)) continue;   // never past the cache
@@ -285,18 +325,19 @@ __device__ __forceinline__ void epi_qkv(const TcGemmParams& p, EpiTile epi, int 
     }
 }
 
+template <int ROWS>
 __device__ __forceinline__ void epi_resid(const TcGemmParams& p, float* red, EpiTile epi, int tile, int r0,
-                                          int t_end, int e) {
+                                          int t_end, int e, int bar = 1) {
     const int n = tile * TC_TILE_N + e;
     const bool ok = n < p.N;
     const float g = ok ? __bfloat162float(p.gain[n]) : 0.f;
     const int warp = e >> 5, lane = e & 31;
-    float y[EPI_ROWS];
+    float y[ROWS];
 #pragma unroll
-    for (int j = 0; j < EPI_ROWS; ++j)
+    for (int j = 0; j < ROWS; ++j)
         y[j] = (ok && r0 + j < t_end) ? __ldcg(p.hidden + (size_t)(r0 + j) * p.N + n) : 0.f;
 #pragma unroll
-    for (int j = 0; j < EPI_ROWS; ++j) {
+    for (int j = 0; j < ROWS; ++j) {
         const int t = r0 + j;
         if (ok && t < t_end) {
             y[j] += epi[j][e];
@@ -309,26 +350,27 @@ __device__ __forceinline__ void epi_resid(const TcGemmParams& p, float* red, Epi
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
-        for (int j = 0; j < EPI_ROWS; ++j) y[j] += __shfl_xor_sync(0xffffffffu, y[j], o);
+        for (int j = 0; j < ROWS; ++j) y[j] += __shfl_xor_sync(0xffffffffu, y[j], o);
     if (lane == 0) {
 #pragma unroll
-        for (int j = 0; j < EPI_ROWS; ++j) red[warp * EPI_ROWS + j] = y[j];
+        for (int j = 0; j < ROWS; ++j) red[warp * ROWS + j] = y[j];
     }
-    epi_bar();
-    if (e < EPI_ROWS && r0 + e < t_end)
+    epi_bar(bar);
+    if (e < ROWS && r0 + e < t_end)
         p.sumsq_out[(size_t)tile * TC_X_ROWS + r0 + e] =
-            (red[e] + red[EPI_ROWS + e]) + (red[2 * EPI_ROWS + e] + red[3 * EPI_ROWS + e]);
-    epi_bar();       // the scratch is reused by the next tile half
+            (red[e] + red[ROWS + e]) + (red[2 * ROWS + e] + red[3 * ROWS + e]);
+    epi_bar(bar);       // the scratch is reused by the next tile half
 }
 
-__device__ __forceinline__ void epi_swiglu(const TcGemmParams& p, float (*epi)[EPI_ROWS][TC_TILE_N + 1], int tile, int r0, int t_end,
+template <int ROWS>
+__device__ __forceinline__ void epi_swiglu(const TcGemmParams& p, float (*epi)[ROWS][TC_TILE_N + 1], int tile, int r0, int t_end,
                                            int e) {
     // the first half of a tile's weight rows are gate rows, the second half the matching up rows
     if (p.mh == 1) {
         if (e >= 64) return;
         const int f = tile * 64 + e;
         if (f >= p.N) return;
-        for (int j = 0; j < EPI_ROWS && r0 + j < t_end; ++j) {
+        for (int j = 0; j < ROWS && r0 + j < t_end; ++j) {
             const float g = epi[0][j][e], u = epi[0][j][e + 64];
             store_terms(g / (1.f + expf(-g)) * u, p.x_out + (size_t)(r0 + j) * p.out_terms * p.xk + f, p.xk, p.out_terms);
         }
@@ -338,31 +380,32 @@ __device__ __forceinline__ void epi_swiglu(const TcGemmParams& p, float (*epi)[E
     for (int h = 0; h < hh; ++h) {
         const int f = tile * 64 * p.mh + h * TC_TILE_N + e;
         if (f >= p.N) break;
-        for (int j = 0; j < EPI_ROWS && r0 + j < t_end; ++j) {
+        for (int j = 0; j < ROWS && r0 + j < t_end; ++j) {
             const float g = epi[h][j][e], u = epi[h + hh][j][e];
             store_terms(g / (1.f + expf(-g)) * u, p.x_out + (size_t)(r0 + j) * p.out_terms * p.xk + f, p.xk, p.out_terms);
         }
     }
 }
 
+template <int ROWS>
 __device__ __forceinline__ void epi_lmhead(const TcGemmParams& p, float4* red4, EpiTile epi, int tile, int r0,
-                                           int t_end, int e) {
+                                           int t_end, int e, int bar = 1) {
     const int v = tile * TC_TILE_N + e;
     const bool ok = v < p.N;
     const int warp = e >> 5, lane = e & 31;
     // Gumbel noise of this token: one draw per sequence, shared by all its rows
-    float u[EPI_ROWS];
+    float u[ROWS];
 #pragma unroll
-    for (int j = 0; j < EPI_ROWS; ++j) {
+    for (int j = 0; j < ROWS; ++j) {
         const int t = r0 + j;
         const bool fresh = j == 0 || t / p.R != (t - 1) / p.R;
         u[j] = (ok && t < t_end && fresh) ? p.uniforms[(size_t)(t / p.R) * p.N + v] : -1.f;
     }
-    float m[EPI_ROWS], sum[EPI_ROWS], bv[EPI_ROWS];
-    int bi[EPI_ROWS];
+    float m[ROWS], sum[ROWS], bv[ROWS];
+    int bi[ROWS];
     float gum = 0.f;
 #pragma unroll
-    for (int j = 0; j < EPI_ROWS; ++j) {
+    for (int j = 0; j < ROWS; ++j) {
         if (u[j] >= 0.f) gum = -logf(-logf(u[j]));
         const bool valid = ok && r0 + j < t_end;
         m[j] = valid ? epi[j][e] : -CUDART_INF_F;
@@ -374,27 +417,27 @@ __device__ __forceinline__ void epi_lmhead(const TcGemmParams& p, float4* red4, 
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
-        for (int j = 0; j < EPI_ROWS; ++j) {
+        for (int j = 0; j < ROWS; ++j) {
             m[j] = fmaxf(m[j], __shfl_xor_sync(0xffffffffu, m[j], o));
             const float v2 = __shfl_xor_sync(0xffffffffu, bv[j], o);
             const int i2 = __shfl_xor_sync(0xffffffffu, bi[j], o);
             if (v2 > bv[j] || (v2 == bv[j] && i2 < bi[j])) { bv[j] = v2; bi[j] = i2; }
         }
 #pragma unroll
-    for (int j = 0; j < EPI_ROWS; ++j) sum[j] = (sum[j] == -CUDART_INF_F) ? 0.f : expf(sum[j] - m[j]);
+    for (int j = 0; j < ROWS; ++j) sum[j] = (sum[j] == -CUDART_INF_F) ? 0.f : expf(sum[j] - m[j]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
-        for (int j = 0; j < EPI_ROWS; ++j) sum[j] += __shfl_xor_sync(0xffffffffu, sum[j], o);
+        for (int j = 0; j < ROWS; ++j) sum[j] += __shfl_xor_sync(0xffffffffu, sum[j], o);
     if (lane == 0) {
 #pragma unroll
-        for (int j = 0; j < EPI_ROWS; ++j) red4[warp * EPI_ROWS + j] = make_float4(m[j], sum[j], bv[j], __int_as_float(bi[j]));
+        for (int j = 0; j < ROWS; ++j) red4[warp * ROWS + j] = make_float4(m[j], sum[j], bv[j], __int_as_float(bi[j]));
     }
-    epi_bar();
-    if (e < EPI_ROWS && r0 + e < t_end) {
+    epi_bar(bar);
+    if (e < ROWS && r0 + e < t_end) {
         float4 a = red4[e];
         for (int w = 1; w < 4; ++w) {
-            const float4 b = red4[w * EPI_ROWS + e];
+            const float4 b = red4[w * ROWS + e];
             const float mm = fmaxf(a.x, b.x);
             const float sa = a.x == -CUDART_INF_F ? 0.f : a.y * expf(a.x - mm);
             const float sb = b.x == -CUDART_INF_F ? 0.f : b.y * expf(b.x - mm);
@@ -412,7 +455,7 @@ __device__ __forceinline__ void epi_lmhead(const TcGemmParams& p, float4* red4, 
         const int tk = p.tok[t] - n0;
         if (tk >= 0 && tk < TC_TILE_N) p.node_z[t] = epi[pr - r0][tk];
     }
-    epi_bar();       // the scratch is reused by the next tile half
+    epi_bar(bar);       // the scratch is reused by the next tile half
 }
 
 }  // namespace tcdev

@@ -387,16 +387,16 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
                         epi_bar();
                         const int t_end = min(T, r0 + EPI_ROWS);
                         if (p.mode == TC_SWIGLU) {
-                            epi_swiglu(p, s.epi, tile, r0, t_end, e);
+                            epi_swiglu<EPI_ROWS>(p, s.epi, tile, r0, t_end, e);
                         } else {
                             for (int h = 0; h < mh; ++h) {
                                 const int t128 = tile * mh + h;
                                 if (t128 * TC_TILE_N >= p.n_rows_total) break;      // half beyond the last weight row
                                 switch (p.mode) {
-                                    case TC_PLAIN: epi_plain(p, s.epi[h], t128, r0, t_end, e); break;
-                                    case TC_QKV: epi_qkv(p, s.epi[h], t128, r0, t_end, e); break;
-                                    case TC_RESID: epi_resid(p, s.red, s.epi[h], t128, r0, t_end, e); break;
-                                    default: epi_lmhead(p, s.red4, s.epi[h], t128, r0, t_end, e); break;
+                                    case TC_PLAIN: epi_plain<EPI_ROWS>(p, s.epi[h], t128, r0, t_end, e); break;
+                                    case TC_QKV: epi_qkv<EPI_ROWS>(p, s.epi[h], t128, r0, t_end, e); break;
+                                    case TC_RESID: epi_resid<EPI_ROWS>(p, s.red, s.epi[h], t128, r0, t_end, e); break;
+                                    default: epi_lmhead<EPI_ROWS>(p, s.red4, s.epi[h], t128, r0, t_end, e); break;
                                 }
                             }
                         }

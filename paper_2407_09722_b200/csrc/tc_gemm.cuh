@@ -41,6 +41,8 @@ struct TcGemmParams {
     unsigned long long* trace;   // MTAD_TRACE builds: [CTA][8] global-timer stamps of this launch, else null
     int csize;             // cluster kernel: CTAs that share a tile's k-range (1..8)
     int rpr;               // cluster kernel: rows per epilogue pass (1..8); pass q is finished by rank q % csize
+    int recv_alias;        // cluster kernel: the receive slots of the exchange lie over the copy ring
+    int ring_bytes;        // cluster kernel: shared memory below the fixed tail (set by the launch)
     int mode;
     int N;                 // output features (bound for stores)
     // Chained phases of one launch: a phase whose operand rows are written by the phase before it reads, per k-block,
@@ -122,11 +124,16 @@ int tc_ctas_per_sm(int T);
 int tc_halves(int T);
 size_t tc_workspace_floats(int n_tiles_max, int max_contrib_max, int rpad_max);
 
-// Cluster variant (tc_gemm_cluster.cu) for calls of up to 32 rows: a cluster of p.csize CTAs per 128-feature tile,
-// partial rows exchanged through distributed shared memory.  tc_cluster_plan fills the decomposition for n_tiles
-// tiles on `slots` co-resident CTAs and returns false when the shape does not suit it (too many rows, more tiles
-// than slots).
-bool tc_cluster_plan(TcGemmParams& p, int n_tiles, int K, int T, int slots);
+// Cluster variants: a cluster of p.csize CTAs per tile of p.mh 128-feature halves, partial rows exchanged through
+// distributed shared memory - tc_gemm_cluster.cu for calls of up to 32 rows (two CTAs on an SM, one half), and
+// tc_gemm_cluster_big.cu beyond (one CTA on an SM, two halves).  tc_cluster_plan fills the decomposition (halves per
+// tile, CTAs per SM, cluster size, rows per pass) for a matrix of n_tiles128 128-feature tiles on `sms` SMs and
+// returns false when the shape does not suit it (more than 256 accumulator columns, more tiles than co-resident
+// CTAs).  p.mode and, for QKV, the segment tiles must be set before the call: a tile never straddles q | k | v.  The
+// weight maps of the launch must have boxes of p.mh halves.
+bool tc_cluster_plan(TcGemmParams& p, int n_tiles128, int K, int T, int sms);
+bool tc_cluster_plan_small(TcGemmParams& p, int n_tiles, int K, int T, int slots);
+cudaError_t launch_tc_cluster_small(const TcMaps& maps, const TcGemmParams& p, bool pdl, cudaStream_t st);
 cudaError_t launch_tc_cluster(const TcMaps& maps, const TcGemmParams& p, bool pdl, cudaStream_t st);
 
 cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p, int ctas, bool pdl, cudaStream_t st);

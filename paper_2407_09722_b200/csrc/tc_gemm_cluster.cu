@@ -26,24 +26,6 @@ namespace {
 constexpr int CL_THREADS = 32 * 7;
 constexpr int CL_EPI_WARP0 = 3;
 
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_arrive_release() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void cluster_wait_acquire() {
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// fp32 store into the shared memory of CTA `rank` of this cluster, at the address that `local_addr` has in this CTA
-__device__ __forceinline__ void st_cluster_f32(uint32_t local_addr, uint32_t rank, float v) {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
-}
-
 struct ClSmem {
     uint8_t* ring;
     float (*epi)[TC_TILE_N + 1];   // [EPI_ROWS][feature]: the rows of the pass being finished
@@ -291,13 +273,13 @@ __global__ void __launch_bounds__(CL_THREADS, 2) tc_gemm_cluster_kernel(const __
             epi_bar();
             if (tile * TC_TILE_N < p.n_rows_total || p.mode == TC_SWIGLU) {
                 switch (p.mode) {
-                    case TC_PLAIN: epi_plain(p, s.epi, tile, r0, t_end, e); break;
-                    case TC_QKV: epi_qkv(p, s.epi, tile, r0, t_end, e); break;
-                    case TC_RESID: epi_resid(p, reinterpret_cast<float*>(s.red4), s.epi, tile, r0, t_end, e); break;
+                    case TC_PLAIN: epi_plain<EPI_ROWS>(p, s.epi, tile, r0, t_end, e); break;
+                    case TC_QKV: epi_qkv<EPI_ROWS>(p, s.epi, tile, r0, t_end, e); break;
+                    case TC_RESID: epi_resid<EPI_ROWS>(p, reinterpret_cast<float*>(s.red4), s.epi, tile, r0, t_end, e); break;
                     case TC_SWIGLU:
-                        epi_swiglu(p, reinterpret_cast<float(*)[EPI_ROWS][TC_TILE_N + 1]>(s.epi), tile, r0, t_end, e);
+                        epi_swiglu<EPI_ROWS>(p, reinterpret_cast<float(*)[EPI_ROWS][TC_TILE_N + 1]>(s.epi), tile, r0, t_end, e);
                         break;
-                    default: epi_lmhead(p, s.red4, s.epi, tile, r0, t_end, e); break;
+                    default: epi_lmhead<EPI_ROWS>(p, s.red4, s.epi, tile, r0, t_end, e); break;
                 }
             }
             epi_bar();
@@ -383,7 +365,7 @@ if (cudaFuncSetAttribute(cl_occupancy_probe_kernel, cudaFuncAttributeMaxDynamicS
 }
 }  // namespace
 
-bool tc_cluster_plan(TcGemmParams& p, int n_tiles, int K, int T, int slots) {
+bool tc_cluster_plan_small(TcGemmParams& p, int n_tiles, int K, int T, int slots) {
     p.n_tiles = n_tiles;
     p.k_blocks = (K + TC_TILE_K - 1) / TC_TILE_K;
     p.T = T;
@@ -410,7 +392,7 @@ bool tc_cluster_plan(TcGemmParams& p, int n_tiles, int K, int T, int slots) {
     return true;
 }
 
-cudaError_t launch_tc_cluster(const TcMaps& maps, const TcGemmParams& p_in, bool pdl, cudaStream_t st) {
+cudaError_t launch_tc_cluster_small(const TcMaps& maps, const TcGemmParams& p_in, bool pdl, cudaStream_t st) {
     TcGemmParams p = p_in;
     if (p.mh != 1 || p.csize < 1 || p.csize > 8 || p.rpr < 1 || p.rpr > EPI_ROWS) return cudaErrorInvalidValue;
     const int acc_cols = p.terms * p.rpad;
