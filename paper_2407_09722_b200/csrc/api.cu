@@ -497,9 +497,19 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
             p.mh = mh; p.n_rows_total = d.d_ffn;
             p.mode = TC_SWIGLU; p.N = d.d_ffn; p.sumsq_in = sc.sumsq_b; p.sumsq_in_parts = dt;
             p.x_out = sc.xf; p.xk = d.d_ffn;
-            if (with_maps) { mp.a0 = wmap(wm->gate, mh, l); mp.a1 = wmap(wm->up, mh, l); }
             mp.x = xd;
-            g.push_back({mp, p, wb * 2.0 * d.d_ffn * d.d_model, false, false});
+            TcGemmParams pa = p, pb = p;
+            static const bool split_on = !(getenv("MTAD_TC_SPLIT") && atoi(getenv("MTAD_TC_SPLIT")) == 0);   // experiment knob
+            if (split_on && tc_ctas_per_sm(T) == 1 && tc_cluster_plan_big_split(pa, pb, up(d.d_ffn, 64), d.d_model, T, kCtas)) {
+                // more tiles than SMs: two cluster launches over two ranges of the tiles
+                if (with_maps) { mp.a0 = wmap(wm->gate, pa.mh, l); mp.a1 = wmap(wm->up, pa.mh, l); }
+                const double all = wb * 2.0 * d.d_ffn * d.d_model, fa = (double)pa.n_tiles / (pa.n_tiles + pb.n_tiles);
+                g.push_back({mp, pa, all * fa, true, false});
+                g.push_back({mp, pb, all * (1.0 - fa), true, false});
+            } else {
+                if (with_maps) { mp.a0 = wmap(wm->gate, mh, l); mp.a1 = wmap(wm->up, mh, l); }
+                g.push_back({mp, p, wb * 2.0 * d.d_ffn * d.d_model, false, false});
+            }
         }
         {   // down projection + residual, emits the next norm's operand rows
             TcGemmParams p = base; TcMaps mp{};

@@ -43,6 +43,7 @@ struct TcGemmParams {
     int rpr;               // cluster kernel: rows per epilogue pass (1..8); pass q is finished by rank q % csize
     int recv_alias;        // cluster kernel: the receive slots of the exchange lie over the copy ring
     int ring_bytes;        // cluster kernel: shared memory below the fixed tail (set by the launch)
+    int tile_base;         // cluster kernel (many rows): first tile of this launch, when a matrix takes two launches
     int mode;
     int N;                 // output features (bound for stores)
     // Chained phases of one launch: a phase whose operand rows are written by the phase before it reads, per k-block,
@@ -132,6 +133,9 @@ size_t tc_workspace_floats(int n_tiles_max, int max_contrib_max, int rpad_max);
 // CTAs).  p.mode and, for QKV, the segment tiles must be set before the call: a tile never straddles q | k | v.  The
 // weight maps of the launch must have boxes of p.mh halves.
 bool tc_cluster_plan(TcGemmParams& p, int n_tiles128, int K, int T, int sms);
+// More tiles than SMs and more than 32 rows: the matrix as two cluster launches over two ranges of its tiles (a and b
+// come in as copies of the launch's parameters with p.mode set).  False when that does not apply.
+bool tc_cluster_plan_big_split(TcGemmParams& a, TcGemmParams& b, int n_tiles128, int K, int T, int sms);
 bool tc_cluster_plan_small(TcGemmParams& p, int n_tiles, int K, int T, int slots);
 cudaError_t launch_tc_cluster_small(const TcMaps& maps, const TcGemmParams& p, bool pdl, cudaStream_t st);
 cudaError_t launch_tc_cluster(const TcMaps& maps, const TcGemmParams& p, bool pdl, cudaStream_t st);

@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(BG_THREADS, 1) tc_gemm_cluster_big_kernel(cons
     const BgSmem s = bg_carve(smem_base, p.ring_bytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = (int)cluster_ctarank();
-    const int tile = (int)blockIdx.x / csize;
+    const int tile = p.tile_base + (int)blockIdx.x / csize;
     const int kb0 = (int)(((long long)rank * p.k_blocks) / csize);
     const int kb1 = (int)(((long long)(rank + 1) * p.k_blocks) / csize);
     const int n_kb = kb1 - kb0;
@@ -478,6 +478,54 @@ bool tc_cluster_plan_big(TcGemmParams& p, int n_tiles128, int K, int T, int sms)
     p.rpr = std::max(1, std::min(rpr, BG_ROWS));
     const BgLayout l = bg_layout(T, p.rpad, p.terms, mh, p.rpr, c);
     return l.stages >= 2 && l.exchange <= l.region;
+}
+
+// A matrix with more tiles than half the SMs (a single launch would leave every CTA a whole tile) as two launches over two ranges of its tiles: the first fills the SMs with small
+// clusters, the second spreads the remaining tiles over large ones (its weights are requested while the first one
+// finishes).  Both read the same operand rows; neither depends on the other.
+bool tc_cluster_plan_big_split(TcGemmParams& a, TcGemmParams& b, int n_tiles128, int K, int T, int sms) {
+    TcGemmParams p = a;
+    p.k_blocks = (K + TC_TILE_K - 1) / TC_TILE_K;
+    p.T = T;
+    p.rpad = (T + 15) / 16 * 16;
+    p.terms = tc_terms(T);
+    p.out_terms = p.terms;
+    p.n_bbox = 1;
+    p.nbuf = 1;
+    p.sliced = 0;
+    p.per_sm = 1;
+    p.recv_alias = 1;
+    const int cols = p.terms * p.rpad;
+    if (n_tiles128 < 1 || cols > 256 || p.mode == TC_QKV) return false;
+    const int mh = 2 * cols <= 512 ? 2 : 1;
+    p.mh = mh;
+    const int n_tiles = (n_tiles128 + mh - 1) / mh;
+    if (2 * n_tiles <= sms || n_tiles >= 2 * sms) return false;    // (up to sms / 2 tiles: one launch of clusters of two or more)
+    int best_a = 0, best_b = 0, best_n = 0;
+    double best_cost = 1e30;
+    for (int ca = 2; ca <= 4 && ca <= p.k_blocks; ++ca) {
+        const int na = std::min(n_tiles - 1, bg_max_active_clusters(ca, sms));
+        const int rest = n_tiles - na;
+        int cb = std::min(std::min(8, sms / rest), p.k_blocks);
+        while (cb >= 1 && bg_max_active_clusters(cb, sms) < rest) --cb;
+        if (na < 1 || cb < 1) continue;
+        const double cost = (double)p.k_blocks / ca + (double)p.k_blocks / cb;      // k-blocks a CTA streams, both launches
+        if (cost < best_cost) { best_cost = cost; best_a = ca; best_b = cb; best_n = na; }
+    }
+    if (!best_a) return false;
+    auto fill = [&](TcGemmParams& q, int tiles, int base, int c) -> bool {
+        q = p;
+        q.n_tiles = tiles;
+        q.tile_base = base;
+        q.total_units = tiles * q.k_blocks;
+        q.csize = c;
+        q.units_per_cta = (q.k_blocks + c - 1) / c;
+        q.max_contrib = c;
+        q.rpr = std::max(1, std::min((T + c - 1) / c, BG_ROWS));
+        const BgLayout l = bg_layout(T, q.rpad, q.terms, mh, q.rpr, c);
+        return l.stages >= 2 && l.exchange <= l.region;
+    };
+    return fill(a, best_n, 0, best_a) && fill(b, n_tiles - best_n, best_n, best_b);
 }
 
 cudaError_t launch_tc_cluster_big(const TcMaps& maps, const TcGemmParams& p_in, bool pdl, cudaStream_t st) {
