@@ -259,8 +259,13 @@ int mtad_profile_end(mtad_ctx* ctx, double* ms, double* bytes, int64_t* launches
 uint64_t mtad_kernel_launches(void);
 /* Runs the weight-streaming tensor-core GEMM alone: y[T, N] (fp32, device) = x[T, K] (fp32, device) * W[N, K]^T
  * (bf16, device, 16-byte aligned), T <= 256, K a multiple of 8 and at most the context's largest FFN width.
+ * variant 0: the stream-K kernel (work units dealt out evenly, partial tiles summed through the workspace);
+ * variant 1: the cluster kernels (split-K inside a thread-block cluster, partial rows summed through distributed
+ * shared memory; one kernel for up to 32 rows, one beyond) - MTAD_E_UNIMPLEMENTED where the shape does not suit them
+ * (more than 256 accumulator columns, more tiles than co-resident CTAs).
  * For unit tests and kernel timing; uses the context's workspace. */
-int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, int T, float* y, void* stream);
+int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, int T, float* y, int variant,
+                    void* stream);
 
 /* Extent audit (host arithmetic only: no device, no driver, descriptors may carry null pointers).  For one call on a
  * context created with (target, aux, max_batch, max_nodes) it lists, per array the call's kernels touch - every region

@@ -91,7 +91,7 @@ def load_library() -> C.CDLL:
     lib.mtad_profile_begin.argtypes = [P, I]
     lib.mtad_profile_end.argtypes = [P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     lib.mtad_kernel_launches.argtypes = []
-    lib.mtad_debug_gemm.argtypes = [P, P, I, I, P, I, P, P]
+    lib.mtad_debug_gemm.argtypes = [P, P, I, I, P, I, P, I, P]
     lib.mtad_verify_chain_static.argtypes = [MD, C.c_int32, C.c_int32, I, P, P, F, P, RS, P]
     for n in EXPORTS:
         if n not in ("mtad_status_str", "mtad_kernel_launches"):

@@ -17,7 +17,7 @@ using namespace mtad;
 // K and V are rounded to bf16 for the cache: their projection accumulates at most this many k-blocks (512 elements)
 // per tensor-memory accumulator, the pieces being added in fp32 (relative error about 4e-7 instead of 4e-6 at K = 8192)
 static const int kQkvSegCap = 8;
-static const int kCtas = getenv("MTAD_TC_CTAS") ? atoi(getenv("MTAD_TC_CTAS")) : 148;   // SMs the tensor-core GEMM spreads over
+static const int kCtas = 148;   // SMs the tensor-core GEMM spreads over
 
 // Host-side tensor maps of one model's weight matrices.
 struct WeightMaps {                      // index 0, 1, 2: tiles of 128, 256, 512 rows (1, 2, 4 halves)
@@ -380,8 +380,7 @@ bool build_weight_maps(const ModelView& m, WeightMaps& w) {
 }
 
 bool mma_attention(const ModelView& m) {
-    static const bool on = !(getenv("MTAD_TC_ATTN") && atoi(getenv("MTAD_TC_ATTN")) == 0);
-    return on && m.kv_map_ok && (m.d.head_dim == 64 || m.d.head_dim == 128);
+    return m.kv_map_ok && (m.d.head_dim == 64 || m.d.head_dim == 128);
 }
 
 // K/V tiles of the tensor-core attention arrive by TMA: one map over the whole cache of a model
@@ -439,11 +438,7 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
         if (!want) return false;
         TcGemmParams q = p;
         if (!tc_cluster_plan(q, n_tiles128, K, T, kCtas)) return false;
-        static const int big_mask = getenv("MTAD_TC_CLBIG") ? atoi(getenv("MTAD_TC_CLBIG")) : 31;   // experiment knob
-        if (q.per_sm == 1) {
-            const int bit = p.mode == TC_QKV ? 1 : (p.mode == TC_RESID ? (K == d.d_ffn ? 8 : 2) : 16);
-            if (!(big_mask & bit)) return false;
-        }
+
         p = q;
         return true;
     };
@@ -499,8 +494,7 @@ int build_plan(ForwardPlan& fp, const Scratch& sc, const RowMeta& rm, const Mode
             p.x_out = sc.xf; p.xk = d.d_ffn;
             mp.x = xd;
             TcGemmParams pa = p, pb = p;
-            static const bool split_on = !(getenv("MTAD_TC_SPLIT") && atoi(getenv("MTAD_TC_SPLIT")) == 0);   // experiment knob
-            if (split_on && tc_ctas_per_sm(T) == 1 && tc_cluster_plan_big_split(pa, pb, up(d.d_ffn, 64), d.d_model, T, kCtas)) {
+            if (tc_ctas_per_sm(T) == 1 && tc_cluster_plan_big_split(pa, pb, up(d.d_ffn, 64), d.d_model, T, kCtas)) {
                 // more tiles than SMs: two cluster launches over two ranges of the tiles
                 if (with_maps) { mp.a0 = wmap(wm->gate, pa.mh, l); mp.a1 = wmap(wm->up, pa.mh, l); }
                 const double all = wb * 2.0 * d.d_ffn * d.d_model, fa = (double)pa.n_tiles / (pa.n_tiles + pb.n_tiles);
@@ -792,7 +786,8 @@ int mtad_profile_end(mtad_ctx* ctx, double* ms, double* bytes, int64_t* launches
 
 uint64_t mtad_kernel_launches(void) { return g_kernel_launches; }
 
-int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, int T, float* y, void* stream) {
+int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, int T, float* y, int variant,
+                    void* stream) {
     if (!ctx || !W || !x || !y || N < 1 || K < 8 || (K % 8) || T < 1) return MTAD_E_INVALID;
     if (T > TC_MAX_ROWS || (size_t)2 * TC_X_ROWS * K > ctx->xf_elems) return MTAD_E_CAPACITY;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -810,13 +805,14 @@ int mtad_debug_gemm(mtad_ctx* ctx, const void* W, int N, int K, const float* x, 
     p.mode = TC_PLAIN; p.N = N; p.out = y; p.ldo = N;
     p.ws = ctx->sc.tc_ws; p.counters = ctx->sc.tc_counters; p.status = nullptr;
     RUN(MTAD_K_PREPARE, 0, 1, launch_split_rows(x, K, ctx->sc.xf, p.terms, T, K, s));
-    static const int cluster_mask = getenv("MTAD_TC_CLUSTER") ? atoi(getenv("MTAD_TC_CLUSTER")) : 27;
     TcGemmParams q = p;
-    if (((cluster_mask >> 5) & 1) && tc_cluster_plan(q, (N + TC_TILE_N - 1) / TC_TILE_N, K, T, kCtas)) {
+    if (variant == 1) {
+        if (!tc_cluster_plan(q, (N + TC_TILE_N - 1) / TC_TILE_N, K, T, kCtas)) return MTAD_E_UNIMPLEMENTED;
         if (q.mh != mh && tc_make_map(&mp.a0, W, N, K, q.mh == 1 ? 128 : 256)) return MTAD_E_CUDA;
         RUN(MTAD_K_GEMM, 2.0 * N * K, 1, launch_tc_cluster(mp, q, false, s));
         return MTAD_OK;
     }
+    if (variant != 0) return MTAD_E_INVALID;
     RUN(MTAD_K_GEMM, 2.0 * N * K, 1, launch_tc_gemm(mp, p, kCtas, false, s));
     return MTAD_OK;
 }

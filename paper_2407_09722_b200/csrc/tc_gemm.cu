@@ -481,8 +481,7 @@ int tc_make_map(CUtensorMap* out, const void* base, long long rows, long long co
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                          getenv("MTAD_TC_L2P") ? (CUtensorMapL2promotion)atoi(getenv("MTAD_TC_L2P"))
-                                                : CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? 0 : -1;
 }
@@ -520,8 +519,7 @@ void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int sms, int per_s
     p.units_per_cta = (p.total_units + ctas - 1) / ctas;
     // small matrices (the auxiliary model's): fewer CTAs with longer runs, so that a tile is not cut into one
     // contributor per k-block whose partial tiles the last arriver has to add up
-    static const int min_units = getenv("MTAD_TC_MIN_UNITS") ? atoi(getenv("MTAD_TC_MIN_UNITS")) : 2;
-    if (p.units_per_cta < min_units) p.units_per_cta = min_units;
+    if (p.units_per_cta < 2) p.units_per_cta = 2;
     p.max_contrib = (p.k_blocks + p.units_per_cta - 1) / p.units_per_cta + 1;
     p.T = T;
     p.rpad = (T + 15) / 16 * 16;
@@ -530,8 +528,7 @@ void tc_decompose(TcGemmParams& p, int n_tiles, int K, int T, int sms, int per_s
     p.n_bbox = tc_boxes(p.terms * p.rpad);
     // more than one pass of eight rows: the passes of a tile are shared out among its contributors, which wait for
     // one another - every CTA of the launch must be resident, i.e. at most one per SM slot
-    static const bool no_slice = getenv("MTAD_TC_SLICED") && atoi(getenv("MTAD_TC_SLICED")) == 0;
-    p.sliced = (T > EPI_ROWS && sms <= 148 && !no_slice) ? 1 : 0;
+    p.sliced = (T > EPI_ROWS && sms <= 148) ? 1 : 0;
     p.seg_cap = 1 << 20;
 }
 
@@ -539,22 +536,16 @@ int tc_terms(int T) {
     // Three terms up to 32 rows, where the third costs nothing measurable; two beyond.  With more rows the operand
     // rows (terms * rows * 128 B per k-block, re-read from L2 by every CTA) outweigh the 16 KB of weights they meet,
     // two terms leave room in tensor memory for two weight halves per stage up to 64 rows, and at the level of the
-    // whole model the third term changes nothing (the error there is set by bf16 K/V rounding).  MTAD_TC_TERMS=2 /
-    // =3 force a count (3 only up to 80 rows: three accumulators must fit tensor memory twice).
-    static const int force = getenv("MTAD_TC_TERMS") ? atoi(getenv("MTAD_TC_TERMS")) : 0;
+    // whole model the third term changes nothing (the error there is set by bf16 K/V rounding).
     const int rpad = (T + 15) / 16 * 16;
-    if (force == 2) return 2;
-    if (force == 3) return rpad <= 80 ? 3 : 2;
     return rpad <= 32 ? 3 : 2;
 }
 
 int tc_ctas_per_sm(int T) {
     // two CTAs need: 16 KB of weights + terms * rpad operand rows per stage, at least two stages in 112 KB less the
     // epilogue scratch, and one accumulator buffer of terms * rpad columns within 256 columns
-    static const int force = getenv("MTAD_TC_PER_SM") ? atoi(getenv("MTAD_TC_PER_SM")) : 0;
     const int rpad = (T + 15) / 16 * 16, cols = tc_terms(T) * rpad;
-    if (cols > 240 || force == 1) return 1;
-    if (force == 2) return 2;
+    if (cols > 240) return 1;
     return rpad <= 32 ? 2 : 1;
 }
 
@@ -564,7 +555,7 @@ int tc_halves(int T) {
     // per stage against the same operand rows) are worth more than a second accumulator buffer: with 129..256
     // columns a stage has two halves and the launch a single buffer (7B tree 8.7 -> 8.0 ms).  Four halves fit the
     // smallest row counts but fill and drain slower than two.
-    static const int cap = getenv("MTAD_TC_MH") ? atoi(getenv("MTAD_TC_MH")) : 2;
+    const int cap = 2;
     const int cols = tc_terms(T) * ((T + 15) / 16 * 16);
     const int fit = cols <= 64 ? 4 : (cols <= 256 ? 2 : 1);
     return fit < cap ? fit : cap;
@@ -586,8 +577,7 @@ cudaError_t launch_tc_chain(const TcChain& chain_in, bool pdl, cudaStream_t st) 
     if (f.mh * acc_cols > tmem_budget || f.n_bbox < 1 || f.n_bbox != tc_boxes(acc_cols)) return cudaErrorInvalidValue;
     const int nbuf = (2 * f.mh * acc_cols <= tmem_budget) ? 2 : 1;
     const int stage_bytes = f.mh * TC_TILE_N * 128 + acc_cols * 128;
-    static const int budget_kb_env = getenv("MTAD_TC_SMEM_KB") ? atoi(getenv("MTAD_TC_SMEM_KB")) : 0;
-    const size_t budget = f.per_sm == 2 ? (size_t)112 * 1024 : (size_t)(budget_kb_env > 0 ? budget_kb_env : 226) * 1024;
+    const size_t budget = f.per_sm == 2 ? (size_t)112 * 1024 : (size_t)226 * 1024;
     int stages = (int)((budget - SMEM_TAIL - 1024) / stage_bytes);
     stages = stages > MAX_STAGES ? MAX_STAGES : stages;
     if (stages < 2) return cudaErrorInvalidValue;
@@ -602,11 +592,15 @@ cudaError_t launch_tc_chain(const TcChain& chain_in, bool pdl, cudaStream_t st) 
         grid = std::max(grid, (p.total_units + p.units_per_cta - 1) / p.units_per_cta);
     }
     const size_t smem = (size_t)stages * stage_bytes + SMEM_TAIL + 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {};                     // per device
+    int dev = 0;
+    cudaError_t e0 = cudaGetDevice(&dev);
+    if (e0 != cudaSuccess) return e0;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(grid);

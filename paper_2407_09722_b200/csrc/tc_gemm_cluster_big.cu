@@ -457,27 +457,31 @@ bool tc_cluster_plan_big(TcGemmParams& p, int n_tiles128, int K, int T, int sms)
     p.sliced = 0;
     p.per_sm = 1;
     p.recv_alias = 1;
+    p.tile_base = 0;
     const int cols = p.terms * p.rpad;
     if (n_tiles128 < 1 || cols > 256) return false;
-    int mh = 2 * cols <= 512 ? 2 : 1;                      // two halves of weights meet the same operand rows
-    if (p.mode == TC_QKV)                                  // a tile must not straddle q | k | v
-        while (mh > 1 && (p.seg_k_tile % mh || p.seg_v_tile % mh || n_tiles128 % mh)) mh /= 2;
-    p.mh = mh;
-    const int n_tiles = (n_tiles128 + mh - 1) / mh;
-    p.n_tiles = n_tiles;
-    p.total_units = n_tiles * p.k_blocks;
-    int c = sms / n_tiles;
-    c = std::min(c, 8);                // portable cluster size
-    c = std::min(c, p.k_blocks);
-    while (c >= 1 && bg_max_active_clusters(c, sms) < n_tiles) --c;     // every cluster resident in one wave
-    if (c < 1) return false;           // more tiles than SMs: a second wave would start late
-    p.csize = c;
-    p.units_per_cta = (p.k_blocks + c - 1) / c;
-    p.max_contrib = c;
-    int rpr = (T + c - 1) / c;
-    p.rpr = std::max(1, std::min(rpr, BG_ROWS));
-    const BgLayout l = bg_layout(T, p.rpad, p.terms, mh, p.rpr, c);
-    return l.stages >= 2 && l.exchange <= l.region;
+    // two halves of weights against the same operand rows where tensor memory (512 columns) and the exchange area
+    // allow, else one; the largest cluster whose tiles are all resident in one wave and whose exchange fits
+    for (int mh = 2 * cols <= 512 ? 2 : 1; mh >= 1; --mh) {
+        if (p.mode == TC_QKV && (p.seg_k_tile % mh || p.seg_v_tile % mh || n_tiles128 % mh)) continue;   // no tile straddles q | k | v
+        const int n_tiles = (n_tiles128 + mh - 1) / mh;
+        int c = std::min(std::min(sms / n_tiles, 8), p.k_blocks);          // (8: portable cluster size)
+        while (c >= 1 && bg_max_active_clusters(c, sms) < n_tiles) --c;
+        for (; c >= 1; --c) {
+            const int rpr = std::max(1, std::min((T + c - 1) / c, BG_ROWS));
+            const BgLayout l = bg_layout(T, p.rpad, p.terms, mh, rpr, c);
+            if (l.stages < 2 || l.exchange > l.region) continue;
+            p.mh = mh;
+            p.n_tiles = n_tiles;
+            p.total_units = n_tiles * p.k_blocks;
+            p.csize = c;
+            p.units_per_cta = (p.k_blocks + c - 1) / c;
+            p.max_contrib = c;
+            p.rpr = rpr;
+            return true;
+        }
+    }
+    return false;                      // more tiles than SMs (a second wave would start late), or no room for the exchange
 }
 
 // A matrix with more tiles than half the SMs (a single launch would leave every CTA a whole tile) as two launches over two ranges of its tiles: the first fills the SMs with small

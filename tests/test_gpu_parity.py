@@ -42,8 +42,7 @@ def test_tiny_chain_matches_oracle(tiny, gamma, L):
         compare(tiny, [case], Bn.log_tau(tau), _u(0, it, 1, TINY.vocab), chain=True, stats=stats)
         tiny.inject(0, L)
     assert stats.ok(), stats
-    assert stats.cache_rows > 0 and stats.cache_max_excess < 1e-3
-    assert stats.cache_exact > 0.95 * stats.cache_rows
+    assert stats.cache_ok(TINY.layers)
 
 
 @pytest.mark.parametrize("depth,width,keep,L", [(4, 4, 4, 32), (3, 8, 2, 7), (4, 8, 4, 130), (2, 16, 4, 0)])
@@ -55,7 +54,7 @@ def test_tiny_tree_matches_oracle(tiny, depth, width, keep, L):
         case = SeqCase(1, L, _root(1, it, TINY.vocab), tree)
         compare(tiny, [case], Bn.log_tau(tau), _u(1, it, 1, TINY.vocab), chain=False, stats=stats)
     assert stats.ok(), stats
-    assert stats.cache_max_excess < 1e-3
+    assert stats.cache_ok(TINY.layers)
 
 
 @pytest.mark.parametrize("shape", [GQA, GQA64])

@@ -35,7 +35,7 @@ def _run(w, shape, capacity, taus, check_cache=True):
 def test_7b_chain_full_depth():
     w = S.WORKLOADS["7b_chain"]
     st = _run(w, w.target, 2048 + 64, [0.1, 0.5])
-    assert st.max_lp_err < 2e-3 and st.cache_max_excess < 1e-3
+    assert st.max_lp_err < 2e-3 and st.cache_ok(w.target.layers)
 
 
 def test_7b_tree_full_depth():
@@ -109,3 +109,13 @@ def test_7b_pair_drafted_tree_two_layers():
     w = S.WORKLOADS["7b_tree"]
     shape = dataclasses.replace(w.target, layers=2)
     batched_iterations(shape, w.aux, [2048], w.gamma, 4, 2048 + 160, 2048 + 160, 2, tree=True, keep_all=True)
+
+
+def test_7b_pair_chain_eight_iterations_two_layers():
+    """Algorithm 1 for eight consecutive iterations at the 7B-shaped pair (target cut to two layers so that the oracle
+    stays affordable, the full-size auxiliary model): draft, verification of the output sequence as a chain, commit of
+    both caches, each iteration starting from the state the one before left on the device, against the oracle."""
+    from tests.test_gpu_draft import batched_iterations
+    w = S.WORKLOADS["7b_chain"]
+    shape = dataclasses.replace(w.target, layers=2)
+    batched_iterations(shape, w.aux, [2048], w.gamma, 4, 2048 + 96, 2048 + 96, 8)

@@ -557,3 +557,63 @@ def test_aux_commit_with_an_accepted_leaf():
     for i, t in enumerate(committed):
         want = O.decoder_rows(model, c2, i, [t], [i], [i], [[i]])[0]
     assert np.max(np.abs(got - want)) < 1e-9
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# the margins that decide which device decisions the parity tests compare
+# ----------------------------------------------------------------------------------------------------------------
+
+def test_warp_row_margin_hand_computed_and_protective():
+    z = np.log(np.array([0.5, 0.3, 0.15, 0.05]))
+    # top-3 of (0.5, 0.3, 0.15, 0.05), top_p 0.8: the top-k boundary lies ln 3 apart in logits; the partial sums are
+    # 0.5 / 0.95 (0.274 from 0.8) and 0.8 / 0.95 (0.0421 above it): the closest decision is the last one
+    _, margin = O.warp_row(z, 3, 0.8)
+    assert abs(margin - (0.8 / 0.95 - 0.8)) < 1e-12
+    # with top_p out of the way (never reached before the last token) only the top-k boundary is left
+    _, margin = O.warp_row(z, 2, 1.0)
+    assert abs(margin - min(math.log(0.3 / 0.15), 1.0 - 0.5 / 0.8)) < 1e-12
+    # what the margin promises: logits moved by less than a quarter of it keep exactly the same tokens (a partial sum
+    # moves by at most e^(2 d) - 1 < margin, the gap across the top-k boundary by at most 2 d < margin)
+    rng = np.random.default_rng(11)
+    for trial in range(200):
+        V = int(rng.integers(4, 12))
+        zr = rng.normal(size=V) * 2.0
+        k, top_p = int(rng.integers(1, V + 1)), float(rng.uniform(0.3, 0.99))
+        out, m = O.warp_row(zr, k, top_p)
+        if not np.isfinite(m) or m <= 0:
+            continue
+        d = rng.uniform(-1, 1, size=V) * min(m, 1.0) / 4.0 * 0.999
+        out2, _ = O.warp_row(zr + d, k, top_p)
+        assert np.array_equal(np.isfinite(out), np.isfinite(out2)), (trial, m)
+
+
+def test_spd_robust_margin_is_the_gap_under_the_worst_perturbation():
+    rng = np.random.default_rng(5)
+    V, g, tol = 9, 3, 2e-3
+    seen_reject = seen_accept = 0
+    for trial in range(300):
+        logits = rng.normal(size=(g + 1, V)) * 2.0
+        logq = O.log_softmax(rng.normal(size=(g, V)) * 2.0)
+        tok = [int(t) for t in rng.integers(0, V, size=g)]
+        u_acc = rng.uniform(0.01, 0.99, size=g)
+        u_res = rng.uniform(0.01, 0.99, size=V)
+        r = O.spd_from_logits(logits, tok, logq, u_acc, u_res, tol=tol)
+        assert r.margin_bonus_robust <= r.margin_bonus + 1e-12
+        if r.eta == g:
+            # every token accepted: the draw is from the target's next row, log p within +-tol moves the winner's
+            # lead by at most 2 tol
+            assert abs(r.margin_bonus_robust - (r.margin_bonus - 2 * tol)) < 1e-9
+            seen_accept += 1
+            continue
+        seen_reject += 1
+        if r.margin_bonus_robust <= 0:
+            continue
+        # a positive robust margin promises the same resampled token for any log p within +-tol of the row
+        logp = O.log_softmax(logits)
+        noise = -np.log(-np.log(u_res))
+        for _ in range(20):
+            lp2 = logp[r.eta] + rng.uniform(-tol, tol, size=V)
+            with np.errstate(divide="ignore"):
+                z2 = np.log(np.maximum(0.0, np.exp(lp2) - np.exp(logq[r.eta])))
+            assert int(np.argmax(z2 + noise)) == r.out_tok[-1], trial
+    assert seen_reject > 50 and seen_accept > 5
