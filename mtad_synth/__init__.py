@@ -199,6 +199,8 @@ WORKLOADS: Dict[str, Workload] = {
     "7b_chain_4l": Workload("7b_chain_4l", _llama(4, 4096, 32, 32, 128, 11008), _llama(2, 768, 12, 12, 64, 3072),
                             batch=1, kind="chain", gamma=4, n_nodes=4, kv_len=(2048, 2048), prompt_len=512,
                             decode_iters=128),
+    "7b_tree_4l": Workload("7b_tree_4l", _llama(4, 4096, 32, 32, 128, 11008), _llama(2, 768, 12, 12, 64, 3072),
+                           batch=1, kind="tree", gamma=4, n_nodes=64, kv_len=(2048, 2048), tree_width=16, tree_keep=4),
     "7b_tree": Workload("7b_tree", _llama(32, 4096, 32, 32, 128, 11008), _llama(2, 768, 12, 12, 64, 3072),
                         batch=1, kind="tree", gamma=4, n_nodes=64, kv_len=(2048, 2048), tree_width=16, tree_keep=4),
     "13b_batched_chain": Workload("13b_batched_chain", _llama(40, 5120, 40, 40, 128, 13824),

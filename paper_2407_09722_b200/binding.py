@@ -303,11 +303,12 @@ class Context:
             self._check(rc, "kv_commit")
         return rc
 
-    def mtad_debug_gemm(self, W: torch.Tensor, x: torch.Tensor, y: torch.Tensor, stream=None, check=True) -> int:
+    def mtad_debug_gemm(self, W: torch.Tensor, x: torch.Tensor, y: torch.Tensor, stream=None, check=True,
+                        variant: int = 0) -> int:
         N, K = W.shape
         T = x.shape[0]
         rc = self._lib.mtad_debug_gemm(self.handle, _ptr(W, torch.bfloat16), N, K, _ptr(x, torch.float32), T,
-                                       _ptr(y, torch.float32), _stream(stream))
+                                       _ptr(y, torch.float32), variant, _stream(stream))
         if check:
             self._check(rc, "mtad_debug_gemm")
         return rc

@@ -17,7 +17,17 @@ from oracle.adapters import oracle_model, bits
 
 LP_TOL = 2e-3          # absolute tolerance on log-probabilities (per token and joint)
 MARGIN = 1e-3          # decisions closer than this to a boundary are counted, not compared
-GEMM_EPS = 8e-6        # error of one projection relative to its largest output (the bound of test_gpu_gemm.py)
+# Error of one projection relative to its largest output; test_gpu_gemm.py holds the GEMM kernels alone to these (about
+# twice what they show).  Up to 32 rows the activations enter as three bf16 terms, i.e. exactly, and what is left is the
+# tensor cores' fp32 accumulation, which grows with the k-blocks summed in one accumulator; beyond 32 rows they enter
+# as two terms (2^-17 relative per element).
+GEMM_EPS_FEW = 1e-6    # up to 32 rows, K <= 2048
+GEMM_EPS_WIDE = 8e-6   # up to 32 rows, K > 2048 (the 7B / 13B / 70B matrices)
+GEMM_EPS_MANY = 6e-6   # more than 32 rows, K <= 2048
+
+
+def gemm_eps(rows: int, k: int) -> float:
+    return GEMM_EPS_WIDE if k > 2048 else (GEMM_EPS_FEW if rows <= 32 else GEMM_EPS_MANY)
 
 
 class GpuModel(DeviceModel):
@@ -92,13 +102,13 @@ class ParityStats:
     cache_scale: float = 0.0
     etas: List[int] = field(default_factory=list)
 
-    def cache_ok(self, layers: int) -> bool:
+    def cache_ok(self, layers: int, gemm_error: float) -> bool:
         """The K/V rows a call appends, against the oracle's (fp64, rounded to bf16 once).
 
         The device rounds its fp32 value y to bf16, the oracle its fp64 value y*.  |y - y*| <= eps * s with s the
-        largest |K/V| value of the call and eps = GEMM_EPS per layer: GEMM_EPS is the bound test_gpu_gemm.py holds the
-        projection alone to (fp32 accumulation of exactly represented operands), and every layer adds one projection's
-        worth to the residual stream the next one reads.  Two things follow.
+        largest |K/V| value of the call and eps = gemm_error per layer: gemm_error (gemm_eps above) is the bound
+        test_gpu_gemm.py holds the projection alone to, and every layer adds one projection's worth to the residual
+        stream the next one reads.  Two things follow.
         (1) Where both sides round the same way the elements are equal; where they do not they are one bf16 step of
         the value apart, at most 2^-7 |y*|; only next to zero can the difference exceed that, and then by no more than
         |y - y*|.  So excess = |got - want| - 2^-7 |want| <= eps * s everywhere.
@@ -106,7 +116,7 @@ class ParityStats:
         2^-8 |y*| apart (at least), so that happens with probability min(1, 2 eps s / (2^-8 |y*|)).  For values spread
         like a normal distribution of standard deviation s / 4 (s is a four-sigma maximum) the mean of that is below
         q (1 + ln(1 / q)) * 0.8 with q = 2048 eps - the bound on the share of unequal elements."""
-        eps = GEMM_EPS * layers
+        eps = gemm_error * layers
         q = 2048.0 * eps
         flips = 0.8 * q * (1.0 + math.log(1.0 / q))
         rate = 1.0 - self.cache_exact / max(self.cache_rows, 1)
@@ -114,12 +124,13 @@ class ParityStats:
               f"{self.cache_max_excess:.2e} (bound {eps * self.cache_scale:.2e})")
         return self.cache_rows > 0 and self.cache_max_excess <= eps * self.cache_scale and rate <= flips
 
-    def ok(self) -> bool:
+    def ok(self, tie_cap: Optional[int] = None) -> bool:
         """Log-probabilities within LP_TOL everywhere; every decision equal except in sequences that have one within
-        MARGIN of going the other way, and those are few: at most a third of the sequences (rounded up).  The margins
-        of a random-init model are spread over several nats, so a share like that already means something is off."""
+        MARGIN of going the other way, and those are few: at most a third of the sequences (rounded up) unless the
+        test states another cap (warped rows add a top-k and a top-p boundary to every row).  The margins of a
+        random-init model are spread over several nats, so a share like that already means something is off."""
         clean = self.n_seq - self.near_ties
-        cap = (self.n_seq + 2) // 3
+        cap = (self.n_seq + 2) // 3 if tie_cap is None else tie_cap
         print(f"parity: {self.n_seq} sequences, {self.near_ties} near a tie (cap {cap}), eta/path/token equal in "
               f"{self.eta_match}/{self.path_match}/{self.tok_match}, largest error lp {self.max_lp_err:.2e} "
               f"LP {self.max_LP_err:.2e} lse {self.max_lse_err:.2e}")

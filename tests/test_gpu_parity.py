@@ -10,7 +10,7 @@ import torch
 import mtad_synth as S
 import paper_2407_09722_b200 as M
 from paper_2407_09722_b200 import binding as Bn
-from tests.parity import GpuModel, SeqCase, ParityStats, compare, run_gpu, LP_TOL
+from tests.parity import GpuModel, SeqCase, ParityStats, compare, run_gpu, LP_TOL, gemm_eps
 
 pytestmark = pytest.mark.gpu
 
@@ -42,7 +42,7 @@ def test_tiny_chain_matches_oracle(tiny, gamma, L):
         compare(tiny, [case], Bn.log_tau(tau), _u(0, it, 1, TINY.vocab), chain=True, stats=stats)
         tiny.inject(0, L)
     assert stats.ok(), stats
-    assert stats.cache_ok(TINY.layers)
+    assert stats.cache_ok(TINY.layers, gemm_eps(gamma + 1, TINY.d_ffn))
 
 
 @pytest.mark.parametrize("depth,width,keep,L", [(4, 4, 4, 32), (3, 8, 2, 7), (4, 8, 4, 130), (2, 16, 4, 0)])
@@ -54,7 +54,7 @@ def test_tiny_tree_matches_oracle(tiny, depth, width, keep, L):
         case = SeqCase(1, L, _root(1, it, TINY.vocab), tree)
         compare(tiny, [case], Bn.log_tau(tau), _u(1, it, 1, TINY.vocab), chain=False, stats=stats)
     assert stats.ok(), stats
-    assert stats.cache_ok(TINY.layers)
+    assert stats.cache_ok(TINY.layers, gemm_eps(1 + depth * width, TINY.d_ffn))
 
 
 @pytest.mark.parametrize("shape", [GQA, GQA64])
