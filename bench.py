@@ -28,7 +28,9 @@ import mtad_synth as S  # noqa: E402
 
 TAU = 0.1
 SEED = 0
-NCU_TRAFFIC_RATIO = 1.022     # (DRAM read + write) / algorithmic bytes of the GEMM launches, ncu on the 4-layer workload
+# (DRAM read + write) / algorithmic bytes of the GEMM launches of one layer, ncu on the 4-layer workloads of the same
+# shape (profiles/tc_gemm_7b_chain_4l.md, profiles/tc_gemm_7b_tree_4l.md); no figure for the other workloads
+NCU_TRAFFIC_RATIO = {"7b_chain": 1.009, "7b_chain_4l": 1.009, "7b_chain_l512": 1.009, "7b_tree": 1.032, "7b_tree_4l": 1.032}
 
 
 def measured_peaks():
@@ -514,14 +516,17 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
     achieved_iso = gemm_iso["bytes"] / (gemm_iso["ms"] * 1e-3) / 1e9 if gemm_iso["ms"] > 0 else 0.0
     prof_total = sum(v["ms"] for v in prof.values())
     alg_per_launch = gemm["bytes"] / max(gemm["launches"], 1)
-    roofline = {"bound": "hbm", "kernel": "tc_gemm_kernel (all weight matrices + LM head)", "achieved": achieved,
+    ratio = NCU_TRAFFIC_RATIO.get(w.name)
+    roofline = {"bound": "hbm",
+                "kernel": "the weight-streaming GEMMs (tc_gemm_cluster_kernel / tc_gemm_cluster_big_kernel / tc_gemm_kernel: "
+                          "all weight matrices + LM head)", "achieved": achieved,
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                 "timing": "CUDA events on the launching stream around every run of consecutive GEMM launches "
                           "(O, gate/up, down, next QKV or LM head), summed and divided by the launches",
                 "algorithmic_bytes_per_launch": alg_per_launch,
                 # DRAM read + write bytes per launch: the ratio to the algorithmic bytes was taken with ncu on the
-                # 4-layer workload (profiles/tc_gemm_7b_chain_4l.md) and scales with the weights streamed
-                "traffic": alg_per_launch * NCU_TRAFFIC_RATIO if NCU_TRAFFIC_RATIO else None,
+                # 4-layer workload of the same shape and scales with the weights streamed
+                "traffic": alg_per_launch * ratio if ratio else None,
                 "launches_per_step": gemm["launches"] / prof_steps,
                 "avg_launch_us": 1e3 * gemm["ms"] / max(gemm["launches"], 1),
                 "share_of_step": gemm["ms"] / prof_total if prof_total else None,

@@ -39,7 +39,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const TcGemmParams& p0 = ch.p[0];
-    const int mh = p0.mh;                              // 128-row weight halves per stage (1, 2 or 4), same in every phase
+    const int mh = p0.mh;                              // 128-row weight halves per stage (1, 2 or 4), the same for the whole launch
     const int a_bytes = mh * TC_TILE_N * 128;
     const int terms = p0.terms;
     const int acc_cols = terms * p0.rpad;              // one column per operand row: the terms of a draft row are neighbours
@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) trace_stamp(p0.trace, 0);
     volatile int* abort_flag = s.abort_flag;
-    // this CTA's share of a phase: units [first, first + count)
+    // this CTA's share of the launch: units [first, first + count)
     auto share = [&](const TcGemmParams& p, int& first, int& count) {
         first = (int)blockIdx.x * p.units_per_cta;
         count = max(min(first + p.units_per_cta, p.total_units) - first, 0);
@@ -92,14 +92,13 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
 
     if (warp == 0) {
         // ---------------- weight producer (one thread) -------------------------------------------------------------
-        // Weights never depend on an earlier step: their copies go out as soon as a stage is free, across phase
-        // boundaries too.  The operand rows of the same stage are brought by the next warp once they exist.
+        // Weights never depend on an earlier step: their copies go out as soon as a stage is free.  The operand rows of the same stage are brought by the next warp once they exist.
         if (lane == 0) {
             int g = 0;
             bool ok = true;
-            for (int ph = 0; ph < ch.n_phases && ok; ++ph) {
-                const TcGemmParams& p = ch.p[ph];
-                const TcMaps& mp = ch.maps[ph];
+            {
+                const TcGemmParams& p = ch.p[0];
+                const TcMaps& mp = ch.maps[0];
                 int first, n_units;
                 share(p, first, n_units);
                 const int nb = a_boxes(p.mode, mh);
@@ -125,38 +124,27 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
         }
     } else if (warp == 1) {
         // ---------------- operand-row producer (one thread) --------------------------------------------------------
-        // The rows of a k-block exist once their producer is finished: the previous kernel for phase 0, the tile of
-        // the previous phase that wrote those 64 columns otherwise.
+        // The rows of a k-block exist once the previous kernel is finished.
         if (lane == 0) {
             int g = 0;
             bool ok = true;
-            for (int ph = 0; ph < ch.n_phases && ok; ++ph) {
-                const TcGemmParams& p = ch.p[ph];
+            {
+                const TcGemmParams& p = ch.p[0];
                 int first, n_units;
                 share(p, first, n_units);
-                if (ph == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
-                if (ph == 0) trace_stamp(p0.trace, 1);
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                trace_stamp(p0.trace, 1);
                 int kb = n_units > 0 ? first % p.k_blocks : 0;
-                int ready_tile = -1;                   // tile of the previous phase known to be finished
                 for (int i = 0; i < n_units && ok; ++i, ++g) {
                     const int st = g % stages;
                     if (g >= stages) {
                         ok = mbar_wait(smem_u32(&s.empty[st]), (((uint32_t)(g / stages)) & 1u) ^ 1u, abort_flag);
                         if (!ok) break;
                     }
-                    if (ph > 0) {
-                        const int need = (kb * TC_TILE_K) / p.dep_feat;
-                        if (need != ready_tile) {
-                            ok = flag_wait(ch.p[ph - 1].tile_done + need, 1, abort_flag);
-                            if (!ok) break;
-                            ready_tile = need;
-                            asm volatile("fence.proxy.async;" ::: "memory");    // the rows are read by TMA next
-                        }
-                    }
                     const uint32_t bar = smem_u32(&s.full[st]);
                     const uint32_t base = smem_u32(s.ring + (size_t)st * stage_bytes) + a_bytes;
                     for (int b = 0; b < n_bbox && !p0.debug_no_operands; ++b)
-                        tma_load_2d(base + b * bbox_rows * 128, &ch.maps[ph].x, bar, kb * TC_TILE_K, b * bbox_rows,
+                        tma_load_2d(base + b * bbox_rows * 128, &ch.maps[0].x, bar, kb * TC_TILE_K, b * bbox_rows,
                                     HINT_KEEP);
                     if (++kb == p.k_blocks) kb = 0;
                 }
@@ -176,10 +164,10 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
         if (lane == 0 && h < mh) {
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bbox_rows >> 3) << 17) |
                                    ((uint32_t)(TC_TILE_N >> 4) << 24);
-            int g = 0, seg = 0;                        // running unit and segment counters over all phases
+            int g = 0, seg = 0;                        // running unit and segment counters
             bool ok = true;
-            for (int ph = 0; ph < ch.n_phases && ok; ++ph) {
-                const TcGemmParams& p = ch.p[ph];
+            {
+                const TcGemmParams& p = ch.p[0];
                 int first, n_units;
                 share(p, first, n_units);
                 const int KB = p.k_blocks;
@@ -228,23 +216,14 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
         const size_t half_floats = (size_t)p0.rpad * TC_TILE_N;
         const size_t part_floats = (size_t)mh * half_floats;
         int seg = 0;
-        bool alive = true;
-        for (int ph = 0; ph < ch.n_phases && alive; ++ph) {
-            const TcGemmParams& p = ch.p[ph];
+        {
+            const TcGemmParams& p = ch.p[0];
             int first, n_units;
             share(p, first, n_units);
             const int KB = p.k_blocks;
-            // everything this phase reads besides its operand rows (row statistics, the residual stream) is final once
-            // the previous kernel (phase 0) or the whole previous phase has finished
-            if (ph == 0) {
-                asm volatile("griddepcontrol.wait;" ::: "memory");
-            } else {
-                if (e == 0) s.flags[0] = flag_wait(ch.p[ph - 1].phase_done, ch.p[ph - 1].n_tiles, abort_flag) ? 1 : 0;
-                epi_bar();
-                alive = s.flags[0] != 0;
-                epi_bar();
-                if (!alive) break;
-            }
+            // everything read here besides the operand rows (row statistics, the residual stream) is final once the
+            // previous kernel has finished
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             // deferred RMSNorm scale of every row
             for (int r = e; r < TC_MAX_ROWS; r += EPI_THREADS) {
                 float v = 1.f;
@@ -273,7 +252,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
                 if (lane == 0) s.flags[1 + (warp - 2 - MAX_HALVES)] = ok ? 1 : 0;
                 epi_bar();
                 if (e == 0 && i + len == n_units) trace_stamp(p0.trace, 4);
-                if (!(s.flags[1] && s.flags[2] && s.flags[3] && s.flags[4])) { alive = false; break; }
+                if (!(s.flags[1] && s.flags[2] && s.flags[3] && s.flags[4])) break;
                 tc_fence_after();
                 // contributors of this tile, in CTA order
                 const int c_first = (tile * KB) / p.units_per_cta;
@@ -353,7 +332,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
                 epi_bar();
                 const int fin = s.flags[0];
                 epi_bar();                                  // flags[0] is rewritten by the next segment
-                if (fin == 2) { alive = false; break; }
+                if (fin == 2) break;
                 if (sliced) { pass0 = slot_idx; pass_step = n_late; }
                 if (e == 0 && i + len == n_units) trace_stamp(p0.trace, fin == 1 ? 6 : 5);
                 if (fin == 1) {
@@ -415,15 +394,6 @@ __global__ void __launch_bounds__(TC_THREADS, 2) tc_gemm_kernel(const __grid_con
                         epi_bar();
                     }
                     if (e == 0 && closer) p.counters[tile] = 0;          // ready for the next launch
-                    if (p.tile_done && closer) {
-                        // publish the finished tile to the phase that reads it as operand rows
-                        __threadfence();
-                        epi_bar();
-                        if (e == 0) {
-                            asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p.tile_done + tile), "r"(1) : "memory");
-                            atomicAdd(p.phase_done, 1);
-                        }
-                    }
                 }
                 i += len;
                 ++seg;
@@ -567,7 +537,6 @@ size_t tc_workspace_floats(int n_tiles_max, int max_contrib_max, int rpad_max) {
 
 cudaError_t launch_tc_chain(const TcChain& chain_in, bool pdl, cudaStream_t st) {
     TcChain ch = chain_in;
-    if (ch.n_phases < 1 || ch.n_phases > TC_MAX_PHASES) return cudaErrorInvalidValue;
     const TcGemmParams& f = ch.p[0];
     if (f.mh != 1 && f.mh != 2 && f.mh != 4) return cudaErrorInvalidValue;
     if (f.terms != 2 && f.terms != 3) return cudaErrorInvalidValue;
@@ -582,8 +551,8 @@ cudaError_t launch_tc_chain(const TcChain& chain_in, bool pdl, cudaStream_t st) 
     stages = stages > MAX_STAGES ? MAX_STAGES : stages;
     if (stages < 2) return cudaErrorInvalidValue;
     int grid = 1;
-    for (int i = 0; i < ch.n_phases; ++i) {
-        TcGemmParams& p = ch.p[i];
+    {
+        TcGemmParams& p = ch.p[0];
         if (p.mh != f.mh || p.rpad != f.rpad || p.T != f.T || p.terms != f.terms || p.per_sm != f.per_sm ||
             p.n_bbox != f.n_bbox)
             return cudaErrorInvalidValue;                  // one ring, one TMEM layout
@@ -618,11 +587,8 @@ cudaError_t launch_tc_chain(const TcChain& chain_in, bool pdl, cudaStream_t st) 
 cudaError_t launch_tc_gemm(const TcMaps& maps, const TcGemmParams& p, int ctas, bool pdl, cudaStream_t st) {
     (void)ctas;
     TcChain ch{};
-    ch.n_phases = 1;
     ch.maps[0] = maps;
     ch.p[0] = p;
-    ch.p[0].tile_done = nullptr;
-    ch.p[0].phase_done = nullptr;
     return launch_tc_chain(ch, pdl, st);
 }
 

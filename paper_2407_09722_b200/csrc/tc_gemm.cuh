@@ -46,12 +46,6 @@ struct TcGemmParams {
     int tile_base;         // cluster kernel (many rows): first tile of this launch, when a matrix takes two launches
     int mode;
     int N;                 // output features (bound for stores)
-    // Chained phases of one launch: a phase whose operand rows are written by the phase before it reads, per k-block,
-    // the flag of the tile that wrote those 64 columns (dep_feat = output features per tile of that phase); every
-    // finished tile sets tile_done[tile] and bumps *phase_done.  Null in a launch of a single phase.
-    int* tile_done;
-    int* phase_done;
-    int dep_feat;
     // split-K fix-up
     float* ws;             // [n_tiles][max_contrib][mh][rpad][128] partial tiles (terms already summed)
     int* counters;         // [n_tiles], zero between launches
@@ -96,14 +90,10 @@ struct TcMaps {
     CUtensorMap x;                  // operand rows [2 * TC_X_ROWS, K]: row terms * t + j = term j of activation row t
 };
 
-// Up to four GEMMs that feed one another (O projection, gate/up, down, next layer's QKV) run as phases of one launch:
-// the weight stream never stops at a phase boundary, and a phase starts on a k-block as soon as the tile that
-// produced those operand columns is final.
-constexpr int TC_MAX_PHASES = 4;
+// What one launch of the stream-K kernel takes: the tensor maps and the parameters, as one kernel argument.
 struct TcChain {
-    int n_phases;
-    TcMaps maps[TC_MAX_PHASES];
-    TcGemmParams p[TC_MAX_PHASES];
+    TcMaps maps[1];
+    TcGemmParams p[1];
 };
 cudaError_t launch_tc_chain(const TcChain& chain, bool pdl, cudaStream_t st);
 
