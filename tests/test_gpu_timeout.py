@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 TINY = S.WORKLOADS["tiny"].target
 
 
-@pytest.mark.parametrize("gamma", [4, 11])      # 15 rows: cluster kernel; 36 rows: stream-K kernel with shared-out passes
+@pytest.mark.parametrize("gamma", [4, 11])      # 5 rows: the few-row cluster kernel and (gate / up) the stream-K kernel; 12 rows x 3 sequences = 36: the many-row cluster kernel
 def test_wait_runs_out_then_context_recovers(gamma):
     gm = GpuModel(TINY, max_batch=3, max_nodes=16, capacity=128)
     V = TINY.vocab
