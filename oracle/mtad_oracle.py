@@ -50,7 +50,7 @@ from __future__ import annotations
 
 import math
 from dataclasses import dataclass, field
-from typing import List, Optional, Sequence
+from typing import List, Optional, Sequence, Tuple
 
 import numpy as np
 
@@ -495,13 +495,15 @@ class DraftResult:
     slot: List[int] = field(default_factory=list)   # per node: its row in the auxiliary cache is base + slot (the
                                                     # k-th beam of layer s has slot s * b + k); -1 for a candidate
                                                     # that was recorded but not kept as a beam (never run)
+    margin_warp: float = float("inf")   # closest warping decision over all beam rows (warp_row); inf without warping
 
 
 def gumbel_top_b(scores: np.ndarray, u: np.ndarray, b: int, with_gap: bool = False):
     """Sample b distinct flat indices without replacement, successive draws proportional to exp(scores):
     the b largest of scores + Gumbel noise, in decreasing order (lowest index first on ties)."""
     y = np.asarray(scores, dtype=np.float64).ravel() - np.log(-np.log(np.asarray(u, dtype=np.float64).ravel()))
-    order = sorted(range(y.size), key=lambda i: (-y[i], i))
+    # an index of probability 0 (score -inf: a token dropped by the warping) cannot be drawn, so fewer than b may come back
+    order = sorted((i for i in range(y.size) if y[i] > NEG_INF), key=lambda i: (-y[i], i))
     if with_gap:
         top = [y[i] for i in order[:b + 1]]
         gap = min((top[k] - top[k + 1] for k in range(len(top) - 1)), default=float("inf"))
@@ -510,7 +512,7 @@ def gumbel_top_b(scores: np.ndarray, u: np.ndarray, b: int, with_gap: bool = Fal
 
 
 def draft_beam(model: OracleModel, cache: np.ndarray, L: int, pending_tok: Sequence[int], gamma: int, b: int,
-               u: np.ndarray, keep_all: bool = False) -> DraftResult:
+               u: np.ndarray, keep_all: bool = False, warp: Optional[Tuple[int, float]] = None) -> DraftResult:
     """Beam sampling of width b for gamma steps (Sec. 2.1): at each step the b kept sequences are drawn without
     replacement from p_beam over (beam, token) pairs, i.e. proportionally to the joint likelihood
     q(beam) * q(token | beam).  Every intermediate beam becomes a tree node (Sec. 3.3).
@@ -524,6 +526,11 @@ def draft_beam(model: OracleModel, cache: np.ndarray, L: int, pending_tok: Seque
     of each of the b beams afterwards, beam by beam, best first.  The beams kept for the next step are, as before,
     the b best of all (beam, token) pairs, which are among those; the others are leaves (slot -1).  Without keep_all a
     layer holds just its b beams, best first (the paper's tree).
+
+    warp = (top_k, top_p): every beam row q(. | beam) is warped as in the paper's experiments (App. F, warp_row) before
+    the sampling, so the draft samples from, and reports the likelihoods of, the warped auxiliary distribution.  Dropped
+    tokens have probability 0 and are never drafted; a step whose rows keep fewer than b (beam, token) pairs in all
+    keeps that many beams, so layers may hold fewer nodes (node ids stay consecutive).
     """
     P = len(pending_tok)
     base = L + P
@@ -537,7 +544,17 @@ def draft_beam(model: OracleModel, cache: np.ndarray, L: int, pending_tok: Seque
                           [L + i for i in range(P)], vis)
     beams = [-1]                                   # node ids of the current beams (-1 = context)
     beam_logq = np.array([0.0])
-    beam_logp = log_softmax(logits[P - 1:P])       # [n_beams, V]
+    margin_warp = float("inf")
+
+    def row_logp(z):                               # [n_beams, V] log q(token | beam), warped if asked for
+        nonlocal margin_warp
+        if warp is None:
+            return log_softmax(z)
+        lp, m = warp_rows(z, warp[0], warp[1])
+        margin_warp = min(margin_warp, m)
+        return lp
+
+    beam_logp = row_logp(logits[P - 1:P])
     root_vis = vis[P - 1]
     node_vis = {-1: root_vis}
     min_gap = float("inf")
@@ -549,7 +566,7 @@ def draft_beam(model: OracleModel, cache: np.ndarray, L: int, pending_tok: Seque
         V = scores.shape[1]
         if keep_all:
             # the layer's nodes: per beam its best perturbed tokens (b * b of the single beam of the first step)
-            per_beam = (b * b) // len(beams)
+            per_beam = b * b if step == 0 else b
             layer = []
             for j in range(len(beams)):
                 own, gap_j = gumbel_top_b(scores[j:j + 1], u[step, j:j + 1, :], per_beam, with_gap=True)
@@ -575,7 +592,7 @@ def draft_beam(model: OracleModel, cache: np.ndarray, L: int, pending_tok: Seque
         if step + 1 < gamma:
             logits = decoder_rows(model, cache, L, [tok[n] for n in beams], [base - 1 + depth[n] for n in beams],
                                   [base + slot[n] for n in beams], [node_vis[n] for n in beams])
-            beam_logp = log_softmax(logits)
+            beam_logp = row_logp(logits)
     best = max(beams, key=lambda n: (logq[n], -n))
     path = []
     n = best
@@ -583,7 +600,7 @@ def draft_beam(model: OracleModel, cache: np.ndarray, L: int, pending_tok: Seque
         path.append(n)
         n = parent[n]
     path.reverse()
-    return DraftResult(tok, parent, depth, logq, path, [logq[n] for n in path], min_gap, slot)
+    return DraftResult(tok, parent, depth, logq, path, [logq[n] for n in path], min_gap, slot, margin_warp)
 
 
 def aux_commit(cache: np.ndarray, L: int, pending_tok: Sequence[int], draft: DraftResult, accepted: Sequence[int],

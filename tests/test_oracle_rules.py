@@ -617,3 +617,54 @@ def test_spd_robust_margin_is_the_gap_under_the_worst_perturbation():
                 z2 = np.log(np.maximum(0.0, np.exp(lp2) - np.exp(logq[r.eta])))
             assert int(np.argmax(z2 + noise)) == r.out_tok[-1], trial
     assert seen_reject > 50 and seen_accept > 5
+
+
+def test_draft_beam_on_warped_rows():
+    """The draft on warped auxiliary rows (App. F): without limits it is the plain draft; with limits every drafted
+    token lies in its row's kept set and its conditional log-likelihood is the warped row's, recomputed by causal
+    decoding from scratch; rows that keep fewer pairs than the beam width give layers with fewer nodes."""
+    from oracle.adapters import oracle_model
+    shape = S.WORKLOADS["tiny"].aux
+    model = oracle_model(S.make_model(shape, 1))
+    gamma, b, L, cap = 3, 3, 0, 48
+    V = shape.vocab
+    pend = S.token_ids(0, 61, 3, V).tolist()
+    u = S.uniforms(0, 62, gamma * b * V).view(gamma, b, V).numpy()
+    mk = lambda: np.zeros((shape.layers, 2, shape.n_kv_heads, cap, shape.head_dim), dtype=np.uint16)
+    base = O.draft_beam(model, mk(), L, pend, gamma, b, u)
+    same = O.draft_beam(model, mk(), L, pend, gamma, b, u, warp=(V, 1.0))
+    assert same.tok == base.tok and same.parent == base.parent and np.allclose(same.logq, base.logq, atol=1e-12)
+
+    def check(dr, top_k, top_p):
+        for n in range(len(dr.tok)):
+            path = []
+            c = n
+            while c >= 0:
+                path.append(c); c = dr.parent[c]
+            path.reverse()
+            seq = pend + [dr.tok[i] for i in path]
+            c2 = mk()
+            for i, t in enumerate(seq[:-1]):
+                lg = O.decoder_rows(model, c2, i, [t], [i], [i], [[i]])
+            row, _ = O.warp_row(lg[0], top_k, top_p)
+            assert np.isfinite(row[seq[-1]]), n                      # never a dropped token
+            parent_lq = dr.logq[dr.parent[n]] if dr.parent[n] >= 0 else 0.0
+            assert abs((dr.logq[n] - parent_lq) - row[seq[-1]]) < 1e-9, n
+
+    w = O.draft_beam(model, mk(), L, pend, gamma, b, u, warp=(5, 0.9))
+    assert np.isfinite(w.margin_warp) and len(w.tok) <= gamma * b and w.depth == sorted(w.depth)
+    check(w, 5, 0.9)
+    # two kept tokens per row and three beams wanted: layers of 2, 3 (of 2 x 2 pairs), 3 nodes
+    w2 = O.draft_beam(model, mk(), L, pend, gamma, b, u, warp=(2, 1.0))
+    assert [w2.depth.count(d) for d in (1, 2, 3)] == [2, 3, 3]
+    assert sorted(w2.slot[n] for n in range(len(w2.tok))) == [0, 1, 3, 4, 5, 6, 7, 8]
+    check(w2, 2, 1.0)
+    # greedy rows (one kept token each): a single chain, whatever the beam width
+    w1 = O.draft_beam(model, mk(), L, pend, gamma, b, u, warp=(1, 1.0))
+    assert w1.parent == [-1, 0, 1] and w1.best_path == [0, 1, 2]
+    check(w1, 1, 1.0)
+    # every candidate kept, on warped rows: the kept beams are those of the plain warped draft
+    wk = O.draft_beam(model, mk(), L, pend, gamma, b, u, keep_all=True, warp=(5, 0.9))
+    kept = {wk.slot[n]: n for n in range(len(wk.tok)) if wk.slot[n] >= 0}
+    assert [wk.tok[kept[k]] for k in sorted(kept)] == [w.tok[n] for n in sorted(range(len(w.tok)), key=lambda n: w.slot[n])]
+    check(wk, 5, 0.9)
