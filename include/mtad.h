@@ -144,6 +144,15 @@ int mtad_seq_hint(mtad_ctx* ctx, int seq, int32_t kv_len);
  * the verify calls are the caller's: mtad_draft itself samples from the unwarped auxiliary distribution. */
 int mtad_set_warp(mtad_ctx* ctx, int top_k, float top_p);
 
+/* The same warping for the auxiliary model's rows in mtad_draft (App. F warps both models): every beam row
+ * q(. | beam) keeps its top_k most likely tokens, renormalised, of these the first ones whose cumulative probability is
+ * larger than top_p, renormalised again; the draft samples from these rows and reports their likelihoods (node_logq,
+ * logq_ref).  A dropped token is never drafted.  When the rows of a step keep fewer (beam, token) pairs than
+ * beam_width, the step keeps that many beams and the layer holds fewer nodes: node ids stay consecutive, n_nodes of
+ * mtad_draft gives the count and becomes a required argument.  top_k = 0 switches it off (the default); limits and
+ * errors as for mtad_set_warp; MTAD_E_INVALID without an auxiliary model.  Host-side setting, no launch. */
+int mtad_set_draft_warp(mtad_ctx* ctx, int top_k, float top_p);
+
 /* Draft with the auxiliary model: beam sampling of width beam_width for gamma steps (Sec. 2.1, the p_beam
  * equation; every intermediate beam becomes a tree node, Sec. 3.3).  At each step the beam_width kept sequences
  * are drawn without replacement, proportionally to their joint likelihood, as the beam_width largest values of

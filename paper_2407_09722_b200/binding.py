@@ -46,7 +46,7 @@ AUDIT_VERIFY, AUDIT_DRAFT, AUDIT_COMMIT = 0, 1, 2
 EXPORTS = ("mtad_workspace_bytes", "mtad_create", "mtad_destroy", "mtad_seq_set", "mtad_seq_get", "mtad_draft",
            "mtad_verify_chain", "mtad_verify_tree", "kv_commit", "mtad_status_str", "mtad_last_cuda_error",
            "mtad_profile_begin", "mtad_profile_end", "mtad_kernel_launches", "mtad_verify_chain_static",
-           "mtad_debug_gemm", "mtad_set_warp", "mtad_profile_grouped",
+           "mtad_debug_gemm", "mtad_set_warp", "mtad_set_draft_warp", "mtad_profile_grouped",
            "mtad_verify_chain_spd", "mtad_seq_hint", "mtad_debug_set_wait", "mtad_audit_extents",
            "mtad_debug_check_canaries", "mtad_debug_region")
 MTAD_STATIC_SCRATCH_BYTES = 16 << 20
@@ -74,6 +74,7 @@ def load_library() -> C.CDLL:
     lib.mtad_seq_set.argtypes = [P, I, C.c_int32, C.c_int32, C.c_int32, I32P, P]
     lib.mtad_seq_get.argtypes = [P, I, I32P, I32P, P]
     lib.mtad_set_warp.argtypes = [P, I, C.c_float]
+    lib.mtad_set_draft_warp.argtypes = [P, I, C.c_float]
     lib.mtad_seq_hint.argtypes = [P, I, C.c_int32]
     lib.mtad_audit_extents.argtypes = [MD, MD, I, I, I, I, I, I, I, C.c_int64, C.POINTER(Extent), I, C.POINTER(I)]
     lib.mtad_debug_set_wait.argtypes = [P, C.c_uint, I]
@@ -236,6 +237,12 @@ class Context:
         rc = self._lib.mtad_set_warp(self.handle, top_k, top_p)
         if check:
             self._check(rc, "mtad_set_warp")
+        return rc
+
+    def mtad_set_draft_warp(self, top_k: int, top_p: float = 1.0, check=True) -> int:
+        rc = self._lib.mtad_set_draft_warp(self.handle, top_k, top_p)
+        if check:
+            self._check(rc, "mtad_set_draft_warp")
         return rc
 
     def mtad_seq_hint(self, seq: int, kv_len: int):

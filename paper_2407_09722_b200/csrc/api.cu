@@ -72,6 +72,8 @@ struct mtad_ctx {
     int debug_no_operands = 0;          // debug: the GEMM kernels' operand-row copies are left out (waits run out)
     int warp_k = 0;                     // 0: unwarped target rows
     float warp_p = 1.f;
+    int dwarp_k = 0;                    // 0: the draft samples from the unwarped auxiliary rows
+    float dwarp_p = 1.f;
     // optional per-kernel-class timing (cudaEvent pairs around each launch)
     bool prof_on = false;
     std::vector<cudaEvent_t> prof_ev;        // pool, used pairwise
@@ -257,6 +259,8 @@ size_t carve(mtad_ctx* c, const mtad_model_desc* t, const mtad_model_desc* a, in
     ds.best_path = k.take<int32_t>((size_t)max_batch * MTAD_MAX_DEPTH, "ds_best_path");
     ds.tree_id = k.take<int32_t>((size_t)max_batch * MTAD_DRAFT_NODES, "ds_tree_id");
     ds.tree2slot = k.take<int32_t>((size_t)max_batch * MTAD_DRAFT_NODES, "ds_tree2slot");
+    ds.nb = k.take<int32_t>((size_t)max_batch * MTAD_MAX_DEPTH, "ds_nb");
+    ds.n_tree = k.take<int32_t>((size_t)max_batch, "ds_n_tree");
     if (c) {
         c->ds = ds;
         c->st = st; c->rm = rm; c->sc = sc;
@@ -841,6 +845,14 @@ int mtad_set_warp(mtad_ctx* ctx, int top_k, float top_p) {
     return MTAD_OK;
 }
 
+int mtad_set_draft_warp(mtad_ctx* ctx, int top_k, float top_p) {
+    if (!ctx || !ctx->has_aux || top_k < 0 || isnan(top_p) || !(top_p > 0.f) || top_p > 1.f) return MTAD_E_INVALID;
+    if (top_k > MTAD_MAX_TOPK) return MTAD_E_CAPACITY;
+    ctx->dwarp_k = top_k;
+    ctx->dwarp_p = top_p;
+    return MTAD_OK;
+}
+
 int mtad_seq_hint(mtad_ctx* ctx, int seq, int32_t kv_len) {
     if (!ctx || seq < 0 || seq >= ctx->max_batch || kv_len < 0) return MTAD_E_INVALID;
     if (kv_len > ctx->target.d.kv_capacity) return MTAD_E_CAPACITY;
@@ -909,6 +921,9 @@ int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_wi
         gamma * beam_width > MTAD_MAX_NODES)
         return MTAD_E_CAPACITY;
     const int keep_all = keep_all_candidates ? 1 : 0;
+    // on warped rows a layer may hold fewer nodes than the beam width: the caller needs the count
+    const bool dwarp = ctx->dwarp_k > 0;
+    if (dwarp && !n_nodes) return MTAD_E_INVALID;
     // the caller's tree: beam_width * beam_width nodes a layer with every candidate kept (a verify call takes
     // MTAD_MAX_NODES at most), and a layer can only be filled from a vocabulary that large
     if (keep_all && (gamma * beam_width * beam_width > MTAD_MAX_NODES || ctx->aux.d.vocab < beam_width * beam_width))
@@ -931,13 +946,20 @@ int mtad_draft(mtad_ctx* ctx, int B, const int32_t* seqs, int gamma, int beam_wi
     for (int step = 0; step < gamma; ++step) {
         const int R = step == 0 ? R0 : beam_width;
         RUN(MTAD_K_PREPARE, 0, 1, launch_draft_prepare(m, ctx->st, ctx->ds, ctx->rm, ctx->sc, sl, B, R, step, beam_width,
-                                                       tc && B * R <= TC_MAX_ROWS, ctx->use_pdl, s));
+                                                       tc && B * R <= TC_MAX_ROWS, dwarp, ctx->use_pdl, s));
         // keys of the auxiliary cache: committed ones, the pending rows and every node drafted so far
         const long long keys_ub = ub + 1 + (long long)step * beam_width;
         int rc;
         if (tc && B * R <= TC_MAX_ROWS) rc = forward_rows_tc(ctx, m, ctx->amaps, B, R, keys_ub, nullptr, nullptr, true, s);
         else rc = forward_rows(ctx, m, B, R, keys_ub, s);
         if (rc != MTAD_OK) return rc;
+        if (dwarp) {
+            // warped rows (kept tokens and their renormalised log-probabilities), then the selection over those
+            RUN(MTAD_K_LMRED, 0, 2, launch_warp_rows_only(m, ctx->rm, ctx->sc, B, R, ctx->dwarp_k, ctx->dwarp_p, uniforms, s));
+            RUN(MTAD_K_LMRED, 0, 1, launch_draft_select_warped(m, ctx->ds, ctx->sc, sl, B, R, step, gamma, beam_width,
+                                                               keep_all, uniforms, out, s));
+            continue;
+        }
         RUN(MTAD_K_LMRED, 0, 2, launch_draft_select(m, ctx->ds, ctx->sc, sl, B, R, step, gamma, beam_width, keep_all, uniforms, out,
                                                      ctx->use_pdl, s));
     }
@@ -1145,6 +1167,12 @@ int mtad_audit_extents(const mtad_model_desc* target, const mtad_model_desc* aux
             au.ws("ds_node_logq", (size_t)(max_batch - 1) * MTAD_DRAFT_NODES + n_last + 1);
             au.ws("ds_node_mask", ((size_t)(max_batch - 1) * MTAD_DRAFT_NODES + n_last) * MTAD_MASK_WORDS + MTAD_MASK_WORDS);
             au.ws("ds_tree_id", (size_t)(max_batch - 1) * MTAD_DRAFT_NODES + n_last + 1);
+            au.ws("ds_nb", (size_t)(max_batch - 1) * MTAD_MAX_DEPTH + step + 1);
+            au.ws("ds_n_tree", (size_t)max_batch);
+            // on warped rows the selection ranks beam x MTAD_MAX_TOPK pairs held in shared memory
+            au.ext("warped selection candidates (shared memory)", (size_t)beam * MTAD_MAX_TOPK,
+                   (size_t)MTAD_MAX_BEAM * MTAD_MAX_TOPK);
+            au.ws("warp_row", (size_t)B * R);
             // node ids of the caller's tree: beam per layer, or beam * beam with every candidate kept (when that fits a
             // verify call); the selection holds the chunks' candidates of all beam rows in shared memory
             const size_t per_layer = gamma * beam * beam <= MTAD_MAX_NODES ? (size_t)beam * beam : (size_t)beam;

@@ -67,6 +67,10 @@ struct DraftState {
     // caller may hold more (mtad_draft with keep_all_candidates): these map between the two numberings.
     int32_t* tree_id;      // [max_batch][MTAD_DRAFT_NODES] beam slot -> node id in the caller's tree
     int32_t* tree2slot;    // [max_batch][MTAD_DRAFT_NODES] node id in the caller's tree -> beam slot, -1: not a beam
+    // Beams kept per step (the beam width, or fewer when the warped rows of a step keep fewer (beam, token) pairs)
+    // and the nodes written to the caller's tree so far.
+    int32_t* nb;           // [max_batch][MTAD_MAX_DEPTH]
+    int32_t* n_tree;       // [max_batch]
 };
 
 struct DraftOut {          // caller's device arrays of mtad_draft
@@ -350,10 +354,15 @@ cudaError_t launch_seq_advance(const SeqState& s, int B, const int32_t* call_seq
                                int max_depth, int max_batch, long long cap, cudaStream_t st);
 cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const DraftState& ds, const RowMeta& rm,
                                  const Scratch& sc, const SeqList& seqs, int B, int R, int step, int beam, bool tc,
-                                 bool pdl, cudaStream_t st);
+                                 bool warped, bool pdl, cudaStream_t st);
 cudaError_t launch_draft_select(const ModelView& m, const DraftState& ds, const Scratch& sc, const SeqList& seqs, int B,
                                 int R, int step, int gamma, int beam, int keep_all, const float* uniforms,
                                 const DraftOut& out, bool pdl, cudaStream_t st);
+cudaError_t launch_draft_select_warped(const ModelView& m, const DraftState& ds, const Scratch& sc, const SeqList& seqs,
+                                       int B, int R, int step, int gamma, int beam, int keep_all, const float* uniforms,
+                                       const DraftOut& out, cudaStream_t st);
+cudaError_t launch_warp_rows_only(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int top_k,
+                                  float top_p, const float* uni, cudaStream_t st);
 cudaError_t launch_aux_commit(const ModelView& aux, const SeqState& s, const DraftState& ds, int B,
                               const int32_t* call_seq_dev, const mtad_result& res, int max_depth, int mode,
                               cudaStream_t st);

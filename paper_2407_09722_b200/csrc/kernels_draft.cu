@@ -54,10 +54,11 @@ __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, in
                                      RopeInv rinv, long long kv_capacity, SeqState s, DraftState ds, RowMeta rm,
                                      float* __restrict__ hidden, float* __restrict__ rope, SeqList seqs, int R, int step,
                                      int beam, const __nv_bfloat16* __restrict__ gain0, __nv_bfloat16* x, int terms,
-                                     float* sumsq_out) {
+                                     float* sumsq_out, __nv_bfloat16* __restrict__ cache, int layers, int max_batch,
+                                     int Hkv) {
     const int t = blockIdx.x, bi = t / R, r = t % R;
     const int seq = seqs.v[bi];
-    __shared__ int sh_tok, sh_pos, sh_ok;
+    __shared__ int sh_tok, sh_pos, sh_ok, sh_hole;
     pdl_wait();               // the sequence and draft state, and every buffer written here, belong to earlier kernels
     pdl_trigger();
     if (threadIdx.x == 0) {
@@ -67,7 +68,7 @@ __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, in
         uint32_t mask[MTAD_MASK_WORDS];
 #pragma unroll
         for (int i = 0; i < MTAD_MASK_WORDS; ++i) mask[i] = 0;
-        int tok = 0, pos = L, vrow = 0;
+        int tok = 0, pos = L, vrow = 0, hole = -1;
         bool active;
         if (step == 0) {
             active = r < P;
@@ -78,7 +79,13 @@ __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, in
                 for (int i = 0; i <= r; ++i) mask[i >> 5] |= 1u << (i & 31);        // causal over the pending rows
             }
         } else {
-            active = r < beam;
+            // the beams the step before kept: the beam width, or fewer on warped rows
+            const int nbp = min(max(ds.nb[seq * MTAD_MAX_DEPTH + step - 1], 0), beam);
+            active = r < nbp;
+            // A beam slot of the layer before that no beam took is a cache row nobody wrote.  This step's rows never
+            // look at it (their masks name ancestors only), but a masked key still meets its value row with weight 0, and
+            // 0 x (whatever the memory held) must stay 0: the row is cleared (cache != null: only then can slots be empty).
+            hole = (cache && !active && r < beam) ? L + P + (step - 1) * beam + r : -1;
             if (active) {
                 const int n = (step - 1) * beam + r;
                 tok = ds.node_tok[seq * MTAD_DRAFT_NODES + n];
@@ -103,7 +110,8 @@ __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, in
         if (r == 0) {
             const bool state_ok = L >= 0 && P >= 1 && P <= MTAD_MAX_DEPTH + 1 && P <= (step == 0 ? R : MTAD_MAX_DEPTH + 1) &&
                                   (long long)L + P + (long long)step * beam <= kv_capacity;
-            rm.n_rows[bi] = !state_ok ? 0 : (step == 0 ? P : beam);
+            const int nbp = step == 0 ? 0 : min(max(ds.nb[seq * MTAD_MAX_DEPTH + step - 1], 0), beam);
+            rm.n_rows[bi] = !state_ok ? 0 : (step == 0 ? P : nbp);
             rm.n_spec[bi] = !state_ok ? 0 : (step == 0 ? P : P + step * beam);
             rm.kv_base[bi] = L;
             rm.call_seq[bi] = seq;
@@ -111,8 +119,15 @@ __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, in
         sh_tok = tok;
         sh_pos = pos;
         sh_ok = active;
+        sh_hole = (hole >= 0 && L >= 0 && (long long)hole < kv_capacity) ? hole : -1;
     }
     __syncthreads();
+    if (sh_hole >= 0) {
+        for (int i = threadIdx.x; i < layers * 2 * Hkv * hd; i += blockDim.x) {
+            const int j = i % hd, head = (i / hd) % Hkv, kv = (i / (hd * Hkv)) & 1, layer = i / (2 * hd * Hkv);
+            cache[idx_cache(layer, max_batch, seq, kv, Hkv, head, kv_capacity, sh_hole, hd) + j] = __float2bfloat16_rn(0.f);
+        }
+    }
     const int tok = sh_tok;
     const bool ok = sh_ok;
     float ss = embed_row(embed + (size_t)tok * d, ok, d, hidden + (size_t)t * d, gain0,
@@ -138,13 +153,15 @@ __global__ void draft_prepare_kernel(const __nv_bfloat16* __restrict__ embed, in
 
 cudaError_t launch_draft_prepare(const ModelView& m, const SeqState& s, const DraftState& ds, const RowMeta& rm,
                                  const Scratch& sc, const SeqList& seqs, int B, int R, int step, int beam, bool tc,
-                                 bool pdl, cudaStream_t st) {
+                                 bool warped, bool pdl, cudaStream_t st) {
     return launch_pdl(draft_prepare_kernel, dim3(B * R), dim3(128), 0, st, pdl,
                       static_cast<const __nv_bfloat16*>(m.d.embed), m.d.d_model, m.d.vocab, m.d.head_dim,
                       rope_inv((double)m.d.rope_base, m.d.head_dim), (long long)m.d.kv_capacity, s, ds, rm, sc.hidden,
                       sc.rope, seqs, R, step, beam,
                       tc ? m.w(0, 0) : (const __nv_bfloat16*)nullptr, tc ? sc.xd : (__nv_bfloat16*)nullptr,
-                      tc_terms(B * R), sc.sumsq_a);
+                      tc_terms(B * R), sc.sumsq_a,
+                      warped ? static_cast<__nv_bfloat16*>(m.d.kv_cache) : (__nv_bfloat16*)nullptr, m.d.layers, m.max_batch,
+                      m.d.n_kv_heads);
 }
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -344,6 +361,7 @@ __global__ void __launch_bounds__(256) draft_pick_kernel(const float* __restrict
         }
     }
     __syncthreads();
+    if (tid == 0) ds.nb[seq * MTAD_MAX_DEPTH + step] = beam;      // every beam slot of the layer is taken
     if (step == gamma - 1 && tid == 0) {
         // x**: the final beam with the highest draft likelihood (lowest tree id on ties), and its prefix likelihoods
         __threadfence_block();
@@ -365,6 +383,168 @@ __global__ void __launch_bounds__(256) draft_pick_kernel(const float* __restrict
         ds.beam[seq] = beam;
         if (out.n_nodes) out.n_nodes[bi] = N;
     }
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// selection on warped rows (App. F): every beam row has been cut to its kept tokens (warp_scan / warp_merge: at most
+// MTAD_MAX_TOPK tokens with renormalised log-probabilities), so the candidates of a step are the at most
+// beam * MTAD_MAX_TOPK (beam, kept token) pairs and one block per sequence ranks them all.  A step may find fewer
+// pairs than beams: it keeps what there is, the layer holds fewer nodes, node ids stay consecutive.
+// ---------------------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) draft_pick_warped_kernel(const WarpRow* __restrict__ rows, int V, int R, int step,
+                                                                int gamma, int beam, int keep_all,
+                                                                const float* __restrict__ uni, DraftState ds,
+                                                                SeqList seqs, DraftOut out) {
+    const int bi = blockIdx.x, seq = seqs.v[bi];
+    const int tid = threadIdx.x;
+    const int P = min(max(ds.npend[seq], 1), step == 0 ? R : MTAD_MAX_DEPTH + 1);
+    const int n_beams = step == 0 ? 1 : min(max(ds.nb[seq * MTAD_MAX_DEPTH + step - 1], 0), beam);
+    const int kpb = (keep_all && step == 0) ? beam * beam : beam;       // nodes a beam may contribute with all kept
+    const int N = gamma * (keep_all ? beam * beam : beam);              // capacity of the caller's arrays
+    constexpr int NC = MTAD_MAX_BEAM * MTAD_MAX_TOPK;
+    __shared__ float s_lq[MTAD_MAX_BEAM];
+    __shared__ int s_slot[MTAD_MAX_BEAM], s_tree[MTAD_MAX_BEAM];
+    __shared__ float s_y[NC], s_lp[NC];
+    __shared__ int s_flat[NC];
+    __shared__ Cand s_w[8];
+    __shared__ float l_y[MTAD_MAX_CAND], l_lp[MTAD_MAX_CAND];
+    __shared__ int l_flat[MTAD_MAX_CAND], l_rank[MTAD_MAX_CAND], l_id[MTAD_MAX_CAND];
+    __shared__ int s_count[2];                       // nodes of the layer, beams kept
+    if (tid < n_beams) {
+        const int slot = step == 0 ? -1 : (step - 1) * beam + tid;
+        s_slot[tid] = slot;
+        s_tree[tid] = slot < 0 ? -1 : ds.tree_id[seq * MTAD_DRAFT_NODES + slot];
+        s_lq[tid] = slot < 0 ? 0.f : ds.node_logq[seq * MTAD_DRAFT_NODES + slot];
+    }
+    __syncthreads();
+    if (tid < NC) {
+        const int j = tid / MTAD_MAX_TOPK, i = tid % MTAD_MAX_TOPK;
+        bool ok = j < n_beams;
+        float y = -CUDART_INF_F, lp = 0.f;
+        int flat = 0x7fffffff;
+        if (ok) {
+            const WarpRow& row = rows[bi * R + (step == 0 ? P - 1 : j)];
+            ok = i < min(row.n, MTAD_MAX_TOPK);
+            if (ok) {
+                const int v = row.idx[i];
+                ok = v >= 0 && v < V;
+                if (ok) {
+                    lp = row.lp[i];
+                    y = (s_lq[j] + lp) - logf(-logf(uni[(((size_t)bi * gamma + step) * beam + j) * V + v]));
+                    flat = j * V + v;
+                }
+            }
+        }
+        s_y[tid] = y; s_lp[tid] = lp; s_flat[tid] = flat;
+    }
+    __syncthreads();
+    // the layer's nodes: the `beam` best pairs of all, or with every candidate kept each beam's kpb best, best first
+    const int n_groups = keep_all ? n_beams : 1, rounds = keep_all ? min(kpb, MTAD_MAX_TOPK) : beam;
+    for (int gidx = 0; gidx < n_groups; ++gidx) {
+        const int lo = keep_all ? gidx * MTAD_MAX_TOPK : 0, hi = keep_all ? lo + MTAD_MAX_TOPK : NC;
+        for (int k = 0; k < rounds; ++k) {
+            Cand best{-CUDART_INF_F, 0x7fffffff};
+            const int i = lo + tid;
+            if (i < hi && s_flat[i] != 0x7fffffff) best = Cand{s_y[i], s_flat[i]};
+            const Cand win = block_best(best, s_w, tid);
+            const bool found = win.flat != 0x7fffffff;
+            if (tid == 0) {
+                const int m = gidx * rounds + k;
+                if (m < MTAD_MAX_CAND) { l_y[m] = found ? win.y : -CUDART_INF_F; l_flat[m] = win.flat; l_rank[m] = -1; }
+            }
+            if (found && best.flat == win.flat) {                     // the owner (pairs are unique) strikes the winner out
+                const int m = gidx * rounds + k;
+                if (m < MTAD_MAX_CAND) l_lp[m] = s_lp[i];
+                s_flat[i] = 0x7fffffff;
+            }
+            __syncthreads();
+        }
+    }
+    const int per_layer = min(n_groups * rounds, MTAD_MAX_CAND);
+    if (tid == 0) {
+        // consecutive node ids for the pairs that exist; the beams kept: the `beam` best of them
+        const int base_id = step == 0 ? 0 : max(ds.n_tree[seq], 0);
+        int cnt = 0;
+        for (int m = 0; m < per_layer; ++m) l_id[m] = l_flat[m] != 0x7fffffff ? base_id + cnt++ : -1;
+        int kept = 0;
+        for (int k = 0; k < beam; ++k) {
+            int bm = -1;
+            for (int m = 0; m < per_layer; ++m)
+                if (l_rank[m] < 0 && l_flat[m] != 0x7fffffff &&
+                    (bm < 0 || before(Cand{l_y[m], l_flat[m]}, Cand{l_y[bm], l_flat[bm]})))
+                    bm = m;
+            if (bm < 0) break;
+            l_rank[bm] = k;
+            ++kept;
+        }
+        s_count[0] = cnt;
+        s_count[1] = kept;
+        ds.nb[seq * MTAD_MAX_DEPTH + step] = kept;
+        ds.n_tree[seq] = base_id + cnt;
+    }
+    __syncthreads();
+    for (int m = tid; m < per_layer; m += 256) {
+        const int n = l_id[m];
+        if (n < 0 || n >= N || n >= MTAD_DRAFT_NODES) continue;
+        const int j = l_flat[m] / V, v = l_flat[m] % V;
+        const float lq = s_lq[j] + l_lp[m];
+        out.tok[bi * N + n] = v;
+        out.parent[bi * N + n] = s_tree[j];
+        out.depth[bi * N + n] = step + 1;
+        out.node_logq[bi * N + n] = lq;
+        const int k = l_rank[m];
+        ds.tree2slot[seq * MTAD_DRAFT_NODES + n] = k >= 0 ? step * beam + k : -1;
+        if (k >= 0) {
+            const int slot = step * beam + k, parent = s_slot[j];
+            ds.node_tok[seq * MTAD_DRAFT_NODES + slot] = v;
+            ds.node_parent[seq * MTAD_DRAFT_NODES + slot] = parent;
+            ds.node_logq[seq * MTAD_DRAFT_NODES + slot] = lq;
+            ds.tree_id[seq * MTAD_DRAFT_NODES + slot] = n;
+            uint32_t* mk = ds.node_mask + ((size_t)seq * MTAD_DRAFT_NODES + slot) * MTAD_MASK_WORDS;
+            for (int i = 0; i < MTAD_MASK_WORDS; ++i) {
+                uint32_t w;
+                if (parent >= 0) w = ds.node_mask[((size_t)seq * MTAD_DRAFT_NODES + parent) * MTAD_MASK_WORDS + i];
+                else {                                        // child of the root: sees all pending rows
+                    const int lo = i * 32;
+                    w = P >= lo + 32 ? 0xffffffffu : (P > lo ? (1u << (P - lo)) - 1u : 0u);
+                }
+                if (((P + slot) >> 5) == i) w |= 1u << ((P + slot) & 31);
+                mk[i] = w;
+            }
+        }
+    }
+    __syncthreads();
+    if (step == gamma - 1 && tid == 0) {
+        // x**: the final beam with the highest draft likelihood (lowest node id on ties), and its prefix likelihoods
+        __threadfence_block();
+        const int kept = s_count[1];
+        int best = -1;
+        for (int k = 0; k < kept; ++k) {
+            const int sl = (gamma - 1) * beam + k;
+            if (best < 0) { best = sl; continue; }
+            const float a = ds.node_logq[seq * MTAD_DRAFT_NODES + sl], b0 = ds.node_logq[seq * MTAD_DRAFT_NODES + best];
+            if (a > b0 || (a == b0 && ds.tree_id[seq * MTAD_DRAFT_NODES + sl] < ds.tree_id[seq * MTAD_DRAFT_NODES + best]))
+                best = sl;
+        }
+        int cur = best;
+        for (int i = gamma - 1; i >= 0 && cur >= 0; --i) {
+            out.best_path[bi * gamma + i] = ds.tree_id[seq * MTAD_DRAFT_NODES + cur];
+            out.logq_ref[bi * gamma + i] = ds.node_logq[seq * MTAD_DRAFT_NODES + cur];
+            ds.best_path[seq * MTAD_MAX_DEPTH + i] = cur;
+            cur = ds.node_parent[seq * MTAD_DRAFT_NODES + cur];
+        }
+        ds.gamma[seq] = gamma;
+        ds.beam[seq] = beam;
+        if (out.n_nodes) out.n_nodes[bi] = ds.n_tree[seq];
+    }
+}
+
+cudaError_t launch_draft_select_warped(const ModelView& m, const DraftState& ds, const Scratch& sc, const SeqList& seqs,
+                                       int B, int R, int step, int gamma, int beam, int keep_all, const float* uniforms,
+                                       const DraftOut& out, cudaStream_t st) {
+    draft_pick_warped_kernel<<<B, 256, 0, st>>>(sc.warp_row, m.d.vocab, R, step, gamma, beam, keep_all, uniforms, ds, seqs,
+                                                out);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_draft_select(const ModelView& m, const DraftState& ds, const Scratch& sc, const SeqList& seqs, int B,

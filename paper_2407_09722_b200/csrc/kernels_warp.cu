@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(32) warp_merge_kernel(const WarpPart* __restri
             if (y > by || (y == by && s_tv[i] < bv)) { by = y; bv = s_tv[i]; blp = lp; }
         }
         // a row of NaN logits ranks no token: flag the sequence, as the unwarped path does
-        if (found == 0 || bv == NONE || !isfinite(lse)) atomicOr(&status[bi], MTAD_ST_NONFINITE);
+        if (status && (found == 0 || bv == NONE || !isfinite(lse))) atomicOr(&status[bi], MTAD_ST_NONFINITE);
         row_lse[t] = lse;
         row_cand[t] = bv == NONE ? 0 : bv;
         row_cand_lp[t] = blp;
@@ -155,6 +155,21 @@ __global__ void warp_node_lp_kernel(const WarpRow* __restrict__ rows, const int3
             if (r.idx[i] == x) lp = r.lp[i];
     }
     node_lp[t] = lp;
+}
+
+// The warped rows alone (kept tokens and their log-probabilities, sc.warp_row), for the draft's selection: `uni` only
+// feeds the row's extra-token draw, which the draft does not use, and may be any [B, V] array of uniforms.
+cudaError_t launch_warp_rows_only(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int top_k,
+                                  float top_p, const float* uni, cudaStream_t st) {
+    const int V = m.d.vocab, T = B * R;
+    int nch = (V + 1023) / 1024;
+    nch = nch < 1 ? 1 : (nch > MTAD_DRAFT_CHUNKS ? MTAD_DRAFT_CHUNKS : nch);
+    warp_scan_kernel<<<dim3(nch, T), 256, 0, st>>>(sc.logits, V, rm.slot, sc.warp_part, nch, top_k);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    warp_merge_kernel<<<T, 32, 0, st>>>(sc.warp_part, nch, top_k, top_p, V, R, uni, rm.slot, sc.warp_row, sc.row_lse,
+                                        sc.row_cand, sc.row_cand_lp, nullptr);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_warp_rows(const ModelView& m, const RowMeta& rm, const Scratch& sc, int B, int R, int top_k,

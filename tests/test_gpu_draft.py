@@ -26,7 +26,15 @@ def draft_gap(keep_all: bool) -> float:
     return 1e-4 if keep_all else 1e-3
 
 
-def _draft_gpu(gm, seq, gamma, b, u, keep_all=False):
+# A draft on warped rows takes two more decisions per beam row (the top-k boundary in logits, the top-p cut in
+# probability), 1 + (gamma - 1) b rows a draft.  On the random-init auxiliary model the rows are nearly flat (the 10th
+# and 11th largest logit of 1024 lie 1e-3..3e-2 apart), so the closest of a draft's decisions is within 1e-3 in five
+# drafts of six; as for the candidate order above, the comparison goes down to 1e-4, five times the asserted error of
+# the device's logits.
+DRAFT_WARP_MARGIN = 1e-4
+
+
+def _draft_gpu(gm, seq, gamma, b, u, keep_all=False, warped=False):
     N = gamma * (b * b if keep_all else b)
     i32 = dict(dtype=torch.int32, device="cuda")
     f32 = dict(dtype=torch.float32, device="cuda")
@@ -36,16 +44,23 @@ def _draft_gpu(gm, seq, gamma, b, u, keep_all=False):
     gm.ctx.mtad_draft([seq], gamma, b, u, out["tok"], out["parent"], out["depth"], out["node_logq"], out["logq_ref"],
                       out["best_path"], keep_all_candidates=keep_all, n_nodes=out["n_nodes"])
     torch.cuda.synchronize()
-    assert out["n_nodes"].tolist() == [N]
+    assert warped or out["n_nodes"].tolist() == [N]
     return out
 
 
 # the last four keep every candidate of the beam sampling: 64-, 12- and 128-node trees (Sec. 3.3 with the tree sizes
 # of the full-size workloads), and the output sequence of such a draft verified as a chain
-@pytest.mark.parametrize("gamma,b,chain,keep_all", [(4, 4, False, False), (3, 2, True, False), (4, 1, True, False),
-                                                    (2, 8, False, False), (4, 4, False, True), (3, 2, False, True),
-                                                    (2, 8, False, True), (3, 3, True, True)])
-def test_draft_verify_commit_iterations(gamma, b, chain, keep_all):
+# the cases with a (top_k, top_p) pair draft from warped auxiliary rows (App. F): top-10 with top_p 0.85 (on a random-init
+# model the ten kept tokens are almost equally likely, so a cut at 0.9 sits on the ninth partial sum and every draft
+# would count as a near tie); two kept tokens a
+# row, so that the first layers hold fewer nodes than the beam width; greedy rows (a single chain whatever the beam
+# width); every candidate kept on warped rows; the output sequence of a warped draft verified as a chain
+@pytest.mark.parametrize("gamma,b,chain,keep_all,warp", [
+    (4, 4, False, False, None), (3, 2, True, False, None), (4, 1, True, False, None), (2, 8, False, False, None),
+    (4, 4, False, True, None), (3, 2, False, True, None), (2, 8, False, True, None), (3, 3, True, True, None),
+    (4, 4, False, False, (10, 0.85)), (3, 3, False, False, (2, 1.0)), (3, 3, False, False, (1, 1.0)),
+    (3, 3, False, True, (5, 0.9)), (4, 4, True, False, (10, 0.85))])
+def test_draft_verify_commit_iterations(gamma, b, chain, keep_all, warp):
     N = gamma * (b * b if keep_all else b)
     gm = GpuModel(W.target, max_batch=2, max_nodes=max(40, N), capacity=320, aux=W.aux, aux_capacity=320)
     seq, L = 1, 24
@@ -53,6 +68,8 @@ def test_draft_verify_commit_iterations(gamma, b, chain, keep_all):
     gm.inject_aux(seq, L)
     root = 5
     gm.ctx.mtad_seq_set(seq, L, root, aux_len=L)
+    if warp:
+        gm.ctx.mtad_set_draft_warp(*warp)
     tcache = gm.cache_bits(seq, L)
     acache = gm.aux_cache_bits(seq, L)
     La, pend = L, [root]
@@ -60,17 +77,21 @@ def test_draft_verify_commit_iterations(gamma, b, chain, keep_all):
     skipped = 0
     leaves = 0                  # accepted paths that end in a node the auxiliary model never ran
     lq_err = 0.0
+    sizes = set()
     for it in range(6):
         u = S.uniforms(0, (31 << 40) | (it * 16 + gamma), gamma * b * V, "cuda").view(1, gamma, b, V)
-        g = _draft_gpu(gm, seq, gamma, b, u, keep_all)
-        dr = O.draft_beam(gm.oracle_aux(), acache, La, pend, gamma, b, u[0].cpu().numpy(), keep_all=keep_all)
-        assert len(dr.tok) == N
-        near = dr.min_gap < draft_gap(keep_all)
+        g = _draft_gpu(gm, seq, gamma, b, u, keep_all, warped=warp is not None)
+        dr = O.draft_beam(gm.oracle_aux(), acache, La, pend, gamma, b, u[0].cpu().numpy(), keep_all=keep_all, warp=warp)
+        n = len(dr.tok)                              # (on warped rows a layer may hold fewer nodes than it has room for)
+        assert n == N or (warp and n < N)
+        sizes.add(n)
+        near = dr.min_gap < draft_gap(keep_all) or dr.margin_warp < DRAFT_WARP_MARGIN
         if not near:
-            assert g["tok"][0].tolist() == dr.tok and g["parent"][0].tolist() == dr.parent
-            assert g["depth"][0].tolist() == dr.depth and g["best_path"][0].tolist() == dr.best_path
-            lq_err = max(lq_err, float(np.max(np.abs(g["node_logq"][0].cpu().numpy() - np.asarray(dr.logq)))))
-            assert np.max(np.abs(g["node_logq"][0].cpu().numpy() - np.asarray(dr.logq))) < LP_TOL
+            assert g["n_nodes"].tolist() == [n]
+            assert g["tok"][0, :n].tolist() == dr.tok and g["parent"][0, :n].tolist() == dr.parent
+            assert g["depth"][0, :n].tolist() == dr.depth and g["best_path"][0].tolist() == dr.best_path
+            lq_err = max(lq_err, float(np.max(np.abs(g["node_logq"][0, :n].cpu().numpy() - np.asarray(dr.logq)))))
+            assert np.max(np.abs(g["node_logq"][0, :n].cpu().numpy() - np.asarray(dr.logq))) < LP_TOL
             assert np.max(np.abs(g["logq_ref"][0].cpu().numpy() - np.asarray(dr.logq_ref))) < LP_TOL
         # The device verifies its own draft, straight from the arrays mtad_draft wrote; next to a tie of the draft
         # it gets the oracle's instead (and its caches are put back on the oracle's trajectory afterwards).
@@ -87,15 +108,19 @@ def test_draft_verify_commit_iterations(gamma, b, chain, keep_all):
             accepted = [dr.best_path[i] for i in r.path]
         else:
             res = M.ResultBuffers(1, N, gamma)
-            d_tok = g["tok"] if not near else torch.tensor(dr.tok, dtype=torch.int32, device="cuda")
-            d_par = g["parent"] if not near else torch.tensor(dr.parent, dtype=torch.int32, device="cuda")
-            gm.ctx.mtad_verify_tree([seq], g["n_nodes"], N, gamma, d_tok, d_par, d_ref, log_tau, bu, res)
+            pad = [0] * (N - n)
+            d_tok = g["tok"] if not near else torch.tensor(dr.tok + pad, dtype=torch.int32, device="cuda")
+            d_par = g["parent"] if not near else torch.tensor(dr.parent + pad, dtype=torch.int32, device="cuda")
+            d_n = g["n_nodes"] if not near else torch.tensor([n], dtype=torch.int32, device="cuda")
+            gm.ctx.mtad_verify_tree([seq], d_n, N, gamma, d_tok, d_par, d_ref, log_tau, bu, res)
             r = O.verify_tree(gm.oracle(), tcache, L, root, dr.tok, dr.parent, ref.astype(np.float64), log_tau,
                               bu[0].cpu().numpy())
             accepted = list(r.path)
         gm.ctx.kv_commit([seq], res)
         h = res.host()
-        assert int(h["status"][0]) == 0
+        # (next to a tie of the draft the device rolls its auxiliary cache forward by its own tree, which the verified
+        # one need not be: a range flag is possible there and the state is replaced below anyway)
+        assert int(h["status"][0]) == 0 or near
         tie = min(r.margin_accept, r.margin_tie, r.margin_bonus) < 1e-3
         L = O.kv_commit(tcache, L, r.path)
         La, pend = O.aux_commit(acache, La, pend, dr, accepted, r.out_tok[-1], gamma)
@@ -109,9 +134,9 @@ def test_draft_verify_commit_iterations(gamma, b, chain, keep_all):
             continue
         assert int(h["eta"][0]) == r.eta and h["out_tok"][0, :r.eta + 1].tolist() == r.out_tok
         assert gm.ctx.mtad_seq_get(seq) == (L, root)
-    print(f"keep_all={keep_all} gamma={gamma} b={b}: skipped {skipped}, paths ending in a not-run node {leaves}, "
-          f"largest node_logq error {lq_err:.2e}")
-    assert skipped <= 3 and lq_err < 2e-5
+    print(f"keep_all={keep_all} gamma={gamma} b={b} warp={warp}: skipped {skipped}, paths ending in a not-run node {leaves}, "
+          f"largest node_logq error {lq_err:.2e}, tree sizes {sorted(sizes)}")
+    assert skipped <= (4 if warp else 3) and lq_err < 2e-5
     assert gm.ctx.mtad_debug_check_canaries() == ""
 
 
