@@ -233,12 +233,13 @@ def throughput(total_ms: float, tokens: float) -> float:
 DRAFT_BEAM = 4          # the paper's smaller beam width
 
 
-def draft_loop(w: S.Workload, steps: int, warmup: int, cap: int):
+def draft_loop(w: S.Workload, steps: int, warmup: int, cap: int, warp=None):
     """Decode iterations in which the auxiliary model drafts by beam sampling, the target verifies and both caches are
     rolled forward.  Chain workloads verify the best beam (Algorithm 1); tree workloads keep every candidate of the
     beam sampling (beam * beam nodes a layer, the workload's tree size) and verify that tree as mtad_draft left it on
     the device (Sec. 3.3).  Returns tokens/s including the draft and the draft's share; a reported extra, not the
-    headline (the headline times the verification path on synthetic drafts)."""
+    headline (the headline times the verification path on synthetic drafts).  warp = (top_k, top_p): both models'
+    rows warped as in the paper's experiments (App. F)."""
     import paper_2407_09722_b200 as M
     from paper_2407_09722_b200.runtime import DeviceModel
     lens = S.kv_lengths(w, SEED)
@@ -250,6 +251,9 @@ def draft_loop(w: S.Workload, steps: int, warmup: int, cap: int):
     N = g * b * b if tree else g * b
     dm = DeviceModel(w.target, B, max(w.n_nodes, N), cap, SEED, aux=w.aux, aux_capacity=cap + g * b + 8)
     ctx = dm.ctx
+    if warp:
+        ctx.mtad_set_warp(*warp)
+        ctx.mtad_set_draft_warp(*warp)
     seqs = list(range(B))
     for s_, L in enumerate(lens):
         dm.inject(s_, L)
@@ -292,7 +296,7 @@ def draft_loop(w: S.Workload, steps: int, warmup: int, cap: int):
     total_ms = ev[0][0].elapsed_time(ev[-1][2])
     accepted = float(acc.item())
     return {"value": accepted / (total_ms * 1e-3), "unit": "tokens/s", "steps": steps, "gamma": g, "beam": b,
-            "nodes": N, "verified_as": "tree" if tree else "chain",
+            "nodes": N, "verified_as": "tree" if tree else "chain", "warp": list(warp) if warp else None,
             "block_efficiency": accepted / (steps * B), "iteration_ms": total_ms / steps,
             "draft_us_median": statistics.median(d_us), "verify_commit_us_median": 1e3 * statistics.median(it_ms)
             - statistics.median(d_us), "device_status": status}
@@ -627,7 +631,8 @@ def run_ours(args, w: S.Workload, rank: int, world: int, local_rank: int):
     del dm, ctx
     torch.cuda.empty_cache()
     if world == 1 and not args.no_draft_loop:
-        line["draft_loop"] = draft_loop(w, min(args.steps, 32), 3, cap)
+        line["draft_loop"] = draft_loop(w, min(args.steps, 32), 3, cap,
+                                        warp=(args.top_k, args.top_p) if args.top_k > 0 else None)
         torch.cuda.empty_cache()
     if world == 1 and not args.no_extras:
         line["read_only_peak_gbs"] = read_only_peak()
