@@ -180,7 +180,14 @@ def test_draft_rejects_bad_arguments():
     assert c.mtad_draft([3], 4, 4, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_INVALID
     # every candidate kept: gamma * b * b nodes must fit a verify call
     assert c.mtad_draft([0], 4, 8, u, t, t, t, f, f, t, check=False, keep_all_candidates=True) == M.binding.MTAD_E_CAPACITY
+    # warped rows: limits as for the target's warping; the node count becomes a required output
+    assert c.mtad_set_draft_warp(17, 0.9, check=False) == M.binding.MTAD_E_CAPACITY
+    assert c.mtad_set_draft_warp(10, 0.0, check=False) == M.binding.MTAD_E_INVALID
+    assert c.mtad_set_draft_warp(10, 0.9, check=False) == 0
+    assert c.mtad_draft([0], 4, 4, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_INVALID       # no n_nodes
+    assert c.mtad_set_draft_warp(0, 1.0, check=False) == 0
     no_aux = GpuModel(W.target, max_batch=1, max_nodes=8, capacity=64)
+    assert no_aux.ctx.mtad_set_draft_warp(10, 0.9, check=False) == M.binding.MTAD_E_INVALID
     assert no_aux.ctx.mtad_draft([0], 4, 4, u, t, t, t, f, f, t, check=False) == M.binding.MTAD_E_INVALID
 
 
