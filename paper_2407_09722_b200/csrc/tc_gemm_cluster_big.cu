@@ -251,45 +251,62 @@ __global__ void __launch_bounds__(BG_THREADS, 1) tc_gemm_cluster_big_kernel(cons
         cluster_arrive_release();
         cluster_wait_acquire();
         // This CTA's partial tile goes to the staging area behind the receive slots, rows in order, [row][half][128]:
-        // the rows of a pass are one contiguous piece.  The groups share out the (half, 16 rows) blocks.
+        // the rows of a pass are one contiguous piece, which one bulk copy takes to the pass's owner.
         float* recv = reinterpret_cast<float*>(s.ring);
         float* stage_out = recv + bg_recv_floats(T, rpr, csize, mh);
-        if (have) {
-            const int nblk = (T + 15) / 16;
-            for (int it = grp; it < mh * nblk; it += BG_GROUPS) {
-                const int h = it / nblk, rb = (it - h * nblk) * 16;
-                const uint32_t t_acc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(h * acc_cols);
-                float v[16];
-                if (n_kb == 0) {
+        const int nblk = (T + 15) / 16;
+        // 16 rows of half h: tensor memory -> staging area
+        auto stage_block = [&](int h, int rb) {
+            const uint32_t t_acc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(h * acc_cols);
+            float v[16];
+            if (n_kb == 0) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = 0.f;
-                } else if (terms == 3) {
-                    float w[48];
-                    tc_ld16(t_acc + 3 * rb, w);
-                    tc_ld32(t_acc + 3 * rb + 16, w + 16);
+                for (int j = 0; j < 16; ++j) v[j] = 0.f;
+            } else if (terms == 3) {
+                float w[48];
+                tc_ld16(t_acc + 3 * rb, w);
+                tc_ld32(t_acc + 3 * rb + 16, w + 16);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = w[3 * j] + (w[3 * j + 1] + w[3 * j + 2]);
-                } else {
-                    float w[32];
-                    tc_ld32(t_acc + 2 * rb, w);
+                for (int j = 0; j < 16; ++j) v[j] = w[3 * j] + (w[3 * j + 1] + w[3 * j + 2]);
+            } else {
+                float w[32];
+                tc_ld32(t_acc + 2 * rb, w);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = w[2 * j] + w[2 * j + 1];
-                }
-#pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    if (rb + j < T) stage_out[((size_t)(rb + j) * mh + h) * TC_TILE_N + feat] = v[j];
+                for (int j = 0; j < 16; ++j) v[j] = w[2 * j] + w[2 * j + 1];
             }
-        }
-        tc_fence_before();
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the copies below read what was just written
-        both_bar();
-        if (e2 == 0) trace_stamp(p.trace, 5);
-        if (have && e2 < n_pass) {
-            const int pass = e2, r0 = pass * rpr, rows = min(T, r0 + rpr) - r0;
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (rb + j < T) stage_out[((size_t)(rb + j) * mh + h) * TC_TILE_N + feat] = v[j];
+        };
+        auto send_pass = [&](int pass) {
+            const int r0 = pass * rpr, rows = min(T, r0 + rpr) - r0;
             const int owner = pass % csize, own = pass / csize;
             const uint32_t dst = smem_u32(recv) + (uint32_t)((own * csize + rank) * rpr * mh * TC_TILE_N) * 4u;
             bulk_copy_to_rank(dst, smem_u32(stage_out + (size_t)r0 * mh * TC_TILE_N), (uint32_t)(rows * mh * TC_TILE_N * 4),
                               smem_u32(s.rfull), (uint32_t)owner);
+        };
+        if (rpr == 8) {
+            // Passes of eight rows sit inside the 16-row blocks: a group stages whole blocks (both halves) and sends a
+            // block's two passes as soon as the block is in the staging area, so that the transfers run while the rest
+            // is still being drained.
+            for (int b = grp; b < nblk; b += BG_GROUPS) {
+                if (have)
+                    for (int h = 0; h < mh; ++h) stage_block(h, b * 16);
+                tc_fence_before();
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the copies read what was just written
+                epi_bar(bar_id);
+                if (have && e < 2 && 2 * b + e < n_pass) send_pass(2 * b + e);
+            }
+            if (e2 == 0) trace_stamp(p.trace, 5);
+        } else {
+            // the groups share out the (half, 16 rows) blocks; the copies go out when everything is staged
+            if (have)
+                for (int it = grp; it < mh * nblk; it += BG_GROUPS) stage_block(it / nblk, (it % nblk) * 16);
+            tc_fence_before();
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            both_bar();
+            if (e2 == 0) trace_stamp(p.trace, 5);
+            if (have && e2 < n_pass) send_pass(e2);
         }
         if (e2 == 0) s.flags[0] = (have && mbar_wait(smem_u32(s.rfull), 0u, abort_flag)) ? 1 : 0;
         both_bar();
