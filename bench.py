@@ -30,7 +30,7 @@ TAU = 0.1
 SEED = 0
 # (DRAM read + write) / algorithmic bytes of the GEMM launches of one layer, ncu on the 4-layer workloads of the same
 # shape (profiles/tc_gemm_7b_chain_4l.md, profiles/tc_gemm_7b_tree_4l.md); no figure for the other workloads
-NCU_TRAFFIC_RATIO = {"7b_chain": 1.009, "7b_chain_4l": 1.009, "7b_chain_l512": 1.009, "7b_tree": 1.032, "7b_tree_4l": 1.032}
+NCU_TRAFFIC_RATIO = {"7b_chain": 1.011, "7b_chain_4l": 1.011, "7b_chain_l512": 1.011, "7b_tree": 1.033, "7b_tree_4l": 1.033}
 
 
 def measured_peaks():
