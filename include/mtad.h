@@ -141,7 +141,7 @@ int mtad_seq_hint(mtad_ctx* ctx, int seq, int32_t kv_len);
  * into the workspace and derive the warped rows from them (row_lse of mtad_result is the log-sum-exp over the kept
  * tokens).  top_k = 0 switches warping off (the default); top_k <= 16 (MTAD_E_CAPACITY beyond), 0 < top_p <= 1
  * (MTAD_E_INVALID otherwise).  Host-side setting of the context, no launch.  The draft log-likelihoods passed to
- * the verify calls are the caller's: mtad_draft itself samples from the unwarped auxiliary distribution. */
+ * the verify calls are the caller's; mtad_set_draft_warp (below) makes mtad_draft sample from warped rows too. */
 int mtad_set_warp(mtad_ctx* ctx, int top_k, float top_p);
 
 /* The same warping for the auxiliary model's rows in mtad_draft (App. F warps both models): every beam row
