@@ -17,7 +17,7 @@ def small_ctx():
     return DeviceModel(S.ModelShape(1, 256, 4, 4, 64, 1408, 4096), max_batch=1, max_nodes=255, capacity=320)
 
 
-def _check(dm, N, K, T, seed, variant=0):
+def _check(dm, N, K, T, seed, variant=0, allow_small_workspace=False):
     W = S.normal_bf16(seed, 1000 + N + K, N * K, 0.02, "cuda").view(N, K)
     x = S.normal_bf16(seed, 2000 + T + K, T * K, 1.0, "cuda").float().view(T, K)
     x = x * (1.0 + 1e-3 * torch.arange(T * K, device="cuda").view(T, K).remainder(7))     # not bf16-representable
@@ -25,6 +25,8 @@ def _check(dm, N, K, T, seed, variant=0):
     rc = dm.ctx.mtad_debug_gemm(W, x, y, variant=variant, check=False)
     if variant == 1 and rc == Bn.MTAD_E_UNIMPLEMENTED:
         return False                                 # the shape does not suit the cluster kernels
+    if allow_small_workspace and rc == Bn.MTAD_E_WORKSPACE:
+        return False                                 # the context's split-K workspace (sized for its model) is too small
     assert rc == 0, rc
     torch.cuda.synchronize()
     ref = x.double() @ W.double().t()
@@ -81,3 +83,21 @@ def test_debug_gemm_7b_shapes():
     for (N, K, T) in [(4096, 4096, 5), (4096, 11008, 5), (32000, 4096, 9)]:
         _check(dm, N, K, T, 2)
         assert _check(dm, N, K, T, 2, variant=1)
+
+
+def test_debug_gemm_seeded_shape_sweep(small_ctx):
+    """Ragged shapes drawn from a seeded generator, through the stream-K kernel and - where the plan takes them - the
+    cluster kernels: row counts on both sides of the 32-row boundary between the two cluster kernels, feature counts
+    that are no multiple of a tile, k that is no multiple of a k-block."""
+    import random
+    rng = random.Random(2407)
+    ran_cluster = ran_stream = 0
+    for i in range(24):
+        T = rng.choice([rng.randint(1, 32), rng.randint(33, 128)])
+        N = rng.randint(1, 32) * 128 - rng.choice([0, 0, 8, 56, 120])
+        K = rng.randint(2, 176) * 8
+        ran = _check(small_ctx, N, K, T, 100 + i, variant=0, allow_small_workspace=True)
+        ran_stream += bool(ran)
+        ran_cluster += bool(_check(small_ctx, N, K, T, 100 + i, variant=1, allow_small_workspace=True))
+    print(f"sweep: {ran_stream} shapes through the stream-K kernel, {ran_cluster} through the cluster kernels")
+    assert ran_stream >= 16 and ran_cluster >= 12
